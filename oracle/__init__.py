@@ -1,0 +1,246 @@
+"""CMPQ oracle: ctypes binding of ``cmpq_oracle.c`` -- TEST INFRASTRUCTURE ONLY.
+
+A plain single-threaded CPU restatement of the CMPQ pass (arxiv 2410.13056,
+Sections 3.2.1 and 3.2.2, Algorithm 1, Section 5.1).  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import this package; the CUDA
+library never does, and this package never imports the CUDA library.
+
+All arrays are numpy arrays; 16-bit float tensors travel as ``uint16`` bit
+patterns together with ``dtype`` (0 = fp16, 1 = bf16).
+"""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+F16 = 0
+BF16 = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cmpq_oracle.c")
+_LIB_PATH = os.path.join(_HERE, "libcmpq_oracle.so")
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with gcc (-O2, no contraction, no fast-math)."""
+    if (not force and os.path.exists(_LIB_PATH)
+            and os.path.getmtime(_LIB_PATH) >= os.path.getmtime(_SRC)):
+        return _LIB_PATH
+    tmp = _LIB_PATH + ".tmp%d" % os.getpid()
+    subprocess.run(["gcc", "-O2", "-ffp-contract=off", "-std=c11", "-Wall", "-shared", "-fPIC",
+                    "-o", tmp, _SRC, "-lm"], check=True)
+    os.replace(tmp, _LIB_PATH)
+    return _LIB_PATH
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_widen.restype = ctypes.c_float
+        _lib.oracle_widen.argtypes = [ctypes.c_uint16, ctypes.c_int]
+        _lib.oracle_packed_words.restype = ctypes.c_int64
+        _lib.oracle_metadata_bits_per_weight.restype = ctypes.c_double
+        _lib.oracle_recon_error.restype = ctypes.c_double
+    return _lib
+
+
+def _p(arr):
+    return None if arr is None else arr.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i64(v):
+    return ctypes.c_int64(int(v))
+
+
+def _c(arr, dt):
+    arr = np.ascontiguousarray(arr, dtype=dt)
+    return arr
+
+
+def widen(u16, dtype):
+    """Exact fp16/bf16 bit pattern -> float32 (element by element through the C routine)."""
+    u16 = _c(u16, np.uint16)
+    out = np.empty(u16.shape, np.float32)
+    flat_in, flat_out = u16.reshape(-1), out.reshape(-1)
+    f = lib().oracle_widen
+    for i in range(flat_in.size):
+        flat_out[i] = f(int(flat_in[i]), dtype)
+    return out
+
+
+def collect_stats(X_u16, dtype, sumsq=None):
+    X_u16 = _c(X_u16, np.uint16)
+    n, d_in = X_u16.shape
+    if sumsq is None:
+        sumsq = np.zeros(d_in, np.float64)
+    lib().oracle_collect_stats(_p(X_u16), dtype, _i64(n), _i64(d_in), _i64(d_in), _p(sumsq))
+    return sumsq
+
+
+def finalize_stats(sumsq):
+    sumsq = _c(sumsq, np.float64)
+    a = np.empty(sumsq.shape[0], np.float32)
+    lib().oracle_finalize_stats(_p(sumsq), _i64(sumsq.shape[0]), _p(a))
+    return a
+
+
+def alloc_counts(d_in, avg_bits):
+    n2, n4 = ctypes.c_int64(), ctypes.c_int64()
+    lib().oracle_alloc_counts(_i64(d_in), ctypes.c_double(avg_bits), ctypes.byref(n2),
+                              ctypes.byref(n4))
+    return n2.value, n4.value
+
+
+def default_counts(d_in, d_out):
+    n_act, n_q = ctypes.c_int64(), ctypes.c_int64()
+    lib().oracle_default_counts(_i64(d_in), _i64(d_out), ctypes.byref(n_act), ctypes.byref(n_q))
+    return n_act.value, n_q.value
+
+
+def allocate_bits(a, avg_bits, mode=0):
+    """Algorithm 1.  Returns (bits uint8[d_in], order int32[d_in])."""
+    a = _c(a, np.float32)
+    d_in = a.shape[0]
+    bits = np.empty(d_in, np.uint8)
+    order = np.empty(d_in, np.int32)
+    rc = lib().oracle_allocate_bits(_p(a), _i64(d_in), ctypes.c_double(avg_bits), int(mode),
+                                    _p(bits), _p(order))
+    if rc:
+        raise ValueError("avg_bits must lie in [2, 4]")
+    return bits, order
+
+
+def lloyd(x, K, T, s=None, trace=False):
+    """Channel K-means.  Returns (lut float32[16], code uint8[N], err float32[N][, sse[T+1]])."""
+    x = _c(x, np.float32)
+    N = x.shape[0]
+    lut = np.zeros(16, np.float32)
+    code = np.empty(N, np.uint8)
+    err = np.empty(N, np.float32)
+    sse = np.zeros(T + 1, np.float64) if trace else None
+    if s is not None:
+        s = _c(s, np.float64)
+    lib().oracle_lloyd(_p(x), _i64(N), int(K), int(T), _p(s), _p(lut), _p(code), _p(err), _p(sse))
+    return (lut, code, err, sse) if trace else (lut, code, err)
+
+
+def extract_outliers(W_u16, dtype, a, bits, n_act, n_q, T, want_fit=False):
+    """Section 3.2.2.  Returns (rows, cols, vals[, lut1, err])."""
+    W_u16 = _c(W_u16, np.uint16)
+    d_in, d_out = W_u16.shape
+    a = _c(a, np.float32)
+    bits = _c(bits, np.uint8)
+    nnz = n_act * d_out + n_q
+    rows = np.empty(nnz, np.int32)
+    cols = np.empty(nnz, np.int32)
+    vals = np.empty(nnz, np.uint16)
+    lut1 = np.zeros((d_in, 16), np.float32) if want_fit else None
+    err = np.zeros((d_in, d_out), np.float32) if want_fit else None
+    rc = lib().oracle_extract_outliers(_p(W_u16), dtype, _i64(d_in), _i64(d_out), _i64(d_out),
+                                       _p(a), _p(bits), _i64(n_act), _i64(n_q), int(T),
+                                       _p(rows), _p(cols), _p(vals), _p(lut1), _p(err))
+    if rc:
+        raise ValueError("bad outlier counts")
+    return (rows, cols, vals, lut1, err) if want_fit else (rows, cols, vals)
+
+
+def quantize_layer(W_u16, dtype, bits, rows, cols, T, sens=None):
+    """Final channel-wise K-means on W - O.  Returns (lut float32[d_in,16], codes uint8[d_in,d_out])."""
+    W_u16 = _c(W_u16, np.uint16)
+    d_in, d_out = W_u16.shape
+    bits = _c(bits, np.uint8)
+    rows = _c(rows, np.int32)
+    cols = _c(cols, np.int32)
+    lut = np.zeros((d_in, 16), np.float32)
+    codes = np.empty((d_in, d_out), np.uint8)
+    if sens is not None:
+        sens = _c(sens, np.float64)
+    rc = lib().oracle_quantize_layer(_p(W_u16), dtype, _i64(d_in), _i64(d_out), _i64(d_out),
+                                     _p(bits), _p(rows), _p(cols), _i64(rows.shape[0]), int(T),
+                                     _p(sens), _p(lut), _p(codes))
+    if rc:
+        raise ValueError("outlier rows must be sorted ascending")
+    return lut, codes
+
+
+def packed_words(bits, d_out):
+    bits = _c(bits, np.uint8)
+    return int(lib().oracle_packed_words(_p(bits), _i64(bits.shape[0]), _i64(d_out)))
+
+
+def pack(codes, bits):
+    """Returns (packed uint32[words], row_off int64[d_in+1], perm int32[d_in], seg_rows int64[3])."""
+    codes = _c(codes, np.uint8)
+    bits = _c(bits, np.uint8)
+    d_in, d_out = codes.shape
+    packed = np.empty(packed_words(bits, d_out), np.uint32)
+    row_off = np.empty(d_in + 1, np.int64)
+    perm = np.empty(d_in, np.int32)
+    seg_rows = np.zeros(3, np.int64)
+    lib().oracle_pack(_p(codes), _p(bits), _i64(d_in), _i64(d_out), _p(packed), _p(row_off),
+                      _p(perm), _p(seg_rows))
+    return packed, row_off, perm, seg_rows
+
+
+def unpack(packed, row_off, perm, bits, d_out):
+    packed = _c(packed, np.uint32)
+    row_off = _c(row_off, np.int64)
+    perm = _c(perm, np.int32)
+    bits = _c(bits, np.uint8)
+    d_in = bits.shape[0]
+    codes = np.empty((d_in, d_out), np.uint8)
+    lib().oracle_unpack(_p(packed), _p(row_off), _p(perm), _p(bits), _i64(d_in), _i64(d_out),
+                        _p(codes))
+    return codes
+
+
+def metadata_bits_per_weight(bits, d_out, tag_bits=4, lut_bits=16):
+    bits = _c(bits, np.uint8)
+    return float(lib().oracle_metadata_bits_per_weight(_p(bits), _i64(bits.shape[0]), _i64(d_out),
+                                                       int(tag_bits), int(lut_bits)))
+
+
+def recon_error(X_u16, W_u16, dtype, lut, codes, rows, cols, vals, t_step=1):
+    """E = ||X (W - What)||_F in fp64, What = lut[code] + O (every t_step-th token)."""
+    X_u16 = _c(X_u16, np.uint16)
+    W_u16 = _c(W_u16, np.uint16)
+    n, d_in = X_u16.shape
+    d_out = W_u16.shape[1]
+    lut = _c(lut, np.float32)
+    codes = _c(codes, np.uint8)
+    rows = _c(rows, np.int32)
+    cols = _c(cols, np.int32)
+    vals = _c(vals, np.uint16)
+    return float(lib().oracle_recon_error(_p(X_u16), _p(W_u16), dtype, _i64(n), _i64(d_in),
+                                          _i64(d_out), _i64(d_in), _i64(d_out), _p(lut), _p(codes),
+                                          _p(rows), _p(cols), _p(vals), _i64(rows.shape[0]),
+                                          _i64(t_step)))
+
+
+def layer_pass(X_u16, W_u16, dtype, avg_bits, n_act, n_q, T):
+    """The whole pass for one layer in the paper's order; returns a dict of all outputs."""
+    X_u16 = _c(X_u16, np.uint16)
+    W_u16 = _c(W_u16, np.uint16)
+    n, d_in = X_u16.shape
+    d_out = W_u16.shape[1]
+    nnz = n_act * d_out + n_q
+    out = dict(a=np.empty(d_in, np.float32), bits=np.empty(d_in, np.uint8),
+               rows=np.empty(nnz, np.int32), cols=np.empty(nnz, np.int32),
+               vals=np.empty(nnz, np.uint16), lut=np.zeros((d_in, 16), np.float32),
+               codes=np.empty((d_in, d_out), np.uint8),
+               packed=np.zeros(d_in * ((d_out * 4 + 31) // 32), np.uint32),
+               row_off=np.empty(d_in + 1, np.int64), perm=np.empty(d_in, np.int32),
+               seg_rows=np.zeros(3, np.int64))
+    rc = lib().oracle_layer_pass(_p(X_u16), _p(W_u16), dtype, _i64(n), _i64(d_in), _i64(d_out),
+                                 _i64(d_in), _i64(d_out), ctypes.c_double(avg_bits), _i64(n_act),
+                                 _i64(n_q), int(T), _p(out["a"]), _p(out["bits"]), _p(out["rows"]),
+                                 _p(out["cols"]), _p(out["vals"]), _p(out["lut"]), _p(out["codes"]),
+                                 _p(out["packed"]), _p(out["row_off"]), _p(out["perm"]),
+                                 _p(out["seg_rows"]))
+    if rc:
+        raise ValueError("oracle_layer_pass failed with %d" % rc)
+    out["packed"] = out["packed"][: int(out["row_off"][-1])]
+    return out

@@ -1,0 +1,122 @@
+"""Seeded synthetic inputs shaped like the paper's LLM layers.
+
+This module holds input generation only -- none of the method's arithmetic -- so
+that the CUDA library's tests, the benchmark and the CPU checker can all be fed
+the same bytes.  Real LLaMA weights and C4 calibration text (Section 4.1 of the
+paper: 128 segments of 2048 tokens) are replaced by random tensors that keep the
+layer shapes, the storage dtype, the heavy-tailed weight entries and the
+channel-wise activation outliers shown in the paper's activation figure.
+
+Recipe
+  W [d_in][d_out] : N(0, 0.02^2); a Bernoulli(0.005) subset of the entries is
+                    replaced by 0.1 * StudentT(df=3); clamped to |w| <= 8;
+                    rounded to the 16-bit dtype; |w| < 2^-24 flushed to +0.
+  X [n][d_in]     : X[t,j] = z * sigma_j, z ~ N(0,1), sigma_j = exp(N(0,1)),
+                    multiplied by 50 on a random set of outlier channels
+                    (a fixed count, or round(0.01 * d_in)); clamped to +-60000
+                    for fp16; rounded to the dtype.
+Generation runs on whatever device is asked for with a torch.Generator seeded
+there, in fixed-size row chunks, so a (seed, device type) pair fixes the bytes.
+"""
+from dataclasses import dataclass, field
+from typing import List, Optional, Tuple
+
+import torch
+
+F16 = 0
+BF16 = 1
+
+_TORCH_DTYPE = {F16: torch.float16, BF16: torch.bfloat16}
+_W_CHUNK_ROWS = 1024
+_X_CHUNK_ROWS = 8192
+
+
+def torch_dtype(dtype_code: int) -> torch.dtype:
+    return _TORCH_DTYPE[dtype_code]
+
+
+def make_weight(d_in: int, d_out: int, dtype_code: int, seed: int, device="cpu") -> torch.Tensor:
+    """Weight matrix in the library's layout: row i = input channel i, d_out contiguous weights."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(int(seed))
+    out = torch.empty((d_in, d_out), dtype=_TORCH_DTYPE[dtype_code], device=dev)
+    for r0 in range(0, d_in, _W_CHUNK_ROWS):
+        r1 = min(d_in, r0 + _W_CHUNK_ROWS)
+        shape = (r1 - r0, d_out)
+        w = torch.randn(shape, generator=g, device=dev, dtype=torch.float32) * 0.02
+        mask = torch.rand(shape, generator=g, device=dev) < 0.005
+        z = torch.randn(shape, generator=g, device=dev, dtype=torch.float32)
+        chi = torch.randn((3,) + shape, generator=g, device=dev, dtype=torch.float32).square().sum(0)
+        t3 = z / torch.sqrt(chi / 3.0)
+        w = torch.where(mask, 0.1 * t3, w).clamp_(-8.0, 8.0)
+        w16 = w.to(_TORCH_DTYPE[dtype_code])
+        w16 = torch.where(w16.float().abs() < 2.0 ** -24, torch.zeros_like(w16), w16)
+        out[r0:r1] = w16
+    return out
+
+
+def make_activations(n_tokens: int, d_in: int, dtype_code: int, seed: int, device="cpu",
+                     n_outlier_channels: Optional[int] = None) -> torch.Tensor:
+    """Calibration activations [n_tokens][d_in] with channel-wise outliers."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(int(seed) + 7919)
+    sigma = torch.exp(torch.randn(d_in, generator=g, device=dev, dtype=torch.float32))
+    if n_outlier_channels is None:
+        n_outlier_channels = int(round(0.01 * d_in))
+    chosen = torch.randperm(d_in, generator=g, device=dev)[:n_outlier_channels]
+    sigma[chosen] *= 50.0
+    out = torch.empty((n_tokens, d_in), dtype=_TORCH_DTYPE[dtype_code], device=dev)
+    for r0 in range(0, n_tokens, _X_CHUNK_ROWS):
+        r1 = min(n_tokens, r0 + _X_CHUNK_ROWS)
+        x = torch.randn((r1 - r0, d_in), generator=g, device=dev, dtype=torch.float32) * sigma
+        if dtype_code == F16:
+            x.clamp_(-60000.0, 60000.0)
+        out[r0:r1] = x.to(_TORCH_DTYPE[dtype_code])
+    return out
+
+
+def as_u16(t: torch.Tensor):
+    """The raw 16-bit patterns of an fp16/bf16 tensor as a numpy uint16 array (host copy)."""
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view("uint16")
+
+
+@dataclass(frozen=True)
+class Layer:
+    d_in: int
+    d_out: int
+
+
+@dataclass(frozen=True)
+class Config:
+    """One workload: layers (d_in, d_out), storage dtype, calibration tokens, budgets, Lloyd iterations."""
+    name: str
+    layers: Tuple[Layer, ...]
+    dtype: int
+    n_tokens: int
+    budgets: Tuple[float, ...]
+    lloyd_iters: int
+    seed: int
+    n_outlier_channels: Optional[int] = None  # None -> round(0.01 * d_in)
+    repeat: int = 1  # how many times the layer list occurs (transformer blocks)
+
+
+# Shapes are given in the paper's orientation: d_in input channels of d_out weights each.
+_ATTN = Layer(4096, 4096)
+_UP = Layer(4096, 11008)
+_DOWN = Layer(11008, 4096)
+
+CONFIGS = {
+    "c1_small": Config("c1_small", (Layer(512, 512),), F16, 512, (3.0,), 10, 0, n_outlier_channels=8),
+    "c2_attn7b": Config("c2_attn7b", (_ATTN,), BF16, 131072, (2.2,), 20, 2000),
+    "c3_mlp7b": Config("c3_mlp7b", (_UP, _DOWN), BF16, 131072, (2.0, 2.5, 3.0, 3.5, 4.0), 20, 3000),
+    "c4_stack7b": Config("c4_stack7b", (_ATTN, _ATTN, _ATTN, _ATTN, _UP, _UP, _DOWN), BF16, 131072,
+                         (3.0,), 20, 4000, repeat=32),
+    "c5_mlp70b": Config("c5_mlp70b", (Layer(8192, 28672), Layer(28672, 8192)), BF16, 65536, (2.5,),
+                        20, 5000),
+}
+
+
+def layer_seed(cfg: Config, layer_index: int) -> int:
+    return cfg.seed + layer_index
