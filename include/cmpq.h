@@ -1,0 +1,159 @@
+/*
+ * cmpq.h -- C ABI of the CMPQ quantization pass for one linear layer on one GPU.
+ *
+ * CMPQ (channel-wise mixed-precision quantization, arxiv 2410.13056) quantizes a
+ * weight matrix W in R^{d_in x d_out} channel by channel, a channel being the row
+ * W_{i,:} that multiplies input feature i (Section 3.2.1).  The pass is:
+ *   statistic   a_j = ||X[:,j]||_2 over the calibration tokens     (Section 3.2.1)
+ *   allocation  c in {2,3,4}^{d_in} for an average budget b         (Algorithm 1)
+ *   outliers    O_act (whole channels, largest a) and O_q (entries a
+ *               provisional K-means fits worst), kept in 16 bits    (Section 3.2.2)
+ *   quantizer   per channel K-means with K = 2^{c_i}, nearest-centroid
+ *               codes                                               (Sections 3, 3.2.1)
+ *   packing     codes grouped by bit width into bit streams         (Sections 5.1, 6)
+ *
+ * Conventions for every entry point
+ *  - All array arguments are DEVICE pointers owned by the caller unless the
+ *    parameter comment says "host".  The library keeps no state and allocates no
+ *    memory; scratch space is the caller's `ws` buffer of at least
+ *    cmpq_workspace_bytes(op, ...) bytes, 256-byte aligned, whose contents are
+ *    undefined before and after the call.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *    only enqueue work; outputs are valid once the stream has been synchronised.
+ *  - Matrices are row-major with a leading dimension in elements (ldx, ldw).
+ *    16-bit floating inputs (cmpq_dtype) are passed as const void*.
+ *  - Arguments are checked on the host before anything is launched.  A call
+ *    returns CMPQ_OK or an error code and never throws, aborts or prints;
+ *    after an error no output has been written.
+ *  - Inputs must be finite.
+ *  - Results are deterministic: the same inputs give the same bytes.
+ */
+#ifndef CMPQ_H_
+#define CMPQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CMPQ_OK = 0,
+    CMPQ_ERR_INVALID_ARG = 1, /* null pointer, negative size, budget outside [2,4], ... */
+    CMPQ_ERR_UNSUPPORTED = 2, /* legal but outside what the kernels handle (see each call) */
+    CMPQ_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than cmpq_workspace_bytes */
+    CMPQ_ERR_CUDA = 4,        /* a CUDA runtime call failed */
+    CMPQ_ERR_INTERNAL = 5
+} cmpq_status;
+
+typedef enum { CMPQ_F16 = 0, CMPQ_BF16 = 1 } cmpq_dtype;
+
+/* How Algorithm 1's "q-quantile" is read.  RANK: the floor(|b-3| d_in + 1/2)
+ * channels with the smallest (b < 3) or largest (b > 3) statistic change width
+ * (at b == 3 exactly: floor(0.01 d_in + 1/2) at each end); equal statistics are
+ * ordered by channel id.  QUANTILE: thresholds are linearly interpolated
+ * quantiles of a and the comparisons are strict, as the algorithm is printed. */
+typedef enum { CMPQ_ALLOC_RANK = 0, CMPQ_ALLOC_QUANTILE = 1 } cmpq_alloc_mode;
+
+typedef enum {
+    CMPQ_OP_COLLECT_STATS = 0,
+    CMPQ_OP_ALLOCATE_BITS = 1,
+    CMPQ_OP_EXTRACT_OUTLIERS = 2,
+    CMPQ_OP_QUANTIZE_LAYER = 3,
+    CMPQ_OP_PACK = 4
+} cmpq_op;
+
+#define CMPQ_LUT_STRIDE 16      /* floats per channel in a look-up table */
+#define CMPQ_MAX_D_OUT 32768    /* one thread block holds one channel */
+#define CMPQ_MAX_D_IN 262144
+#define CMPQ_MAX_LLOYD_ITERS 1000
+
+/* ---- statistic (Section 3.2.1: per-channel L2 norm of the activation matrix X) --------------
+ * sumsq[j] += sum_t X[t*ldx + j]^2 for the n_tokens rows given; call it once per chunk of
+ * calibration tokens after zeroing sumsq (fp64, d_in entries).  Squares are formed in fp32
+ * (exact for 16-bit inputs), partial sums in fp32 over at most 64 rows, the rest in fp64 in
+ * a fixed order.  n_tokens may be 0.  X is [n_tokens][ldx] of `dt`, ldx >= d_in.
+ * ws: cmpq_workspace_bytes(CMPQ_OP_COLLECT_STATS, d_in, 0). */
+cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                               int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
+                               void* stream);
+
+/* a[j] = (float) sqrt(sumsq[j]). */
+cmpq_status cmpq_finalize_stats(const double* sumsq, int64_t d_in, float* a, void* stream);
+
+/* ---- allocation (Algorithm 1) ------------------------------------------------------------------
+ * bits[i] in {2,3,4} from the statistic a (fp32, d_in entries, finite, >= 0) and the average
+ * budget avg_bits in [2,4] (else CMPQ_ERR_INVALID_ARG).  order (optional, may be NULL) receives
+ * the channel ids sorted ascending by (a, id).
+ * ws: cmpq_workspace_bytes(CMPQ_OP_ALLOCATE_BITS, d_in, 0). */
+cmpq_status cmpq_allocate_bits(const float* a, int64_t d_in, double avg_bits, cmpq_alloc_mode mode,
+                               uint8_t* bits, int32_t* order, void* ws, size_t ws_bytes,
+                               void* stream);
+
+/* ---- outlier protection (Section 3.2.2) ------------------------------------------------------
+ * O_act: the n_act channels with the largest (a, id), kept whole.  W' = W with those rows set
+ * to +0.  Every channel of W' is fitted by K-means with K = 2^bits[i] and lloyd_iters updates
+ * (start, tie and rounding rules: see cmpq_quantize_layer).  O_q: the n_q entries outside O_act
+ * rows with the largest fp32 error |W' - W'_q|, equal errors by smaller i*d_out + j.
+ * Output: the union as coordinate lists sorted by (row, col); vals are the original 16-bit
+ * patterns of W.  nnz_out must equal n_act*d_out + n_q (the arrays' length).
+ * W is [d_in][ldw] of `dt`, ldw >= d_out, 1 <= d_out <= CMPQ_MAX_D_OUT.
+ * 0 <= n_act <= d_in, 0 <= n_q <= (d_in - n_act)*d_out.
+ * ws: cmpq_workspace_bytes(CMPQ_OP_EXTRACT_OUTLIERS, d_in, d_out)  (holds one fp32 per weight). */
+cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                  int64_t ldw, const float* a, const uint8_t* bits, int64_t n_act,
+                                  int64_t n_q, int lloyd_iters, int32_t* rows, int32_t* cols,
+                                  uint16_t* vals, int64_t nnz_out, void* ws, size_t ws_bytes,
+                                  void* stream);
+
+/* ---- channel-wise non-uniform quantization (Sections 3 and 3.2.1, final step of 3.2.2) -------
+ * W'' = W with the nnz listed positions (sorted by (row, col), e.g. from cmpq_extract_outliers;
+ * rows/cols may be NULL when nnz == 0) set to +0.  For every channel i, K = 2^bits[i]:
+ *   start       c_k = the ((2k+1) d_out)/(2K)-th smallest value (integer division)
+ *   assignment  the first k minimising fabsf(x - c_k) in fp32
+ *   update      c_k = (float)(sum of members in fp64 / count); an empty cluster keeps c_k
+ * exactly lloyd_iters updates (1..CMPQ_MAX_LLOYD_ITERS; 0 is allowed and returns the start),
+ * then a last assignment.  lut: [d_in][CMPQ_LUT_STRIDE] fp32, the first K entries valid, the
+ * rest 0.  codes: [d_in][d_out] uint8.
+ * sens: must be NULL (the paper's K-means is unweighted); non-NULL gives CMPQ_ERR_UNSUPPORTED.
+ * inexact_rows (optional device int32, caller zeroes it): incremented for every channel whose
+ * dynamic range is so wide that fp64 cluster sums may depend on the order of summation; when
+ * it stays 0 the centroids are independent of the summation order, hence reproducible bit
+ * for bit by any other correct implementation.
+ * sweeps (optional device uint64, caller zeroes it): receives the total number of
+ * (weight, centroid) distance evaluations performed, for throughput accounting.
+ * ws: cmpq_workspace_bytes(CMPQ_OP_QUANTIZE_LAYER, d_in, d_out). */
+cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                int64_t ldw, const uint8_t* bits, const int32_t* rows,
+                                const int32_t* cols, int64_t nnz, int lloyd_iters,
+                                const float* sens, float* lut, uint8_t* codes,
+                                int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
+                                size_t ws_bytes, void* stream);
+
+/* ---- packing (accounting of Section 5.1; per-precision sub-matrices of Section 6) -----------
+ * Three segments in the order 2-, 3-, 4-bit channels, channels by ascending id inside a
+ * segment.  perm[r] = channel stored at position r; row_off[r] = its first 32-bit word
+ * (row_off[d_in] = total words = cmpq_packed_words); seg_rows[0..2] = channels per segment.
+ * A channel's codes form an LSB-first bit stream (code j at bits [j*c, (j+1)*c)) cut into
+ * little-endian 32-bit words, the last one zero padded.  packed must hold
+ * cmpq_packed_words() words.  seg_rows is a DEVICE array of 3 int64.
+ * ws: cmpq_workspace_bytes(CMPQ_OP_PACK, d_in, d_out). */
+cmpq_status cmpq_pack(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
+                      uint32_t* packed, int64_t* row_off, int32_t* perm, int64_t* seg_rows,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/* ---- host helpers (pure functions, no GPU work) ----------------------------------------------- */
+size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out);
+/* Algorithm 1 in rank form: how many channels get 2 and 4 bits. */
+void cmpq_alloc_counts(int64_t d_in, double avg_bits, int64_t* n2, int64_t* n4);
+/* Section 3.2.2 budget: n_act = 45*d_in/10000, n_q = 5*d_in*d_out/10000 (integer division). */
+void cmpq_default_counts(int64_t d_in, int64_t d_out, int64_t* n_act, int64_t* n_q);
+/* Sum over channels of ceil(d_out*bits/32); bits_host is a HOST array. */
+int64_t cmpq_packed_words(const uint8_t* bits_host, int64_t d_in, int64_t d_out);
+const char* cmpq_status_string(cmpq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CMPQ_H_ */

@@ -1,0 +1,155 @@
+"""Thin ctypes binding of the C ABI in include/cmpq.h.
+
+Argument marshalling only: every step of the pass runs in the CUDA library.  Tensors are
+torch CUDA tensors (torch is used for device memory and streams, nothing else); each function
+has the name and the argument order of its C counterpart, enqueues work on the current torch
+stream and raises CmpqError when the library returns a non-zero status.  There is no CPU
+fallback: if libcmpq.so is missing or does not load, the first call raises.
+"""
+import ctypes
+import os
+
+import torch
+
+F16, BF16 = 0, 1
+ALLOC_RANK, ALLOC_QUANTILE = 0, 1
+OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK = range(5)
+LUT_STRIDE = 16
+
+EXPORTS = (
+    "cmpq_collect_stats", "cmpq_finalize_stats", "cmpq_allocate_bits", "cmpq_extract_outliers",
+    "cmpq_quantize_layer", "cmpq_pack", "cmpq_workspace_bytes", "cmpq_alloc_counts",
+    "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
+)
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
+_lib = None
+
+
+class CmpqError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        msg = lib().cmpq_status_string(self.status).decode()
+        super().__init__("%s failed: %s (status %d)" % (where, msg, self.status))
+
+
+def lib():
+    """Loads libcmpq.so once; raises if it was not built (run paper_2410_13056_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing: build it with "
+                               "`python -m paper_2410_13056_b200.build`" % _LIB_PATH)
+        L = ctypes.CDLL(_LIB_PATH)
+        i64, vp, dbl, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_double, ctypes.c_size_t
+        ci = ctypes.c_int
+        L.cmpq_collect_stats.argtypes = [vp, ci, i64, i64, i64, vp, vp, sz, vp]
+        L.cmpq_finalize_stats.argtypes = [vp, i64, vp, vp]
+        L.cmpq_allocate_bits.argtypes = [vp, i64, dbl, ci, vp, vp, vp, sz, vp]
+        L.cmpq_extract_outliers.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp,
+                                            i64, vp, sz, vp]
+        L.cmpq_quantize_layer.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp,
+                                          vp, vp, sz, vp]
+        L.cmpq_pack.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp]
+        for name in ("cmpq_collect_stats", "cmpq_finalize_stats", "cmpq_allocate_bits",
+                     "cmpq_extract_outliers", "cmpq_quantize_layer", "cmpq_pack"):
+            getattr(L, name).restype = ci
+        L.cmpq_workspace_bytes.argtypes = [ci, i64, i64]
+        L.cmpq_workspace_bytes.restype = sz
+        L.cmpq_alloc_counts.argtypes = [i64, dbl, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.cmpq_alloc_counts.restype = None
+        L.cmpq_default_counts.argtypes = [i64, i64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.cmpq_default_counts.restype = None
+        L.cmpq_packed_words.argtypes = [vp, i64, i64]
+        L.cmpq_packed_words.restype = i64
+        L.cmpq_status_string.argtypes = [ci]
+        L.cmpq_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status, where):
+    if status != 0:
+        raise CmpqError(status, where)
+
+
+def dtype_code(t):
+    if t.dtype == torch.float16:
+        return F16
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("expected a float16 or bfloat16 tensor, got %s" % t.dtype)
+
+
+def cmpq_workspace_bytes(op, d_in, d_out=0):
+    return int(lib().cmpq_workspace_bytes(op, d_in, d_out))
+
+
+def workspace(op, d_in, d_out=0, device="cuda"):
+    """A fresh scratch buffer of the size the given call needs."""
+    return torch.empty(max(256, cmpq_workspace_bytes(op, d_in, d_out)), dtype=torch.uint8, device=device)
+
+
+def cmpq_alloc_counts(d_in, avg_bits):
+    n2, n4 = ctypes.c_int64(), ctypes.c_int64()
+    lib().cmpq_alloc_counts(d_in, avg_bits, ctypes.byref(n2), ctypes.byref(n4))
+    return n2.value, n4.value
+
+
+def cmpq_default_counts(d_in, d_out):
+    n_act, n_q = ctypes.c_int64(), ctypes.c_int64()
+    lib().cmpq_default_counts(d_in, d_out, ctypes.byref(n_act), ctypes.byref(n_q))
+    return n_act.value, n_q.value
+
+
+def cmpq_packed_words(bits_host, d_out):
+    """bits_host: a CPU uint8 tensor."""
+    b = bits_host.contiguous()
+    return int(lib().cmpq_packed_words(ctypes.c_void_p(b.data_ptr()), b.numel(), d_out))
+
+
+def cmpq_collect_stats(X, sumsq, ws):
+    """sumsq (float64 [d_in]) += column sums of squares of X ([n_tokens][d_in], fp16/bf16)."""
+    n, d_in = X.shape
+    _check(lib().cmpq_collect_stats(_ptr(X), dtype_code(X), n, d_in, X.stride(0) if n > 0 else d_in,
+                                    _ptr(sumsq), _ptr(ws), ws.numel(), _stream()), "cmpq_collect_stats")
+
+
+def cmpq_finalize_stats(sumsq, a):
+    _check(lib().cmpq_finalize_stats(_ptr(sumsq), sumsq.numel(), _ptr(a), _stream()), "cmpq_finalize_stats")
+
+
+def cmpq_allocate_bits(a, avg_bits, mode, bits, order, ws):
+    _check(lib().cmpq_allocate_bits(_ptr(a), a.numel(), float(avg_bits), int(mode), _ptr(bits), _ptr(order),
+                                    _ptr(ws), ws.numel(), _stream()), "cmpq_allocate_bits")
+
+
+def cmpq_extract_outliers(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, ws):
+    d_in, d_out = W.shape
+    _check(lib().cmpq_extract_outliers(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
+                                       n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals),
+                                       rows.numel(), _ptr(ws), ws.numel(), _stream()), "cmpq_extract_outliers")
+
+
+def cmpq_quantize_layer(W, bits, rows, cols, lloyd_iters, lut, codes, ws, sens=None, inexact_rows=None,
+                        sweeps=None):
+    d_in, d_out = W.shape
+    nnz = 0 if rows is None else rows.numel()
+    _check(lib().cmpq_quantize_layer(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(bits),
+                                     _ptr(rows) if nnz else None, _ptr(cols) if nnz else None, nnz,
+                                     lloyd_iters, _ptr(sens), _ptr(lut), _ptr(codes), _ptr(inexact_rows),
+                                     _ptr(sweeps), _ptr(ws), ws.numel(), _stream()), "cmpq_quantize_layer")
+
+
+def cmpq_pack(codes, bits, packed, row_off, perm, seg_rows, ws):
+    d_in, d_out = codes.shape
+    _check(lib().cmpq_pack(_ptr(codes), _ptr(bits), d_in, d_out, _ptr(packed), _ptr(row_off), _ptr(perm),
+                           _ptr(seg_rows), _ptr(ws), ws.numel(), _stream()), "cmpq_pack")

@@ -1,0 +1,34 @@
+// Host-only helpers of the C ABI.
+#include "common.cuh"
+
+using namespace cmpq;
+
+extern "C" size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out) {
+    if (d_in < 1 || d_in > CMPQ_MAX_D_IN) return 0;
+    switch (op) {
+        case CMPQ_OP_COLLECT_STATS: return stats_ws_bytes(d_in);
+        case CMPQ_OP_ALLOCATE_BITS: return alloc_ws_bytes(d_in);
+        case CMPQ_OP_EXTRACT_OUTLIERS:
+            if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+            return outliers_ws_bytes(d_in, d_out);
+        case CMPQ_OP_QUANTIZE_LAYER:
+            if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+            return quantize_ws_bytes(d_in, d_out);
+        case CMPQ_OP_PACK:
+            if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+            return pack_ws_bytes(d_in, d_out);
+    }
+    return 0;
+}
+
+extern "C" const char* cmpq_status_string(cmpq_status s) {
+    switch (s) {
+        case CMPQ_OK: return "ok";
+        case CMPQ_ERR_INVALID_ARG: return "invalid argument";
+        case CMPQ_ERR_UNSUPPORTED: return "unsupported argument combination";
+        case CMPQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CMPQ_ERR_CUDA: return "CUDA runtime error";
+        case CMPQ_ERR_INTERNAL: return "internal error";
+    }
+    return "unknown status";
+}

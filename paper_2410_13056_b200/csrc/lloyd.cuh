@@ -1,0 +1,36 @@
+// Channel-wise K-means of CMPQ (Section 3.2.1; quantizer of Section 3): launch interface.
+#pragma once
+
+#include "common.cuh"
+
+namespace cmpq {
+
+// What one launch of the channel kernel reads and writes.
+struct LloydArgs {
+    const uint16_t* W;       // [d_in][ldw] 16-bit weights
+    int64_t d_in, d_out, ldw;
+    const uint8_t* bits;     // [d_in] in {2,3,4}
+    int iters;               // centroid updates T
+    // provisional fit (Section 3.2.2): rows flagged in skip_row are not fitted, every other
+    // row writes err[i*d_out + j] = |x - nearest centroid|
+    const uint8_t* skip_row; // [d_in] or NULL
+    float* err;              // [d_in*d_out] or NULL
+    // final fit: positions row_ptr[i]..row_ptr[i+1] of cols are set to +0 before fitting
+    const int64_t* row_ptr;  // [d_in+1] or NULL
+    const int32_t* cols;     // [nnz] or NULL
+    float* lut;              // [d_in][16] or NULL
+    uint8_t* codes;          // [d_in][d_out] or NULL
+    int32_t* inexact_rows;   // optional counter
+    unsigned long long* sweeps;  // optional counter of distance evaluations
+};
+
+cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
+
+// Fills row_ptr[0..d_in] from a row-sorted coordinate list.
+cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64_t* row_ptr,
+                           cudaStream_t st);
+
+// rank[i] = position of channel i in the ascending order of (a, id).
+cmpq_status launch_rank(const float* a, int64_t d_in, int32_t* rank, cudaStream_t st);
+
+}  // namespace cmpq

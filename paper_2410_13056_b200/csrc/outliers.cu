@@ -1,0 +1,313 @@
+// Outlier protection of CMPQ (Section 3.2.2).
+//
+//   O_act  the n_act channels with the largest activation statistic are kept whole
+//   O_q    after a provisional channel-wise K-means of W' = W - O_act, the n_q entries with the
+//          largest error |W' - W'_q| are kept as well (equal errors: smaller linear index first)
+//
+// The provisional fit writes one fp32 error per weight.  Errors are non-negative, so their
+// bit patterns order like integers: an exact three-pass radix select (12 + 10 + 10 bits) finds
+// the bit pattern tau of the n_q-th largest error and how many entries equal to tau still
+// belong to the set.  Per-row counts and one scan over the rows then give every row its slice
+// of the output, and each row writes its entries in column order, which yields the list sorted
+// by (row, col) without a sort.
+#include "lloyd.cuh"
+
+namespace cmpq {
+
+constexpr int kSelBins = 4096;
+constexpr int kSelThreads = 256;
+
+struct SelectState {
+    uint32_t prefix;        // bits of tau fixed so far
+    uint32_t mask;          // which bits are fixed
+    long long remaining;    // entries still to take among those matching prefix
+    uint32_t tau;           // final threshold pattern
+    long long take_equal;   // entries equal to tau that belong to the set
+};
+
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_totals, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    __syncthreads();  // warp_totals may still be read from a previous call
+    if (lane == 31) warp_totals[warp] = incl;
+    __syncthreads();
+    int base = 0, all = 0;
+    for (int w = 0; w < nwarps; ++w) {
+        int t = warp_totals[w];
+        if (w < warp) base += t;
+        all += t;
+    }
+    total = all;
+    return base + incl - v;
+}
+
+__global__ void mark_act_rows_kernel(const int32_t* __restrict__ rank, int64_t d_in, int64_t n_act,
+                                     uint8_t* __restrict__ is_act) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < d_in) is_act[i] = rank[i] >= d_in - n_act ? 1 : 0;
+}
+
+__global__ void select_init_kernel(SelectState* st, long long n_q) {
+    st->prefix = 0; st->mask = 0; st->remaining = n_q; st->tau = 0xffffffffu; st->take_equal = 0;
+}
+
+// hist[d] += number of errors in non-act rows whose fixed bits match the prefix and whose
+// digit (err >> shift) & (bins-1) equals d.  One block handles whole rows.
+__global__ void __launch_bounds__(kSelThreads)
+select_hist_kernel(const float* __restrict__ err, const uint8_t* __restrict__ is_act, int64_t d_in,
+                   int64_t d_out, const SelectState* __restrict__ st, int shift, int bins,
+                   unsigned int* __restrict__ hist) {
+    __shared__ unsigned int local[kSelBins];
+    for (int b = threadIdx.x; b < bins; b += blockDim.x) local[b] = 0;
+    __syncthreads();
+    const uint32_t prefix = st->prefix, mask = st->mask;
+    for (int64_t row = blockIdx.x; row < d_in; row += gridDim.x) {
+        if (is_act[row]) continue;
+        const uint32_t* e = reinterpret_cast<const uint32_t*>(err + row * d_out);
+        for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
+            uint32_t u = e[j];
+            if ((u & mask) == prefix) atomicAdd(&local[(u >> shift) & (bins - 1)], 1u);
+        }
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < bins; b += blockDim.x)
+        if (local[b]) atomicAdd(&hist[b], local[b]);
+}
+
+// Walks the histogram from the largest digit down to the one that holds the remaining-th
+// largest entry, fixes that digit in the prefix and clears the histogram for the next pass.
+__global__ void __launch_bounds__(1024)
+select_digit_kernel(unsigned int* __restrict__ hist, int shift, int bins, SelectState* st, int final_pass) {
+    __shared__ int warp_totals[32];
+    __shared__ int found_digit;
+    __shared__ long long found_above;
+    const int per = kSelBins / 1024;  // 4 bins per thread, descending digit order
+    const long long remaining = st->remaining;
+    int v[per], s = 0;
+#pragma unroll
+    for (int t = 0; t < per; ++t) {
+        int d = bins - 1 - (threadIdx.x * per + t);
+        v[t] = d >= 0 ? (int)hist[d] : 0;
+        s += v[t];
+    }
+    if (threadIdx.x == 0) found_digit = -1;
+    int total;
+    long long above = block_exclusive_scan(s, warp_totals, total);  // entries with a larger digit
+    if (remaining > 0 && above < remaining && remaining <= above + s) {
+#pragma unroll
+        for (int t = 0; t < per; ++t) {
+            if (above < remaining && remaining <= above + v[t]) {
+                found_digit = bins - 1 - (threadIdx.x * per + t);
+                found_above = above;
+            }
+            above += v[t];
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && found_digit >= 0) {
+        st->prefix |= (uint32_t)found_digit << shift;
+        st->mask |= (uint32_t)(bins - 1) << shift;
+        st->remaining = remaining - found_above;
+        if (final_pass) { st->tau = st->prefix; st->take_equal = st->remaining; }
+    }
+    for (int b = threadIdx.x; b < bins; b += blockDim.x) hist[b] = 0;
+}
+
+// Per row: how many errors exceed tau and how many equal it.
+__global__ void __launch_bounds__(kSelThreads)
+row_count_kernel(const float* __restrict__ err, const uint8_t* __restrict__ is_act, int64_t d_out,
+                 const SelectState* __restrict__ st, int32_t* __restrict__ gt,
+                 int32_t* __restrict__ eq) {
+    __shared__ int sg, se;
+    const int64_t row = blockIdx.x;
+    if (threadIdx.x == 0) { sg = 0; se = 0; }
+    __syncthreads();
+    int g = 0, q = 0;
+    if (!is_act[row]) {
+        const uint32_t tau = st->tau;
+        const uint32_t* e = reinterpret_cast<const uint32_t*>(err + row * d_out);
+        for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
+            uint32_t u = e[j];
+            g += u > tau ? 1 : 0;
+            q += u == tau ? 1 : 0;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        g += __shfl_xor_sync(0xffffffffu, g, o);
+        q += __shfl_xor_sync(0xffffffffu, q, o);
+    }
+    if ((threadIdx.x & 31) == 0) { if (g) atomicAdd(&sg, g); if (q) atomicAdd(&se, q); }
+    __syncthreads();
+    if (threadIdx.x == 0) { gt[row] = sg; eq[row] = se; }
+}
+
+// One block walks the rows in order: entries equal to tau are taken from the lowest rows first
+// until take_equal is used up; row_start is the exclusive scan of the rows' output counts.
+__global__ void __launch_bounds__(1024)
+row_scan_kernel(const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
+                const uint8_t* __restrict__ is_act, int64_t d_in, int64_t d_out,
+                const SelectState* __restrict__ st, int32_t* __restrict__ take_eq,
+                int64_t* __restrict__ row_start) {
+    __shared__ int warp_totals[32];
+    const long long take_equal = st->take_equal;
+    long long eq_before = 0, out_before = 0;
+    for (int64_t base = 0; base < d_in; base += blockDim.x) {
+        int64_t i = base + threadIdx.x;
+        int e = i < d_in ? eq[i] : 0;
+        int tot_e;
+        long long my_eq_before = eq_before + block_exclusive_scan(e, warp_totals, tot_e);
+        long long room = take_equal - my_eq_before;
+        int te = room <= 0 ? 0 : (room < e ? (int)room : e);
+        int sel = 0;
+        if (i < d_in) sel = is_act[i] ? (int)d_out : gt[i] + te;
+        int tot_s;
+        long long my_out_before = out_before + block_exclusive_scan(sel, warp_totals, tot_s);
+        if (i < d_in) { take_eq[i] = te; row_start[i] = my_out_before; }
+        eq_before += tot_e;
+        out_before += tot_s;
+    }
+    if (threadIdx.x == 0) row_start[d_in] = out_before;
+}
+
+// Each row writes its kept entries in column order.
+__global__ void __launch_bounds__(kSelThreads)
+emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __restrict__ err,
+            const uint8_t* __restrict__ is_act, int64_t d_out, const SelectState* __restrict__ st,
+            const int32_t* __restrict__ take_eq, const int64_t* __restrict__ row_start,
+            int32_t* __restrict__ rows, int32_t* __restrict__ cols, uint16_t* __restrict__ vals) {
+    __shared__ int warp_totals[32];
+    const int64_t row = blockIdx.x;
+    const int64_t out0 = row_start[row];
+    if (row_start[row + 1] == out0) return;
+    const bool act = is_act[row] != 0;
+    const uint32_t tau = st->tau;
+    const int te = take_eq[row];
+    const uint32_t* e = reinterpret_cast<const uint32_t*>(err + row * d_out);
+    const uint16_t* w = W + row * ldw;
+    int eq_seen = 0, written = 0;
+    for (int64_t base = 0; base < d_out; base += blockDim.x) {
+        int64_t j = base + threadIdx.x;
+        bool in = j < d_out;
+        uint32_t u = (in && !act) ? e[j] : 0u;
+        int is_eq = (in && !act && u == tau) ? 1 : 0;
+        int tot_eq;
+        int eq_rank = eq_seen + block_exclusive_scan(is_eq, warp_totals, tot_eq);
+        int keep = in && (act || u > tau || (is_eq && eq_rank < te)) ? 1 : 0;
+        int tot_keep;
+        int pos = written + block_exclusive_scan(keep, warp_totals, tot_keep);
+        if (keep) {
+            rows[out0 + pos] = (int32_t)row;
+            cols[out0 + pos] = (int32_t)j;
+            vals[out0 + pos] = w[j];
+        }
+        eq_seen += tot_eq;
+        written += tot_keep;
+    }
+}
+
+struct OutlierWs {
+    float* err;
+    int32_t* rank;
+    uint8_t* is_act;
+    unsigned int* hist;
+    SelectState* state;
+    int32_t* gt;
+    int32_t* eq;
+    int32_t* take_eq;
+    int64_t* row_start;
+};
+
+static OutlierWs carve(Workspace& w, int64_t d_in, int64_t d_out) {
+    OutlierWs o;
+    o.err = w.take<float>((size_t)d_in * (size_t)d_out);
+    o.rank = w.take<int32_t>(d_in);
+    o.is_act = w.take<uint8_t>(d_in);
+    o.hist = w.take<unsigned int>(kSelBins);
+    o.state = w.take<SelectState>(1);
+    o.gt = w.take<int32_t>(d_in);
+    o.eq = w.take<int32_t>(d_in);
+    o.take_eq = w.take<int32_t>(d_in);
+    o.row_start = w.take<int64_t>(d_in + 1);
+    return o;
+}
+
+size_t outliers_ws_bytes(int64_t d_in, int64_t d_out) {
+    Workspace w(nullptr, 0);
+    carve(w, d_in, d_out);
+    return w.used;
+}
+
+}  // namespace cmpq
+
+using namespace cmpq;
+
+extern "C" void cmpq_default_counts(int64_t d_in, int64_t d_out, int64_t* n_act, int64_t* n_q) {
+    if (n_act) *n_act = (45 * d_in) / 10000;
+    if (n_q) *n_q = (5 * d_in * d_out) / 10000;
+}
+
+extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                             int64_t ldw, const float* a, const uint8_t* bits,
+                                             int64_t n_act, int64_t n_q, int lloyd_iters,
+                                             int32_t* rows, int32_t* cols, uint16_t* vals,
+                                             int64_t nnz_out, void* ws, size_t ws_bytes, void* stream) {
+    if (!W || !a || !bits) return CMPQ_ERR_INVALID_ARG;
+    if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
+    if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT || ldw < d_out)
+        return CMPQ_ERR_INVALID_ARG;
+    if (n_act < 0 || n_act > d_in || n_q < 0 || n_q > (d_in - n_act) * d_out) return CMPQ_ERR_INVALID_ARG;
+    if (nnz_out != n_act * d_out + n_q) return CMPQ_ERR_INVALID_ARG;
+    if (nnz_out > 0 && (!rows || !cols || !vals)) return CMPQ_ERR_INVALID_ARG;
+    if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(W, 2)) return CMPQ_ERR_INVALID_ARG;
+    if (d_in * d_out > 0x7fffffffLL) return CMPQ_ERR_UNSUPPORTED;  // 32-bit counters in the select
+    if (!ws || !aligned_to(ws, 256) || ws_bytes < outliers_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Workspace wsp(ws, ws_bytes);
+    OutlierWs o = carve(wsp, d_in, d_out);
+    const unsigned row_blocks = (unsigned)((d_in + 255) / 256);
+
+    cmpq_status s = launch_rank(a, d_in, o.rank, st);
+    if (s != CMPQ_OK) return s;
+    mark_act_rows_kernel<<<row_blocks, 256, 0, st>>>(o.rank, d_in, n_act, o.is_act);
+
+    if (n_q > 0) {
+        LloydArgs la{};
+        la.W = static_cast<const uint16_t*>(W);
+        la.d_in = d_in; la.d_out = d_out; la.ldw = ldw;
+        la.bits = bits;
+        la.iters = lloyd_iters;
+        la.skip_row = o.is_act;
+        la.err = o.err;
+        s = launch_lloyd(la, dt, st);
+        if (s != CMPQ_OK) return s;
+    }
+
+    select_init_kernel<<<1, 1, 0, st>>>(o.state, (long long)n_q);
+    if (cudaMemsetAsync(o.hist, 0, kSelBins * sizeof(unsigned int), st) != cudaSuccess) return CMPQ_ERR_CUDA;
+    if (n_q > 0) {
+        int sms = sm_count();
+        if (sms <= 0) return CMPQ_ERR_CUDA;
+        unsigned hist_blocks = (unsigned)((int64_t)sms * 8 < d_in ? (int64_t)sms * 8 : d_in);
+        const int shifts[3] = {20, 10, 0};
+        const int bins[3] = {4096, 1024, 1024};
+        for (int p = 0; p < 3; ++p) {
+            select_hist_kernel<<<hist_blocks, kSelThreads, 0, st>>>(o.err, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist);
+            select_digit_kernel<<<1, 1024, 0, st>>>(o.hist, shifts[p], bins[p], o.state, p == 2);
+        }
+        row_count_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(o.err, o.is_act, d_out, o.state, o.gt, o.eq);
+    } else {
+        if (cudaMemsetAsync(o.gt, 0, (size_t)d_in * sizeof(int32_t), st) != cudaSuccess) return CMPQ_ERR_CUDA;
+        if (cudaMemsetAsync(o.eq, 0, (size_t)d_in * sizeof(int32_t), st) != cudaSuccess) return CMPQ_ERR_CUDA;
+    }
+    row_scan_kernel<<<1, 1024, 0, st>>>(o.gt, o.eq, o.is_act, d_in, d_out, o.state, o.take_eq, o.row_start);
+    if (nnz_out > 0)
+        emit_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(static_cast<const uint16_t*>(W), ldw, o.err, o.is_act, d_out, o.state, o.take_eq, o.row_start, rows, cols, vals);
+    return launch_status();
+}

@@ -1,0 +1,216 @@
+// Activation statistic of CMPQ (Section 3.2.1): per input channel j the sum over the
+// calibration tokens of X[t,j]^2, whose square root is the channel's L2 norm a_j.
+//
+// HBM-bound column reduction.  A warp reads 512 contiguous bytes of a row with one 128-bit
+// load per lane (8 adjacent columns per thread), eight warps of a block take eight rows at a
+// time, four rows are in flight per thread.  Squares are exact in fp32; a thread keeps fp32
+// partial sums for at most kFlushRows of its rows and folds them into fp64.  The blocks of
+// one column tile write fp64 partials to the work space; a second kernel adds them in a fixed
+// order, so the result does not depend on scheduling.
+#include "common.cuh"
+
+namespace cmpq {
+
+constexpr int kStatsThreads = 256;
+constexpr int kStatsWarps = kStatsThreads / 32;
+constexpr int kTileCols = 256;       // columns per block: 32 lanes x 8 columns
+constexpr int kFlushRows = 32;       // rows a thread sums in fp32 before folding into fp64
+constexpr int kMaxRowBlocks = 2048;  // upper bound used to size the work space
+constexpr int kCtasPerSm = 8;
+
+int sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return n;
+}
+
+static int64_t col_tiles(int64_t d_in) { return (d_in + kTileCols - 1) / kTileCols; }
+
+// Row blocks per column tile for a device with `sms` SMs: enough blocks to fill every SM
+// kCtasPerSm times, never more than kMaxRowBlocks / col_tiles (work-space bound).
+static int64_t row_blocks_for(int64_t d_in, int64_t n_tokens, int sms) {
+    int64_t ct = col_tiles(d_in);
+    int64_t want = ((int64_t)sms * kCtasPerSm + ct - 1) / ct;
+    int64_t cap = kMaxRowBlocks / ct;
+    if (cap < 1) cap = 1;
+    if (want > cap) want = cap;
+    int64_t by_rows = (n_tokens + kStatsWarps - 1) / kStatsWarps;  // at least one row per warp
+    if (want > by_rows) want = by_rows;
+    if (want < 1) want = 1;
+    return want;
+}
+
+size_t stats_ws_bytes(int64_t d_in) {
+    int64_t ct = col_tiles(d_in);
+    int64_t rb = kMaxRowBlocks / ct;
+    if (rb < 1) rb = 1;
+    return round_up((size_t)rb * (size_t)ct * kTileCols * sizeof(double), 256);
+}
+
+template <int DT>
+__device__ __forceinline__ void accumulate8(const uint4& v, float (&acc)[8]) {
+    float2 p0 = widen16x2<DT>(v.x), p1 = widen16x2<DT>(v.y);
+    float2 p2 = widen16x2<DT>(v.z), p3 = widen16x2<DT>(v.w);
+    acc[0] = fmaf(p0.x, p0.x, acc[0]);
+    acc[1] = fmaf(p0.y, p0.y, acc[1]);
+    acc[2] = fmaf(p1.x, p1.x, acc[2]);
+    acc[3] = fmaf(p1.y, p1.y, acc[3]);
+    acc[4] = fmaf(p2.x, p2.x, acc[4]);
+    acc[5] = fmaf(p2.y, p2.y, acc[5]);
+    acc[6] = fmaf(p3.x, p3.x, acc[6]);
+    acc[7] = fmaf(p3.y, p3.y, acc[7]);
+}
+
+// partial[(row_block * tiles + tile) * kTileCols + c] = sum over the block's rows of X[t, tile*256+c]^2
+template <int DT>
+__global__ void __launch_bounds__(kStatsThreads)
+stats_partial_vec_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64_t d_in, int64_t ldx,
+                         int64_t rows_per_block, double* __restrict__ partial) {
+    __shared__ double red[kStatsWarps][kTileCols];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t tile = blockIdx.x;
+    const int64_t col = tile * kTileCols + lane * 8;
+    const int64_t r0 = (int64_t)blockIdx.y * rows_per_block;
+    int64_t r1 = r0 + rows_per_block;
+    if (r1 > n_tokens) r1 = n_tokens;
+
+    double total[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) total[i] = 0.0;
+
+    if (col < d_in) {
+        const uint16_t* p = X + col;
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        int since_flush = 0;
+        int64_t r = r0 + warp;
+        for (; r + 3 * kStatsWarps < r1; r += 4 * kStatsWarps) {
+            uint4 v0 = __ldcs(reinterpret_cast<const uint4*>(p + r * ldx));
+            uint4 v1 = __ldcs(reinterpret_cast<const uint4*>(p + (r + kStatsWarps) * ldx));
+            uint4 v2 = __ldcs(reinterpret_cast<const uint4*>(p + (r + 2 * kStatsWarps) * ldx));
+            uint4 v3 = __ldcs(reinterpret_cast<const uint4*>(p + (r + 3 * kStatsWarps) * ldx));
+            accumulate8<DT>(v0, acc);
+            accumulate8<DT>(v1, acc);
+            accumulate8<DT>(v2, acc);
+            accumulate8<DT>(v3, acc);
+            since_flush += 4;
+            if (since_flush >= kFlushRows) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { total[i] += (double)acc[i]; acc[i] = 0.f; }
+                since_flush = 0;
+            }
+        }
+        for (; r < r1; r += kStatsWarps) {
+            uint4 v0 = __ldcs(reinterpret_cast<const uint4*>(p + r * ldx));
+            accumulate8<DT>(v0, acc);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) total[i] += (double)acc[i];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) red[warp][lane * 8 + i] = total[i];
+    __syncthreads();
+    // thread c adds the eight warps' sums of column c in warp order
+    const int c = threadIdx.x;
+    double s = 0.0;
+#pragma unroll
+    for (int w = 0; w < kStatsWarps; ++w) s += red[w][c];
+    partial[((int64_t)blockIdx.y * gridDim.x + tile) * kTileCols + c] = s;
+}
+
+// Same contract for inputs that cannot be read with aligned 128-bit loads: one column per thread.
+template <int DT>
+__global__ void __launch_bounds__(kStatsThreads)
+stats_partial_scalar_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64_t d_in,
+                            int64_t ldx, int64_t rows_per_block, double* __restrict__ partial) {
+    const int64_t tile = blockIdx.x;
+    const int64_t col = tile * kTileCols + threadIdx.x;
+    const int64_t r0 = (int64_t)blockIdx.y * rows_per_block;
+    int64_t r1 = r0 + rows_per_block;
+    if (r1 > n_tokens) r1 = n_tokens;
+    double total = 0.0;
+    if (col < d_in) {
+        float acc = 0.f;
+        int since_flush = 0;
+        for (int64_t r = r0; r < r1; ++r) {
+            float x = widen16<DT>(X[r * ldx + col]);
+            acc = fmaf(x, x, acc);
+            if (++since_flush == kFlushRows) { total += (double)acc; acc = 0.f; since_flush = 0; }
+        }
+        total += (double)acc;
+    }
+    partial[((int64_t)blockIdx.y * gridDim.x + tile) * kTileCols + threadIdx.x] = total;
+}
+
+// sumsq[j] += sum over row blocks (ascending) of partial[rb][j]
+__global__ void stats_combine_kernel(const double* __restrict__ partial, int64_t row_blocks,
+                                     int64_t padded_cols, int64_t d_in, double* __restrict__ sumsq) {
+    int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d_in) return;
+    double s = 0.0;
+    for (int64_t rb = 0; rb < row_blocks; ++rb) s += partial[rb * padded_cols + j];
+    sumsq[j] += s;
+}
+
+__global__ void stats_finalize_kernel(const double* __restrict__ sumsq, int64_t d_in,
+                                      float* __restrict__ a) {
+    int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < d_in) a[j] = (float)sqrt(sumsq[j]);
+}
+
+// Launches the two statistic kernels with `partial` as scratch (row_blocks * tiles * 256 doubles).
+cmpq_status launch_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                 int64_t ldx, double* sumsq, double* partial, int64_t row_blocks,
+                                 cudaStream_t st) {
+    const int64_t ct = col_tiles(d_in);
+    const int64_t rows_per_block = (n_tokens + row_blocks - 1) / row_blocks;
+    const bool vec = aligned_to(X, 16) && (ldx % 8 == 0) && (d_in % 8 == 0);
+    dim3 grid((unsigned)ct, (unsigned)row_blocks);
+    const uint16_t* Xp = static_cast<const uint16_t*>(X);
+    if (vec) {
+        if (dt == CMPQ_F16)
+            stats_partial_vec_kernel<CMPQ_F16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+        else
+            stats_partial_vec_kernel<CMPQ_BF16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+    } else {
+        if (dt == CMPQ_F16)
+            stats_partial_scalar_kernel<CMPQ_F16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+        else
+            stats_partial_scalar_kernel<CMPQ_BF16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+    }
+    stats_combine_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, st>>>(partial, row_blocks, ct * kTileCols, d_in, sumsq);
+    return launch_status();
+}
+
+int64_t stats_row_blocks(int64_t d_in, int64_t n_tokens) {
+    int sms = sm_count();
+    if (sms <= 0) return 0;
+    return row_blocks_for(d_in, n_tokens, sms);
+}
+
+}  // namespace cmpq
+
+using namespace cmpq;
+
+extern "C" cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                          int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
+                                          void* stream) {
+    if (!sumsq || n_tokens < 0 || d_in < 1 || d_in > CMPQ_MAX_D_IN || ldx < d_in) return CMPQ_ERR_INVALID_ARG;
+    if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
+    if (n_tokens > 0 && !X) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(X, 2) || !aligned_to(sumsq, 8)) return CMPQ_ERR_INVALID_ARG;
+    if (!ws || !aligned_to(ws, 256) || ws_bytes < stats_ws_bytes(d_in)) return CMPQ_ERR_WORKSPACE;
+    if (n_tokens == 0) return CMPQ_OK;
+    int64_t rb = stats_row_blocks(d_in, n_tokens);
+    if (rb <= 0) return CMPQ_ERR_CUDA;
+    return launch_collect_stats(X, dt, n_tokens, d_in, ldx, sumsq, static_cast<double*>(ws), rb,
+                                static_cast<cudaStream_t>(stream));
+}
+
+extern "C" cmpq_status cmpq_finalize_stats(const double* sumsq, int64_t d_in, float* a, void* stream) {
+    if (!sumsq || !a || d_in < 1 || d_in > CMPQ_MAX_D_IN) return CMPQ_ERR_INVALID_ARG;
+    stats_finalize_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(sumsq, d_in, a);
+    return launch_status();
+}

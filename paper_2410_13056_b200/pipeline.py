@@ -1,0 +1,86 @@
+"""The whole CMPQ pass for one linear layer as a chain of C-ABI calls.
+
+LayerQuantizer owns the device buffers of one layer shape (outputs and scratch, allocated once
+through torch) and enqueues, on the current stream and without host synchronisation, the calls
+in the paper's order: statistic (Section 3.2.1) -> Algorithm 1 -> outlier protection
+(Section 3.2.2) -> channel-wise K-means and codes -> packing (Section 5.1).  It computes
+nothing itself.
+"""
+from dataclasses import dataclass
+
+import torch
+
+from . import binding as B
+
+
+@dataclass
+class LayerResult:
+    """Views of the quantizer's output buffers (overwritten by the next run)."""
+    a: torch.Tensor          # [d_in] fp32 activation statistic
+    bits: torch.Tensor       # [d_in] uint8 in {2,3,4}
+    rows: torch.Tensor       # [nnz] int32 outlier coordinates, sorted by (row, col)
+    cols: torch.Tensor       # [nnz] int32
+    vals: torch.Tensor       # [nnz] int16 raw 16-bit patterns of the kept weights
+    lut: torch.Tensor        # [d_in][16] fp32 centroids
+    codes: torch.Tensor      # [d_in][d_out] uint8
+    packed: torch.Tensor     # [words] int32 bit streams
+    row_off: torch.Tensor    # [d_in+1] int64 word offsets in segment order
+    perm: torch.Tensor       # [d_in] int32 channel ids in segment order
+    seg_rows: torch.Tensor   # [3] int64 channels per width 2,3,4
+    inexact_rows: torch.Tensor  # [1] int32
+    sweeps: torch.Tensor     # [1] int64 distance evaluations of the final fit
+
+
+class LayerQuantizer:
+    def __init__(self, d_in, d_out, device="cuda", n_act=None, n_q=None):
+        self.d_in, self.d_out = int(d_in), int(d_out)
+        self.device = torch.device(device)
+        da, dq = B.cmpq_default_counts(self.d_in, self.d_out)
+        self.n_act = da if n_act is None else int(n_act)
+        self.n_q = dq if n_q is None else int(n_q)
+        self.nnz = self.n_act * self.d_out + self.n_q
+        dev = self.device
+        ws_bytes = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out) for op in range(5))
+        self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+        self.sumsq = torch.empty(self.d_in, dtype=torch.float64, device=dev)
+        self.a = torch.empty(self.d_in, dtype=torch.float32, device=dev)
+        self.bits = torch.empty(self.d_in, dtype=torch.uint8, device=dev)
+        self.rows = torch.empty(self.nnz, dtype=torch.int32, device=dev)
+        self.cols = torch.empty(self.nnz, dtype=torch.int32, device=dev)
+        self.vals = torch.empty(self.nnz, dtype=torch.int16, device=dev)
+        self.lut = torch.empty((self.d_in, B.LUT_STRIDE), dtype=torch.float32, device=dev)
+        self.codes = torch.empty((self.d_in, self.d_out), dtype=torch.uint8, device=dev)
+        max_words = self.d_in * ((self.d_out * 4 + 31) // 32)
+        self.packed = torch.empty(max_words, dtype=torch.int32, device=dev)
+        self.row_off = torch.empty(self.d_in + 1, dtype=torch.int64, device=dev)
+        self.perm = torch.empty(self.d_in, dtype=torch.int32, device=dev)
+        self.seg_rows = torch.empty(3, dtype=torch.int64, device=dev)
+        self.counters = torch.zeros(4, dtype=torch.int64, device=dev)
+
+    def packed_words(self, avg_bits):
+        """Words the rank-form allocation produces for this budget (no device read needed)."""
+        n2, n4 = B.cmpq_alloc_counts(self.d_in, avg_bits)
+        n3 = self.d_in - n2 - n4
+        w = lambda c: (self.d_out * c + 31) // 32
+        return n2 * w(2) + n3 * w(3) + n4 * w(4)
+
+    def run(self, X, W, avg_bits, lloyd_iters, stats_only=False):
+        """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out]."""
+        assert W.shape == (self.d_in, self.d_out) and X.shape[1] == self.d_in
+        self.sumsq.zero_()
+        self.counters.zero_()
+        B.cmpq_collect_stats(X, self.sumsq, self.ws)
+        B.cmpq_finalize_stats(self.sumsq, self.a)
+        if stats_only:
+            return None
+        B.cmpq_allocate_bits(self.a, avg_bits, B.ALLOC_RANK, self.bits, None, self.ws)
+        B.cmpq_extract_outliers(W, self.a, self.bits, self.n_act, self.n_q, lloyd_iters, self.rows,
+                                self.cols, self.vals, self.ws)
+        inexact = self.counters[0:1].view(torch.int32)[0:1]
+        sweeps = self.counters[1:2]
+        B.cmpq_quantize_layer(W, self.bits, self.rows, self.cols, lloyd_iters, self.lut, self.codes,
+                              self.ws, inexact_rows=inexact, sweeps=sweeps)
+        B.cmpq_pack(self.codes, self.bits, self.packed, self.row_off, self.perm, self.seg_rows, self.ws)
+        words = self.packed_words(avg_bits)
+        return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
+                           self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)

@@ -1,0 +1,146 @@
+"""GPU parity of the whole pass (the chain of C-ABI calls) on the small workload in full and on
+the Llama-shaped workloads through samples and properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2410_13056_b200 import binding as B
+from paper_2410_13056_b200 import inputs
+from paper_2410_13056_b200.pipeline import LayerQuantizer
+
+pytestmark = pytest.mark.gpu
+
+
+def _np(r):
+    out = {k: getattr(r, k).cpu().numpy() for k in ("a", "bits", "rows", "cols", "lut", "codes", "row_off",
+                                                     "perm", "seg_rows")}
+    out["vals"] = r.vals.cpu().numpy().view(np.uint16)
+    out["packed"] = r.packed.cpu().numpy().view(np.uint32)
+    return out
+
+
+def _chain_with_gpu_statistic(Wu, dtype, a_gpu, b, n_act, n_q, T):
+    """The checker's steps 2..8 fed with the statistic the GPU produced (the statistic itself is
+    compared within tolerance; everything after it must then agree bit for bit)."""
+    bits, _ = oracle.allocate_bits(a_gpu, b)
+    rows, cols, vals = oracle.extract_outliers(Wu, dtype, a_gpu, bits, n_act, n_q, T)
+    lut, codes = oracle.quantize_layer(Wu, dtype, bits, rows, cols, T)
+    packed, row_off, perm, seg = oracle.pack(codes, bits)
+    return dict(bits=bits, rows=rows, cols=cols, vals=vals, lut=lut, codes=codes, packed=packed,
+                row_off=row_off, perm=perm, seg_rows=seg)
+
+
+def test_small_workload_full_parity():
+    cfg = inputs.CONFIGS["c1_small"]
+    L = cfg.layers[0]
+    W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, cfg.seed, device="cuda")
+    X = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, cfg.seed, device="cuda",
+                                n_outlier_channels=cfg.n_outlier_channels)
+    q = LayerQuantizer(L.d_in, L.d_out)
+    assert (q.n_act, q.n_q, q.nnz) == (2, 131, 1155)
+    g = _np(q.run(X, W, 3.0, cfg.lloyd_iters))
+    Xu, Wu = inputs.as_u16(X), inputs.as_u16(W)
+    ref = oracle.layer_pass(Xu, Wu, cfg.dtype, 3.0, q.n_act, q.n_q, cfg.lloyd_iters)
+    np.testing.assert_allclose(g["a"], ref["a"], rtol=1e-5)
+    for k in ("bits", "rows", "cols", "vals", "codes", "packed", "row_off", "perm", "seg_rows"):
+        assert np.array_equal(g[k], ref[k]), k
+    np.testing.assert_allclose(g["lut"], ref["lut"], rtol=1e-4)
+    assert g["packed"].nbytes == 98304 and int(q.counters[0].item()) == 0
+    # reconstruction error ||X (W - What)||_F: both sides evaluated by the checker in fp64
+    Eg = oracle.recon_error(Xu, Wu, cfg.dtype, g["lut"], g["codes"], g["rows"], g["cols"], g["vals"])
+    Er = oracle.recon_error(Xu, Wu, cfg.dtype, ref["lut"], ref["codes"], ref["rows"], ref["cols"], ref["vals"])
+    assert Eg == pytest.approx(Er, rel=1e-4)
+    # and on the device in fp32 from the library's own outputs
+    What = torch.gather(q.lut, 1, q.codes.long())
+    What[q.rows.long(), q.cols.long()] += W[q.rows.long(), q.cols.long()].float()
+    E32 = torch.linalg.norm(X.float() @ (W.float() - What)).item()
+    assert E32 == pytest.approx(Er, rel=1e-4)
+    # a second run gives the same bytes
+    g2 = _np(q.run(X, W, 3.0, cfg.lloyd_iters))
+    for k in g:
+        assert np.array_equal(g[k], g2[k]), k
+
+
+@pytest.mark.parametrize("b", [2.0, 2.2, 3.0, 3.5, 4.0])
+def test_midsize_layer_all_budgets(b):
+    d_in, d_out, n, T = 256, 1536, 2048, 12
+    W = inputs.make_weight(d_in, d_out, inputs.BF16, 31, device="cuda")
+    X = inputs.make_activations(n, d_in, inputs.BF16, 31, device="cuda")
+    q = LayerQuantizer(d_in, d_out)
+    g = _np(q.run(X, W, b, T))
+    Xu, Wu = inputs.as_u16(X), inputs.as_u16(W)
+    a_ref = oracle.finalize_stats(oracle.collect_stats(Xu, inputs.BF16))
+    np.testing.assert_allclose(g["a"], a_ref, rtol=1e-5)
+    ref = _chain_with_gpu_statistic(Wu, inputs.BF16, g["a"], b, q.n_act, q.n_q, T)
+    for k, v in ref.items():
+        if k == "lut":
+            np.testing.assert_allclose(g[k], v, rtol=1e-4)
+        else:
+            assert np.array_equal(g[k], v), k
+    assert abs(g["bits"].mean() - b) <= 0.5 / d_in or b == 3.0
+
+
+def test_llama_attention_shape_sampled_parity():
+    """The benchmark's workload (4096 x 4096 bf16, 131072 tokens, 2.2 bits, 20 iterations) in the
+    launch configuration the benchmark uses; the checker verifies sampled channels and global
+    properties instead of re-running everything."""
+    cfg = inputs.CONFIGS["c2_attn7b"]
+    L = cfg.layers[0]
+    b, T = cfg.budgets[0], cfg.lloyd_iters
+    W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, cfg.seed, device="cuda")
+    X = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, cfg.seed, device="cuda")
+    q = LayerQuantizer(L.d_in, L.d_out)
+    r = q.run(X, W, b, T)
+    g = _np(r)
+    assert int(q.counters[0].item()) == 0
+    # statistic: sampled columns against the checker (fp64, token order)
+    colsel = np.array([0, 1, 7, 8, 255, 256, 1000, 2047, 4095] + list(np.argsort(g["a"])[-4:]))
+    Xs = X[:, torch.from_numpy(colsel).cuda()].contiguous()
+    a_ref = oracle.finalize_stats(oracle.collect_stats(inputs.as_u16(Xs), cfg.dtype))
+    np.testing.assert_allclose(g["a"][colsel], a_ref, rtol=1e-5)
+    # allocation: exact, from the GPU statistic
+    bits_ref, order_ref = oracle.allocate_bits(g["a"], b)
+    assert np.array_equal(g["bits"], bits_ref)
+    assert (g["bits"] == 2).sum() == 3277 and (g["bits"] == 4).sum() == 0
+    # outlier list: structure and O_act rows
+    d_in, d_out = L.d_in, L.d_out
+    assert (q.n_act, q.n_q, q.nnz) == (18, 8388, 82116)
+    lin = g["rows"].astype(np.int64) * d_out + g["cols"]
+    assert np.all(np.diff(lin) > 0)
+    Wu = inputs.as_u16(W)
+    assert np.array_equal(g["vals"], Wu[g["rows"], g["cols"]])
+    per_row = np.bincount(g["rows"], minlength=d_in)
+    act_rows = np.sort(order_ref[d_in - q.n_act:])
+    assert np.array_equal(np.flatnonzero(per_row == d_out), act_rows)
+    assert per_row[per_row < d_out].sum() == q.n_q
+    # O_q: the provisional fit of sampled rows reproduces exactly the entries taken in those rows,
+    # and no error left behind in a sampled row exceeds the smallest error taken anywhere sampled
+    is_act = np.zeros(d_in, bool); is_act[act_rows] = True
+    sample = [i for i in (0, 1, 17, 511, 2048, 4095, int(np.argmax(per_row * ~is_act))) if not is_act[i]]
+    Wf = W.float().cpu().numpy()
+    taken_min, left_max = np.inf, 0.0
+    for i in sample:
+        _, _, err = oracle.lloyd(Wf[i], 1 << int(bits_ref[i]), T)
+        mine = g["cols"][g["rows"] == i]
+        mask = np.zeros(d_out, bool); mask[mine] = True
+        if mask.any():
+            taken_min = min(taken_min, err[mask].min())
+        left_max = max(left_max, err[~mask].max())
+        if mask.any() and (~mask).any():
+            assert err[mask].min() >= err[~mask].max()
+    assert left_max <= taken_min
+    # final fit: sampled channels (all widths present, an O_act row, the row with most O_q entries)
+    sample2 = sample + [int(act_rows[0]), int(np.flatnonzero(bits_ref == 3)[0]), int(np.flatnonzero(bits_ref == 2)[-1])]
+    for i in sample2:
+        x = Wf[i].copy()
+        x[g["cols"][g["rows"] == i]] = 0
+        lut, code, _ = oracle.lloyd(x, 1 << int(bits_ref[i]), T)
+        assert np.array_equal(code, g["codes"][i]), i
+        np.testing.assert_allclose(g["lut"][i], lut, rtol=1e-4)
+    assert g["codes"].max() < 8 and np.all(g["codes"][bits_ref == 2] < 4)
+    # packing: full comparison against the checker's packer (cheap), 4 613 632 bytes at 2.2 bits
+    packed, row_off, perm, seg = oracle.pack(g["codes"], g["bits"])
+    assert np.array_equal(g["packed"], packed) and np.array_equal(g["row_off"], row_off)
+    assert np.array_equal(g["perm"], perm) and np.array_equal(g["seg_rows"], seg)
+    assert g["packed"].nbytes == 4613632

@@ -1,0 +1,190 @@
+"""GPU parity: every C-ABI call against the CPU checker on the same seeded inputs.
+Bit-exact for bits, order, outlier lists, codes and packed words; the statistic within 1e-5
+relative (fp32 partial sums over at most 32 rows, fp64 above); centroids within 1e-4 relative
+(expected equal bit for bit while no channel is flagged as inexact)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2410_13056_b200 import binding as B
+from paper_2410_13056_b200 import inputs
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+STAT_RTOL = 1e-5
+LUT_RTOL = 1e-4
+
+
+def _lut_close(got, ref, W_absmax):
+    np.testing.assert_allclose(got, ref, rtol=LUT_RTOL, atol=LUT_RTOL * W_absmax * 1e-3)
+
+
+# ----------------------------------------------------------------------------- statistic
+@pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
+@pytest.mark.parametrize("n,d_in", [(512, 512), (1000, 264), (37, 1544), (3000, 4096), (1, 8), (9, 2056)])
+def test_stats_vector_path(dtype, n, d_in):
+    X = inputs.make_activations(n, d_in, dtype, 5, device="cuda", n_outlier_channels=3)
+    sumsq, a = G.gpu_stats(X)
+    ref = oracle.finalize_stats(oracle.collect_stats(inputs.as_u16(X), dtype))
+    np.testing.assert_allclose(a, ref, rtol=STAT_RTOL)
+    assert np.array_equal(a, np.sqrt(sumsq).astype(np.float32))
+
+
+@pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
+def test_stats_ragged_strided_and_chunked(dtype):
+    # d_in not a multiple of 8 -> scalar path; a column slice of a wider matrix -> ldx > d_in
+    X = inputs.make_activations(777, 301, dtype, 6, device="cuda")
+    _, a = G.gpu_stats(X)
+    ref = oracle.finalize_stats(oracle.collect_stats(inputs.as_u16(X), dtype))
+    np.testing.assert_allclose(a, ref, rtol=STAT_RTOL)
+    Xw = inputs.make_activations(500, 640, dtype, 7, device="cuda")
+    for view in (Xw[:, 64:576], Xw[:, 3:260]):          # aligned slice, misaligned slice
+        _, a = G.gpu_stats(view)
+        ref = oracle.finalize_stats(oracle.collect_stats(inputs.as_u16(view.contiguous()), dtype))
+        np.testing.assert_allclose(a, ref, rtol=STAT_RTOL)
+    # accumulation over three chunks of tokens, one of them empty
+    s1, a1 = G.gpu_stats(Xw, chunks=1)
+    s3, a3 = G.gpu_stats(Xw, chunks=3)
+    np.testing.assert_allclose(s3, s1, rtol=1e-6)
+    sumsq = torch.ones(640, dtype=torch.float64, device="cuda")
+    B.cmpq_collect_stats(Xw[:0], sumsq, B.workspace(B.OP_COLLECT_STATS, 640))
+    assert torch.all(sumsq == 1.0)
+
+
+def test_stats_closed_forms_and_determinism():
+    X = torch.zeros(4096, 512, dtype=torch.bfloat16, device="cuda")
+    X[:, 0] = 1.5
+    X[100, 1] = -3.0
+    X[:, 2] = 2.0 ** -20
+    _, a = G.gpu_stats(X)
+    assert a[0] == np.float32(1.5 * 64) and a[1] == 3.0 and a[2] == np.float32(2.0 ** -20 * 64) and a[3] == 0
+    Y = inputs.make_activations(5000, 1024, inputs.BF16, 8, device="cuda")
+    s1, _ = G.gpu_stats(Y)
+    s2, _ = G.gpu_stats(Y)
+    assert np.array_equal(s1, s2)
+
+
+# ----------------------------------------------------------------------------- Algorithm 1
+@pytest.mark.parametrize("d_in", [1, 5, 512, 4096, 11008, 28672])
+@pytest.mark.parametrize("b", [2.0, 2.2, 2.5, 3.0, 3.7, 4.0])
+def test_allocation_bit_exact(d_in, b):
+    rng = np.random.default_rng(d_in + int(b * 10))
+    a = np.exp(rng.standard_normal(d_in)).astype(np.float32)
+    a[rng.integers(0, d_in, d_in // 7)] = a[0]            # ties
+    for mode in (B.ALLOC_RANK, B.ALLOC_QUANTILE):
+        bits, order = G.gpu_allocate(a, b, mode)
+        rbits, rorder = oracle.allocate_bits(a, b, mode)
+        assert np.array_equal(order, rorder)
+        assert np.array_equal(bits, rbits)
+    bits, _ = G.gpu_allocate(a, b, want_order=False)
+    assert np.array_equal(bits, oracle.allocate_bits(a, b)[0])
+
+
+# ----------------------------------------------------------------------------- K-means, outliers
+def _case(d_in, d_out, dtype, seed, b):
+    W = inputs.make_weight(d_in, d_out, dtype, seed, device="cuda")
+    rng = np.random.default_rng(seed)
+    a = np.exp(rng.standard_normal(d_in)).astype(np.float32)
+    bits, _ = oracle.allocate_bits(a, b)
+    return W, inputs.as_u16(W), a, bits
+
+
+@pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
+@pytest.mark.parametrize("d_in,d_out,T", [(96, 512, 10), (40, 1000, 6), (24, 4096, 20), (12, 11008, 5),
+                                          (6, 28672, 4), (50, 37, 12), (64, 16, 30), (9, 1, 3), (5, 32768, 2)])
+def test_quantize_layer_matches_checker(dtype, d_in, d_out, T):
+    W, Wu, a, bits = _case(d_in, d_out, dtype, 21 + d_out, 3.0)
+    bits[: d_in // 3] = 2
+    bits[d_in // 3: 2 * d_in // 3] = 4
+    rng = np.random.default_rng(d_out)
+    nnz = min(d_in * d_out // 50, 500)
+    lin = np.sort(rng.choice(d_in * d_out, nnz, replace=False))
+    rows, cols = (lin // d_out).astype(np.int32), (lin % d_out).astype(np.int32)
+    lut, codes, inexact, sweeps = G.gpu_quantize(W, bits, rows, cols, T)
+    rlut, rcodes = oracle.quantize_layer(Wu, dtype, bits, rows, cols, T)
+    assert inexact == 0
+    assert np.array_equal(codes, rcodes)
+    assert np.array_equal(lut.view(np.uint32), rlut.view(np.uint32))   # stronger than LUT_RTOL
+    _lut_close(lut, rlut, 8.0)
+    assert 0 < sweeps <= (T + 1) * d_out * int((1 << bits.astype(np.int64)).sum())
+
+
+def test_quantize_layer_degenerate_channels():
+    d_out = 256
+    rows_ = []
+    rows_.append(np.zeros(d_out))                                       # all zero
+    rows_.append(np.full(d_out, 0.375))                                 # constant
+    rows_.append(np.where(np.arange(d_out) % 8 == 0, -3.0, 1.0))        # two values
+    z = np.zeros(d_out); z[::2] = -0.0; rows_.append(z)                 # signed zeros
+    r = np.zeros(d_out); r[:5] = [1, 2, 3, 4, 5]; rows_.append(r)       # mass on one value -> duplicate starts
+    rows_.append(np.linspace(-1, 1, d_out))
+    rows_.append(np.arange(d_out) % 3 - 1.0)                            # three values
+    Wt = torch.tensor(np.stack(rows_), dtype=torch.float16).cuda()
+    Wu = inputs.as_u16(Wt)
+    none = np.zeros(0, np.int32)
+    for c in (2, 3, 4):
+        for T in (0, 1, 3, 25):
+            bits = np.full(len(rows_), c, np.uint8)
+            lut, codes, inexact, _ = G.gpu_quantize(Wt, bits, none, none, T)
+            rlut, rcodes = oracle.quantize_layer(Wu, inputs.F16, bits, none, none, T)
+            assert np.array_equal(codes, rcodes), (c, T)
+            assert np.array_equal(lut.view(np.uint32), rlut.view(np.uint32)), (c, T)
+
+
+def test_wide_dynamic_range_is_flagged_not_hidden():
+    d_out = 512
+    x = np.random.default_rng(0).standard_normal((4, d_out)).astype(np.float32)
+    x[1, 0] = 2.0 ** 60
+    x[1, 1] = 2.0 ** -60
+    Wt = torch.tensor(x, dtype=torch.bfloat16).cuda()
+    bits = np.full(4, 3, np.uint8)
+    none = np.zeros(0, np.int32)
+    lut, codes, inexact, _ = G.gpu_quantize(Wt, bits, none, none, 10)
+    assert inexact == 1
+    rlut, rcodes = oracle.quantize_layer(inputs.as_u16(Wt), inputs.BF16, bits, none, none, 10)
+    np.testing.assert_allclose(lut, rlut, rtol=LUT_RTOL)
+
+
+@pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
+@pytest.mark.parametrize("d_in,d_out,n_act,n_q,T", [(64, 512, 2, 40, 8), (48, 1000, 0, 77, 5), (40, 300, 3, 0, 5),
+                                                    (33, 4096, 1, 500, 10), (20, 64, 0, 0, 3), (16, 11008, 1, 88, 4),
+                                                    (10, 50, 2, 8 * 50, 4)])
+def test_extract_outliers_bit_exact(dtype, d_in, d_out, n_act, n_q, T):
+    W, Wu, a, bits = _case(d_in, d_out, dtype, 77 + d_in, 2.5)
+    rows, cols, vals = G.gpu_extract(W, a, bits, n_act, n_q, T)
+    rr, rc, rv = oracle.extract_outliers(Wu, dtype, a, bits, n_act, n_q, T)
+    assert np.array_equal(rows, rr) and np.array_equal(cols, rc) and np.array_equal(vals, rv)
+
+
+def test_extract_outliers_ties_across_rows():
+    d_in, d_out = 12, 128
+    base = (np.linspace(-1, 1, d_out) ** 3).astype(np.float16)
+    Wt = torch.from_numpy(np.tile(base, (d_in, 1))).cuda()
+    a = np.arange(d_in, dtype=np.float32)
+    bits = np.full(d_in, 2, np.uint8)
+    for n_q in (1, 7, 11, 12, 30):
+        got = G.gpu_extract(Wt, a, bits, 1, n_q, 4)
+        ref = oracle.extract_outliers(inputs.as_u16(Wt), inputs.F16, a, bits, 1, n_q, 4)
+        for g, r in zip(got, ref):
+            assert np.array_equal(g, r), n_q
+
+
+# ----------------------------------------------------------------------------- packing
+@pytest.mark.parametrize("d_in,d_out", [(23, 1), (23, 31), (23, 32), (23, 33), (40, 100), (16, 4096), (9, 11008),
+                                        (300, 512), (7, 28672), (5, 1000)])
+def test_pack_bit_exact(d_in, d_out):
+    rng = np.random.default_rng(d_in * d_out)
+    bits = rng.integers(2, 5, d_in).astype(np.uint8)
+    codes = (rng.integers(0, 16, (d_in, d_out)) & ((1 << bits[:, None]) - 1)).astype(np.uint8)
+    got = G.gpu_pack(codes, bits)
+    ref = oracle.pack(codes, bits)
+    for g, r, name in zip(got, ref, ("packed", "row_off", "perm", "seg_rows")):
+        assert np.array_equal(g, r), name
+    for only in (2, 3, 4):                                   # single-width layers leave segments empty
+        b1 = np.full(d_in, only, np.uint8)
+        c1 = codes & ((1 << only) - 1)
+        for g, r in zip(G.gpu_pack(c1, b1), oracle.pack(c1, b1)):
+            assert np.array_equal(g, r)
