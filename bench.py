@@ -1,0 +1,286 @@
+"""Benchmark of the CMPQ quantization pass: weights quantized per second on one Llama-7B-shaped
+attention projection (4096 x 4096 bf16 weights, 131072 calibration tokens, 20 Lloyd iterations).
+
+A step is one whole pass over one layer: statistic -> Algorithm 1 -> outlier protection (with its
+provisional K-means) -> final K-means and codes -> packing.  `value` is measured with the inputs
+resident in HBM, `e2e` through the same public call with pinned HOST buffers (copies timed).
+`--impl reference` times the plain CPU checker instead (on a bounded sample of the same layer).
+With N > 1 ranks (torchrun) every rank quantizes its own layer -- layers are independent, so
+there is no collective on the data path -- and `value` is the aggregate.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "weights quantized/sec (Mparams/s) at avg 3.0 bits; % of HBM / FP32 roofline"
+UNIT = "Mparams/s"
+WORKLOAD = "c2_attn7b"
+METRIC_BUDGET = 3.0          # the metric is quoted at an average of 3.0 bits
+SM_COUNT, FP32_LANES_PER_SM = 148, 128
+CPU_BASELINE_CHANNELS = 4096   # cpu_baseline leg: the whole layer (about 15 s on one core)
+REFERENCE_ARM_CHANNELS = 1024  # --impl reference: a quarter of the layer per step
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), float(p.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        out, _ = self.proc.communicate(timeout=10)
+        clocks, max_clock, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) != 6:
+                continue
+            try:
+                clocks.append(float(parts[0]))
+                max_clock = float(parts[1])
+            except ValueError:
+                continue
+            for name, flag in zip(names, parts[2:]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [c for c in clocks if max_clock and c > 0.3 * max_clock] or clocks
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max_clock,
+                "reasons": sorted(reasons), "samples": len(clocks)}
+
+
+def _visible_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        ids = [v for v in vis.split(",") if v]
+        if local_rank < len(ids) and ids[local_rank].isdigit():
+            return int(ids[local_rank])
+    return local_rank
+
+
+def cpu_reference_sample(cfg, layer, channels):
+    """Inputs of the CPU leg: `channels` input channels of the layer with all of their d_out weights
+    and all calibration tokens, so the work per weight is that of the full layer."""
+    from paper_2410_13056_b200 import inputs
+    import oracle
+
+    W = inputs.make_weight(channels, layer.d_out, cfg.dtype, cfg.seed)
+    X = inputs.make_activations(cfg.n_tokens, channels, cfg.dtype, cfg.seed)
+    n_act, n_q = oracle.default_counts(channels, layer.d_out)
+    return inputs.as_u16(X), inputs.as_u16(W), n_act, n_q
+
+
+def time_cpu_reference(cfg, layer, budget, steps, warmup, channels):
+    import oracle
+
+    oracle.build()
+    Xu, Wu, n_act, n_q = cpu_reference_sample(cfg, layer, channels)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.layer_pass(Xu, Wu, cfg.dtype, budget, n_act, n_q, cfg.lloyd_iters)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    params = Wu.shape[0] * Wu.shape[1]
+    sec = sum(times) / len(times)
+    sample = ("%d of %d input channels x %d weights, all %d tokens, one thread"
+              % (Wu.shape[0], layer.d_in, layer.d_out, cfg.n_tokens))
+    return params / sec / 1e6, sec, sample
+
+
+def run_reference(args, cfg, layer):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    value, sec, sample = time_cpu_reference(cfg, layer, METRIC_BUDGET, args.steps, max(args.warmup, 0),
+                                            REFERENCE_ARM_CHANNELS)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD + " shape at avg 3.0 bits, CPU checker on a sample", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2410_13056_b200 import inputs
+
+    cfg = inputs.CONFIGS[WORKLOAD]
+    layer = cfg.layers[0]
+    if args.impl == "reference":
+        run_reference(args, cfg, layer)
+        return
+
+    import torch
+    from paper_2410_13056_b200.pipeline import LayerQuantizer, KERNELS_PER_RUN
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    warmup = max(args.warmup, 3)
+    steps = args.steps
+    seed = cfg.seed + 100 * rank   # every rank quantizes its own layer
+    W = inputs.make_weight(layer.d_in, layer.d_out, cfg.dtype, seed, device="cuda")
+    X = inputs.make_activations(cfg.n_tokens, layer.d_in, cfg.dtype, seed, device="cuda")
+    q = LayerQuantizer(layer.d_in, layer.d_out)
+    params = layer.d_in * layer.d_out
+
+    def timed(budget, k, ev=None):
+        for _ in range(warmup):
+            q.run(X, W, budget, cfg.lloyd_iters)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(k):
+            q.run(X, W, budget, cfg.lloyd_iters, events=None if ev is None else ev[i])
+        e1.record()
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1)) / k
+
+    # device-resident throughput at the metric's budget, per-call events for the roofline
+    sampler = ClockSampler(_visible_index(local_rank))
+    events = [dict() for _ in range(steps)]
+    sampler.start()
+    ms = timed(METRIC_BUDGET, steps, events)
+    clocks = sampler.stop()
+    value = world * params / (ms * 1e-3) / 1e6
+    sweeps_evals = int(q.counters[1].item())
+    per_call = {}
+    for name in events[0]:
+        per_call[name] = statistics.mean(e[name][0].elapsed_time(e[name][1]) for e in events)
+    ms_22 = timed(cfg.budgets[0], max(3, steps // 2))
+
+    # roofline of the dominant kernel: the channel K-means of the final fit (cmpq_quantize_layer is
+    # that kernel plus a microsecond-sized index kernel); 2 ops (subtract, compare/select) per
+    # (weight, centroid) distance evaluation actually executed
+    hbm_peak, sm_max_mhz, peak_kind = _peaks()
+    alu_peak_tflops = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    lloyd_ms = per_call["cmpq_quantize_layer"]
+    achieved = 2.0 * sweeps_evals / (lloyd_ms * 1e-3) / 1e12
+    stats_ms = per_call["cmpq_collect_stats"]
+    stats_gbs = X.numel() * 2 / (stats_ms * 1e-3) / 1e9
+    pack_ms = per_call["cmpq_pack"]
+    pack_gbs = params * (1 + METRIC_BUDGET / 8) / (pack_ms * 1e-3) / 1e9
+    roofline = {"bound": "alu", "kernel": "lloyd_kernel (final fit)", "achieved": achieved,
+                "peak": alu_peak_tflops, "unit": "TFLOP/s", "frac": achieved / alu_peak_tflops,
+                "peak_kind": "148 SMs x 128 fp32 lanes x %.0f MHz, one op per lane per clock" % sm_max_mhz,
+                "traffic": None,
+                "other_kernels": {
+                    "stats": {"bound": "hbm", "achieved": stats_gbs, "peak": hbm_peak, "unit": "GB/s",
+                              "frac": stats_gbs / hbm_peak, "peak_kind": peak_kind},
+                    "pack": {"bound": "hbm", "achieved": pack_gbs, "peak": hbm_peak, "unit": "GB/s",
+                             "frac": pack_gbs / hbm_peak, "peak_kind": peak_kind}}}
+
+    # end to end through the public call with host buffers
+    Xh = torch.empty(X.shape, dtype=X.dtype, pin_memory=True)
+    Wh = torch.empty(W.shape, dtype=W.dtype, pin_memory=True)
+    Xh.copy_(X)
+    Wh.copy_(W)
+    host_out = q.make_host_outputs(METRIC_BUDGET)
+    e2e_steps = max(3, min(steps, 5))
+    for _ in range(2):
+        q.run_host(Xh, Wh, METRIC_BUDGET, cfg.lloyd_iters, host_out)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        q.run_host(Xh, Wh, METRIC_BUDGET, cfg.lloyd_iters, host_out)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    e2e = {"value": world * params / (e2e_ms * 1e-3) / 1e6, "unit": UNIT,
+           "h2d_bytes_per_step": Xh.numel() * 2 + Wh.numel() * 2,
+           "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in host_out.values()),
+           "ms_per_step": e2e_ms}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, sec, sample = time_cpu_reference(cfg, layer, METRIC_BUDGET, 1, 0, CPU_BASELINE_CHANNELS)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                        "seconds": sec}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "c2_attn7b: W 4096x4096 bf16, X 131072x4096 bf16, 20 Lloyd iterations, "
+                                   "avg 3.0 bits (the metric's budget); one layer per step per GPU",
+                       "l2": "inputs larger than L2 (X is 1 GiB per step)",
+                       "n_act": q.n_act, "n_q": q.n_q},
+            "at_config_budget": {"avg_bits": cfg.budgets[0], "value": world * params / (ms_22 * 1e-3) / 1e6,
+                                 "unit": UNIT, "ms_per_step": ms_22},
+            "per_call_ms": per_call,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_RUN * steps,
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -12,6 +12,11 @@ import torch
 
 from . import binding as B
 
+# CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0:
+# statistic 2 + finalize 1, allocation 2, outliers 13 (rank, mark, K-means, select init, 3 x
+# (histogram, digit), row count, row scan, emit), final fit 2, packing 2.
+KERNELS_PER_RUN = 22
+
 
 @dataclass
 class LayerResult:
@@ -64,23 +69,60 @@ class LayerQuantizer:
         w = lambda c: (self.d_out * c + 31) // 32
         return n2 * w(2) + n3 * w(3) + n4 * w(4)
 
-    def run(self, X, W, avg_bits, lloyd_iters, stats_only=False):
-        """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out]."""
+    def run(self, X, W, avg_bits, lloyd_iters, events=None):
+        """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
+        events (optional dict) receives a (start, end) CUDA event pair per C-ABI call."""
         assert W.shape == (self.d_in, self.d_out) and X.shape[1] == self.d_in
+
+        def call(name, fn, *args, **kw):
+            if events is None:
+                fn(*args, **kw)
+                return
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(*args, **kw)
+            e1.record()
+            events[name] = (e0, e1)
+
         self.sumsq.zero_()
         self.counters.zero_()
-        B.cmpq_collect_stats(X, self.sumsq, self.ws)
-        B.cmpq_finalize_stats(self.sumsq, self.a)
-        if stats_only:
-            return None
-        B.cmpq_allocate_bits(self.a, avg_bits, B.ALLOC_RANK, self.bits, None, self.ws)
-        B.cmpq_extract_outliers(W, self.a, self.bits, self.n_act, self.n_q, lloyd_iters, self.rows,
-                                self.cols, self.vals, self.ws)
         inexact = self.counters[0:1].view(torch.int32)[0:1]
         sweeps = self.counters[1:2]
-        B.cmpq_quantize_layer(W, self.bits, self.rows, self.cols, lloyd_iters, self.lut, self.codes,
-                              self.ws, inexact_rows=inexact, sweeps=sweeps)
-        B.cmpq_pack(self.codes, self.bits, self.packed, self.row_off, self.perm, self.seg_rows, self.ws)
+        call("cmpq_collect_stats", B.cmpq_collect_stats, X, self.sumsq, self.ws)
+        call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
+        call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
+             self.ws)
+        call("cmpq_extract_outliers", B.cmpq_extract_outliers, W, self.a, self.bits, self.n_act, self.n_q,
+             lloyd_iters, self.rows, self.cols, self.vals, self.ws)
+        call("cmpq_quantize_layer", B.cmpq_quantize_layer, W, self.bits, self.rows, self.cols, lloyd_iters,
+             self.lut, self.codes, self.ws, inexact_rows=inexact, sweeps=sweeps)
+        call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
+             self.seg_rows, self.ws)
         words = self.packed_words(avg_bits)
         return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
                            self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)
+
+    # ---- host-buffer entry: the same pass with the copies a caller holding host tensors pays ----
+    def make_host_outputs(self, avg_bits):
+        """Pinned host tensors for everything a caller stores for one quantized layer."""
+        words = self.packed_words(avg_bits)
+        pin = lambda t, n=None: torch.empty(t.shape if n is None else (n,), dtype=t.dtype, pin_memory=True)
+        return {"bits": pin(self.bits), "rows": pin(self.rows), "cols": pin(self.cols), "vals": pin(self.vals),
+                "lut": pin(self.lut), "packed": pin(self.packed, words), "row_off": pin(self.row_off),
+                "perm": pin(self.perm), "seg_rows": pin(self.seg_rows), "counters": pin(self.counters)}
+
+    def run_host(self, X_host, W_host, avg_bits, lloyd_iters, host_out):
+        """X_host, W_host: pinned host tensors.  Copies them in, runs the pass, copies the stored
+        representation (not the byte codes) back into host_out and waits for it."""
+        if not hasattr(self, "_Xd") or self._Xd.shape != X_host.shape or self._Xd.dtype != X_host.dtype:
+            self._Xd = torch.empty(X_host.shape, dtype=X_host.dtype, device=self.device)
+            self._Wd = torch.empty(W_host.shape, dtype=W_host.dtype, device=self.device)
+        self._Xd.copy_(X_host, non_blocking=True)
+        self._Wd.copy_(W_host, non_blocking=True)
+        r = self.run(self._Xd, self._Wd, avg_bits, lloyd_iters)
+        src = {"bits": r.bits, "rows": r.rows, "cols": r.cols, "vals": r.vals, "lut": r.lut, "packed": r.packed,
+               "row_off": r.row_off, "perm": r.perm, "seg_rows": r.seg_rows, "counters": self.counters}
+        for k, t in host_out.items():
+            t.copy_(src[k], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return host_out
