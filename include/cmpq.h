@@ -79,6 +79,22 @@ cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, i
                                int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
                                void* stream);
 
+/* Same result as cmpq_collect_stats without any work space: the partial sums live in a fixed
+ * 2 MiB array inside the library (the paper has no counterpart; this exists for callers that
+ * cannot allocate device memory: code running inside another framework's memory plan, code that
+ * must avoid the device-wide synchronisation an allocation implies, plug-ins that only receive
+ * input and output buffers).  The array is held by every GPU that loads the library until the
+ * process exits.  d_in <= CMPQ_STATIC_MAX_D_IN, else CMPQ_ERR_UNSUPPORTED; other checks as above.
+ * The call allocates and frees nothing.  The first call on each device looks up the array's
+ * device address (make that call before any stream capture starts).  All calls on a device share
+ * the array: two calls whose kernels may overlap on the GPU (different streams, no ordering
+ * between them) race on it; calls on one stream are safe.  Nothing needs clearing between calls:
+ * each call overwrites every partial it later reads.  The number of partial sums may differ
+ * from cmpq_collect_stats, so results agree to rounding (about 1e-7 relative), not bit for bit. */
+#define CMPQ_STATIC_MAX_D_IN 32768
+cmpq_status cmpq_collect_stats_static(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                      int64_t ldx, double* sumsq, void* stream);
+
 /* a[j] = (float) sqrt(sumsq[j]). */
 cmpq_status cmpq_finalize_stats(const double* sumsq, int64_t d_in, float* a, void* stream);
 

@@ -17,7 +17,7 @@ OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_P
 LUT_STRIDE = 16
 
 EXPORTS = (
-    "cmpq_collect_stats", "cmpq_finalize_stats", "cmpq_allocate_bits", "cmpq_extract_outliers",
+    "cmpq_collect_stats", "cmpq_collect_stats_static", "cmpq_finalize_stats", "cmpq_allocate_bits", "cmpq_extract_outliers",
     "cmpq_quantize_layer", "cmpq_pack", "cmpq_workspace_bytes", "cmpq_alloc_counts",
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
 )
@@ -44,6 +44,7 @@ def lib():
         i64, vp, dbl, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_double, ctypes.c_size_t
         ci = ctypes.c_int
         L.cmpq_collect_stats.argtypes = [vp, ci, i64, i64, i64, vp, vp, sz, vp]
+        L.cmpq_collect_stats_static.argtypes = [vp, ci, i64, i64, i64, vp, vp]
         L.cmpq_finalize_stats.argtypes = [vp, i64, vp, vp]
         L.cmpq_allocate_bits.argtypes = [vp, i64, dbl, ci, vp, vp, vp, sz, vp]
         L.cmpq_extract_outliers.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp,
@@ -51,7 +52,7 @@ def lib():
         L.cmpq_quantize_layer.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp,
                                           vp, vp, sz, vp]
         L.cmpq_pack.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp]
-        for name in ("cmpq_collect_stats", "cmpq_finalize_stats", "cmpq_allocate_bits",
+        for name in ("cmpq_collect_stats", "cmpq_collect_stats_static", "cmpq_finalize_stats", "cmpq_allocate_bits",
                      "cmpq_extract_outliers", "cmpq_quantize_layer", "cmpq_pack"):
             getattr(L, name).restype = ci
         L.cmpq_workspace_bytes.argtypes = [ci, i64, i64]
@@ -121,6 +122,14 @@ def cmpq_collect_stats(X, sumsq, ws):
     n, d_in = X.shape
     _check(lib().cmpq_collect_stats(_ptr(X), dtype_code(X), n, d_in, X.stride(0) if n > 0 else d_in,
                                     _ptr(sumsq), _ptr(ws), ws.numel(), _stream()), "cmpq_collect_stats")
+
+
+def cmpq_collect_stats_static(X, sumsq):
+    """cmpq_collect_stats for callers that cannot provide a work space: the scratch is a fixed array
+    inside the library (d_in <= 32768).  Calls on different streams must not overlap."""
+    n, d_in = X.shape
+    _check(lib().cmpq_collect_stats_static(_ptr(X), dtype_code(X), n, d_in, X.stride(0) if n > 0 else d_in,
+                                           _ptr(sumsq), _stream()), "cmpq_collect_stats_static")
 
 
 def cmpq_finalize_stats(sumsq, a):
