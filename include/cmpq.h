@@ -72,7 +72,7 @@ typedef enum {
 /* ---- statistic (Section 3.2.1: per-channel L2 norm of the activation matrix X) --------------
  * sumsq[j] += sum_t X[t*ldx + j]^2 for the n_tokens rows given; call it once per chunk of
  * calibration tokens after zeroing sumsq (fp64, d_in entries).  Squares are formed in fp32
- * (exact for 16-bit inputs), partial sums in fp32 over at most 64 rows, the rest in fp64 in
+ * (exact for 16-bit inputs), partial sums in fp32 over at most 32 rows, the rest in fp64 in
  * a fixed order.  n_tokens may be 0.  X is [n_tokens][ldx] of `dt`, ldx >= d_in.
  * ws: cmpq_workspace_bytes(CMPQ_OP_COLLECT_STATS, d_in, 0). */
 cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,

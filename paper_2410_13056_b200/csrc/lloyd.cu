@@ -2,19 +2,27 @@
 // Section 3: each weight is replaced by its nearest centroid).
 //
 // One thread block fits one channel.  The channel is read from HBM once, widened to fp32 and
-// kept in shared memory for all iterations together with its current codes, so an iteration
-// moves no HBM bytes.  Nothing here is a dense contraction: the work is K subtract / compare
-// steps per weight per sweep on the fp32 pipes, so no tensor cores are used.
+// kept in REGISTERS (E weights per thread) for all iterations together with its codes, so an
+// iteration moves no HBM bytes and no shared-memory bytes either.  Nothing here is a dense
+// contraction: the work is K subtract / compare steps per weight per sweep on the fp32 pipes, so
+// no tensor cores are used.
 //
 //   start       K order statistics of the channel, found by a two-level counting select on the
 //               16-bit keys (256 buckets by high byte, then 256 by low byte inside the buckets
 //               that hold a target) -- no sort
-//   sweep       every thread assigns its weights to the first nearest centroid (centroids in
-//               registers, fp32 |x - c_k|, strict '<' scan)
-//   update      cluster sums are kept in fp64 and counts in int32.  The first sweep, and any
-//               sweep after one that moved more than 1/8 of the weights, rebuilds them from
-//               scratch (per-warp partials added in warp order); otherwise only the weights
-//               whose code changed are moved between clusters with shared-memory atomics.
+//   sweep       defined as: the first k minimising fabsf(x - c_k) (fp32, strict '<' scan).
+//               When the centroids are strictly increasing and every gap exceeds 2^-22 times the
+//               channel's value range, two values x - c_k and x - c_{k-1} can never round to the
+//               same float, and then that first minimum equals the number of k >= 1 with
+//               fabsf(x - c_k) < fabsf(x - c_{k-1}); the sweep counts those with one subtract, one
+//               compare and one predicated add per (weight, centroid).  Otherwise it runs the
+//               plain scan.  Codes of four weights are accumulated in one float (base 16), so
+//               an unchanged group costs one compare.
+//   update      cluster sums are kept in fp64 and counts in int32.  The first sweep rebuilds them
+//               from scratch (per-warp partials added in warp order); later sweeps list the
+//               weights whose code changed and move only those between clusters (
+//               per-warp partial changes, no atomics on the sums); a sweep that changes more than
+//               1/8 of the weights rebuilds instead.
 //               16-bit weights of bounded dynamic range make every such sum exact in fp64, so
 //               the order of the additions cannot change the result
 //   stop        a sweep that changes no code ends the loop early: later iterations would
@@ -27,13 +35,8 @@ constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
 
 struct alignas(16) LloydShared {
-    union {
-        int hist2[kMaxK][256];  // second-level counts, one row per distinct target bucket
-        struct {
-            double wsum[kMaxWarps][kMaxK];  // per-warp cluster sums of a rebuild
-            int wcnt[kMaxWarps][kMaxK];
-        } acc;
-    } u;
+    double wsum[kMaxWarps][kMaxK];  // per-warp cluster sums of a rebuild
+    int wcnt[kMaxWarps][kMaxK];
     int hist1[256];
     int excl1[257];
     double S[kMaxK];
@@ -43,10 +46,25 @@ struct alignas(16) LloydShared {
     int tgt_resid[kMaxK];
     int tgt_slot[kMaxK];
     unsigned char slot_of_bucket[256];
-    int changed;
-    int max_top;   // largest exponent of a non-zero weight
-    int min_ulp;   // exponent of the smallest unit in the last place among non-zero weights
+    int changed[2];     // weights whose code changed in the current sweep (by sweep parity)
+    int list_count[2];  // entries appended to the change list (may exceed its capacity)
+    int fast;         // centroids strictly increasing with safe gaps
+    float vmin, vmax; // value range of the channel
+    float wlo[kMaxWarps], whi[kMaxWarps];  // per-warp value range, largest exponent, smallest ulp
+    int wtop[kMaxWarps], wulp[kMaxWarps];
 };
+// dynamic shared memory after LloydShared: scratch region (lloyd_scratch_bytes), then float xs[N]
+
+// Bytes of the multi-purpose scratch region: second-level histogram (start), change list (N/8
+// entries), removed-column bitmap (load).
+__host__ __device__ inline int lloyd_scratch_bytes(int N) {
+    int hist2 = kMaxK * 256 * (int)sizeof(int);
+    int list = (N >> 3) * 4;
+    int bitmap = ((N + 31) / 32) * 4;
+    int m = hist2 > list ? hist2 : list;
+    m = m > bitmap ? m : bitmap;
+    return (m + 15) & ~15;
+}
 
 template <int DT>
 __device__ __forceinline__ uint32_t sort_key16(float x) {
@@ -62,18 +80,6 @@ __device__ __forceinline__ float value_of_key16(uint32_t key) {
     return widen16<DT>((uint16_t)h);
 }
 
-template <int K>
-__device__ __forceinline__ int nearest(float x, const float (&c)[K]) {
-    float best = fabsf(x - c[0]);
-    int bk = 0;
-#pragma unroll
-    for (int k = 1; k < K; ++k) {
-        float d = fabsf(x - c[k]);
-        if (d < best) { best = d; bk = k; }
-    }
-    return bk;
-}
-
 __device__ __forceinline__ int warp_sum(int v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -86,15 +92,30 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
+// Code of one weight by the defining scan: first k minimising |x - c_k|.
+template <int K>
+__device__ __forceinline__ int nearest_scan(float x, const float (&c)[K]) {
+    float best = fabsf(x - c[0]);
+    int bk = 0;
+#pragma unroll
+    for (int k = 1; k < K; ++k) {
+        float d = fabsf(x - c[k]);
+        if (d < best) { best = d; bk = k; }
+    }
+    return bk;
+}
+
 // The K starting centroids: the ((2k+1) N)/(2K)-th smallest values of the channel.
-template <int DT, int K>
-__device__ void select_start(const float* xs, int N, LloydShared& sh) {
+template <int DT, int K, int E>
+__device__ void select_start(const float (&x)[E], int nval, int N, LloydShared& sh, int* hist2) {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = nthr >> 5;
     for (int b = tid; b < 256; b += nthr) { sh.hist1[b] = 0; sh.slot_of_bucket[b] = 0xff; }
-    for (int b = tid; b < K * 256; b += nthr) (&sh.u.hist2[0][0])[b] = 0;
+    for (int b = tid; b < K * 256; b += nthr) hist2[b] = 0;
     __syncthreads();
-    for (int j = tid; j < N; j += nthr) atomicAdd(&sh.hist1[sort_key16<DT>(xs[j]) >> 8], 1);
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nval) atomicAdd(&sh.hist1[sort_key16<DT>(x[e]) >> 8], 1);
     __syncthreads();
     if (warp == 0) {  // exclusive prefix of the 256 bucket counts
         int v[8], s = 0;
@@ -132,14 +153,17 @@ __device__ void select_start(const float* xs, int N, LloydShared& sh) {
         }
     }
     __syncthreads();
-    for (int j = tid; j < N; j += nthr) {
-        uint32_t key = sort_key16<DT>(xs[j]);
-        int slot = sh.slot_of_bucket[key >> 8];
-        if (slot != 0xff) atomicAdd(&sh.u.hist2[slot][key & 0xff], 1);
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        if (e < nval) {
+            uint32_t key = sort_key16<DT>(x[e]);
+            int slot = sh.slot_of_bucket[key >> 8];
+            if (slot != 0xff) atomicAdd(&hist2[slot * 256 + (key & 0xff)], 1);
+        }
     }
     __syncthreads();
     for (int k = warp; k < K; k += nwarps) {  // one warp resolves one target inside its bucket
-        const int* h = sh.u.hist2[sh.tgt_slot[k]];
+        const int* h = hist2 + sh.tgt_slot[k] * 256;
         const int resid = sh.tgt_resid[k];
         int v[8], s = 0;
 #pragma unroll
@@ -160,183 +184,391 @@ __device__ void select_start(const float* xs, int N, LloydShared& sh) {
     __syncthreads();
 }
 
-// Rebuilds S and n from the codes in shared memory (per-warp partials, added in warp order).
+// Warp 0 decides whether the counting sweep is valid for the centroids now in sh.c.
 template <int K>
-__device__ void rebuild_sums(const float* xs, const unsigned char* code, int N, LloydShared& sh) {
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    const int nwarps = nthr >> 5;
+__device__ __forceinline__ void decide_fast(LloydShared& sh) {
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        float ck = sh.c[lane < K ? lane : K - 1];
+        float cp = __shfl_up_sync(0xffffffffu, ck, 1);
+        double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+        bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
+        ok = __all_sync(0xffffffffu, ok);
+        if (lane == 0) sh.fast = ok ? 1 : 0;
+    }
+}
+
+// Per-warp cluster sums and counts of all weights, from the codes in registers.
+template <int K, int E>
+__device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 7) / 8], int nval,
+                                 LloydShared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int code[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) code[e] = (e < nval) ? (int)((cw[e >> 3] >> (4 * (e & 7))) & 15u) : -1;
+#pragma unroll 1
     for (int k = 0; k < K; ++k) {
         double s = 0.0;
         int cnt = 0;
-        for (int j = tid; j < N; j += nthr) {
-            bool mine = code[j] == k;
-            s += mine ? (double)xs[j] : 0.0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            bool mine = code[e] == k;
+            s += mine ? (double)x[e] : 0.0;
             cnt += mine ? 1 : 0;
         }
         s = warp_sum(s);
         cnt = warp_sum(cnt);
-        if (lane == 0) { sh.u.acc.wsum[warp][k] = s; sh.u.acc.wcnt[warp][k] = cnt; }
+        if (lane == 0) { sh.wsum[warp][k] = s; sh.wcnt[warp][k] = cnt; }
     }
-    __syncthreads();
-    if (tid < K) {
-        double s = 0.0;
-        int cnt = 0;
-        for (int w = 0; w < nwarps; ++w) { s += sh.u.acc.wsum[w][tid]; cnt += sh.u.acc.wcnt[w][tid]; }
-        sh.S[tid] = s;
-        sh.n[tid] = cnt;
-    }
-    __syncthreads();
 }
 
-template <int DT, int K>
-__device__ void fit_channel(const LloydArgs& a, int64_t row, float* xs, unsigned char* code,
-                            LloydShared& sh) {
+// Per-warp changes of the cluster sums and counts caused by the listed weights.  Thread t looks
+// after cluster t mod K and every (nthr/K)-th list entry; lanes with the same cluster are combined
+// with shuffles, so no two threads ever add to the same address.
+template <int K>
+__device__ void list_partials(const uint32_t* list, int L, const float* xs, LloydShared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k = tid & (K - 1), seg = tid / K, nseg = blockDim.x / K;
+    double ds = 0.0;
+    int dn = 0;
+    for (int t = seg; t < L; t += nseg) {
+        const uint32_t en = list[t];  // column | old code << 16 | new code << 20
+        const int o = (en >> 16) & 15, nw = (en >> 20) & 15;
+        const double xv = (double)xs[en & 0xffffu];
+        if (nw == k) { ds += xv; ++dn; }
+        if (o == k) { ds -= xv; --dn; }
+    }
+#pragma unroll
+    for (int o = K; o < 32; o <<= 1) {
+        ds += __shfl_xor_sync(0xffffffffu, ds, o);
+        dn += __shfl_xor_sync(0xffffffffu, dn, o);
+    }
+    if (lane < K) { sh.wsum[warp][lane] = ds; sh.wcnt[warp][lane] = dn; }
+}
+
+// Warp 0: combine the per-warp partials into S and n (absolute after a rebuild, as a change after
+// a list pass), move every non-empty cluster's centroid to its mean and decide whether the counting
+// sweep is valid for the new centroids.
+template <int K>
+__device__ __forceinline__ void update_centroids(LloydShared& sh, bool absolute) {
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x, nwarps = blockDim.x >> 5;
+        float ck = 0.f;
+        if (lane < K) {
+            double s = 0.0;
+            int cnt = 0;
+            for (int w = 0; w < nwarps; ++w) { s += sh.wsum[w][lane]; cnt += sh.wcnt[w][lane]; }
+            if (!absolute) { s += sh.S[lane]; cnt += sh.n[lane]; }
+            sh.S[lane] = s;
+            sh.n[lane] = cnt;
+            ck = sh.c[lane];
+            if (cnt > 0) { ck = __double2float_rn(__ddiv_rn(s, (double)cnt)); sh.c[lane] = ck; }
+        }
+        ck = __shfl_sync(0xffffffffu, ck, lane < K ? lane : K - 1);
+        float cp = __shfl_up_sync(0xffffffffu, ck, 1);
+        double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+        bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
+        ok = __all_sync(0xffffffffu, ok);
+        if (lane == 0) sh.fast = ok ? 1 : 0;
+    }
+}
+
+template <int DT, int K, int E>
+__device__ void fit_channel(const LloydArgs& a, int64_t row, float (&x)[E], int nval, LloydShared& sh,
+                            unsigned char* dyn, const float* xs) {
+    constexpr int G = E / 4;          // float accumulators: codes of 4 weights each, base 16
+    constexpr int WORDS = (E + 7) / 8;  // packed codes: 8 weights per 32-bit word
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
     const int N = (int)a.d_out;
     const int T = a.iters;
+    uint32_t* list = reinterpret_cast<uint32_t*>(dyn);
+    const int list_cap = N >> 3;
 
-    select_start<DT, K>(xs, N, sh);
+    select_start<DT, K, E>(x, nval, N, sh, reinterpret_cast<int*>(dyn));
+    if (tid < 2) { sh.changed[tid] = 0; sh.list_count[tid] = 0; }
+    decide_fast<K>(sh);
+    __syncthreads();
 
+    uint32_t cw[WORDS];
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) cw[w] = 0;
     float c[K];
-    bool rebuild = true;  // the first sweep has no previous codes
     int sweeps_done = 0;
+    int prev_changed = N;
     for (int it = 0; it <= T; ++it) {
 #pragma unroll
         for (int k = 0; k < K; ++k) c[k] = sh.c[k];
-        if (tid == 0) sh.changed = 0;
-        __syncthreads();
-        const bool last = (it == T);
-        const bool first = (it == 0);
-        int changed = 0;
-        for (int j = tid; j < N; j += nthr) {
-            float x = xs[j];
-            int nk = nearest<K>(x, c);
-            int ok = first ? -1 : (int)code[j];
-            if (nk != ok) {
-                ++changed;
-                code[j] = (unsigned char)nk;
-                if (!rebuild && !last) {
-                    atomicAdd(&sh.S[nk], (double)x);
-                    atomicAdd(&sh.S[ok], -(double)x);
-                    atomicAdd(&sh.n[nk], 1);
-                    atomicAdd(&sh.n[ok], -1);
+        const bool fast = sh.fast != 0;
+        const bool last = (it == T), first = (it == 0);
+        const bool use_list = !first && !last && prev_changed <= list_cap;
+        const int par = it & 1;
+
+        uint32_t half[G];  // 16 bits: the codes of weights 4g..4g+3
+        if (fast) {
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                // 2^23 + sum code_u 16^u is exact in fp32, so the low mantissa bits are the codes
+                float acc = 8388608.f;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float xv = x[4 * g + u];
+                    const float inc = (float)(1 << (4 * u));
+                    float dp = fabsf(xv - c[0]);
+#pragma unroll
+                    for (int k = 1; k < K; ++k) {
+                        float d = fabsf(xv - c[k]);
+                        if (d < dp) acc += inc;
+                        dp = d;
+                    }
+                }
+                half[g] = __float_as_uint(acc);
+            }
+        } else {
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                uint32_t p = 0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) p |= (uint32_t)nearest_scan<K>(x[4 * g + u], c) << (4 * u);
+                half[g] = p;
+            }
+        }
+        uint32_t nw[WORDS];
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w)
+            nw[w] = (2 * w + 1 < G) ? __byte_perm(half[2 * w], half[2 * w + 1], 0x5410) : (half[2 * w] & 0xffffu);
+        ++sweeps_done;
+
+        // weights whose code changed (few once the fit settles)
+        uint32_t any = 0;
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) any |= nw[w] ^ cw[w];
+        int nch = 0;
+        if (first) {
+            nch = nval;
+        } else if (any) {
+            uint32_t m[WORDS];  // bit 4i set: weight i of the word changed
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) {
+                uint32_t xr = nw[w] ^ cw[w];
+                m[w] = (xr | (xr >> 1) | (xr >> 2) | (xr >> 3)) & 0x11111111u;
+                nch += __popc(m[w]);
+            }
+            if (use_list) {
+                int pos = atomicAdd(&sh.list_count[par], nch);
+#pragma unroll
+                for (int w = 0; w < WORDS; ++w) {
+                    uint32_t mm = m[w];
+                    while (mm) {
+                        const int b = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        const int e = 8 * w + (b >> 2);
+                        const uint32_t j = (uint32_t)(((e >> 2) * nthr + tid) * 4 + (e & 3));
+                        if (pos < list_cap)
+                            list[pos] = j | (((cw[w] >> b) & 15u) << 16) | (((nw[w] >> b) & 15u) << 20);
+                        ++pos;
+                    }
                 }
             }
         }
-        ++sweeps_done;
-        changed = warp_sum(changed);
-        if (lane == 0 && changed) atomicAdd(&sh.changed, changed);
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) cw[w] = nw[w];
+        nch = warp_sum(nch);
+        if (lane == 0 && nch) atomicAdd(&sh.changed[par], nch);
         __syncthreads();
-        const int total_changed = sh.changed;
+        const int total_changed = sh.changed[par];
+        const int L = sh.list_count[par];
+        if (tid == 0) { sh.changed[par ^ 1] = 0; sh.list_count[par ^ 1] = 0; }
+        prev_changed = total_changed;
         if (last || total_changed == 0) break;  // uniform: every thread reads the same value
-        if (rebuild) rebuild_sums<K>(xs, code, N, sh);
-        if (tid < K && sh.n[tid] > 0)
-            sh.c[tid] = __double2float_rn(__ddiv_rn(sh.S[tid], (double)sh.n[tid]));
-        rebuild = total_changed > (N >> 3);
+        const bool by_list = use_list && L <= list_cap;
+        if (by_list) list_partials<K>(list, L, xs, sh);
+        else rebuild_partials<K, E>(x, cw, nval, sh);
+        __syncthreads();
+        update_centroids<K>(sh, !by_list);
         __syncthreads();
     }
 
-    // outputs
-#pragma unroll
-    for (int k = 0; k < K; ++k) c[k] = sh.c[k];
+    // outputs: thread owns weights j = (g * nthr + tid) * 4 + u
     if (a.lut && tid < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + tid] = tid < K ? sh.c[tid] : 0.f;
-    if (a.codes) {
-        uint8_t* out = a.codes + row * a.d_out;
-        if ((a.d_out & 3) == 0) {
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(code);
-            uint32_t* dst = reinterpret_cast<uint32_t*>(out);
-            for (int j = tid; j < (N >> 2); j += nthr) dst[j] = src[j];
-        } else {
-            for (int j = tid; j < N; j += nthr) out[j] = code[j];
+    const bool vec4 = (a.d_out & 3) == 0;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const int j0 = (g * nthr + tid) * 4;
+        if (j0 >= N) continue;
+        const uint32_t p = (cw[g >> 1] >> (16 * (g & 1))) & 0xffffu;
+        if (a.codes) {
+            uint8_t* out = a.codes + row * a.d_out + j0;
+            if (vec4) {
+                uint32_t w = (p & 15u) | (((p >> 4) & 15u) << 8) | (((p >> 8) & 15u) << 16) | (((p >> 12) & 15u) << 24);
+                *reinterpret_cast<uint32_t*>(out) = w;
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (j0 + u < N) out[u] = (uint8_t)((p >> (4 * u)) & 15u);
+            }
         }
-    }
-    if (a.err) {
-        float* out = a.err + row * a.d_out;
-        for (int j = tid; j < N; j += nthr) out[j] = fabsf(xs[j] - sh.c[code[j]]);
+        if (a.err) {
+            float* out = a.err + row * a.d_out + j0;
+            float ev[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) ev[u] = fabsf(x[4 * g + u] - sh.c[(p >> (4 * u)) & 15u]);
+            if (vec4) {
+                *reinterpret_cast<float4*>(out) = make_float4(ev[0], ev[1], ev[2], ev[3]);
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (j0 + u < N) out[u] = ev[u];
+            }
+        }
     }
     if (a.sweeps && tid == 0)
         atomicAdd(a.sweeps, (unsigned long long)sweeps_done * (unsigned long long)N * (unsigned long long)K);
 }
 
-template <int DT>
-__global__ void __launch_bounds__(1024)
+template <int DT, int E, int MAXT>
+__global__ void __launch_bounds__(MAXT)
 lloyd_kernel(const LloydArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int64_t row = blockIdx.x;
     if (a.skip_row && a.skip_row[row]) return;
     const int N = (int)a.d_out;
-    const int npad = (N + 15) & ~15;
     LloydShared& sh = *reinterpret_cast<LloydShared*>(smem_raw);
-    float* xs = reinterpret_cast<float*>(smem_raw + sizeof(LloydShared));
-    unsigned char* code = reinterpret_cast<unsigned char*>(xs + npad);
+    unsigned char* dyn = smem_raw + sizeof(LloydShared);          // hist2 / change list / bitmap
+    float* xs = reinterpret_cast<float*>(dyn + lloyd_scratch_bytes(N));  // fp32 copy of the channel
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
 
-    if (tid == 0) { sh.max_top = -100000; sh.min_ulp = 100000; }
-    const uint16_t* w = a.W + row * a.ldw;
-    for (int j = tid; j < N; j += nthr) {
-        float x = widen16<DT>(w[j]);
-        xs[j] = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
+    // removed positions (outliers of this row) are marked in a bitmap over the columns
+    uint32_t* removed = reinterpret_cast<uint32_t*>(dyn);
+    int64_t p0 = 0, p1 = 0;
+    if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
+    const bool has_removed = p1 > p0;
+    if (has_removed) {
+        for (int w = tid; w < (N + 31) / 32; w += nthr) removed[w] = 0;
+        __syncthreads();
+        for (int64_t p = p0 + tid; p < p1; p += nthr) {
+            int col = a.cols[p];
+            atomicOr(&removed[col >> 5], 1u << (col & 31));
+        }
     }
     __syncthreads();
-    if (a.row_ptr) {
-        const int64_t p0 = a.row_ptr[row], p1 = a.row_ptr[row + 1];
-        for (int64_t p = p0 + tid; p < p1; p += nthr) xs[a.cols[p]] = 0.f;
-        __syncthreads();
+
+    // thread owns weights j = (g * nthr + tid) * 4 + u, u = 0..3; valid ones form a prefix
+    const uint16_t* w = a.W + row * a.ldw;
+    const bool vec = ((a.ldw & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 7) == 0);
+    float x[E];
+    int nval = 0;
+#pragma unroll
+    for (int g = 0; g < E / 4; ++g) {
+        const int j0 = (g * nthr + tid) * 4;
+        uint16_t h[4] = {0, 0, 0, 0};
+        if (j0 + 3 < N && vec) {
+            uint2 v = *reinterpret_cast<const uint2*>(w + j0);
+            h[0] = (uint16_t)(v.x & 0xffff); h[1] = (uint16_t)(v.x >> 16);
+            h[2] = (uint16_t)(v.y & 0xffff); h[3] = (uint16_t)(v.y >> 16);
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (j0 + u < N) h[u] = w[j0 + u];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            float v = widen16<DT>(h[u]);
+            const int j = j0 + u;
+            if (j < N) {
+                ++nval;
+                if (has_removed && ((removed[j >> 5] >> (j & 31)) & 1)) v = 0.f;
+                v = (v == 0.f) ? 0.f : v;  // -0 and +0 are the same point
+                xs[j] = v;
+            } else {
+                v = __int_as_float(0x7f800000);  // padding: +inf always gets code 0 and never changes
+            }
+            x[4 * g + u] = v;
+        }
     }
-    if (a.inexact_rows) {
+    // value range (for the gap test) and exactness diagnostics
+    {
+        float lo = __int_as_float(0x7f800000), hi = __int_as_float(0xff800000);
         int top = -100000, ulp = 100000;
-        for (int j = tid; j < N; j += nthr) {
-            uint32_t u = __float_as_uint(xs[j]) & 0x7fffffffu;
-            if (u) {
-                int e = (int)(u >> 23);
-                uint32_t m = u & 0x7fffffu;
-                int t, q;
-                if (e) { t = e - 127; q = e - 150 + (__ffs(m | 0x800000u) - 1); }
-                else   { t = (31 - __clz(m)) - 149; q = (__ffs(m) - 1) - 149; }
-                top = max(top, t);
-                ulp = min(ulp, q);
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (e < nval) {
+                lo = fminf(lo, x[e]);
+                hi = fmaxf(hi, x[e]);
+                uint32_t u = __float_as_uint(x[e]) & 0x7fffffffu;
+                if (u) {
+                    int ex = (int)(u >> 23);
+                    uint32_t m = u & 0x7fffffu;
+                    int t, q;
+                    if (ex) { t = ex - 127; q = ex - 150 + (__ffs(m | 0x800000u) - 1); }
+                    else    { t = (31 - __clz(m)) - 149; q = (__ffs(m) - 1) - 149; }
+                    top = max(top, t);
+                    ulp = min(ulp, q);
+                }
             }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
             top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
             ulp = min(ulp, __shfl_xor_sync(0xffffffffu, ulp, o));
         }
-        if (lane == 0) { atomicMax(&sh.max_top, top); atomicMin(&sh.min_ulp, ulp); }
-        __syncthreads();
-        if (tid == 0 && sh.max_top > -100000) {
-            // sums and differences of up to 2N weights stay exact in fp64 while
-            // 2 N 2^(top+1) / 2^ulp <= 2^53
-            int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
-            if (log2n + 1 + (sh.max_top + 1 - sh.min_ulp) > 53) atomicAdd(a.inexact_rows, 1);
+        const int warp = tid >> 5, nwarps = nthr >> 5;
+        if (lane == 0) { sh.wlo[warp] = lo; sh.whi[warp] = hi; sh.wtop[warp] = top; sh.wulp[warp] = ulp; }
+        __syncthreads();  // also: every thread is done with the removed-column bitmap
+        if (tid == 0) {
+            for (int wv = 1; wv < nwarps; ++wv) {
+                lo = fminf(lo, sh.wlo[wv]);
+                hi = fmaxf(hi, sh.whi[wv]);
+                top = max(top, sh.wtop[wv]);
+                ulp = min(ulp, sh.wulp[wv]);
+            }
+            sh.vmin = lo;
+            sh.vmax = hi;
+            if (a.inexact_rows && top > -100000) {
+                // sums and differences of up to 2N weights stay exact in fp64 while
+                // 2 N 2^(top+1) / 2^ulp <= 2^53
+                int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
+                if (log2n + 1 + (top + 1 - ulp) > 53) atomicAdd(a.inexact_rows, 1);
+            }
         }
+        __syncthreads();
     }
     const int bits = a.bits[row];
-    if (bits == 2) fit_channel<DT, 4>(a, row, xs, code, sh);
-    else if (bits == 3) fit_channel<DT, 8>(a, row, xs, code, sh);
-    else fit_channel<DT, 16>(a, row, xs, code, sh);
+    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, dyn, xs);
+    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, dyn, xs);
+    else fit_channel<DT, 16, E>(a, row, x, nval, sh, dyn, xs);
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out) {
-    size_t npad = ((size_t)d_out + 15) & ~(size_t)15;
-    return sizeof(LloydShared) + npad * 5;
+    return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * sizeof(float);
 }
 
-static int lloyd_threads(int64_t d_out) {
-    int64_t t = (d_out + 15) / 16;
-    t = (t + 31) / 32 * 32;
-    if (t < 64) t = 64;
-    if (t > 1024) t = 1024;
-    return (int)t;
+template <int DT, int E, int MAXT>
+static cmpq_status launch_variant(const LloydArgs& args, int threads, cudaStream_t st) {
+    const size_t smem = lloyd_smem_bytes(args.d_out);
+    auto kern = lloyd_kernel<DT, E, MAXT>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return CMPQ_ERR_CUDA;
+    kern<<<(unsigned)args.d_in, threads, smem, st>>>(args);
+    return launch_status();
+}
+
+template <int DT>
+static cmpq_status launch_dt(const LloydArgs& args, cudaStream_t st) {
+    const int64_t N = args.d_out;
+    auto threads_for = [N](int e) {
+        int64_t t = (N + e - 1) / e;
+        t = (t + 31) / 32 * 32;
+        return (int)(t < 32 ? 32 : t);
+    };
+    if (N <= 2048) return launch_variant<DT, 4, 512>(args, threads_for(4), st);
+    if (N <= 16384) return launch_variant<DT, 16, 1024>(args, threads_for(16), st);
+    return launch_variant<DT, 32, 1024>(args, threads_for(32), st);
 }
 
 cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st) {
-    const size_t smem = lloyd_smem_bytes(args.d_out);
-    auto kern = dt == CMPQ_F16 ? lloyd_kernel<CMPQ_F16> : lloyd_kernel<CMPQ_BF16>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return CMPQ_ERR_CUDA;
-    kern<<<(unsigned)args.d_in, lloyd_threads(args.d_out), smem, st>>>(args);
-    return launch_status();
+    return dt == CMPQ_F16 ? launch_dt<CMPQ_F16>(args, st) : launch_dt<CMPQ_BF16>(args, st);
 }
 
 // row_ptr[r] = first position p with rows[p] >= r; every thread owns one position and fills the

@@ -1,0 +1,85 @@
+"""Small, self-ending runs of single C-ABI calls, meant to be captured by a profiler.
+
+    python -m paper_2410_13056_b200.profile_cases lloyd --d-in 1184 --d-out 4096 --bits 3 --launches 3
+    python -m paper_2410_13056_b200.profile_cases stats --tokens 32768 --d-in 4096 --launches 3
+    python -m paper_2410_13056_b200.profile_cases pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
+    python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
+
+Each case prints the mean CUDA-event time per call; every run holds well under 1 GB on the device.
+"""
+import argparse
+
+import torch
+
+from . import binding as B
+from . import inputs
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers"])
+    ap.add_argument("--d-in", type=int, default=1184)
+    ap.add_argument("--d-out", type=int, default=4096)
+    ap.add_argument("--tokens", type=int, default=32768)
+    ap.add_argument("--bits", type=int, default=3)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16"])
+    a = ap.parse_args()
+    dt = inputs.BF16 if a.dtype == "bf16" else inputs.F16
+    torch.cuda.set_device(0)
+    d_in, d_out = a.d_in, a.d_out
+    bits = torch.full((d_in,), a.bits, dtype=torch.uint8, device="cuda")
+
+    if a.case == "stats":
+        X = inputs.make_activations(a.tokens, d_in, dt, 1, device="cuda")
+        sumsq = torch.zeros(d_in, dtype=torch.float64, device="cuda")
+        ws = B.workspace(B.OP_COLLECT_STATS, d_in)
+        fn = lambda: B.cmpq_collect_stats(X, sumsq, ws)
+        work = "%.1f MB read" % (X.numel() * 2 / 1e6)
+    elif a.case == "pack":
+        codes = torch.randint(0, 1 << a.bits, (d_in, d_out), dtype=torch.uint8, device="cuda")
+        words = d_in * ((d_out * a.bits + 31) // 32)
+        packed = torch.empty(words, dtype=torch.int32, device="cuda")
+        row_off = torch.empty(d_in + 1, dtype=torch.int64, device="cuda")
+        perm = torch.empty(d_in, dtype=torch.int32, device="cuda")
+        seg = torch.empty(3, dtype=torch.int64, device="cuda")
+        ws = B.workspace(B.OP_PACK, d_in, d_out)
+        fn = lambda: B.cmpq_pack(codes, bits, packed, row_off, perm, seg, ws)
+        work = "%.1f MB read + %.1f MB written" % (codes.numel() / 1e6, words * 4 / 1e6)
+    else:
+        W = inputs.make_weight(d_in, d_out, dt, 1, device="cuda")
+        if a.case == "lloyd":
+            lut = torch.empty((d_in, 16), dtype=torch.float32, device="cuda")
+            codes = torch.empty((d_in, d_out), dtype=torch.uint8, device="cuda")
+            counters = torch.zeros(2, dtype=torch.int64, device="cuda")
+            ws = B.workspace(B.OP_QUANTIZE_LAYER, d_in, d_out)
+            fn = lambda: B.cmpq_quantize_layer(W, bits, None, None, a.iters, lut, codes, ws,
+                                               sweeps=counters[1:2])
+            work = "%d channels x %d weights, K=%d, T=%d" % (d_in, d_out, 1 << a.bits, a.iters)
+        else:
+            n_act, n_q = B.cmpq_default_counts(d_in, d_out)
+            nnz = n_act * d_out + n_q
+            rows = torch.empty(nnz, dtype=torch.int32, device="cuda")
+            cols = torch.empty(nnz, dtype=torch.int32, device="cuda")
+            vals = torch.empty(nnz, dtype=torch.int16, device="cuda")
+            av = torch.rand(d_in, device="cuda")
+            ws = B.workspace(B.OP_EXTRACT_OUTLIERS, d_in, d_out)
+            fn = lambda: B.cmpq_extract_outliers(W, av, bits, n_act, n_q, a.iters, rows, cols, vals, ws)
+            work = "%d channels x %d weights, K=%d, T=%d, nnz=%d" % (d_in, d_out, 1 << a.bits, a.iters, nnz)
+
+    fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.launches):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    print("%s: %s; %.4f ms per call over %d calls" % (a.case, work, e0.elapsed_time(e1) / a.launches, a.launches))
+    if a.case == "lloyd":
+        print("distance evaluations per call: %d" % (int(counters[1].item()) // (a.launches + 1)))
+
+
+if __name__ == "__main__":
+    main()
