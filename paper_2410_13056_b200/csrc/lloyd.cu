@@ -1,69 +1,65 @@
 // Channel-wise K-means of CMPQ (Section 3.2.1: K-means per channel W_{i,:} with K = 2^bits;
 // Section 3: each weight is replaced by its nearest centroid).
 //
-// One thread block fits one channel.  The channel is read from HBM once, widened to fp32 and
-// kept in REGISTERS (E weights per thread) for all iterations together with its codes, so an
-// iteration moves no HBM bytes and no shared-memory bytes either.  Nothing here is a dense
-// contraction: the work is K subtract / compare steps per weight per sweep on the fp32 pipes, so
-// no tensor cores are used.
+// One thread block fits one channel.  Nothing here is a dense contraction: the work is K
+// subtract / compare steps per weight per sweep on the fp32 pipes, so no tensor cores are used.
 //
-//   start       K order statistics of the channel, found by a two-level counting select on the
-//               16-bit keys (256 buckets by high byte, then 256 by low byte inside the buckets
-//               that hold a target) -- no sort
-//   sweep       defined as: the first k minimising fabsf(x - c_k) (fp32, strict '<' scan).
-//               When the centroids are strictly increasing and every gap exceeds 2^-22 times the
-//               channel's value range, two values x - c_k and x - c_{k-1} can never round to the
-//               same float, and then that first minimum equals the number of k >= 1 with
-//               fabsf(x - c_k) < fabsf(x - c_{k-1}); the sweep counts those with one subtract, one
-//               compare and one predicated add per (weight, centroid).  Otherwise it runs the
-//               plain scan.  Codes of four weights are accumulated in one float (base 16), so
-//               an unchanged group costs one compare.
-//   update      cluster sums are kept in fp64 and counts in int32.  The first sweep rebuilds them
-//               from scratch (per-warp partials added in warp order); later sweeps list the
-//               weights whose code changed and move only those between clusters (
-//               per-warp partial changes, no atomics on the sums); a sweep that changes more than
-//               1/8 of the weights rebuilds instead.
-//               16-bit weights of bounded dynamic range make every such sum exact in fp64, so
-//               the order of the additions cannot change the result
-//   stop        a sweep that changes no code ends the loop early: later iterations would
-//               repeat it exactly
+//   load        the channel is read from HBM once, removed positions are zeroed, and the weights
+//               are SORTED by value inside the block with a two-level counting sort on their
+//               16-bit keys (high byte, then low byte inside each high-byte bucket).  Thread t
+//               then keeps the E consecutive order statistics [E t, E t + E) in REGISTERS for all
+//               iterations, so an iteration moves no HBM bytes.
+//   start       the K order statistics xs[((2k+1) N)/(2K)] are read straight from the sorted array
+//   sweep       defined as: the first k minimising fabsf(x - c_k) (fp32, strict '<' scan), for
+//               every weight and every centroid.  When the centroids are strictly increasing and
+//               every gap exceeds 2^-22 times the channel's value range, x - c_k and x - c_{k-1}
+//               can never round to the same float, and then that first minimum equals the number
+//               of k >= 1 with fabsf(x - c_k) < fabsf(x - c_{k-1}); the sweep counts those with one
+//               subtract, one compare and one predicated add per (weight, centroid) and the codes
+//               are non-decreasing along the sorted order.  Otherwise it runs the plain scan.
+//   update      with non-decreasing codes a cluster is a run [B_k, B_{k+1}) of the sorted order:
+//               its count is B_{k+1} - B_k and its sum a difference of fp64 prefix sums (per-thread
+//               totals scanned once at load, plus at most E-1 weights of the thread that holds the
+//               boundary).  The boundaries come from K-1 warp votes.  16-bit weights of bounded
+//               dynamic range make these fp64 sums exact, so they equal the sums taken in any
+//               other order.  Without the ordering guarantee the sums are rebuilt by plain
+//               per-cluster accumulation.
+//   stop        a sweep that moves no boundary (changes no code) ends the loop early: later
+//               iterations would repeat it exactly
+//   output      codes / errors are put back into column order through shared memory and stored
+//               with coalesced writes
 #include "lloyd.cuh"
 
 namespace cmpq {
 
 constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
+constexpr int kMaxThreads = 1024;
 
 struct alignas(16) LloydShared {
-    double wsum[kMaxWarps][kMaxK];  // per-warp cluster sums of a rebuild
-    int wcnt[kMaxWarps][kMaxK];
+    double pt[kMaxThreads + 1];     // exclusive prefix over threads of the threads' fp64 totals
+    double wsum[kMaxWarps][kMaxK];  // per-warp cluster sums (rebuild path), per-warp totals (scan)
+    int wcnt[kMaxWarps][kMaxK];     // per-warp cluster counts (rebuild) / threads below boundary k
     int hist1[256];
     int excl1[257];
-    double S[kMaxK];
-    int n[kMaxK];
+    int bucket_rank[256];           // rank of a high-byte bucket among the non-empty ones, or -1
     float c[kMaxK];
-    int tgt_bucket[kMaxK];
-    int tgt_resid[kMaxK];
-    int tgt_slot[kMaxK];
-    unsigned char slot_of_bucket[256];
-    int changed[2];     // weights whose code changed in the current sweep (by sweep parity)
-    int list_count[2];  // entries appended to the change list (may exceed its capacity)
-    int fast;         // centroids strictly increasing with safe gaps
-    float vmin, vmax; // value range of the channel
-    float wlo[kMaxWarps], whi[kMaxWarps];  // per-warp value range, largest exponent, smallest ulp
+    int bound[kMaxK + 1];           // B_k of the last ordered sweep
+    int bound_valid;
+    int n_nonempty;
+    int fast;                       // centroids strictly increasing with safe gaps
+    int stop;
+    float vmin, vmax;               // value range of the channel
+    float wlo[kMaxWarps], whi[kMaxWarps];
     int wtop[kMaxWarps], wulp[kMaxWarps];
 };
-// dynamic shared memory after LloydShared: scratch region (lloyd_scratch_bytes), then float xs[N]
+// dynamic shared memory after LloydShared:
+//   scratch (lloyd_scratch_bytes): removed-column bitmap during the load, second-level histogram
+//                                  during the sort, then the threads' packed codes
+//   sorted  (4 bytes per weight):  key << 16 | column, ascending; reused for the output staging
 
-// Bytes of the multi-purpose scratch region: second-level histogram (start), change list (N/8
-// entries), removed-column bitmap (load).
-__host__ __device__ inline int lloyd_scratch_bytes(int N) {
-    int hist2 = kMaxK * 256 * (int)sizeof(int);
-    int list = (N >> 3) * 4;
-    int bitmap = ((N + 31) / 32) * 4;
-    int m = hist2 > list ? hist2 : list;
-    m = m > bitmap ? m : bitmap;
-    return (m + 15) & ~15;
+__host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
+    return kMaxK * 256 * (int)sizeof(int);  // 16 KiB >= 16 bytes x 1024 threads >= 32768 bits
 }
 
 template <int DT>
@@ -92,6 +88,25 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
+// exclusive prefix of 256 counters by one warp (8 per lane, in place allowed); returns the total
+__device__ __forceinline__ int warp_scan256(const int* in, int* out_excl) {
+    const int lane = threadIdx.x & 31;
+    int v[8], s = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { v[t] = in[lane * 8 + t]; s += v[t]; }
+    int incl = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    int run = incl - s;
+    __syncwarp();
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { out_excl[lane * 8 + t] = run; run += v[t]; }
+    return __shfl_sync(0xffffffffu, incl, 31);
+}
+
 // Code of one weight by the defining scan: first k minimising |x - c_k|.
 template <int K>
 __device__ __forceinline__ int nearest_scan(float x, const float (&c)[K]) {
@@ -105,22 +120,26 @@ __device__ __forceinline__ int nearest_scan(float x, const float (&c)[K]) {
     return bk;
 }
 
-// The K starting centroids: the ((2k+1) N)/(2K)-th smallest values of the channel.
-template <int DT, int K, int E>
-__device__ void select_start(const float (&x)[E], int nval, int N, LloydShared& sh, int* hist2) {
+// Sorts the block's weights by 16-bit key into `sorted` (key << 16 | column).  key[e] belongs to
+// column ((e >> 2) * nthr + tid) * 4 + (e & 3); the first nval of a thread's keys are real.
+template <int E>
+__device__ void sort_channel(const uint32_t (&key)[E], int nval, LloydShared& sh, int* hist2,
+                             uint32_t* sorted) {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = nthr >> 5;
-    for (int b = tid; b < 256; b += nthr) { sh.hist1[b] = 0; sh.slot_of_bucket[b] = 0xff; }
-    for (int b = tid; b < K * 256; b += nthr) hist2[b] = 0;
+    for (int b = tid; b < 256; b += nthr) sh.hist1[b] = 0;
     __syncthreads();
 #pragma unroll
     for (int e = 0; e < E; ++e)
-        if (e < nval) atomicAdd(&sh.hist1[sort_key16<DT>(x[e]) >> 8], 1);
+        if (e < nval) atomicAdd(&sh.hist1[key[e] >> 8], 1);
     __syncthreads();
-    if (warp == 0) {  // exclusive prefix of the 256 bucket counts
-        int v[8], s = 0;
+    if (warp == 0) {
+        int total = warp_scan256(sh.hist1, sh.excl1);
+        if (lane == 0) sh.excl1[256] = total;
+        // rank of every non-empty bucket among the non-empty ones
+        int flag[8], s = 0;
 #pragma unroll
-        for (int t = 0; t < 8; ++t) { v[t] = sh.hist1[lane * 8 + t]; s += v[t]; }
+        for (int t = 0; t < 8; ++t) { flag[t] = sh.hist1[lane * 8 + t] > 0; s += flag[t]; }
         int incl = s;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -129,76 +148,52 @@ __device__ void select_start(const float (&x)[E], int nval, int N, LloydShared& 
         }
         int run = incl - s;
 #pragma unroll
-        for (int t = 0; t < 8; ++t) { sh.excl1[lane * 8 + t] = run; run += v[t]; }
-        if (lane == 31) sh.excl1[256] = run;
+        for (int t = 0; t < 8; ++t) { sh.bucket_rank[lane * 8 + t] = flag[t] ? run : -1; run += flag[t]; }
+        if (lane == 31) sh.n_nonempty = incl;
     }
     __syncthreads();
-    if (tid < K) {
-        int pos = (int)(((long long)(2 * tid + 1) * N) / (2 * K));
-        int lo = 0, hi = 256;  // last bucket b with excl1[b] <= pos
-        while (hi - lo > 1) {
-            int mid = (lo + hi) >> 1;
-            if (sh.excl1[mid] <= pos) lo = mid; else hi = mid;
-        }
-        sh.tgt_bucket[tid] = lo;
-        sh.tgt_resid[tid] = pos - sh.excl1[lo];
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int slots = 0;
-        for (int k = 0; k < K; ++k) {
-            int b = sh.tgt_bucket[k];
-            if (k == 0 || b != sh.tgt_bucket[k - 1]) sh.slot_of_bucket[b] = (unsigned char)slots++;
-            sh.tgt_slot[k] = sh.slot_of_bucket[b];
-        }
-    }
-    __syncthreads();
+    const int ngroups = (sh.n_nonempty + kMaxK - 1) / kMaxK;  // 16 buckets are refined at a time
+    for (int grp = 0; grp < ngroups; ++grp) {
+        for (int b = tid; b < kMaxK * 256; b += nthr) hist2[b] = 0;
+        __syncthreads();
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        if (e < nval) {
-            uint32_t key = sort_key16<DT>(x[e]);
-            int slot = sh.slot_of_bucket[key >> 8];
-            if (slot != 0xff) atomicAdd(&hist2[slot * 256 + (key & 0xff)], 1);
+        for (int e = 0; e < E; ++e) {
+            if (e < nval) {
+                int r = sh.bucket_rank[key[e] >> 8];
+                if ((r >> 4) == grp) atomicAdd(&hist2[(r & 15) * 256 + (key[e] & 0xff)], 1);
+            }
         }
-    }
-    __syncthreads();
-    for (int k = warp; k < K; k += nwarps) {  // one warp resolves one target inside its bucket
-        const int* h = hist2 + sh.tgt_slot[k] * 256;
-        const int resid = sh.tgt_resid[k];
-        int v[8], s = 0;
+        __syncthreads();
+        for (int s = warp; s < kMaxK; s += nwarps) warp_scan256(hist2 + s * 256, hist2 + s * 256);
+        __syncthreads();
 #pragma unroll
-        for (int t = 0; t < 8; ++t) { v[t] = h[lane * 8 + t]; s += v[t]; }
-        int incl = s;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
+        for (int e = 0; e < E; ++e) {
+            if (e < nval) {
+                int r = sh.bucket_rank[key[e] >> 8];
+                if ((r >> 4) == grp) {
+                    int pos = sh.excl1[key[e] >> 8] + atomicAdd(&hist2[(r & 15) * 256 + (key[e] & 0xff)], 1);
+                    uint32_t col = (uint32_t)(((e >> 2) * nthr + tid) * 4 + (e & 3));
+                    sorted[pos] = (key[e] << 16) | col;
+                }
+            }
         }
-        int run = incl - s;
-        if (resid >= run && resid < incl) {
-            int t = 0;
-            while (resid >= run + v[t]) { run += v[t]; ++t; }
-            sh.c[k] = value_of_key16<DT>((uint32_t)(sh.tgt_bucket[k] << 8) | (uint32_t)(lane * 8 + t));
-        }
+        __syncthreads();
     }
-    __syncthreads();
 }
 
-// Warp 0 decides whether the counting sweep is valid for the centroids now in sh.c.
+// Warp 0 decides whether the counting sweep is valid for the new centroids (lane k holds c_k).
 template <int K>
-__device__ __forceinline__ void decide_fast(LloydShared& sh) {
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        float ck = sh.c[lane < K ? lane : K - 1];
-        float cp = __shfl_up_sync(0xffffffffu, ck, 1);
-        double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
-        bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
-        ok = __all_sync(0xffffffffu, ok);
-        if (lane == 0) sh.fast = ok ? 1 : 0;
-    }
+__device__ __forceinline__ void decide_fast_warp0(LloydShared& sh, float ck_lane) {
+    const int lane = threadIdx.x;
+    float ck = __shfl_sync(0xffffffffu, ck_lane, lane < K ? lane : K - 1);
+    float cp = __shfl_up_sync(0xffffffffu, ck, 1);
+    double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+    bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
+    ok = __all_sync(0xffffffffu, ok);
+    if (lane == 0) sh.fast = ok ? 1 : 0;
 }
 
-// Per-warp cluster sums and counts of all weights, from the codes in registers.
+// Per-warp cluster sums and counts of all weights, from the codes in registers (any order).
 template <int K, int E>
 __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 7) / 8], int nval,
                                  LloydShared& sh) {
@@ -222,35 +217,10 @@ __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 
     }
 }
 
-// Per-warp changes of the cluster sums and counts caused by the listed weights.  Thread t looks
-// after cluster t mod K and every (nthr/K)-th list entry; lanes with the same cluster are combined
-// with shuffles, so no two threads ever add to the same address.
+// Warp 0, rebuild path: combine the per-warp partials, move every non-empty cluster's centroid to
+// its mean, decide the next sweep's mode.
 template <int K>
-__device__ void list_partials(const uint32_t* list, int L, const float* xs, LloydShared& sh) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int k = tid & (K - 1), seg = tid / K, nseg = blockDim.x / K;
-    double ds = 0.0;
-    int dn = 0;
-    for (int t = seg; t < L; t += nseg) {
-        const uint32_t en = list[t];  // column | old code << 16 | new code << 20
-        const int o = (en >> 16) & 15, nw = (en >> 20) & 15;
-        const double xv = (double)xs[en & 0xffffu];
-        if (nw == k) { ds += xv; ++dn; }
-        if (o == k) { ds -= xv; --dn; }
-    }
-#pragma unroll
-    for (int o = K; o < 32; o <<= 1) {
-        ds += __shfl_xor_sync(0xffffffffu, ds, o);
-        dn += __shfl_xor_sync(0xffffffffu, dn, o);
-    }
-    if (lane < K) { sh.wsum[warp][lane] = ds; sh.wcnt[warp][lane] = dn; }
-}
-
-// Warp 0: combine the per-warp partials into S and n (absolute after a rebuild, as a change after
-// a list pass), move every non-empty cluster's centroid to its mean and decide whether the counting
-// sweep is valid for the new centroids.
-template <int K>
-__device__ __forceinline__ void update_centroids(LloydShared& sh, bool absolute) {
+__device__ __forceinline__ void update_from_partials(LloydShared& sh) {
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x, nwarps = blockDim.x >> 5;
         float ck = 0.f;
@@ -258,50 +228,100 @@ __device__ __forceinline__ void update_centroids(LloydShared& sh, bool absolute)
             double s = 0.0;
             int cnt = 0;
             for (int w = 0; w < nwarps; ++w) { s += sh.wsum[w][lane]; cnt += sh.wcnt[w][lane]; }
-            if (!absolute) { s += sh.S[lane]; cnt += sh.n[lane]; }
-            sh.S[lane] = s;
-            sh.n[lane] = cnt;
             ck = sh.c[lane];
             if (cnt > 0) { ck = __double2float_rn(__ddiv_rn(s, (double)cnt)); sh.c[lane] = ck; }
         }
-        ck = __shfl_sync(0xffffffffu, ck, lane < K ? lane : K - 1);
-        float cp = __shfl_up_sync(0xffffffffu, ck, 1);
-        double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
-        bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
-        ok = __all_sync(0xffffffffu, ok);
-        if (lane == 0) sh.fast = ok ? 1 : 0;
+        decide_fast_warp0<K>(sh, ck);
+        if (lane == 0) sh.bound_valid = 0;
+    }
+}
+
+// Warp 0, ordered path: boundaries from the warps' votes, cluster sums from prefix sums.
+//   sh.wcnt[w][k] = threads of warp w whose last code is < k  (k = 1..K-1)
+//   codes_s[t]    = packed codes of thread t
+template <int DT, int K, int E>
+__device__ __forceinline__ void update_from_boundaries(LloydShared& sh, const uint32_t* codes_s,
+                                                       const uint32_t* sorted, int N) {
+    constexpr int WORDS = (E + 7) / 8;
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x, nwarps = blockDim.x >> 5, nthr = blockDim.x;
+        // lane k (0..K) evaluates B_k = number of weights with a code below k, and the fp64
+        // prefix sum of the first B_k sorted weights
+        int B = 0;
+        double P = 0.0;
+        if (lane <= K) {
+            if (lane == K) {
+                B = N;
+            } else if (lane > 0) {
+                int t = 0;
+                for (int w = 0; w < nwarps; ++w) t += sh.wcnt[w][lane];
+                B = t * E;
+                if (t < nthr) {
+                    int q = 0;
+#pragma unroll
+                    for (int w = 0; w < WORDS; ++w) {
+                        uint32_t word = codes_s[t * WORDS + w];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (8 * w + i < E) q += ((int)((word >> (4 * i)) & 15u) < lane) ? 1 : 0;
+                    }
+                    B += q;
+                }
+                B = B < N ? B : N;
+            }
+            const int t = B / E, r = B - t * E;
+            P = sh.pt[t];
+            for (int e = 0; e < r; ++e) P += (double)value_of_key16<DT>(sorted[t * E + e] >> 16);
+        }
+        const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
+        const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
+        float ck = 0.f;
+        bool moved = false;
+        if (lane < K) {
+            const int cnt = Bn - B;
+            ck = sh.c[lane];
+            if (cnt > 0) { ck = __double2float_rn(__ddiv_rn(Pn - P, (double)cnt)); sh.c[lane] = ck; }
+            moved = !sh.bound_valid || sh.bound[lane] != B;
+            sh.bound[lane] = B;
+        }
+        moved = __any_sync(0xffffffffu, moved);
+        decide_fast_warp0<K>(sh, ck);
+        if (lane == 0) { sh.stop = moved ? 0 : 1; sh.bound_valid = 1; }
     }
 }
 
 template <int DT, int K, int E>
-__device__ void fit_channel(const LloydArgs& a, int64_t row, float (&x)[E], int nval, LloydShared& sh,
-                            unsigned char* dyn, const float* xs) {
-    constexpr int G = E / 4;          // float accumulators: codes of 4 weights each, base 16
+__device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
+                            LloydShared& sh, uint32_t* codes_s, uint32_t* sorted) {
+    constexpr int G = E / 4;            // float accumulators: codes of 4 weights each, base 16
     constexpr int WORDS = (E + 7) / 8;  // packed codes: 8 weights per 32-bit word
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int N = (int)a.d_out;
     const int T = a.iters;
-    uint32_t* list = reinterpret_cast<uint32_t*>(dyn);
-    const int list_cap = N >> 3;
 
-    select_start<DT, K, E>(x, nval, N, sh, reinterpret_cast<int*>(dyn));
-    if (tid < 2) { sh.changed[tid] = 0; sh.list_count[tid] = 0; }
-    decide_fast<K>(sh);
+    // start: K evenly spaced order statistics
+    if (tid < 32) {
+        float ck = 0.f;
+        if (tid < K) {
+            int pos = (int)(((long long)(2 * tid + 1) * N) / (2 * K));
+            ck = value_of_key16<DT>(sorted[pos] >> 16);
+            sh.c[tid] = ck;
+        }
+        decide_fast_warp0<K>(sh, ck);
+        if (tid == 0) { sh.bound_valid = 0; sh.stop = 0; }
+    }
     __syncthreads();
 
     uint32_t cw[WORDS];
 #pragma unroll
-    for (int w = 0; w < WORDS; ++w) cw[w] = 0;
+    for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;
     float c[K];
     int sweeps_done = 0;
-    int prev_changed = N;
     for (int it = 0; it <= T; ++it) {
 #pragma unroll
         for (int k = 0; k < K; ++k) c[k] = sh.c[k];
         const bool fast = sh.fast != 0;
-        const bool last = (it == T), first = (it == 0);
-        const bool use_list = !first && !last && prev_changed <= list_cap;
-        const int par = it & 1;
+        const bool last = (it == T);
 
         uint32_t half[G];  // 16 bits: the codes of weights 4g..4g+3
         if (fast) {
@@ -337,89 +357,65 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, float (&x)[E], int 
         for (int w = 0; w < WORDS; ++w)
             nw[w] = (2 * w + 1 < G) ? __byte_perm(half[2 * w], half[2 * w + 1], 0x5410) : (half[2 * w] & 0xffffu);
         ++sweeps_done;
-
-        // weights whose code changed (few once the fit settles)
         uint32_t any = 0;
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w) any |= nw[w] ^ cw[w];
-        int nch = 0;
-        if (first) {
-            nch = nval;
-        } else if (any) {
-            uint32_t m[WORDS];  // bit 4i set: weight i of the word changed
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) {
-                uint32_t xr = nw[w] ^ cw[w];
-                m[w] = (xr | (xr >> 1) | (xr >> 2) | (xr >> 3)) & 0x11111111u;
-                nch += __popc(m[w]);
-            }
-            if (use_list) {
-                int pos = atomicAdd(&sh.list_count[par], nch);
-#pragma unroll
-                for (int w = 0; w < WORDS; ++w) {
-                    uint32_t mm = m[w];
-                    while (mm) {
-                        const int b = __ffs(mm) - 1;
-                        mm &= mm - 1;
-                        const int e = 8 * w + (b >> 2);
-                        const uint32_t j = (uint32_t)(((e >> 2) * nthr + tid) * 4 + (e & 3));
-                        if (pos < list_cap)
-                            list[pos] = j | (((cw[w] >> b) & 15u) << 16) | (((nw[w] >> b) & 15u) << 20);
-                        ++pos;
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int w = 0; w < WORDS; ++w) cw[w] = nw[w];
-        nch = warp_sum(nch);
-        if (lane == 0 && nch) atomicAdd(&sh.changed[par], nch);
-        __syncthreads();
-        const int total_changed = sh.changed[par];
-        const int L = sh.list_count[par];
-        if (tid == 0) { sh.changed[par ^ 1] = 0; sh.list_count[par ^ 1] = 0; }
-        prev_changed = total_changed;
-        if (last || total_changed == 0) break;  // uniform: every thread reads the same value
-        const bool by_list = use_list && L <= list_cap;
-        if (by_list) list_partials<K>(list, L, xs, sh);
-        else rebuild_partials<K, E>(x, cw, nval, sh);
-        __syncthreads();
-        update_centroids<K>(sh, !by_list);
-        __syncthreads();
-    }
+        for (int w = 0; w < WORDS; ++w) { any |= nw[w] ^ cw[w]; cw[w] = nw[w]; }
+        if (last) break;
 
-    // outputs: thread owns weights j = (g * nthr + tid) * 4 + u
+        if (fast) {
+            // codes are non-decreasing along the sorted order: publish them and vote the boundaries
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) codes_s[tid * WORDS + w] = cw[w];
+            const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
+#pragma unroll
+            for (int k = 1; k < K; ++k) {
+                unsigned m = __ballot_sync(0xffffffffu, c_last < k);
+                if (lane == 0) sh.wcnt[warp][k] = __popc(m);
+            }
+            __syncthreads();
+            update_from_boundaries<DT, K, E>(sh, codes_s, sorted, N);
+            __syncthreads();
+            if (sh.stop) break;
+        } else {
+            const int changed = __syncthreads_or(any != 0);
+            if (!changed) break;
+            rebuild_partials<K, E>(x, cw, nval, sh);
+            __syncthreads();
+            update_from_partials<K>(sh);
+            __syncthreads();
+        }
+    }
+    __syncthreads();  // warp 0 is done with `sorted`
+
+    // outputs, staged through shared memory back into column order
     if (a.lut && tid < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + tid] = tid < K ? sh.c[tid] : 0.f;
-    const bool vec4 = (a.d_out & 3) == 0;
+    uint32_t colv[E];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        const int j0 = (g * nthr + tid) * 4;
-        if (j0 >= N) continue;
-        const uint32_t p = (cw[g >> 1] >> (16 * (g & 1))) & 0xffffu;
-        if (a.codes) {
-            uint8_t* out = a.codes + row * a.d_out + j0;
-            if (vec4) {
-                uint32_t w = (p & 15u) | (((p >> 4) & 15u) << 8) | (((p >> 8) & 15u) << 16) | (((p >> 12) & 15u) << 24);
-                *reinterpret_cast<uint32_t*>(out) = w;
-            } else {
+    for (int e = 0; e < E; ++e) colv[e] = (e < nval) ? (sorted[tid * E + e] & 0xffffu) : 0u;
+    __syncthreads();  // every thread has its columns: `sorted` may be overwritten
+    if (a.codes) {
+        uint8_t* stage = reinterpret_cast<uint8_t*>(sorted);
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (j0 + u < N) out[u] = (uint8_t)((p >> (4 * u)) & 15u);
-            }
+        for (int e = 0; e < E; ++e)
+            if (e < nval) stage[colv[e]] = (uint8_t)((cw[e >> 3] >> (4 * (e & 7))) & 15u);
+        __syncthreads();
+        uint8_t* out = a.codes + row * a.d_out;
+        if ((a.d_out & 3) == 0) {
+            const uint32_t* s4 = reinterpret_cast<const uint32_t*>(stage);
+            uint32_t* o4 = reinterpret_cast<uint32_t*>(out);
+            for (int j = tid; j < (N >> 2); j += nthr) o4[j] = s4[j];
+        } else {
+            for (int j = tid; j < N; j += nthr) out[j] = stage[j];
         }
-        if (a.err) {
-            float* out = a.err + row * a.d_out + j0;
-            float ev[4];
+    }
+    if (a.err) {
+        float* stage = reinterpret_cast<float*>(sorted);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) ev[u] = fabsf(x[4 * g + u] - sh.c[(p >> (4 * u)) & 15u]);
-            if (vec4) {
-                *reinterpret_cast<float4*>(out) = make_float4(ev[0], ev[1], ev[2], ev[3]);
-            } else {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (j0 + u < N) out[u] = ev[u];
-            }
-        }
+        for (int e = 0; e < E; ++e)
+            if (e < nval) stage[colv[e]] = fabsf(x[e] - sh.c[(cw[e >> 3] >> (4 * (e & 7))) & 15u]);
+        __syncthreads();
+        float* out = a.err + row * a.d_out;
+        for (int j = tid; j < N; j += nthr) out[j] = stage[j];
     }
     if (a.sweeps && tid == 0)
         atomicAdd(a.sweeps, (unsigned long long)sweeps_done * (unsigned long long)N * (unsigned long long)K);
@@ -433,12 +429,13 @@ lloyd_kernel(const LloydArgs a) {
     if (a.skip_row && a.skip_row[row]) return;
     const int N = (int)a.d_out;
     LloydShared& sh = *reinterpret_cast<LloydShared*>(smem_raw);
-    unsigned char* dyn = smem_raw + sizeof(LloydShared);          // hist2 / change list / bitmap
-    float* xs = reinterpret_cast<float*>(dyn + lloyd_scratch_bytes(N));  // fp32 copy of the channel
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
+    unsigned char* scratch = smem_raw + sizeof(LloydShared);
+    uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int nwarps = nthr >> 5;
 
     // removed positions (outliers of this row) are marked in a bitmap over the columns
-    uint32_t* removed = reinterpret_cast<uint32_t*>(dyn);
+    uint32_t* removed = reinterpret_cast<uint32_t*>(scratch);
     int64_t p0 = 0, p1 = 0;
     if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
     const bool has_removed = p1 > p0;
@@ -449,63 +446,55 @@ lloyd_kernel(const LloydArgs a) {
             int col = a.cols[p];
             atomicOr(&removed[col >> 5], 1u << (col & 31));
         }
+        __syncthreads();
     }
-    __syncthreads();
 
-    // thread owns weights j = (g * nthr + tid) * 4 + u, u = 0..3; valid ones form a prefix
+    // column layout for the load: thread owns columns (g * nthr + tid) * 4 + u
     const uint16_t* w = a.W + row * a.ldw;
     const bool vec = ((a.ldw & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 7) == 0);
-    float x[E];
-    int nval = 0;
-#pragma unroll
-    for (int g = 0; g < E / 4; ++g) {
-        const int j0 = (g * nthr + tid) * 4;
-        uint16_t h[4] = {0, 0, 0, 0};
-        if (j0 + 3 < N && vec) {
-            uint2 v = *reinterpret_cast<const uint2*>(w + j0);
-            h[0] = (uint16_t)(v.x & 0xffff); h[1] = (uint16_t)(v.x >> 16);
-            h[2] = (uint16_t)(v.y & 0xffff); h[3] = (uint16_t)(v.y >> 16);
-        } else {
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (j0 + u < N) h[u] = w[j0 + u];
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            float v = widen16<DT>(h[u]);
-            const int j = j0 + u;
-            if (j < N) {
-                ++nval;
-                if (has_removed && ((removed[j >> 5] >> (j & 31)) & 1)) v = 0.f;
-                v = (v == 0.f) ? 0.f : v;  // -0 and +0 are the same point
-                xs[j] = v;
-            } else {
-                v = __int_as_float(0x7f800000);  // padding: +inf always gets code 0 and never changes
-            }
-            x[4 * g + u] = v;
-        }
-    }
-    // value range (for the gap test) and exactness diagnostics
+    uint32_t key[E];
+    int nval_cols = 0;
     {
         float lo = __int_as_float(0x7f800000), hi = __int_as_float(0xff800000);
         int top = -100000, ulp = 100000;
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            if (e < nval) {
-                lo = fminf(lo, x[e]);
-                hi = fmaxf(hi, x[e]);
-                uint32_t u = __float_as_uint(x[e]) & 0x7fffffffu;
-                if (u) {
-                    int ex = (int)(u >> 23);
-                    uint32_t m = u & 0x7fffffu;
-                    int t, q;
-                    if (ex) { t = ex - 127; q = ex - 150 + (__ffs(m | 0x800000u) - 1); }
-                    else    { t = (31 - __clz(m)) - 149; q = (__ffs(m) - 1) - 149; }
-                    top = max(top, t);
-                    ulp = min(ulp, q);
+        for (int g = 0; g < E / 4; ++g) {
+            const int j0 = (g * nthr + tid) * 4;
+            uint16_t h[4] = {0, 0, 0, 0};
+            if (j0 + 3 < N && vec) {
+                uint2 v = *reinterpret_cast<const uint2*>(w + j0);
+                h[0] = (uint16_t)(v.x & 0xffff); h[1] = (uint16_t)(v.x >> 16);
+                h[2] = (uint16_t)(v.y & 0xffff); h[3] = (uint16_t)(v.y >> 16);
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (j0 + u < N) h[u] = w[j0 + u];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = j0 + u;
+                float v = widen16<DT>(h[u]);
+                if (j < N) {
+                    ++nval_cols;
+                    if (has_removed && ((removed[j >> 5] >> (j & 31)) & 1)) v = 0.f;
+                    v = (v == 0.f) ? 0.f : v;  // -0 and +0 are the same point
+                    lo = fminf(lo, v);
+                    hi = fmaxf(hi, v);
+                    uint32_t ub = __float_as_uint(v) & 0x7fffffffu;
+                    if (ub) {
+                        int ex = (int)(ub >> 23);
+                        uint32_t m = ub & 0x7fffffu;
+                        int t, q;
+                        if (ex) { t = ex - 127; q = ex - 150 + (__ffs(m | 0x800000u) - 1); }
+                        else    { t = (31 - __clz(m)) - 149; q = (__ffs(m) - 1) - 149; }
+                        top = max(top, t);
+                        ulp = min(ulp, q);
+                    }
                 }
+                key[4 * g + u] = sort_key16<DT>(v);
             }
         }
+        // value range (for the gap test) and exactness diagnostics
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
@@ -513,7 +502,6 @@ lloyd_kernel(const LloydArgs a) {
             top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
             ulp = min(ulp, __shfl_xor_sync(0xffffffffu, ulp, o));
         }
-        const int warp = tid >> 5, nwarps = nthr >> 5;
         if (lane == 0) { sh.wlo[warp] = lo; sh.whi[warp] = hi; sh.wtop[warp] = top; sh.wulp[warp] = ulp; }
         __syncthreads();  // also: every thread is done with the removed-column bitmap
         if (tid == 0) {
@@ -532,16 +520,51 @@ lloyd_kernel(const LloydArgs a) {
                 if (log2n + 1 + (top + 1 - ulp) > 53) atomicAdd(a.inexact_rows, 1);
             }
         }
+    }
+
+    sort_channel<E>(key, nval_cols, sh, reinterpret_cast<int*>(scratch), sorted);
+
+    // sorted layout: thread t keeps order statistics [E t, E t + E); padding repeats the maximum
+    float x[E];
+    int nval = N - tid * E;
+    nval = nval < 0 ? 0 : (nval > E ? E : nval);
+    {
+        const float vlast = value_of_key16<DT>(sorted[N - 1] >> 16);
+        double tot = 0.0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (e < nval) {
+                x[e] = value_of_key16<DT>(sorted[tid * E + e] >> 16);
+                tot += (double)x[e];
+            } else {
+                x[e] = vlast;
+            }
+        }
+        // exclusive scan of the thread totals over the block
+        double incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) sh.wsum[warp][0] = incl;
+        __syncthreads();
+        double base = 0.0;
+        for (int wv = 0; wv < warp; ++wv) base += sh.wsum[wv][0];
+        sh.pt[tid] = base + incl - tot;
+        if (tid == nthr - 1) sh.pt[nthr] = base + incl;
         __syncthreads();
     }
+
+    uint32_t* codes_s = reinterpret_cast<uint32_t*>(scratch);
     const int bits = a.bits[row];
-    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, dyn, xs);
-    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, dyn, xs);
-    else fit_channel<DT, 16, E>(a, row, x, nval, sh, dyn, xs);
+    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
+    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
+    else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out) {
-    return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * sizeof(float);
+    return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4;
 }
 
 template <int DT, int E, int MAXT>
