@@ -44,6 +44,8 @@ struct alignas(16) LloydShared {
     int excl1[257];
     int bucket_rank[256];           // rank of a high-byte bucket among the non-empty ones, or -1
     float c[kMaxK];
+    double part_sum[kMaxK];         // boundary k inside a thread: sum / count of that thread's
+    int part_cnt[kMaxK];            //   weights with a code below k
     int bound[kMaxK + 1];           // B_k of the last ordered sweep
     int bound_valid;
     int n_nonempty;
@@ -236,42 +238,78 @@ __device__ __forceinline__ void update_from_partials(LloydShared& sh) {
     }
 }
 
-// Warp 0, ordered path: boundaries from the warps' votes, cluster sums from prefix sums.
-//   sh.wcnt[w][k] = threads of warp w whose last code is < k  (k = 1..K-1)
-//   codes_s[t]    = packed codes of thread t
-template <int DT, int K, int E>
-__device__ __forceinline__ void update_from_boundaries(LloydShared& sh, const uint32_t* codes_s,
-                                                       const uint32_t* sorted, int N) {
+// Number of the E packed 4-bit codes that are below k (byte-wise SWAR compare of the even and the
+// odd nibbles: n + 128 - k has bit 7 set exactly when n >= k).
+template <int E>
+struct PackedCodes { uint32_t w[(E + 7) / 8]; };
+
+template <int E>
+__device__ __forceinline__ int count_below(const PackedCodes<E>& pc, int k) {
     constexpr int WORDS = (E + 7) / 8;
+    const uint32_t (&cw)[WORDS] = pc.w;
+    const uint32_t kk = (uint32_t)k * 0x01010101u;
+    int ge = 0;
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) {
+        uint32_t ev = cw[w] & 0x0f0f0f0fu, od = (cw[w] >> 4) & 0x0f0f0f0fu;
+        ge += __popc(((ev | 0x80808080u) - kk) & 0x80808080u) + __popc(((od | 0x80808080u) - kk) & 0x80808080u);
+    }
+    // a word holding fewer than 8 codes has zero padding nibbles: they compare as "below"
+    return 8 * WORDS - ge - (8 * WORDS - E);
+}
+
+// A thread whose codes differ holds boundaries c_first < k <= c_last in its interior.  For each it
+// publishes how many of its weights lie below the boundary and their fp64 sum (the shorter side
+// is added up; the other side follows from the thread's total).  `mine` = the thread's sorted run.
+template <int DT, int E>
+__device__ __noinline__ void boundary_partials(PackedCodes<E> cw, int c_first, int c_last, int nval,
+                                               const uint32_t* mine, LloydShared& sh) {
+    const int tid = threadIdx.x;
+#pragma unroll 1
+    for (int k = c_first + 1; k <= c_last; ++k) {
+        const int q = count_below<E>(cw, k);
+        double s0 = 0.0, s1 = 0.0;
+        const bool low_side = 2 * q <= nval;
+        const int e0 = low_side ? 0 : q, e1 = low_side ? q : nval;
+        int e = e0;
+#pragma unroll 1
+        for (; e + 1 < e1; e += 2) {
+            s0 += (double)value_of_key16<DT>(mine[e] >> 16);
+            s1 += (double)value_of_key16<DT>(mine[e + 1] >> 16);
+        }
+        if (e < e1) s0 += (double)value_of_key16<DT>(mine[e] >> 16);
+        double s = s0 + s1;
+        if (!low_side) s = (sh.pt[tid + 1] - sh.pt[tid]) - s;
+        sh.part_sum[k] = s;
+        sh.part_cnt[k] = q;
+    }
+}
+
+// Warp 0, ordered path: boundaries from the warps' votes, cluster sums from prefix sums.
+//   sh.wcnt[w][k]  = threads of warp w whose last code is < k  (k = 1..K-1)
+//   first_code_s[t] = packed codes of thread t's first eight weights
+//   sh.part_*[k]   = written this sweep by the thread that holds boundary k in its interior
+template <int K, int E>
+__device__ __forceinline__ void update_from_boundaries(LloydShared& sh, const uint32_t* first_code_s, int N) {
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x, nwarps = blockDim.x >> 5, nthr = blockDim.x;
         // lane k (0..K) evaluates B_k = number of weights with a code below k, and the fp64
-        // prefix sum of the first B_k sorted weights
+        // sum P_k of those weights
         int B = 0;
         double P = 0.0;
-        if (lane <= K) {
-            if (lane == K) {
-                B = N;
-            } else if (lane > 0) {
-                int t = 0;
-                for (int w = 0; w < nwarps; ++w) t += sh.wcnt[w][lane];
-                B = t * E;
-                if (t < nthr) {
-                    int q = 0;
-#pragma unroll
-                    for (int w = 0; w < WORDS; ++w) {
-                        uint32_t word = codes_s[t * WORDS + w];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (8 * w + i < E) q += ((int)((word >> (4 * i)) & 15u) < lane) ? 1 : 0;
-                    }
-                    B += q;
-                }
-                B = B < N ? B : N;
-            }
-            const int t = B / E, r = B - t * E;
+        if (lane == K) {
+            B = N;
+            P = sh.pt[nthr];
+        } else if (lane > 0 && lane < K) {
+            int t = 0;
+            for (int w = 0; w < nwarps; ++w) t += sh.wcnt[w][lane];
+            B = t * E;
             P = sh.pt[t];
-            for (int e = 0; e < r; ++e) P += (double)value_of_key16<DT>(sorted[t * E + e] >> 16);
+            if (t < nthr && (int)(first_code_s[t] & 15u) < lane) {  // boundary inside thread t
+                B += sh.part_cnt[lane];
+                P += sh.part_sum[lane];
+            }
+            if (B >= N) { B = N; P = sh.pt[nthr]; }
         }
         const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
         const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
@@ -363,17 +401,24 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         if (last) break;
 
         if (fast) {
-            // codes are non-decreasing along the sorted order: publish them and vote the boundaries
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) codes_s[tid * WORDS + w] = cw[w];
+            // codes are non-decreasing along the sorted order: vote the boundaries; a thread with
+            // a boundary in its interior also publishes the sum and count of its weights below it
+            codes_s[tid] = cw[0];
+            const int c_first = (int)(cw[0] & 15u);
             const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
 #pragma unroll
             for (int k = 1; k < K; ++k) {
                 unsigned m = __ballot_sync(0xffffffffu, c_last < k);
                 if (lane == 0) sh.wcnt[warp][k] = __popc(m);
             }
+            if (c_first != c_last) {
+                PackedCodes<E> pc;
+#pragma unroll
+                for (int w = 0; w < WORDS; ++w) pc.w[w] = cw[w];
+                boundary_partials<DT, E>(pc, c_first, c_last, nval, sorted + tid * E, sh);
+            }
             __syncthreads();
-            update_from_boundaries<DT, K, E>(sh, codes_s, sorted, N);
+            update_from_boundaries<K, E>(sh, codes_s, N);
             __syncthreads();
             if (sh.stop) break;
         } else {
