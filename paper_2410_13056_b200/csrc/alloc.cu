@@ -9,7 +9,7 @@
 namespace cmpq {
 
 constexpr int kRankThreads = 256;
-constexpr int kRankSlice = 2048;  // candidates one block compares against
+constexpr int kRankSlice = 256;   // candidates one block compares against
 
 size_t alloc_ws_bytes(int64_t d_in) {
     return 2 * round_up((size_t)d_in * sizeof(int32_t), 256);

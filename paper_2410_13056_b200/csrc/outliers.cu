@@ -175,30 +175,82 @@ row_scan_kernel(const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
     if (threadIdx.x == 0) row_start[d_in] = out_before;
 }
 
-// Each row writes its kept entries in column order.
+// Each row writes its kept entries in column order.  Rows of O_act are copied whole.  In the
+// other rows kept entries are rare: candidates (error >= tau) are gathered into a short list in
+// shared memory, ordered by column by counting, and the first take_eq[row] of those equal to tau
+// are kept next to all larger ones.  A row with more candidates than the list holds falls back
+// to a scan-based ordered compaction.
+constexpr int kEmitListCap = 1024;
+
 __global__ void __launch_bounds__(kSelThreads)
 emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __restrict__ err,
             const uint8_t* __restrict__ is_act, int64_t d_out, const SelectState* __restrict__ st,
+            const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
             const int32_t* __restrict__ take_eq, const int64_t* __restrict__ row_start,
             int32_t* __restrict__ rows, int32_t* __restrict__ cols, uint16_t* __restrict__ vals) {
     __shared__ int warp_totals[32];
+    __shared__ int list_col[kEmitListCap];
+    __shared__ unsigned char list_eq[kEmitListCap];
+    __shared__ int list_n;
     const int64_t row = blockIdx.x;
     const int64_t out0 = row_start[row];
     if (row_start[row + 1] == out0) return;
-    const bool act = is_act[row] != 0;
+    const uint16_t* w = W + row * ldw;
+    if (is_act[row]) {
+        for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
+            rows[out0 + j] = (int32_t)row;
+            cols[out0 + j] = (int32_t)j;
+            vals[out0 + j] = w[j];
+        }
+        return;
+    }
     const uint32_t tau = st->tau;
     const int te = take_eq[row];
     const uint32_t* e = reinterpret_cast<const uint32_t*>(err + row * d_out);
-    const uint16_t* w = W + row * ldw;
+    const int ncand = gt[row] + eq[row];
+    if (ncand <= kEmitListCap) {
+        if (threadIdx.x == 0) list_n = 0;
+        __syncthreads();
+        for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
+            uint32_t u = e[j];
+            if (u >= tau) {
+                int p = atomicAdd(&list_n, 1);
+                list_col[p] = (int)j;
+                list_eq[p] = u == tau ? 1 : 0;
+            }
+        }
+        __syncthreads();
+        const int n = list_n;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int c = list_col[i];
+            const int is_eq = list_eq[i];
+            int before = 0, eq_before = 0;   // candidates / tau-candidates in lower columns
+            for (int t = 0; t < n; ++t) {
+                int lower = list_col[t] < c ? 1 : 0;
+                before += lower;
+                eq_before += lower & list_eq[t];
+            }
+            const bool keep = !is_eq || eq_before < te;
+            if (keep) {
+                // dropped tau-candidates are exactly those of tau-rank >= te, all after the kept ones
+                int dropped_before = eq_before > te ? eq_before - te : 0;
+                int64_t pos = out0 + before - dropped_before;
+                rows[pos] = (int32_t)row;
+                cols[pos] = c;
+                vals[pos] = w[c];
+            }
+        }
+        return;
+    }
     int eq_seen = 0, written = 0;
     for (int64_t base = 0; base < d_out; base += blockDim.x) {
         int64_t j = base + threadIdx.x;
         bool in = j < d_out;
-        uint32_t u = (in && !act) ? e[j] : 0u;
-        int is_eq = (in && !act && u == tau) ? 1 : 0;
+        uint32_t u = in ? e[j] : 0u;
+        int is_eq = (in && u == tau) ? 1 : 0;
         int tot_eq;
         int eq_rank = eq_seen + block_exclusive_scan(is_eq, warp_totals, tot_eq);
-        int keep = in && (act || u > tau || (is_eq && eq_rank < te)) ? 1 : 0;
+        int keep = in && (u > tau || (is_eq && eq_rank < te)) ? 1 : 0;
         int tot_keep;
         int pos = written + block_exclusive_scan(keep, warp_totals, tot_keep);
         if (keep) {
@@ -308,6 +360,6 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
     }
     row_scan_kernel<<<1, 1024, 0, st>>>(o.gt, o.eq, o.is_act, d_in, d_out, o.state, o.take_eq, o.row_start);
     if (nnz_out > 0)
-        emit_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(static_cast<const uint16_t*>(W), ldw, o.err, o.is_act, d_out, o.state, o.take_eq, o.row_start, rows, cols, vals);
+        emit_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(static_cast<const uint16_t*>(W), ldw, o.err, o.is_act, d_out, o.state, o.gt, o.eq, o.take_eq, o.row_start, rows, cols, vals);
     return launch_status();
 }
