@@ -173,12 +173,10 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    from paper_2410_13056_b200 import sharding
+
     def max_over_ranks(x):
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.max_over_ranks(x, device="cuda")
 
     warmup = max(args.warmup, 3)
     steps = args.steps
