@@ -37,27 +37,24 @@ constexpr int kMaxWarps = 32;
 constexpr int kMaxThreads = 1024;
 
 struct alignas(16) LloydShared {
-    double pt[kMaxThreads + 1];     // exclusive prefix over threads of the threads' fp64 totals
-    double wsum[kMaxWarps][kMaxK];  // per-warp cluster sums (rebuild path), per-warp totals (scan)
-    int wcnt[kMaxWarps][kMaxK];     // per-warp cluster counts (rebuild) / threads below boundary k
+    double pt[kMaxThreads + 1];        // exclusive prefix over threads of the threads' fp64 totals
+    // exchanged once per sweep, double-buffered by sweep parity so that one barrier per sweep is enough
+    double wsum[2][kMaxWarps][kMaxK];  // per-warp cluster sums (rebuild path); [0][w][0]: totals (scan)
+    int wcnt[2][kMaxWarps][kMaxK];     // per-warp cluster counts (rebuild) / threads below boundary k
+    double part_sum[2][kMaxK];         // boundary k inside a thread: sum / count of that thread's
+    int part_cnt[2][kMaxK];            //   weights with a code below k
     int hist1[256];
     int excl1[257];
-    int bucket_rank[256];           // rank of a high-byte bucket among the non-empty ones, or -1
-    float c[kMaxK];
-    double part_sum[kMaxK];         // boundary k inside a thread: sum / count of that thread's
-    int part_cnt[kMaxK];            //   weights with a code below k
-    int bound[kMaxK + 1];           // B_k of the last ordered sweep
-    int bound_valid;
+    int bucket_rank[256];              // rank of a high-byte bucket among the non-empty ones, or -1
+    float c[kMaxK];                    // final centroids (for the outputs)
     int n_nonempty;
-    int fast;                       // centroids strictly increasing with safe gaps
-    int stop;
-    float vmin, vmax;               // value range of the channel
+    float vmin, vmax;                  // value range of the channel
     float wlo[kMaxWarps], whi[kMaxWarps];
     int wtop[kMaxWarps], wulp[kMaxWarps];
 };
 // dynamic shared memory after LloydShared:
 //   scratch (lloyd_scratch_bytes): removed-column bitmap during the load, second-level histogram
-//                                  during the sort, then the threads' packed codes
+//                                  during the sort, then the threads' first code words (2 x 4 B)
 //   sorted  (4 bytes per weight):  key << 16 | column, ascending; reused for the output staging
 
 __host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
@@ -183,22 +180,21 @@ __device__ void sort_channel(const uint32_t (&key)[E], int nval, LloydShared& sh
     }
 }
 
-// Warp 0 decides whether the counting sweep is valid for the new centroids (lane k holds c_k).
+// Whether the counting sweep is valid for the centroids (lane k holds c_k): strictly increasing
+// with every gap above 2^-22 of the channel's value range.  Same answer in every lane.
 template <int K>
-__device__ __forceinline__ void decide_fast_warp0(LloydShared& sh, float ck_lane) {
-    const int lane = threadIdx.x;
+__device__ __forceinline__ bool counting_sweep_valid(float ck_lane, double need) {
+    const int lane = threadIdx.x & 31;
     float ck = __shfl_sync(0xffffffffu, ck_lane, lane < K ? lane : K - 1);
     float cp = __shfl_up_sync(0xffffffffu, ck, 1);
-    double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
     bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
-    ok = __all_sync(0xffffffffu, ok);
-    if (lane == 0) sh.fast = ok ? 1 : 0;
+    return __all_sync(0xffffffffu, ok);
 }
 
 // Per-warp cluster sums and counts of all weights, from the codes in registers (any order).
 template <int K, int E>
 __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 7) / 8], int nval,
-                                 LloydShared& sh) {
+                                 LloydShared& sh, int par) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int code[E];
 #pragma unroll
@@ -215,27 +211,22 @@ __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 
         }
         s = warp_sum(s);
         cnt = warp_sum(cnt);
-        if (lane == 0) { sh.wsum[warp][k] = s; sh.wcnt[warp][k] = cnt; }
+        if (lane == 0) { sh.wsum[par][warp][k] = s; sh.wcnt[par][warp][k] = cnt; }
     }
 }
 
-// Warp 0, rebuild path: combine the per-warp partials, move every non-empty cluster's centroid to
-// its mean, decide the next sweep's mode.
+// Rebuild path, every warp for itself: lane k combines the per-warp partials of cluster k and moves
+// the centroid to the mean if the cluster has members.
 template <int K>
-__device__ __forceinline__ void update_from_partials(LloydShared& sh) {
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x, nwarps = blockDim.x >> 5;
-        float ck = 0.f;
-        if (lane < K) {
-            double s = 0.0;
-            int cnt = 0;
-            for (int w = 0; w < nwarps; ++w) { s += sh.wsum[w][lane]; cnt += sh.wcnt[w][lane]; }
-            ck = sh.c[lane];
-            if (cnt > 0) { ck = __double2float_rn(__ddiv_rn(s, (double)cnt)); sh.c[lane] = ck; }
-        }
-        decide_fast_warp0<K>(sh, ck);
-        if (lane == 0) sh.bound_valid = 0;
+__device__ __forceinline__ float centroid_from_partials(const LloydShared& sh, int par, float ck) {
+    const int lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    if (lane < K) {
+        double s = 0.0;
+        int cnt = 0;
+        for (int w = 0; w < nwarps; ++w) { s += sh.wsum[par][w][lane]; cnt += sh.wcnt[par][w][lane]; }
+        if (cnt > 0) ck = __double2float_rn(__ddiv_rn(s, (double)cnt));
     }
+    return ck;
 }
 
 // Number of the E packed 4-bit codes that are below k (byte-wise SWAR compare of the even and the
@@ -263,7 +254,7 @@ __device__ __forceinline__ int count_below(const PackedCodes<E>& pc, int k) {
 // is added up; the other side follows from the thread's total).  `mine` = the thread's sorted run.
 template <int DT, int E>
 __device__ __noinline__ void boundary_partials(PackedCodes<E> cw, int c_first, int c_last, int nval,
-                                               const uint32_t* mine, LloydShared& sh) {
+                                               const uint32_t* mine, LloydShared& sh, int par) {
     const int tid = threadIdx.x;
 #pragma unroll 1
     for (int k = c_first + 1; k <= c_last; ++k) {
@@ -280,75 +271,67 @@ __device__ __noinline__ void boundary_partials(PackedCodes<E> cw, int c_first, i
         if (e < e1) s0 += (double)value_of_key16<DT>(mine[e] >> 16);
         double s = s0 + s1;
         if (!low_side) s = (sh.pt[tid + 1] - sh.pt[tid]) - s;
-        sh.part_sum[k] = s;
-        sh.part_cnt[k] = q;
+        sh.part_sum[par][k] = s;
+        sh.part_cnt[par][k] = q;
     }
 }
 
-// Warp 0, ordered path: boundaries from the warps' votes, cluster sums from prefix sums.
-//   sh.wcnt[w][k]  = threads of warp w whose last code is < k  (k = 1..K-1)
-//   first_code_s[t] = packed codes of thread t's first eight weights
-//   sh.part_*[k]   = written this sweep by the thread that holds boundary k in its interior
+// Ordered path, every warp for itself: lane k (0..K) evaluates B_k = number of weights with a code
+// below k and the fp64 sum P_k of those weights; cluster k is the run [B_k, B_{k+1}).
+//   sh.wcnt[par][w][k]  = threads of warp w whose last code is < k  (k = 1..K-1)
+//   first_code_s[t]     = packed codes of thread t's first eight weights
+//   sh.part_*[par][k]   = written this sweep by the thread that holds boundary k in its interior
+// Returns the new centroid of cluster `lane` (the old one if the cluster is empty); B_out = B_lane.
 template <int K, int E>
-__device__ __forceinline__ void update_from_boundaries(LloydShared& sh, const uint32_t* first_code_s, int N) {
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x, nwarps = blockDim.x >> 5, nthr = blockDim.x;
-        // lane k (0..K) evaluates B_k = number of weights with a code below k, and the fp64
-        // sum P_k of those weights
-        int B = 0;
-        double P = 0.0;
-        if (lane == K) {
-            B = N;
-            P = sh.pt[nthr];
-        } else if (lane > 0 && lane < K) {
-            int t = 0;
-            for (int w = 0; w < nwarps; ++w) t += sh.wcnt[w][lane];
-            B = t * E;
-            P = sh.pt[t];
-            if (t < nthr && (int)(first_code_s[t] & 15u) < lane) {  // boundary inside thread t
-                B += sh.part_cnt[lane];
-                P += sh.part_sum[lane];
-            }
-            if (B >= N) { B = N; P = sh.pt[nthr]; }
+__device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh, int par,
+                                                          const uint32_t* first_code_s, int N, float ck,
+                                                          int& B_out) {
+    const int lane = threadIdx.x & 31, nwarps = blockDim.x >> 5, nthr = blockDim.x;
+    int B = 0;
+    double P = 0.0;
+    if (lane == K) {
+        B = N;
+        P = sh.pt[nthr];
+    } else if (lane > 0 && lane < K) {
+        int t = 0;
+        for (int w = 0; w < nwarps; ++w) t += sh.wcnt[par][w][lane];
+        B = t * E;
+        P = sh.pt[t];
+        if (t < nthr && (int)(first_code_s[t] & 15u) < lane) {  // boundary inside thread t
+            B += sh.part_cnt[par][lane];
+            P += sh.part_sum[par][lane];
         }
-        const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
-        const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
-        float ck = 0.f;
-        bool moved = false;
-        if (lane < K) {
-            const int cnt = Bn - B;
-            ck = sh.c[lane];
-            if (cnt > 0) { ck = __double2float_rn(__ddiv_rn(Pn - P, (double)cnt)); sh.c[lane] = ck; }
-            moved = !sh.bound_valid || sh.bound[lane] != B;
-            sh.bound[lane] = B;
-        }
-        moved = __any_sync(0xffffffffu, moved);
-        decide_fast_warp0<K>(sh, ck);
-        if (lane == 0) { sh.stop = moved ? 0 : 1; sh.bound_valid = 1; }
+        if (B >= N) { B = N; P = sh.pt[nthr]; }
     }
+    const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
+    const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
+    if (lane < K) {
+        const int cnt = Bn - B;
+        if (cnt > 0) ck = __double2float_rn(__ddiv_rn(Pn - P, (double)cnt));
+    }
+    B_out = B;
+    return ck;
 }
 
 template <int DT, int K, int E>
 __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
-                            LloydShared& sh, uint32_t* codes_s, uint32_t* sorted) {
+                            LloydShared& sh, uint32_t* first_code_s, uint32_t* sorted) {
     constexpr int G = E / 4;            // float accumulators: codes of 4 weights each, base 16
     constexpr int WORDS = (E + 7) / 8;  // packed codes: 8 weights per 32-bit word
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int N = (int)a.d_out;
     const int T = a.iters;
+    const double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
 
-    // start: K evenly spaced order statistics
-    if (tid < 32) {
-        float ck = 0.f;
-        if (tid < K) {
-            int pos = (int)(((long long)(2 * tid + 1) * N) / (2 * K));
-            ck = value_of_key16<DT>(sorted[pos] >> 16);
-            sh.c[tid] = ck;
-        }
-        decide_fast_warp0<K>(sh, ck);
-        if (tid == 0) { sh.bound_valid = 0; sh.stop = 0; }
+    // Every warp keeps the centroids itself (lane k holds c_k) and repeats the tiny update, so that
+    // a sweep needs a single block-wide barrier.  All warps compute identical values.
+    float ck_lane = 0.f;
+    if (lane < K) {
+        int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
+        ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
     }
-    __syncthreads();
+    bool fast = counting_sweep_valid<K>(ck_lane, need);
+    int B_prev = -1;  // lane k: B_k of the previous ordered sweep (-1: none)
 
     uint32_t cw[WORDS];
 #pragma unroll
@@ -357,9 +340,9 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
     int sweeps_done = 0;
     for (int it = 0; it <= T; ++it) {
 #pragma unroll
-        for (int k = 0; k < K; ++k) c[k] = sh.c[k];
-        const bool fast = sh.fast != 0;
+        for (int k = 0; k < K; ++k) c[k] = __shfl_sync(0xffffffffu, ck_lane, k);
         const bool last = (it == T);
+        const int par = it & 1;
 
         uint32_t half[G];  // 16 bits: the codes of weights 4g..4g+3
         if (fast) {
@@ -401,36 +384,45 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         if (last) break;
 
         if (fast) {
-            // codes are non-decreasing along the sorted order: vote the boundaries; a thread with
-            // a boundary in its interior also publishes the sum and count of its weights below it
-            codes_s[tid] = cw[0];
+            // codes are non-decreasing along the sorted order.  Lane k finds, by bisection over the
+            // lanes' last codes, how many threads of this warp lie entirely below boundary k; a thread
+            // with a boundary in its interior also publishes the sum and count of its weights below it.
+            first_code_s[par * nthr + tid] = cw[0];
             const int c_first = (int)(cw[0] & 15u);
             const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
+            int below = 0;
 #pragma unroll
-            for (int k = 1; k < K; ++k) {
-                unsigned m = __ballot_sync(0xffffffffu, c_last < k);
-                if (lane == 0) sh.wcnt[warp][k] = __popc(m);
+            for (int step = 16; step > 0; step >>= 1) {
+                int probe = __shfl_sync(0xffffffffu, c_last, below + step - 1);
+                if (probe < lane) below += step;
             }
+            if (__shfl_sync(0xffffffffu, c_last, 31) < lane) below = 32;
+            if (lane > 0 && lane < K) sh.wcnt[par][warp][lane] = below;
             if (c_first != c_last) {
                 PackedCodes<E> pc;
 #pragma unroll
                 for (int w = 0; w < WORDS; ++w) pc.w[w] = cw[w];
-                boundary_partials<DT, E>(pc, c_first, c_last, nval, sorted + tid * E, sh);
+                boundary_partials<DT, E>(pc, c_first, c_last, nval, sorted + tid * E, sh, par);
             }
             __syncthreads();
-            update_from_boundaries<K, E>(sh, codes_s, N);
-            __syncthreads();
-            if (sh.stop) break;
+            int B;
+            ck_lane = centroid_from_boundaries<K, E>(sh, par, first_code_s + par * nthr, N, ck_lane, B);
+            const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
+            B_prev = B;
+            fast = counting_sweep_valid<K>(ck_lane, need);
+            if (!moved) break;  // same decision in every warp
         } else {
             const int changed = __syncthreads_or(any != 0);
             if (!changed) break;
-            rebuild_partials<K, E>(x, cw, nval, sh);
+            rebuild_partials<K, E>(x, cw, nval, sh, par);
             __syncthreads();
-            update_from_partials<K>(sh);
-            __syncthreads();
+            ck_lane = centroid_from_partials<K>(sh, par, ck_lane);
+            fast = counting_sweep_valid<K>(ck_lane, need);
+            B_prev = -1;
         }
     }
-    __syncthreads();  // warp 0 is done with `sorted`
+    if (warp == 0 && lane < K) sh.c[lane] = ck_lane;
+    __syncthreads();  // centroids published; no thread reads keys from `sorted` after this point
 
     // outputs, staged through shared memory back into column order
     if (a.lut && tid < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + tid] = tid < K ? sh.c[tid] : 0.f;
@@ -592,20 +584,20 @@ lloyd_kernel(const LloydArgs a) {
             double up = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += up;
         }
-        if (lane == 31) sh.wsum[warp][0] = incl;
+        if (lane == 31) sh.wsum[0][warp][0] = incl;
         __syncthreads();
         double base = 0.0;
-        for (int wv = 0; wv < warp; ++wv) base += sh.wsum[wv][0];
+        for (int wv = 0; wv < warp; ++wv) base += sh.wsum[0][wv][0];
         sh.pt[tid] = base + incl - tot;
         if (tid == nthr - 1) sh.pt[nthr] = base + incl;
         __syncthreads();
     }
 
-    uint32_t* codes_s = reinterpret_cast<uint32_t*>(scratch);
+    uint32_t* first_code_s = reinterpret_cast<uint32_t*>(scratch);
     const int bits = a.bits[row];
-    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
-    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
-    else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
+    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, first_code_s, sorted);
+    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, first_code_s, sorted);
+    else fit_channel<DT, 16, E>(a, row, x, nval, sh, first_code_s, sorted);
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out) {
