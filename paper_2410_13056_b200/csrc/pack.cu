@@ -16,82 +16,97 @@ size_t pack_ws_bytes(int64_t d_in, int64_t) {
 }
 
 // Single block: segment sizes, perm, row_off (segment order) and word_off (by channel id).
+// Thread t owns the consecutive channels [t R, t R + R); the three per-width counts travel through
+// one block-wide scan packed into a 64-bit integer (21 bits each, d_in <= 2^18).
 __global__ void __launch_bounds__(1024)
 pack_layout_kernel(const uint8_t* __restrict__ bits, int64_t d_in, int64_t d_out,
                    int64_t* __restrict__ row_off, int32_t* __restrict__ perm,
                    int64_t* __restrict__ seg_rows, int64_t* __restrict__ word_off) {
-    __shared__ int warp_tot[3][32];
-    __shared__ long long seg_count[3];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    // pass 1: channels per width
-    long long cnt[3] = {0, 0, 0};
-    for (int64_t i = threadIdx.x; i < d_in; i += blockDim.x) {
+    __shared__ unsigned long long warp_tot[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int64_t R = (d_in + blockDim.x - 1) / blockDim.x;
+    const int64_t i0 = (int64_t)tid * R;
+    const int64_t i1 = i0 + R < d_in ? i0 + R : d_in;
+    unsigned long long mine = 0;
+    for (int64_t i = i0; i < i1; ++i) {
         int c = bits[i];
-        cnt[0] += c == 2; cnt[1] += c == 3; cnt[2] += c == 4;
+        if (c >= 2 && c <= 4) mine += 1ull << (21 * (c - 2));
     }
-    if (threadIdx.x < 3) seg_count[threadIdx.x] = 0;
-    __syncthreads();
+    unsigned long long incl = mine;
 #pragma unroll
-    for (int s = 0; s < 3; ++s) {
-        long long v = cnt[s];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0 && v) atomicAdd((unsigned long long*)&seg_count[s], (unsigned long long)v);
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
     }
+    if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    long long words[3], seg_base[3], seg_word_base[3];
+    unsigned long long base = 0, total = 0;
+    for (int w = 0; w < nwarps; ++w) {
+        unsigned long long t = warp_tot[w];
+        if (w < warp) base += t;
+        total += t;
+    }
+    const unsigned long long before = base + incl - mine;
+    long long seen[3], count[3], words[3], seg_base[3], seg_word_base[3];
     long long rb = 0, wb = 0;
 #pragma unroll
-    for (int s = 0; s < 3; ++s) {
-        words[s] = (d_out * (s + 2) + 31) / 32;
-        seg_base[s] = rb;
-        seg_word_base[s] = wb;
-        rb += seg_count[s];
-        wb += seg_count[s] * words[s];
+    for (int sgm = 0; sgm < 3; ++sgm) {
+        seen[sgm] = (long long)((before >> (21 * sgm)) & 0x1fffffull);
+        count[sgm] = (long long)((total >> (21 * sgm)) & 0x1fffffull);
+        words[sgm] = (d_out * (sgm + 2) + 31) / 32;
+        seg_base[sgm] = rb;
+        seg_word_base[sgm] = wb;
+        rb += count[sgm];
+        wb += count[sgm] * words[sgm];
     }
-    if (threadIdx.x < 3) seg_rows[threadIdx.x] = seg_count[threadIdx.x];
-    if (threadIdx.x == 0) row_off[d_in] = wb;
-    // pass 2: position of every channel among the channels of its width (ascending id)
-    long long seen[3] = {0, 0, 0};
-    for (int64_t base = 0; base < d_in; base += blockDim.x) {
-        int64_t i = base + threadIdx.x;
-        int c = i < d_in ? bits[i] : 0;
-        int excl[3];
-        __syncthreads();
-#pragma unroll
-        for (int s = 0; s < 3; ++s) {
-            unsigned m = __ballot_sync(0xffffffffu, c == s + 2);
-            excl[s] = __popc(m & ((1u << lane) - 1));
-            if (lane == 0) warp_tot[s][warp] = __popc(m);
-        }
-        __syncthreads();
-        long long tot[3] = {0, 0, 0};
-#pragma unroll
-        for (int s = 0; s < 3; ++s) {
-            int before = 0, all = 0;
-            for (int w = 0; w < nwarps; ++w) {
-                int t = warp_tot[s][w];
-                if (w < warp) before += t;
-                all += t;
-            }
-            excl[s] += before;
-            tot[s] = all;
-        }
-        if (i < d_in && c >= 2 && c <= 4) {
-            int s = c - 2;
-            long long pos = seen[s] + excl[s];
-            long long r = seg_base[s] + pos;
-            long long off = seg_word_base[s] + pos * words[s];
-            perm[r] = (int32_t)i;
-            row_off[r] = off;
-            word_off[i] = off;
-        }
-#pragma unroll
-        for (int s = 0; s < 3; ++s) seen[s] += tot[s];
+    if (tid < 3) seg_rows[tid] = count[tid];
+    if (tid == 0) row_off[d_in] = wb;
+    for (int64_t i = i0; i < i1; ++i) {
+        int c = bits[i];
+        if (c < 2 || c > 4) continue;
+        int sgm = c - 2;
+        long long pos = seen[sgm]++;
+        long long r = seg_base[sgm] + pos;
+        long long off = seg_word_base[sgm] + pos * words[sgm];
+        perm[r] = (int32_t)i;
+        row_off[r] = off;
+        word_off[i] = off;
     }
 }
 
-// One thread packs 32 consecutive codes of one channel.
+// Four codes held one per byte -> one 4C-bit field (C bits each, first code lowest).
+template <int C>
+__device__ __forceinline__ uint32_t squeeze4(uint32_t x) {
+    constexpr uint32_t m1 = ((1u << (2 * C)) - 1u) * 0x00010001u;
+    constexpr uint32_t m2 = (C == 4) ? 0xffffu : ((1u << (4 * C)) - 1u);
+    x &= ((1u << C) - 1u) * 0x01010101u;  // ignore anything above the channel's width
+    uint32_t t = (x | (x >> (8 - C))) & m1;
+    return (t | (t >> (16 - 2 * C))) & m2;
+}
+
+template <int C>
+__device__ __forceinline__ void pack32(const uint32_t (&b)[8], uint32_t (&w)[4]) {
+    uint32_t r[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) r[q] = squeeze4<C>(b[q]);
+    if (C == 2) {
+        w[0] = r[0] | (r[1] << 8) | (r[2] << 16) | (r[3] << 24);
+        w[1] = r[4] | (r[5] << 8) | (r[6] << 16) | (r[7] << 24);
+        w[2] = w[3] = 0;
+    } else if (C == 3) {
+        w[0] = r[0] | (r[1] << 12) | (r[2] << 24);
+        w[1] = (r[2] >> 8) | (r[3] << 4) | (r[4] << 16) | (r[5] << 28);
+        w[2] = (r[5] >> 4) | (r[6] << 8) | (r[7] << 20);
+        w[3] = 0;
+    } else {
+        w[0] = r[0] | (r[1] << 16);
+        w[1] = r[2] | (r[3] << 16);
+        w[2] = r[4] | (r[5] << 16);
+        w[3] = r[6] | (r[7] << 16);
+    }
+}
+
+// One thread packs 32 consecutive codes of one channel into C consecutive words.
 __global__ void __launch_bounds__(kPackThreads)
 pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ bits, int64_t d_out,
             const int64_t* __restrict__ word_off, uint32_t* __restrict__ packed, int vec_ok) {
@@ -120,23 +135,12 @@ pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ bits,
             b[q] = w;
         }
     }
-    // 128-bit little-endian bit stream of the 32 codes, c bits each
-    unsigned long long lo = 0, hi = 0;
-    const uint32_t cmask = (1u << c) - 1u;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        unsigned long long code = (b[j >> 2] >> (8 * (j & 3))) & cmask;
-        int pos = j * c;
-        if (pos < 64) {
-            lo |= code << pos;
-            if (pos + c > 64) hi |= code >> (64 - pos);
-        } else {
-            hi |= code << (pos - 64);
-        }
-    }
+    uint32_t w[4];
+    if (c == 2) pack32<2>(b, w);
+    else if (c == 3) pack32<3>(b, w);
+    else pack32<4>(b, w);
     uint32_t* dst = packed + word_off[row] + g * c;
     const int nwords = (cnt * c + 31) / 32;
-    uint32_t w[4] = {(uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32)};
 #pragma unroll
     for (int t = 0; t < 4; ++t)
         if (t < nwords) dst[t] = w[t];

@@ -16,7 +16,7 @@ constexpr int kStatsWarps = kStatsThreads / 32;
 constexpr int kTileCols = 256;       // columns per block: 32 lanes x 8 columns
 constexpr int kFlushRows = 32;       // rows a thread sums in fp32 before folding into fp64
 constexpr int kMaxRowBlocks = 2048;  // upper bound used to size the work space
-constexpr int kCtasPerSm = 8;
+constexpr int kCtasPerSm = 5;       // resident blocks per SM of the vector kernel (48 registers)
 
 int sm_count() {
     int dev = 0, n = 0;
@@ -27,11 +27,11 @@ int sm_count() {
 
 static int64_t col_tiles(int64_t d_in) { return (d_in + kTileCols - 1) / kTileCols; }
 
-// Row blocks per column tile for a device with `sms` SMs: enough blocks to fill every SM
-// kCtasPerSm times, never more than kMaxRowBlocks / col_tiles (work-space bound).
+// Row blocks per column tile for a device with `sms` SMs: as many blocks as are resident at once
+// (one full wave, no tail), never more than kMaxRowBlocks / col_tiles (work-space bound).
 static int64_t row_blocks_for(int64_t d_in, int64_t n_tokens, int sms) {
     int64_t ct = col_tiles(d_in);
-    int64_t want = ((int64_t)sms * kCtasPerSm + ct - 1) / ct;
+    int64_t want = ((int64_t)sms * kCtasPerSm) / ct;
     int64_t cap = kMaxRowBlocks / ct;
     if (cap < 1) cap = 1;
     if (want > cap) want = cap;
@@ -63,21 +63,21 @@ __device__ __forceinline__ void accumulate8(const uint4& v, float (&acc)[8]) {
 }
 
 // partial[(row_block * tiles + tile) * kTileCols + c] = sum over the block's rows of X[t, tile*256+c]^2
+// The fp64 running totals live in shared memory (slot [warp][i][lane] for column lane*8+i: conflict
+// free), which keeps the register count low enough for 5 resident blocks per SM.
 template <int DT>
-__global__ void __launch_bounds__(kStatsThreads)
+__global__ void __launch_bounds__(kStatsThreads, 5)
 stats_partial_vec_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64_t d_in, int64_t ldx,
                          int64_t rows_per_block, double* __restrict__ partial) {
-    __shared__ double red[kStatsWarps][kTileCols];
+    __shared__ double red[kStatsWarps][8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t tile = blockIdx.x;
     const int64_t col = tile * kTileCols + lane * 8;
     const int64_t r0 = (int64_t)blockIdx.y * rows_per_block;
     int64_t r1 = r0 + rows_per_block;
     if (r1 > n_tokens) r1 = n_tokens;
-
-    double total[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) total[i] = 0.0;
+    for (int i = 0; i < 8; ++i) red[warp][i][lane] = 0.0;
 
     if (col < d_in) {
         const uint16_t* p = X + col;
@@ -98,7 +98,7 @@ stats_partial_vec_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64
             since_flush += 4;
             if (since_flush >= kFlushRows) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { total[i] += (double)acc[i]; acc[i] = 0.f; }
+                for (int i = 0; i < 8; ++i) { red[warp][i][lane] += (double)acc[i]; acc[i] = 0.f; }
                 since_flush = 0;
             }
         }
@@ -107,16 +107,14 @@ stats_partial_vec_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64
             accumulate8<DT>(v0, acc);
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) total[i] += (double)acc[i];
+        for (int i = 0; i < 8; ++i) red[warp][i][lane] += (double)acc[i];
     }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) red[warp][lane * 8 + i] = total[i];
     __syncthreads();
     // thread c adds the eight warps' sums of column c in warp order
     const int c = threadIdx.x;
     double s = 0.0;
 #pragma unroll
-    for (int w = 0; w < kStatsWarps; ++w) s += red[w][c];
+    for (int w = 0; w < kStatsWarps; ++w) s += red[w][c & 7][c >> 3];
     partial[((int64_t)blockIdx.y * gridDim.x + tile) * kTileCols + c] = s;
 }
 
