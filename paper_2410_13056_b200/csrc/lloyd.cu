@@ -34,13 +34,12 @@ namespace cmpq {
 
 constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
-constexpr int kMaxThreads = 1024;
 
 struct alignas(16) LloydShared {
-    double pt[kMaxThreads + 1];        // exclusive prefix over threads of the threads' fp64 totals
+    double* pt;                        // [nthr + 1] exclusive prefix over threads of their fp64 totals
     // exchanged once per sweep, double-buffered by sweep parity so that one barrier per sweep is enough
-    double wsum[2][kMaxWarps][kMaxK];  // per-warp cluster sums (rebuild path); [0][w][0]: totals (scan)
-    int wcnt[2][kMaxWarps][kMaxK];     // per-warp cluster counts (rebuild) / threads below boundary k
+    double (*wsum)[kMaxK];             // [2 * nwarps][K] per-warp cluster sums (rebuild path)
+    int (*wcnt)[kMaxK];                // [2 * nwarps][K] per-warp counts (rebuild) / threads below boundary k
     double part_sum[2][kMaxK];         // boundary k inside a thread: sum / count of that thread's
     int part_cnt[2][kMaxK];            //   weights with a code below k
     int hist1[256];
@@ -56,6 +55,8 @@ struct alignas(16) LloydShared {
 //   scratch (lloyd_scratch_bytes): removed-column bitmap during the load, second-level histogram
 //                                  during the sort, then the threads' first code words (2 x 4 B)
 //   sorted  (4 bytes per weight):  key << 16 | column, ascending; reused for the output staging
+
+__host__ __device__ inline size_t lloyd_pt_bytes(int nthr) { return (((size_t)nthr + 1) * sizeof(double) + 15) & ~(size_t)15; }
 
 __host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
     return kMaxK * 256 * (int)sizeof(int);  // 16 KiB >= 16 bytes x 1024 threads >= 32768 bits
@@ -195,7 +196,7 @@ __device__ __forceinline__ bool counting_sweep_valid(float ck_lane, double need)
 template <int K, int E>
 __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 7) / 8], int nval,
                                  LloydShared& sh, int par) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_ = blockDim.x >> 5;
     int code[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) code[e] = (e < nval) ? (int)((cw[e >> 3] >> (4 * (e & 7))) & 15u) : -1;
@@ -211,7 +212,7 @@ __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 
         }
         s = warp_sum(s);
         cnt = warp_sum(cnt);
-        if (lane == 0) { sh.wsum[par][warp][k] = s; sh.wcnt[par][warp][k] = cnt; }
+        if (lane == 0) { sh.wsum[par * nwarps_ + warp][k] = s; sh.wcnt[par * nwarps_ + warp][k] = cnt; }
     }
 }
 
@@ -223,7 +224,7 @@ __device__ __forceinline__ float centroid_from_partials(const LloydShared& sh, i
     if (lane < K) {
         double s = 0.0;
         int cnt = 0;
-        for (int w = 0; w < nwarps; ++w) { s += sh.wsum[par][w][lane]; cnt += sh.wcnt[par][w][lane]; }
+        for (int w = 0; w < nwarps; ++w) { s += sh.wsum[par * nwarps + w][lane]; cnt += sh.wcnt[par * nwarps + w][lane]; }
         if (cnt > 0) ck = __double2float_rn(__ddiv_rn(s, (double)cnt));
     }
     return ck;
@@ -294,7 +295,7 @@ __device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh,
         P = sh.pt[nthr];
     } else if (lane > 0 && lane < K) {
         int t = 0;
-        for (int w = 0; w < nwarps; ++w) t += sh.wcnt[par][w][lane];
+        for (int w = 0; w < nwarps; ++w) t += sh.wcnt[par * nwarps + w][lane];
         B = t * E;
         P = sh.pt[t];
         if (t < nthr && (int)(first_code_s[t] & 15u) < lane) {  // boundary inside thread t
@@ -397,7 +398,7 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
                 if (probe < lane) below += step;
             }
             if (__shfl_sync(0xffffffffu, c_last, 31) < lane) below = 32;
-            if (lane > 0 && lane < K) sh.wcnt[par][warp][lane] = below;
+            if (lane > 0 && lane < K) sh.wcnt[par * (nthr >> 5) + warp][lane] = below;
             if (c_first != c_last) {
                 PackedCodes<E> pc;
 #pragma unroll
@@ -458,18 +459,24 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         atomicAdd(a.sweeps, (unsigned long long)sweeps_done * (unsigned long long)N * (unsigned long long)K);
 }
 
-template <int DT, int E, int MAXT>
-__global__ void __launch_bounds__(MAXT)
+template <int DT, int E, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
 lloyd_kernel(const LloydArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int64_t row = blockIdx.x;
     if (a.skip_row && a.skip_row[row]) return;
     const int N = (int)a.d_out;
     LloydShared& sh = *reinterpret_cast<LloydShared*>(smem_raw);
-    unsigned char* scratch = smem_raw + sizeof(LloydShared);
-    uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = nthr >> 5;
+    unsigned char* scratch = smem_raw + sizeof(LloydShared);
+    uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
+    unsigned char* tail = reinterpret_cast<unsigned char*>(sorted) + (((size_t)N + 3) & ~(size_t)3) * 4;
+    if (tid == 0) {  // published by the first barrier below, long before anyone uses them
+        sh.pt = reinterpret_cast<double*>(tail);
+        sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr));
+        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr) + (size_t)2 * nwarps * kMaxK * sizeof(double));
+    }
 
     // removed positions (outliers of this row) are marked in a bitmap over the columns
     uint32_t* removed = reinterpret_cast<uint32_t*>(scratch);
@@ -584,10 +591,10 @@ lloyd_kernel(const LloydArgs a) {
             double up = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += up;
         }
-        if (lane == 31) sh.wsum[0][warp][0] = incl;
+        if (lane == 31) sh.wsum[warp][0] = incl;
         __syncthreads();
         double base = 0.0;
-        for (int wv = 0; wv < warp; ++wv) base += sh.wsum[0][wv][0];
+        for (int wv = 0; wv < warp; ++wv) base += sh.wsum[wv][0];
         sh.pt[tid] = base + incl - tot;
         if (tid == nthr - 1) sh.pt[nthr] = base + incl;
         __syncthreads();
@@ -600,14 +607,16 @@ lloyd_kernel(const LloydArgs a) {
     else fit_channel<DT, 16, E>(a, row, x, nval, sh, first_code_s, sorted);
 }
 
-static size_t lloyd_smem_bytes(int64_t d_out) {
-    return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4;
+static size_t lloyd_smem_bytes(int64_t d_out, int threads) {
+    const size_t nwarps = (size_t)threads / 32;
+    return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4 +
+           lloyd_pt_bytes(threads) + 2 * nwarps * kMaxK * (sizeof(double) + sizeof(int));
 }
 
-template <int DT, int E, int MAXT>
+template <int DT, int E, int MAXT, int MINB>
 static cmpq_status launch_variant(const LloydArgs& args, int threads, cudaStream_t st) {
-    const size_t smem = lloyd_smem_bytes(args.d_out);
-    auto kern = lloyd_kernel<DT, E, MAXT>;
+    const size_t smem = lloyd_smem_bytes(args.d_out, threads);
+    auto kern = lloyd_kernel<DT, E, MAXT, MINB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
     kern<<<(unsigned)args.d_in, threads, smem, st>>>(args);
@@ -622,9 +631,10 @@ static cmpq_status launch_dt(const LloydArgs& args, cudaStream_t st) {
         t = (t + 31) / 32 * 32;
         return (int)(t < 32 ? 32 : t);
     };
-    if (N <= 2048) return launch_variant<DT, 4, 512>(args, threads_for(4), st);
-    if (N <= 16384) return launch_variant<DT, 16, 1024>(args, threads_for(16), st);
-    return launch_variant<DT, 32, 1024>(args, threads_for(32), st);
+    if (N <= 2048) return launch_variant<DT, 4, 512, 1>(args, threads_for(4), st);
+    if (N <= 4096) return launch_variant<DT, 16, 256, 4>(args, threads_for(16), st);
+    if (N <= 16384) return launch_variant<DT, 16, 1024, 1>(args, threads_for(16), st);
+    return launch_variant<DT, 32, 1024, 1>(args, threads_for(32), st);
 }
 
 cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st) {
