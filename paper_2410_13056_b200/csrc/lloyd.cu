@@ -219,8 +219,8 @@ __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 
 // Rebuild path, every warp for itself: lane k combines the per-warp partials of cluster k and moves
 // the centroid to the mean if the cluster has members.
 template <int K>
-__device__ __forceinline__ float centroid_from_partials(const LloydShared& sh, int par, float ck) {
-    const int lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+__device__ __forceinline__ float centroid_from_partials(const LloydShared& sh, int par, float ck, int nwarps) {
+    const int lane = threadIdx.x & 31;
     if (lane < K) {
         double s = 0.0;
         int cnt = 0;
@@ -286,8 +286,8 @@ __device__ __noinline__ void boundary_partials(PackedCodes<E> cw, int c_first, i
 template <int K, int E>
 __device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh, int par,
                                                           const uint32_t* first_code_s, int N, float ck,
-                                                          int& B_out) {
-    const int lane = threadIdx.x & 31, nwarps = blockDim.x >> 5, nthr = blockDim.x;
+                                                          int& B_out, int nwarps) {
+    const int lane = threadIdx.x & 31, nthr = blockDim.x;
     int B = 0;
     double P = 0.0;
     if (lane == K) {
@@ -314,118 +314,54 @@ __device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh,
     return ck;
 }
 
-template <int DT, int K, int E>
-__device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
-                            LloydShared& sh, uint32_t* first_code_s, uint32_t* sorted) {
-    constexpr int G = E / 4;            // float accumulators: codes of 4 weights each, base 16
-    constexpr int WORDS = (E + 7) / 8;  // packed codes: 8 weights per 32-bit word
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    const int N = (int)a.d_out;
-    const int T = a.iters;
-    const double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
-
-    // Every warp keeps the centroids itself (lane k holds c_k) and repeats the tiny update, so that
-    // a sweep needs a single block-wide barrier.  All warps compute identical values.
-    float ck_lane = 0.f;
-    if (lane < K) {
-        int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
-        ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
-    }
-    bool fast = counting_sweep_valid<K>(ck_lane, need);
-    int B_prev = -1;  // lane k: B_k of the previous ordered sweep (-1: none)
-
-    uint32_t cw[WORDS];
+// One sweep over a thread's E weights: their codes for the centroids c, packed 8 per word.
+template <int K, int E>
+__device__ __forceinline__ void sweep_codes(const float (&x)[E], const float (&c)[K], bool fast,
+                                            uint32_t (&nw)[(E + 7) / 8]) {
+    constexpr int G = E / 4, WORDS = (E + 7) / 8;
+    uint32_t half[G];  // 16 bits: the codes of weights 4g..4g+3
+    if (fast) {
 #pragma unroll
-    for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;
-    float c[K];
-    int sweeps_done = 0;
-    for (int it = 0; it <= T; ++it) {
+        for (int g = 0; g < G; ++g) {
+            // 2^23 + sum code_u 16^u is exact in fp32, so the low mantissa bits are the codes
+            float acc = 8388608.f;
 #pragma unroll
-        for (int k = 0; k < K; ++k) c[k] = __shfl_sync(0xffffffffu, ck_lane, k);
-        const bool last = (it == T);
-        const int par = it & 1;
-
-        uint32_t half[G];  // 16 bits: the codes of weights 4g..4g+3
-        if (fast) {
+            for (int u = 0; u < 4; ++u) {
+                const float xv = x[4 * g + u];
+                const float inc = (float)(1 << (4 * u));
+                float dp = fabsf(xv - c[0]);
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                // 2^23 + sum code_u 16^u is exact in fp32, so the low mantissa bits are the codes
-                float acc = 8388608.f;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float xv = x[4 * g + u];
-                    const float inc = (float)(1 << (4 * u));
-                    float dp = fabsf(xv - c[0]);
-#pragma unroll
-                    for (int k = 1; k < K; ++k) {
-                        float d = fabsf(xv - c[k]);
-                        if (d < dp) acc += inc;
-                        dp = d;
-                    }
+                for (int k = 1; k < K; ++k) {
+                    float d = fabsf(xv - c[k]);
+                    if (d < dp) acc += inc;
+                    dp = d;
                 }
-                half[g] = __float_as_uint(acc);
             }
-        } else {
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                uint32_t p = 0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) p |= (uint32_t)nearest_scan<K>(x[4 * g + u], c) << (4 * u);
-                half[g] = p;
-            }
+            half[g] = __float_as_uint(acc);
         }
-        uint32_t nw[WORDS];
+    } else {
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w)
-            nw[w] = (2 * w + 1 < G) ? __byte_perm(half[2 * w], half[2 * w + 1], 0x5410) : (half[2 * w] & 0xffffu);
-        ++sweeps_done;
-        uint32_t any = 0;
+        for (int g = 0; g < G; ++g) {
+            uint32_t p = 0;
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w) { any |= nw[w] ^ cw[w]; cw[w] = nw[w]; }
-        if (last) break;
-
-        if (fast) {
-            // codes are non-decreasing along the sorted order.  Lane k finds, by bisection over the
-            // lanes' last codes, how many threads of this warp lie entirely below boundary k; a thread
-            // with a boundary in its interior also publishes the sum and count of its weights below it.
-            first_code_s[par * nthr + tid] = cw[0];
-            const int c_first = (int)(cw[0] & 15u);
-            const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
-            int below = 0;
-#pragma unroll
-            for (int step = 16; step > 0; step >>= 1) {
-                int probe = __shfl_sync(0xffffffffu, c_last, below + step - 1);
-                if (probe < lane) below += step;
-            }
-            if (__shfl_sync(0xffffffffu, c_last, 31) < lane) below = 32;
-            if (lane > 0 && lane < K) sh.wcnt[par * (nthr >> 5) + warp][lane] = below;
-            if (c_first != c_last) {
-                PackedCodes<E> pc;
-#pragma unroll
-                for (int w = 0; w < WORDS; ++w) pc.w[w] = cw[w];
-                boundary_partials<DT, E>(pc, c_first, c_last, nval, sorted + tid * E, sh, par);
-            }
-            __syncthreads();
-            int B;
-            ck_lane = centroid_from_boundaries<K, E>(sh, par, first_code_s + par * nthr, N, ck_lane, B);
-            const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
-            B_prev = B;
-            fast = counting_sweep_valid<K>(ck_lane, need);
-            if (!moved) break;  // same decision in every warp
-        } else {
-            const int changed = __syncthreads_or(any != 0);
-            if (!changed) break;
-            rebuild_partials<K, E>(x, cw, nval, sh, par);
-            __syncthreads();
-            ck_lane = centroid_from_partials<K>(sh, par, ck_lane);
-            fast = counting_sweep_valid<K>(ck_lane, need);
-            B_prev = -1;
+            for (int u = 0; u < 4; ++u) p |= (uint32_t)nearest_scan<K>(x[4 * g + u], c) << (4 * u);
+            half[g] = p;
         }
     }
-    if (warp == 0 && lane < K) sh.c[lane] = ck_lane;
-    __syncthreads();  // centroids published; no thread reads keys from `sorted` after this point
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w)
+        nw[w] = (2 * w + 1 < G) ? __byte_perm(half[2 * w], half[2 * w + 1], 0x5410) : (half[2 * w] & 0xffffu);
+}
 
-    // outputs, staged through shared memory back into column order
+// Outputs of one channel, staged through shared memory back into column order.  Called by every
+// thread of the block after a barrier that follows the last read of keys from `sorted`; sh.c holds
+// the final centroids.
+template <int E>
+__device__ void write_outputs(const LloydArgs& a, int64_t row, int K, const LloydShared& sh, uint32_t* sorted,
+                              const float (&x)[E], const uint32_t (&cw)[(E + 7) / 8], int nval,
+                              int sweeps_done) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int N = (int)a.d_out;
     if (a.lut && tid < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + tid] = tid < K ? sh.c[tid] : 0.f;
     uint32_t colv[E];
 #pragma unroll
@@ -459,25 +395,96 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         atomicAdd(a.sweeps, (unsigned long long)sweeps_done * (unsigned long long)N * (unsigned long long)K);
 }
 
-template <int DT, int E, int MAXT, int MINB>
-__global__ void __launch_bounds__(MAXT, MINB)
-lloyd_kernel(const LloydArgs a) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int64_t row = blockIdx.x;
-    if (a.skip_row && a.skip_row[row]) return;
+template <int DT, int K, int E>
+__device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
+                            LloydShared& sh, uint32_t* first_code_s, uint32_t* sorted) {
+    constexpr int WORDS = (E + 7) / 8;  // packed codes: 8 weights per 32-bit word
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int N = (int)a.d_out;
-    LloydShared& sh = *reinterpret_cast<LloydShared*>(smem_raw);
+    const int T = a.iters;
+    const double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+
+    // Every warp keeps the centroids itself (lane k holds c_k) and repeats the tiny update, so that
+    // a sweep needs a single block-wide barrier.  All warps compute identical values.
+    float ck_lane = 0.f;
+    if (lane < K) {
+        int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
+        ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
+    }
+    bool fast = counting_sweep_valid<K>(ck_lane, need);
+    int B_prev = -1;  // lane k: B_k of the previous ordered sweep (-1: none)
+
+    uint32_t cw[WORDS];
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;
+    float c[K];
+    int sweeps_done = 0;
+    for (int it = 0; it <= T; ++it) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) c[k] = __shfl_sync(0xffffffffu, ck_lane, k);
+        const bool last = (it == T);
+        const int par = it & 1;
+
+        uint32_t nw[WORDS];
+        sweep_codes<K, E>(x, c, fast, nw);
+        ++sweeps_done;
+        uint32_t any = 0;
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) { any |= nw[w] ^ cw[w]; cw[w] = nw[w]; }
+        if (last) break;
+
+        if (fast) {
+            // codes are non-decreasing along the sorted order.  Lane k finds, by bisection over the
+            // lanes' last codes, how many threads of this warp lie entirely below boundary k; a thread
+            // with a boundary in its interior also publishes the sum and count of its weights below it.
+            first_code_s[par * nthr + tid] = cw[0];
+            const int c_first = (int)(cw[0] & 15u);
+            const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
+            int below = 0;
+#pragma unroll
+            for (int step = 16; step > 0; step >>= 1) {
+                int probe = __shfl_sync(0xffffffffu, c_last, below + step - 1);
+                if (probe < lane) below += step;
+            }
+            if (__shfl_sync(0xffffffffu, c_last, 31) < lane) below = 32;
+            if (lane > 0 && lane < K) sh.wcnt[par * (nthr >> 5) + warp][lane] = below;
+            if (c_first != c_last) {
+                PackedCodes<E> pc;
+#pragma unroll
+                for (int w = 0; w < WORDS; ++w) pc.w[w] = cw[w];
+                boundary_partials<DT, E>(pc, c_first, c_last, nval, sorted + tid * E, sh, par);
+            }
+            __syncthreads();
+            int B;
+            ck_lane = centroid_from_boundaries<K, E>(sh, par, first_code_s + par * nthr, N, ck_lane, B, nthr >> 5);
+            const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
+            B_prev = B;
+            fast = counting_sweep_valid<K>(ck_lane, need);
+            if (!moved) break;  // same decision in every warp
+        } else {
+            const int changed = __syncthreads_or(any != 0);
+            if (!changed) break;
+            rebuild_partials<K, E>(x, cw, nval, sh, par);
+            __syncthreads();
+            ck_lane = centroid_from_partials<K>(sh, par, ck_lane, nthr >> 5);
+            fast = counting_sweep_valid<K>(ck_lane, need);
+            B_prev = -1;
+        }
+    }
+    if (warp == 0 && lane < K) sh.c[lane] = ck_lane;
+    __syncthreads();  // centroids published; no thread reads keys from `sorted` after this point
+    write_outputs<E>(a, row, K, sh, sorted, x, cw, nval, sweeps_done);
+}
+
+// One-time work for a channel, by every thread of the block: read the row, zero the removed
+// positions, note the value range and the exactness diagnostics, sort it into `sorted`, load this
+// thread's run of E order statistics into x and scan the threads' fp64 totals into sh.pt.
+template <int DT, int E>
+__device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh, unsigned char* scratch,
+                                uint32_t* sorted, float (&x)[E], int& nval_out) {
+    const int N = (int)a.d_out;
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = nthr >> 5;
-    unsigned char* scratch = smem_raw + sizeof(LloydShared);
-    uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
-    unsigned char* tail = reinterpret_cast<unsigned char*>(sorted) + (((size_t)N + 3) & ~(size_t)3) * 4;
-    if (tid == 0) {  // published by the first barrier below, long before anyone uses them
-        sh.pt = reinterpret_cast<double*>(tail);
-        sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr));
-        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr) + (size_t)2 * nwarps * kMaxK * sizeof(double));
-    }
-
     // removed positions (outliers of this row) are marked in a bitmap over the columns
     uint32_t* removed = reinterpret_cast<uint32_t*>(scratch);
     int64_t p0 = 0, p1 = 0;
@@ -569,7 +576,6 @@ lloyd_kernel(const LloydArgs a) {
     sort_channel<E>(key, nval_cols, sh, reinterpret_cast<int*>(scratch), sorted);
 
     // sorted layout: thread t keeps order statistics [E t, E t + E); padding repeats the maximum
-    float x[E];
     int nval = N - tid * E;
     nval = nval < 0 ? 0 : (nval > E ? E : nval);
     {
@@ -599,6 +605,32 @@ lloyd_kernel(const LloydArgs a) {
         if (tid == nthr - 1) sh.pt[nthr] = base + incl;
         __syncthreads();
     }
+
+    nval_out = nval;
+}
+
+template <int DT, int E, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
+lloyd_kernel(const LloydArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int64_t row = blockIdx.x;
+    if (a.skip_row && a.skip_row[row]) return;
+    const int N = (int)a.d_out;
+    LloydShared& sh = *reinterpret_cast<LloydShared*>(smem_raw);
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int nwarps = nthr >> 5;
+    unsigned char* scratch = smem_raw + sizeof(LloydShared);
+    uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
+    unsigned char* tail = reinterpret_cast<unsigned char*>(sorted) + (((size_t)N + 3) & ~(size_t)3) * 4;
+    if (tid == 0) {  // published by the first barrier below, long before anyone uses them
+        sh.pt = reinterpret_cast<double*>(tail);
+        sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr));
+        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr) + (size_t)2 * nwarps * kMaxK * sizeof(double));
+    }
+
+    float x[E];
+    int nval;
+    prepare_channel<DT, E>(a, row, sh, scratch, sorted, x, nval);
 
     uint32_t* first_code_s = reinterpret_cast<uint32_t*>(scratch);
     const int bits = a.bits[row];
