@@ -81,31 +81,34 @@ def test_midsize_layer_all_budgets(b):
     assert abs(g["bits"].mean() - b) <= 0.5 / d_in or b == 3.0
 
 
-def test_llama_attention_shape_sampled_parity():
-    """The benchmark's workload (4096 x 4096 bf16, 131072 tokens, 2.2 bits, 20 iterations) in the
-    launch configuration the benchmark uses; the checker verifies sampled channels and global
-    properties instead of re-running everything."""
-    cfg = inputs.CONFIGS["c2_attn7b"]
-    L = cfg.layers[0]
-    b, T = cfg.budgets[0], cfg.lloyd_iters
-    W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, cfg.seed, device="cuda")
-    X = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, cfg.seed, device="cuda")
-    q = LayerQuantizer(L.d_in, L.d_out)
+def _sampled_parity(cfg_name, layer_index, b):
+    """One full-size layer through the quantizer in the launch configuration the benchmark uses; the
+    checker verifies sampled channels and properties that hold at any size instead of re-running
+    everything (a full single-threaded run would take minutes)."""
+    cfg = inputs.CONFIGS[cfg_name]
+    L = cfg.layers[layer_index]
+    T = cfg.lloyd_iters
+    d_in, d_out = L.d_in, L.d_out
+    seed = inputs.layer_seed(cfg, layer_index)
+    W = inputs.make_weight(d_in, d_out, cfg.dtype, seed, device="cuda")
+    X = inputs.make_activations(cfg.n_tokens, d_in, cfg.dtype, seed, device="cuda")
+    q = LayerQuantizer(d_in, d_out)
     r = q.run(X, W, b, T)
     g = _np(r)
     assert int(q.counters[0].item()) == 0
+    assert (q.n_act, q.n_q) == oracle.default_counts(d_in, d_out)
     # statistic: sampled columns against the checker (fp64, token order)
-    colsel = np.array([0, 1, 7, 8, 255, 256, 1000, 2047, 4095] + list(np.argsort(g["a"])[-4:]))
+    colsel = np.unique(np.array([0, 1, 7, 8, 255, 256, d_in // 2, d_in - 1] + list(np.argsort(g["a"])[-4:])))
     Xs = X[:, torch.from_numpy(colsel).cuda()].contiguous()
     a_ref = oracle.finalize_stats(oracle.collect_stats(inputs.as_u16(Xs), cfg.dtype))
     np.testing.assert_allclose(g["a"][colsel], a_ref, rtol=1e-5)
+    del X, Xs
     # allocation: exact, from the GPU statistic
     bits_ref, order_ref = oracle.allocate_bits(g["a"], b)
     assert np.array_equal(g["bits"], bits_ref)
-    assert (g["bits"] == 2).sum() == 3277 and (g["bits"] == 4).sum() == 0
+    n2, n4 = oracle.alloc_counts(d_in, b)
+    assert (g["bits"] == 2).sum() == n2 and (g["bits"] == 4).sum() == n4
     # outlier list: structure and O_act rows
-    d_in, d_out = L.d_in, L.d_out
-    assert (q.n_act, q.n_q, q.nnz) == (18, 8388, 82116)
     lin = g["rows"].astype(np.int64) * d_out + g["cols"]
     assert np.all(np.diff(lin) > 0)
     Wu = inputs.as_u16(W)
@@ -115,32 +118,59 @@ def test_llama_attention_shape_sampled_parity():
     assert np.array_equal(np.flatnonzero(per_row == d_out), act_rows)
     assert per_row[per_row < d_out].sum() == q.n_q
     # O_q: the provisional fit of sampled rows reproduces exactly the entries taken in those rows,
-    # and no error left behind in a sampled row exceeds the smallest error taken anywhere sampled
-    is_act = np.zeros(d_in, bool); is_act[act_rows] = True
-    sample = [i for i in (0, 1, 17, 511, 2048, 4095, int(np.argmax(per_row * ~is_act))) if not is_act[i]]
-    Wf = W.float().cpu().numpy()
+    # and no error left behind in a sampled row exceeds the smallest error taken in any sampled row
+    is_act = np.zeros(d_in, bool)
+    is_act[act_rows] = True
+    sample = [i for i in (0, 1, 17, d_in // 8, d_in // 2, d_in - 1, int(np.argmax(per_row * ~is_act))) if not is_act[i]]
     taken_min, left_max = np.inf, 0.0
     for i in sample:
-        _, _, err = oracle.lloyd(Wf[i], 1 << int(bits_ref[i]), T)
-        mine = g["cols"][g["rows"] == i]
-        mask = np.zeros(d_out, bool); mask[mine] = True
+        xi = W[i].float().cpu().numpy()
+        _, _, err = oracle.lloyd(xi, 1 << int(bits_ref[i]), T)
+        mask = np.zeros(d_out, bool)
+        mask[g["cols"][g["rows"] == i]] = True
         if mask.any():
             taken_min = min(taken_min, err[mask].min())
-        left_max = max(left_max, err[~mask].max())
-        if mask.any() and (~mask).any():
             assert err[mask].min() >= err[~mask].max()
+        left_max = max(left_max, err[~mask].max())
     assert left_max <= taken_min
-    # final fit: sampled channels (all widths present, an O_act row, the row with most O_q entries)
-    sample2 = sample + [int(act_rows[0]), int(np.flatnonzero(bits_ref == 3)[0]), int(np.flatnonzero(bits_ref == 2)[-1])]
+    # final fit: sampled channels (every width present, an O_act row, the row with most O_q entries)
+    sample2 = sample + [int(act_rows[0])] + [int(np.flatnonzero(bits_ref == c)[k]) for c in (2, 3, 4)
+                                              for k in (0, -1) if (bits_ref == c).any()]
     for i in sample2:
-        x = Wf[i].copy()
-        x[g["cols"][g["rows"] == i]] = 0
-        lut, code, _ = oracle.lloyd(x, 1 << int(bits_ref[i]), T)
+        xi = W[i].float().cpu().numpy()
+        xi[g["cols"][g["rows"] == i]] = 0
+        lut, code, _ = oracle.lloyd(xi, 1 << int(bits_ref[i]), T)
         assert np.array_equal(code, g["codes"][i]), i
         np.testing.assert_allclose(g["lut"][i], lut, rtol=1e-4)
-    assert g["codes"].max() < 8 and np.all(g["codes"][bits_ref == 2] < 4)
-    # packing: full comparison against the checker's packer (cheap), 4 613 632 bytes at 2.2 bits
+        assert np.array_equal(g["lut"][i].view(np.uint32), lut.view(np.uint32)), i
+    assert np.all(g["codes"] < (1 << g["bits"].astype(np.int64))[:, None])
+    # packing: full comparison against the checker's packer
     packed, row_off, perm, seg = oracle.pack(g["codes"], g["bits"])
     assert np.array_equal(g["packed"], packed) and np.array_equal(g["row_off"], row_off)
     assert np.array_equal(g["perm"], perm) and np.array_equal(g["seg_rows"], seg)
-    assert g["packed"].nbytes == 4613632
+    return g, q
+
+
+def test_llama_attention_shape_sampled_parity():
+    """The benchmark's workload shape (4096 x 4096 bf16, 131072 tokens, 20 iterations) at its own 2.2-bit
+    budget and at the metric's 3.0 bits."""
+    g, q = _sampled_parity("c2_attn7b", 0, 2.2)
+    assert (q.n_act, q.n_q, q.nnz) == (18, 8388, 82116)
+    assert (g["bits"] == 2).sum() == 3277 and g["packed"].nbytes == 4613632
+    g, q = _sampled_parity("c2_attn7b", 0, 3.0)
+    assert g["packed"].nbytes == 4096 * 4096 * 3 // 8
+
+
+@pytest.mark.parametrize("layer_index,b", [(0, 2.5), (1, 3.5)])
+def test_llama_mlp_shapes_sampled_parity(layer_index, b):
+    """4096 x 11008 (up) and 11008 x 4096 (down) with 131072 calibration tokens."""
+    g, q = _sampled_parity("c3_mlp7b", layer_index, b)
+    assert q.nnz == (220688 if layer_index == 0 else 223248)
+
+
+@pytest.mark.parametrize("layer_index", [0, 1])
+def test_llama70b_mlp_shapes_sampled_parity(layer_index):
+    """8192 x 28672 and 28672 x 8192 with 65536 calibration tokens at 2.5 bits."""
+    g, q = _sampled_parity("c5_mlp70b", layer_index, 2.5)
+    assert q.nnz == (1149632 if layer_index == 0 else 1174208)
+    assert g["packed"].nbytes == 8192 * 28672 * 5 // 16
