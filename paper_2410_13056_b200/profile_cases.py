@@ -4,6 +4,9 @@
     python -m paper_2410_13056_b200.profile_cases stats --tokens 32768 --d-in 4096 --launches 3
     python -m paper_2410_13056_b200.profile_cases pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
     python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
+    python -m paper_2410_13056_b200.profile_cases layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
+
+`layer` runs the whole pass on one layer of a named workload and prints the time per C-ABI call.
 
 Each case prints the mean CUDA-event time per call; every run holds well under 1 GB on the device.
 """
@@ -15,9 +18,42 @@ from . import binding as B
 from . import inputs
 
 
+def run_layer(a):
+    from .pipeline import LayerQuantizer
+
+    cfg = inputs.CONFIGS[a.config]
+    L = cfg.layers[a.layer]
+    seed = inputs.layer_seed(cfg, a.layer)
+    W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, seed, device="cuda")
+    X = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, seed, device="cuda")
+    q = LayerQuantizer(L.d_in, L.d_out)
+    for _ in range(2):
+        q.run(X, W, a.budget, cfg.lloyd_iters)
+    torch.cuda.synchronize()
+    evs = [dict() for _ in range(a.launches)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(a.launches):
+        q.run(X, W, a.budget, cfg.lloyd_iters, events=evs[i])
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / a.launches
+    params = L.d_in * L.d_out
+    print("layer %s[%d] d_in=%d d_out=%d tokens=%d budget=%.2f T=%d: %.3f ms per pass, %.0f Mparams/s"
+          % (a.config, a.layer, L.d_in, L.d_out, cfg.n_tokens, a.budget, cfg.lloyd_iters, ms, params / ms / 1e3))
+    for name in evs[0]:
+        t = sum(e[name][0].elapsed_time(e[name][1]) for e in evs) / a.launches
+        print("   %-24s %.3f ms" % (name, t))
+    print("   final-fit distance evaluations: %d, inexact rows: %d"
+          % (int(q.counters[1].item()), int(q.counters[0].item() & 0xffffffff)))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers"])
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "layer"])
+    ap.add_argument("--config", default="c2_attn7b")
+    ap.add_argument("--layer", type=int, default=0)
+    ap.add_argument("--budget", type=float, default=3.0)
     ap.add_argument("--d-in", type=int, default=1184)
     ap.add_argument("--d-out", type=int, default=4096)
     ap.add_argument("--tokens", type=int, default=32768)
@@ -28,6 +64,9 @@ def main():
     a = ap.parse_args()
     dt = inputs.BF16 if a.dtype == "bf16" else inputs.F16
     torch.cuda.set_device(0)
+    if a.case == "layer":
+        run_layer(a)
+        return
     d_in, d_out = a.d_in, a.d_out
     bits = torch.full((d_in,), a.bits, dtype=torch.uint8, device="cuda")
 
