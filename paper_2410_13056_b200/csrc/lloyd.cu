@@ -30,22 +30,27 @@
 //               with coalesced writes
 #include "lloyd.cuh"
 
+#ifndef CMPQ_SINGLE_WARP_UPDATE
+#define CMPQ_SINGLE_WARP_UPDATE 0
+#endif
+
 namespace cmpq {
 
 constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
+constexpr bool kSingleWarpUpdate = CMPQ_SINGLE_WARP_UPDATE;  // ordered path: warp 0 updates, second barrier
 
 struct alignas(16) LloydShared {
-    double* pt;                        // [nthr + 1] exclusive prefix over threads of their fp64 totals
+    double* pt4;                       // [nthr E / 4 + 1] fp64 sum of the first 4 i sorted weights
     // exchanged once per sweep, double-buffered by sweep parity so that one barrier per sweep is enough
     double (*wsum)[kMaxK];             // [2 * nwarps][K] per-warp cluster sums (rebuild path)
     int (*wcnt)[kMaxK];                // [2 * nwarps][K] per-warp counts (rebuild) / threads below boundary k
-    double part_sum[2][kMaxK];         // boundary k inside a thread: sum / count of that thread's
-    int part_cnt[2][kMaxK];            //   weights with a code below k
+    int part_cnt[2][kMaxK];            // boundary k inside a thread: that thread's weights with a code below k
     int hist1[256];
     int excl1[257];
     int bucket_rank[256];              // rank of a high-byte bucket among the non-empty ones, or -1
-    float c[kMaxK];                    // final centroids (for the outputs)
+    float c[kMaxK];                    // centroids (single-warp update; final ones for the outputs)
+    int flag_fast, flag_moved;         // single-warp update: decisions of warp 0
     int n_nonempty;
     float vmin, vmax;                  // value range of the channel
     float wlo[kMaxWarps], whi[kMaxWarps];
@@ -56,7 +61,7 @@ struct alignas(16) LloydShared {
 //                                  during the sort, then the threads' first code words (2 x 4 B)
 //   sorted  (4 bytes per weight):  key << 16 | column, ascending; reused for the output staging
 
-__host__ __device__ inline size_t lloyd_pt_bytes(int nthr) { return (((size_t)nthr + 1) * sizeof(double) + 15) & ~(size_t)15; }
+__host__ __device__ inline size_t lloyd_pt_bytes(int nthr, int E) { return (((size_t)nthr * E / 4 + 1) * sizeof(double) + 15) & ~(size_t)15; }
 
 __host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
     return kMaxK * 256 * (int)sizeof(int);  // 16 KiB >= 16 bytes x 1024 threads >= 32768 bits
@@ -250,59 +255,35 @@ __device__ __forceinline__ int count_below(const PackedCodes<E>& pc, int k) {
     return 8 * WORDS - ge - (8 * WORDS - E);
 }
 
-// A thread whose codes differ holds boundaries c_first < k <= c_last in its interior.  For each it
-// publishes how many of its weights lie below the boundary and their fp64 sum (the shorter side
-// is added up; the other side follows from the thread's total).  `mine` = the thread's sorted run.
-template <int DT, int E>
-__device__ __noinline__ void boundary_partials(PackedCodes<E> cw, int c_first, int c_last, int nval,
-                                               const uint32_t* mine, LloydShared& sh, int par) {
-    const int tid = threadIdx.x;
-#pragma unroll 1
-    for (int k = c_first + 1; k <= c_last; ++k) {
-        const int q = count_below<E>(cw, k);
-        double s0 = 0.0, s1 = 0.0;
-        const bool low_side = 2 * q <= nval;
-        const int e0 = low_side ? 0 : q, e1 = low_side ? q : nval;
-        int e = e0;
-#pragma unroll 1
-        for (; e + 1 < e1; e += 2) {
-            s0 += (double)value_of_key16<DT>(mine[e] >> 16);
-            s1 += (double)value_of_key16<DT>(mine[e + 1] >> 16);
-        }
-        if (e < e1) s0 += (double)value_of_key16<DT>(mine[e] >> 16);
-        double s = s0 + s1;
-        if (!low_side) s = (sh.pt[tid + 1] - sh.pt[tid]) - s;
-        sh.part_sum[par][k] = s;
-        sh.part_cnt[par][k] = q;
-    }
-}
-
-// Ordered path, every warp for itself: lane k (0..K) evaluates B_k = number of weights with a code
-// below k and the fp64 sum P_k of those weights; cluster k is the run [B_k, B_{k+1}).
-//   sh.wcnt[par][w][k]  = threads of warp w whose last code is < k  (k = 1..K-1)
-//   first_code_s[t]     = packed codes of thread t's first eight weights
-//   sh.part_*[par][k]   = written this sweep by the thread that holds boundary k in its interior
+// Ordered path: lane k (0..K) evaluates B_k = number of weights with a code below k and the fp64
+// sum P_k of those weights (prefix table at every fourth weight plus at most three weights read from
+// the sorted array); cluster k is the run [B_k, B_{k+1}).
+//   sh.wcnt[par][w][k]   = threads of warp w whose last code is < k  (k = 1..K-1)
+//   first_code_s[t]      = packed codes of thread t's first eight weights
+//   sh.part_cnt[par][k]  = written this sweep by the thread that holds boundary k in its interior
 // Returns the new centroid of cluster `lane` (the old one if the cluster is empty); B_out = B_lane.
-template <int K, int E>
+template <int DT, int K, int E>
 __device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh, int par,
-                                                          const uint32_t* first_code_s, int N, float ck,
-                                                          int& B_out, int nwarps) {
+                                                          const uint32_t* first_code_s, const uint32_t* sorted,
+                                                          int N, float ck, int& B_out, int nwarps) {
     const int lane = threadIdx.x & 31, nthr = blockDim.x;
     int B = 0;
-    double P = 0.0;
     if (lane == K) {
         B = N;
-        P = sh.pt[nthr];
     } else if (lane > 0 && lane < K) {
         int t = 0;
         for (int w = 0; w < nwarps; ++w) t += sh.wcnt[par * nwarps + w][lane];
         B = t * E;
-        P = sh.pt[t];
-        if (t < nthr && (int)(first_code_s[t] & 15u) < lane) {  // boundary inside thread t
-            B += sh.part_cnt[par][lane];
-            P += sh.part_sum[par][lane];
-        }
-        if (B >= N) { B = N; P = sh.pt[nthr]; }
+        if (t < nthr && (int)(first_code_s[t] & 15u) < lane) B += sh.part_cnt[par][lane];  // inside thread t
+        if (B > N) B = N;
+    }
+    double P = 0.0;
+    if (lane <= K) {
+        const int q = B >> 2, r = B & 3;
+        P = sh.pt4[q];
+#pragma unroll
+        for (int e = 0; e < 3; ++e)
+            if (e < r) P += (double)value_of_key16<DT>(sorted[4 * q + e] >> 16);
     }
     const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
     const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
@@ -440,27 +421,48 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
             first_code_s[par * nthr + tid] = cw[0];
             const int c_first = (int)(cw[0] & 15u);
             const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
-            int below = 0;
-#pragma unroll
-            for (int step = 16; step > 0; step >>= 1) {
-                int probe = __shfl_sync(0xffffffffu, c_last, below + step - 1);
-                if (probe < lane) below += step;
+            // lane k: how many threads of this warp lie entirely below boundary k.  The last codes are
+            // non-decreasing along the lanes: everything below the first lane's code counts 0, everything
+            // above the last lane's code counts 32, and a lane whose successor has a larger code owns the
+            // boundaries in between
+            {
+                const int c0 = __shfl_sync(0xffffffffu, c_last, 0), c31 = __shfl_sync(0xffffffffu, c_last, 31);
+                const int c_next = __shfl_down_sync(0xffffffffu, c_last, 1);
+                int* cnt_row = sh.wcnt[par * (nthr >> 5) + warp];
+                if (lane > 0 && lane < K) {
+                    if (lane <= c0) cnt_row[lane] = 0;
+                    else if (lane > c31) cnt_row[lane] = 32;
+                }
+                if (lane < 31 && c_next > c_last)
+                    for (int k = c_last + 1; k <= c_next; ++k) cnt_row[k] = lane + 1;
             }
-            if (__shfl_sync(0xffffffffu, c_last, 31) < lane) below = 32;
-            if (lane > 0 && lane < K) sh.wcnt[par * (nthr >> 5) + warp][lane] = below;
-            if (c_first != c_last) {
+            if (c_first != c_last) {  // boundaries inside this thread: its weights below each of them
                 PackedCodes<E> pc;
 #pragma unroll
                 for (int w = 0; w < WORDS; ++w) pc.w[w] = cw[w];
-                boundary_partials<DT, E>(pc, c_first, c_last, nval, sorted + tid * E, sh, par);
+                for (int k = c_first + 1; k <= c_last; ++k) sh.part_cnt[par][k] = count_below<E>(pc, k);
             }
             __syncthreads();
-            int B;
-            ck_lane = centroid_from_boundaries<K, E>(sh, par, first_code_s + par * nthr, N, ck_lane, B, nthr >> 5);
-            const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
-            B_prev = B;
-            fast = counting_sweep_valid<K>(ck_lane, need);
-            if (!moved) break;  // same decision in every warp
+            if (!kSingleWarpUpdate || warp == 0) {
+                int B;
+                ck_lane = centroid_from_boundaries<DT, K, E>(sh, par, first_code_s + par * nthr, sorted, N, ck_lane,
+                                                             B, nthr >> 5);
+                const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
+                B_prev = B;
+                fast = counting_sweep_valid<K>(ck_lane, need);
+                if (kSingleWarpUpdate) {
+                    if (lane < K) sh.c[lane] = ck_lane;
+                    if (lane == 0) { sh.flag_fast = fast ? 1 : 0; sh.flag_moved = moved ? 1 : 0; }
+                } else if (!moved) {
+                    break;  // same decision in every warp
+                }
+            }
+            if (kSingleWarpUpdate) {
+                __syncthreads();
+                if (lane < K) ck_lane = sh.c[lane];
+                fast = sh.flag_fast != 0;
+                if (!sh.flag_moved) break;
+            }
         } else {
             const int changed = __syncthreads_or(any != 0);
             if (!changed) break;
@@ -478,7 +480,7 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
 
 // One-time work for a channel, by every thread of the block: read the row, zero the removed
 // positions, note the value range and the exactness diagnostics, sort it into `sorted`, load this
-// thread's run of E order statistics into x and scan the threads' fp64 totals into sh.pt.
+// thread's run of E order statistics into x and build the fp64 prefix table sh.pt4.
 template <int DT, int E>
 __device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh, unsigned char* scratch,
                                 uint32_t* sorted, float (&x)[E], int& nval_out) {
@@ -590,7 +592,7 @@ __device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh
                 x[e] = vlast;
             }
         }
-        // exclusive scan of the thread totals over the block
+        // exclusive scan of the thread totals over the block, then the table at every fourth weight
         double incl = tot;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -599,10 +601,16 @@ __device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh
         }
         if (lane == 31) sh.wsum[warp][0] = incl;
         __syncthreads();
-        double base = 0.0;
-        for (int wv = 0; wv < warp; ++wv) base += sh.wsum[wv][0];
-        sh.pt[tid] = base + incl - tot;
-        if (tid == nthr - 1) sh.pt[nthr] = base + incl;
+        double run = incl - tot;
+        for (int wv = 0; wv < warp; ++wv) run += sh.wsum[wv][0];
+#pragma unroll
+        for (int g = 0; g < E / 4; ++g) {
+            sh.pt4[tid * (E / 4) + g] = run;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (4 * g + u < nval) run += (double)x[4 * g + u];
+        }
+        if (tid == nthr - 1) sh.pt4[nthr * (E / 4)] = run;
         __syncthreads();
     }
 
@@ -623,9 +631,9 @@ lloyd_kernel(const LloydArgs a) {
     uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
     unsigned char* tail = reinterpret_cast<unsigned char*>(sorted) + (((size_t)N + 3) & ~(size_t)3) * 4;
     if (tid == 0) {  // published by the first barrier below, long before anyone uses them
-        sh.pt = reinterpret_cast<double*>(tail);
-        sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr));
-        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr) + (size_t)2 * nwarps * kMaxK * sizeof(double));
+        sh.pt4 = reinterpret_cast<double*>(tail);
+        sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr, E));
+        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr, E) + (size_t)2 * nwarps * kMaxK * sizeof(double));
     }
 
     float x[E];
@@ -639,15 +647,15 @@ lloyd_kernel(const LloydArgs a) {
     else fit_channel<DT, 16, E>(a, row, x, nval, sh, first_code_s, sorted);
 }
 
-static size_t lloyd_smem_bytes(int64_t d_out, int threads) {
+static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
     const size_t nwarps = (size_t)threads / 32;
     return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4 +
-           lloyd_pt_bytes(threads) + 2 * nwarps * kMaxK * (sizeof(double) + sizeof(int));
+           lloyd_pt_bytes(threads, E) + 2 * nwarps * kMaxK * (sizeof(double) + sizeof(int));
 }
 
 template <int DT, int E, int MAXT, int MINB>
 static cmpq_status launch_variant(const LloydArgs& args, int threads, cudaStream_t st) {
-    const size_t smem = lloyd_smem_bytes(args.d_out, threads);
+    const size_t smem = lloyd_smem_bytes(args.d_out, threads, E);
     auto kern = lloyd_kernel<DT, E, MAXT, MINB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
