@@ -30,27 +30,20 @@
 //               with coalesced writes
 #include "lloyd.cuh"
 
-#ifndef CMPQ_SINGLE_WARP_UPDATE
-#define CMPQ_SINGLE_WARP_UPDATE 0
-#endif
-
 namespace cmpq {
 
 constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
-constexpr bool kSingleWarpUpdate = CMPQ_SINGLE_WARP_UPDATE;  // ordered path: warp 0 updates, second barrier
 
 struct alignas(16) LloydShared {
     double* pt4;                       // [nthr E / 4 + 1] fp64 sum of the first 4 i sorted weights
-    // exchanged once per sweep, double-buffered by sweep parity so that one barrier per sweep is enough
-    double (*wsum)[kMaxK];             // [2 * nwarps][K] per-warp cluster sums (rebuild path)
-    int (*wcnt)[kMaxK];                // [2 * nwarps][K] per-warp counts (rebuild) / threads below boundary k
-    int part_cnt[2][kMaxK];            // boundary k inside a thread: that thread's weights with a code below k
+    double (*wsum)[kMaxK];             // [nwarps][K] per-warp cluster sums (rebuild path)
+    int (*wcnt)[kMaxK];                // [nwarps][K] per-warp counts (rebuild) / threads below boundary k
     int hist1[256];
     int excl1[257];
     int bucket_rank[256];              // rank of a high-byte bucket among the non-empty ones, or -1
-    float c[kMaxK];                    // centroids (single-warp update; final ones for the outputs)
-    int flag_fast, flag_moved;         // single-warp update: decisions of warp 0
+    float c[kMaxK];                    // centroids for the next sweep, written by warp 0
+    int flag_fast, flag_moved;         // warp 0's decisions: counting sweep valid / a boundary moved
     int n_nonempty;
     float vmin, vmax;                  // value range of the channel
     float wlo[kMaxWarps], whi[kMaxWarps];
@@ -58,7 +51,7 @@ struct alignas(16) LloydShared {
 };
 // dynamic shared memory after LloydShared:
 //   scratch (lloyd_scratch_bytes): removed-column bitmap during the load, second-level histogram
-//                                  during the sort, then the threads' first code words (2 x 4 B)
+//                                  during the sort, then the threads' packed codes
 //   sorted  (4 bytes per weight):  key << 16 | column, ascending; reused for the output staging
 
 __host__ __device__ inline size_t lloyd_pt_bytes(int nthr, int E) { return (((size_t)nthr * E / 4 + 1) * sizeof(double) + 15) & ~(size_t)15; }
@@ -200,8 +193,8 @@ __device__ __forceinline__ bool counting_sweep_valid(float ck_lane, double need)
 // Per-warp cluster sums and counts of all weights, from the codes in registers (any order).
 template <int K, int E>
 __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 7) / 8], int nval,
-                                 LloydShared& sh, int par) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_ = blockDim.x >> 5;
+                                 LloydShared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int code[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) code[e] = (e < nval) ? (int)((cw[e >> 3] >> (4 * (e & 7))) & 15u) : -1;
@@ -217,19 +210,19 @@ __device__ void rebuild_partials(const float (&x)[E], const uint32_t (&cw)[(E + 
         }
         s = warp_sum(s);
         cnt = warp_sum(cnt);
-        if (lane == 0) { sh.wsum[par * nwarps_ + warp][k] = s; sh.wcnt[par * nwarps_ + warp][k] = cnt; }
+        if (lane == 0) { sh.wsum[warp][k] = s; sh.wcnt[warp][k] = cnt; }
     }
 }
 
-// Rebuild path, every warp for itself: lane k combines the per-warp partials of cluster k and moves
+// Rebuild path, warp 0: lane k combines the per-warp partials of cluster k and moves
 // the centroid to the mean if the cluster has members.
 template <int K>
-__device__ __forceinline__ float centroid_from_partials(const LloydShared& sh, int par, float ck, int nwarps) {
+__device__ __forceinline__ float centroid_from_partials(const LloydShared& sh, float ck, int nwarps) {
     const int lane = threadIdx.x & 31;
     if (lane < K) {
         double s = 0.0;
         int cnt = 0;
-        for (int w = 0; w < nwarps; ++w) { s += sh.wsum[par * nwarps + w][lane]; cnt += sh.wcnt[par * nwarps + w][lane]; }
+        for (int w = 0; w < nwarps; ++w) { s += sh.wsum[w][lane]; cnt += sh.wcnt[w][lane]; }
         if (cnt > 0) ck = __double2float_rn(__ddiv_rn(s, (double)cnt));
     }
     return ck;
@@ -255,26 +248,31 @@ __device__ __forceinline__ int count_below(const PackedCodes<E>& pc, int k) {
     return 8 * WORDS - ge - (8 * WORDS - E);
 }
 
-// Ordered path: lane k (0..K) evaluates B_k = number of weights with a code below k and the fp64
-// sum P_k of those weights (prefix table at every fourth weight plus at most three weights read from
-// the sorted array); cluster k is the run [B_k, B_{k+1}).
-//   sh.wcnt[par][w][k]   = threads of warp w whose last code is < k  (k = 1..K-1)
-//   first_code_s[t]      = packed codes of thread t's first eight weights
-//   sh.part_cnt[par][k]  = written this sweep by the thread that holds boundary k in its interior
+// Ordered path, warp 0: lane k (0..K) evaluates B_k = number of weights with a code below k and the
+// fp64 sum P_k of those weights (prefix table at every fourth weight plus at most three weights read
+// from the sorted array); cluster k is the run [B_k, B_{k+1}).
+//   sh.wcnt[w][k]  = threads of warp w whose last code is < k  (k = 1..K-1)
+//   codes_s[t]     = packed codes of thread t
 // Returns the new centroid of cluster `lane` (the old one if the cluster is empty); B_out = B_lane.
 template <int DT, int K, int E>
-__device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh, int par,
-                                                          const uint32_t* first_code_s, const uint32_t* sorted,
-                                                          int N, float ck, int& B_out, int nwarps) {
+__device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh, const uint32_t* codes_s,
+                                                          const uint32_t* sorted, int N, float ck, int& B_out,
+                                                          int nwarps) {
+    constexpr int WORDS = (E + 7) / 8;
     const int lane = threadIdx.x & 31, nthr = blockDim.x;
     int B = 0;
     if (lane == K) {
         B = N;
     } else if (lane > 0 && lane < K) {
         int t = 0;
-        for (int w = 0; w < nwarps; ++w) t += sh.wcnt[par * nwarps + w][lane];
+        for (int w = 0; w < nwarps; ++w) t += sh.wcnt[w][lane];
         B = t * E;
-        if (t < nthr && (int)(first_code_s[t] & 15u) < lane) B += sh.part_cnt[par][lane];  // inside thread t
+        if (t < nthr) {  // thread t is the first whose last code reaches k: its weights below k
+            PackedCodes<E> pc;
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) pc.w[w] = codes_s[t * WORDS + w];
+            B += count_below<E>(pc, lane);
+        }
         if (B > N) B = N;
     }
     double P = 0.0;
@@ -378,22 +376,27 @@ __device__ void write_outputs(const LloydArgs& a, int64_t row, int K, const Lloy
 
 template <int DT, int K, int E>
 __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
-                            LloydShared& sh, uint32_t* first_code_s, uint32_t* sorted) {
+                            LloydShared& sh, uint32_t* codes_s, uint32_t* sorted) {
     constexpr int WORDS = (E + 7) / 8;  // packed codes: 8 weights per 32-bit word
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int N = (int)a.d_out;
     const int T = a.iters;
     const double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
 
-    // Every warp keeps the centroids itself (lane k holds c_k) and repeats the tiny update, so that
-    // a sweep needs a single block-wide barrier.  All warps compute identical values.
+    // Warp 0 owns the centroids (lane k holds c_k) and publishes them, with the mode of the next
+    // sweep, in shared memory; a sweep costs two barriers and the update is computed once.
     float ck_lane = 0.f;
-    if (lane < K) {
-        int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
-        ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
+    int B_prev = -1;  // warp 0, lane k: B_k of the previous ordered sweep (-1: none)
+    if (warp == 0) {
+        if (lane < K) {
+            int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
+            ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
+            sh.c[lane] = ck_lane;
+        }
+        const bool f = counting_sweep_valid<K>(ck_lane, need);
+        if (lane == 0) { sh.flag_fast = f ? 1 : 0; sh.flag_moved = 1; }
     }
-    bool fast = counting_sweep_valid<K>(ck_lane, need);
-    int B_prev = -1;  // lane k: B_k of the previous ordered sweep (-1: none)
+    __syncthreads();
 
     uint32_t cw[WORDS];
 #pragma unroll
@@ -402,9 +405,9 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
     int sweeps_done = 0;
     for (int it = 0; it <= T; ++it) {
 #pragma unroll
-        for (int k = 0; k < K; ++k) c[k] = __shfl_sync(0xffffffffu, ck_lane, k);
+        for (int k = 0; k < K; ++k) c[k] = sh.c[k];
+        const bool fast = sh.flag_fast != 0;
         const bool last = (it == T);
-        const int par = it & 1;
 
         uint32_t nw[WORDS];
         sweep_codes<K, E>(x, c, fast, nw);
@@ -415,66 +418,50 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         if (last) break;
 
         if (fast) {
-            // codes are non-decreasing along the sorted order.  Lane k finds, by bisection over the
-            // lanes' last codes, how many threads of this warp lie entirely below boundary k; a thread
-            // with a boundary in its interior also publishes the sum and count of its weights below it.
-            first_code_s[par * nthr + tid] = cw[0];
-            const int c_first = (int)(cw[0] & 15u);
-            const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
-            // lane k: how many threads of this warp lie entirely below boundary k.  The last codes are
-            // non-decreasing along the lanes: everything below the first lane's code counts 0, everything
-            // above the last lane's code counts 32, and a lane whose successor has a larger code owns the
-            // boundaries in between
-            {
-                const int c0 = __shfl_sync(0xffffffffu, c_last, 0), c31 = __shfl_sync(0xffffffffu, c_last, 31);
-                const int c_next = __shfl_down_sync(0xffffffffu, c_last, 1);
-                int* cnt_row = sh.wcnt[par * (nthr >> 5) + warp];
-                if (lane > 0 && lane < K) {
-                    if (lane <= c0) cnt_row[lane] = 0;
-                    else if (lane > c31) cnt_row[lane] = 32;
-                }
-                if (lane < 31 && c_next > c_last)
-                    for (int k = c_last + 1; k <= c_next; ++k) cnt_row[k] = lane + 1;
-            }
-            if (c_first != c_last) {  // boundaries inside this thread: its weights below each of them
-                PackedCodes<E> pc;
+            // codes are non-decreasing along the sorted order: publish them and, per warp, how many of
+            // its threads lie entirely below each boundary.  The threads' last codes are non-decreasing
+            // along the lanes: a boundary at or below the first lane's code counts 0, one above the last
+            // lane's code counts 32, and a lane whose successor has a larger code owns those in between.
 #pragma unroll
-                for (int w = 0; w < WORDS; ++w) pc.w[w] = cw[w];
-                for (int k = c_first + 1; k <= c_last; ++k) sh.part_cnt[par][k] = count_below<E>(pc, k);
+            for (int w = 0; w < WORDS; ++w) codes_s[tid * WORDS + w] = cw[w];
+            const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
+            const int c0 = __shfl_sync(0xffffffffu, c_last, 0), c31 = __shfl_sync(0xffffffffu, c_last, 31);
+            const int c_next = __shfl_down_sync(0xffffffffu, c_last, 1);
+            int* cnt_row = sh.wcnt[warp];
+            if (lane > 0 && lane < K) {
+                if (lane <= c0) cnt_row[lane] = 0;
+                else if (lane > c31) cnt_row[lane] = 32;
             }
+            if (lane < 31 && c_next > c_last)
+                for (int k = c_last + 1; k <= c_next; ++k) cnt_row[k] = lane + 1;
             __syncthreads();
-            if (!kSingleWarpUpdate || warp == 0) {
+            if (warp == 0) {
                 int B;
-                ck_lane = centroid_from_boundaries<DT, K, E>(sh, par, first_code_s + par * nthr, sorted, N, ck_lane,
-                                                             B, nthr >> 5);
+                ck_lane = centroid_from_boundaries<DT, K, E>(sh, codes_s, sorted, N, ck_lane, B, nthr >> 5);
                 const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
                 B_prev = B;
-                fast = counting_sweep_valid<K>(ck_lane, need);
-                if (kSingleWarpUpdate) {
-                    if (lane < K) sh.c[lane] = ck_lane;
-                    if (lane == 0) { sh.flag_fast = fast ? 1 : 0; sh.flag_moved = moved ? 1 : 0; }
-                } else if (!moved) {
-                    break;  // same decision in every warp
-                }
+                const bool f = counting_sweep_valid<K>(ck_lane, need);
+                if (lane < K) sh.c[lane] = ck_lane;
+                if (lane == 0) { sh.flag_fast = f ? 1 : 0; sh.flag_moved = moved ? 1 : 0; }
             }
-            if (kSingleWarpUpdate) {
-                __syncthreads();
-                if (lane < K) ck_lane = sh.c[lane];
-                fast = sh.flag_fast != 0;
-                if (!sh.flag_moved) break;
-            }
+            __syncthreads();
+            if (!sh.flag_moved) break;  // no boundary moved: later sweeps would repeat this one
         } else {
             const int changed = __syncthreads_or(any != 0);
             if (!changed) break;
-            rebuild_partials<K, E>(x, cw, nval, sh, par);
+            rebuild_partials<K, E>(x, cw, nval, sh);
             __syncthreads();
-            ck_lane = centroid_from_partials<K>(sh, par, ck_lane, nthr >> 5);
-            fast = counting_sweep_valid<K>(ck_lane, need);
-            B_prev = -1;
+            if (warp == 0) {
+                ck_lane = centroid_from_partials<K>(sh, ck_lane, nthr >> 5);
+                const bool f = counting_sweep_valid<K>(ck_lane, need);
+                if (lane < K) sh.c[lane] = ck_lane;
+                if (lane == 0) sh.flag_fast = f ? 1 : 0;
+                B_prev = -1;
+            }
+            __syncthreads();
         }
     }
-    if (warp == 0 && lane < K) sh.c[lane] = ck_lane;
-    __syncthreads();  // centroids published; no thread reads keys from `sorted` after this point
+    __syncthreads();  // sh.c holds the final centroids; no thread reads keys from `sorted` after this point
     write_outputs<E>(a, row, K, sh, sorted, x, cw, nval, sweeps_done);
 }
 
@@ -633,24 +620,24 @@ lloyd_kernel(const LloydArgs a) {
     if (tid == 0) {  // published by the first barrier below, long before anyone uses them
         sh.pt4 = reinterpret_cast<double*>(tail);
         sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr, E));
-        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr, E) + (size_t)2 * nwarps * kMaxK * sizeof(double));
+        sh.wcnt = reinterpret_cast<int (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr, E) + (size_t)nwarps * kMaxK * sizeof(double));
     }
 
     float x[E];
     int nval;
     prepare_channel<DT, E>(a, row, sh, scratch, sorted, x, nval);
 
-    uint32_t* first_code_s = reinterpret_cast<uint32_t*>(scratch);
+    uint32_t* codes_s = reinterpret_cast<uint32_t*>(scratch);  // [nthr][WORDS], at most 16 KiB
     const int bits = a.bits[row];
-    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, first_code_s, sorted);
-    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, first_code_s, sorted);
-    else fit_channel<DT, 16, E>(a, row, x, nval, sh, first_code_s, sorted);
+    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
+    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
+    else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
     const size_t nwarps = (size_t)threads / 32;
     return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4 +
-           lloyd_pt_bytes(threads, E) + 2 * nwarps * kMaxK * (sizeof(double) + sizeof(int));
+           lloyd_pt_bytes(threads, E) + nwarps * kMaxK * (sizeof(double) + sizeof(int));
 }
 
 template <int DT, int E, int MAXT, int MINB>
