@@ -660,6 +660,8 @@ static cmpq_status launch_dt(const LloydArgs& args, cudaStream_t st) {
     };
     if (N <= 2048) return launch_variant<DT, 4, 512, 1>(args, threads_for(4), st);
     if (N <= 4096) return launch_variant<DT, 16, 256, 4>(args, threads_for(16), st);
+    if (N <= 8192) return launch_variant<DT, 16, 512, 2>(args, threads_for(16), st);
+    if (N <= 12288) return launch_variant<DT, 32, 384, 2>(args, threads_for(32), st);
     if (N <= 16384) return launch_variant<DT, 16, 1024, 1>(args, threads_for(16), st);
     return launch_variant<DT, 32, 1024, 1>(args, threads_for(32), st);
 }
