@@ -56,6 +56,14 @@ struct alignas(16) LloydShared {
 
 __host__ __device__ inline size_t lloyd_pt_bytes(int nthr, int E) { return (((size_t)nthr * E / 4 + 1) * sizeof(double) + 15) & ~(size_t)15; }
 
+__host__ __device__ inline size_t lloyd_codes_bytes(int nthr, int E) { return (size_t)nthr * ((E + 7) / 8) * 4; }
+__host__ __device__ inline size_t lloyd_tail_bytes(int nthr, int E) {
+    return lloyd_pt_bytes(nthr, E) + (size_t)(nthr / 32) * 16 * (sizeof(double) + sizeof(int));
+}
+__host__ __device__ inline bool lloyd_tail_fits_scratch(int nthr, int E) {
+    return lloyd_codes_bytes(nthr, E) + lloyd_tail_bytes(nthr, E) <= (size_t)16 * 256 * sizeof(int);
+}
+
 __host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
     return kMaxK * 256 * (int)sizeof(int);  // 16 KiB >= 16 bytes x 1024 threads >= 32768 bits
 }
@@ -616,7 +624,11 @@ lloyd_kernel(const LloydArgs a) {
     const int nwarps = nthr >> 5;
     unsigned char* scratch = smem_raw + sizeof(LloydShared);
     uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
-    unsigned char* tail = reinterpret_cast<unsigned char*>(sorted) + (((size_t)N + 3) & ~(size_t)3) * 4;
+    // prefix table and per-warp exchange arrays: inside the scratch region (behind the packed codes)
+    // when they fit there -- they are first written after the sort is done with it -- else behind `sorted`
+    unsigned char* tail = lloyd_tail_fits_scratch(nthr, E)
+                              ? scratch + lloyd_codes_bytes(nthr, E)
+                              : reinterpret_cast<unsigned char*>(sorted) + (((size_t)N + 3) & ~(size_t)3) * 4;
     if (tid == 0) {  // published by the first barrier below, long before anyone uses them
         sh.pt4 = reinterpret_cast<double*>(tail);
         sh.wsum = reinterpret_cast<double (*)[kMaxK]>(tail + lloyd_pt_bytes(nthr, E));
@@ -635,9 +647,9 @@ lloyd_kernel(const LloydArgs a) {
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
-    const size_t nwarps = (size_t)threads / 32;
-    return sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4 +
-           lloyd_pt_bytes(threads, E) + nwarps * kMaxK * (sizeof(double) + sizeof(int));
+    size_t bytes = sizeof(LloydShared) + (size_t)lloyd_scratch_bytes((int)d_out) + (((size_t)d_out + 3) & ~(size_t)3) * 4;
+    if (!lloyd_tail_fits_scratch(threads, E)) bytes += lloyd_tail_bytes(threads, E);
+    return bytes;
 }
 
 template <int DT, int E, int MAXT, int MINB>
