@@ -43,6 +43,7 @@ struct alignas(16) LloydShared {
     int excl1[257];
     int bucket_rank[256];              // rank of a high-byte bucket among the non-empty ones, or -1
     float c[kMaxK];                    // centroids for the next sweep, written by warp 0
+    int below_total[kMaxK];            // ordered path: threads of the block entirely below boundary k
     int flag_fast, flag_moved;         // warp 0's decisions: counting sweep valid / a boundary moved
     int n_nonempty;
     float vmin, vmax;                  // value range of the channel
@@ -259,21 +260,20 @@ __device__ __forceinline__ int count_below(const PackedCodes<E>& pc, int k) {
 // Ordered path, warp 0: lane k (0..K) evaluates B_k = number of weights with a code below k and the
 // fp64 sum P_k of those weights (prefix table at every fourth weight plus at most three weights read
 // from the sorted array); cluster k is the run [B_k, B_{k+1}).
-//   sh.wcnt[w][k]  = threads of warp w whose last code is < k  (k = 1..K-1)
-//   codes_s[t]     = packed codes of thread t
+//   sh.below_total[k] = threads whose last code is < k  (k = 1..K-1); read and cleared here
+//   codes_s[t]        = packed codes of thread t
 // Returns the new centroid of cluster `lane` (the old one if the cluster is empty); B_out = B_lane.
 template <int DT, int K, int E>
-__device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh, const uint32_t* codes_s,
-                                                          const uint32_t* sorted, int N, float ck, int& B_out,
-                                                          int nwarps) {
+__device__ __forceinline__ float centroid_from_boundaries(LloydShared& sh, const uint32_t* codes_s,
+                                                          const uint32_t* sorted, int N, float ck, int& B_out) {
     constexpr int WORDS = (E + 7) / 8;
     const int lane = threadIdx.x & 31, nthr = blockDim.x;
     int B = 0;
     if (lane == K) {
         B = N;
     } else if (lane > 0 && lane < K) {
-        int t = 0;
-        for (int w = 0; w < nwarps; ++w) t += sh.wcnt[w][lane];
+        const int t = sh.below_total[lane];
+        sh.below_total[lane] = 0;
         B = t * E;
         if (t < nthr) {  // thread t is the first whose last code reaches k: its weights below k
             PackedCodes<E> pc;
@@ -286,10 +286,16 @@ __device__ __forceinline__ float centroid_from_boundaries(const LloydShared& sh,
     double P = 0.0;
     if (lane <= K) {
         const int q = B >> 2, r = B & 3;
+        double tail[3];  // the three loads are independent of r, so they overlap
+#pragma unroll
+        for (int e = 0; e < 3; ++e) {
+            const int idx = 4 * q + e < N ? 4 * q + e : N - 1;
+            tail[e] = (double)value_of_key16<DT>(sorted[idx] >> 16);
+        }
         P = sh.pt4[q];
 #pragma unroll
         for (int e = 0; e < 3; ++e)
-            if (e < r) P += (double)value_of_key16<DT>(sorted[4 * q + e] >> 16);
+            if (e < r) P += tail[e];
     }
     const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
     const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
@@ -403,6 +409,7 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         }
         const bool f = counting_sweep_valid<K>(ck_lane, need);
         if (lane == 0) { sh.flag_fast = f ? 1 : 0; sh.flag_moved = 1; }
+        if (lane < kMaxK) sh.below_total[lane] = 0;
     }
     __syncthreads();
 
@@ -426,26 +433,22 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
         if (last) break;
 
         if (fast) {
-            // codes are non-decreasing along the sorted order: publish them and, per warp, how many of
-            // its threads lie entirely below each boundary.  The threads' last codes are non-decreasing
-            // along the lanes: a boundary at or below the first lane's code counts 0, one above the last
-            // lane's code counts 32, and a lane whose successor has a larger code owns those in between.
+            // codes are non-decreasing along the sorted order: publish them and add, per warp, how many of
+            // its threads lie entirely below each boundary to the block's totals.  The threads' last codes are non-decreasing
+            // along the lanes: a boundary at or below the first lane's code adds nothing, one above the last
+            // lane's code adds 32, and a lane whose successor has a larger code owns those in between.
 #pragma unroll
             for (int w = 0; w < WORDS; ++w) codes_s[tid * WORDS + w] = cw[w];
             const int c_last = (int)((cw[WORDS - 1] >> (4 * ((E - 1) & 7))) & 15u);
-            const int c0 = __shfl_sync(0xffffffffu, c_last, 0), c31 = __shfl_sync(0xffffffffu, c_last, 31);
+            const int c31 = __shfl_sync(0xffffffffu, c_last, 31);
             const int c_next = __shfl_down_sync(0xffffffffu, c_last, 1);
-            int* cnt_row = sh.wcnt[warp];
-            if (lane > 0 && lane < K) {
-                if (lane <= c0) cnt_row[lane] = 0;
-                else if (lane > c31) cnt_row[lane] = 32;
-            }
+            if (lane > 0 && lane < K && lane > c31) atomicAdd(&sh.below_total[lane], 32);
             if (lane < 31 && c_next > c_last)
-                for (int k = c_last + 1; k <= c_next; ++k) cnt_row[k] = lane + 1;
+                for (int k = c_last + 1; k <= c_next; ++k) atomicAdd(&sh.below_total[k], lane + 1);
             __syncthreads();
             if (warp == 0) {
                 int B;
-                ck_lane = centroid_from_boundaries<DT, K, E>(sh, codes_s, sorted, N, ck_lane, B, nthr >> 5);
+                ck_lane = centroid_from_boundaries<DT, K, E>(sh, codes_s, sorted, N, ck_lane, B);
                 const bool moved = __any_sync(0xffffffffu, lane < K && B != B_prev);
                 B_prev = B;
                 const bool f = counting_sweep_valid<K>(ck_lane, need);
