@@ -34,6 +34,8 @@ namespace cmpq {
 
 constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
+constexpr int kSortSlots = 32;  // high-byte buckets refined per pass of the sort's second level
+static_assert(CMPQ_MAX_D_OUT < 65536, "the sort's second-level counters are 16 bits wide");
 
 struct alignas(16) LloydShared {
     double* pt4;                       // [nthr E / 4 + 1] fp64 sum of the first 4 i sorted weights
@@ -66,7 +68,8 @@ __host__ __device__ inline bool lloyd_tail_fits_scratch(int nthr, int E) {
 }
 
 __host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
-    return kMaxK * 256 * (int)sizeof(int);  // 16 KiB >= 16 bytes x 1024 threads >= 32768 bits
+    // 16 KiB = kSortSlots x 256 16-bit counters >= 16 bytes x 1024 threads >= 32768 bits
+    return kSortSlots * 128 * (int)sizeof(uint32_t);
 }
 
 template <int DT>
@@ -114,6 +117,33 @@ __device__ __forceinline__ int warp_scan256(const int* in, int* out_excl) {
     return __shfl_sync(0xffffffffu, incl, 31);
 }
 
+// In-place exclusive prefix of 256 16-bit counters packed two per word (128 words, 16-byte
+// aligned), by one warp: 4 words per lane.
+__device__ __forceinline__ void warp_scan256_packed(uint32_t* h) {
+    const int lane = threadIdx.x & 31;
+    uint4 v = reinterpret_cast<uint4*>(h)[lane];
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t s = 0;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) s += (w[t] & 0xffffu) + (w[t] >> 16);
+    uint32_t incl = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    uint32_t run = incl - s;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        uint32_t lo = run;
+        run += w[t] & 0xffffu;
+        uint32_t hi = run;
+        run += w[t] >> 16;
+        w[t] = lo | (hi << 16);
+    }
+    reinterpret_cast<uint4*>(h)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // Code of one weight by the defining scan: first k minimising |x - c_k|.
 template <int K>
 __device__ __forceinline__ int nearest_scan(float x, const float (&c)[K]) {
@@ -159,26 +189,34 @@ __device__ void sort_channel(const uint32_t (&key)[E], int nval, LloydShared& sh
         if (lane == 31) sh.n_nonempty = incl;
     }
     __syncthreads();
-    const int ngroups = (sh.n_nonempty + kMaxK - 1) / kMaxK;  // 16 buckets are refined at a time
+    // Second level: the low byte inside each non-empty high-byte bucket, kSortSlots buckets at a
+    // time.  Two 16-bit counters share a word (a channel has at most 32768 weights, so neither a
+    // count nor a prefix inside one bucket reaches 2^16 and the halves never carry into each other).
+    uint32_t* h2 = reinterpret_cast<uint32_t*>(hist2);
+    const int ngroups = (sh.n_nonempty + kSortSlots - 1) / kSortSlots;
     for (int grp = 0; grp < ngroups; ++grp) {
-        for (int b = tid; b < kMaxK * 256; b += nthr) hist2[b] = 0;
+        for (int b = tid; b < kSortSlots * 32; b += nthr) reinterpret_cast<uint4*>(h2)[b] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             if (e < nval) {
                 int r = sh.bucket_rank[key[e] >> 8];
-                if ((r >> 4) == grp) atomicAdd(&hist2[(r & 15) * 256 + (key[e] & 0xff)], 1);
+                uint32_t lo = key[e] & 0xffu;
+                if ((r >> 5) == grp) atomicAdd(&h2[(r & 31) * 128 + (lo >> 1)], 1u << (16 * (lo & 1u)));
             }
         }
         __syncthreads();
-        for (int s = warp; s < kMaxK; s += nwarps) warp_scan256(hist2 + s * 256, hist2 + s * 256);
+        for (int s = warp; s < kSortSlots; s += nwarps) warp_scan256_packed(h2 + s * 128);
         __syncthreads();
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             if (e < nval) {
                 int r = sh.bucket_rank[key[e] >> 8];
-                if ((r >> 4) == grp) {
-                    int pos = sh.excl1[key[e] >> 8] + atomicAdd(&hist2[(r & 15) * 256 + (key[e] & 0xff)], 1);
+                uint32_t lo = key[e] & 0xffu;
+                if ((r >> 5) == grp) {
+                    uint32_t sh16 = 16 * (lo & 1u);
+                    uint32_t old = atomicAdd(&h2[(r & 31) * 128 + (lo >> 1)], 1u << sh16);
+                    int pos = sh.excl1[key[e] >> 8] + (int)((old >> sh16) & 0xffffu);
                     uint32_t col = (uint32_t)(((e >> 2) * nthr + tid) * 4 + (e & 3));
                     sorted[pos] = (key[e] << 16) | col;
                 }
