@@ -56,6 +56,17 @@ typedef enum { CMPQ_F16 = 0, CMPQ_BF16 = 1 } cmpq_dtype;
  * quantiles of a and the comparisons are strict, as the algorithm is printed. */
 typedef enum { CMPQ_ALLOC_RANK = 0, CMPQ_ALLOC_QUANTILE = 1 } cmpq_alloc_mode;
 
+/* How the K-means kernels find the nearest centroid of every weight (Section 3: each weight goes
+ * to its nearest centroid; the rule itself is stated at cmpq_quantize_layer and is the same for
+ * both).  Both give bit-identical centroids, codes and errors.
+ *   CMPQ_ASSIGN_ORDERED    (default) the channel is sorted once; while the centroids are strictly
+ *                          increasing with safe gaps, a cluster is a run of the sorted order and an
+ *                          iteration only searches the K-1 run boundaries and reads prefix sums.
+ *                          Iterations whose centroids do not allow this fall back to all pairs.
+ *   CMPQ_ASSIGN_ALL_PAIRS  every iteration evaluates every (weight, centroid) pair on the fp32
+ *                          pipes: the brute-force formulation, kept for measuring ALU throughput. */
+typedef enum { CMPQ_ASSIGN_ORDERED = 0, CMPQ_ASSIGN_ALL_PAIRS = 1 } cmpq_lloyd_assignment;
+
 typedef enum {
     CMPQ_OP_COLLECT_STATS = 0,
     CMPQ_OP_ALLOCATE_BITS = 1,
@@ -137,8 +148,10 @@ cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, in
  * dynamic range is so wide that fp64 cluster sums may depend on the order of summation; when
  * it stays 0 the centroids are independent of the summation order, hence reproducible bit
  * for bit by any other correct implementation.
- * sweeps (optional device uint64, caller zeroes it): receives the total number of
- * (weight, centroid) distance evaluations performed, for throughput accounting.
+ * sweeps (optional device uint64, caller zeroes it): receives, summed over the channels,
+ * (assignment steps executed) * d_out * K, i.e. the number of (weight, centroid) distance
+ * evaluations that assigning every weight against every centroid costs.  CMPQ_ASSIGN_ALL_PAIRS
+ * performs exactly that many; CMPQ_ASSIGN_ORDERED reaches the same result with far fewer.
  * ws: cmpq_workspace_bytes(CMPQ_OP_QUANTIZE_LAYER, d_in, d_out). */
 cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
                                 int64_t ldw, const uint8_t* bits, const int32_t* rows,
@@ -146,6 +159,12 @@ cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int6
                                 const float* sens, float* lut, uint8_t* codes,
                                 int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
                                 size_t ws_bytes, void* stream);
+
+/* Process-wide choice of the assignment method used by cmpq_extract_outliers and
+ * cmpq_quantize_layer from the next call on (host state, no GPU work; thread-safe).
+ * CMPQ_ERR_INVALID_ARG for an unknown value. */
+cmpq_status cmpq_set_lloyd_assignment(cmpq_lloyd_assignment mode);
+cmpq_lloyd_assignment cmpq_get_lloyd_assignment(void);
 
 /* ---- packing (accounting of Section 5.1; per-precision sub-matrices of Section 6) -----------
  * Three segments in the order 2-, 3-, 4-bit channels, channels by ascending id inside a

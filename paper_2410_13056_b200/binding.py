@@ -13,6 +13,7 @@ import torch
 
 F16, BF16 = 0, 1
 ALLOC_RANK, ALLOC_QUANTILE = 0, 1
+ASSIGN_ORDERED, ASSIGN_ALL_PAIRS = 0, 1
 OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK = range(5)
 LUT_STRIDE = 16
 
@@ -20,6 +21,7 @@ EXPORTS = (
     "cmpq_collect_stats", "cmpq_collect_stats_static", "cmpq_finalize_stats", "cmpq_allocate_bits", "cmpq_extract_outliers",
     "cmpq_quantize_layer", "cmpq_pack", "cmpq_workspace_bytes", "cmpq_alloc_counts",
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
+    "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -63,6 +65,10 @@ def lib():
         L.cmpq_default_counts.restype = None
         L.cmpq_packed_words.argtypes = [vp, i64, i64]
         L.cmpq_packed_words.restype = i64
+        L.cmpq_set_lloyd_assignment.argtypes = [ci]
+        L.cmpq_set_lloyd_assignment.restype = ci
+        L.cmpq_get_lloyd_assignment.argtypes = []
+        L.cmpq_get_lloyd_assignment.restype = ci
         L.cmpq_status_string.argtypes = [ci]
         L.cmpq_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -97,6 +103,15 @@ def cmpq_workspace_bytes(op, d_in, d_out=0):
 def workspace(op, d_in, d_out=0, device="cuda"):
     """A fresh scratch buffer of the size the given call needs."""
     return torch.empty(max(256, cmpq_workspace_bytes(op, d_in, d_out)), dtype=torch.uint8, device=device)
+
+
+def cmpq_set_lloyd_assignment(mode):
+    """ASSIGN_ORDERED (default) or ASSIGN_ALL_PAIRS for the K-means calls that follow."""
+    _check(lib().cmpq_set_lloyd_assignment(int(mode)), "cmpq_set_lloyd_assignment")
+
+
+def cmpq_get_lloyd_assignment():
+    return int(lib().cmpq_get_lloyd_assignment())
 
 
 def cmpq_alloc_counts(d_in, avg_bits):

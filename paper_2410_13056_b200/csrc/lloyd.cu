@@ -30,6 +30,8 @@
 //               with coalesced writes
 #include "lloyd.cuh"
 
+#include <atomic>
+
 namespace cmpq {
 
 constexpr int kMaxK = 16;
@@ -47,6 +49,8 @@ struct alignas(16) LloydShared {
     float c[kMaxK];                    // centroids for the next sweep, written by warp 0
     int below_total[kMaxK];            // ordered path: threads of the block entirely below boundary k
     int flag_fast, flag_moved;         // warp 0's decisions: counting sweep valid / a boundary moved
+    int bound[kMaxK + 1];              // ordered search: B_k of the last search, published by warp 0
+    int pub_it, pub_done, pub_sweeps;  // ordered search: updates done, fit finished, searches counted
     int n_nonempty;
     float vmin, vmax;                  // value range of the channel
     float wlo[kMaxWarps], whi[kMaxWarps];
@@ -295,32 +299,14 @@ __device__ __forceinline__ int count_below(const PackedCodes<E>& pc, int k) {
     return 8 * WORDS - ge - (8 * WORDS - E);
 }
 
-// Ordered path, warp 0: lane k (0..K) evaluates B_k = number of weights with a code below k and the
-// fp64 sum P_k of those weights (prefix table at every fourth weight plus at most three weights read
-// from the sorted array); cluster k is the run [B_k, B_{k+1}).
-//   sh.below_total[k] = threads whose last code is < k  (k = 1..K-1); read and cleared here
-//   codes_s[t]        = packed codes of thread t
-// Returns the new centroid of cluster `lane` (the old one if the cluster is empty); B_out = B_lane.
-template <int DT, int K, int E>
-__device__ __forceinline__ float centroid_from_boundaries(LloydShared& sh, const uint32_t* codes_s,
-                                                          const uint32_t* sorted, int N, float ck, int& B_out) {
-    constexpr int WORDS = (E + 7) / 8;
-    const int lane = threadIdx.x & 31, nthr = blockDim.x;
-    int B = 0;
-    if (lane == K) {
-        B = N;
-    } else if (lane > 0 && lane < K) {
-        const int t = sh.below_total[lane];
-        sh.below_total[lane] = 0;
-        B = t * E;
-        if (t < nthr) {  // thread t is the first whose last code reaches k: its weights below k
-            PackedCodes<E> pc;
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) pc.w[w] = codes_s[t * WORDS + w];
-            B += count_below<E>(pc, lane);
-        }
-        if (B > N) B = N;
-    }
+// Warp 0, lane k (0..K) holds B_k = number of weights (in sorted order) before cluster k, B_0 = 0
+// and B_K = N: cluster k is the run [B_k, B_{k+1}) of the sorted order.  Its fp64 sum is a
+// difference of prefix sums P_k (table at every fourth weight plus at most three weights read from
+// the sorted array).  Returns the new centroid of cluster `lane` (the old one if the run is empty).
+template <int DT, int K>
+__device__ __forceinline__ float centroid_from_runs(const LloydShared& sh, const uint32_t* sorted, int N,
+                                                    float ck, int B) {
+    const int lane = threadIdx.x & 31;
     double P = 0.0;
     if (lane <= K) {
         const int q = B >> 2, r = B & 3;
@@ -341,8 +327,103 @@ __device__ __forceinline__ float centroid_from_boundaries(LloydShared& sh, const
         const int cnt = Bn - B;
         if (cnt > 0) ck = __double2float_rn(__ddiv_rn(Pn - P, (double)cnt));
     }
-    B_out = B;
     return ck;
+}
+
+// All-pairs path, warp 0: lane k (0..K) evaluates B_k = number of weights with a code below k from
+//   sh.below_total[k] = threads whose last code is < k  (k = 1..K-1); read and cleared here
+//   codes_s[t]        = packed codes of thread t
+// and returns the new centroid of cluster `lane`; B_out = B_lane.
+template <int DT, int K, int E>
+__device__ __forceinline__ float centroid_from_boundaries(LloydShared& sh, const uint32_t* codes_s,
+                                                          const uint32_t* sorted, int N, float ck, int& B_out) {
+    constexpr int WORDS = (E + 7) / 8;
+    const int lane = threadIdx.x & 31, nthr = blockDim.x;
+    int B = 0;
+    if (lane == K) {
+        B = N;
+    } else if (lane > 0 && lane < K) {
+        const int t = sh.below_total[lane];
+        sh.below_total[lane] = 0;
+        B = t * E;
+        if (t < nthr) {  // thread t is the first whose last code reaches k: its weights below k
+            PackedCodes<E> pc;
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) pc.w[w] = codes_s[t * WORDS + w];
+            B += count_below<E>(pc, lane);
+        }
+        if (B > N) B = N;
+    }
+    B_out = B;
+    return centroid_from_runs<DT, K>(sh, sorted, N, ck, B);
+}
+
+// Ordered search, warp 0 (lane k holds c_k; the centroids pass counting_sweep_valid): the
+// predicate fabsf(x - c_k) < fabsf(x - c_{k-1}) is then false on a prefix of the sorted order and true
+// on the rest, so B_k -- the number of weights for which it is false -- is found by probing
+// sorted weights instead of evaluating all of them: every half warp narrows the interval of one
+// boundary by 16 probes per round, two boundaries per round per warp, kBatch pairs interleaved.
+// Returns B_lane for lanes 1..K-1, 0 in lane 0, N in lane K.
+template <int DT, int K>
+__device__ __forceinline__ int search_boundaries(const uint32_t* sorted, int N, float ck_lane) {
+    constexpr int PAIRS = K / 2;
+    constexpr int kBatch = PAIRS < 4 ? PAIRS : 4;
+    const int lane = threadIdx.x & 31, half = lane >> 4, j = lane & 15;
+    int B = (lane == K) ? N : 0;
+#pragma unroll
+    for (int p0 = 0; p0 < PAIRS; p0 += kBatch) {
+        float ck[kBatch], cm[kBatch];
+        int lo[kBatch], hi[kBatch];
+#pragma unroll
+        for (int p = 0; p < kBatch; ++p) {
+            const int k = 1 + 2 * (p0 + p) + half;
+            const int kk = k < K ? k : K - 1;
+            ck[p] = __shfl_sync(0xffffffffu, ck_lane, kk);
+            cm[p] = __shfl_sync(0xffffffffu, ck_lane, kk - 1);
+            lo[p] = 0;
+            hi[p] = k < K ? N : 0;  // k = K has no boundary: empty interval
+        }
+        // an interval of length len shrinks to at most step - 1 per round; the probe stride is made odd
+        // so that the 16 probes of a boundary fall into 16 different shared-memory banks
+        for (int len = N; len > 0; len = (((len + 15) >> 4) | 1) - 1) {
+            // staged so that the kBatch independent chains overlap: addresses and loads, predicates,
+            // votes, interval updates
+            int step[kBatch];
+            float v[kBatch];
+            bool inb[kBatch];
+#pragma unroll
+            for (int p = 0; p < kBatch; ++p) {
+                const int cur = hi[p] - lo[p];
+                step[p] = ((cur + 15) >> 4) | 1;
+                const int pos = lo[p] + j * step[p] + step[p] - 1;
+                inb[p] = pos < hi[p];  // false for an empty interval; positions from hi on are known to be true
+                const int idx = pos < N ? pos : N - 1;
+                v[p] = value_of_key16<DT>(sorted[idx] >> 16);
+            }
+            uint32_t m[kBatch];
+#pragma unroll
+            for (int p = 0; p < kBatch; ++p) {
+                const bool is_false = inb[p] && !(fabsf(v[p] - ck[p]) < fabsf(v[p] - cm[p]));
+                m[p] = __ballot_sync(0xffffffffu, is_false);
+            }
+#pragma unroll
+            for (int p = 0; p < kBatch; ++p) {
+                const int nf = __popc((m[p] >> (16 * half)) & 0xffffu);
+                // an empty interval has nf = 0 and keeps lo = hi
+                lo[p] += nf * step[p];
+                const int cap = lo[p] + step[p] - 1;
+                if (nf < 16) hi[p] = hi[p] < cap ? hi[p] : cap;
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < kBatch; ++p) {
+            const int b0 = __shfl_sync(0xffffffffu, lo[p], 0);
+            const int b1 = __shfl_sync(0xffffffffu, lo[p], 16);
+            if (lane == 1 + 2 * (p0 + p)) B = b0;
+            if (lane == 2 + 2 * (p0 + p) && lane < K) B = b1;
+        }
+    }
+    return B;
 }
 
 // One sweep over a thread's E weights: their codes for the centroids c, packed 8 per word.
@@ -514,6 +595,128 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
     write_outputs<E>(a, row, K, sh, sorted, x, cw, nval, sweeps_done);
 }
 
+// The same fit with the ordered search in place of the all-pairs sweeps.  While the centroids pass
+// counting_sweep_valid, warp 0 runs whole iterations alone (search the K-1 boundaries, compare
+// them with the previous ones, update from the prefix table) and the other warps wait at a
+// barrier; an iteration whose centroids fail the test is done by the whole block with the plain
+// scan and per-cluster accumulation, exactly as in fit_channel.  The last assignment turns the
+// final boundaries into codes (or is a plain scan when the final centroids fail the test).
+template <int DT, int K, int E>
+__device__ void fit_channel_ordered(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
+                                    LloydShared& sh, uint32_t* sorted) {
+    constexpr int WORDS = (E + 7) / 8;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int N = (int)a.d_out;
+    const int T = a.iters;
+    const double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+
+    // warp 0 only: lane k holds c_k and B_k
+    float ck_lane = 0.f;
+    int B_prev = -1, it0 = 0, searches = 0;
+    bool valid0 = false, conv0 = false;
+    if (warp == 0) {
+        if (lane < K) {
+            int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
+            ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
+        }
+        valid0 = counting_sweep_valid<K>(ck_lane, need);
+    }
+
+    uint32_t cw[WORDS];
+#pragma unroll
+    for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;  // no plain sweep yet: the next one counts as a change
+    int plain_sweeps = 0, it_after_plain = -1;
+    bool codes_ready = false;  // cw holds the final codes (a plain sweep that changed nothing)
+    bool valid = false;
+    for (;;) {
+        if (warp == 0) {
+            while (it0 < T && valid0) {
+                const int B = search_boundaries<DT, K>(sorted, N, ck_lane);
+                ++searches;
+                const bool moved = __any_sync(0xffffffffu, lane > 0 && lane < K && B != B_prev);
+                B_prev = B;
+                if (!moved) { conv0 = true; break; }  // same runs as before: the update would repeat itself
+                ck_lane = centroid_from_runs<DT, K>(sh, sorted, N, ck_lane, B);
+                ++it0;
+                valid0 = counting_sweep_valid<K>(ck_lane, need);
+            }
+            if (valid0 && !conv0 && it0 == T) {  // last assignment
+                B_prev = search_boundaries<DT, K>(sorted, N, ck_lane);
+                ++searches;
+            }
+            if (lane < K) sh.c[lane] = ck_lane;
+            if (lane <= K) sh.bound[lane] = B_prev;
+            if (lane == 0) {
+                sh.flag_fast = valid0 ? 1 : 0;
+                sh.pub_it = it0;
+                sh.pub_done = (conv0 || it0 == T) ? 1 : 0;
+                sh.pub_sweeps = searches;
+            }
+        }
+        __syncthreads();
+        valid = sh.flag_fast != 0;
+        if (sh.pub_done) break;
+
+        // the centroids are not safe for the ordered search: one plain iteration by the block
+        const int it_pub = sh.pub_it;
+        if (it_pub != it_after_plain) {  // ordered iterations ran since the last plain sweep: its codes are stale
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;
+        }
+        float c[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) c[k] = sh.c[k];
+        uint32_t nw[WORDS];
+        sweep_codes<K, E>(x, c, false, nw);
+        ++plain_sweeps;
+        uint32_t any = 0;
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) { any |= nw[w] ^ cw[w]; cw[w] = nw[w]; }
+        const int changed = __syncthreads_or(any != 0);
+        if (!changed) { codes_ready = true; break; }
+        rebuild_partials<K, E>(x, cw, nval, sh);
+        __syncthreads();
+        if (warp == 0) {
+            ck_lane = centroid_from_partials<K>(sh, ck_lane, nthr >> 5);
+            ++it0;
+            valid0 = counting_sweep_valid<K>(ck_lane, need);
+            B_prev = -1;
+        }
+        it_after_plain = it_pub + 1;
+    }
+
+    if (!codes_ready) {
+        if (valid) {
+            // codes from the final boundaries: position i of the sorted order has code #{k : B_k <= i}
+            const int idx0 = tid * E;
+            int cf = 0, cl = 0;
+#pragma unroll
+            for (int k = 1; k < K; ++k) {
+                const int b = sh.bound[k];
+                cf += (idx0 >= b) ? 1 : 0;
+                cl += (idx0 + E - 1 >= b) ? 1 : 0;
+            }
+#pragma unroll
+            for (int w = 0; w < WORDS; ++w) cw[w] = (uint32_t)cf * 0x11111111u;
+            for (int k = cf + 1; k <= cl; ++k) {
+                const int b = sh.bound[k] - idx0;  // in [1, E-1]
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if (e >= b) cw[e >> 3] += 1u << (4 * (e & 7));
+            }
+        } else {
+            float c[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k) c[k] = sh.c[k];
+            sweep_codes<K, E>(x, c, false, cw);
+            ++plain_sweeps;
+        }
+    }
+    const int sweeps_done = plain_sweeps + sh.pub_sweeps;
+    __syncthreads();  // sh.c holds the final centroids; no thread reads keys from `sorted` after this point
+    write_outputs<E>(a, row, K, sh, sorted, x, cw, nval, sweeps_done);
+}
+
 // One-time work for a channel, by every thread of the block: read the row, zero the removed
 // positions, note the value range and the exactness diagnostics, sort it into `sorted`, load this
 // thread's run of E order statistics into x and build the fp64 prefix table sh.pt4.
@@ -653,7 +856,7 @@ __device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh
     nval_out = nval;
 }
 
-template <int DT, int E, int MAXT, int MINB>
+template <int DT, int E, int MAXT, int MINB, bool ORDERED>
 __global__ void __launch_bounds__(MAXT, MINB)
 lloyd_kernel(const LloydArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -661,7 +864,7 @@ lloyd_kernel(const LloydArgs a) {
     if (a.skip_row && a.skip_row[row]) return;
     const int N = (int)a.d_out;
     LloydShared& sh = *reinterpret_cast<LloydShared*>(smem_raw);
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, nthr = blockDim.x;
     const int nwarps = nthr >> 5;
     unsigned char* scratch = smem_raw + sizeof(LloydShared);
     uint32_t* sorted = reinterpret_cast<uint32_t*>(scratch + lloyd_scratch_bytes(N));
@@ -682,9 +885,15 @@ lloyd_kernel(const LloydArgs a) {
 
     uint32_t* codes_s = reinterpret_cast<uint32_t*>(scratch);  // [nthr][WORDS], at most 16 KiB
     const int bits = a.bits[row];
-    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
-    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
-    else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
+    if (ORDERED) {
+        if (bits == 2) fit_channel_ordered<DT, 4, E>(a, row, x, nval, sh, sorted);
+        else if (bits == 3) fit_channel_ordered<DT, 8, E>(a, row, x, nval, sh, sorted);
+        else fit_channel_ordered<DT, 16, E>(a, row, x, nval, sh, sorted);
+    } else {
+        if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
+        else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
+        else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
+    }
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
@@ -696,7 +905,7 @@ static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
 template <int DT, int E, int MAXT, int MINB>
 static cmpq_status launch_variant(const LloydArgs& args, int threads, cudaStream_t st) {
     const size_t smem = lloyd_smem_bytes(args.d_out, threads, E);
-    auto kern = lloyd_kernel<DT, E, MAXT, MINB>;
+    auto kern = args.all_pairs ? lloyd_kernel<DT, E, MAXT, MINB, false> : lloyd_kernel<DT, E, MAXT, MINB, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
     kern<<<(unsigned)args.d_in, threads, smem, st>>>(args);
@@ -718,6 +927,10 @@ static cmpq_status launch_dt(const LloydArgs& args, cudaStream_t st) {
     if (N <= 16384) return launch_variant<DT, 16, 1024, 1>(args, threads_for(16), st);
     return launch_variant<DT, 32, 1024, 1>(args, threads_for(32), st);
 }
+
+static std::atomic<int> g_assignment{CMPQ_ASSIGN_ORDERED};
+
+cmpq_lloyd_assignment lloyd_assignment() { return (cmpq_lloyd_assignment)g_assignment.load(); }
 
 cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st) {
     return dt == CMPQ_F16 ? launch_dt<CMPQ_F16>(args, st) : launch_dt<CMPQ_BF16>(args, st);
@@ -752,6 +965,14 @@ size_t quantize_ws_bytes(int64_t d_in, int64_t) {
 
 using namespace cmpq;
 
+extern "C" cmpq_status cmpq_set_lloyd_assignment(cmpq_lloyd_assignment mode) {
+    if (mode != CMPQ_ASSIGN_ORDERED && mode != CMPQ_ASSIGN_ALL_PAIRS) return CMPQ_ERR_INVALID_ARG;
+    g_assignment.store((int)mode);
+    return CMPQ_OK;
+}
+
+extern "C" cmpq_lloyd_assignment cmpq_get_lloyd_assignment(void) { return lloyd_assignment(); }
+
 extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
                                            int64_t ldw, const uint8_t* bits, const int32_t* rows,
                                            const int32_t* cols, int64_t nnz, int lloyd_iters,
@@ -782,5 +1003,6 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
     a.codes = codes;
     a.inexact_rows = inexact_rows;
     a.sweeps = sweeps;
+    a.all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
     return launch_lloyd(a, dt, st);
 }

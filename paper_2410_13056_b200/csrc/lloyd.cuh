@@ -22,7 +22,11 @@ struct LloydArgs {
     uint8_t* codes;          // [d_in][d_out] or NULL
     int32_t* inexact_rows;   // optional counter
     unsigned long long* sweeps;  // optional counter of distance evaluations
+    bool all_pairs;          // assignment by evaluating every (weight, centroid) pair
 };
+
+// The process-wide choice made by cmpq_set_lloyd_assignment.
+cmpq_lloyd_assignment lloyd_assignment();
 
 cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
 

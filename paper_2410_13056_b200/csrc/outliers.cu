@@ -337,6 +337,7 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
         la.iters = lloyd_iters;
         la.skip_row = o.is_act;
         la.err = o.err;
+        la.all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
         s = launch_lloyd(la, dt, st);
         if (s != CMPQ_OK) return s;
     }

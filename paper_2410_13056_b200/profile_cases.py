@@ -61,9 +61,12 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16"])
+    ap.add_argument("--assign", default="ordered", choices=["ordered", "all_pairs"],
+                    help="assignment method of the K-means kernels")
     a = ap.parse_args()
     dt = inputs.BF16 if a.dtype == "bf16" else inputs.F16
     torch.cuda.set_device(0)
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS if a.assign == "all_pairs" else B.ASSIGN_ORDERED)
     if a.case == "layer":
         run_layer(a)
         return

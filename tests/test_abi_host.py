@@ -95,6 +95,16 @@ def test_bad_arguments_are_refused_on_the_host(L):
     assert L.cmpq_pack(p, p, 8, 16, p, p, p, p, ws, 8, None) == WORKSPACE
 
 
+def test_assignment_method_is_host_state(L):
+    assert L.cmpq_get_lloyd_assignment() == B.ASSIGN_ORDERED          # the default
+    assert L.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS) == 0
+    assert L.cmpq_get_lloyd_assignment() == B.ASSIGN_ALL_PAIRS
+    assert L.cmpq_set_lloyd_assignment(7) == 1                        # unknown value: refused, unchanged
+    assert L.cmpq_get_lloyd_assignment() == B.ASSIGN_ALL_PAIRS
+    assert L.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED) == 0
+    assert B.cmpq_get_lloyd_assignment() == B.ASSIGN_ORDERED
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "_LIB_PATH", "/nonexistent/libcmpq.so")

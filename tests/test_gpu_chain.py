@@ -31,7 +31,14 @@ def _chain_with_gpu_statistic(Wu, dtype, a_gpu, b, n_act, n_q, T):
                 row_off=row_off, perm=perm, seg_rows=seg)
 
 
-def test_small_workload_full_parity():
+@pytest.fixture(params=["ordered", "all_pairs"])
+def assignment(request):
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS if request.param == "all_pairs" else B.ASSIGN_ORDERED)
+    yield request.param
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED)
+
+
+def test_small_workload_full_parity(assignment):
     cfg = inputs.CONFIGS["c1_small"]
     L = cfg.layers[0]
     W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, cfg.seed, device="cuda")

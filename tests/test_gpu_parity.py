@@ -18,6 +18,14 @@ STAT_RTOL = 1e-5
 LUT_RTOL = 1e-4
 
 
+@pytest.fixture(params=["ordered", "all_pairs"])
+def assignment(request):
+    """Runs a K-means test once per assignment method of the library; both must match the checker."""
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS if request.param == "all_pairs" else B.ASSIGN_ORDERED)
+    yield request.param
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED)
+
+
 def _lut_close(got, ref, W_absmax):
     np.testing.assert_allclose(got, ref, rtol=LUT_RTOL, atol=LUT_RTOL * W_absmax * 1e-3)
 
@@ -95,7 +103,7 @@ def _case(d_in, d_out, dtype, seed, b):
 @pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
 @pytest.mark.parametrize("d_in,d_out,T", [(96, 512, 10), (40, 1000, 6), (24, 4096, 20), (12, 11008, 5),
                                           (6, 28672, 4), (50, 37, 12), (64, 16, 30), (9, 1, 3), (5, 32768, 2)])
-def test_quantize_layer_matches_checker(dtype, d_in, d_out, T):
+def test_quantize_layer_matches_checker(dtype, d_in, d_out, T, assignment):
     W, Wu, a, bits = _case(d_in, d_out, dtype, 21 + d_out, 3.0)
     bits[: d_in // 3] = 2
     bits[d_in // 3: 2 * d_in // 3] = 4
@@ -112,7 +120,7 @@ def test_quantize_layer_matches_checker(dtype, d_in, d_out, T):
     assert 0 < sweeps <= (T + 1) * d_out * int((1 << bits.astype(np.int64)).sum())
 
 
-def test_quantize_layer_degenerate_channels():
+def test_quantize_layer_degenerate_channels(assignment):
     d_out = 256
     rows_ = []
     rows_.append(np.zeros(d_out))                                       # all zero
@@ -134,7 +142,7 @@ def test_quantize_layer_degenerate_channels():
             assert np.array_equal(lut.view(np.uint32), rlut.view(np.uint32)), (c, T)
 
 
-def test_wide_dynamic_range_is_flagged_not_hidden():
+def test_wide_dynamic_range_is_flagged_not_hidden(assignment):
     d_out = 512
     x = np.random.default_rng(0).standard_normal((4, d_out)).astype(np.float32)
     x[1, 0] = 2.0 ** 60
@@ -152,14 +160,14 @@ def test_wide_dynamic_range_is_flagged_not_hidden():
 @pytest.mark.parametrize("d_in,d_out,n_act,n_q,T", [(64, 512, 2, 40, 8), (48, 1000, 0, 77, 5), (40, 300, 3, 0, 5),
                                                     (33, 4096, 1, 500, 10), (20, 64, 0, 0, 3), (16, 11008, 1, 88, 4),
                                                     (10, 50, 2, 8 * 50, 4)])
-def test_extract_outliers_bit_exact(dtype, d_in, d_out, n_act, n_q, T):
+def test_extract_outliers_bit_exact(dtype, d_in, d_out, n_act, n_q, T, assignment):
     W, Wu, a, bits = _case(d_in, d_out, dtype, 77 + d_in, 2.5)
     rows, cols, vals = G.gpu_extract(W, a, bits, n_act, n_q, T)
     rr, rc, rv = oracle.extract_outliers(Wu, dtype, a, bits, n_act, n_q, T)
     assert np.array_equal(rows, rr) and np.array_equal(cols, rc) and np.array_equal(vals, rv)
 
 
-def test_extract_outliers_ties_across_rows():
+def test_extract_outliers_ties_across_rows(assignment):
     d_in, d_out = 12, 128
     base = (np.linspace(-1, 1, d_out) ** 3).astype(np.float16)
     Wt = torch.from_numpy(np.tile(base, (d_in, 1))).cuda()
