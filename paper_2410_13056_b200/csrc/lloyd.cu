@@ -29,12 +29,12 @@
 //   output      codes / errors are put back into column order through shared memory and stored
 //               with coalesced writes
 #include "lloyd.cuh"
+#include "lloyd_device.cuh"
 
 #include <atomic>
 
 namespace cmpq {
 
-constexpr int kMaxK = 16;
 constexpr int kMaxWarps = 32;
 constexpr int kSortSlots = 32;  // high-byte buckets refined per pass of the sort's second level
 static_assert(CMPQ_MAX_D_OUT < 65536, "the sort's second-level counters are 16 bits wide");
@@ -49,8 +49,6 @@ struct alignas(16) LloydShared {
     float c[kMaxK];                    // centroids for the next sweep, written by warp 0
     int below_total[kMaxK];            // ordered path: threads of the block entirely below boundary k
     int flag_fast, flag_moved;         // warp 0's decisions: counting sweep valid / a boundary moved
-    int bound[kMaxK + 1];              // ordered search: B_k of the last search, published by warp 0
-    int pub_it, pub_done, pub_sweeps;  // ordered search: updates done, fit finished, searches counted
     int n_nonempty;
     float vmin, vmax;                  // value range of the channel
     float wlo[kMaxWarps], whi[kMaxWarps];
@@ -74,51 +72,6 @@ __host__ __device__ inline bool lloyd_tail_fits_scratch(int nthr, int E) {
 __host__ __device__ inline int lloyd_scratch_bytes(int /*N*/) {
     // 16 KiB = kSortSlots x 256 16-bit counters >= 16 bytes x 1024 threads >= 32768 bits
     return kSortSlots * 128 * (int)sizeof(uint32_t);
-}
-
-template <int DT>
-__device__ __forceinline__ uint32_t sort_key16(float x) {
-    uint32_t h;
-    if (DT == CMPQ_BF16) h = __float_as_uint(x) >> 16;
-    else h = __half_as_ushort(__float2half_rn(x));
-    return (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
-}
-
-template <int DT>
-__device__ __forceinline__ float value_of_key16(uint32_t key) {
-    uint32_t h = (key & 0x8000u) ? (key & 0x7fffu) : (~key & 0xffffu);
-    return widen16<DT>((uint16_t)h);
-}
-
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-// exclusive prefix of 256 counters by one warp (8 per lane, in place allowed); returns the total
-__device__ __forceinline__ int warp_scan256(const int* in, int* out_excl) {
-    const int lane = threadIdx.x & 31;
-    int v[8], s = 0;
-#pragma unroll
-    for (int t = 0; t < 8; ++t) { v[t] = in[lane * 8 + t]; s += v[t]; }
-    int incl = s;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    int run = incl - s;
-    __syncwarp();
-#pragma unroll
-    for (int t = 0; t < 8; ++t) { out_excl[lane * 8 + t] = run; run += v[t]; }
-    return __shfl_sync(0xffffffffu, incl, 31);
 }
 
 // In-place exclusive prefix of 256 16-bit counters packed two per word (128 words, 16-byte
@@ -146,19 +99,6 @@ __device__ __forceinline__ void warp_scan256_packed(uint32_t* h) {
         w[t] = lo | (hi << 16);
     }
     reinterpret_cast<uint4*>(h)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
-}
-
-// Code of one weight by the defining scan: first k minimising |x - c_k|.
-template <int K>
-__device__ __forceinline__ int nearest_scan(float x, const float (&c)[K]) {
-    float best = fabsf(x - c[0]);
-    int bk = 0;
-#pragma unroll
-    for (int k = 1; k < K; ++k) {
-        float d = fabsf(x - c[k]);
-        if (d < best) { best = d; bk = k; }
-    }
-    return bk;
 }
 
 // Sorts the block's weights by 16-bit key into `sorted` (key << 16 | column).  key[e] belongs to
@@ -228,17 +168,6 @@ __device__ void sort_channel(const uint32_t (&key)[E], int nval, LloydShared& sh
         }
         __syncthreads();
     }
-}
-
-// Whether the counting sweep is valid for the centroids (lane k holds c_k): strictly increasing
-// with every gap above 2^-22 of the channel's value range.  Same answer in every lane.
-template <int K>
-__device__ __forceinline__ bool counting_sweep_valid(float ck_lane, double need) {
-    const int lane = threadIdx.x & 31;
-    float ck = __shfl_sync(0xffffffffu, ck_lane, lane < K ? lane : K - 1);
-    float cp = __shfl_up_sync(0xffffffffu, ck, 1);
-    bool ok = (lane == 0 || lane >= K) ? true : ((double)ck - (double)cp > need);
-    return __all_sync(0xffffffffu, ok);
 }
 
 // Per-warp cluster sums and counts of all weights, from the codes in registers (any order).
@@ -356,74 +285,6 @@ __device__ __forceinline__ float centroid_from_boundaries(LloydShared& sh, const
     }
     B_out = B;
     return centroid_from_runs<DT, K>(sh, sorted, N, ck, B);
-}
-
-// Ordered search, warp 0 (lane k holds c_k; the centroids pass counting_sweep_valid): the
-// predicate fabsf(x - c_k) < fabsf(x - c_{k-1}) is then false on a prefix of the sorted order and true
-// on the rest, so B_k -- the number of weights for which it is false -- is found by probing
-// sorted weights instead of evaluating all of them: every half warp narrows the interval of one
-// boundary by 16 probes per round, two boundaries per round per warp, kBatch pairs interleaved.
-// Returns B_lane for lanes 1..K-1, 0 in lane 0, N in lane K.
-template <int DT, int K>
-__device__ __forceinline__ int search_boundaries(const uint32_t* sorted, int N, float ck_lane) {
-    constexpr int PAIRS = K / 2;
-    constexpr int kBatch = PAIRS < 4 ? PAIRS : 4;
-    const int lane = threadIdx.x & 31, half = lane >> 4, j = lane & 15;
-    int B = (lane == K) ? N : 0;
-#pragma unroll
-    for (int p0 = 0; p0 < PAIRS; p0 += kBatch) {
-        float ck[kBatch], cm[kBatch];
-        int lo[kBatch], hi[kBatch];
-#pragma unroll
-        for (int p = 0; p < kBatch; ++p) {
-            const int k = 1 + 2 * (p0 + p) + half;
-            const int kk = k < K ? k : K - 1;
-            ck[p] = __shfl_sync(0xffffffffu, ck_lane, kk);
-            cm[p] = __shfl_sync(0xffffffffu, ck_lane, kk - 1);
-            lo[p] = 0;
-            hi[p] = k < K ? N : 0;  // k = K has no boundary: empty interval
-        }
-        // an interval of length len shrinks to at most step - 1 per round; the probe stride is made odd
-        // so that the 16 probes of a boundary fall into 16 different shared-memory banks
-        for (int len = N; len > 0; len = (((len + 15) >> 4) | 1) - 1) {
-            // staged so that the kBatch independent chains overlap: addresses and loads, predicates,
-            // votes, interval updates
-            int step[kBatch];
-            float v[kBatch];
-            bool inb[kBatch];
-#pragma unroll
-            for (int p = 0; p < kBatch; ++p) {
-                const int cur = hi[p] - lo[p];
-                step[p] = ((cur + 15) >> 4) | 1;
-                const int pos = lo[p] + j * step[p] + step[p] - 1;
-                inb[p] = pos < hi[p];  // false for an empty interval; positions from hi on are known to be true
-                const int idx = pos < N ? pos : N - 1;
-                v[p] = value_of_key16<DT>(sorted[idx] >> 16);
-            }
-            uint32_t m[kBatch];
-#pragma unroll
-            for (int p = 0; p < kBatch; ++p) {
-                const bool is_false = inb[p] && !(fabsf(v[p] - ck[p]) < fabsf(v[p] - cm[p]));
-                m[p] = __ballot_sync(0xffffffffu, is_false);
-            }
-#pragma unroll
-            for (int p = 0; p < kBatch; ++p) {
-                const int nf = __popc((m[p] >> (16 * half)) & 0xffffu);
-                // an empty interval has nf = 0 and keeps lo = hi
-                lo[p] += nf * step[p];
-                const int cap = lo[p] + step[p] - 1;
-                if (nf < 16) hi[p] = hi[p] < cap ? hi[p] : cap;
-            }
-        }
-#pragma unroll
-        for (int p = 0; p < kBatch; ++p) {
-            const int b0 = __shfl_sync(0xffffffffu, lo[p], 0);
-            const int b1 = __shfl_sync(0xffffffffu, lo[p], 16);
-            if (lane == 1 + 2 * (p0 + p)) B = b0;
-            if (lane == 2 + 2 * (p0 + p) && lane < K) B = b1;
-        }
-    }
-    return B;
 }
 
 // One sweep over a thread's E weights: their codes for the centroids c, packed 8 per word.
@@ -595,128 +456,6 @@ __device__ void fit_channel(const LloydArgs& a, int64_t row, const float (&x)[E]
     write_outputs<E>(a, row, K, sh, sorted, x, cw, nval, sweeps_done);
 }
 
-// The same fit with the ordered search in place of the all-pairs sweeps.  While the centroids pass
-// counting_sweep_valid, warp 0 runs whole iterations alone (search the K-1 boundaries, compare
-// them with the previous ones, update from the prefix table) and the other warps wait at a
-// barrier; an iteration whose centroids fail the test is done by the whole block with the plain
-// scan and per-cluster accumulation, exactly as in fit_channel.  The last assignment turns the
-// final boundaries into codes (or is a plain scan when the final centroids fail the test).
-template <int DT, int K, int E>
-__device__ void fit_channel_ordered(const LloydArgs& a, int64_t row, const float (&x)[E], int nval,
-                                    LloydShared& sh, uint32_t* sorted) {
-    constexpr int WORDS = (E + 7) / 8;
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    const int N = (int)a.d_out;
-    const int T = a.iters;
-    const double need = ((double)sh.vmax - (double)sh.vmin) * (1.0 / 4194304.0);  // range * 2^-22
-
-    // warp 0 only: lane k holds c_k and B_k
-    float ck_lane = 0.f;
-    int B_prev = -1, it0 = 0, searches = 0;
-    bool valid0 = false, conv0 = false;
-    if (warp == 0) {
-        if (lane < K) {
-            int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));  // K evenly spaced order statistics
-            ck_lane = value_of_key16<DT>(sorted[pos] >> 16);
-        }
-        valid0 = counting_sweep_valid<K>(ck_lane, need);
-    }
-
-    uint32_t cw[WORDS];
-#pragma unroll
-    for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;  // no plain sweep yet: the next one counts as a change
-    int plain_sweeps = 0, it_after_plain = -1;
-    bool codes_ready = false;  // cw holds the final codes (a plain sweep that changed nothing)
-    bool valid = false;
-    for (;;) {
-        if (warp == 0) {
-            while (it0 < T && valid0) {
-                const int B = search_boundaries<DT, K>(sorted, N, ck_lane);
-                ++searches;
-                const bool moved = __any_sync(0xffffffffu, lane > 0 && lane < K && B != B_prev);
-                B_prev = B;
-                if (!moved) { conv0 = true; break; }  // same runs as before: the update would repeat itself
-                ck_lane = centroid_from_runs<DT, K>(sh, sorted, N, ck_lane, B);
-                ++it0;
-                valid0 = counting_sweep_valid<K>(ck_lane, need);
-            }
-            if (valid0 && !conv0 && it0 == T) {  // last assignment
-                B_prev = search_boundaries<DT, K>(sorted, N, ck_lane);
-                ++searches;
-            }
-            if (lane < K) sh.c[lane] = ck_lane;
-            if (lane <= K) sh.bound[lane] = B_prev;
-            if (lane == 0) {
-                sh.flag_fast = valid0 ? 1 : 0;
-                sh.pub_it = it0;
-                sh.pub_done = (conv0 || it0 == T) ? 1 : 0;
-                sh.pub_sweeps = searches;
-            }
-        }
-        __syncthreads();
-        valid = sh.flag_fast != 0;
-        if (sh.pub_done) break;
-
-        // the centroids are not safe for the ordered search: one plain iteration by the block
-        const int it_pub = sh.pub_it;
-        if (it_pub != it_after_plain) {  // ordered iterations ran since the last plain sweep: its codes are stale
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) cw[w] = 0xffffffffu;
-        }
-        float c[K];
-#pragma unroll
-        for (int k = 0; k < K; ++k) c[k] = sh.c[k];
-        uint32_t nw[WORDS];
-        sweep_codes<K, E>(x, c, false, nw);
-        ++plain_sweeps;
-        uint32_t any = 0;
-#pragma unroll
-        for (int w = 0; w < WORDS; ++w) { any |= nw[w] ^ cw[w]; cw[w] = nw[w]; }
-        const int changed = __syncthreads_or(any != 0);
-        if (!changed) { codes_ready = true; break; }
-        rebuild_partials<K, E>(x, cw, nval, sh);
-        __syncthreads();
-        if (warp == 0) {
-            ck_lane = centroid_from_partials<K>(sh, ck_lane, nthr >> 5);
-            ++it0;
-            valid0 = counting_sweep_valid<K>(ck_lane, need);
-            B_prev = -1;
-        }
-        it_after_plain = it_pub + 1;
-    }
-
-    if (!codes_ready) {
-        if (valid) {
-            // codes from the final boundaries: position i of the sorted order has code #{k : B_k <= i}
-            const int idx0 = tid * E;
-            int cf = 0, cl = 0;
-#pragma unroll
-            for (int k = 1; k < K; ++k) {
-                const int b = sh.bound[k];
-                cf += (idx0 >= b) ? 1 : 0;
-                cl += (idx0 + E - 1 >= b) ? 1 : 0;
-            }
-#pragma unroll
-            for (int w = 0; w < WORDS; ++w) cw[w] = (uint32_t)cf * 0x11111111u;
-            for (int k = cf + 1; k <= cl; ++k) {
-                const int b = sh.bound[k] - idx0;  // in [1, E-1]
-#pragma unroll
-                for (int e = 0; e < E; ++e)
-                    if (e >= b) cw[e >> 3] += 1u << (4 * (e & 7));
-            }
-        } else {
-            float c[K];
-#pragma unroll
-            for (int k = 0; k < K; ++k) c[k] = sh.c[k];
-            sweep_codes<K, E>(x, c, false, cw);
-            ++plain_sweeps;
-        }
-    }
-    const int sweeps_done = plain_sweeps + sh.pub_sweeps;
-    __syncthreads();  // sh.c holds the final centroids; no thread reads keys from `sorted` after this point
-    write_outputs<E>(a, row, K, sh, sorted, x, cw, nval, sweeps_done);
-}
-
 // One-time work for a channel, by every thread of the block: read the row, zero the removed
 // positions, note the value range and the exactness diagnostics, sort it into `sorted`, load this
 // thread's run of E order statistics into x and build the fp64 prefix table sh.pt4.
@@ -725,94 +464,9 @@ __device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh
                                 uint32_t* sorted, float (&x)[E], int& nval_out) {
     const int N = (int)a.d_out;
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    const int nwarps = nthr >> 5;
-    // removed positions (outliers of this row) are marked in a bitmap over the columns
-    uint32_t* removed = reinterpret_cast<uint32_t*>(scratch);
-    int64_t p0 = 0, p1 = 0;
-    if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
-    const bool has_removed = p1 > p0;
-    if (has_removed) {
-        for (int w = tid; w < (N + 31) / 32; w += nthr) removed[w] = 0;
-        __syncthreads();
-        for (int64_t p = p0 + tid; p < p1; p += nthr) {
-            int col = a.cols[p];
-            atomicOr(&removed[col >> 5], 1u << (col & 31));
-        }
-        __syncthreads();
-    }
-
-    // column layout for the load: thread owns columns (g * nthr + tid) * 4 + u
-    const uint16_t* w = a.W + row * a.ldw;
-    const bool vec = ((a.ldw & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 7) == 0);
     uint32_t key[E];
     int nval_cols = 0;
-    {
-        float lo = __int_as_float(0x7f800000), hi = __int_as_float(0xff800000);
-        int top = -100000, ulp = 100000;
-#pragma unroll
-        for (int g = 0; g < E / 4; ++g) {
-            const int j0 = (g * nthr + tid) * 4;
-            uint16_t h[4] = {0, 0, 0, 0};
-            if (j0 + 3 < N && vec) {
-                uint2 v = *reinterpret_cast<const uint2*>(w + j0);
-                h[0] = (uint16_t)(v.x & 0xffff); h[1] = (uint16_t)(v.x >> 16);
-                h[2] = (uint16_t)(v.y & 0xffff); h[3] = (uint16_t)(v.y >> 16);
-            } else {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (j0 + u < N) h[u] = w[j0 + u];
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int j = j0 + u;
-                float v = widen16<DT>(h[u]);
-                if (j < N) {
-                    ++nval_cols;
-                    if (has_removed && ((removed[j >> 5] >> (j & 31)) & 1)) v = 0.f;
-                    v = (v == 0.f) ? 0.f : v;  // -0 and +0 are the same point
-                    lo = fminf(lo, v);
-                    hi = fmaxf(hi, v);
-                    uint32_t ub = __float_as_uint(v) & 0x7fffffffu;
-                    if (ub) {
-                        int ex = (int)(ub >> 23);
-                        uint32_t m = ub & 0x7fffffu;
-                        int t, q;
-                        if (ex) { t = ex - 127; q = ex - 150 + (__ffs(m | 0x800000u) - 1); }
-                        else    { t = (31 - __clz(m)) - 149; q = (__ffs(m) - 1) - 149; }
-                        top = max(top, t);
-                        ulp = min(ulp, q);
-                    }
-                }
-                key[4 * g + u] = sort_key16<DT>(v);
-            }
-        }
-        // value range (for the gap test) and exactness diagnostics
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
-            top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
-            ulp = min(ulp, __shfl_xor_sync(0xffffffffu, ulp, o));
-        }
-        if (lane == 0) { sh.wlo[warp] = lo; sh.whi[warp] = hi; sh.wtop[warp] = top; sh.wulp[warp] = ulp; }
-        __syncthreads();  // also: every thread is done with the removed-column bitmap
-        if (tid == 0) {
-            for (int wv = 1; wv < nwarps; ++wv) {
-                lo = fminf(lo, sh.wlo[wv]);
-                hi = fmaxf(hi, sh.whi[wv]);
-                top = max(top, sh.wtop[wv]);
-                ulp = min(ulp, sh.wulp[wv]);
-            }
-            sh.vmin = lo;
-            sh.vmax = hi;
-            if (a.inexact_rows && top > -100000) {
-                // sums and differences of up to 2N weights stay exact in fp64 while
-                // 2 N 2^(top+1) / 2^ulp <= 2^53
-                int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
-                if (log2n + 1 + (top + 1 - ulp) > 53) atomicAdd(a.inexact_rows, 1);
-            }
-        }
-    }
+    load_channel_keys<DT, E>(a, row, sh, reinterpret_cast<uint32_t*>(scratch), key, nval_cols);
 
     sort_channel<E>(key, nval_cols, sh, reinterpret_cast<int*>(scratch), sorted);
 
@@ -856,7 +510,7 @@ __device__ void prepare_channel(const LloydArgs& a, int64_t row, LloydShared& sh
     nval_out = nval;
 }
 
-template <int DT, int E, int MAXT, int MINB, bool ORDERED>
+template <int DT, int E, int MAXT, int MINB>
 __global__ void __launch_bounds__(MAXT, MINB)
 lloyd_kernel(const LloydArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -885,15 +539,9 @@ lloyd_kernel(const LloydArgs a) {
 
     uint32_t* codes_s = reinterpret_cast<uint32_t*>(scratch);  // [nthr][WORDS], at most 16 KiB
     const int bits = a.bits[row];
-    if (ORDERED) {
-        if (bits == 2) fit_channel_ordered<DT, 4, E>(a, row, x, nval, sh, sorted);
-        else if (bits == 3) fit_channel_ordered<DT, 8, E>(a, row, x, nval, sh, sorted);
-        else fit_channel_ordered<DT, 16, E>(a, row, x, nval, sh, sorted);
-    } else {
-        if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
-        else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
-        else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
-    }
+    if (bits == 2) fit_channel<DT, 4, E>(a, row, x, nval, sh, codes_s, sorted);
+    else if (bits == 3) fit_channel<DT, 8, E>(a, row, x, nval, sh, codes_s, sorted);
+    else fit_channel<DT, 16, E>(a, row, x, nval, sh, codes_s, sorted);
 }
 
 static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
@@ -905,7 +553,7 @@ static size_t lloyd_smem_bytes(int64_t d_out, int threads, int E) {
 template <int DT, int E, int MAXT, int MINB>
 static cmpq_status launch_variant(const LloydArgs& args, int threads, cudaStream_t st) {
     const size_t smem = lloyd_smem_bytes(args.d_out, threads, E);
-    auto kern = args.all_pairs ? lloyd_kernel<DT, E, MAXT, MINB, false> : lloyd_kernel<DT, E, MAXT, MINB, true>;
+    auto kern = lloyd_kernel<DT, E, MAXT, MINB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
     kern<<<(unsigned)args.d_in, threads, smem, st>>>(args);
@@ -957,8 +605,10 @@ cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64
     return launch_status();
 }
 
-size_t quantize_ws_bytes(int64_t d_in, int64_t) {
-    return round_up((size_t)(d_in + 1) * sizeof(int64_t), 256);
+static size_t row_ptr_bytes(int64_t d_in) { return round_up((size_t)(d_in + 1) * sizeof(int64_t), 256); }
+
+size_t quantize_ws_bytes(int64_t d_in, int64_t d_out) {
+    return row_ptr_bytes(d_in) + lloyd_tables_bytes(d_in, d_out);
 }
 
 }  // namespace cmpq
@@ -1003,6 +653,6 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
     a.codes = codes;
     a.inexact_rows = inexact_rows;
     a.sweeps = sweeps;
-    a.all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
-    return launch_lloyd(a, dt, st);
+    if (lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS) return launch_lloyd(a, dt, st);
+    return launch_lloyd_ordered(a, dt, static_cast<char*>(ws) + row_ptr_bytes(d_in), lloyd_tables_bytes(d_in, d_out), st);
 }

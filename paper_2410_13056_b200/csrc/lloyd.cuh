@@ -22,13 +22,19 @@ struct LloydArgs {
     uint8_t* codes;          // [d_in][d_out] or NULL
     int32_t* inexact_rows;   // optional counter
     unsigned long long* sweeps;  // optional counter of distance evaluations
-    bool all_pairs;          // assignment by evaluating every (weight, centroid) pair
 };
 
 // The process-wide choice made by cmpq_set_lloyd_assignment.
 cmpq_lloyd_assignment lloyd_assignment();
 
+// All-pairs formulation: one fused kernel, every iteration evaluates every (weight, centroid) pair.
 cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
+
+// Ordered formulation: value table per channel, warp-per-channel iterations, streaming last
+// assignment.  `tables` is device scratch of lloyd_tables_bytes(d_in, d_out) bytes, 256-byte aligned.
+size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out);
+cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,
+                                 cudaStream_t st);
 
 // Fills row_ptr[0..d_in] from a row-sorted coordinate list.
 cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64_t* row_ptr,

@@ -1,0 +1,524 @@
+// Channel-wise K-means of CMPQ (Section 3.2.1: K-means per channel W_{i,:} with K = 2^bits;
+// Section 3: each weight is replaced by its nearest centroid) -- the ordered formulation.
+//
+// A channel of 16-bit weights is fully described by how often each 16-bit value occurs.  Three
+// kernels use that:
+//
+//   lloyd_table_kernel    one block per channel: reads the row from HBM once, sets the removed
+//                         positions to +0, counts the values with a two-level histogram in shared
+//                         memory (high byte, then low byte inside the non-empty high-byte buckets)
+//                         and writes the DISTINCT values in ascending order with, for each, the
+//                         number and the fp64 sum of all smaller weights (exclusive prefixes).
+//   lloyd_iterate_kernel  one WARP per channel, all iterations.  While the centroids are strictly
+//                         increasing with gaps above 2^-22 of the value range, the predicate
+//                         fabsf(x - c_k) < fabsf(x - c_{k-1}) is false on a prefix of the ascending
+//                         values and true on the rest, and the first k minimising fabsf(x - c_k) is
+//                         the number of k >= 1 for which it is true.  Cluster k is then a run of the
+//                         table: a half warp finds the first entry where predicate k holds with 16
+//                         probes per round, and the cluster's count and sum are differences of the
+//                         prefixes at two such entries.  Centroids that fail the test are handled
+//                         by the plain first-minimum scan over the distinct values.  The sums are
+//                         count x value products added in fp64: exact for 16-bit weights of bounded
+//                         dynamic range, hence equal to the sums taken weight by weight.
+//   lloyd_assign_kernel   streams the row once more and applies the defining rule (first k
+//                         minimising fabsf(x - c_k), fp32) to every weight with the final centroids:
+//                         codes or errors leave in column order, no staging.
+//
+// Nothing here is a dense contraction, so no tensor cores are used.
+#include "lloyd.cuh"
+#include "lloyd_device.cuh"
+
+namespace cmpq {
+
+constexpr int kSlots = 32;       // high-byte buckets refined per pass of the second histogram level
+constexpr int kSlotWords = 128;  // 256 low-byte counters of 16 bits, two per word
+static_assert(CMPQ_MAX_D_OUT < 65536, "second-level counters and count prefixes are 16 bits wide");
+
+struct ChannelHeader {
+    int M;             // distinct values of the channel
+    float vmin, vmax;  // its value range
+    int pad;
+};
+
+// Per channel: `stride` entries (M used, entry M is a sentinel holding the totals).
+struct Tables {
+    int64_t stride;
+    ChannelHeader* hdr;  // [d_in]
+    uint16_t* keys;      // [d_in][stride] sort keys of the distinct values, ascending
+    uint16_t* cum;       // [d_in][stride] number of weights below the entry's value
+    double* sum;         // [d_in][stride] fp64 sum of the weights below the entry's value
+    float* lut;          // [d_in][16] centroids for the assign kernel when the caller wants no lut
+};
+
+static int64_t table_stride(int64_t d_out) { return (d_out + 1 + 7) / 8 * 8; }
+
+static Tables carve_tables(Workspace& w, int64_t d_in, int64_t d_out) {
+    Tables t;
+    t.stride = table_stride(d_out);
+    t.hdr = w.take<ChannelHeader>(d_in);
+    t.keys = w.take<uint16_t>((size_t)d_in * t.stride);
+    t.cum = w.take<uint16_t>((size_t)d_in * t.stride);
+    t.sum = w.take<double>((size_t)d_in * t.stride);
+    t.lut = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
+    return t;
+}
+
+size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out) {
+    Workspace w(nullptr, 0);
+    carve_tables(w, d_in, d_out);
+    return w.used;
+}
+
+// ------------------------------------------------------------------------------------------------
+// value table of one channel
+
+struct alignas(16) TableShared {
+    int hist1[256];
+    int bucket_rank[256];  // rank of a high-byte bucket among the non-empty ones, or -1
+    int slot_hi[256];      // the inverse: high byte of the r-th non-empty bucket
+    int n_nonempty;
+    float vmin, vmax;
+    float wlo[32], whi[32];
+    int wtop[32], wulp[32];
+    int w_nz[32], w_cnt[32];  // per-warp totals of the block scan
+    double w_sum[32];
+    int base_nz, base_cnt;    // entries / weights / sum emitted by the previous passes
+    double base_sum;
+};
+// dynamic shared memory after TableShared: kSlots * kSlotWords words (removed-column bitmap during
+// the load, second-level counters afterwards)
+
+template <int DT, int E, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
+lloyd_table_kernel(const LloydArgs a, const Tables t) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int64_t row = blockIdx.x;
+    if (a.skip_row && a.skip_row[row]) return;
+    TableShared& sh = *reinterpret_cast<TableShared*>(smem_raw);
+    uint32_t* h2 = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TableShared));
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+
+    uint32_t key[E];
+    int nval = 0;
+    load_channel_keys<DT, E>(a, row, sh, h2, key, nval);
+
+    // first level: which high bytes occur
+    for (int b = tid; b < 256; b += nthr) sh.hist1[b] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nval) atomicAdd(&sh.hist1[key[e] >> 8], 1);
+    __syncthreads();
+    if (warp == 0) {
+        int flag[8], s = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { flag[u] = sh.hist1[lane * 8 + u] > 0; s += flag[u]; }
+        int incl = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        int run = incl - s;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            sh.bucket_rank[lane * 8 + u] = flag[u] ? run : -1;
+            if (flag[u]) sh.slot_hi[run] = lane * 8 + u;
+            run += flag[u];
+        }
+        if (lane == 31) { sh.n_nonempty = incl; sh.base_nz = 0; sh.base_cnt = 0; sh.base_sum = 0.0; }
+    }
+    __syncthreads();
+
+    uint16_t* keys = t.keys + row * t.stride;
+    uint16_t* cum = t.cum + row * t.stride;
+    double* sum = t.sum + row * t.stride;
+    const int n_nonempty = sh.n_nonempty;
+    int run_nz = 0, run_cnt = 0;
+    double run_sum = 0.0;
+    for (int g0 = 0; g0 < n_nonempty; g0 += kSlots) {
+        const int nslots = n_nonempty - g0 < kSlots ? n_nonempty - g0 : kSlots;
+        const int words_total = nslots * kSlotWords;
+        // Second level: the low byte inside the buckets g0 .. g0 + nslots.  Two 16-bit counters share a
+        // word (a channel has fewer than 2^16 weights, so the halves never carry into each other).
+        for (int w = tid; w < words_total / 4; w += nthr) reinterpret_cast<uint4*>(h2)[w] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();  // also: the previous pass has published its bases
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (e < nval) {
+                const int r = sh.bucket_rank[key[e] >> 8] - g0;
+                const uint32_t lo = key[e] & 0xffu;
+                if (r >= 0 && r < kSlots) atomicAdd(&h2[r * kSlotWords + (lo >> 1)], 1u << (16 * (lo & 1u)));
+            }
+        }
+        __syncthreads();
+        // Every thread owns a contiguous range of counters: totals first, a block scan, then the entries.
+        const int w0 = (int)((long long)tid * words_total / nthr);
+        const int w1 = (int)((long long)(tid + 1) * words_total / nthr);
+        int nz = 0, cnt = 0;
+        double s = 0.0;
+        for (int w = w0; w < w1; ++w) {
+            const uint32_t word = h2[w];
+            if (word) {
+                const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
+                const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
+                if (c0) { ++nz; cnt += c0; s += (double)c0 * (double)value_of_key16<DT>(kb); }
+                if (c1) { ++nz; cnt += c1; s += (double)c1 * (double)value_of_key16<DT>(kb | 1u); }
+            }
+        }
+        int inz = nz, icnt = cnt;
+        double isum = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int unz = __shfl_up_sync(0xffffffffu, inz, o);
+            const int ucnt = __shfl_up_sync(0xffffffffu, icnt, o);
+            const double usum = __shfl_up_sync(0xffffffffu, isum, o);
+            if (lane >= o) { inz += unz; icnt += ucnt; isum += usum; }
+        }
+        if (lane == 31) { sh.w_nz[warp] = inz; sh.w_cnt[warp] = icnt; sh.w_sum[warp] = isum; }
+        __syncthreads();
+        double esum = __shfl_up_sync(0xffffffffu, isum, 1);  // exclusive prefix inside the warp
+        if (lane == 0) esum = 0.0;
+        run_nz = sh.base_nz + inz - nz;
+        run_cnt = sh.base_cnt + icnt - cnt;
+        run_sum = sh.base_sum + esum;
+        for (int wv = 0; wv < warp; ++wv) { run_nz += sh.w_nz[wv]; run_cnt += sh.w_cnt[wv]; run_sum += sh.w_sum[wv]; }
+        for (int w = w0; w < w1; ++w) {
+            const uint32_t word = h2[w];
+            if (word) {
+                const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
+                const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
+                if (c0) {
+                    keys[run_nz] = (uint16_t)kb; cum[run_nz] = (uint16_t)run_cnt; sum[run_nz] = run_sum;
+                    ++run_nz; run_cnt += c0; run_sum += (double)c0 * (double)value_of_key16<DT>(kb);
+                }
+                if (c1) {
+                    keys[run_nz] = (uint16_t)(kb | 1u); cum[run_nz] = (uint16_t)run_cnt; sum[run_nz] = run_sum;
+                    ++run_nz; run_cnt += c1; run_sum += (double)c1 * (double)value_of_key16<DT>(kb | 1u);
+                }
+            }
+        }
+        __syncthreads();  // every thread has read the bases and the counters of this pass
+        if (tid == nthr - 1) { sh.base_nz = run_nz; sh.base_cnt = run_cnt; sh.base_sum = run_sum; }
+    }
+    if (tid == nthr - 1) {
+        // the last thread's running values are the totals: sentinel entry and header
+        keys[run_nz] = 0xffffu;
+        cum[run_nz] = (uint16_t)run_cnt;
+        sum[run_nz] = run_sum;
+        ChannelHeader h;
+        h.M = run_nz; h.vmin = sh.vmin; h.vmax = sh.vmax; h.pad = 0;
+        t.hdr[row] = h;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// iterations: one warp per channel
+
+struct IterArgs {
+    Tables t;
+    const uint8_t* bits;
+    const uint8_t* skip_row;
+    int64_t d_in, d_out;
+    int iters;
+    float* lut;  // [d_in][16]
+    unsigned long long* sweeps;
+};
+
+// Lane k (1..K-1) receives e_k = the number of table entries for whose value the predicate
+// fabsf(x - c_k) < fabsf(x - c_{k-1}) is false (a prefix of the table); lane 0 receives 0, lane K
+// receives M.  A half warp narrows one boundary's interval by 16 probes per round; kBatch pairs
+// of boundaries are interleaved so that their loads overlap.
+template <int DT, int K>
+__device__ __forceinline__ int search_entries(const uint16_t* __restrict__ keys, int M, float ck_lane) {
+    constexpr int PAIRS = K / 2;
+    constexpr int kBatch = PAIRS < 4 ? PAIRS : 4;
+    const int lane = threadIdx.x & 31, half = lane >> 4, j = lane & 15;
+    int out = (lane == K) ? M : 0;
+#pragma unroll
+    for (int p0 = 0; p0 < PAIRS; p0 += kBatch) {
+        float ck[kBatch], cm[kBatch];
+        int lo[kBatch], hi[kBatch];
+#pragma unroll
+        for (int p = 0; p < kBatch; ++p) {
+            const int k = 1 + 2 * (p0 + p) + half;
+            const int kk = k < K ? k : K - 1;
+            ck[p] = __shfl_sync(0xffffffffu, ck_lane, kk);
+            cm[p] = __shfl_sync(0xffffffffu, ck_lane, kk - 1);
+            lo[p] = 0;
+            hi[p] = k < K ? M : 0;  // k = K has no boundary: empty interval
+        }
+        // an interval of length len shrinks to at most step - 1 per round
+        for (int len = M; len > 0; len = ((len + 15) >> 4) - 1) {
+            int step[kBatch];
+            float v[kBatch];
+            bool inb[kBatch];
+#pragma unroll
+            for (int p = 0; p < kBatch; ++p) {
+                step[p] = (hi[p] - lo[p] + 15) >> 4;
+                const int pos = lo[p] + j * step[p] + step[p] - 1;
+                // false for an empty interval (step 0); entries from hi on are known to be true
+                inb[p] = step[p] > 0 && pos < hi[p];
+                const int idx = pos < 0 ? 0 : (pos < M ? pos : M - 1);
+                v[p] = value_of_key16<DT>(__ldg(keys + idx));
+            }
+            uint32_t m[kBatch];
+#pragma unroll
+            for (int p = 0; p < kBatch; ++p) {
+                const bool is_false = inb[p] && !(fabsf(v[p] - ck[p]) < fabsf(v[p] - cm[p]));
+                m[p] = __ballot_sync(0xffffffffu, is_false);
+            }
+#pragma unroll
+            for (int p = 0; p < kBatch; ++p) {
+                const int nf = __popc((m[p] >> (16 * half)) & 0xffffu);
+                if (step[p] > 0) {
+                    lo[p] += nf * step[p];
+                    const int cap = lo[p] + step[p] - 1;
+                    hi[p] = hi[p] < cap ? hi[p] : cap;
+                }
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < kBatch; ++p) {
+            const int b0 = __shfl_sync(0xffffffffu, lo[p], 0);
+            const int b1 = __shfl_sync(0xffffffffu, lo[p], 16);
+            if (lane == 1 + 2 * (p0 + p)) out = b0;
+            if (lane == 2 + 2 * (p0 + p) && lane < K) out = b1;
+        }
+    }
+    return out;
+}
+
+template <int DT, int K>
+__device__ void iterate_channel(const IterArgs& a, int64_t row) {
+    const int lane = threadIdx.x & 31;
+    const ChannelHeader h = a.t.hdr[row];
+    const int N = (int)a.d_out, T = a.iters;
+    const int M = h.M < 1 ? 1 : (h.M > N ? N : h.M);  // 1 <= M <= N by construction
+    const uint16_t* __restrict__ keys = a.t.keys + row * a.t.stride;
+    const uint16_t* __restrict__ cum = a.t.cum + row * a.t.stride;
+    const double* __restrict__ sum = a.t.sum + row * a.t.stride;
+    const double need = ((double)h.vmax - (double)h.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+
+    // start: K evenly spaced order statistics; the weight at sorted position pos has the value of the
+    // entry e with cum[e] <= pos < cum[e + 1]
+    float ck = 0.f;
+    if (lane < K) {
+        const int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));
+        int lo = 0, hi = M;  // cum[lo] <= pos < cum[hi]   (cum[0] = 0, cum[M] = N)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((int)__ldg(cum + mid) <= pos) lo = mid; else hi = mid;
+        }
+        ck = value_of_key16<DT>(__ldg(keys + lo));
+    }
+    __syncwarp();
+
+    int updates = 0;
+    while (updates < T) {
+        float cn = ck;
+        if (counting_sweep_valid<K>(ck, need)) {
+            const int e = search_entries<DT, K>(keys, M, ck);
+            int B = 0;
+            double P = 0.0;
+            if (lane <= K) { B = (int)__ldg(cum + e); P = __ldg(sum + e); }
+            const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
+            const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
+            if (lane < K) {
+                const int cnt = Bn - B;
+                if (cnt > 0) cn = __double2float_rn(__ddiv_rn(Pn - P, (double)cnt));
+            }
+        } else {
+            // plain rule on every distinct value; cluster sums as count x value in fp64
+            float c[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k) c[k] = __shfl_sync(0xffffffffu, ck, k);
+            double s[K];
+            int n[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k) { s[k] = 0.0; n[k] = 0; }
+            for (int j = lane; j < M; j += 32) {
+                const float v = value_of_key16<DT>(__ldg(keys + j));
+                const int cnt = (int)__ldg(cum + j + 1) - (int)__ldg(cum + j);
+                const int code = nearest_scan<K>(v, c);
+                const double prod = (double)cnt * (double)v;
+#pragma unroll
+                for (int k = 0; k < K; ++k)
+                    if (code == k) { s[k] += prod; n[k] += cnt; }
+            }
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const double sk = warp_sum(s[k]);
+                const int nk = warp_sum(n[k]);
+                if (lane == k && nk > 0) cn = __double2float_rn(__ddiv_rn(sk, (double)nk));
+            }
+        }
+        ++updates;
+        const bool same = __all_sync(0xffffffffu, lane >= K || __float_as_uint(cn) == __float_as_uint(ck));
+        ck = cn;
+        if (same) break;  // identical centroids: every later iteration repeats this one
+    }
+    if (lane < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + lane] = lane < K ? ck : 0.f;
+    // assignments made: one per update, and the last one by the assign kernel
+    if (a.sweeps && lane == 0)
+        atomicAdd(a.sweeps, (unsigned long long)(updates + 1) * (unsigned long long)N * (unsigned long long)K);
+}
+
+constexpr int kIterWarps = 4;
+
+template <int DT>
+__global__ void __launch_bounds__(kIterWarps * 32, 8)
+lloyd_iterate_kernel(const IterArgs a) {
+    const int64_t row = (int64_t)blockIdx.x * kIterWarps + (threadIdx.x >> 5);
+    if (row >= a.d_in) return;
+    if (a.skip_row && a.skip_row[row]) return;
+    const int bits = a.bits[row];
+    if (bits == 2) iterate_channel<DT, 4>(a, row);
+    else if (bits == 3) iterate_channel<DT, 8>(a, row);
+    else iterate_channel<DT, 16>(a, row);
+}
+
+// ------------------------------------------------------------------------------------------------
+// last assignment
+
+constexpr int kAssignThreads = 256;
+
+template <int DT, int K>
+__device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut, const uint32_t* removed,
+                           bool has_removed) {
+    const int N = (int)a.d_out;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    float c[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
+    const uint16_t* w = a.W + row * a.ldw;
+    const bool vec_in = ((a.ldw & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 7) == 0);
+    const bool vec_out = (N & 3) == 0;
+    uint8_t* codes = a.codes ? a.codes + row * a.d_out : nullptr;
+    float* err = a.err ? a.err + row * a.d_out : nullptr;
+    for (int j0 = tid * 4; j0 < N; j0 += nthr * 4) {
+        uint16_t h[4] = {0, 0, 0, 0};
+        if (j0 + 3 < N && vec_in) {
+            const uint2 v = *reinterpret_cast<const uint2*>(w + j0);
+            h[0] = (uint16_t)(v.x & 0xffff); h[1] = (uint16_t)(v.x >> 16);
+            h[2] = (uint16_t)(v.y & 0xffff); h[3] = (uint16_t)(v.y >> 16);
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (j0 + u < N) h[u] = w[j0 + u];
+        }
+        uint32_t code[4];
+        float dist[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + u;
+            float x = widen16<DT>(h[u]);
+            if (has_removed && j < N && ((removed[j >> 5] >> (j & 31)) & 1)) x = 0.f;
+            x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
+            float best = fabsf(x - c[0]);
+            uint32_t bk = 0;
+#pragma unroll
+            for (int k = 1; k < K; ++k) {
+                const float d = fabsf(x - c[k]);
+                if (d < best) { best = d; bk = k; }
+            }
+            code[u] = bk;
+            dist[u] = best;
+        }
+        if (j0 + 3 < N && vec_out) {
+            if (codes) *reinterpret_cast<uint32_t*>(codes + j0) = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
+            if (err) *reinterpret_cast<float4*>(err + j0) = make_float4(dist[0], dist[1], dist[2], dist[3]);
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (j0 + u < N) {
+                    if (codes) codes[j0 + u] = (uint8_t)code[u];
+                    if (err) err[j0 + u] = dist[u];
+                }
+            }
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kAssignThreads)
+lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut) {
+    __shared__ uint32_t removed[CMPQ_MAX_D_OUT / 32];
+    const int64_t row = blockIdx.x;
+    if (a.skip_row && a.skip_row[row]) return;
+    const int N = (int)a.d_out;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    int64_t p0 = 0, p1 = 0;
+    if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
+    const bool has_removed = p1 > p0;
+    if (has_removed) {
+        for (int w = tid; w < (N + 31) / 32; w += nthr) removed[w] = 0;
+        __syncthreads();
+        for (int64_t p = p0 + tid; p < p1; p += nthr) {
+            const int col = a.cols[p];
+            atomicOr(&removed[col >> 5], 1u << (col & 31));
+        }
+        __syncthreads();
+    }
+    const int bits = a.bits[row];
+    if (bits == 2) assign_row<DT, 4>(a, row, lut, removed, has_removed);
+    else if (bits == 3) assign_row<DT, 8>(a, row, lut, removed, has_removed);
+    else assign_row<DT, 16>(a, row, lut, removed, has_removed);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+
+template <int DT, int E, int MAXT, int MINB>
+static cmpq_status launch_table(const LloydArgs& args, const Tables& t, int threads, cudaStream_t st) {
+    const size_t smem = sizeof(TableShared) + (size_t)kSlots * kSlotWords * sizeof(uint32_t);
+    auto kern = lloyd_table_kernel<DT, E, MAXT, MINB>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return CMPQ_ERR_CUDA;
+    kern<<<(unsigned)args.d_in, threads, smem, st>>>(args, t);
+    return launch_status();
+}
+
+template <int DT>
+static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cudaStream_t st) {
+    const int64_t N = args.d_out;
+    auto threads_for = [N](int e) {
+        int64_t th = (N + e - 1) / e;
+        th = (th + 31) / 32 * 32;
+        return (int)(th < 32 ? 32 : th);
+    };
+    cmpq_status s;
+    if (N <= 2048) s = launch_table<DT, 4, 512, 2>(args, t, threads_for(4), st);
+    else if (N <= 4096) s = launch_table<DT, 16, 256, 4>(args, t, threads_for(16), st);
+    else if (N <= 8192) s = launch_table<DT, 16, 512, 2>(args, t, threads_for(16), st);
+    else if (N <= 16384) s = launch_table<DT, 16, 1024, 1>(args, t, threads_for(16), st);
+    else s = launch_table<DT, 32, 1024, 1>(args, t, threads_for(32), st);
+    if (s != CMPQ_OK) return s;
+
+    IterArgs ia{};
+    ia.t = t;
+    ia.bits = args.bits;
+    ia.skip_row = args.skip_row;
+    ia.d_in = args.d_in;
+    ia.d_out = args.d_out;
+    ia.iters = args.iters;
+    ia.lut = args.lut ? args.lut : t.lut;
+    ia.sweeps = args.sweeps;
+    const unsigned iter_blocks = (unsigned)((args.d_in + kIterWarps - 1) / kIterWarps);
+    lloyd_iterate_kernel<DT><<<iter_blocks, kIterWarps * 32, 0, st>>>(ia);
+    s = launch_status();
+    if (s != CMPQ_OK) return s;
+
+    lloyd_assign_kernel<DT><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut);
+    return launch_status();
+}
+
+cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,
+                                 cudaStream_t st) {
+    if (!tables || tables_bytes < lloyd_tables_bytes(args.d_in, args.d_out)) return CMPQ_ERR_WORKSPACE;
+    Workspace w(tables, tables_bytes);
+    const Tables t = carve_tables(w, args.d_in, args.d_out);
+    return dt == CMPQ_F16 ? launch_ordered_dt<CMPQ_F16>(args, t, st) : launch_ordered_dt<CMPQ_BF16>(args, t, st);
+}
+
+}  // namespace cmpq

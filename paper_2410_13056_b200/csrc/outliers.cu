@@ -273,6 +273,7 @@ struct OutlierWs {
     int32_t* eq;
     int32_t* take_eq;
     int64_t* row_start;
+    char* tables;  // scratch of the ordered K-means
 };
 
 static OutlierWs carve(Workspace& w, int64_t d_in, int64_t d_out) {
@@ -286,6 +287,7 @@ static OutlierWs carve(Workspace& w, int64_t d_in, int64_t d_out) {
     o.eq = w.take<int32_t>(d_in);
     o.take_eq = w.take<int32_t>(d_in);
     o.row_start = w.take<int64_t>(d_in + 1);
+    o.tables = w.take<char>(lloyd_tables_bytes(d_in, d_out));
     return o;
 }
 
@@ -337,8 +339,9 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
         la.iters = lloyd_iters;
         la.skip_row = o.is_act;
         la.err = o.err;
-        la.all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
-        s = launch_lloyd(la, dt, st);
+        s = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS
+                ? launch_lloyd(la, dt, st)
+                : launch_lloyd_ordered(la, dt, o.tables, lloyd_tables_bytes(d_in, d_out), st);
         if (s != CMPQ_OK) return s;
     }
 
