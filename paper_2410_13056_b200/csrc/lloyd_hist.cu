@@ -8,15 +8,17 @@
 //                         positions to +0, counts the values with a two-level histogram in shared
 //                         memory (high byte, then low byte inside the non-empty high-byte buckets)
 //                         and writes the DISTINCT values in ascending order with, for each, the
-//                         number and the fp64 sum of all smaller weights (exclusive prefixes).
+//                         number of smaller weights (exclusive prefix of the counts).
 //   lloyd_iterate_kernel  one WARP per channel, all iterations.  While the centroids are strictly
 //                         increasing with gaps above 2^-22 of the value range, the predicate
 //                         fabsf(x - c_k) < fabsf(x - c_{k-1}) is false on a prefix of the ascending
 //                         values and true on the rest, and the first k minimising fabsf(x - c_k) is
 //                         the number of k >= 1 for which it is true.  Cluster k is then a run of the
 //                         table: a half warp finds the first entry where predicate k holds with 16
-//                         probes per round, and the cluster's count and sum are differences of the
-//                         prefixes at two such entries.  Centroids that fail the test are handled
+//                         probes per round, and the cluster's count and sum are differences of
+//                         prefix counts and prefix sums at two such entries (the warp builds the
+//                         prefix sums once, at every eighth entry; table and sums stay in shared
+//                         memory when they fit).  Centroids that fail the test are handled
 //                         by the plain first-minimum scan over the distinct values.  The sums are
 //                         count x value products added in fp64: exact for 16-bit weights of bounded
 //                         dynamic range, hence equal to the sums taken weight by weight.
@@ -46,8 +48,9 @@ struct Tables {
     ChannelHeader* hdr;  // [d_in]
     uint16_t* keys;      // [d_in][stride] sort keys of the distinct values, ascending
     uint16_t* cum;       // [d_in][stride] number of weights below the entry's value
-    double* sum;         // [d_in][stride] fp64 sum of the weights below the entry's value
+    double* sum;         // [d_in][stride] scratch of the iterate kernel for tables too large for shared memory
     float* lut;          // [d_in][16] centroids for the assign kernel when the caller wants no lut
+    float* thr;          // [d_in][16] value thresholds of the last assignment ([0]: 1 if valid)
 };
 
 static int64_t table_stride(int64_t d_out) { return (d_out + 1 + 7) / 8 * 8; }
@@ -60,6 +63,7 @@ static Tables carve_tables(Workspace& w, int64_t d_in, int64_t d_out) {
     t.cum = w.take<uint16_t>((size_t)d_in * t.stride);
     t.sum = w.take<double>((size_t)d_in * t.stride);
     t.lut = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
+    t.thr = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
     return t;
 }
 
@@ -81,9 +85,7 @@ struct alignas(16) TableShared {
     float wlo[32], whi[32];
     int wtop[32], wulp[32];
     int w_nz[32], w_cnt[32];  // per-warp totals of the block scan
-    double w_sum[32];
-    int base_nz, base_cnt;    // entries / weights / sum emitted by the previous passes
-    double base_sum;
+    int base_nz, base_cnt;    // entries / weights emitted by the previous passes
 };
 // dynamic shared memory after TableShared: kSlots * kSlotWords words (removed-column bitmap during
 // the load, second-level counters afterwards)
@@ -126,16 +128,14 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
             if (flag[u]) sh.slot_hi[run] = lane * 8 + u;
             run += flag[u];
         }
-        if (lane == 31) { sh.n_nonempty = incl; sh.base_nz = 0; sh.base_cnt = 0; sh.base_sum = 0.0; }
+        if (lane == 31) { sh.n_nonempty = incl; sh.base_nz = 0; sh.base_cnt = 0; }
     }
     __syncthreads();
 
     uint16_t* keys = t.keys + row * t.stride;
     uint16_t* cum = t.cum + row * t.stride;
-    double* sum = t.sum + row * t.stride;
     const int n_nonempty = sh.n_nonempty;
     int run_nz = 0, run_cnt = 0;
-    double run_sum = 0.0;
     for (int g0 = 0; g0 < n_nonempty; g0 += kSlots) {
         const int nslots = n_nonempty - g0 < kSlots ? n_nonempty - g0 : kSlots;
         const int words_total = nslots * kSlotWords;
@@ -156,56 +156,40 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         const int w0 = (int)((long long)tid * words_total / nthr);
         const int w1 = (int)((long long)(tid + 1) * words_total / nthr);
         int nz = 0, cnt = 0;
-        double s = 0.0;
         for (int w = w0; w < w1; ++w) {
             const uint32_t word = h2[w];
-            if (word) {
-                const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
-                const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-                if (c0) { ++nz; cnt += c0; s += (double)c0 * (double)value_of_key16<DT>(kb); }
-                if (c1) { ++nz; cnt += c1; s += (double)c1 * (double)value_of_key16<DT>(kb | 1u); }
-            }
+            const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
+            nz += (c0 ? 1 : 0) + (c1 ? 1 : 0);
+            cnt += c0 + c1;
         }
         int inz = nz, icnt = cnt;
-        double isum = s;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int unz = __shfl_up_sync(0xffffffffu, inz, o);
             const int ucnt = __shfl_up_sync(0xffffffffu, icnt, o);
-            const double usum = __shfl_up_sync(0xffffffffu, isum, o);
-            if (lane >= o) { inz += unz; icnt += ucnt; isum += usum; }
+            if (lane >= o) { inz += unz; icnt += ucnt; }
         }
-        if (lane == 31) { sh.w_nz[warp] = inz; sh.w_cnt[warp] = icnt; sh.w_sum[warp] = isum; }
+        if (lane == 31) { sh.w_nz[warp] = inz; sh.w_cnt[warp] = icnt; }
         __syncthreads();
-        double esum = __shfl_up_sync(0xffffffffu, isum, 1);  // exclusive prefix inside the warp
-        if (lane == 0) esum = 0.0;
         run_nz = sh.base_nz + inz - nz;
         run_cnt = sh.base_cnt + icnt - cnt;
-        run_sum = sh.base_sum + esum;
-        for (int wv = 0; wv < warp; ++wv) { run_nz += sh.w_nz[wv]; run_cnt += sh.w_cnt[wv]; run_sum += sh.w_sum[wv]; }
+        for (int wv = 0; wv < warp; ++wv) { run_nz += sh.w_nz[wv]; run_cnt += sh.w_cnt[wv]; }
         for (int w = w0; w < w1; ++w) {
             const uint32_t word = h2[w];
             if (word) {
                 const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
                 const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-                if (c0) {
-                    keys[run_nz] = (uint16_t)kb; cum[run_nz] = (uint16_t)run_cnt; sum[run_nz] = run_sum;
-                    ++run_nz; run_cnt += c0; run_sum += (double)c0 * (double)value_of_key16<DT>(kb);
-                }
-                if (c1) {
-                    keys[run_nz] = (uint16_t)(kb | 1u); cum[run_nz] = (uint16_t)run_cnt; sum[run_nz] = run_sum;
-                    ++run_nz; run_cnt += c1; run_sum += (double)c1 * (double)value_of_key16<DT>(kb | 1u);
-                }
+                if (c0) { keys[run_nz] = (uint16_t)kb; cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c0; }
+                if (c1) { keys[run_nz] = (uint16_t)(kb | 1u); cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c1; }
             }
         }
         __syncthreads();  // every thread has read the bases and the counters of this pass
-        if (tid == nthr - 1) { sh.base_nz = run_nz; sh.base_cnt = run_cnt; sh.base_sum = run_sum; }
+        if (tid == nthr - 1) { sh.base_nz = run_nz; sh.base_cnt = run_cnt; }
     }
     if (tid == nthr - 1) {
         // the last thread's running values are the totals: sentinel entry and header
         keys[run_nz] = 0xffffu;
         cum[run_nz] = (uint16_t)run_cnt;
-        sum[run_nz] = run_sum;
         ChannelHeader h;
         h.M = run_nz; h.vmin = sh.vmin; h.vmax = sh.vmax; h.pad = 0;
         t.hdr[row] = h;
@@ -230,7 +214,7 @@ struct IterArgs {
 // receives M.  A half warp narrows one boundary's interval by 16 probes per round; kBatch pairs
 // of boundaries are interleaved so that their loads overlap.
 template <int DT, int K>
-__device__ __forceinline__ int search_entries(const uint16_t* __restrict__ keys, int M, float ck_lane) {
+__device__ __forceinline__ int search_entries(const uint16_t* keys, int M, float ck_lane) {
     constexpr int PAIRS = K / 2;
     constexpr int kBatch = PAIRS < 4 ? PAIRS : 4;
     const int lane = threadIdx.x & 31, half = lane >> 4, j = lane & 15;
@@ -260,7 +244,7 @@ __device__ __forceinline__ int search_entries(const uint16_t* __restrict__ keys,
                 // false for an empty interval (step 0); entries from hi on are known to be true
                 inb[p] = step[p] > 0 && pos < hi[p];
                 const int idx = pos < 0 ? 0 : (pos < M ? pos : M - 1);
-                v[p] = value_of_key16<DT>(__ldg(keys + idx));
+                v[p] = value_of_key16<DT>(keys[idx]);
             }
             uint32_t m[kBatch];
 #pragma unroll
@@ -289,15 +273,84 @@ __device__ __forceinline__ int search_entries(const uint16_t* __restrict__ keys,
     return out;
 }
 
+constexpr int kIterWarps = 4;
+constexpr int kIterCap = 2048;  // distinct values of a channel whose table fits the warp's shared memory
+
+struct alignas(16) IterShared {
+    uint16_t keys[kIterCap];
+    uint16_t cum[kIterCap + 8];
+    double coarse[kIterCap / 8 + 1];
+};
+
+// fp64 sum of all weights below entry e (0 <= e <= M): the prefix stored for entry 8 (e / 8)
+// plus at most seven count x value products.
+template <int DT>
+__device__ __forceinline__ double prefix_sum_at(const uint16_t* keys, const uint16_t* cum, const double* coarse,
+                                                int e) {
+    const int j0 = e & ~7;
+    double P = coarse[e >> 3];
+    int c_prev = (int)cum[j0];
+#pragma unroll
+    for (int u = 0; u < 7; ++u) {
+        if (j0 + u < e) {
+            const int c_next = (int)cum[j0 + u + 1];
+            P += (double)(c_next - c_prev) * (double)value_of_key16<DT>(keys[j0 + u]);
+            c_prev = c_next;
+        }
+    }
+    return P;
+}
+
 template <int DT, int K>
-__device__ void iterate_channel(const IterArgs& a, int64_t row) {
+__device__ void iterate_channel(const IterArgs& a, int64_t row, IterShared& sm) {
     const int lane = threadIdx.x & 31;
     const ChannelHeader h = a.t.hdr[row];
     const int N = (int)a.d_out, T = a.iters;
     const int M = h.M < 1 ? 1 : (h.M > N ? N : h.M);  // 1 <= M <= N by construction
-    const uint16_t* __restrict__ keys = a.t.keys + row * a.t.stride;
-    const uint16_t* __restrict__ cum = a.t.cum + row * a.t.stride;
-    const double* __restrict__ sum = a.t.sum + row * a.t.stride;
+    const uint16_t* keys = a.t.keys + row * a.t.stride;
+    const uint16_t* cum = a.t.cum + row * a.t.stride;
+    double* coarse = a.t.sum + row * a.t.stride;  // global scratch, used when the table is too large
+    if (M <= kIterCap) {  // the rows are 16-byte aligned and padded to a multiple of 8 entries
+        for (int i = lane; i < (M + 7) / 8; i += 32)
+            reinterpret_cast<uint4*>(sm.keys)[i] = __ldg(reinterpret_cast<const uint4*>(keys) + i);
+        for (int i = lane; i < (M + 1 + 7) / 8; i += 32)  // with the sentinel cum[M] = d_out
+            reinterpret_cast<uint4*>(sm.cum)[i] = __ldg(reinterpret_cast<const uint4*>(cum) + i);
+        keys = sm.keys;
+        cum = sm.cum;
+        coarse = sm.coarse;
+    }
+    __syncwarp();
+    // prefix sums at every eighth entry: each lane sums a contiguous range of groups of eight entries,
+    // the lane totals are scanned, then every group receives its base
+    {
+        const int groups = (M >> 3) + 1;  // coarse[g] for g = 0 .. M / 8
+        const int per_lane = (groups + 31) / 32;
+        const int g_begin = lane * per_lane;
+        double local = 0.0;
+        for (int g = g_begin; g < g_begin + per_lane && g < groups; ++g) {
+            coarse[g] = local;
+            int c_prev = (int)cum[g * 8 < M ? g * 8 : M];
+            for (int u = 0; u < 8; ++u) {
+                const int j = g * 8 + u;
+                if (j < M) {
+                    const int c_next = (int)cum[j + 1];
+                    local += (double)(c_next - c_prev) * (double)value_of_key16<DT>(keys[j]);
+                    c_prev = c_next;
+                }
+            }
+        }
+        double incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        double base = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) base = 0.0;
+        for (int g = g_begin; g < g_begin + per_lane && g < groups; ++g) coarse[g] += base;
+        __threadfence_block();  // the sums may live in global memory: make them visible to the other lanes
+        __syncwarp();
+    }
     const double need = ((double)h.vmax - (double)h.vmin) * (1.0 / 4194304.0);  // range * 2^-22
 
     // start: K evenly spaced order statistics; the weight at sorted position pos has the value of the
@@ -308,9 +361,9 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row) {
         int lo = 0, hi = M;  // cum[lo] <= pos < cum[hi]   (cum[0] = 0, cum[M] = N)
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if ((int)__ldg(cum + mid) <= pos) lo = mid; else hi = mid;
+            if ((int)cum[mid] <= pos) lo = mid; else hi = mid;
         }
-        ck = value_of_key16<DT>(__ldg(keys + lo));
+        ck = value_of_key16<DT>(keys[lo]);
     }
     __syncwarp();
 
@@ -321,7 +374,7 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row) {
             const int e = search_entries<DT, K>(keys, M, ck);
             int B = 0;
             double P = 0.0;
-            if (lane <= K) { B = (int)__ldg(cum + e); P = __ldg(sum + e); }
+            if (lane <= K) { B = (int)cum[e]; P = prefix_sum_at<DT>(keys, cum, coarse, e); }
             const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
             const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
             if (lane < K) {
@@ -338,8 +391,8 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row) {
 #pragma unroll
             for (int k = 0; k < K; ++k) { s[k] = 0.0; n[k] = 0; }
             for (int j = lane; j < M; j += 32) {
-                const float v = value_of_key16<DT>(__ldg(keys + j));
-                const int cnt = (int)__ldg(cum + j + 1) - (int)__ldg(cum + j);
+                const float v = value_of_key16<DT>(keys[j]);
+                const int cnt = (int)cum[j + 1] - (int)cum[j];
                 const int code = nearest_scan<K>(v, c);
                 const double prod = (double)cnt * (double)v;
 #pragma unroll
@@ -359,23 +412,34 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row) {
         if (same) break;  // identical centroids: every later iteration repeats this one
     }
     if (lane < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + lane] = lane < K ? ck : 0.f;
+    // Last assignment: when the final centroids pass the test, predicate k holds exactly for the values
+    // from the first entry where it is true, so the assign kernel only compares with K-1 thresholds.
+    {
+        const bool ok = counting_sweep_valid<K>(ck, need);
+        float thr = ok ? 1.f : 0.f;
+        if (ok) {
+            const int e = search_entries<DT, K>(keys, M, ck);
+            if (lane > 0 && lane < K) thr = e < M ? value_of_key16<DT>(keys[e]) : __int_as_float(0x7f800000);
+        }
+        if (lane < CMPQ_LUT_STRIDE) a.t.thr[row * CMPQ_LUT_STRIDE + lane] = lane < K ? thr : 0.f;
+    }
     // assignments made: one per update, and the last one by the assign kernel
     if (a.sweeps && lane == 0)
         atomicAdd(a.sweeps, (unsigned long long)(updates + 1) * (unsigned long long)N * (unsigned long long)K);
 }
 
-constexpr int kIterWarps = 4;
-
 template <int DT>
-__global__ void __launch_bounds__(kIterWarps * 32, 8)
+__global__ void __launch_bounds__(kIterWarps * 32, 5)
 lloyd_iterate_kernel(const IterArgs a) {
-    const int64_t row = (int64_t)blockIdx.x * kIterWarps + (threadIdx.x >> 5);
+    __shared__ IterShared sm[kIterWarps];
+    const int warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * kIterWarps + warp;
     if (row >= a.d_in) return;
     if (a.skip_row && a.skip_row[row]) return;
     const int bits = a.bits[row];
-    if (bits == 2) iterate_channel<DT, 4>(a, row);
-    else if (bits == 3) iterate_channel<DT, 8>(a, row);
-    else iterate_channel<DT, 16>(a, row);
+    if (bits == 2) iterate_channel<DT, 4>(a, row, sm[warp]);
+    else if (bits == 3) iterate_channel<DT, 8>(a, row, sm[warp]);
+    else iterate_channel<DT, 16>(a, row, sm[warp]);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -384,13 +448,18 @@ lloyd_iterate_kernel(const IterArgs a) {
 constexpr int kAssignThreads = 256;
 
 template <int DT, int K>
-__device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut, const uint32_t* removed,
-                           bool has_removed) {
+__device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut,
+                           const float* __restrict__ thr, const uint32_t* removed, bool has_removed) {
     const int N = (int)a.d_out;
     const int tid = threadIdx.x, nthr = blockDim.x;
     float c[K];
 #pragma unroll
     for (int k = 0; k < K; ++k) c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
+    // t[0] != 0: the code of x is the number of k >= 1 with x >= t[k] (see lloyd_iterate_kernel)
+    float t[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
+    const bool by_threshold = t[0] != 0.f;
     const uint16_t* w = a.W + row * a.ldw;
     const bool vec_in = ((a.ldw & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 7) == 0);
     const bool vec_out = (N & 3) == 0;
@@ -415,15 +484,28 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
             float x = widen16<DT>(h[u]);
             if (has_removed && j < N && ((removed[j >> 5] >> (j & 31)) & 1)) x = 0.f;
             x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
-            float best = fabsf(x - c[0]);
-            uint32_t bk = 0;
+            if (by_threshold) {
+                uint32_t bk = 0;
+                float cc = c[0];
 #pragma unroll
-            for (int k = 1; k < K; ++k) {
-                const float d = fabsf(x - c[k]);
-                if (d < best) { best = d; bk = k; }
+                for (int k = 1; k < K; ++k) {
+                    const bool ge = x >= t[k];
+                    bk += ge ? 1u : 0u;
+                    cc = ge ? c[k] : cc;  // thresholds ascend: the last one reached is the code's
+                }
+                code[u] = bk;
+                dist[u] = fabsf(x - cc);
+            } else {
+                float best = fabsf(x - c[0]);
+                uint32_t bk = 0;
+#pragma unroll
+                for (int k = 1; k < K; ++k) {
+                    const float d = fabsf(x - c[k]);
+                    if (d < best) { best = d; bk = k; }
+                }
+                code[u] = bk;
+                dist[u] = best;
             }
-            code[u] = bk;
-            dist[u] = best;
         }
         if (j0 + 3 < N && vec_out) {
             if (codes) *reinterpret_cast<uint32_t*>(codes + j0) = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
@@ -442,7 +524,7 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
 
 template <int DT>
 __global__ void __launch_bounds__(kAssignThreads)
-lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut) {
+lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut, const float* __restrict__ thr) {
     __shared__ uint32_t removed[CMPQ_MAX_D_OUT / 32];
     const int64_t row = blockIdx.x;
     if (a.skip_row && a.skip_row[row]) return;
@@ -461,9 +543,9 @@ lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut) {
         __syncthreads();
     }
     const int bits = a.bits[row];
-    if (bits == 2) assign_row<DT, 4>(a, row, lut, removed, has_removed);
-    else if (bits == 3) assign_row<DT, 8>(a, row, lut, removed, has_removed);
-    else assign_row<DT, 16>(a, row, lut, removed, has_removed);
+    if (bits == 2) assign_row<DT, 4>(a, row, lut, thr, removed, has_removed);
+    else if (bits == 3) assign_row<DT, 8>(a, row, lut, thr, removed, has_removed);
+    else assign_row<DT, 16>(a, row, lut, thr, removed, has_removed);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -509,7 +591,7 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cud
     s = launch_status();
     if (s != CMPQ_OK) return s;
 
-    lloyd_assign_kernel<DT><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut);
+    lloyd_assign_kernel<DT><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
     return launch_status();
 }
 
