@@ -27,6 +27,9 @@ METRIC_BUDGET = 3.0          # the metric is quoted at an average of 3.0 bits
 SM_COUNT, FP32_LANES_PER_SM = 148, 128
 CPU_BASELINE_CHANNELS = 4096   # cpu_baseline leg: the whole layer (about 15 s on one core)
 REFERENCE_ARM_CHANNELS = 1024  # --impl reference: a quarter of the layer per step
+# dram__bytes_read.sum + dram__bytes_write.sum of lloyd_table_kernel per weight, from the ncu capture
+# summarised under profiles/ (None while no capture of the current kernel exists)
+LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT = None
 
 
 def _peaks():
@@ -156,7 +159,8 @@ def main():
         return
 
     import torch
-    from paper_2410_13056_b200.pipeline import LayerQuantizer, KERNELS_PER_RUN
+    from paper_2410_13056_b200 import binding as B
+    from paper_2410_13056_b200.pipeline import LayerQuantizer, kernels_per_run
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -205,32 +209,79 @@ def main():
     ms = timed(METRIC_BUDGET, steps, events)
     clocks = sampler.stop()
     value = world * params / (ms * 1e-3) / 1e6
-    sweeps_evals = int(q.counters[1].item())
     per_call = {}
     for name in events[0]:
-        per_call[name] = statistics.mean(e[name][0].elapsed_time(e[name][1]) for e in events)
+        if name != "final_fit_kernels":
+            per_call[name] = statistics.mean(e[name][0].elapsed_time(e[name][1]) for e in events)
+    phases = [e["final_fit_kernels"] for e in events]
+    kernel_ms = {
+        "lloyd_table_kernel": statistics.mean(p[0].elapsed_time(p[1]) for p in phases),
+        "lloyd_iterate_kernel": statistics.mean(p[1].elapsed_time(p[2]) for p in phases),
+        "lloyd_assign_kernel": statistics.mean(p[2].elapsed_time(p[3]) for p in phases),
+    }
     ms_22 = timed(cfg.budgets[0], max(3, steps // 2))
 
-    # roofline of the dominant kernel: the channel K-means of the final fit (cmpq_quantize_layer is
-    # that kernel plus a microsecond-sized index kernel); 2 ops (subtract, compare/select) per
-    # (weight, centroid) distance evaluation actually executed
+    # Roofline of the dominant kernel.  With the default (ordered) assignment a K-means call is three
+    # kernels, timed live by events the library records between them; the value-table kernel takes
+    # the largest share of a step (it runs in both fits).  It has to read every weight once (2 B)
+    # and nothing else of comparable size, so it is held against the HBM peak.
     hbm_peak, sm_max_mhz, peak_kind = _peaks()
-    alu_peak_tflops = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
-    lloyd_ms = per_call["cmpq_quantize_layer"]
-    achieved = 2.0 * sweeps_evals / (lloyd_ms * 1e-3) / 1e12
+    table_gbs = params * 2 / (kernel_ms["lloyd_table_kernel"] * 1e-3) / 1e9
+    assign_gbs = params * 3 / (kernel_ms["lloyd_assign_kernel"] * 1e-3) / 1e9
     stats_ms = per_call["cmpq_collect_stats"]
     stats_gbs = X.numel() * 2 / (stats_ms * 1e-3) / 1e9
     pack_ms = per_call["cmpq_pack"]
     pack_gbs = params * (1 + METRIC_BUDGET / 8) / (pack_ms * 1e-3) / 1e9
-    roofline = {"bound": "alu", "kernel": "lloyd_kernel (final fit)", "achieved": achieved,
-                "peak": alu_peak_tflops, "unit": "TFLOP/s", "frac": achieved / alu_peak_tflops,
-                "peak_kind": "148 SMs x 128 fp32 lanes x %.0f MHz, one op per lane per clock" % sm_max_mhz,
-                "traffic": None,
+
+    # The all-pairs formulation (every weight against every centroid in every iteration), timed on
+    # the same layer after the timed region: 2 ops (subtract, compare/select) per evaluation it executes.
+    alu_peak_tflops = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    q.run(X, W, METRIC_BUDGET, cfg.lloyd_iters)  # bits and outlier list of the metric's budget
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS)
+    try:
+        ap_calls = 5
+        def all_pairs_call():
+            q.counters.zero_()
+            B.cmpq_quantize_layer(W, q.bits, q.rows, q.cols, cfg.lloyd_iters, q.lut, q.codes, q.ws,
+                                  sweeps=q.counters[1:2])
+        for _ in range(2):
+            all_pairs_call()
+        torch.cuda.synchronize()
+        ap_ms = 0.0
+        for _ in range(ap_calls):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q.counters.zero_()
+            e0.record()
+            B.cmpq_quantize_layer(W, q.bits, q.rows, q.cols, cfg.lloyd_iters, q.lut, q.codes, q.ws,
+                                  sweeps=q.counters[1:2])
+            e1.record()
+            torch.cuda.synchronize()
+            ap_ms += e0.elapsed_time(e1) / ap_calls
+        ap_evals = int(q.counters[1].item())
+    finally:
+        B.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED)
+    ap_tflops = 2.0 * ap_evals / (ap_ms * 1e-3) / 1e12
+
+    roofline = {"bound": "hbm", "kernel": "lloyd_table_kernel (final fit)", "achieved": table_gbs,
+                "peak": hbm_peak, "unit": "GB/s", "frac": table_gbs / hbm_peak, "peak_kind": peak_kind,
+                "traffic": LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT * params if LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT else None,
+                "note": "algorithmic bytes: each 16-bit weight read once; the kernel is bound by "
+                        "shared-memory histogram work, not by HBM",
+                "kernel_ms": kernel_ms,
                 "other_kernels": {
                     "stats": {"bound": "hbm", "achieved": stats_gbs, "peak": hbm_peak, "unit": "GB/s",
                               "frac": stats_gbs / hbm_peak, "peak_kind": peak_kind},
                     "pack": {"bound": "hbm", "achieved": pack_gbs, "peak": hbm_peak, "unit": "GB/s",
-                             "frac": pack_gbs / hbm_peak, "peak_kind": peak_kind}}}
+                             "frac": pack_gbs / hbm_peak, "peak_kind": peak_kind},
+                    "lloyd_assign": {"bound": "hbm", "achieved": assign_gbs, "peak": hbm_peak, "unit": "GB/s",
+                                     "frac": assign_gbs / hbm_peak, "peak_kind": peak_kind},
+                    "lloyd_all_pairs": {
+                        "bound": "alu", "kernel": "lloyd_kernel (CMPQ_ASSIGN_ALL_PAIRS, final fit)",
+                        "achieved": ap_tflops, "peak": alu_peak_tflops, "unit": "TFLOP/s",
+                        "frac": ap_tflops / alu_peak_tflops, "ms": ap_ms,
+                        "peak_kind": "148 SMs x 128 fp32 lanes x %.0f MHz, one op per lane per clock" % sm_max_mhz,
+                        "note": "brute-force formulation, not on the default path: the ordered "
+                                "assignment reaches the same codes and centroids without this work"}}}
 
     # end to end through the public call with host buffers
     Xh = torch.empty(X.shape, dtype=X.dtype, pin_memory=True)
@@ -272,7 +323,7 @@ def main():
             "at_config_budget": {"avg_bits": cfg.budgets[0], "value": world * params / (ms_22 * 1e-3) / 1e6,
                                  "unit": UNIT, "ms_per_step": ms_22},
             "per_call_ms": per_call,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_RUN * steps,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_run(B.ASSIGN_ORDERED) * steps,
             "roofline": roofline, "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))

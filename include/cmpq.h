@@ -166,6 +166,14 @@ cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int6
 cmpq_status cmpq_set_lloyd_assignment(cmpq_lloyd_assignment mode);
 cmpq_lloyd_assignment cmpq_get_lloyd_assignment(void);
 
+/* Timing aid for CMPQ_ASSIGN_ORDERED, which runs three kernels per K-means call (value table,
+ * iterations, last assignment): the four cudaEvent_t handles given here are recorded on the call's
+ * stream before the first and after each of the three kernels by the NEXT cmpq_extract_outliers or
+ * cmpq_quantize_layer call, once; the library keeps no reference afterwards.  Pass four NULLs to
+ * cancel; any other mix of NULLs is CMPQ_ERR_INVALID_ARG.  The events stay owned by the caller. */
+cmpq_status cmpq_lloyd_phase_events(void* before_table, void* after_table, void* after_iterate,
+                                    void* after_assign);
+
 /* ---- packing (accounting of Section 5.1; per-precision sub-matrices of Section 6) -----------
  * Three segments in the order 2-, 3-, 4-bit channels, channels by ascending id inside a
  * segment.  perm[r] = channel stored at position r; row_off[r] = its first 32-bit word

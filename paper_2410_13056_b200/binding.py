@@ -21,7 +21,7 @@ EXPORTS = (
     "cmpq_collect_stats", "cmpq_collect_stats_static", "cmpq_finalize_stats", "cmpq_allocate_bits", "cmpq_extract_outliers",
     "cmpq_quantize_layer", "cmpq_pack", "cmpq_workspace_bytes", "cmpq_alloc_counts",
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
-    "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment",
+    "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment", "cmpq_lloyd_phase_events",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -69,6 +69,8 @@ def lib():
         L.cmpq_set_lloyd_assignment.restype = ci
         L.cmpq_get_lloyd_assignment.argtypes = []
         L.cmpq_get_lloyd_assignment.restype = ci
+        L.cmpq_lloyd_phase_events.argtypes = [vp, vp, vp, vp]
+        L.cmpq_lloyd_phase_events.restype = ci
         L.cmpq_status_string.argtypes = [ci]
         L.cmpq_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -112,6 +114,19 @@ def cmpq_set_lloyd_assignment(mode):
 
 def cmpq_get_lloyd_assignment():
     return int(lib().cmpq_get_lloyd_assignment())
+
+
+def cmpq_lloyd_phase_events(events):
+    """`events`: four torch.cuda.Event(enable_timing=True) that the next ordered K-means call records
+    before its table kernel and after its table, iterate and assign kernels; None cancels."""
+    if events is None:
+        _check(lib().cmpq_lloyd_phase_events(None, None, None, None), "cmpq_lloyd_phase_events")
+        return
+    handles = []
+    for ev in events:
+        ev.record()  # torch creates the CUDA event lazily: make sure the handle exists
+        handles.append(ctypes.c_void_p(ev.cuda_event))
+    _check(lib().cmpq_lloyd_phase_events(*handles), "cmpq_lloyd_phase_events")
 
 
 def cmpq_alloc_counts(d_in, avg_bits):

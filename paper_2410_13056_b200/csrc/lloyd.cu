@@ -623,6 +623,18 @@ extern "C" cmpq_status cmpq_set_lloyd_assignment(cmpq_lloyd_assignment mode) {
 
 extern "C" cmpq_lloyd_assignment cmpq_get_lloyd_assignment(void) { return lloyd_assignment(); }
 
+extern "C" cmpq_status cmpq_lloyd_phase_events(void* before_table, void* after_table, void* after_iterate,
+                                               void* after_assign) {
+    if (!before_table && !after_table && !after_iterate && !after_assign) {
+        set_lloyd_phase_events(nullptr);
+        return CMPQ_OK;
+    }
+    if (!before_table || !after_table || !after_iterate || !after_assign) return CMPQ_ERR_INVALID_ARG;
+    void* ev[4] = {before_table, after_table, after_iterate, after_assign};
+    set_lloyd_phase_events(ev);
+    return CMPQ_OK;
+}
+
 extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
                                            int64_t ldw, const uint8_t* bits, const int32_t* rows,
                                            const int32_t* cols, int64_t nnz, int lloyd_iters,

@@ -33,6 +33,8 @@ cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
 // Ordered formulation: value table per channel, warp-per-channel iterations, streaming last
 // assignment.  `tables` is device scratch of lloyd_tables_bytes(d_in, d_out) bytes, 256-byte aligned.
 size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out);
+// events[0..3] (cudaEvent_t, or NULL to clear): recorded around the three kernels of the next ordered launch.
+void set_lloyd_phase_events(void* const* events);
 cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,
                                  cudaStream_t st);
 

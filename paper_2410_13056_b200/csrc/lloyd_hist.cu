@@ -30,6 +30,8 @@
 #include "lloyd.cuh"
 #include "lloyd_device.cuh"
 
+#include <mutex>
+
 namespace cmpq {
 
 constexpr int kSlots = 32;       // high-byte buckets refined per pass of the second histogram level
@@ -447,83 +449,106 @@ lloyd_iterate_kernel(const IterArgs a) {
 
 constexpr int kAssignThreads = 256;
 
-template <int DT, int K>
+// Code (and distance) of one weight.  by_threshold: the code is the number of k >= 1 with
+// x >= t[k] (thresholds from lloyd_iterate_kernel); otherwise the defining scan.
+template <int K, bool ERR>
+__device__ __forceinline__ void assign_one(float x, const float (&c)[K], const float (&t)[K], bool by_threshold,
+                                           uint32_t& code, float& dist) {
+    if (by_threshold) {
+        uint32_t bk = 0;
+        float cc = c[0];
+#pragma unroll
+        for (int k = 1; k < K; ++k) {
+            const bool ge = x >= t[k];
+            bk += ge ? 1u : 0u;
+            if (ERR) cc = ge ? c[k] : cc;  // thresholds ascend: the last one reached is the code's
+        }
+        code = bk;
+        dist = ERR ? fabsf(x - cc) : 0.f;
+    } else {
+        float best = fabsf(x - c[0]);
+        uint32_t bk = 0;
+#pragma unroll
+        for (int k = 1; k < K; ++k) {
+            const float d = fabsf(x - c[k]);
+            if (d < best) { best = d; bk = k; }
+        }
+        code = bk;
+        dist = best;
+    }
+}
+
+// One row, 8 weights per thread and step (one 128-bit load when the layout allows).
+template <int DT, int K, bool ERR>
 __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut,
                            const float* __restrict__ thr, const uint32_t* removed, bool has_removed) {
     const int N = (int)a.d_out;
     const int tid = threadIdx.x, nthr = blockDim.x;
-    float c[K];
+    float c[K], t[K];
 #pragma unroll
-    for (int k = 0; k < K; ++k) c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
-    // t[0] != 0: the code of x is the number of k >= 1 with x >= t[k] (see lloyd_iterate_kernel)
-    float t[K];
-#pragma unroll
-    for (int k = 0; k < K; ++k) t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
+    for (int k = 0; k < K; ++k) {
+        c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
+        t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
+    }
     const bool by_threshold = t[0] != 0.f;
     const uint16_t* w = a.W + row * a.ldw;
-    const bool vec_in = ((a.ldw & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 7) == 0);
-    const bool vec_out = (N & 3) == 0;
+    const bool vec_in = ((a.ldw & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 15) == 0);
+    const bool vec_out = (N & 7) == 0;
     uint8_t* codes = a.codes ? a.codes + row * a.d_out : nullptr;
     float* err = a.err ? a.err + row * a.d_out : nullptr;
-    for (int j0 = tid * 4; j0 < N; j0 += nthr * 4) {
-        uint16_t h[4] = {0, 0, 0, 0};
-        if (j0 + 3 < N && vec_in) {
-            const uint2 v = *reinterpret_cast<const uint2*>(w + j0);
-            h[0] = (uint16_t)(v.x & 0xffff); h[1] = (uint16_t)(v.x >> 16);
-            h[2] = (uint16_t)(v.y & 0xffff); h[3] = (uint16_t)(v.y >> 16);
+#pragma unroll 2
+    for (int j0 = tid * 8; j0 < N; j0 += nthr * 8) {
+        uint32_t pk[4] = {0u, 0u, 0u, 0u};  // 8 weights, two per word
+        if (j0 + 7 < N && vec_in) {
+            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(w + j0));
+            pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
         } else {
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (j0 + u < N) h[u] = w[j0 + u];
+            for (int u = 0; u < 8; ++u)
+                if (j0 + u < N) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
         }
-        uint32_t code[4];
-        float dist[4];
+        uint32_t mask = 0;  // removed positions among the 8
+        if (has_removed) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = j0 + u;
-            float x = widen16<DT>(h[u]);
-            if (has_removed && j < N && ((removed[j >> 5] >> (j & 31)) & 1)) x = 0.f;
-            x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
-            if (by_threshold) {
-                uint32_t bk = 0;
-                float cc = c[0];
-#pragma unroll
-                for (int k = 1; k < K; ++k) {
-                    const bool ge = x >= t[k];
-                    bk += ge ? 1u : 0u;
-                    cc = ge ? c[k] : cc;  // thresholds ascend: the last one reached is the code's
-                }
-                code[u] = bk;
-                dist[u] = fabsf(x - cc);
-            } else {
-                float best = fabsf(x - c[0]);
-                uint32_t bk = 0;
-#pragma unroll
-                for (int k = 1; k < K; ++k) {
-                    const float d = fabsf(x - c[k]);
-                    if (d < best) { best = d; bk = k; }
-                }
-                code[u] = bk;
-                dist[u] = best;
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                if (j < N) mask |= ((removed[j >> 5] >> (j & 31)) & 1u) << u;
             }
         }
-        if (j0 + 3 < N && vec_out) {
-            if (codes) *reinterpret_cast<uint32_t*>(codes + j0) = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
-            if (err) *reinterpret_cast<float4*>(err + j0) = make_float4(dist[0], dist[1], dist[2], dist[3]);
+        uint32_t code[8];
+        float dist[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            float x = widen16<DT>((uint16_t)(pk[u >> 1] >> (16 * (u & 1))));
+            if ((mask >> u) & 1u) x = 0.f;
+            x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
+            assign_one<K, ERR>(x, c, t, by_threshold, code[u], dist[u]);
+        }
+        if (j0 + 7 < N && vec_out) {
+            if (codes) {
+                uint2 o;
+                o.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
+                o.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
+                *reinterpret_cast<uint2*>(codes + j0) = o;
+            }
+            if (ERR && err) {
+                *reinterpret_cast<float4*>(err + j0) = make_float4(dist[0], dist[1], dist[2], dist[3]);
+                *reinterpret_cast<float4*>(err + j0 + 4) = make_float4(dist[4], dist[5], dist[6], dist[7]);
+            }
         } else {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 if (j0 + u < N) {
                     if (codes) codes[j0 + u] = (uint8_t)code[u];
-                    if (err) err[j0 + u] = dist[u];
+                    if (ERR && err) err[j0 + u] = dist[u];
                 }
             }
         }
     }
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kAssignThreads)
+template <int DT, bool ERR>
+__global__ void __launch_bounds__(kAssignThreads, ERR ? 4 : 6)
 lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut, const float* __restrict__ thr) {
     __shared__ uint32_t removed[CMPQ_MAX_D_OUT / 32];
     const int64_t row = blockIdx.x;
@@ -543,9 +568,9 @@ lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut, const floa
         __syncthreads();
     }
     const int bits = a.bits[row];
-    if (bits == 2) assign_row<DT, 4>(a, row, lut, thr, removed, has_removed);
-    else if (bits == 3) assign_row<DT, 8>(a, row, lut, thr, removed, has_removed);
-    else assign_row<DT, 16>(a, row, lut, thr, removed, has_removed);
+    if (bits == 2) assign_row<DT, 4, ERR>(a, row, lut, thr, removed, has_removed);
+    else if (bits == 3) assign_row<DT, 8, ERR>(a, row, lut, thr, removed, has_removed);
+    else assign_row<DT, 16, ERR>(a, row, lut, thr, removed, has_removed);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -561,8 +586,26 @@ static cmpq_status launch_table(const LloydArgs& args, const Tables& t, int thre
     return launch_status();
 }
 
+// Optional timing of the three kernels: events supplied by cmpq_lloyd_phase_events are recorded
+// around them by the next ordered launch, once.
+static std::mutex g_phase_mutex;
+static cudaEvent_t g_phase_events[4] = {nullptr, nullptr, nullptr, nullptr};
+
+void set_lloyd_phase_events(void* const* events) {
+    std::lock_guard<std::mutex> lock(g_phase_mutex);
+    for (int i = 0; i < 4; ++i) g_phase_events[i] = events ? static_cast<cudaEvent_t>(events[i]) : nullptr;
+}
+
+static void take_phase_events(cudaEvent_t (&ev)[4]) {
+    std::lock_guard<std::mutex> lock(g_phase_mutex);
+    for (int i = 0; i < 4; ++i) { ev[i] = g_phase_events[i]; g_phase_events[i] = nullptr; }
+}
+
 template <int DT>
 static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cudaStream_t st) {
+    cudaEvent_t ev[4];
+    take_phase_events(ev);
+    if (ev[0]) cudaEventRecord(ev[0], st);
     const int64_t N = args.d_out;
     auto threads_for = [N](int e) {
         int64_t th = (N + e - 1) / e;
@@ -576,6 +619,7 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cud
     else if (N <= 16384) s = launch_table<DT, 16, 1024, 1>(args, t, threads_for(16), st);
     else s = launch_table<DT, 32, 1024, 1>(args, t, threads_for(32), st);
     if (s != CMPQ_OK) return s;
+    if (ev[1]) cudaEventRecord(ev[1], st);
 
     IterArgs ia{};
     ia.t = t;
@@ -590,9 +634,13 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cud
     lloyd_iterate_kernel<DT><<<iter_blocks, kIterWarps * 32, 0, st>>>(ia);
     s = launch_status();
     if (s != CMPQ_OK) return s;
+    if (ev[2]) cudaEventRecord(ev[2], st);
 
-    lloyd_assign_kernel<DT><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
-    return launch_status();
+    if (args.err) lloyd_assign_kernel<DT, true><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
+    else lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
+    s = launch_status();
+    if (ev[3]) cudaEventRecord(ev[3], st);
+    return s;
 }
 
 cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,

@@ -13,9 +13,17 @@ import torch
 from . import binding as B
 
 # CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0:
-# statistic 2 + finalize 1, allocation 2, outliers 13 (rank, mark, K-means, select init, 3 x
-# (histogram, digit), row count, row scan, emit), final fit 2, packing 2.
-KERNELS_PER_RUN = 22
+# statistic 2 + finalize 1, allocation 2, outliers 12 + the K-means (rank, mark, select init, 3 x
+# (histogram, digit), row count, row scan, emit), final fit 1 (row index) + the K-means, packing 2.
+# A K-means call is 3 kernels (table, iterate, assign) by default, 1 with ASSIGN_ALL_PAIRS.
+def kernels_per_run(assignment=None):
+    if assignment is None:
+        assignment = B.cmpq_get_lloyd_assignment()
+    per_kmeans = 1 if assignment == B.ASSIGN_ALL_PAIRS else 3
+    return 20 + 2 * per_kmeans
+
+
+KERNELS_PER_RUN = 26  # with the default assignment
 
 
 @dataclass
@@ -71,7 +79,8 @@ class LayerQuantizer:
 
     def run(self, X, W, avg_bits, lloyd_iters, events=None):
         """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
-        events (optional dict) receives a (start, end) CUDA event pair per C-ABI call."""
+        events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and, under
+        "final_fit_kernels", the four events around the three kernels of the final K-means."""
         assert W.shape == (self.d_in, self.d_out) and X.shape[1] == self.d_in
 
         def call(name, fn, *args, **kw):
@@ -94,6 +103,11 @@ class LayerQuantizer:
              self.ws)
         call("cmpq_extract_outliers", B.cmpq_extract_outliers, W, self.a, self.bits, self.n_act, self.n_q,
              lloyd_iters, self.rows, self.cols, self.vals, self.ws)
+        if events is not None and B.cmpq_get_lloyd_assignment() == B.ASSIGN_ORDERED:
+            # the three kernels of the final fit, timed separately
+            phase = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            B.cmpq_lloyd_phase_events(phase)
+            events["final_fit_kernels"] = phase
         call("cmpq_quantize_layer", B.cmpq_quantize_layer, W, self.bits, self.rows, self.cols, lloyd_iters,
              self.lut, self.codes, self.ws, inexact_rows=inexact, sweeps=sweeps)
         call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
