@@ -111,7 +111,7 @@ __device__ __forceinline__ void load_channel_keys(const LloydArgs& a, int64_t ro
     nval_cols = 0;
     {
         float lo = __int_as_float(0x7f800000), hi = __int_as_float(0xff800000);
-        int top = -100000, ulp = 100000;
+        uint32_t amax = 0u, amin1 = 0xffffffffu;  // largest |x| pattern; smallest non-zero |x| pattern minus 1
 #pragma unroll
         for (int g = 0; g < E / 4; ++g) {
             const int j0 = (g * nthr + tid) * 4;
@@ -135,44 +135,68 @@ __device__ __forceinline__ void load_channel_keys(const LloydArgs& a, int64_t ro
                     v = (v == 0.f) ? 0.f : v;  // -0 and +0 are the same point
                     lo = fminf(lo, v);
                     hi = fmaxf(hi, v);
-                    uint32_t ub = __float_as_uint(v) & 0x7fffffffu;
-                    if (ub) {
-                        int ex = (int)(ub >> 23);
-                        uint32_t m = ub & 0x7fffffu;
-                        int t, q;
-                        if (ex) { t = ex - 127; q = ex - 150 + (__ffs(m | 0x800000u) - 1); }
-                        else    { t = (31 - __clz(m)) - 149; q = (__ffs(m) - 1) - 149; }
-                        top = max(top, t);
-                        ulp = min(ulp, q);
-                    }
+                    const uint32_t ub = __float_as_uint(v) & 0x7fffffffu;
+                    amax = max(amax, ub);
+                    amin1 = min(amin1, ub - 1u);  // zero wraps to the largest value
                 }
                 key[4 * g + u] = sort_key16<DT>(v);
             }
         }
-        // value range (for the gap test) and exactness diagnostics
+        // value range (for the gap test) and the magnitude range (for the exactness test)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
             hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
-            top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
-            ulp = min(ulp, __shfl_xor_sync(0xffffffffu, ulp, o));
+            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
         }
-        if (lane == 0) { sh.wlo[warp] = lo; sh.whi[warp] = hi; sh.wtop[warp] = top; sh.wulp[warp] = ulp; }
+        if (lane == 0) { sh.wlo[warp] = lo; sh.whi[warp] = hi; sh.wtop[warp] = (int)amax; sh.wulp[warp] = (int)amin1; }
         __syncthreads();  // also: every thread is done with the removed-column bitmap
+        // every warp reduces the per-warp values again, so the decision below is the same in all threads
+        amax = lane < nwarps ? (uint32_t)sh.wtop[lane] : 0u;
+        amin1 = lane < nwarps ? (uint32_t)sh.wulp[lane] : 0xffffffffu;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
+        }
         if (tid == 0) {
             for (int wv = 1; wv < nwarps; ++wv) {
                 lo = fminf(lo, sh.wlo[wv]);
                 hi = fmaxf(hi, sh.whi[wv]);
-                top = max(top, sh.wtop[wv]);
-                ulp = min(ulp, sh.wulp[wv]);
             }
             sh.vmin = lo;
             sh.vmax = hi;
-            if (a.inexact_rows && top > -100000) {
-                // sums and differences of up to 2N weights stay exact in fp64 while
-                // 2 N 2^(top+1) / 2^ulp <= 2^53
-                int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
-                if (log2n + 1 + (top + 1 - ulp) > 53) atomicAdd(a.inexact_rows, 1);
+        }
+        // Sums and differences of up to 2N weights stay exact in fp64 while 2 N 2^(top+1) / 2^q <= 2^53,
+        // top = exponent of the largest magnitude, 2^q = smallest unit in the last place of a non-zero
+        // weight.  First with a lower bound of q from the smallest magnitude's exponent and the trailing
+        // zero bits every widened 16-bit value has; only a channel that fails this is examined bit by bit.
+        if (a.inexact_rows && amax != 0u) {
+            const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
+            const int ex_max = (int)(amax >> 23), ex_min = (int)((amin1 + 1u) >> 23);
+            const int top = ex_max ? ex_max - 127 : (31 - __clz(amax)) - 149;
+            const int q_low = (ex_min ? ex_min - 150 : -149) + (DT == CMPQ_BF16 ? 16 : 13);
+            if (log2n + 1 + (top + 1 - q_low) > 53) {  // same value in every thread of the block
+                int q = 100000;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const uint32_t ub = __float_as_uint(value_of_key16<DT>(key[e])) & 0x7fffffffu;
+                    if (e < nval_cols && ub) {
+                        const int ex = (int)(ub >> 23);
+                        const uint32_t m = ub & 0x7fffffu;
+                        q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) q = min(q, __shfl_xor_sync(0xffffffffu, q, o));
+                __syncthreads();  // every warp has read wtop / wulp
+                if (lane == 0) sh.wulp[warp] = q;
+                __syncthreads();
+                if (tid == 0) {
+                    for (int wv = 1; wv < nwarps; ++wv) q = min(q, sh.wulp[wv]);
+                    if (log2n + 1 + (top + 1 - q) > 53) atomicAdd(a.inexact_rows, 1);
+                }
             }
         }
     }

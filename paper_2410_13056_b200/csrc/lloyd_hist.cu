@@ -30,6 +30,8 @@
 #include "lloyd.cuh"
 #include "lloyd_device.cuh"
 
+#include <cuda_bf16.h>
+
 #include <mutex>
 
 namespace cmpq {
@@ -207,6 +209,7 @@ struct IterArgs {
     const uint8_t* skip_row;
     int64_t d_in, d_out;
     int iters;
+    int cap;     // table entries a warp can stage in shared memory (multiple of 8)
     float* lut;  // [d_in][16]
     unsigned long long* sweeps;
 };
@@ -276,13 +279,12 @@ __device__ __forceinline__ int search_entries(const uint16_t* keys, int M, float
 }
 
 constexpr int kIterWarps = 4;
-constexpr int kIterCap = 2048;  // distinct values of a channel whose table fits the warp's shared memory
 
-struct alignas(16) IterShared {
-    uint16_t keys[kIterCap];
-    uint16_t cum[kIterCap + 8];
-    double coarse[kIterCap / 8 + 1];
-};
+// Shared memory of one warp of the iterate kernel: the channel's table when it has at most `cap`
+// distinct values (cap is a multiple of 8, chosen by the host from d_out).
+__host__ __device__ inline size_t iter_warp_bytes(int cap) {
+    return (size_t)cap * 2 + (size_t)(cap + 8) * 2 + (size_t)(cap / 8 + 1) * 8 + 8;  // keys, cum, coarse sums
+}
 
 // fp64 sum of all weights below entry e (0 <= e <= M): the prefix stored for entry 8 (e / 8)
 // plus at most seven count x value products.
@@ -304,7 +306,7 @@ __device__ __forceinline__ double prefix_sum_at(const uint16_t* keys, const uint
 }
 
 template <int DT, int K>
-__device__ void iterate_channel(const IterArgs& a, int64_t row, IterShared& sm) {
+__device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* warp_smem) {
     const int lane = threadIdx.x & 31;
     const ChannelHeader h = a.t.hdr[row];
     const int N = (int)a.d_out, T = a.iters;
@@ -312,14 +314,17 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, IterShared& sm) 
     const uint16_t* keys = a.t.keys + row * a.t.stride;
     const uint16_t* cum = a.t.cum + row * a.t.stride;
     double* coarse = a.t.sum + row * a.t.stride;  // global scratch, used when the table is too large
-    if (M <= kIterCap) {  // the rows are 16-byte aligned and padded to a multiple of 8 entries
+    if (M <= a.cap) {  // the rows are 16-byte aligned and padded to a multiple of 8 entries
+        double* s_coarse = reinterpret_cast<double*>(warp_smem);
+        uint16_t* s_keys = reinterpret_cast<uint16_t*>(s_coarse + a.cap / 8 + 1 + 1);
+        uint16_t* s_cum = s_keys + a.cap;
         for (int i = lane; i < (M + 7) / 8; i += 32)
-            reinterpret_cast<uint4*>(sm.keys)[i] = __ldg(reinterpret_cast<const uint4*>(keys) + i);
+            reinterpret_cast<uint4*>(s_keys)[i] = __ldg(reinterpret_cast<const uint4*>(keys) + i);
         for (int i = lane; i < (M + 1 + 7) / 8; i += 32)  // with the sentinel cum[M] = d_out
-            reinterpret_cast<uint4*>(sm.cum)[i] = __ldg(reinterpret_cast<const uint4*>(cum) + i);
-        keys = sm.keys;
-        cum = sm.cum;
-        coarse = sm.coarse;
+            reinterpret_cast<uint4*>(s_cum)[i] = __ldg(reinterpret_cast<const uint4*>(cum) + i);
+        keys = s_keys;
+        cum = s_cum;
+        coarse = s_coarse;
     }
     __syncwarp();
     // prefix sums at every eighth entry: each lane sums a contiguous range of groups of eight entries,
@@ -431,23 +436,48 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, IterShared& sm) 
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kIterWarps * 32, 5)
+__global__ void __launch_bounds__(kIterWarps * 32, 7)
 lloyd_iterate_kernel(const IterArgs a) {
-    __shared__ IterShared sm[kIterWarps];
+    extern __shared__ __align__(16) unsigned char iter_smem[];
     const int warp = threadIdx.x >> 5;
+    unsigned char* warp_smem = iter_smem + (size_t)warp * iter_warp_bytes(a.cap);
     const int64_t row = (int64_t)blockIdx.x * kIterWarps + warp;
     if (row >= a.d_in) return;
     if (a.skip_row && a.skip_row[row]) return;
     const int bits = a.bits[row];
-    if (bits == 2) iterate_channel<DT, 4>(a, row, sm[warp]);
-    else if (bits == 3) iterate_channel<DT, 8>(a, row, sm[warp]);
-    else iterate_channel<DT, 16>(a, row, sm[warp]);
+    if (bits == 2) iterate_channel<DT, 4>(a, row, warp_smem);
+    else if (bits == 3) iterate_channel<DT, 8>(a, row, warp_smem);
+    else iterate_channel<DT, 16>(a, row, warp_smem);
 }
 
 // ------------------------------------------------------------------------------------------------
 // last assignment
 
 constexpr int kAssignThreads = 256;
+
+// Two weights at once in their 16-bit storage type: acc += (x >= t) per half, as 1.0 or 0.0.
+template <int DT>
+__device__ __forceinline__ uint32_t add_ge_x2(uint32_t acc, uint32_t x2, uint32_t t2) {
+    if (DT == CMPQ_BF16) {
+        const __nv_bfloat162 r = __hadd2(*reinterpret_cast<const __nv_bfloat162*>(&acc),
+                                         __hge2(*reinterpret_cast<const __nv_bfloat162*>(&x2),
+                                                *reinterpret_cast<const __nv_bfloat162*>(&t2)));
+        return *reinterpret_cast<const uint32_t*>(&r);
+    } else {
+        const __half2 r = __hadd2(*reinterpret_cast<const __half2*>(&acc),
+                                  __hge2(*reinterpret_cast<const __half2*>(&x2), *reinterpret_cast<const __half2*>(&t2)));
+        return *reinterpret_cast<const uint32_t*>(&r);
+    }
+}
+
+// A threshold (a value of the channel or +infinity, so exact in the storage type) in both halves.
+template <int DT>
+__device__ __forceinline__ uint32_t threshold_x2(float t) {
+    uint32_t h;
+    if (DT == CMPQ_BF16) h = __float_as_uint(t) >> 16;
+    else h = __half_as_ushort(__float2half_rn(t));
+    return h | (h << 16);
+}
 
 // Code (and distance) of one weight.  by_threshold: the code is the number of k >= 1 with
 // x >= t[k] (thresholds from lloyd_iterate_kernel); otherwise the defining scan.
@@ -460,7 +490,7 @@ __device__ __forceinline__ void assign_one(float x, const float (&c)[K], const f
 #pragma unroll
         for (int k = 1; k < K; ++k) {
             const bool ge = x >= t[k];
-            bk += ge ? 1u : 0u;
+            if (!ERR) bk += ge ? 1u : 0u;   // the provisional fit (ERR) asks for distances only
             if (ERR) cc = ge ? c[k] : cc;  // thresholds ascend: the last one reached is the code's
         }
         code = bk;
@@ -479,9 +509,17 @@ __device__ __forceinline__ void assign_one(float x, const float (&c)[K], const f
 }
 
 // One row, 8 weights per thread and step (one 128-bit load when the layout allows).
+// removed positions of the row: a bitmap over the columns (nrem > kShortList) or a short list
+struct RemovedCols {
+    const uint32_t* bitmap;
+    const int* list;
+    int nrem;
+};
+constexpr int kShortList = 16;
+
 template <int DT, int K, bool ERR>
 __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut,
-                           const float* __restrict__ thr, const uint32_t* removed, bool has_removed) {
+                           const float* __restrict__ thr, const RemovedCols& rem, uint4 first) {
     const int N = (int)a.d_out;
     const int tid = threadIdx.x, nthr = blockDim.x;
     float c[K], t[K];
@@ -491,6 +529,12 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
         t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
     }
     const bool by_threshold = t[0] != 0.f;
+    // codes only, by thresholds: two weights per compare in the storage type.  A count c sits in
+    // the low mantissa bits of 128 + c (bf16) or 1024 + c (fp16).
+    uint32_t t2[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) t2[k] = threshold_x2<DT>(t[k]);
+    const uint32_t acc0 = DT == CMPQ_BF16 ? 0x43004300u : 0x64006400u;
     const uint16_t* w = a.W + row * a.ldw;
     const bool vec_in = ((a.ldw & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 15) == 0);
     const bool vec_out = (N & 7) == 0;
@@ -500,7 +544,8 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
     for (int j0 = tid * 8; j0 < N; j0 += nthr * 8) {
         uint32_t pk[4] = {0u, 0u, 0u, 0u};  // 8 weights, two per word
         if (j0 + 7 < N && vec_in) {
-            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(w + j0));
+            // the first step's weights were requested before anything else in the kernel
+            const uint4 v = j0 == tid * 8 ? first : __ldcs(reinterpret_cast<const uint4*>(w + j0));
             pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
         } else {
 #pragma unroll
@@ -508,12 +553,31 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
                 if (j0 + u < N) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
         }
         uint32_t mask = 0;  // removed positions among the 8
-        if (has_removed) {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int j = j0 + u;
-                if (j < N) mask |= ((removed[j >> 5] >> (j & 31)) & 1u) << u;
+        if (rem.nrem > kShortList) {
+            mask = (rem.bitmap[j0 >> 5] >> (j0 & 31)) & 0xffu;  // j0 is a multiple of 8
+        } else {
+            for (int i = 0; i < rem.nrem; ++i) {
+                const unsigned d = (unsigned)(rem.list[i] - j0);
+                if (d < 8u) mask |= 1u << d;
             }
+        }
+        if (!ERR && codes && by_threshold && j0 + 7 < N && vec_out) {
+            uint32_t r[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t x2 = pk[q];
+                if ((mask >> (2 * q)) & 1u) x2 &= 0xffff0000u;      // removed positions become +0
+                if ((mask >> (2 * q + 1)) & 1u) x2 &= 0x0000ffffu;
+                uint32_t acc = acc0;
+#pragma unroll
+                for (int k = 1; k < K; ++k) acc = add_ge_x2<DT>(acc, x2, t2[k]);
+                r[q] = acc & 0x000f000fu;
+            }
+            uint2 o;
+            o.x = __byte_perm(r[0], r[1], 0x6420);
+            o.y = __byte_perm(r[2], r[3], 0x6420);
+            *reinterpret_cast<uint2*>(codes + j0) = o;
+            continue;
         }
         uint32_t code[8];
         float dist[8];
@@ -550,27 +614,38 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
 template <int DT, bool ERR>
 __global__ void __launch_bounds__(kAssignThreads, ERR ? 4 : 6)
 lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut, const float* __restrict__ thr) {
-    __shared__ uint32_t removed[CMPQ_MAX_D_OUT / 32];
+    __shared__ uint32_t bitmap[CMPQ_MAX_D_OUT / 32];
+    __shared__ int list[kShortList];
     const int64_t row = blockIdx.x;
-    if (a.skip_row && a.skip_row[row]) return;
     const int N = (int)a.d_out;
     const int tid = threadIdx.x, nthr = blockDim.x;
+    // request this thread's first 8 weights before the row's metadata: the loads overlap
+    uint4 first = make_uint4(0u, 0u, 0u, 0u);
+    if (tid * 8 + 7 < N && ((a.ldw & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & 15) == 0))
+        first = __ldcs(reinterpret_cast<const uint4*>(a.W + row * a.ldw + tid * 8));
+    if (a.skip_row && a.skip_row[row]) return;
     int64_t p0 = 0, p1 = 0;
     if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
-    const bool has_removed = p1 > p0;
-    if (has_removed) {
-        for (int w = tid; w < (N + 31) / 32; w += nthr) removed[w] = 0;
+    RemovedCols rem;
+    rem.bitmap = bitmap;
+    rem.list = list;
+    rem.nrem = (int)(p1 - p0);
+    if (rem.nrem > kShortList) {
+        for (int w = tid; w < (N + 31) / 32; w += nthr) bitmap[w] = 0;
         __syncthreads();
         for (int64_t p = p0 + tid; p < p1; p += nthr) {
             const int col = a.cols[p];
-            atomicOr(&removed[col >> 5], 1u << (col & 31));
+            atomicOr(&bitmap[col >> 5], 1u << (col & 31));
         }
+        __syncthreads();
+    } else if (rem.nrem > 0) {
+        if (tid < rem.nrem) list[tid] = a.cols[p0 + tid];
         __syncthreads();
     }
     const int bits = a.bits[row];
-    if (bits == 2) assign_row<DT, 4, ERR>(a, row, lut, thr, removed, has_removed);
-    else if (bits == 3) assign_row<DT, 8, ERR>(a, row, lut, thr, removed, has_removed);
-    else assign_row<DT, 16, ERR>(a, row, lut, thr, removed, has_removed);
+    if (bits == 2) assign_row<DT, 4, ERR>(a, row, lut, thr, rem, first);
+    else if (bits == 3) assign_row<DT, 8, ERR>(a, row, lut, thr, rem, first);
+    else assign_row<DT, 16, ERR>(a, row, lut, thr, rem, first);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -603,6 +678,7 @@ static void take_phase_events(cudaEvent_t (&ev)[4]) {
 
 template <int DT>
 static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cudaStream_t st) {
+    if (args.err && args.codes) return CMPQ_ERR_INTERNAL;  // the assign kernel writes one or the other
     cudaEvent_t ev[4];
     take_phase_events(ev);
     if (ev[0]) cudaEventRecord(ev[0], st);
@@ -630,8 +706,15 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cud
     ia.iters = args.iters;
     ia.lut = args.lut ? args.lut : t.lut;
     ia.sweeps = args.sweeps;
+    // distinct 16-bit values grow slowly with the channel length (about 1400 at 4096 weights, 2300 at
+    // 28672 for Gaussian-like bf16 weights); longer tables are read from global memory
+    ia.cap = N <= 4096 ? 1536 : (N <= 12288 ? 2048 : 3072);
+    const size_t iter_smem = (size_t)kIterWarps * iter_warp_bytes(ia.cap);
+    if (cudaFuncSetAttribute(lloyd_iterate_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)iter_smem) !=
+        cudaSuccess)
+        return CMPQ_ERR_CUDA;
     const unsigned iter_blocks = (unsigned)((args.d_in + kIterWarps - 1) / kIterWarps);
-    lloyd_iterate_kernel<DT><<<iter_blocks, kIterWarps * 32, 0, st>>>(ia);
+    lloyd_iterate_kernel<DT><<<iter_blocks, kIterWarps * 32, iter_smem, st>>>(ia);
     s = launch_status();
     if (s != CMPQ_OK) return s;
     if (ev[2]) cudaEventRecord(ev[2], st);
