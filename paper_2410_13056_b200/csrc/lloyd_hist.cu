@@ -14,8 +14,9 @@
 //                         fabsf(x - c_k) < fabsf(x - c_{k-1}) is false on a prefix of the ascending
 //                         values and true on the rest, and the first k minimising fabsf(x - c_k) is
 //                         the number of k >= 1 for which it is true.  Cluster k is then a run of the
-//                         table: a half warp finds the first entry where predicate k holds with 16
-//                         probes per round, and the cluster's count and sum are differences of
+//                         table: lane k finds the first entry where predicate k holds (galloping
+//                         from the previous boundary, then bisection), and the cluster's count and
+//                         sum are differences of
 //                         prefix counts and prefix sums at two such entries (the warp builds the
 //                         prefix sums once, at every eighth entry; table and sums stay in shared
 //                         memory when they fit).  Centroids that fail the test are handled
@@ -216,66 +217,47 @@ struct IterArgs {
 
 // Lane k (1..K-1) receives e_k = the number of table entries for whose value the predicate
 // fabsf(x - c_k) < fabsf(x - c_{k-1}) is false (a prefix of the table); lane 0 receives 0, lane K
-// receives M.  A half warp narrows one boundary's interval by 16 probes per round; kBatch pairs
-// of boundaries are interleaved so that their loads overlap.
+// receives M.  Every lane searches its own boundary: the warp's instruction stream then serves all
+// K-1 boundaries at once, which matters because the kernel is bound by instruction issue.  e_prev
+// (the lane's result of the previous iteration, or -1) starts a galloping search next to the old
+// boundary -- boundaries move by a few entries per iteration -- followed by bisection.
 template <int DT, int K>
-__device__ __forceinline__ int search_entries(const uint16_t* keys, int M, float ck_lane) {
-    constexpr int PAIRS = K / 2;
-    constexpr int kBatch = PAIRS < 4 ? PAIRS : 4;
-    const int lane = threadIdx.x & 31, half = lane >> 4, j = lane & 15;
-    int out = (lane == K) ? M : 0;
-#pragma unroll
-    for (int p0 = 0; p0 < PAIRS; p0 += kBatch) {
-        float ck[kBatch], cm[kBatch];
-        int lo[kBatch], hi[kBatch];
-#pragma unroll
-        for (int p = 0; p < kBatch; ++p) {
-            const int k = 1 + 2 * (p0 + p) + half;
-            const int kk = k < K ? k : K - 1;
-            ck[p] = __shfl_sync(0xffffffffu, ck_lane, kk);
-            cm[p] = __shfl_sync(0xffffffffu, ck_lane, kk - 1);
-            lo[p] = 0;
-            hi[p] = k < K ? M : 0;  // k = K has no boundary: empty interval
-        }
-        // an interval of length len shrinks to at most step - 1 per round
-        for (int len = M; len > 0; len = ((len + 15) >> 4) - 1) {
-            int step[kBatch];
-            float v[kBatch];
-            bool inb[kBatch];
-#pragma unroll
-            for (int p = 0; p < kBatch; ++p) {
-                step[p] = (hi[p] - lo[p] + 15) >> 4;
-                const int pos = lo[p] + j * step[p] + step[p] - 1;
-                // false for an empty interval (step 0); entries from hi on are known to be true
-                inb[p] = step[p] > 0 && pos < hi[p];
-                const int idx = pos < 0 ? 0 : (pos < M ? pos : M - 1);
-                v[p] = value_of_key16<DT>(keys[idx]);
-            }
-            uint32_t m[kBatch];
-#pragma unroll
-            for (int p = 0; p < kBatch; ++p) {
-                const bool is_false = inb[p] && !(fabsf(v[p] - ck[p]) < fabsf(v[p] - cm[p]));
-                m[p] = __ballot_sync(0xffffffffu, is_false);
-            }
-#pragma unroll
-            for (int p = 0; p < kBatch; ++p) {
-                const int nf = __popc((m[p] >> (16 * half)) & 0xffffu);
-                if (step[p] > 0) {
-                    lo[p] += nf * step[p];
-                    const int cap = lo[p] + step[p] - 1;
-                    hi[p] = hi[p] < cap ? hi[p] : cap;
+__device__ __forceinline__ int search_entries(const uint16_t* keys, int M, float ck_lane, int e_prev) {
+    const int lane = threadIdx.x & 31;
+    const float cm = __shfl_up_sync(0xffffffffu, ck_lane, 1);  // c_{k-1}
+    const float ck = ck_lane;
+    int lo = 0, hi = 0;  // the predicate is false for entries < lo and true for entries >= hi
+    if (lane > 0 && lane < K) {
+        hi = M;
+        auto pred = [&](int i) {
+            const float v = value_of_key16<DT>(keys[i]);
+            return fabsf(v - ck) < fabsf(v - cm);
+        };
+        if (e_prev >= 0) {
+            const int p = e_prev < M ? e_prev : M;
+            if (p >= M || pred(p)) {  // the boundary is at or below p: gallop downwards
+                hi = p;
+                for (int step = 1;; step <<= 1) {
+                    const int q = hi - step;
+                    if (q < 0) break;
+                    if (pred(q)) { hi = q; } else { lo = q + 1; break; }
+                }
+            } else {                  // the boundary is above p: gallop upwards
+                lo = p + 1;
+                for (int step = 1;; step <<= 1) {
+                    const int q = lo - 1 + step;
+                    if (q >= M) break;
+                    if (pred(q)) { hi = q; break; } else { lo = q + 1; }
                 }
             }
         }
-#pragma unroll
-        for (int p = 0; p < kBatch; ++p) {
-            const int b0 = __shfl_sync(0xffffffffu, lo[p], 0);
-            const int b1 = __shfl_sync(0xffffffffu, lo[p], 16);
-            if (lane == 1 + 2 * (p0 + p)) out = b0;
-            if (lane == 2 + 2 * (p0 + p) && lane < K) out = b1;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (pred(mid)) hi = mid; else lo = mid + 1;
         }
     }
-    return out;
+    __syncwarp();
+    return lane == K ? M : lo;
 }
 
 constexpr int kIterWarps = 4;
@@ -375,10 +357,12 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* w
     __syncwarp();
 
     int updates = 0;
+    int e_prev = -1;  // this lane's boundary of the previous ordered search
     while (updates < T) {
         float cn = ck;
         if (counting_sweep_valid<K>(ck, need)) {
-            const int e = search_entries<DT, K>(keys, M, ck);
+            const int e = search_entries<DT, K>(keys, M, ck, e_prev);
+            e_prev = e;
             int B = 0;
             double P = 0.0;
             if (lane <= K) { B = (int)cum[e]; P = prefix_sum_at<DT>(keys, cum, coarse, e); }
@@ -425,7 +409,7 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* w
         const bool ok = counting_sweep_valid<K>(ck, need);
         float thr = ok ? 1.f : 0.f;
         if (ok) {
-            const int e = search_entries<DT, K>(keys, M, ck);
+            const int e = search_entries<DT, K>(keys, M, ck, e_prev);
             if (lane > 0 && lane < K) thr = e < M ? value_of_key16<DT>(keys[e]) : __int_as_float(0x7f800000);
         }
         if (lane < CMPQ_LUT_STRIDE) a.t.thr[row * CMPQ_LUT_STRIDE + lane] = lane < K ? thr : 0.f;

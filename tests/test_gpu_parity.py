@@ -196,3 +196,22 @@ def test_pack_bit_exact(d_in, d_out):
         c1 = codes & ((1 << only) - 1)
         for g, r in zip(G.gpu_pack(c1, b1), oracle.pack(c1, b1)):
             assert np.array_equal(g, r)
+
+
+# ----------------------------------------------------------------------------- timing aid
+def test_phase_events_bracket_the_three_kernels_once():
+    W, Wu, a, bits = _case(64, 2048, inputs.BF16, 5, 3.0)
+    none = np.zeros(0, np.int32)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    B.cmpq_lloyd_phase_events(ev)
+    lut1, codes1, _, _ = G.gpu_quantize(W, bits, none, none, 6)
+    torch.cuda.synchronize()
+    spans = [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
+    assert all(s > 0 for s in spans)
+    # the hook is consumed by one call; a second call is neither timed nor changed by it
+    lut2, codes2, _, _ = G.gpu_quantize(W, bits, none, none, 6)
+    assert np.array_equal(codes1, codes2) and np.array_equal(lut1, lut2)
+    B.cmpq_lloyd_phase_events(ev)
+    B.cmpq_lloyd_phase_events(None)   # cancel
+    with pytest.raises(B.CmpqError):
+        B._check(B.lib().cmpq_lloyd_phase_events(1, None, None, None), "cmpq_lloyd_phase_events")
