@@ -268,20 +268,31 @@ __host__ __device__ inline size_t iter_warp_bytes(int cap) {
     return (size_t)cap * 2 + (size_t)(cap + 8) * 2 + (size_t)(cap / 8 + 1) * 8 + 8;  // keys, cum, coarse sums
 }
 
+// Eight consecutive 16-bit table entries starting at a multiple of 8 (16-byte aligned), one load.
+struct Eight {
+    uint32_t w[4];
+    __device__ __forceinline__ uint32_t at(int u) const { return (w[u >> 1] >> (16 * (u & 1))) & 0xffffu; }
+};
+__device__ __forceinline__ Eight load_eight(const uint16_t* p) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    Eight r;
+    r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w;
+    return r;
+}
+
 // fp64 sum of all weights below entry e (0 <= e <= M): the prefix stored for entry 8 (e / 8)
 // plus at most seven count x value products.
 template <int DT>
 __device__ __forceinline__ double prefix_sum_at(const uint16_t* keys, const uint16_t* cum, const double* coarse,
                                                 int e) {
-    const int j0 = e & ~7;
+    const int j0 = e & ~7, r = e & 7;
     double P = coarse[e >> 3];
-    int c_prev = (int)cum[j0];
+    const Eight k8 = load_eight(keys + j0), c8 = load_eight(cum + j0);
 #pragma unroll
     for (int u = 0; u < 7; ++u) {
-        if (j0 + u < e) {
-            const int c_next = (int)cum[j0 + u + 1];
-            P += (double)(c_next - c_prev) * (double)value_of_key16<DT>(keys[j0 + u]);
-            c_prev = c_next;
+        if (u < r) {
+            const int cnt = (int)c8.at(u + 1) - (int)c8.at(u);
+            P += (double)cnt * (double)value_of_key16<DT>(k8.at(u));
         }
     }
     return P;
@@ -318,13 +329,13 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* w
         double local = 0.0;
         for (int g = g_begin; g < g_begin + per_lane && g < groups; ++g) {
             coarse[g] = local;
-            int c_prev = (int)cum[g * 8 < M ? g * 8 : M];
+            const Eight k8 = load_eight(keys + g * 8), c8 = load_eight(cum + g * 8);
+            const int c_end = g * 8 + 8 <= M ? (int)cum[g * 8 + 8] : 0;
+#pragma unroll
             for (int u = 0; u < 8; ++u) {
-                const int j = g * 8 + u;
-                if (j < M) {
-                    const int c_next = (int)cum[j + 1];
-                    local += (double)(c_next - c_prev) * (double)value_of_key16<DT>(keys[j]);
-                    c_prev = c_next;
+                if (g * 8 + u < M) {
+                    const int c_next = u < 7 ? (int)c8.at(u + 1) : c_end;
+                    local += (double)(c_next - (int)c8.at(u)) * (double)value_of_key16<DT>(k8.at(u));
                 }
             }
         }
