@@ -42,9 +42,7 @@ constexpr int kSlotWords = 128;  // 256 low-byte counters of 16 bits, two per wo
 static_assert(CMPQ_MAX_D_OUT < 65536, "second-level counters and count prefixes are 16 bits wide");
 
 struct ChannelHeader {
-    int M;             // distinct values of the channel
-    float vmin, vmax;  // its value range
-    int pad;
+    int M;  // distinct values of the channel
 };
 
 // Per channel: `stride` entries (M used, entry M is a sentinel holding the totals).
@@ -81,19 +79,20 @@ size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out) {
 // ------------------------------------------------------------------------------------------------
 // value table of one channel
 
+constexpr int kShortList = 16;  // removed positions of a row kept as a list up to this many, else as a bitmap
+
 struct alignas(16) TableShared {
-    int hist1[256];
+    int hist1[256];        // 1 where the high byte occurs
     int bucket_rank[256];  // rank of a high-byte bucket among the non-empty ones, or -1
     int slot_hi[256];      // the inverse: high byte of the r-th non-empty bucket
     int n_nonempty;
-    float vmin, vmax;
-    float wlo[32], whi[32];
-    int wtop[32], wulp[32];
+    int wtop[32], wulp[32];   // per-warp magnitude range (largest pattern, smallest non-zero pattern - 1)
     int w_nz[32], w_cnt[32];  // per-warp totals of the block scan
     int base_nz, base_cnt;    // entries / weights emitted by the previous passes
+    int rem_list[kShortList];
 };
-// dynamic shared memory after TableShared: kSlots * kSlotWords words (removed-column bitmap during
-// the load, second-level counters afterwards)
+// dynamic shared memory after TableShared: kSlots * kSlotWords words of second-level counters, then
+// a bitmap of d_out bits for rows with many removed positions
 
 template <int DT, int E, int MAXT, int MINB>
 __global__ void __launch_bounds__(MAXT, MINB)
@@ -103,30 +102,104 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     if (a.skip_row && a.skip_row[row]) return;
     TableShared& sh = *reinterpret_cast<TableShared*>(smem_raw);
     uint32_t* h2 = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TableShared));
+    uint32_t* bitmap = h2 + kSlots * kSlotWords;
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int nwarps = nthr >> 5;
+    const int N = (int)a.d_out;
 
-    uint32_t key[E];
-    int nval = 0;
-    load_channel_keys<DT, E>(a, row, sh, h2, key, nval);
-
-    // first level: which high bytes occur
-    for (int b = tid; b < 256; b += nthr) sh.hist1[b] = 0;
-    __syncthreads();
+    // The weights are requested first (the order of the columns does not matter for a histogram:
+    // a thread takes VEC consecutive ones per load), then the row's metadata.
+    constexpr int VEC = E >= 8 ? 8 : 4;
+    constexpr int G = E / VEC;
+    const uint16_t* w = a.W + row * a.ldw;
+    const bool vec = ((a.ldw & (VEC - 1)) == 0) && ((reinterpret_cast<uintptr_t>(a.W) & (2 * VEC - 1)) == 0);
+    uint32_t raw[E / 2];  // two weights per word
 #pragma unroll
-    for (int e = 0; e < E; ++e)
-        if (e < nval) atomicAdd(&sh.hist1[key[e] >> 8], 1);
+    for (int g = 0; g < G; ++g) {
+        const int j0 = (g * nthr + tid) * VEC;
+        if (j0 + VEC - 1 < N && vec) {
+            if (VEC == 8) {
+                const uint4 v = __ldcs(reinterpret_cast<const uint4*>(w + j0));
+                raw[4 * g] = v.x; raw[4 * g + 1] = v.y; raw[4 * g + 2] = v.z; raw[4 * g + 3] = v.w;
+            } else {
+                const uint2 v = __ldcs(reinterpret_cast<const uint2*>(w + j0));
+                raw[2 * g] = v.x; raw[2 * g + 1] = v.y;
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < VEC; u += 2) {
+                const uint32_t a0 = j0 + u < N ? w[j0 + u] : 0u, a1 = j0 + u + 1 < N ? w[j0 + u + 1] : 0u;
+                raw[(g * VEC + u) / 2] = a0 | (a1 << 16);
+            }
+        }
+    }
+    int64_t p0 = 0, p1 = 0;
+    if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
+    const int nrem = (int)(p1 - p0);
+    for (int b = tid; b < 256; b += nthr) sh.hist1[b] = 0;
+    for (int i = tid; i < kSlots * kSlotWords / 4; i += nthr) reinterpret_cast<uint4*>(h2)[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (nrem > kShortList) {
+        for (int i = tid; i < (N + 31) / 32; i += nthr) bitmap[i] = 0;
+        __syncthreads();
+        for (int64_t p = p0 + tid; p < p1; p += nthr) {
+            const int col = a.cols[p];
+            atomicOr(&bitmap[col >> 5], 1u << (col & 31));
+        }
+    } else if (tid < nrem) {
+        sh.rem_list[tid] = a.cols[p0 + tid];
+    }
+    __syncthreads();
+
+    // keys (removed positions and -0 become +0), which high bytes occur, range of the magnitudes
+    uint32_t key[E];
+    uint32_t valid = 0;  // bit e: key[e] is a weight of the row
+    uint32_t amax = 0u, amin1 = 0xffffffffu;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const int j0 = (g * nthr + tid) * VEC;
+        uint32_t rm = 0;  // removed positions among the VEC
+        if (nrem > kShortList) {
+            rm = j0 < N ? (bitmap[j0 >> 5] >> (j0 & 31)) & ((1u << VEC) - 1u) : 0u;  // j0 is a multiple of VEC
+        } else {
+            for (int i = 0; i < nrem; ++i) {
+                const unsigned d = (unsigned)(sh.rem_list[i] - j0);
+                if (d < (unsigned)VEC) rm |= 1u << d;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < VEC; ++u) {
+            const int e = g * VEC + u;
+            uint32_t h = (raw[e >> 1] >> (16 * (e & 1))) & 0xffffu;
+            if ((rm >> u) & 1u) h = 0u;
+            if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
+            const uint32_t ub = h & 0x7fffu;
+            key[e] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+            if (j0 + u < N) {
+                valid |= 1u << e;
+                amax = max(amax, ub);
+                amin1 = min(amin1, ub - 1u);  // zero wraps to the largest value
+                sh.hist1[key[e] >> 8] = 1;
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
+    }
+    if (lane == 0) { sh.wtop[warp] = (int)amax; sh.wulp[warp] = (int)amin1; }
     __syncthreads();
     if (warp == 0) {
-        int flag[8], s = 0;
+        int flag[8], sum = 0;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { flag[u] = sh.hist1[lane * 8 + u] > 0; s += flag[u]; }
-        int incl = s;
+        for (int u = 0; u < 8; ++u) { flag[u] = sh.hist1[lane * 8 + u]; sum += flag[u]; }
+        int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             int up = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += up;
         }
-        int run = incl - s;
+        int run = incl - sum;
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             sh.bucket_rank[lane * 8 + u] = flag[u] ? run : -1;
@@ -134,6 +207,47 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
             run += flag[u];
         }
         if (lane == 31) { sh.n_nonempty = incl; sh.base_nz = 0; sh.base_cnt = 0; }
+    }
+    // Exactness of fp64 sums (see load_channel_keys): first from the magnitude range alone, bit by bit
+    // only for a channel that fails that.  Every warp reduces the per-warp ranges, so the decision is
+    // the same in all threads.
+    if (a.inexact_rows) {
+        amax = lane < nwarps ? (uint32_t)sh.wtop[lane] : 0u;
+        amin1 = lane < nwarps ? (uint32_t)sh.wulp[lane] : 0xffffffffu;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
+        }
+        if (amax != 0u) {
+            const uint32_t fmax = __float_as_uint(widen16<DT>((uint16_t)amax));
+            const uint32_t fmin = __float_as_uint(widen16<DT>((uint16_t)(amin1 + 1u)));
+            const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
+            const int ex_max = (int)(fmax >> 23), ex_min = (int)(fmin >> 23);
+            const int top = ex_max ? ex_max - 127 : (31 - __clz(fmax)) - 149;
+            const int q_low = (ex_min ? ex_min - 150 : -149) + (DT == CMPQ_BF16 ? 16 : 13);
+            if (log2n + 1 + (top + 1 - q_low) > 53) {
+                int q = 100000;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const uint32_t ub = __float_as_uint(value_of_key16<DT>(key[e])) & 0x7fffffffu;
+                    if (((valid >> e) & 1u) && ub) {
+                        const int ex = (int)(ub >> 23);
+                        const uint32_t m = ub & 0x7fffffu;
+                        q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) q = min(q, __shfl_xor_sync(0xffffffffu, q, o));
+                __syncthreads();  // every warp has read wtop / wulp
+                if (lane == 0) sh.wulp[warp] = q;
+                __syncthreads();
+                if (tid == 0) {
+                    for (int wv = 1; wv < nwarps; ++wv) q = min(q, sh.wulp[wv]);
+                    if (log2n + 1 + (top + 1 - q) > 53) atomicAdd(a.inexact_rows, 1);
+                }
+            }
+        }
     }
     __syncthreads();
 
@@ -146,11 +260,13 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         const int words_total = nslots * kSlotWords;
         // Second level: the low byte inside the buckets g0 .. g0 + nslots.  Two 16-bit counters share a
         // word (a channel has fewer than 2^16 weights, so the halves never carry into each other).
-        for (int w = tid; w < words_total / 4; w += nthr) reinterpret_cast<uint4*>(h2)[w] = make_uint4(0u, 0u, 0u, 0u);
-        __syncthreads();  // also: the previous pass has published its bases
+        if (g0 > 0) {  // the counters of the first pass were cleared at the start
+            for (int w = tid; w < words_total / 4; w += nthr) reinterpret_cast<uint4*>(h2)[w] = make_uint4(0u, 0u, 0u, 0u);
+            __syncthreads();  // also: the previous pass has published its bases
+        }
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if (e < nval) {
+            if ((valid >> e) & 1u) {
                 const int r = sh.bucket_rank[key[e] >> 8] - g0;
                 const uint32_t lo = key[e] & 0xffu;
                 if (r >= 0 && r < kSlots) atomicAdd(&h2[r * kSlotWords + (lo >> 1)], 1u << (16 * (lo & 1u)));
@@ -196,7 +312,7 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         keys[run_nz] = 0xffffu;
         cum[run_nz] = (uint16_t)run_cnt;
         ChannelHeader h;
-        h.M = run_nz; h.vmin = sh.vmin; h.vmax = sh.vmax; h.pad = 0;
+        h.M = run_nz;
         t.hdr[row] = h;
     }
 }
@@ -351,7 +467,8 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* w
         __threadfence_block();  // the sums may live in global memory: make them visible to the other lanes
         __syncwarp();
     }
-    const double need = ((double)h.vmax - (double)h.vmin) * (1.0 / 4194304.0);  // range * 2^-22
+    // range * 2^-22, the range being last minus first value of the table
+    const double need = ((double)value_of_key16<DT>(keys[M - 1]) - (double)value_of_key16<DT>(keys[0])) * (1.0 / 4194304.0);
 
     // start: K evenly spaced order statistics; the weight at sorted position pos has the value of the
     // entry e with cum[e] <= pos < cum[e + 1]
@@ -510,8 +627,6 @@ struct RemovedCols {
     const int* list;
     int nrem;
 };
-constexpr int kShortList = 16;
-
 template <int DT, int K, bool ERR>
 __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut,
                            const float* __restrict__ thr, const RemovedCols& rem, uint4 first) {
@@ -648,7 +763,8 @@ lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut, const floa
 
 template <int DT, int E, int MAXT, int MINB>
 static cmpq_status launch_table(const LloydArgs& args, const Tables& t, int threads, cudaStream_t st) {
-    const size_t smem = sizeof(TableShared) + (size_t)kSlots * kSlotWords * sizeof(uint32_t);
+    const size_t smem = sizeof(TableShared) + (size_t)kSlots * kSlotWords * sizeof(uint32_t) +
+                        (((size_t)args.d_out + 31) / 32) * sizeof(uint32_t);
     auto kern = lloyd_table_kernel<DT, E, MAXT, MINB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
