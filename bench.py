@@ -29,7 +29,7 @@ CPU_BASELINE_CHANNELS = 4096   # cpu_baseline leg: the whole layer (about 15 s o
 REFERENCE_ARM_CHANNELS = 1024  # --impl reference: a quarter of the layer per step
 # dram__bytes_read.sum + dram__bytes_write.sum of lloyd_table_kernel per weight, from the ncu capture
 # summarised under profiles/ (None while no capture of the current kernel exists)
-LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT = None
+LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT = 9761536 / (1184 * 4096)
 
 
 def _peaks():

@@ -650,7 +650,7 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
     const bool vec_out = (N & 7) == 0;
     uint8_t* codes = a.codes ? a.codes + row * a.d_out : nullptr;
     float* err = a.err ? a.err + row * a.d_out : nullptr;
-#pragma unroll 2
+#pragma unroll 1
     for (int j0 = tid * 8; j0 < N; j0 += nthr * 8) {
         uint32_t pk[4] = {0u, 0u, 0u, 0u};  // 8 weights, two per word
         if (j0 + 7 < N && vec_in) {

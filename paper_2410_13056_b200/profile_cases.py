@@ -42,6 +42,11 @@ def run_layer(a):
     print("layer %s[%d] d_in=%d d_out=%d tokens=%d budget=%.2f T=%d: %.3f ms per pass, %.0f Mparams/s"
           % (a.config, a.layer, L.d_in, L.d_out, cfg.n_tokens, a.budget, cfg.lloyd_iters, ms, params / ms / 1e3))
     for name in evs[0]:
+        if name == "final_fit_kernels":
+            for i, kernel in enumerate(("table", "iterate", "assign")):
+                t = sum(e[name][i].elapsed_time(e[name][i + 1]) for e in evs) / a.launches
+                print("      final fit, %-12s %.3f ms" % (kernel + " kernel", t))
+            continue
         t = sum(e[name][0].elapsed_time(e[name][1]) for e in evs) / a.launches
         print("   %-24s %.3f ms" % (name, t))
     print("   final-fit distance evaluations: %d, inexact rows: %d"
