@@ -157,18 +157,39 @@ row_scan_kernel(const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
     __shared__ int warp_totals[32];
     const long long take_equal = st->take_equal;
     long long eq_before = 0, out_before = 0;
-    for (int64_t base = 0; base < d_in; base += blockDim.x) {
-        int64_t i = base + threadIdx.x;
-        int e = i < d_in ? eq[i] : 0;
+    // every thread owns kPer consecutive rows of a chunk: two block scans per chunk, loads up front
+    constexpr int kPer = 4;
+    for (int64_t base = 0; base < d_in; base += (int64_t)blockDim.x * kPer) {
+        const int64_t i0 = base + (int64_t)threadIdx.x * kPer;
+        int e[kPer], g[kPer], act[kPer];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            const bool in = i0 + u < d_in;
+            e[u] = in ? eq[i0 + u] : 0;
+            g[u] = in ? gt[i0 + u] : 0;
+            act[u] = in ? is_act[i0 + u] : 0;
+        }
+        int e_sum = 0;
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) e_sum += e[u];
         int tot_e;
-        long long my_eq_before = eq_before + block_exclusive_scan(e, warp_totals, tot_e);
-        long long room = take_equal - my_eq_before;
-        int te = room <= 0 ? 0 : (room < e ? (int)room : e);
-        int sel = 0;
-        if (i < d_in) sel = is_act[i] ? (int)d_out : gt[i] + te;
+        long long my_eq_before = eq_before + block_exclusive_scan(e_sum, warp_totals, tot_e);
+        int te[kPer], sel[kPer], sel_sum = 0;
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            const long long room = take_equal - my_eq_before;
+            te[u] = room <= 0 ? 0 : (room < e[u] ? (int)room : e[u]);
+            my_eq_before += e[u];
+            sel[u] = i0 + u < d_in ? (act[u] ? (int)d_out : g[u] + te[u]) : 0;
+            sel_sum += sel[u];
+        }
         int tot_s;
-        long long my_out_before = out_before + block_exclusive_scan(sel, warp_totals, tot_s);
-        if (i < d_in) { take_eq[i] = te; row_start[i] = my_out_before; }
+        long long my_out_before = out_before + block_exclusive_scan(sel_sum, warp_totals, tot_s);
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            if (i0 + u < d_in) { take_eq[i0 + u] = te[u]; row_start[i0 + u] = my_out_before; }
+            my_out_before += sel[u];
+        }
         eq_before += tot_e;
         out_before += tot_s;
     }

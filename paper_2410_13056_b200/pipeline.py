@@ -116,6 +116,31 @@ class LayerQuantizer:
         return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
                            self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)
 
+    def run_graphed(self, X, W, avg_bits, lloyd_iters):
+        """The same pass replayed from a CUDA graph: the 26 launches of a pass are short enough for launch
+        overhead to show, and nothing in the pass depends on values read back by the host.  The graph is
+        captured on the first call for a given (X, W, budget, iterations) and replayed afterwards; X
+        and W must keep their addresses (their contents may change).  Results as in run()."""
+        key = (X.data_ptr(), W.data_ptr(), tuple(X.shape), float(avg_bits), int(lloyd_iters),
+               B.cmpq_get_lloyd_assignment())
+        if not hasattr(self, "_graphs"):
+            self._graphs = {}
+        entry = self._graphs.get(key)
+        if entry is None:
+            cur = torch.cuda.current_stream()
+            side = torch.cuda.Stream()
+            side.wait_stream(cur)
+            with torch.cuda.stream(side):  # first-use initialisation must not be captured
+                self.run(X, W, avg_bits, lloyd_iters)
+            cur.wait_stream(side)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                result = self.run(X, W, avg_bits, lloyd_iters)
+            entry = (graph, result)
+            self._graphs[key] = entry
+        entry[0].replay()
+        return entry[1]
+
     # ---- host-buffer entry: the same pass with the copies a caller holding host tensors pays ----
     def make_host_outputs(self, avg_bits):
         """Pinned host tensors for everything a caller stores for one quantized layer."""
@@ -133,7 +158,7 @@ class LayerQuantizer:
             self._Wd = torch.empty(W_host.shape, dtype=W_host.dtype, device=self.device)
         self._Xd.copy_(X_host, non_blocking=True)
         self._Wd.copy_(W_host, non_blocking=True)
-        r = self.run(self._Xd, self._Wd, avg_bits, lloyd_iters)
+        r = self.run_graphed(self._Xd, self._Wd, avg_bits, lloyd_iters)
         src = {"bits": r.bits, "rows": r.rows, "cols": r.cols, "vals": r.vals, "lut": r.lut, "packed": r.packed,
                "row_off": r.row_off, "perm": r.perm, "seg_rows": r.seg_rows, "counters": self.counters}
         for k, t in host_out.items():

@@ -181,3 +181,20 @@ def test_llama70b_mlp_shapes_sampled_parity(layer_index):
     g, q = _sampled_parity("c5_mlp70b", layer_index, 2.5)
     assert q.nnz == (1149632 if layer_index == 0 else 1174208)
     assert g["packed"].nbytes == 8192 * 28672 * 5 // 16
+
+
+def test_graph_replay_gives_the_same_bytes_as_the_eager_pass():
+    d_in, d_out, n, T = 192, 1024, 1024, 8
+    W = inputs.make_weight(d_in, d_out, inputs.BF16, 7, device="cuda")
+    X = inputs.make_activations(n, d_in, inputs.BF16, 7, device="cuda")
+    q = LayerQuantizer(d_in, d_out)
+    eager = _np(q.run(X, W, 2.5, T))
+    first = _np(q.run_graphed(X, W, 2.5, T))       # captures, then replays once
+    W2 = inputs.make_weight(d_in, d_out, inputs.BF16, 8, device="cuda")
+    W.copy_(W2)                                       # same address, new contents
+    replay = _np(q.run_graphed(X, W, 2.5, T))
+    again = _np(q.run(X, W, 2.5, T))
+    for k in eager:
+        assert np.array_equal(eager[k], first[k]), k
+        assert np.array_equal(replay[k], again[k]), k
+    assert not np.array_equal(eager["codes"], replay["codes"])
