@@ -33,6 +33,20 @@ cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
 // Ordered formulation: value table per channel, warp-per-channel iterations, streaming last
 // assignment.  `tables` is device scratch of lloyd_tables_bytes(d_in, d_out) bytes, 256-byte aligned.
 size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out);
+// Selection of the worst-fitted entries on the tables of a provisional ordered fit made with neither codes
+// nor errors requested (state: the radix select's SelectState; see outliers.cu for the procedure).
+cmpq_status launch_table_select_hist(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
+                                     const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
+                                     int shift, int bins, unsigned int* hist, cudaStream_t st);
+cmpq_status launch_table_row_count(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
+                                   const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
+                                   int32_t* gt, int32_t* eq, cudaStream_t st);
+cmpq_status launch_table_emit(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint16_t* W, int64_t ldw,
+                              const uint8_t* bits, const uint8_t* is_act, int64_t d_in, int64_t d_out,
+                              const void* state, const int32_t* gt, const int32_t* eq, const int32_t* take_eq,
+                              const int64_t* row_start, int32_t* rows, int32_t* cols, uint16_t* vals,
+                              cudaStream_t st);
+
 // events[0..3] (cudaEvent_t, or NULL to clear): recorded around the three kernels of the next ordered launch.
 void set_lloyd_phase_events(void* const* events);
 cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,

@@ -30,6 +30,7 @@
 // Nothing here is a dense contraction, so no tensor cores are used.
 #include "lloyd.cuh"
 #include "lloyd_device.cuh"
+#include "select.cuh"
 
 #include <cuda_bf16.h>
 
@@ -759,6 +760,294 @@ lloyd_assign_kernel(const LloydArgs a, const float* __restrict__ lut, const floa
 }
 
 // ------------------------------------------------------------------------------------------------
+// Selection of the worst-fitted entries (Section 3.2.2) on the value tables.  The error of a
+// weight depends only on its value, so the radix select and the per-row counts weigh the error of
+// every DISTINCT value with its count instead of reading one error per weight, and the errors are
+// never written to memory; the emit kernel recomputes them for the rows that keep entries.
+
+// Centroids and thresholds of a row of the provisional fit, and the error of a value under them.
+template <int K>
+struct RowFit {
+    float c[K], t[K];
+    bool by_threshold;
+    __device__ __forceinline__ void load(const float* __restrict__ lut, const float* __restrict__ thr, int64_t row) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
+            t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
+        }
+        by_threshold = t[0] != 0.f;
+    }
+    __device__ __forceinline__ uint32_t err_bits(float x) const {
+        uint32_t code;
+        float dist;
+        assign_one<K, true>(x, c, t, by_threshold, code, dist);
+        return __float_as_uint(dist);
+    }
+};
+
+constexpr int kTableSelWarps = 8;
+
+template <int DT, int K>
+__device__ __forceinline__ void table_hist_row(const Tables& t, int64_t row, uint32_t prefix, uint32_t mask, int shift,
+                                               int bins, unsigned int* local) {
+    const int lane = threadIdx.x & 31;
+    RowFit<K> fit;
+    fit.load(t.lut, t.thr, row);
+    const int M = t.hdr[row].M;
+    const uint16_t* keys = t.keys + row * t.stride;
+    const uint16_t* cum = t.cum + row * t.stride;
+    // eight entries per lane and step: two 128-bit loads, the eight errors are independent
+    for (int j0 = lane * 8; j0 < M; j0 += 256) {
+        const Eight k8 = load_eight(keys + j0), c8 = load_eight(cum + j0);
+        const uint32_t c_end = j0 + 8 <= M ? cum[j0 + 8] : 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (j0 + u < M) {
+                const uint32_t e = fit.err_bits(value_of_key16<DT>(k8.at(u)));
+                const uint32_t cnt = (u < 7 ? c8.at(u + 1) : c_end) - c8.at(u);
+                if ((e & mask) == prefix) atomicAdd(&local[(e >> shift) & (bins - 1)], cnt);
+            }
+        }
+    }
+}
+
+// hist[d] += number of weights in non-act rows whose error has the fixed bits of the prefix and the
+// digit d at `shift`.  One warp per row, block-local histogram first.
+template <int DT>
+__global__ void __launch_bounds__(kTableSelWarps * 32)
+table_select_hist_kernel(const Tables t, const uint8_t* __restrict__ bits, const uint8_t* __restrict__ is_act,
+                         int64_t d_in, const SelectState* __restrict__ st, int shift, int bins,
+                         unsigned int* __restrict__ hist) {
+    __shared__ unsigned int local[kSelBins];
+    for (int b = threadIdx.x; b < bins; b += blockDim.x) local[b] = 0;
+    __syncthreads();
+    const uint32_t prefix = st->prefix, mask = st->mask;
+    const int warp = threadIdx.x >> 5;
+    for (int64_t row = (int64_t)blockIdx.x * kTableSelWarps + warp; row < d_in; row += (int64_t)gridDim.x * kTableSelWarps) {
+        if (is_act[row]) continue;
+        const int b = bits[row];
+        if (b == 2) table_hist_row<DT, 4>(t, row, prefix, mask, shift, bins, local);
+        else if (b == 3) table_hist_row<DT, 8>(t, row, prefix, mask, shift, bins, local);
+        else table_hist_row<DT, 16>(t, row, prefix, mask, shift, bins, local);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < bins; b += blockDim.x)
+        if (local[b]) atomicAdd(&hist[b], local[b]);
+}
+
+template <int DT, int K>
+__device__ __forceinline__ void table_count_row(const Tables& t, int64_t row, uint32_t tau, int& g, int& q) {
+    const int lane = threadIdx.x & 31;
+    RowFit<K> fit;
+    fit.load(t.lut, t.thr, row);
+    const int M = t.hdr[row].M;
+    const uint16_t* keys = t.keys + row * t.stride;
+    const uint16_t* cum = t.cum + row * t.stride;
+    for (int j0 = lane * 8; j0 < M; j0 += 256) {
+        const Eight k8 = load_eight(keys + j0), c8 = load_eight(cum + j0);
+        const uint32_t c_end = j0 + 8 <= M ? cum[j0 + 8] : 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (j0 + u < M) {
+                const uint32_t e = fit.err_bits(value_of_key16<DT>(k8.at(u)));
+                const int cnt = (int)((u < 7 ? c8.at(u + 1) : c_end) - c8.at(u));
+                g += e > tau ? cnt : 0;
+                q += e == tau ? cnt : 0;
+            }
+        }
+    }
+}
+
+// Per row: how many errors exceed tau and how many equal it.  One warp per row.
+template <int DT>
+__global__ void __launch_bounds__(kTableSelWarps * 32)
+table_row_count_kernel(const Tables t, const uint8_t* __restrict__ bits, const uint8_t* __restrict__ is_act,
+                       int64_t d_in, const SelectState* __restrict__ st, int32_t* __restrict__ gt,
+                       int32_t* __restrict__ eq) {
+    const int64_t row = (int64_t)blockIdx.x * kTableSelWarps + (threadIdx.x >> 5);
+    if (row >= d_in) return;
+    int g = 0, q = 0;
+    if (!is_act[row]) {
+        const uint32_t tau = st->tau;
+        const int b = bits[row];
+        if (b == 2) table_count_row<DT, 4>(t, row, tau, g, q);
+        else if (b == 3) table_count_row<DT, 8>(t, row, tau, g, q);
+        else table_count_row<DT, 16>(t, row, tau, g, q);
+    }
+    g = warp_sum(g);
+    q = warp_sum(q);
+    if ((threadIdx.x & 31) == 0) { gt[row] = g; eq[row] = q; }
+}
+
+// Kept entries of one non-act row in column order; errors recomputed from the weights.  Same
+// procedure as the emit kernel that reads materialised errors: candidates (error >= tau) go to a
+// short list that is ordered by counting; a row with more candidates uses scan-based compaction.
+template <int DT, int K>
+__device__ void table_emit_row(const uint16_t* __restrict__ w, int64_t d_out, const Tables& t, int64_t row,
+                               uint32_t tau, int te, int ncand, int64_t out0, int32_t* __restrict__ rows,
+                               int32_t* __restrict__ cols, uint16_t* __restrict__ vals, int* warp_totals,
+                               int* list_col, unsigned char* list_eq, int* list_n) {
+    RowFit<K> fit;
+    fit.load(t.lut, t.thr, row);
+    auto err_at = [&](int64_t j) {
+        float x = widen16<DT>(w[j]);
+        x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
+        return fit.err_bits(x);
+    };
+    if (ncand <= kEmitListCap) {
+        if (threadIdx.x == 0) *list_n = 0;
+        __syncthreads();
+        const bool vec = ((reinterpret_cast<uintptr_t>(w) & 15) == 0);
+        for (int64_t j0 = (int64_t)threadIdx.x * 8; j0 < d_out; j0 += (int64_t)blockDim.x * 8) {
+            uint32_t pk[4] = {0u, 0u, 0u, 0u};
+            if (j0 + 7 < d_out && vec) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(w + j0));
+                pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
+            } else {
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (j0 + u < d_out) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float x = widen16<DT>((uint16_t)(pk[u >> 1] >> (16 * (u & 1))));
+                x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
+                const uint32_t e = fit.err_bits(x);
+                if (j0 + u < d_out && e >= tau) {
+                    const int p = atomicAdd(list_n, 1);
+                    if (p < kEmitListCap) {
+                        list_col[p] = (int)(j0 + u);
+                        list_eq[p] = e == tau ? 1 : 0;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        const int n = *list_n < kEmitListCap ? *list_n : kEmitListCap;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int c = list_col[i];
+            const int is_eq = list_eq[i];
+            int before = 0, eq_before = 0;  // candidates / tau-candidates in lower columns
+            for (int u = 0; u < n; ++u) {
+                const int lower = list_col[u] < c ? 1 : 0;
+                before += lower;
+                eq_before += lower & list_eq[u];
+            }
+            const bool keep = !is_eq || eq_before < te;
+            if (keep) {
+                // dropped tau-candidates are exactly those of tau-rank >= te, all after the kept ones
+                const int dropped_before = eq_before > te ? eq_before - te : 0;
+                const int64_t pos = out0 + before - dropped_before;
+                rows[pos] = (int32_t)row;
+                cols[pos] = c;
+                vals[pos] = w[c];
+            }
+        }
+        return;
+    }
+    int eq_seen = 0, written = 0;
+    for (int64_t base = 0; base < d_out; base += blockDim.x) {
+        const int64_t j = base + threadIdx.x;
+        const bool in = j < d_out;
+        const uint32_t u = in ? err_at(j) : 0u;
+        const int is_eq = (in && u == tau) ? 1 : 0;
+        int tot_eq;
+        const int eq_rank = eq_seen + block_exclusive_scan(is_eq, warp_totals, tot_eq);
+        const int keep = in && (u > tau || (is_eq && eq_rank < te)) ? 1 : 0;
+        int tot_keep;
+        const int pos = written + block_exclusive_scan(keep, warp_totals, tot_keep);
+        if (keep) {
+            rows[out0 + pos] = (int32_t)row;
+            cols[out0 + pos] = (int32_t)j;
+            vals[out0 + pos] = w[j];
+        }
+        eq_seen += tot_eq;
+        written += tot_keep;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kSelThreads)
+table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, const uint8_t* __restrict__ bits,
+                  const uint8_t* __restrict__ is_act, int64_t d_out, const SelectState* __restrict__ st,
+                  const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
+                  const int32_t* __restrict__ take_eq, const int64_t* __restrict__ row_start,
+                  int32_t* __restrict__ rows, int32_t* __restrict__ cols, uint16_t* __restrict__ vals) {
+    __shared__ int warp_totals[32];
+    __shared__ int list_col[kEmitListCap];
+    __shared__ unsigned char list_eq[kEmitListCap];
+    __shared__ int list_n;
+    const int64_t row = blockIdx.x;
+    const int64_t out0 = row_start[row];
+    if (row_start[row + 1] == out0) return;
+    const uint16_t* w = W + row * ldw;
+    if (is_act[row]) {
+        for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
+            rows[out0 + j] = (int32_t)row;
+            cols[out0 + j] = (int32_t)j;
+            vals[out0 + j] = w[j];
+        }
+        return;
+    }
+    const uint32_t tau = st->tau;
+    const int te = take_eq[row];
+    const int ncand = gt[row] + eq[row];
+    const int b = bits[row];
+    if (b == 2) table_emit_row<DT, 4>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
+    else if (b == 3) table_emit_row<DT, 8>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
+    else table_emit_row<DT, 16>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
+}
+
+static Tables tables_at(void* tables, size_t tables_bytes, int64_t d_in, int64_t d_out) {
+    Workspace w(tables, tables_bytes);
+    return carve_tables(w, d_in, d_out);
+}
+
+cmpq_status launch_table_select_hist(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
+                                     const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
+                                     int shift, int bins, unsigned int* hist, cudaStream_t st) {
+    const Tables t = tables_at(tables, tables_bytes, d_in, d_out);
+    const int sms = sm_count();
+    if (sms <= 0) return CMPQ_ERR_CUDA;
+    int64_t blocks = (d_in + kTableSelWarps - 1) / kTableSelWarps;
+    if (blocks > (int64_t)sms * 4) blocks = (int64_t)sms * 4;
+    const SelectState* ss = static_cast<const SelectState*>(state);
+    if (dt == CMPQ_F16)
+        table_select_hist_kernel<CMPQ_F16><<<(unsigned)blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, shift, bins, hist);
+    else
+        table_select_hist_kernel<CMPQ_BF16><<<(unsigned)blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, shift, bins, hist);
+    return launch_status();
+}
+
+cmpq_status launch_table_row_count(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
+                                   const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
+                                   int32_t* gt, int32_t* eq, cudaStream_t st) {
+    const Tables t = tables_at(tables, tables_bytes, d_in, d_out);
+    const unsigned blocks = (unsigned)((d_in + kTableSelWarps - 1) / kTableSelWarps);
+    const SelectState* ss = static_cast<const SelectState*>(state);
+    if (dt == CMPQ_F16)
+        table_row_count_kernel<CMPQ_F16><<<blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, gt, eq);
+    else
+        table_row_count_kernel<CMPQ_BF16><<<blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, gt, eq);
+    return launch_status();
+}
+
+cmpq_status launch_table_emit(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint16_t* W, int64_t ldw,
+                              const uint8_t* bits, const uint8_t* is_act, int64_t d_in, int64_t d_out,
+                              const void* state, const int32_t* gt, const int32_t* eq, const int32_t* take_eq,
+                              const int64_t* row_start, int32_t* rows, int32_t* cols, uint16_t* vals,
+                              cudaStream_t st) {
+    const Tables t = tables_at(tables, tables_bytes, d_in, d_out);
+    const SelectState* ss = static_cast<const SelectState*>(state);
+    if (dt == CMPQ_F16)
+        table_emit_kernel<CMPQ_F16><<<(unsigned)d_in, kSelThreads, 0, st>>>(W, ldw, t, bits, is_act, d_out, ss, gt, eq, take_eq, row_start, rows, cols, vals);
+    else
+        table_emit_kernel<CMPQ_BF16><<<(unsigned)d_in, kSelThreads, 0, st>>>(W, ldw, t, bits, is_act, d_out, ss, gt, eq, take_eq, row_start, rows, cols, vals);
+    return launch_status();
+}
+
+// ------------------------------------------------------------------------------------------------
 // host side
 
 template <int DT, int E, int MAXT, int MINB>
@@ -830,8 +1119,9 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cud
     if (s != CMPQ_OK) return s;
     if (ev[2]) cudaEventRecord(ev[2], st);
 
+    // neither codes nor errors wanted: the fit alone (centroids and thresholds stay in the tables)
     if (args.err) lloyd_assign_kernel<DT, true><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
-    else lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
+    else if (args.codes) lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
     s = launch_status();
     if (ev[3]) cudaEventRecord(ev[3], st);
     return s;

@@ -4,47 +4,22 @@
 //   O_q    after a provisional channel-wise K-means of W' = W - O_act, the n_q entries with the
 //          largest error |W' - W'_q| are kept as well (equal errors: smaller linear index first)
 //
-// The provisional fit writes one fp32 error per weight.  Errors are non-negative, so their
+// Errors are non-negative, so their
 // bit patterns order like integers: an exact three-pass radix select (12 + 10 + 10 bits) finds
 // the bit pattern tau of the n_q-th largest error and how many entries equal to tau still
 // belong to the set.  Per-row counts and one scan over the rows then give every row its slice
 // of the output, and each row writes its entries in column order, which yields the list sorted
 // by (row, col) without a sort.
+//
+// Where the errors come from depends on the K-means formulation.  The all-pairs kernel writes one
+// fp32 error per weight and the kernels in this file read them.  The ordered formulation never
+// writes them: the error of a weight depends only on its value, so the select and the per-row
+// counts run on the value tables of the fit (every distinct value weighed with its count) and the
+// emit step recomputes the errors of the rows that keep entries (kernels in lloyd_hist.cu).
 #include "lloyd.cuh"
+#include "select.cuh"
 
 namespace cmpq {
-
-constexpr int kSelBins = 4096;
-constexpr int kSelThreads = 256;
-
-struct SelectState {
-    uint32_t prefix;        // bits of tau fixed so far
-    uint32_t mask;          // which bits are fixed
-    long long remaining;    // entries still to take among those matching prefix
-    uint32_t tau;           // final threshold pattern
-    long long take_equal;   // entries equal to tau that belong to the set
-};
-
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_totals, int& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    int incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    __syncthreads();  // warp_totals may still be read from a previous call
-    if (lane == 31) warp_totals[warp] = incl;
-    __syncthreads();
-    int base = 0, all = 0;
-    for (int w = 0; w < nwarps; ++w) {
-        int t = warp_totals[w];
-        if (w < warp) base += t;
-        all += t;
-    }
-    total = all;
-    return base + incl - v;
-}
 
 __global__ void mark_act_rows_kernel(const int32_t* __restrict__ rank, int64_t d_in, int64_t n_act,
                                      uint8_t* __restrict__ is_act) {
@@ -201,8 +176,6 @@ row_scan_kernel(const int32_t* __restrict__ gt, const int32_t* __restrict__ eq,
 // shared memory, ordered by column by counting, and the first take_eq[row] of those equal to tau
 // are kept next to all larger ones.  A row with more candidates than the list holds falls back
 // to a scan-based ordered compaction.
-constexpr int kEmitListCap = 1024;
-
 __global__ void __launch_bounds__(kSelThreads)
 emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __restrict__ err,
             const uint8_t* __restrict__ is_act, int64_t d_out, const SelectState* __restrict__ st,
@@ -348,6 +321,10 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
     OutlierWs o = carve(wsp, d_in, d_out);
     const unsigned row_blocks = (unsigned)((d_in + 255) / 256);
 
+    const bool all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
+    const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
+    const uint16_t* Wp = static_cast<const uint16_t*>(W);
+
     cmpq_status s = launch_rank(a, d_in, o.rank, st);
     if (s != CMPQ_OK) return s;
     mark_act_rows_kernel<<<row_blocks, 256, 0, st>>>(o.rank, d_in, n_act, o.is_act);
@@ -359,10 +336,10 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
         la.bits = bits;
         la.iters = lloyd_iters;
         la.skip_row = o.is_act;
-        la.err = o.err;
-        s = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS
-                ? launch_lloyd(la, dt, st)
-                : launch_lloyd_ordered(la, dt, o.tables, lloyd_tables_bytes(d_in, d_out), st);
+        // all pairs: one fp32 error per weight is written; ordered: the fit alone, errors are then
+        // taken from the value tables
+        la.err = all_pairs ? o.err : nullptr;
+        s = all_pairs ? launch_lloyd(la, dt, st) : launch_lloyd_ordered(la, dt, o.tables, tables_bytes, st);
         if (s != CMPQ_OK) return s;
     }
 
@@ -375,16 +352,31 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
         const int shifts[3] = {20, 10, 0};
         const int bins[3] = {4096, 1024, 1024};
         for (int p = 0; p < 3; ++p) {
-            select_hist_kernel<<<hist_blocks, kSelThreads, 0, st>>>(o.err, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist);
+            if (all_pairs) {
+                select_hist_kernel<<<hist_blocks, kSelThreads, 0, st>>>(o.err, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist);
+            } else {
+                s = launch_table_select_hist(o.tables, tables_bytes, dt, bits, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist, st);
+                if (s != CMPQ_OK) return s;
+            }
             select_digit_kernel<<<1, 1024, 0, st>>>(o.hist, shifts[p], bins[p], o.state, p == 2);
         }
-        row_count_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(o.err, o.is_act, d_out, o.state, o.gt, o.eq);
+        if (all_pairs) {
+            row_count_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(o.err, o.is_act, d_out, o.state, o.gt, o.eq);
+        } else {
+            s = launch_table_row_count(o.tables, tables_bytes, dt, bits, o.is_act, d_in, d_out, o.state, o.gt, o.eq, st);
+            if (s != CMPQ_OK) return s;
+        }
     } else {
         if (cudaMemsetAsync(o.gt, 0, (size_t)d_in * sizeof(int32_t), st) != cudaSuccess) return CMPQ_ERR_CUDA;
         if (cudaMemsetAsync(o.eq, 0, (size_t)d_in * sizeof(int32_t), st) != cudaSuccess) return CMPQ_ERR_CUDA;
     }
     row_scan_kernel<<<1, 1024, 0, st>>>(o.gt, o.eq, o.is_act, d_in, d_out, o.state, o.take_eq, o.row_start);
-    if (nnz_out > 0)
-        emit_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(static_cast<const uint16_t*>(W), ldw, o.err, o.is_act, d_out, o.state, o.gt, o.eq, o.take_eq, o.row_start, rows, cols, vals);
+    if (nnz_out > 0) {
+        // with n_q == 0 no row outside O_act keeps anything, so neither errors nor tables are read
+        if (all_pairs || n_q == 0)
+            emit_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(Wp, ldw, o.err, o.is_act, d_out, o.state, o.gt, o.eq, o.take_eq, o.row_start, rows, cols, vals);
+        else
+            return launch_table_emit(o.tables, tables_bytes, dt, Wp, ldw, bits, o.is_act, d_in, d_out, o.state, o.gt, o.eq, o.take_eq, o.row_start, rows, cols, vals, st);
+    }
     return launch_status();
 }

@@ -15,15 +15,16 @@ from . import binding as B
 # CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0:
 # statistic 2 + finalize 1, allocation 2, outliers 12 + the K-means (rank, mark, select init, 3 x
 # (histogram, digit), row count, row scan, emit), final fit 1 (row index) + the K-means, packing 2.
-# A K-means call is 3 kernels (table, iterate, assign) by default, 1 with ASSIGN_ALL_PAIRS.
+# The K-means is 1 kernel per fit with ASSIGN_ALL_PAIRS; by default the final fit is 3 kernels (table,
+# iterate, assign) and the provisional fit 2 (its errors are never written: the selection works on the
+# value tables).
 def kernels_per_run(assignment=None):
     if assignment is None:
         assignment = B.cmpq_get_lloyd_assignment()
-    per_kmeans = 1 if assignment == B.ASSIGN_ALL_PAIRS else 3
-    return 20 + 2 * per_kmeans
+    return 20 + (2 if assignment == B.ASSIGN_ALL_PAIRS else 5)
 
 
-KERNELS_PER_RUN = 26  # with the default assignment
+KERNELS_PER_RUN = 25  # with the default assignment
 
 
 @dataclass
