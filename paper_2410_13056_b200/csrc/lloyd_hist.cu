@@ -351,21 +351,18 @@ __device__ __forceinline__ int search_entries(const uint16_t* keys, int M, float
             return fabsf(v - ck) < fabsf(v - cm);
         };
         if (e_prev >= 0) {
+            // gallop away from the old boundary p, downwards if the predicate holds at p and upwards if
+            // not, in one loop for both directions (lanes of both kinds then share the instructions)
             const int p = e_prev < M ? e_prev : M;
-            if (p >= M || pred(p)) {  // the boundary is at or below p: gallop downwards
-                hi = p;
-                for (int step = 1;; step <<= 1) {
-                    const int q = hi - step;
-                    if (q < 0) break;
-                    if (pred(q)) { hi = q; } else { lo = q + 1; break; }
-                }
-            } else {                  // the boundary is above p: gallop upwards
-                lo = p + 1;
-                for (int step = 1;; step <<= 1) {
-                    const int q = lo - 1 + step;
-                    if (q >= M) break;
-                    if (pred(q)) { hi = q; break; } else { lo = q + 1; }
-                }
+            const bool down = p >= M || pred(p);
+            if (down) hi = p; else lo = p + 1;
+            bool open = true;
+            for (int step = 1; open; step <<= 1) {
+                const int q = down ? hi - step : lo - 1 + step;
+                if (q < 0 || q >= M) break;  // ran off the table: the bracket is [0, hi] or [lo, M]
+                const bool t = pred(q);
+                if (t) hi = q; else lo = q + 1;
+                open = (t == down);          // closed by the first false (down) or the first true (up)
             }
         }
         while (lo < hi) {
