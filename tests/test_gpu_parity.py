@@ -215,3 +215,55 @@ def test_phase_events_bracket_the_three_kernels_once():
     B.cmpq_lloyd_phase_events(None)   # cancel
     with pytest.raises(B.CmpqError):
         B._check(B.lib().cmpq_lloyd_phase_events(1, None, None, None), "cmpq_lloyd_phase_events")
+
+
+# ----------------------------------------------------------------------------- value tables: less common shapes
+def _log_uniform(d_in, d_out, lo_exp, hi_exp, seed, tdt):
+    """Weights with magnitudes spread evenly over many binades and both signs: many distinct 16-bit
+    values and many occupied high bytes, unlike Gaussian-like weights."""
+    rng = np.random.default_rng(seed)
+    mag = np.exp2(rng.uniform(lo_exp, hi_exp, (d_in, d_out)))
+    sign = np.where(rng.random((d_in, d_out)) < 0.5, -1.0, 1.0)
+    return torch.tensor(mag * sign, dtype=torch.float32).to(tdt).cuda()
+
+
+@pytest.mark.parametrize("dtype,tdt,d_in,d_out,lo,hi", [
+    (inputs.BF16, torch.bfloat16, 12, 768, -20, 13),     # more than 32 occupied high bytes: several table passes
+    (inputs.BF16, torch.bfloat16, 3, 32768, -9, 3),      # more distinct values than a warp stages in shared memory
+    (inputs.F16, torch.float16, 6, 8192, -14, 3),        # fp16: both at once
+])
+def test_quantize_layer_wide_value_tables(dtype, tdt, d_in, d_out, lo, hi, assignment):
+    W = _log_uniform(d_in, d_out, lo, hi, 3 + d_out, tdt)
+    Wu = inputs.as_u16(W)
+    bits = np.array([2, 3, 4] * d_in, np.uint8)[:d_in]
+    none = np.zeros(0, np.int32)
+    assert max(len(np.unique(r)) for r in Wu) > 600   # the shapes above rely on many distinct values
+    lut, codes, inexact, _ = G.gpu_quantize(W, bits, none, none, 9)
+    rlut, rcodes = oracle.quantize_layer(Wu, dtype, bits, none, none, 9)
+    assert inexact == 0
+    assert np.array_equal(codes, rcodes)
+    assert np.array_equal(lut.view(np.uint32), rlut.view(np.uint32))
+
+
+@pytest.mark.parametrize("per_row", [1, 15, 16, 17, 40])
+def test_quantize_layer_removed_positions_list_and_bitmap(per_row, assignment):
+    d_in, d_out, T = 10, 2048, 7
+    W, Wu, a, bits = _case(d_in, d_out, inputs.BF16, 99, 3.0)
+    rng = np.random.default_rng(per_row)
+    lin = np.sort(np.concatenate([i * d_out + rng.choice(d_out, per_row, replace=False) for i in range(d_in)]))
+    rows, cols = (lin // d_out).astype(np.int32), (lin % d_out).astype(np.int32)
+    lut, codes, inexact, _ = G.gpu_quantize(W, bits, rows, cols, T)
+    rlut, rcodes = oracle.quantize_layer(Wu, inputs.BF16, bits, rows, cols, T)
+    assert np.array_equal(codes, rcodes)
+    assert np.array_equal(lut.view(np.uint32), rlut.view(np.uint32))
+
+
+def test_extract_outliers_wide_value_tables(assignment):
+    d_in, d_out = 9, 4096
+    W = _log_uniform(d_in, d_out, -12, 2, 17, torch.float16)
+    a = np.arange(d_in, dtype=np.float32)[::-1].copy()
+    bits = np.array([2, 3, 4] * 3, np.uint8)
+    got = G.gpu_extract(W, a, bits, 1, 300, 6)
+    ref = oracle.extract_outliers(inputs.as_u16(W), inputs.F16, a, bits, 1, 300, 6)
+    for g, r in zip(got, ref):
+        assert np.array_equal(g, r)
