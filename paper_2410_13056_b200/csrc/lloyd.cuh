@@ -36,8 +36,8 @@ size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out);
 // Selection of the worst-fitted entries on the tables of a provisional ordered fit made with neither codes
 // nor errors requested (state: the radix select's SelectState; see outliers.cu for the procedure).
 cmpq_status launch_table_select_hist(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
-                                     const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
-                                     int shift, int bins, unsigned int* hist, cudaStream_t st);
+                                     const uint8_t* is_act, int64_t d_in, int64_t d_out, void* state,
+                                     int shift, int bins, int final_pass, unsigned int* hist, cudaStream_t st);
 cmpq_status launch_table_row_count(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
                                    const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
                                    int32_t* gt, int32_t* eq, cudaStream_t st);

@@ -814,9 +814,11 @@ __device__ __forceinline__ void table_hist_row(const Tables& t, int64_t row, uin
 template <int DT>
 __global__ void __launch_bounds__(kTableSelWarps * 32)
 table_select_hist_kernel(const Tables t, const uint8_t* __restrict__ bits, const uint8_t* __restrict__ is_act,
-                         int64_t d_in, const SelectState* __restrict__ st, int shift, int bins,
-                         unsigned int* __restrict__ hist) {
+                         int64_t d_in, SelectState* st, int shift, int bins, int final_pass, unsigned int* hist) {
     __shared__ unsigned int local[kSelBins];
+    __shared__ int warp_totals[32];
+    __shared__ int found_digit, is_last;
+    __shared__ long long found_above;
     for (int b = threadIdx.x; b < bins; b += blockDim.x) local[b] = 0;
     __syncthreads();
     const uint32_t prefix = st->prefix, mask = st->mask;
@@ -831,6 +833,17 @@ table_select_hist_kernel(const Tables t, const uint8_t* __restrict__ bits, const
     __syncthreads();
     for (int b = threadIdx.x; b < bins; b += blockDim.x)
         if (local[b]) atomicAdd(&hist[b], local[b]);
+    // The block that finishes last fixes the digit (no block waits for another: a counter tells which
+    // one is last) and leaves the histogram and the counter cleared for the next pass.
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(&st->done, 1u) == gridDim.x - 1 ? 1 : 0;
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        select_digit_block<kTableSelWarps * 32>(hist, shift, bins, st, final_pass, warp_totals, &found_digit, &found_above);
+        if (threadIdx.x == 0) st->done = 0;
+    }
 }
 
 template <int DT, int K>
@@ -1002,18 +1015,18 @@ static Tables tables_at(void* tables, size_t tables_bytes, int64_t d_in, int64_t
 }
 
 cmpq_status launch_table_select_hist(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
-                                     const uint8_t* is_act, int64_t d_in, int64_t d_out, const void* state,
-                                     int shift, int bins, unsigned int* hist, cudaStream_t st) {
+                                     const uint8_t* is_act, int64_t d_in, int64_t d_out, void* state,
+                                     int shift, int bins, int final_pass, unsigned int* hist, cudaStream_t st) {
     const Tables t = tables_at(tables, tables_bytes, d_in, d_out);
     const int sms = sm_count();
     if (sms <= 0) return CMPQ_ERR_CUDA;
     int64_t blocks = (d_in + kTableSelWarps - 1) / kTableSelWarps;
     if (blocks > (int64_t)sms * 4) blocks = (int64_t)sms * 4;
-    const SelectState* ss = static_cast<const SelectState*>(state);
+    SelectState* ss = static_cast<SelectState*>(state);
     if (dt == CMPQ_F16)
-        table_select_hist_kernel<CMPQ_F16><<<(unsigned)blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, shift, bins, hist);
+        table_select_hist_kernel<CMPQ_F16><<<(unsigned)blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, shift, bins, final_pass, hist);
     else
-        table_select_hist_kernel<CMPQ_BF16><<<(unsigned)blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, shift, bins, hist);
+        table_select_hist_kernel<CMPQ_BF16><<<(unsigned)blocks, kTableSelWarps * 32, 0, st>>>(t, bits, is_act, d_in, ss, shift, bins, final_pass, hist);
     return launch_status();
 }
 

@@ -28,7 +28,7 @@ __global__ void mark_act_rows_kernel(const int32_t* __restrict__ rank, int64_t d
 }
 
 __global__ void select_init_kernel(SelectState* st, long long n_q) {
-    st->prefix = 0; st->mask = 0; st->remaining = n_q; st->tau = 0xffffffffu; st->take_equal = 0;
+    st->prefix = 0; st->mask = 0; st->remaining = n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0;
 }
 
 // hist[d] += number of errors in non-act rows whose fixed bits match the prefix and whose
@@ -54,43 +54,12 @@ select_hist_kernel(const float* __restrict__ err, const uint8_t* __restrict__ is
         if (local[b]) atomicAdd(&hist[b], local[b]);
 }
 
-// Walks the histogram from the largest digit down to the one that holds the remaining-th
-// largest entry, fixes that digit in the prefix and clears the histogram for the next pass.
 __global__ void __launch_bounds__(1024)
 select_digit_kernel(unsigned int* __restrict__ hist, int shift, int bins, SelectState* st, int final_pass) {
     __shared__ int warp_totals[32];
     __shared__ int found_digit;
     __shared__ long long found_above;
-    const int per = kSelBins / 1024;  // 4 bins per thread, descending digit order
-    const long long remaining = st->remaining;
-    int v[per], s = 0;
-#pragma unroll
-    for (int t = 0; t < per; ++t) {
-        int d = bins - 1 - (threadIdx.x * per + t);
-        v[t] = d >= 0 ? (int)hist[d] : 0;
-        s += v[t];
-    }
-    if (threadIdx.x == 0) found_digit = -1;
-    int total;
-    long long above = block_exclusive_scan(s, warp_totals, total);  // entries with a larger digit
-    if (remaining > 0 && above < remaining && remaining <= above + s) {
-#pragma unroll
-        for (int t = 0; t < per; ++t) {
-            if (above < remaining && remaining <= above + v[t]) {
-                found_digit = bins - 1 - (threadIdx.x * per + t);
-                found_above = above;
-            }
-            above += v[t];
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0 && found_digit >= 0) {
-        st->prefix |= (uint32_t)found_digit << shift;
-        st->mask |= (uint32_t)(bins - 1) << shift;
-        st->remaining = remaining - found_above;
-        if (final_pass) { st->tau = st->prefix; st->take_equal = st->remaining; }
-    }
-    for (int b = threadIdx.x; b < bins; b += blockDim.x) hist[b] = 0;
+    select_digit_block<1024>(hist, shift, bins, st, final_pass, warp_totals, &found_digit, &found_above);
 }
 
 // Per row: how many errors exceed tau and how many equal it.
@@ -354,11 +323,11 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
         for (int p = 0; p < 3; ++p) {
             if (all_pairs) {
                 select_hist_kernel<<<hist_blocks, kSelThreads, 0, st>>>(o.err, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist);
-            } else {
-                s = launch_table_select_hist(o.tables, tables_bytes, dt, bits, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist, st);
+                select_digit_kernel<<<1, 1024, 0, st>>>(o.hist, shifts[p], bins[p], o.state, p == 2);
+            } else {  // the last block of the histogram kernel to finish also fixes the digit
+                s = launch_table_select_hist(o.tables, tables_bytes, dt, bits, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], p == 2, o.hist, st);
                 if (s != CMPQ_OK) return s;
             }
-            select_digit_kernel<<<1, 1024, 0, st>>>(o.hist, shifts[p], bins[p], o.state, p == 2);
         }
         if (all_pairs) {
             row_count_kernel<<<(unsigned)d_in, kSelThreads, 0, st>>>(o.err, o.is_act, d_out, o.state, o.gt, o.eq);

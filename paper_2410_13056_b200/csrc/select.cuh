@@ -15,6 +15,7 @@ struct SelectState {
     long long remaining;    // entries still to take among those matching prefix
     uint32_t tau;           // final threshold pattern
     long long take_equal;   // entries equal to tau that belong to the set
+    unsigned int done;      // blocks of the running histogram kernel that have added their counts
 };
 
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_totals, int& total) {
@@ -36,6 +37,45 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_totals, int
     }
     total = all;
     return base + incl - v;
+}
+
+// One block: walks the histogram from the largest digit down to the one that holds the
+// remaining-th largest entry, fixes that digit in the prefix and clears the histogram for the next
+// pass.  THREADS = blockDim.x; the histogram is read past the L1 cache (other blocks wrote it).
+template <int THREADS>
+__device__ __forceinline__ void select_digit_block(unsigned int* hist, int shift, int bins, SelectState* st,
+                                                   int final_pass, int* warp_totals, int* found_digit,
+                                                   long long* found_above) {
+    constexpr int per = kSelBins / THREADS;  // bins per thread, descending digit order
+    const long long remaining = st->remaining;
+    int v[per], s = 0;
+#pragma unroll
+    for (int t = 0; t < per; ++t) {
+        const int d = bins - 1 - (threadIdx.x * per + t);
+        v[t] = d >= 0 ? (int)__ldcg(hist + d) : 0;
+        s += v[t];
+    }
+    if (threadIdx.x == 0) *found_digit = -1;
+    int total;
+    long long above = block_exclusive_scan(s, warp_totals, total);  // entries with a larger digit
+    if (remaining > 0 && above < remaining && remaining <= above + s) {
+#pragma unroll
+        for (int t = 0; t < per; ++t) {
+            if (above < remaining && remaining <= above + v[t]) {
+                *found_digit = bins - 1 - (threadIdx.x * per + t);
+                *found_above = above;
+            }
+            above += v[t];
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && *found_digit >= 0) {
+        st->prefix |= (uint32_t)*found_digit << shift;
+        st->mask |= (uint32_t)(bins - 1) << shift;
+        st->remaining = remaining - *found_above;
+        if (final_pass) { st->tau = st->prefix; st->take_equal = st->remaining; }
+    }
+    for (int b = threadIdx.x; b < bins; b += THREADS) hist[b] = 0;
 }
 
 constexpr int kEmitListCap = 1024;  // candidates of a row ordered in shared memory; more: scan-based compaction

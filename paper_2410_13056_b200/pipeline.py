@@ -12,19 +12,16 @@ import torch
 
 from . import binding as B
 
-# CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0:
-# statistic 2 + finalize 1, allocation 2, outliers 12 + the K-means (rank, mark, select init, 3 x
-# (histogram, digit), row count, row scan, emit), final fit 1 (row index) + the K-means, packing 2.
-# The K-means is 1 kernel per fit with ASSIGN_ALL_PAIRS; by default the final fit is 3 kernels (table,
-# iterate, assign) and the provisional fit 2 (its errors are never written: the selection works on the
-# value tables).
+# CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0.
+# ASSIGN_ALL_PAIRS: statistic 2 + finalize 1, allocation 2, outliers 13 (rank, mark, K-means, select init,
+# 3 x (histogram, digit), row count, row scan, emit), final fit 2 (row index, K-means), packing 2 = 22.
+# Default: the provisional fit is 2 kernels (table, iterate; its errors are never written), the three digit
+# steps run inside the histogram kernels, the final fit is row index + 3 (table, iterate, assign) = 22 as well.
 def kernels_per_run(assignment=None):
-    if assignment is None:
-        assignment = B.cmpq_get_lloyd_assignment()
-    return 20 + (2 if assignment == B.ASSIGN_ALL_PAIRS else 5)
+    return 22
 
 
-KERNELS_PER_RUN = 25  # with the default assignment
+KERNELS_PER_RUN = 22
 
 
 @dataclass
