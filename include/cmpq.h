@@ -72,7 +72,8 @@ typedef enum {
     CMPQ_OP_ALLOCATE_BITS = 1,
     CMPQ_OP_EXTRACT_OUTLIERS = 2,
     CMPQ_OP_QUANTIZE_LAYER = 3,
-    CMPQ_OP_PACK = 4
+    CMPQ_OP_PACK = 4,
+    CMPQ_OP_PROTECT_AND_QUANTIZE = 5
 } cmpq_op;
 
 #define CMPQ_LUT_STRIDE 16      /* floats per channel in a look-up table */
@@ -159,6 +160,20 @@ cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int6
                                 const float* sens, float* lut, uint8_t* codes,
                                 int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
                                 size_t ws_bytes, void* stream);
+
+/* ---- outlier protection and quantization in one call (Section 3.2.2 with its final step) -------
+ * Exactly cmpq_extract_outliers followed by cmpq_quantize_layer on the list it produced: the same
+ * arguments, the same outputs bit for bit (rows/cols/vals, lut, codes, inexact_rows, sweeps of the
+ * final fit).  Knowing both steps lets the library derive the value tables of the final fit from
+ * those of the provisional fit (the two weight matrices differ only at the kept entries) instead
+ * of reading and counting every weight a second time.
+ * ws: cmpq_workspace_bytes(CMPQ_OP_PROTECT_AND_QUANTIZE, d_in, d_out). */
+cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                      int64_t ldw, const float* a, const uint8_t* bits, int64_t n_act,
+                                      int64_t n_q, int lloyd_iters, int32_t* rows, int32_t* cols,
+                                      uint16_t* vals, int64_t nnz_out, float* lut, uint8_t* codes,
+                                      int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
+                                      size_t ws_bytes, void* stream);
 
 /* Process-wide choice of the assignment method used by cmpq_extract_outliers and
  * cmpq_quantize_layer from the next call on (host state, no GPU work; thread-safe).

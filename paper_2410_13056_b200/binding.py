@@ -14,7 +14,7 @@ import torch
 F16, BF16 = 0, 1
 ALLOC_RANK, ALLOC_QUANTILE = 0, 1
 ASSIGN_ORDERED, ASSIGN_ALL_PAIRS = 0, 1
-OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK = range(5)
+OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK, OP_PROTECT_AND_QUANTIZE = range(6)
 LUT_STRIDE = 16
 
 EXPORTS = (
@@ -22,6 +22,7 @@ EXPORTS = (
     "cmpq_quantize_layer", "cmpq_pack", "cmpq_workspace_bytes", "cmpq_alloc_counts",
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
     "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment", "cmpq_lloyd_phase_events",
+    "cmpq_protect_and_quantize",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -54,6 +55,9 @@ def lib():
         L.cmpq_quantize_layer.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp,
                                           vp, vp, sz, vp]
         L.cmpq_pack.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.cmpq_protect_and_quantize.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
+                                                vp, vp, vp, vp, sz, vp]
+        L.cmpq_protect_and_quantize.restype = ci
         for name in ("cmpq_collect_stats", "cmpq_collect_stats_static", "cmpq_finalize_stats", "cmpq_allocate_bits",
                      "cmpq_extract_outliers", "cmpq_quantize_layer", "cmpq_pack"):
             getattr(L, name).restype = ci
@@ -186,6 +190,16 @@ def cmpq_quantize_layer(W, bits, rows, cols, lloyd_iters, lut, codes, ws, sens=N
                                      _ptr(rows) if nnz else None, _ptr(cols) if nnz else None, nnz,
                                      lloyd_iters, _ptr(sens), _ptr(lut), _ptr(codes), _ptr(inexact_rows),
                                      _ptr(sweeps), _ptr(ws), ws.numel(), _stream()), "cmpq_quantize_layer")
+
+
+def cmpq_protect_and_quantize(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, ws,
+                              inexact_rows=None, sweeps=None):
+    d_in, d_out = W.shape
+    nnz = n_act * d_out + n_q
+    _check(lib().cmpq_protect_and_quantize(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
+                                           n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz,
+                                           _ptr(lut), _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(ws),
+                                           ws.numel(), _stream()), "cmpq_protect_and_quantize")
 
 
 def cmpq_pack(codes, bits, packed, row_off, perm, seg_rows, ws):

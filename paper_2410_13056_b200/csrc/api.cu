@@ -17,6 +17,9 @@ extern "C" size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out) 
         case CMPQ_OP_PACK:
             if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
             return pack_ws_bytes(d_in, d_out);
+        case CMPQ_OP_PROTECT_AND_QUANTIZE:
+            if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+            return protect_quantize_ws_bytes(d_in, d_out);
     }
     return 0;
 }

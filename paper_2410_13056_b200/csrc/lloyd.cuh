@@ -33,6 +33,11 @@ cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
 // Ordered formulation: value table per channel, warp-per-channel iterations, streaming last
 // assignment.  `tables` is device scratch of lloyd_tables_bytes(d_in, d_out) bytes, 256-byte aligned.
 size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out);
+// Final fit whose value tables are derived from those a provisional ordered fit of the same weights left
+// in prov_tables (args.row_ptr / args.cols: the positions removed since; skip_rebuild: d_in bytes of scratch).
+cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, void* prov_tables, void* tables,
+                                         size_t tables_bytes, uint8_t* skip_rebuild, cudaStream_t st);
+
 // Selection of the worst-fitted entries on the tables of a provisional ordered fit made with neither codes
 // nor errors requested (state: the radix select's SelectState; see outliers.cu for the procedure).
 cmpq_status launch_table_select_hist(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,

@@ -1087,23 +1087,30 @@ static void take_phase_events(cudaEvent_t (&ev)[4]) {
 }
 
 template <int DT>
-static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, cudaStream_t st) {
-    if (args.err && args.codes) return CMPQ_ERR_INTERNAL;  // the assign kernel writes one or the other
-    cudaEvent_t ev[4];
-    take_phase_events(ev);
-    if (ev[0]) cudaEventRecord(ev[0], st);
+static cmpq_status launch_table_dt(const LloydArgs& args, const Tables& t, cudaStream_t st) {
     const int64_t N = args.d_out;
     auto threads_for = [N](int e) {
         int64_t th = (N + e - 1) / e;
         th = (th + 31) / 32 * 32;
         return (int)(th < 32 ? 32 : th);
     };
-    cmpq_status s;
-    if (N <= 2048) s = launch_table<DT, 4, 512, 2>(args, t, threads_for(4), st);
-    else if (N <= 4096) s = launch_table<DT, 16, 256, 4>(args, t, threads_for(16), st);
-    else if (N <= 8192) s = launch_table<DT, 16, 512, 2>(args, t, threads_for(16), st);
-    else if (N <= 16384) s = launch_table<DT, 16, 1024, 1>(args, t, threads_for(16), st);
-    else s = launch_table<DT, 32, 1024, 1>(args, t, threads_for(32), st);
+    if (N <= 2048) return launch_table<DT, 4, 512, 2>(args, t, threads_for(4), st);
+    if (N <= 4096) return launch_table<DT, 16, 256, 4>(args, t, threads_for(16), st);
+    if (N <= 8192) return launch_table<DT, 16, 512, 2>(args, t, threads_for(16), st);
+    if (N <= 16384) return launch_table<DT, 16, 1024, 1>(args, t, threads_for(16), st);
+    return launch_table<DT, 32, 1024, 1>(args, t, threads_for(32), st);
+}
+
+// tables_ready: the value tables of every row to be fitted are in place already (skip the table kernel)
+template <int DT>
+static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, bool tables_ready, cudaStream_t st) {
+    if (args.err && args.codes) return CMPQ_ERR_INTERNAL;  // the assign kernel writes one or the other
+    cudaEvent_t ev[4];
+    take_phase_events(ev);
+    if (ev[0]) cudaEventRecord(ev[0], st);
+    const int64_t N = args.d_out;
+    cmpq_status s = CMPQ_OK;
+    if (!tables_ready) s = launch_table_dt<DT>(args, t, st);
     if (s != CMPQ_OK) return s;
     if (ev[1]) cudaEventRecord(ev[1], st);
 
@@ -1142,7 +1149,150 @@ cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tab
     if (!tables || tables_bytes < lloyd_tables_bytes(args.d_in, args.d_out)) return CMPQ_ERR_WORKSPACE;
     Workspace w(tables, tables_bytes);
     const Tables t = carve_tables(w, args.d_in, args.d_out);
-    return dt == CMPQ_F16 ? launch_ordered_dt<CMPQ_F16>(args, t, st) : launch_ordered_dt<CMPQ_BF16>(args, t, st);
+    return dt == CMPQ_F16 ? launch_ordered_dt<CMPQ_F16>(args, t, false, st) : launch_ordered_dt<CMPQ_BF16>(args, t, false, st);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Final fit from the tables of the provisional fit.  W'' differs from W' only at the positions of
+// O_q (and the O_act rows are all zero in both), so the table of a row of W'' is the table of the
+// same row of W' with the counts of the removed values moved to the value +0.  One warp per row
+// does that for rows with at most kPatchCap removed positions; a row whose every position is
+// removed gets the one-entry table of an all-zero channel; the few other rows are flagged and
+// rebuilt from the weights by the table kernel.
+
+constexpr int kPatchCap = 64;
+constexpr int kPatchWarps = 8;
+
+template <int DT>
+__global__ void __launch_bounds__(kPatchWarps * 32)
+lloyd_patch_tables_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables src, const Tables dst,
+                          const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ cols, int64_t d_in,
+                          int64_t d_out, int32_t* inexact_rows, uint8_t* __restrict__ skip_rebuild) {
+    __shared__ uint32_t removed_keys[kPatchWarps][kPatchCap];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * kPatchWarps + warp;
+    if (row >= d_in) return;
+    const int N = (int)d_out;
+    const int64_t p0 = row_ptr[row];
+    const int64_t nrem64 = row_ptr[row + 1] - p0;
+    uint16_t* dkeys = dst.keys + row * dst.stride;
+    uint16_t* dcum = dst.cum + row * dst.stride;
+    const uint32_t kZeroKey = 0x8000u;  // sort key of +0
+    if (nrem64 >= N) {  // an all-zero channel
+        if (lane == 0) {
+            dkeys[0] = (uint16_t)kZeroKey; dcum[0] = 0;
+            dkeys[1] = 0xffffu; dcum[1] = (uint16_t)N;
+            ChannelHeader h; h.M = 1; dst.hdr[row] = h;
+            skip_rebuild[row] = 1;
+        }
+        return;
+    }
+    if (nrem64 > kPatchCap) {
+        if (lane == 0) skip_rebuild[row] = 0;
+        return;
+    }
+    if (lane == 0) skip_rebuild[row] = 1;
+    const int nrem = (int)nrem64;
+    uint32_t* rk = removed_keys[warp];
+    for (int i = lane; i < nrem; i += 32) {
+        uint32_t h = W[row * ldw + cols[p0 + i]];
+        if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
+        rk[i] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+    }
+    __syncwarp();
+    const int M = src.hdr[row].M;
+    const uint16_t* skeys = src.keys + row * src.stride;
+    const uint16_t* scum = src.cum + row * src.stride;
+    // where +0 sits in the old table, or would sit
+    int lo = 0, hi = M;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if ((uint32_t)skeys[mid] >= kZeroKey) hi = mid; else lo = mid + 1;
+    }
+    const int pos0 = lo;
+    const bool present = pos0 < M && (uint32_t)skeys[pos0] == kZeroKey;
+    const int ins = (nrem > 0 && !present) ? 1 : 0;  // +0 becomes a new entry
+    const int Mm = M + ins;
+    int out = 0, run = 0;
+    uint32_t amax = 0u;
+    int q = 100000;
+    for (int base = 0; base < Mm; base += 32) {
+        const int i = base + lane;
+        uint32_t key = 0u;
+        int cnt = 0;
+        if (i < Mm) {
+            if (ins && i == pos0) {
+                key = kZeroKey;
+            } else {
+                const int j = (ins && i > pos0) ? i - 1 : i;
+                key = skeys[j];
+                cnt = (int)scum[j + 1] - (int)scum[j];
+            }
+            for (int r = 0; r < nrem; ++r) cnt -= rk[r] == key ? 1 : 0;
+            if (key == kZeroKey) cnt += nrem;
+        }
+        const bool keep = cnt > 0;
+        const uint32_t votes = __ballot_sync(0xffffffffu, keep);
+        int incl = keep ? cnt : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (keep) {
+            const int o = out + __popc(votes & ((1u << lane) - 1u));
+            dkeys[o] = (uint16_t)key;
+            dcum[o] = (uint16_t)(run + incl - cnt);
+            const uint32_t ub = __float_as_uint(value_of_key16<DT>(key)) & 0x7fffffffu;
+            if (ub) {
+                amax = max(amax, ub);
+                const int ex = (int)(ub >> 23);
+                const uint32_t m = ub & 0x7fffffu;
+                q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
+            }
+        }
+        out += __popc(votes);
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) {
+        dkeys[out] = 0xffffu;
+        dcum[out] = (uint16_t)run;
+        ChannelHeader h; h.M = out; dst.hdr[row] = h;
+    }
+    if (inexact_rows) {  // the exactness test of the table kernel, on the new table
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            q = min(q, __shfl_xor_sync(0xffffffffu, q, o));
+        }
+        if (lane == 0 && amax != 0u) {
+            const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
+            const int ex_max = (int)(amax >> 23);
+            const int top = ex_max ? ex_max - 127 : (31 - __clz(amax)) - 149;
+            if (log2n + 1 + (top + 1 - q) > 53) atomicAdd(inexact_rows, 1);
+        }
+    }
+}
+
+// args: the final fit (row_ptr / cols = the removed positions, skip_row unused).  prov_tables: the
+// tables the provisional fit left; tables: scratch of the final fit; skip_rebuild: d_in bytes.
+cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, void* prov_tables, void* tables,
+                                         size_t tables_bytes, uint8_t* skip_rebuild, cudaStream_t st) {
+    if (!prov_tables || !tables || tables_bytes < lloyd_tables_bytes(args.d_in, args.d_out)) return CMPQ_ERR_WORKSPACE;
+    const Tables src = tables_at(prov_tables, tables_bytes, args.d_in, args.d_out);
+    const Tables dst = tables_at(tables, tables_bytes, args.d_in, args.d_out);
+    const unsigned blocks = (unsigned)((args.d_in + kPatchWarps - 1) / kPatchWarps);
+    if (dt == CMPQ_F16)
+        lloyd_patch_tables_kernel<CMPQ_F16><<<blocks, kPatchWarps * 32, 0, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild);
+    else
+        lloyd_patch_tables_kernel<CMPQ_BF16><<<blocks, kPatchWarps * 32, 0, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild);
+    cmpq_status s = launch_status();
+    if (s != CMPQ_OK) return s;
+    LloydArgs rebuild = args;  // rows with too many removed positions for the patch: from the weights
+    rebuild.skip_row = skip_rebuild;
+    s = dt == CMPQ_F16 ? launch_table_dt<CMPQ_F16>(rebuild, dst, st) : launch_table_dt<CMPQ_BF16>(rebuild, dst, st);
+    if (s != CMPQ_OK) return s;
+    return dt == CMPQ_F16 ? launch_ordered_dt<CMPQ_F16>(args, dst, true, st) : launch_ordered_dt<CMPQ_BF16>(args, dst, true, st);
 }
 
 }  // namespace cmpq

@@ -260,6 +260,14 @@ size_t outliers_ws_bytes(int64_t d_in, int64_t d_out) {
     return w.used;
 }
 
+cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw, const float* a,
+                         const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
+                         int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st);
+static cmpq_status check_extract_args(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                      const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                      int lloyd_iters, const int32_t* rows, const int32_t* cols,
+                                      const uint16_t* vals, int64_t nnz_out);
+
 }  // namespace cmpq
 
 using namespace cmpq;
@@ -274,20 +282,20 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
                                              int64_t n_act, int64_t n_q, int lloyd_iters,
                                              int32_t* rows, int32_t* cols, uint16_t* vals,
                                              int64_t nnz_out, void* ws, size_t ws_bytes, void* stream) {
-    if (!W || !a || !bits) return CMPQ_ERR_INVALID_ARG;
-    if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
-    if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT || ldw < d_out)
-        return CMPQ_ERR_INVALID_ARG;
-    if (n_act < 0 || n_act > d_in || n_q < 0 || n_q > (d_in - n_act) * d_out) return CMPQ_ERR_INVALID_ARG;
-    if (nnz_out != n_act * d_out + n_q) return CMPQ_ERR_INVALID_ARG;
-    if (nnz_out > 0 && (!rows || !cols || !vals)) return CMPQ_ERR_INVALID_ARG;
-    if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
-    if (!aligned_to(W, 2)) return CMPQ_ERR_INVALID_ARG;
-    if (d_in * d_out > 0x7fffffffLL) return CMPQ_ERR_UNSUPPORTED;  // 32-bit counters in the select
+    const cmpq_status chk = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
+    if (chk != CMPQ_OK) return chk;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < outliers_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     Workspace wsp(ws, ws_bytes);
     OutlierWs o = carve(wsp, d_in, d_out);
+    return extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, o,
+                        static_cast<cudaStream_t>(stream));
+}
+
+namespace cmpq {
+
+cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw, const float* a,
+                         const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
+                         int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st) {
     const unsigned row_blocks = (unsigned)((d_in + 255) / 256);
 
     const bool all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
@@ -349,3 +357,83 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
     }
     return launch_status();
 }
+
+static cmpq_status check_extract_args(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                      const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                      int lloyd_iters, const int32_t* rows, const int32_t* cols,
+                                      const uint16_t* vals, int64_t nnz_out) {
+    if (!W || !a || !bits) return CMPQ_ERR_INVALID_ARG;
+    if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
+    if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT || ldw < d_out)
+        return CMPQ_ERR_INVALID_ARG;
+    if (n_act < 0 || n_act > d_in || n_q < 0 || n_q > (d_in - n_act) * d_out) return CMPQ_ERR_INVALID_ARG;
+    if (nnz_out != n_act * d_out + n_q) return CMPQ_ERR_INVALID_ARG;
+    if (nnz_out > 0 && (!rows || !cols || !vals)) return CMPQ_ERR_INVALID_ARG;
+    if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(W, 2)) return CMPQ_ERR_INVALID_ARG;
+    if (d_in * d_out > 0x7fffffffLL) return CMPQ_ERR_UNSUPPORTED;  // 32-bit counters in the select
+    return CMPQ_OK;
+}
+
+// work space of the fused call: the outlier step's, then the final fit's row index, tables and a
+// byte per row
+struct FusedWs {
+    OutlierWs o;
+    int64_t* row_ptr;
+    char* tables;
+    uint8_t* skip_rebuild;
+};
+
+static FusedWs carve_fused(Workspace& w, int64_t d_in, int64_t d_out) {
+    FusedWs f;
+    f.o = carve(w, d_in, d_out);
+    f.row_ptr = w.take<int64_t>(d_in + 1);
+    f.tables = w.take<char>(lloyd_tables_bytes(d_in, d_out));
+    f.skip_rebuild = w.take<uint8_t>(d_in);
+    return f;
+}
+
+size_t protect_quantize_ws_bytes(int64_t d_in, int64_t d_out) {
+    Workspace w(nullptr, 0);
+    carve_fused(w, d_in, d_out);
+    return w.used;
+}
+
+}  // namespace cmpq
+
+extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                                 int64_t ldw, const float* a, const uint8_t* bits,
+                                                 int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
+                                                 int32_t* cols, uint16_t* vals, int64_t nnz_out, float* lut,
+                                                 uint8_t* codes, int32_t* inexact_rows,
+                                                 unsigned long long* sweeps, void* ws, size_t ws_bytes,
+                                                 void* stream) {
+    cmpq_status s = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
+    if (s != CMPQ_OK) return s;
+    if (!lut || !codes || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
+    if (!ws || !aligned_to(ws, 256) || ws_bytes < protect_quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Workspace wsp(ws, ws_bytes);
+    const FusedWs f = carve_fused(wsp, d_in, d_out);
+    s = extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, f.o, st);
+    if (s != CMPQ_OK) return s;
+    s = launch_row_ptr(rows, nnz_out, d_in, f.row_ptr, st);
+    if (s != CMPQ_OK) return s;
+    LloydArgs la{};
+    la.W = static_cast<const uint16_t*>(W);
+    la.d_in = d_in; la.d_out = d_out; la.ldw = ldw;
+    la.bits = bits;
+    la.iters = lloyd_iters;
+    la.row_ptr = f.row_ptr;
+    la.cols = cols;
+    la.lut = lut;
+    la.codes = codes;
+    la.inexact_rows = inexact_rows;
+    la.sweeps = sweeps;
+    const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
+    if (lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS) return launch_lloyd(la, dt, st);
+    // the provisional fit ran (and left its tables) only when entries had to be selected
+    if (n_q > 0) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, f.skip_rebuild, st);
+    return launch_lloyd_ordered(la, dt, f.tables, tables_bytes, st);
+}
+

@@ -17,8 +17,12 @@ from . import binding as B
 # 3 x (histogram, digit), row count, row scan, emit), final fit 2 (row index, K-means), packing 2 = 22.
 # Default: the provisional fit is 2 kernels (table, iterate; its errors are never written), the three digit
 # steps run inside the histogram kernels, the final fit is row index + 3 (table, iterate, assign) = 22 as well.
-def kernels_per_run(assignment=None):
-    return 22
+# Fused (cmpq_protect_and_quantize, default path): the final fit's table kernel is replaced by the patch
+# kernel plus a table-kernel launch that only rebuilds rows with many removed positions = 23.
+def kernels_per_run(assignment=None, fused=False):
+    if assignment is None:
+        assignment = B.cmpq_get_lloyd_assignment()
+    return 23 if (fused and assignment != B.ASSIGN_ALL_PAIRS) else 22
 
 
 KERNELS_PER_RUN = 22
@@ -51,7 +55,7 @@ class LayerQuantizer:
         self.n_q = dq if n_q is None else int(n_q)
         self.nnz = self.n_act * self.d_out + self.n_q
         dev = self.device
-        ws_bytes = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out) for op in range(5))
+        ws_bytes = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out) for op in range(6))
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
         self.sumsq = torch.empty(self.d_in, dtype=torch.float64, device=dev)
         self.a = torch.empty(self.d_in, dtype=torch.float32, device=dev)
@@ -75,10 +79,16 @@ class LayerQuantizer:
         w = lambda c: (self.d_out * c + 31) // 32
         return n2 * w(2) + n3 * w(3) + n4 * w(4)
 
-    def run(self, X, W, avg_bits, lloyd_iters, events=None):
+    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None):
         """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
-        events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and, under
-        "final_fit_kernels", the four events around the three kernels of the final K-means."""
+        fused (default: True unless events are asked for): outlier protection and final fit through
+        cmpq_protect_and_quantize, which derives the final fit's value tables from the provisional
+        fit's; otherwise cmpq_extract_outliers and cmpq_quantize_layer one after the other (same
+        results).  events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and,
+        when not fused, under "final_fit_kernels" the four events around the three kernels of the
+        final K-means."""
+        if fused is None:
+            fused = events is None
         assert W.shape == (self.d_in, self.d_out) and X.shape[1] == self.d_in
 
         def call(name, fn, *args, **kw):
@@ -99,6 +109,19 @@ class LayerQuantizer:
         call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
         call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
              self.ws)
+        if fused:
+            call("cmpq_protect_and_quantize", B.cmpq_protect_and_quantize, W, self.a, self.bits, self.n_act,
+                 self.n_q, lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.ws,
+                 inexact_rows=inexact, sweeps=sweeps)
+        else:
+            self._protect_then_quantize(call, W, lloyd_iters, events, inexact, sweeps)
+        call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
+             self.seg_rows, self.ws)
+        words = self.packed_words(avg_bits)
+        return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
+                           self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)
+
+    def _protect_then_quantize(self, call, W, lloyd_iters, events, inexact, sweeps):
         call("cmpq_extract_outliers", B.cmpq_extract_outliers, W, self.a, self.bits, self.n_act, self.n_q,
              lloyd_iters, self.rows, self.cols, self.vals, self.ws)
         if events is not None and B.cmpq_get_lloyd_assignment() == B.ASSIGN_ORDERED:
@@ -108,11 +131,6 @@ class LayerQuantizer:
             events["final_fit_kernels"] = phase
         call("cmpq_quantize_layer", B.cmpq_quantize_layer, W, self.bits, self.rows, self.cols, lloyd_iters,
              self.lut, self.codes, self.ws, inexact_rows=inexact, sweeps=sweeps)
-        call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
-             self.seg_rows, self.ws)
-        words = self.packed_words(avg_bits)
-        return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
-                           self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)
 
     def run_graphed(self, X, W, avg_bits, lloyd_iters):
         """The same pass replayed from a CUDA graph: the 26 launches of a pass are short enough for launch

@@ -53,10 +53,12 @@ def test_default_counts_and_packed_words_match_the_checker(L):
 def test_workspace_sizes(L):
     assert B.cmpq_workspace_bytes(B.OP_EXTRACT_OUTLIERS, 4096, 4096) >= 4 * 4096 * 4096
     assert B.cmpq_workspace_bytes(B.OP_COLLECT_STATS, 4096) <= 8 << 20
-    for op in range(5):
+    for op in range(6):
         assert B.cmpq_workspace_bytes(op, 512, 512) % 256 == 0
         assert B.cmpq_workspace_bytes(op, 0, 512) == 0          # d_in out of range
     assert B.cmpq_workspace_bytes(B.OP_PACK, 512, 1 << 20) == 0   # d_out out of range
+    assert (B.cmpq_workspace_bytes(B.OP_PROTECT_AND_QUANTIZE, 512, 512)
+            > B.cmpq_workspace_bytes(B.OP_EXTRACT_OUTLIERS, 512, 512))
 
 
 def test_bad_arguments_are_refused_on_the_host(L):
@@ -90,6 +92,12 @@ def test_bad_arguments_are_refused_on_the_host(L):
     assert L.cmpq_quantize_layer(*q(nnz=3)) == INVALID                                     # list missing
     assert L.cmpq_quantize_layer(*q(d_out=0)) == INVALID
     assert L.cmpq_quantize_layer(*q(iters=2000)) == INVALID
+    # outlier protection and final fit in one call: the checks of both
+    f = lambda n_act=1, n_q=3, nnz=19, lut=p, codes=p, wsb=1 << 30: (p, 0, 8, 16, 16, p, p, n_act, n_q, 5, p, p, p, nnz, lut, codes, None, None, ws, wsb, None)
+    assert L.cmpq_protect_and_quantize(*f(nnz=18)) == INVALID
+    assert L.cmpq_protect_and_quantize(*f(lut=None)) == INVALID
+    assert L.cmpq_protect_and_quantize(*f(codes=None)) == INVALID
+    assert L.cmpq_protect_and_quantize(*f(wsb=64)) == WORKSPACE
     # pack
     assert L.cmpq_pack(p, p, 8, 16, None, p, p, p, ws, 1 << 30, None) == INVALID
     assert L.cmpq_pack(p, p, 8, 16, p, p, p, p, ws, 8, None) == WORKSPACE

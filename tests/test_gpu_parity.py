@@ -267,3 +267,36 @@ def test_extract_outliers_wide_value_tables(assignment):
     ref = oracle.extract_outliers(inputs.as_u16(W), inputs.F16, a, bits, 1, 300, 6)
     for g, r in zip(got, ref):
         assert np.array_equal(g, r)
+
+
+# ----------------------------------------------------------------------------- fused protection + final fit
+@pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
+@pytest.mark.parametrize("d_in,d_out,n_act,n_q,T", [(64, 512, 2, 40, 8), (33, 4096, 1, 500, 10), (20, 64, 0, 0, 3),
+                                                    (6, 1024, 1, 900, 5), (10, 50, 2, 8 * 50, 4), (40, 300, 3, 0, 5),
+                                                    (5, 1, 1, 2, 3)])
+def test_protect_and_quantize_equals_the_two_calls(dtype, d_in, d_out, n_act, n_q, T, assignment):
+    W, Wu, a, bits = _case(d_in, d_out, dtype, 55 + d_in, 2.8)
+    bits[::3] = 4
+    rows, cols, vals = G.gpu_extract(W, a, bits, n_act, n_q, T)
+    lut, codes, inexact, sweeps = G.gpu_quantize(W, bits, rows, cols, T)
+    nnz = n_act * d_out + n_q
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    r2 = torch.full((max(nnz, 1),), -1, dtype=torch.int32, device="cuda")
+    c2 = torch.full((max(nnz, 1),), -1, dtype=torch.int32, device="cuda")
+    v2 = torch.zeros(max(nnz, 1), dtype=torch.int16, device="cuda")
+    lut2 = torch.full((d_in, 16), -7.0, dtype=torch.float32, device="cuda")
+    codes2 = torch.full((d_in, d_out), 255, dtype=torch.uint8, device="cuda")
+    counters = torch.zeros(2, dtype=torch.int64, device="cuda")
+    B.cmpq_protect_and_quantize(W, dev(a), dev(bits), n_act, n_q, T, r2[:nnz], c2[:nnz], v2[:nnz], lut2, codes2,
+                                B.workspace(B.OP_PROTECT_AND_QUANTIZE, d_in, d_out),
+                                inexact_rows=counters[0:1].view(torch.int32)[0:1], sweeps=counters[1:2])
+    torch.cuda.synchronize()
+    assert np.array_equal(r2[:nnz].cpu().numpy(), rows) and np.array_equal(c2[:nnz].cpu().numpy(), cols)
+    assert np.array_equal(v2[:nnz].cpu().numpy().view(np.uint16), vals)
+    assert np.array_equal(codes2.cpu().numpy(), codes)
+    assert np.array_equal(lut2.cpu().numpy().view(np.uint32), lut.view(np.uint32))
+    c = counters.cpu().numpy()
+    assert int(c[0] & 0xffffffff) == inexact and int(c[1]) == sweeps
+    # and against the checker
+    rlut, rcodes = oracle.quantize_layer(Wu, dtype, bits, rows, cols, T)
+    assert np.array_equal(codes2.cpu().numpy(), rcodes)
