@@ -324,13 +324,16 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": "c2_attn7b: W 4096x4096 bf16, X 131072x4096 bf16, 20 Lloyd iterations, "
                                    "avg 3.0 bits (the metric's budget); one layer per step per GPU",
-                       "launch": "the pass is captured once in a CUDA graph and replayed (LayerQuantizer.run_graphed)",
+                       "launch": "the pass is captured once in a CUDA graph and replayed (LayerQuantizer.run_graphed); "
+                                 "outlier protection and final fit through cmpq_protect_and_quantize. per_call_ms and "
+                                 "kernel_ms come from eager passes that call cmpq_extract_outliers and "
+                                 "cmpq_quantize_layer separately (same results, the final fit rebuilds its tables)",
                        "l2": "inputs larger than L2 (X is 1 GiB per step)",
                        "n_act": q.n_act, "n_q": q.n_q},
             "at_config_budget": {"avg_bits": cfg.budgets[0], "value": world * params / (ms_22 * 1e-3) / 1e6,
                                  "unit": UNIT, "ms_per_step": ms_22},
             "per_call_ms": per_call, "ms_per_step_with_events": ms_instrumented,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_run(B.ASSIGN_ORDERED) * steps,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_run(B.ASSIGN_ORDERED, fused=True) * steps,
             "roofline": roofline, "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))

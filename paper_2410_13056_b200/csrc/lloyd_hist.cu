@@ -1161,13 +1161,14 @@ cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tab
 // rebuilt from the weights by the table kernel.
 
 constexpr int kPatchCap = 64;
-constexpr int kPatchWarps = 8;
+constexpr int kPatchWarps = 4;
 
 template <int DT>
 __global__ void __launch_bounds__(kPatchWarps * 32)
 lloyd_patch_tables_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables src, const Tables dst,
                           const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ cols, int64_t d_in,
-                          int64_t d_out, int32_t* inexact_rows, uint8_t* __restrict__ skip_rebuild) {
+                          int64_t d_out, int32_t* inexact_rows, uint8_t* __restrict__ skip_rebuild, int cap) {
+    extern __shared__ __align__(16) unsigned char patch_smem[];  // per warp: cap keys, cap + 8 count prefixes
     __shared__ uint32_t removed_keys[kPatchWarps][kPatchCap];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row = (int64_t)blockIdx.x * kPatchWarps + warp;
@@ -1203,6 +1204,17 @@ lloyd_patch_tables_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tab
     const int M = src.hdr[row].M;
     const uint16_t* skeys = src.keys + row * src.stride;
     const uint16_t* scum = src.cum + row * src.stride;
+    if (M <= cap) {  // stage the old table in shared memory: all its loads are in flight at once
+        uint16_t* s_keys = reinterpret_cast<uint16_t*>(patch_smem + (size_t)warp * (4 * (size_t)cap + 16));
+        uint16_t* s_cum = s_keys + cap;
+        for (int i = lane; i < (M + 7) / 8; i += 32)
+            reinterpret_cast<uint4*>(s_keys)[i] = __ldg(reinterpret_cast<const uint4*>(skeys) + i);
+        for (int i = lane; i < (M + 1 + 7) / 8; i += 32)
+            reinterpret_cast<uint4*>(s_cum)[i] = __ldg(reinterpret_cast<const uint4*>(scum) + i);
+        __syncwarp();
+        skeys = s_keys;
+        scum = s_cum;
+    }
     // where +0 sits in the old table, or would sit
     int lo = 0, hi = M;
     while (lo < hi) {
@@ -1282,10 +1294,15 @@ cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, v
     const Tables src = tables_at(prov_tables, tables_bytes, args.d_in, args.d_out);
     const Tables dst = tables_at(tables, tables_bytes, args.d_in, args.d_out);
     const unsigned blocks = (unsigned)((args.d_in + kPatchWarps - 1) / kPatchWarps);
+    const int cap = args.d_out <= 4096 ? 1536 : (args.d_out <= 12288 ? 2048 : 3072);  // as in the iterate kernel
+    const size_t smem = (size_t)kPatchWarps * (4 * (size_t)cap + 16);
+    if (cudaFuncSetAttribute(lloyd_patch_tables_kernel<CMPQ_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(lloyd_patch_tables_kernel<CMPQ_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return CMPQ_ERR_CUDA;
     if (dt == CMPQ_F16)
-        lloyd_patch_tables_kernel<CMPQ_F16><<<blocks, kPatchWarps * 32, 0, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild);
+        lloyd_patch_tables_kernel<CMPQ_F16><<<blocks, kPatchWarps * 32, smem, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild, cap);
     else
-        lloyd_patch_tables_kernel<CMPQ_BF16><<<blocks, kPatchWarps * 32, 0, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild);
+        lloyd_patch_tables_kernel<CMPQ_BF16><<<blocks, kPatchWarps * 32, smem, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild, cap);
     cmpq_status s = launch_status();
     if (s != CMPQ_OK) return s;
     LloydArgs rebuild = args;  // rows with too many removed positions for the patch: from the weights

@@ -55,7 +55,7 @@ def run_layer(a):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "layer"])
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer"])
     ap.add_argument("--config", default="c2_attn7b")
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--budget", type=float, default=3.0)
@@ -111,8 +111,15 @@ def main():
             cols = torch.empty(nnz, dtype=torch.int32, device="cuda")
             vals = torch.empty(nnz, dtype=torch.int16, device="cuda")
             av = torch.rand(d_in, device="cuda")
-            ws = B.workspace(B.OP_EXTRACT_OUTLIERS, d_in, d_out)
-            fn = lambda: B.cmpq_extract_outliers(W, av, bits, n_act, n_q, a.iters, rows, cols, vals, ws)
+            if a.case == "protect":  # outlier protection and final fit in one call
+                lut = torch.empty((d_in, 16), dtype=torch.float32, device="cuda")
+                codes = torch.empty((d_in, d_out), dtype=torch.uint8, device="cuda")
+                ws = B.workspace(B.OP_PROTECT_AND_QUANTIZE, d_in, d_out)
+                fn = lambda: B.cmpq_protect_and_quantize(W, av, bits, n_act, n_q, a.iters, rows, cols, vals, lut,
+                                                         codes, ws)
+            else:
+                ws = B.workspace(B.OP_EXTRACT_OUTLIERS, d_in, d_out)
+                fn = lambda: B.cmpq_extract_outliers(W, av, bits, n_act, n_q, a.iters, rows, cols, vals, ws)
             work = "%d channels x %d weights, K=%d, T=%d, nnz=%d" % (d_in, d_out, 1 << a.bits, a.iters, nnz)
 
     fn()
