@@ -34,7 +34,7 @@ def run_layer(a):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(a.launches):
-        q.run(X, W, a.budget, cfg.lloyd_iters, events=evs[i])
+        q.run(X, W, a.budget, cfg.lloyd_iters, events=evs[i], fused=a.fused)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / a.launches
@@ -66,6 +66,8 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16"])
+    ap.add_argument("--fused", action="store_true",
+                    help="layer case: outlier protection and final fit through cmpq_protect_and_quantize")
     ap.add_argument("--assign", default="ordered", choices=["ordered", "all_pairs"],
                     help="assignment method of the K-means kernels")
     a = ap.parse_args()
