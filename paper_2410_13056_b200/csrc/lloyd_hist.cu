@@ -43,7 +43,8 @@ constexpr int kSlotWords = 128;  // 256 low-byte counters of 16 bits, two per wo
 static_assert(CMPQ_MAX_D_OUT < 65536, "second-level counters and count prefixes are 16 bits wide");
 
 struct ChannelHeader {
-    int M;  // distinct values of the channel
+    int M;        // distinct values of the channel
+    int suspect;  // 1 if the magnitude range alone does not prove the fp64 sums exact
 };
 
 // Per channel: `stride` entries (M used, entry M is a sentinel holding the totals).
@@ -212,7 +213,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     // Exactness of fp64 sums (see load_channel_keys): first from the magnitude range alone, bit by bit
     // only for a channel that fails that.  Every warp reduces the per-warp ranges, so the decision is
     // the same in all threads.
-    if (a.inexact_rows) {
+    bool suspect = false;  // kept in the header: a later fit of a subset of these weights can skip the test
+    {
         amax = lane < nwarps ? (uint32_t)sh.wtop[lane] : 0u;
         amin1 = lane < nwarps ? (uint32_t)sh.wulp[lane] : 0xffffffffu;
 #pragma unroll
@@ -227,7 +229,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
             const int ex_max = (int)(fmax >> 23), ex_min = (int)(fmin >> 23);
             const int top = ex_max ? ex_max - 127 : (31 - __clz(fmax)) - 149;
             const int q_low = (ex_min ? ex_min - 150 : -149) + (DT == CMPQ_BF16 ? 16 : 13);
-            if (log2n + 1 + (top + 1 - q_low) > 53) {
+            suspect = log2n + 1 + (top + 1 - q_low) > 53;
+            if (suspect && a.inexact_rows) {
                 int q = 100000;
 #pragma unroll
                 for (int e = 0; e < E; ++e) {
@@ -314,6 +317,7 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         cum[run_nz] = (uint16_t)run_cnt;
         ChannelHeader h;
         h.M = run_nz;
+        h.suspect = suspect ? 1 : 0;
         t.hdr[row] = h;
     }
 }
@@ -1183,7 +1187,7 @@ lloyd_patch_tables_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tab
         if (lane == 0) {
             dkeys[0] = (uint16_t)kZeroKey; dcum[0] = 0;
             dkeys[1] = 0xffffu; dcum[1] = (uint16_t)N;
-            ChannelHeader h; h.M = 1; dst.hdr[row] = h;
+            ChannelHeader h; h.M = 1; h.suspect = 0; dst.hdr[row] = h;
             skip_rebuild[row] = 1;
         }
         return;
@@ -1225,53 +1229,62 @@ lloyd_patch_tables_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tab
     const bool present = pos0 < M && (uint32_t)skeys[pos0] == kZeroKey;
     const int ins = (nrem > 0 && !present) ? 1 : 0;  // +0 becomes a new entry
     const int Mm = M + ins;
-    int out = 0, run = 0;
+    // The magnitude range of the old table proved its sums exact: so are those of any subset with zeros
+    // added, and the bit-by-bit test is skipped.
+    const bool test = inexact_rows && src.hdr[row].suspect;
+    int deleted = 0;  // entries dropped so far (their count fell to zero)
     uint32_t amax = 0u;
     int q = 100000;
     for (int base = 0; base < Mm; base += 32) {
         const int i = base + lane;
-        uint32_t key = 0u;
-        int cnt = 0;
-        if (i < Mm) {
+        const bool valid = i < Mm;
+        uint32_t key = kZeroKey;
+        int cnt = 0, below = 0;  // weights with this value / with a smaller value in the old table
+        if (valid) {
             if (ins && i == pos0) {
-                key = kZeroKey;
+                below = (int)scum[pos0];
             } else {
                 const int j = (ins && i > pos0) ? i - 1 : i;
                 key = skeys[j];
-                cnt = (int)scum[j + 1] - (int)scum[j];
+                below = (int)scum[j];
+                cnt = (int)scum[j + 1] - below;
             }
-            for (int r = 0; r < nrem; ++r) cnt -= rk[r] == key ? 1 : 0;
-            if (key == kZeroKey) cnt += nrem;
+            int eq = 0, lt = 0;
+            for (int r = 0; r < nrem; ++r) {
+                const uint32_t k = rk[r];
+                eq += k == key ? 1 : 0;
+                lt += k < key ? 1 : 0;
+            }
+            cnt -= eq;
+            below -= lt;
+            if (key == kZeroKey) cnt += nrem;      // the removed weights are zeros now
+            if (key > kZeroKey) below += nrem;
         }
         const bool keep = cnt > 0;
-        const uint32_t votes = __ballot_sync(0xffffffffu, keep);
-        int incl = keep ? cnt : 0;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
+        const uint32_t gone = __ballot_sync(0xffffffffu, valid && !keep);
         if (keep) {
-            const int o = out + __popc(votes & ((1u << lane) - 1u));
+            const int o = i - deleted - __popc(gone & ((1u << lane) - 1u));
             dkeys[o] = (uint16_t)key;
-            dcum[o] = (uint16_t)(run + incl - cnt);
-            const uint32_t ub = __float_as_uint(value_of_key16<DT>(key)) & 0x7fffffffu;
-            if (ub) {
-                amax = max(amax, ub);
-                const int ex = (int)(ub >> 23);
-                const uint32_t m = ub & 0x7fffffu;
-                q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
+            dcum[o] = (uint16_t)below;
+            if (test) {
+                const uint32_t ub = __float_as_uint(value_of_key16<DT>(key)) & 0x7fffffffu;
+                if (ub) {
+                    amax = max(amax, ub);
+                    const int ex = (int)(ub >> 23);
+                    const uint32_t m = ub & 0x7fffffu;
+                    q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
+                }
             }
         }
-        out += __popc(votes);
-        run += __shfl_sync(0xffffffffu, incl, 31);
+        deleted += __popc(gone);
     }
     if (lane == 0) {
+        const int out = Mm - deleted;
         dkeys[out] = 0xffffu;
-        dcum[out] = (uint16_t)run;
-        ChannelHeader h; h.M = out; dst.hdr[row] = h;
+        dcum[out] = (uint16_t)N;
+        ChannelHeader h; h.M = out; h.suspect = src.hdr[row].suspect; dst.hdr[row] = h;
     }
-    if (inexact_rows) {  // the exactness test of the table kernel, on the new table
+    if (test) {  // the exactness test of the table kernel, on the new table
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
