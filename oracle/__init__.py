@@ -220,6 +220,36 @@ def recon_error(X_u16, W_u16, dtype, lut, codes, rows, cols, vals, t_step=1):
                                           _i64(t_step)))
 
 
+def matvec(x_u16, dtype, lut, codes, rows, cols, vals):
+    """Inference product of one token (Section 6): returns (y float64[d_out], yabs float64[d_out])."""
+    x_u16 = _c(x_u16, np.uint16)
+    lut = _c(lut, np.float32)
+    codes = _c(codes, np.uint8)
+    rows = _c(rows, np.int32)
+    cols = _c(cols, np.int32)
+    vals = _c(vals, np.uint16)
+    d_in, d_out = codes.shape
+    y = np.empty(d_out, np.float64)
+    yabs = np.empty(d_out, np.float64)
+    lib().oracle_matvec(_p(x_u16), dtype, _i64(d_in), _i64(d_out), _p(lut), _p(codes), _p(rows),
+                        _p(cols), _p(vals), _i64(rows.shape[0]), _p(y), _p(yabs))
+    return y, yabs
+
+
+def outliers_by_column(rows, cols, vals, d_out):
+    """Outlier list regrouped by column.  Returns (col_ptr int64[d_out+1], rows int32, vals uint16)."""
+    rows = _c(rows, np.int32)
+    cols = _c(cols, np.int32)
+    vals = _c(vals, np.uint16)
+    nnz = rows.shape[0]
+    col_ptr = np.empty(d_out + 1, np.int64)
+    c_rows = np.empty(nnz, np.int32)
+    c_vals = np.empty(nnz, np.uint16)
+    lib().oracle_outliers_by_column(_p(rows), _p(cols), _p(vals), _i64(nnz), _i64(d_out),
+                                    _p(col_ptr), _p(c_rows), _p(c_vals))
+    return col_ptr, c_rows, c_vals
+
+
 def layer_pass(X_u16, W_u16, dtype, avg_bits, n_act, n_q, T):
     """The whole pass for one layer in the paper's order; returns a dict of all outputs."""
     X_u16 = _c(X_u16, np.uint16)

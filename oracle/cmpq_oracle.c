@@ -22,7 +22,9 @@
  * Pins (tests/test_oracle_*.py): closed forms for the statistic, allocation
  * invariants and numpy argsort, exhaustive optimal 1-D clustering on <= 16
  * points, sklearn's Lloyd from the same start, full-sort top-k, pack/unpack
- * round trip, and the storage figures the paper prints.
+ * round trip, the storage figures the paper prints; for the inference product:
+ * unit inputs, exactly representable layers, a dense float64 matrix product and
+ * the reconstruction error of the same layer.
  * Parity unpinned: none of the paper's perplexity tables can pin the
  * reconstruction error (no model weights exist here); oracle_recon_error is
  * pinned only against a dense float64 numpy evaluation of the same definition.
@@ -456,6 +458,61 @@ double oracle_recon_error(const uint16_t* X, const uint16_t* W, int dtype, int64
     free(y);
     free(D);
     return sqrt(total);
+}
+
+/* ---------------------------------------------------------------------------
+ * Step 10.  Inference product of one token with the quantized layer (Section 6,
+ * the figure of the real quantization process): the input is split by the
+ * precision of its channels, each part multiplies its 2-, 3- or 4-bit weight
+ * sub-matrix, the outliers multiply the original 16-bit input, and everything
+ * is accumulated:
+ *     y_j = sum_i x_i * lut_i[code_{ij}]  +  sum_{(i,j,v) in O} x_i * v .
+ * Grouping by precision only reorders the sum over i, so the definition is
+ * written out directly from the byte codes, in fp64, channel by channel.
+ * yabs_j (optional) = sum of the absolute values of the same terms: the scale
+ * a floating-point error bound of any summation order is stated against.
+ * ------------------------------------------------------------------------- */
+void oracle_matvec(const uint16_t* x, int dtype, int64_t d_in, int64_t d_out, const float* lut,
+                   const uint8_t* codes, const int32_t* rows, const int32_t* cols,
+                   const uint16_t* vals, int64_t nnz, double* y, double* yabs) {
+    for (int64_t j = 0; j < d_out; ++j) {
+        y[j] = 0.0;
+        if (yabs) yabs[j] = 0.0;
+    }
+    for (int64_t i = 0; i < d_in; ++i) {
+        double xi = (double)oracle_widen(x[i], dtype);
+        for (int64_t j = 0; j < d_out; ++j) {
+            double t = xi * (double)lut[i * 16 + codes[i * d_out + j]];
+            y[j] += t;
+            if (yabs) yabs[j] += fabs(t);
+        }
+    }
+    for (int64_t p = 0; p < nnz; ++p) {
+        double t = (double)oracle_widen(x[rows[p]], dtype) * (double)oracle_widen(vals[p], dtype);
+        y[cols[p]] += t;
+        if (yabs) yabs[cols[p]] += fabs(t);
+    }
+}
+
+/* The outlier list regrouped by output column (the paper keeps the outliers in a
+ * compressed sparse format for the inference kernel, Section 6): col_ptr[j] ..
+ * col_ptr[j+1] delimits the entries of column j, inside a column ascending by
+ * row.  Plain definition: stable counting by column of a list that is already
+ * sorted by (row, col). */
+void oracle_outliers_by_column(const int32_t* rows, const int32_t* cols, const uint16_t* vals,
+                               int64_t nnz, int64_t d_out, int64_t* col_ptr, int32_t* c_rows,
+                               uint16_t* c_vals) {
+    for (int64_t j = 0; j <= d_out; ++j) col_ptr[j] = 0;
+    for (int64_t p = 0; p < nnz; ++p) ++col_ptr[cols[p] + 1];
+    for (int64_t j = 0; j < d_out; ++j) col_ptr[j + 1] += col_ptr[j];
+    int64_t* next = (int64_t*)malloc((size_t)(d_out + 1) * sizeof(int64_t));
+    memcpy(next, col_ptr, (size_t)(d_out + 1) * sizeof(int64_t));
+    for (int64_t p = 0; p < nnz; ++p) {
+        int64_t q = next[cols[p]]++;
+        c_rows[q] = rows[p];
+        c_vals[q] = vals[p];
+    }
+    free(next);
 }
 
 /* Whole pass for one layer, in the paper's order (used by the timed CPU
