@@ -11,6 +11,7 @@
  *   quantizer   per channel K-means with K = 2^{c_i}, nearest-centroid
  *               codes                                               (Sections 3, 3.2.1)
  *   packing     codes grouped by bit width into bit streams         (Sections 5.1, 6)
+ * and, for the quantized layer, the product of one token with it   (Section 6).
  *
  * Conventions for every entry point
  *  - All array arguments are DEVICE pointers owned by the caller unless the
@@ -73,7 +74,9 @@ typedef enum {
     CMPQ_OP_EXTRACT_OUTLIERS = 2,
     CMPQ_OP_QUANTIZE_LAYER = 3,
     CMPQ_OP_PACK = 4,
-    CMPQ_OP_PROTECT_AND_QUANTIZE = 5
+    CMPQ_OP_PROTECT_AND_QUANTIZE = 5,
+    CMPQ_OP_OUTLIERS_BY_COLUMN = 6, /* d_in is ignored */
+    CMPQ_OP_MATVEC = 7
 } cmpq_op;
 
 #define CMPQ_LUT_STRIDE 16      /* floats per channel in a look-up table */
@@ -200,6 +203,37 @@ cmpq_status cmpq_lloyd_phase_events(void* before_table, void* after_table, void*
 cmpq_status cmpq_pack(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
                       uint32_t* packed, int64_t* row_off, int32_t* perm, int64_t* seg_rows,
                       void* ws, size_t ws_bytes, void* stream);
+
+/* ---- inference product of one token (Section 6: the figure of the real quantization process) ----
+ * The input vector is split by the precision of its channels, every part multiplies its 2-, 3- or
+ * 4-bit weight sub-matrix through the channel's look-up table, the 16-bit outliers multiply the
+ * original input, and all products are accumulated:
+ *     y[j] = sum_i x[i] * lut[i][code_ij]  +  sum over outliers (i, j, v) of x[i] * v .
+ * packed, row_off, perm, seg_rows: exactly what cmpq_pack wrote for a [d_in][d_out] layer (the
+ * codes are read from the packed segments; the byte codes are not needed).  lut: [d_in][16] fp32
+ * as written by cmpq_quantize_layer.  x: d_in values of `dt`.  col_ptr / c_rows / c_vals: the
+ * outliers grouped by column as written by cmpq_outliers_by_column (values of the same `dt`), or
+ * three NULLs for a layer without outliers.  y: d_out fp32.  y16 (optional, may be NULL): the same
+ * result rounded to nearest even into `dt` (the paper accumulates into 16-bit outputs).
+ * Arithmetic: fp32; x[i]*lut[i][k] is formed once per table entry, a column's sum is taken over
+ * blocks of channels in a fixed order, so the result is deterministic and differs from the exact
+ * sum by at most a few hundred units of 2^-24 relative to sum_i |x[i] * w_ij|.
+ * 1 <= d_out <= CMPQ_MAX_D_OUT.  ws: cmpq_workspace_bytes(CMPQ_OP_MATVEC, d_in, d_out). */
+cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
+                        const int64_t* seg_rows, const float* lut, int64_t d_in, int64_t d_out,
+                        const void* x, cmpq_dtype dt, const int64_t* col_ptr, const int32_t* c_rows,
+                        const uint16_t* c_vals, float* y, void* y16, void* ws, size_t ws_bytes,
+                        void* stream);
+
+/* The outlier list of cmpq_extract_outliers (sorted by (row, col)) regrouped by output column for
+ * cmpq_matvec (Section 6 keeps the outliers in a compressed sparse format): col_ptr[j] ..
+ * col_ptr[j+1] (d_out + 1 int64) delimits column j's entries in c_rows / c_vals (nnz entries
+ * each), which are ascending by row inside a column.  (row, col) pairs must be distinct and
+ * 0 <= col < d_out.  nnz may be 0 (then only col_ptr is written and the list pointers may be NULL).
+ * ws: cmpq_workspace_bytes(CMPQ_OP_OUTLIERS_BY_COLUMN, 1, d_out). */
+cmpq_status cmpq_outliers_by_column(const int32_t* rows, const int32_t* cols, const uint16_t* vals,
+                                    int64_t nnz, int64_t d_out, int64_t* col_ptr, int32_t* c_rows,
+                                    uint16_t* c_vals, void* ws, size_t ws_bytes, void* stream);
 
 /* ---- host helpers (pure functions, no GPU work) ----------------------------------------------- */
 size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out);

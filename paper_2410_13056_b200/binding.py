@@ -14,7 +14,8 @@ import torch
 F16, BF16 = 0, 1
 ALLOC_RANK, ALLOC_QUANTILE = 0, 1
 ASSIGN_ORDERED, ASSIGN_ALL_PAIRS = 0, 1
-OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK, OP_PROTECT_AND_QUANTIZE = range(6)
+(OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK, OP_PROTECT_AND_QUANTIZE,
+ OP_OUTLIERS_BY_COLUMN, OP_MATVEC) = range(8)
 LUT_STRIDE = 16
 
 EXPORTS = (
@@ -22,7 +23,7 @@ EXPORTS = (
     "cmpq_quantize_layer", "cmpq_pack", "cmpq_workspace_bytes", "cmpq_alloc_counts",
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
     "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment", "cmpq_lloyd_phase_events",
-    "cmpq_protect_and_quantize",
+    "cmpq_protect_and_quantize", "cmpq_matvec", "cmpq_outliers_by_column",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -58,6 +59,10 @@ def lib():
         L.cmpq_protect_and_quantize.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
                                                 vp, vp, vp, vp, sz, vp]
         L.cmpq_protect_and_quantize.restype = ci
+        L.cmpq_matvec.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, ci, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.cmpq_matvec.restype = ci
+        L.cmpq_outliers_by_column.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, sz, vp]
+        L.cmpq_outliers_by_column.restype = ci
         for name in ("cmpq_collect_stats", "cmpq_collect_stats_static", "cmpq_finalize_stats", "cmpq_allocate_bits",
                      "cmpq_extract_outliers", "cmpq_quantize_layer", "cmpq_pack"):
             getattr(L, name).restype = ci
@@ -206,3 +211,22 @@ def cmpq_pack(codes, bits, packed, row_off, perm, seg_rows, ws):
     d_in, d_out = codes.shape
     _check(lib().cmpq_pack(_ptr(codes), _ptr(bits), d_in, d_out, _ptr(packed), _ptr(row_off), _ptr(perm),
                            _ptr(seg_rows), _ptr(ws), ws.numel(), _stream()), "cmpq_pack")
+
+
+def cmpq_outliers_by_column(rows, cols, vals, d_out, col_ptr, c_rows, c_vals, ws):
+    """Regroups the (row, col)-sorted outlier list by column: col_ptr int64 [d_out+1], c_rows int32 [nnz],
+    c_vals 16-bit patterns [nnz]."""
+    nnz = 0 if rows is None else rows.numel()
+    _check(lib().cmpq_outliers_by_column(_ptr(rows) if nnz else None, _ptr(cols) if nnz else None,
+                                         _ptr(vals) if nnz else None, nnz, d_out, _ptr(col_ptr),
+                                         _ptr(c_rows) if nnz else None, _ptr(c_vals) if nnz else None,
+                                         _ptr(ws), ws.numel(), _stream()), "cmpq_outliers_by_column")
+
+
+def cmpq_matvec(packed, row_off, perm, seg_rows, lut, x, col_ptr, c_rows, c_vals, y, y16, ws):
+    """y (float32 [d_out]) = x (fp16/bf16 [d_in]) times the quantized layer read from its packed segments,
+    plus the outlier products; y16 (optional) receives y rounded to x's dtype."""
+    d_in, d_out = x.numel(), y.numel()
+    _check(lib().cmpq_matvec(_ptr(packed), _ptr(row_off), _ptr(perm), _ptr(seg_rows), _ptr(lut), d_in, d_out,
+                             _ptr(x), dtype_code(x), _ptr(col_ptr), _ptr(c_rows), _ptr(c_vals), _ptr(y),
+                             _ptr(y16), _ptr(ws), ws.numel(), _stream()), "cmpq_matvec")

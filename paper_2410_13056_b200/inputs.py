@@ -82,6 +82,38 @@ def as_u16(t: torch.Tensor):
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view("uint16")
 
 
+def make_quantized_layer(d_in: int, d_out: int, counts: Tuple[int, int, int], dtype_code: int, seed: int,
+                         n_act: int = 0, n_q: int = 0):
+    """A random ALREADY-QUANTIZED layer for the inference product, as host numpy arrays: bit widths with
+    counts[0], counts[1], counts[2] channels of 2, 3, 4 bits at random positions, uniformly random byte
+    codes below 2^bits, ascending N(0, 0.02^2) look-up tables (unused entries 0), an outlier list of
+    n_act whole random rows plus n_q distinct random entries elsewhere (sorted by (row, col), values
+    0.1 * N(0,1) in the dtype), and one input token with the channel scales of make_activations.
+    Nothing here quantizes anything: the arrays only have the shapes and value ranges a quantized
+    layer has."""
+    import numpy as np
+
+    assert sum(counts) == d_in
+    g = np.random.default_rng(int(seed))
+    bits = np.repeat(np.array([2, 3, 4], np.uint8), counts)[g.permutation(d_in)]
+    codes = (g.integers(0, 16, size=(d_in, d_out), dtype=np.uint8) & ((1 << bits) - 1)[:, None]).astype(np.uint8)
+    lut = np.sort(g.normal(0.0, 0.02, size=(d_in, 16)).astype(np.float32), axis=1)
+    lut[np.arange(16)[None, :] >= (1 << bits.astype(np.int64))[:, None]] = 0.0
+    act_rows = np.sort(g.choice(d_in, size=n_act, replace=False)) if n_act else np.zeros(0, np.int64)
+    lin = [np.add.outer(act_rows * d_out, np.arange(d_out)).reshape(-1)]
+    if n_q:
+        free_rows = np.setdiff1d(np.arange(d_in), act_rows)
+        pick = g.choice(free_rows.size * d_out, size=n_q, replace=False)
+        lin.append(free_rows[pick // d_out] * d_out + pick % d_out)
+    lin = np.sort(np.concatenate(lin).astype(np.int64))
+    rows, cols = (lin // d_out).astype(np.int32), (lin % d_out).astype(np.int32)
+    vals = as_u16(torch.from_numpy(0.1 * g.normal(size=lin.size)).to(_TORCH_DTYPE[dtype_code]))
+    sigma = np.exp(g.normal(size=d_in))
+    sigma[g.permutation(d_in)[: int(round(0.01 * d_in))]] *= 50.0
+    x = torch.from_numpy(g.normal(size=d_in) * sigma).to(_TORCH_DTYPE[dtype_code])
+    return dict(bits=bits, codes=codes, lut=lut, rows=rows, cols=cols, vals=vals, x=as_u16(x))
+
+
 @dataclass(frozen=True)
 class Layer:
     d_in: int

@@ -181,3 +181,37 @@ class LayerQuantizer:
             t.copy_(src[k], non_blocking=True)
         torch.cuda.current_stream().synchronize()
         return host_out
+
+
+class QuantizedLinear:
+    """A quantized layer held the way inference reads it (Section 6 of the paper): packed 2/3/4-bit
+    segments, look-up tables and the outliers grouped by column.  matvec(x) enqueues y = x (W_q + O)
+    for one token; it computes nothing itself."""
+
+    def __init__(self, packed, row_off, perm, seg_rows, lut, rows, cols, vals, d_out):
+        self.d_in, self.d_out = int(lut.shape[0]), int(d_out)
+        self.packed, self.row_off, self.perm, self.seg_rows, self.lut = packed, row_off, perm, seg_rows, lut
+        dev = lut.device
+        nnz = 0 if rows is None else rows.numel()
+        self.col_ptr = self.c_rows = self.c_vals = None
+        if nnz:
+            self.col_ptr = torch.empty(self.d_out + 1, dtype=torch.int64, device=dev)
+            self.c_rows = torch.empty(nnz, dtype=torch.int32, device=dev)
+            self.c_vals = torch.empty(nnz, dtype=torch.int16, device=dev)
+            B.cmpq_outliers_by_column(rows, cols, vals, self.d_out, self.col_ptr, self.c_rows, self.c_vals,
+                                      B.workspace(B.OP_OUTLIERS_BY_COLUMN, 1, self.d_out, device=dev))
+        self.ws = B.workspace(B.OP_MATVEC, self.d_in, self.d_out, device=dev)
+        self.y = torch.empty(self.d_out, dtype=torch.float32, device=dev)
+
+    @classmethod
+    def from_result(cls, r: "LayerResult"):
+        return cls(r.packed, r.row_off, r.perm, r.seg_rows, r.lut, r.rows, r.cols, r.vals, r.codes.shape[1])
+
+    def packed_bytes(self):
+        return self.packed.numel() * 4
+
+    def matvec(self, x, y16=None):
+        """x: [d_in] fp16/bf16 on the device.  Returns the fp32 result buffer (overwritten by the next call)."""
+        B.cmpq_matvec(self.packed, self.row_off, self.perm, self.seg_rows, self.lut, x, self.col_ptr, self.c_rows,
+                      self.c_vals, self.y, y16, self.ws)
+        return self.y

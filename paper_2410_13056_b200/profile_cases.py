@@ -4,6 +4,7 @@
     python -m paper_2410_13056_b200.profile_cases stats --tokens 32768 --d-in 4096 --launches 3
     python -m paper_2410_13056_b200.profile_cases pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
     python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
+    python -m paper_2410_13056_b200.profile_cases matvec --d-in 8192 --d-out 28672 --budget 2.5 --launches 20
     python -m paper_2410_13056_b200.profile_cases layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
 
 `layer` runs the whole pass on one layer of a named workload and prints the time per C-ABI call.
@@ -53,9 +54,63 @@ def run_layer(a):
           % (int(q.counters[1].item()), int(q.counters[0].item() & 0xffffffff)))
 
 
+def run_matvec(a, dt):
+    """The inference product on a random quantized layer (codes are random, so no quantization runs):
+    widths split as the rank-form allocation splits them for the budget."""
+    from .pipeline import QuantizedLinear
+
+    d_in, d_out = a.d_in, a.d_out
+    n2, n4 = B.cmpq_alloc_counts(d_in, a.budget)
+    n_act, n_q = B.cmpq_default_counts(d_in, d_out)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(5)
+    bits = torch.full((d_in,), 3, dtype=torch.uint8, device="cuda")
+    order = torch.randperm(d_in, generator=g, device="cuda")
+    bits[order[:n2]] = 2
+    bits[order[d_in - n4:]] = 4
+    codes = torch.randint(0, 16, (d_in, d_out), dtype=torch.uint8, device="cuda", generator=g)
+    codes &= ((1 << bits.int()) - 1).to(torch.uint8)[:, None]
+    lut = torch.sort(torch.randn((d_in, 16), device="cuda", generator=g) * 0.02, dim=1).values.contiguous()
+    words = B.cmpq_packed_words(bits.cpu(), d_out)
+    packed = torch.empty(words, dtype=torch.int32, device="cuda")
+    row_off = torch.empty(d_in + 1, dtype=torch.int64, device="cuda")
+    perm = torch.empty(d_in, dtype=torch.int32, device="cuda")
+    seg = torch.empty(3, dtype=torch.int64, device="cuda")
+    B.cmpq_pack(codes, bits, packed, row_off, perm, seg, B.workspace(B.OP_PACK, d_in, d_out))
+    nnz = n_act * d_out + n_q
+    lin = torch.unique(torch.randint(0, d_in * d_out, (nnz + nnz // 8 + 64,), generator=g, device="cuda"))[:nnz]
+    nnz = lin.numel()
+    rows, cols = (lin // d_out).int(), (lin % d_out).int()
+    vals = (torch.randn(nnz, device="cuda", generator=g) * 0.1).to(inputs.torch_dtype(dt)).view(torch.int16)
+    x = torch.randn(d_in, device="cuda", generator=g).to(inputs.torch_dtype(dt))
+    layer = QuantizedLinear(packed, row_off, perm, seg, lut, rows, cols, vals, d_out)
+    y16 = torch.empty(d_out, dtype=inputs.torch_dtype(dt), device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # larger than L2
+    for _ in range(3):
+        layer.matvec(x, y16)
+    torch.cuda.synchronize()
+    cold = warm = 0.0
+    for _ in range(a.launches):
+        flush.zero_()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        layer.matvec(x, y16)
+        e1.record()
+        layer.matvec(x, y16)
+        e2.record()
+        torch.cuda.synchronize()
+        cold += e0.elapsed_time(e1) / a.launches
+        warm += e1.elapsed_time(e2) / a.launches
+    algo = words * 4 + d_in * 64 + nnz * 6 + d_in * 2 + d_out * 4
+    print("matvec: d_in=%d d_out=%d avg %.2f bits (%d/%d/%d channels of 2/3/4 bits), nnz=%d; %.1f MB packed, "
+          "%.1f MB algorithmic" % (d_in, d_out, a.budget, n2, d_in - n2 - n4, n4, nnz, words * 4 / 1e6, algo / 1e6))
+    print("   L2 flushed before the call: %.4f ms (%.0f GB/s); directly repeated: %.4f ms (%.0f GB/s); %d calls"
+          % (cold, algo / cold / 1e6, warm, algo / warm / 1e6, a.launches))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer"])
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec"])
     ap.add_argument("--config", default="c2_attn7b")
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--budget", type=float, default=3.0)
@@ -76,6 +131,9 @@ def main():
     B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS if a.assign == "all_pairs" else B.ASSIGN_ORDERED)
     if a.case == "layer":
         run_layer(a)
+        return
+    if a.case == "matvec":
+        run_matvec(a, dt)
         return
     d_in, d_out = a.d_in, a.d_out
     bits = torch.full((d_in,), a.bits, dtype=torch.uint8, device="cuda")
