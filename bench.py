@@ -27,8 +27,12 @@ METRIC_BUDGET = 3.0          # the metric is quoted at an average of 3.0 bits
 SM_COUNT, FP32_LANES_PER_SM = 148, 128
 CPU_BASELINE_CHANNELS = 4096   # cpu_baseline leg: the whole layer (about 15 s on one core)
 REFERENCE_ARM_CHANNELS = 1024  # --impl reference: a quarter of the layer per step
-# dram__bytes_read.sum + dram__bytes_write.sum of lloyd_table_kernel per weight, from the ncu capture
-# summarised under profiles/ (None while no capture of the current kernel exists)
+# dram__bytes_read.sum and dram__bytes_write.sum of stats_partial_vec_kernel from the ncu capture summarised
+# under profiles/ (32768 x 4096 bf16 activations: 268.44 MB algorithmic).  Reads grow with the rows, the
+# written fp64 partial sums do not.  None while no capture of the current kernel exists.
+STATS_DRAM_READ_PER_INPUT_BYTE = 268.45e6 / (32768 * 4096 * 2)
+STATS_DRAM_WRITE_BYTES = 3.58e6
+# the same for lloyd_table_kernel, per weight
 LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT = 9761536 / (1184 * 4096)
 
 
@@ -227,10 +231,10 @@ def main():
     }
     ms_22 = timed(cfg.budgets[0], max(3, steps // 2))
 
-    # Roofline of the dominant kernel.  With the default (ordered) assignment a K-means call is three
-    # kernels, timed live by events the library records between them; the value-table kernel takes
-    # the largest share of a step (it runs in both fits).  It has to read every weight once (2 B)
-    # and nothing else of comparable size, so it is held against the HBM peak.
+    # Roofline of the dominant kernel.  By time per step the largest kernel is the statistic's column
+    # reduction (about a quarter of the pass; the K-means work is spread over five smaller kernels).  It has
+    # to read X once (2 bytes per activation) and nothing else of comparable size: HBM bound.  Its duration is
+    # taken from the events around cmpq_collect_stats (the reduction plus its microsecond-sized combine step).
     hbm_peak, sm_max_mhz, peak_kind = _peaks()
     table_gbs = params * 2 / (kernel_ms["lloyd_table_kernel"] * 1e-3) / 1e9
     assign_gbs = params * 3 / (kernel_ms["lloyd_assign_kernel"] * 1e-3) / 1e9
@@ -268,15 +272,22 @@ def main():
         B.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED)
     ap_tflops = 2.0 * ap_evals / (ap_ms * 1e-3) / 1e12
 
-    roofline = {"bound": "hbm", "kernel": "lloyd_table_kernel (final fit)", "achieved": table_gbs,
-                "peak": hbm_peak, "unit": "GB/s", "frac": table_gbs / hbm_peak, "peak_kind": peak_kind,
-                "traffic": LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT * params if LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT else None,
-                "note": "algorithmic bytes: each 16-bit weight read once; the kernel is bound by "
-                        "shared-memory histogram work, not by HBM",
+    stats_bytes = X.numel() * 2
+    roofline = {"bound": "hbm", "kernel": "stats_partial_vec_kernel (cmpq_collect_stats)", "achieved": stats_gbs,
+                "peak": hbm_peak, "unit": "GB/s", "frac": stats_gbs / hbm_peak, "peak_kind": peak_kind,
+                "traffic": (STATS_DRAM_READ_PER_INPUT_BYTE * stats_bytes + STATS_DRAM_WRITE_BYTES
+                            if STATS_DRAM_READ_PER_INPUT_BYTE else None),
+                "note": "algorithmic bytes: every 16-bit activation read once (%d bytes per launch); the largest "
+                        "kernel of the step by time" % stats_bytes,
+                "ms": stats_ms, "share_of_step": stats_ms / ms,
                 "kernel_ms": kernel_ms,
                 "other_kernels": {
-                    "stats": {"bound": "hbm", "achieved": stats_gbs, "peak": hbm_peak, "unit": "GB/s",
-                              "frac": stats_gbs / hbm_peak, "peak_kind": peak_kind},
+                    "lloyd_table": {"bound": "hbm", "kernel": "lloyd_table_kernel (final fit, separate calls)",
+                                    "achieved": table_gbs, "peak": hbm_peak, "unit": "GB/s",
+                                    "frac": table_gbs / hbm_peak, "peak_kind": peak_kind,
+                                    "traffic": LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT * params,
+                                    "note": "each 16-bit weight read once; bound by shared-memory histogram "
+                                            "work, not by HBM"},
                     "pack": {"bound": "hbm", "achieved": pack_gbs, "peak": hbm_peak, "unit": "GB/s",
                              "frac": pack_gbs / hbm_peak, "peak_kind": peak_kind},
                     "lloyd_assign": {"bound": "hbm", "achieved": assign_gbs, "peak": hbm_peak, "unit": "GB/s",
@@ -310,6 +321,33 @@ def main():
            "h2d_bytes_per_step": Xh.numel() * 2 + Wh.numel() * 2,
            "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in host_out.values()),
            "ms_per_step": e2e_ms}
+
+    # the quantized layer in use: the product of one token with it (cmpq_matvec), read from the packed
+    # segments this pass wrote; L2 is flushed before every timed call (the layer itself is only 6 MB)
+    from paper_2410_13056_b200.pipeline import QuantizedLinear
+    res = q.run(X, W, METRIC_BUDGET, cfg.lloyd_iters)
+    qlin = QuantizedLinear.from_result(res)
+    y16 = torch.empty(layer.d_out, dtype=X.dtype, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        qlin.matvec(X[0], y16)
+    mv_ms = []
+    for i in range(30):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        qlin.matvec(X[i], y16)
+        e1.record()
+        torch.cuda.synchronize()
+        mv_ms.append(e0.elapsed_time(e1))
+    mv_ms = statistics.median(mv_ms)
+    mv_bytes = qlin.packed_bytes() + layer.d_in * 64 + q.nnz * 6 + layer.d_in * 2 + layer.d_out * 6
+    matvec = {"call": "cmpq_matvec (2 kernels)", "ms": mv_ms, "bound": "hbm", "achieved": mv_bytes / (mv_ms * 1e-3) / 1e9,
+              "peak": hbm_peak, "unit": "GB/s", "frac": mv_bytes / (mv_ms * 1e-3) / 1e9 / hbm_peak,
+              "peak_kind": peak_kind, "algorithmic_bytes": mv_bytes,
+              "note": "one token; packed codes + tables + outliers read once; at this size two launches and "
+                      "shared-memory table look-ups bound it, not HBM"}
+    roofline["other_kernels"]["matvec"] = matvec
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -16,13 +16,19 @@ constexpr int kMvRowsPerWarp = 8;                     // channels a warp keeps i
 constexpr int kMvRowsPerPass = kMvWarps * kMvRowsPerWarp;
 constexpr int kMvCols = 1024;                         // output columns per block: 32 lanes x 32 columns
 constexpr int kMvPad = kMvCols + 32;                  // one pad float per 32 columns: conflict-free both ways
+#ifndef CMPQ_MV_MIN_BLOCKS
+#define CMPQ_MV_MIN_BLOCKS 2                          // resident blocks per SM the partial kernel is compiled for
+#endif
 
-// Channels per block (a multiple of kMvRowsPerPass), chosen so that large layers still fill the GPU a few
-// times over while their partial sums stay small beside the code stream.
+// Channels per block: a multiple m <= 8 of kMvRowsPerPass, grown with the layer.  Measured on B200 the time
+// hardly depends on m once there are a few blocks per SM (67 to 75 us for m = 2..12 at 8192 x 28672), single
+// passes lose 20 % there (nothing to overlap the first loads with) and small layers want m = 1 or 2 to spread
+// over every SM: aim at two to four resident rounds.
 static int matvec_rows_per_block(int64_t d_in, int64_t d_out) {
     const int64_t tiles = (d_out + kMvCols - 1) / kMvCols;
     const int64_t blocks = tiles * ((d_in + kMvRowsPerPass - 1) / kMvRowsPerPass + 2);
-    int64_t m = blocks / 592;
+    const int sms = sm_count();
+    int64_t m = blocks / (4 * (int64_t)(sms > 0 ? sms : 148));
     if (m < 1) m = 1;
     if (m > 8) m = 8;
     return (int)(m * kMvRowsPerPass);
@@ -32,8 +38,9 @@ static int64_t matvec_max_chunks(int64_t d_in, int rows_per_block) {
     return (d_in + rows_per_block - 1) / rows_per_block + 2;  // three segments: at most two extra ragged chunks
 }
 
+// Sized for the smallest block (the most chunks), so the size does not depend on the device.
 size_t matvec_ws_bytes(int64_t d_in, int64_t d_out) {
-    return round_up((size_t)matvec_max_chunks(d_in, matvec_rows_per_block(d_in, d_out)) * (size_t)d_out * sizeof(float), 256);
+    return round_up((size_t)matvec_max_chunks(d_in, kMvRowsPerPass) * (size_t)d_out * sizeof(float), 256);
 }
 
 size_t by_column_ws_bytes(int64_t d_out) { return round_up((size_t)(d_out + 1) * sizeof(int), 256); }
@@ -69,98 +76,269 @@ __device__ __forceinline__ int64_t matvec_total_chunks(const int64_t* __restrict
     return (seg_rows[0] + rb - 1) / rb + (seg_rows[1] + rb - 1) / rb + (seg_rows[2] + rb - 1) / rb;
 }
 
-// Code t (0..31) of a group of 32 codes held LSB-first in C words, as a byte offset into a float table.
-template <int C, int T>
-__device__ __forceinline__ uint32_t code_offset(const uint32_t (&w)[C]) {
-    constexpr int pos = C * T, word = pos / 32, sh = pos % 32;
+// ---- two channels per look-up ------------------------------------------------------------------------
+// Two channels a, b of the same width C share one table of 2^(2C) sums  T[cb << C | ca] = t_a[ca] + t_b[cb]
+// (t_i[k] = x_i * lut_i[k]), so one shared-memory load and one addition serve two weights.  The index
+// streams are formed 32 columns at a time with word-wide logic: with M = the bits of every even-numbered
+// code,  U = (wa & M) | ((wb & M) << C)  holds the 2C-bit indices of the even columns back to back, and
+// V = ((wa & ~M) >> C) | (wb & ~M)  those of the odd columns (shifts run across the C words of the group).
+
+// Mask word `word` of the even-numbered codes of width C: bit i of the stream is set iff (i mod 2C) < C.
+template <int C>
+__host__ __device__ constexpr uint32_t even_code_mask(int word) {
+    uint32_t m = 0;
+    for (int j = 0; j < 32; ++j)
+        if (((word * 32 + j) % (2 * C)) < C) m |= 1u << j;
+    return m;
+}
+
+template <int C>
+__device__ __forceinline__ void pair_streams(const uint32_t (&wa)[C], const uint32_t (&wb)[C], uint32_t (&U)[C],
+                                             uint32_t (&V)[C]) {
+    uint32_t be[C], ao[C];
+#pragma unroll
+    for (int k = 0; k < C; ++k) {
+        be[k] = wb[k] & even_code_mask<C>(k);
+        ao[k] = wa[k] & ~even_code_mask<C>(k);
+    }
+#pragma unroll
+    for (int k = 0; k < C; ++k) {
+        const uint32_t up = (be[k] << C) | (k > 0 ? be[k > 0 ? k - 1 : 0] >> (32 - C) : 0u);
+        const uint32_t down = (ao[k] >> C) | (k + 1 < C ? ao[k + 1 < C ? k + 1 : k] << (32 - C) : 0u);
+        U[k] = (wa[k] & even_code_mask<C>(k)) | up;
+        V[k] = down | (wb[k] & ~even_code_mask<C>(k));
+    }
+}
+
+// Shared-memory address of table entry number S, an F-bit field at bit F*S of a stream of C words: the
+// field is moved straight to bits [2, 2+F) (a byte offset into floats) and OR-ed into the table's address,
+// which is aligned to the table's size, so one shift and one three-input logic operation produce the address.
+template <int C, int F, int S>
+__device__ __forceinline__ uint32_t entry_address(const uint32_t (&st)[C], uint32_t table_addr) {
+    constexpr int pos = F * S, word = pos / 32, sh = pos % 32;
+    constexpr uint32_t mask = ((1u << F) - 1u) << 2;
     uint32_t v;
-    if (sh + C <= 32) v = w[word] >> sh;
-    else v = __funnelshift_r(w[word], w[(word + 1 < C) ? word + 1 : word], sh);
-    return (v & ((1u << C) - 1u)) << 2;
+    if constexpr (sh + F > 32) v = __funnelshift_r(st[word], st[(word + 1 < C) ? word + 1 : word], sh - 2);
+    else if constexpr (sh >= 2) v = st[word] >> (sh - 2);
+    else v = st[word] << (2 - sh);
+    return (v & mask) | table_addr;
 }
 
-template <int C, int T>
+template <int BYTE_OFFSET>
+__device__ __forceinline__ float load_shared_float(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(BYTE_OFFSET) : "memory");
+    return v;
+}
+
+// acc[2s] += T_P[U_s], acc[2s+1] += T_P[V_s] for the 16 even and 16 odd columns of the group.
+template <int C, int P, int S>
 struct MvAccumulate {
-    static __device__ __forceinline__ void run(const uint32_t (&w)[C], const char* table, float (&acc)[32]) {
-        acc[T] += *reinterpret_cast<const float*>(table + code_offset<C, T>(w));
-        MvAccumulate<C, T + 1>::run(w, table, acc);
+    static __device__ __forceinline__ void run(const uint32_t (&U)[C], const uint32_t (&V)[C], uint32_t table_addr,
+                                               float (&acc)[32]) {
+        constexpr int table_bytes = 4 << (2 * C);
+        acc[2 * S] += load_shared_float<P * table_bytes>(entry_address<C, 2 * C, S>(U, table_addr));
+        acc[2 * S + 1] += load_shared_float<P * table_bytes>(entry_address<C, 2 * C, S>(V, table_addr));
+        MvAccumulate<C, P, S + 1>::run(U, V, table_addr, acc);
     }
 };
-template <int C>
-struct MvAccumulate<C, 32> {
-    static __device__ __forceinline__ void run(const uint32_t (&)[C], const char*, float (&)[32]) {}
+template <int C, int P>
+struct MvAccumulate<C, P, 16> {
+    static __device__ __forceinline__ void run(const uint32_t (&)[C], const uint32_t (&)[C], uint32_t, float (&)[32]) {}
 };
 
-// The C words of one group of 32 codes; words at or beyond `valid` read as 0.
-template <int C>
-__device__ __forceinline__ void load_group(const uint32_t* __restrict__ p, int valid, bool vec, uint32_t (&w)[C]) {
-    if (C == 2 && vec && valid >= 2) {
-        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
-        w[0] = v.x;
-        w[1] = v.y;
-    } else if (C == 4 && vec && valid >= 4) {
-        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
-        w[0] = v.x;
-        w[1] = v.y;
-        w[2] = v.z;
-        w[3] = v.w;
-    } else {
-#pragma unroll
-        for (int t = 0; t < C; ++t) w[t] = (t < valid) ? __ldcs(p + t) : 0u;
+template <int C, int P>
+struct MvPairs {
+    static __device__ __forceinline__ void run(const uint32_t (&w)[kMvRowsPerWarp][C], uint32_t table_addr,
+                                               float (&acc)[32]) {
+        uint32_t U[C], V[C];
+        pair_streams<C>(w[2 * P], w[2 * P + 1], U, V);
+        MvAccumulate<C, P, 0>::run(U, V, table_addr, acc);
+        MvPairs<C, P + 1>::run(w, table_addr, acc);
     }
+};
+template <int C>
+struct MvPairs<C, kMvRowsPerWarp / 2> {
+    static __device__ __forceinline__ void run(const uint32_t (&)[kMvRowsPerWarp][C], uint32_t, float (&)[32]) {}
+};
+
+// One channel per look-up, for 4-bit channels: a pair table would have 256 entries, whose bank conflicts
+// and construction cost more than the second load saves, so each row reads its own 16 values directly.
+template <int C, int Q, int T>
+struct MvAccumulateRow {
+    static __device__ __forceinline__ void run(const uint32_t (&w)[C], uint32_t values_addr, float (&acc)[32]) {
+        acc[T] += load_shared_float<Q * 64>(entry_address<C, C, T>(w, values_addr));
+        MvAccumulateRow<C, Q, T + 1>::run(w, values_addr, acc);
+    }
+};
+template <int C, int Q>
+struct MvAccumulateRow<C, Q, 32> {
+    static __device__ __forceinline__ void run(const uint32_t (&)[C], uint32_t, float (&)[32]) {}
+};
+template <int C, int Q>
+struct MvRows {
+    static __device__ __forceinline__ void run(const uint32_t (&w)[kMvRowsPerWarp][C], uint32_t values_addr,
+                                               float (&acc)[32]) {
+        MvAccumulateRow<C, Q, 0>::run(w[Q], values_addr, acc);
+        MvRows<C, Q + 1>::run(w, values_addr, acc);
+    }
+};
+template <int C>
+struct MvRows<C, kMvRowsPerWarp> {
+    static __device__ __forceinline__ void run(const uint32_t (&)[kMvRowsPerWarp][C], uint32_t, float (&)[32]) {}
+};
+
+template <int C>
+constexpr bool kMvUsePairs = (C < 4);
+
+// ---- staging of the code words: asynchronous copies into a per-lane slot of shared memory -------------
+// Every lane copies the C words of its own group for each row of a pass; word t of row q of lane l lands at
+// stage[(q * C + t) * 32 + l] (conflict free).  Only the copying lane reads its words back, so waiting for
+// the lane's own copy group is all the synchronisation the data needs.  Words at or beyond `valid`, and
+// rows past the end, are zero-filled (a copy of source size 0 reads nothing).
+template <int BYTES>
+__device__ __forceinline__ void async_copy(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"(dst), "l"(src), "n"(BYTES), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// One warp, up to kMvRowsPerWarp stored rows [r, r_end): every lane adds its 32 columns.
-template <int C, int DT>
-__device__ __forceinline__ void matvec_rows(const uint32_t* __restrict__ packed, const int64_t* __restrict__ row_off,
-                                            const int32_t* __restrict__ perm, const float* __restrict__ lut,
-                                            const uint16_t* __restrict__ x, int64_t r, int64_t r_end, int64_t group,
-                                            int valid_words, bool base_vec, float* table /* [rows][16] of this warp */,
-                                            float (&acc)[32]) {
+// Within a segment every channel has the same number of words, so the word offset of stored row r is
+// off0 + (r - r0) * words_per_row with off0 = row_off[r0]: no load stands between a row and its copies.
+template <int C>
+__device__ __forceinline__ void stage_rows(const uint32_t* __restrict__ packed, int64_t off0, int64_t r0,
+                                           int64_t words_per_row, int64_t r, int64_t r_end, int64_t group,
+                                           int valid_words, uint32_t stage_addr /* shared address of this warp's stage */) {
     const int lane = threadIdx.x & 31;
-    // table[q][k] = x_i * lut_i[k] for the rows of this pass: one multiplication per table entry instead
-    // of one per weight
-#pragma unroll
-    for (int q = 0; q < kMvRowsPerWarp / 2; ++q) {
-        const int rr = 2 * q + (lane >> 4);
-        float v = 0.0f;
-        if (r + rr < r_end) {
-            const int32_t i = perm[r + rr];
-            v = widen16<DT>(x[i]) * lut[(int64_t)i * CMPQ_LUT_STRIDE + (lane & 15)];
-        }
-        table[rr * 16 + (lane & 15)] = v;
-    }
-    uint32_t w[kMvRowsPerWarp][C];
 #pragma unroll
     for (int q = 0; q < kMvRowsPerWarp; ++q) {
-        if (r + q < r_end && valid_words > 0) {
-            const int64_t off = row_off[r + q] + group * C;
-            const bool vec = base_vec && (C == 2 ? (off & 1) == 0 : (off & 3) == 0);
-            load_group<C>(packed + off, valid_words, vec, w[q]);
-        } else {
+        const bool row_ok = (r + q < r_end) && valid_words > 0;
+        const uint32_t* src = row_ok ? packed + off0 + (r + q - r0) * words_per_row + group * C : packed;
 #pragma unroll
-            for (int t = 0; t < C; ++t) w[q][t] = 0u;
-        }
+        for (int t = 0; t < C; ++t)
+            async_copy<4>(stage_addr + ((q * C + t) * 32 + lane) * 4, row_ok && t < valid_words ? src + t : packed,
+                          row_ok && t < valid_words ? 4 : 0);
     }
-    __syncwarp();
+}
+
+// The table values x_i * lut_i[k] of a pass are fetched in three steps spread over three passes, so that
+// no step waits for the one before it: channel ids (perm) two passes ahead, the raw x_i and lut_i[k] one
+// pass ahead, the product when the pass starts.  This lane holds rows 2q + (lane >> 4), entry k = lane & 15.
+struct MvIds {
+    int32_t i[kMvRowsPerWarp / 2];  // -1: no such row
+};
+struct MvRaw {
+    uint16_t x[kMvRowsPerWarp / 2];
+    float l[kMvRowsPerWarp / 2];
+};
+
+__device__ __forceinline__ MvIds load_ids(const int32_t* __restrict__ perm, int64_t r, int64_t r_end) {
+    const int lane = threadIdx.x & 31;
+    MvIds ids;
 #pragma unroll
-    for (int q = 0; q < kMvRowsPerWarp; ++q)
-        MvAccumulate<C, 0>::run(w[q], reinterpret_cast<const char*>(table + q * 16), acc);
-    __syncwarp();
+    for (int q = 0; q < kMvRowsPerWarp / 2; ++q) {
+        const int64_t row = r + 2 * q + (lane >> 4);
+        ids.i[q] = row < r_end ? perm[row] : -1;
+    }
+    return ids;
+}
+
+__device__ __forceinline__ MvRaw load_raw(const MvIds& ids, const float* __restrict__ lut,
+                                          const uint16_t* __restrict__ x) {
+    const int lane = threadIdx.x & 31;
+    MvRaw raw;
+#pragma unroll
+    for (int q = 0; q < kMvRowsPerWarp / 2; ++q) {
+        raw.x[q] = ids.i[q] >= 0 ? x[ids.i[q]] : (uint16_t)0;
+        raw.l[q] = ids.i[q] >= 0 ? lut[(int64_t)ids.i[q] * CMPQ_LUT_STRIDE + (lane & 15)] : 0.0f;
+    }
+    return raw;
+}
+
+constexpr int kMvWarpTableBytes = (kMvRowsPerWarp / 2) * (4 << 8);   // four pair tables of 4-bit channels
+constexpr int kMvWarpValueFloats = kMvRowsPerWarp * 16;              // t_i[k] of the rows of a pass
+constexpr int kMvWarpStageBytes = kMvRowsPerWarp * 4 * 32 * 4;       // one pass of 4-bit code words
+constexpr int kMvStages = 2;
+constexpr int kMvTableRegion = kMvWarps * (kMvWarpTableBytes + kMvWarpValueFloats * 4);
+constexpr int kMvSharedBytes = 1024 + kMvTableRegion + kMvWarps * kMvStages * kMvWarpStageBytes;
+static_assert(kMvTableRegion >= kMvWarps * kMvPad * 4, "the reduction staging reuses the table space");
+
+// One warp, all its passes over the chunk's rows: pass p computes while the words of pass p + 1 arrive.
+template <int C, int DT>
+__device__ __forceinline__ void matvec_warp(const uint32_t* __restrict__ packed, int64_t off0, int64_t r0,
+                                            int64_t words_per_row, const int32_t* __restrict__ perm,
+                                            const float* __restrict__ lut, const uint16_t* __restrict__ x,
+                                            int64_t r_first, int64_t r_end, int64_t group, int valid_words,
+                                            float* values, float* tables, uint32_t stage_addr, float (&acc)[32]) {
+    const int lane = threadIdx.x & 31;
+    if (r_first >= r_end) return;
+    stage_rows<C>(packed, off0, r0, words_per_row, r_first, r_end, group, valid_words, stage_addr);
+    async_commit();
+    MvRaw raw_now = load_raw(load_ids(perm, r_first, r_end), lut, x);
+    MvIds ids_next = load_ids(perm, r_first + kMvRowsPerPass, r_end);
+    int buf = 0;
+    for (int64_t r = r_first; r < r_end; r += kMvRowsPerPass) {
+        const int64_t rn = r + kMvRowsPerPass;
+        if (rn < r_end)
+            stage_rows<C>(packed, off0, r0, words_per_row, rn, r_end, group, valid_words,
+                          stage_addr + (buf ^ 1) * kMvWarpStageBytes);
+        async_commit();
+        const MvRaw raw_next = load_raw(ids_next, lut, x);            // used in the next pass
+        ids_next = load_ids(perm, rn + kMvRowsPerPass, r_end);        // used in the next pass
+        // values[q][k] of this pass, then the pair tables: entry e of pair p = values[2p][e mod 2^C] +
+        // values[2p+1][e div 2^C]
+#pragma unroll
+        for (int q = 0; q < kMvRowsPerWarp / 2; ++q)
+            values[(2 * q + (lane >> 4)) * 16 + (lane & 15)] = widen16<DT>(raw_now.x[q]) * raw_now.l[q];
+        __syncwarp();
+        if constexpr (kMvUsePairs<C>) {
+            constexpr int E = 1 << (2 * C);
+#pragma unroll
+            for (int idx0 = 0; idx0 < (kMvRowsPerWarp / 2) * E; idx0 += 32) {
+                const int idx = idx0 + lane, pr = idx / E, e = idx % E;
+                tables[idx] = values[(2 * pr) * 16 + (e & ((1 << C) - 1))] + values[(2 * pr + 1) * 16 + (e >> C)];
+            }
+        }
+        async_wait<1>();  // the words of this pass have arrived (the next pass's group may still be in flight)
+        uint32_t w[kMvRowsPerWarp][C];
+        const uint32_t* st = reinterpret_cast<const uint32_t*>(__cvta_shared_to_generic(stage_addr + buf * kMvWarpStageBytes));
+#pragma unroll
+        for (int q = 0; q < kMvRowsPerWarp; ++q)
+#pragma unroll
+            for (int t = 0; t < C; ++t) w[q][t] = st[(q * C + t) * 32 + lane];
+        __syncwarp();
+        if constexpr (kMvUsePairs<C>) MvPairs<C, 0>::run(w, (uint32_t)__cvta_generic_to_shared(tables), acc);
+        else MvRows<C, 0>::run(w, (uint32_t)__cvta_generic_to_shared(values), acc);
+        __syncwarp();
+        raw_now = raw_next;
+        buf ^= 1;
+    }
+    async_wait<0>();
 }
 
 // partial[slot][j] = sum over the chunk's channels of x_i * lut_i[code_ij].
 template <int DT>
-__global__ void __launch_bounds__(kMvThreads)
+__global__ void __launch_bounds__(kMvThreads, CMPQ_MV_MIN_BLOCKS)
 matvec_partial_kernel(const uint32_t* __restrict__ packed, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ perm, const int64_t* __restrict__ seg_rows,
                       const float* __restrict__ lut, const uint16_t* __restrict__ x, int64_t d_out,
-                      int rows_per_block, int base_align, float* __restrict__ partial) {
-    __shared__ float tables[kMvWarps][kMvRowsPerWarp * 16];
-    __shared__ float red[kMvWarps][kMvPad];
+                      int rows_per_block, float* __restrict__ partial) {
+    extern __shared__ __align__(16) unsigned char raw[];
     const MvChunk ch = matvec_chunk(seg_rows, blockIdx.y, rows_per_block);
     if (ch.c == 0) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // the pair tables must sit on a multiple of their size (1 KB for 4-bit channels): align by hand
+    const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(raw);
+    const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
+    unsigned char* base = raw + (base_addr - raw_addr);
+    float* tables = reinterpret_cast<float*>(base + warp * kMvWarpTableBytes);
+    float* values = reinterpret_cast<float*>(base + kMvWarps * kMvWarpTableBytes) + warp * kMvWarpValueFloats;
+    float* red = reinterpret_cast<float*>(base);  // [kMvWarps][kMvPad], used after the tables
+    const uint32_t stage_addr = base_addr + kMvTableRegion + warp * kMvStages * kMvWarpStageBytes;
     const int64_t group = (int64_t)blockIdx.x * 32 + lane;  // group of 32 columns
     const int64_t words_per_row = (d_out * ch.c + 31) / 32;
     const int64_t left = words_per_row - group * ch.c;
@@ -168,26 +346,28 @@ matvec_partial_kernel(const uint32_t* __restrict__ packed, const int64_t* __rest
     float acc[32];
 #pragma unroll
     for (int t = 0; t < 32; ++t) acc[t] = 0.0f;
-    for (int64_t r = ch.r0 + warp * kMvRowsPerWarp; r < ch.r1; r += kMvRowsPerPass) {
-        if (ch.c == 2)
-            matvec_rows<2, DT>(packed, row_off, perm, lut, x, r, ch.r1, group, valid_words, base_align >= 8,
-                               tables[warp], acc);
-        else if (ch.c == 3)
-            matvec_rows<3, DT>(packed, row_off, perm, lut, x, r, ch.r1, group, valid_words, false, tables[warp], acc);
-        else
-            matvec_rows<4, DT>(packed, row_off, perm, lut, x, r, ch.r1, group, valid_words, base_align >= 16,
-                               tables[warp], acc);
-    }
+    const int64_t r_first = ch.r0 + warp * kMvRowsPerWarp;
+    const int64_t off0 = row_off[ch.r0];
+    if (ch.c == 2)
+        matvec_warp<2, DT>(packed, off0, ch.r0, words_per_row, perm, lut, x, r_first, ch.r1, group, valid_words, values,
+                           tables, stage_addr, acc);
+    else if (ch.c == 3)
+        matvec_warp<3, DT>(packed, off0, ch.r0, words_per_row, perm, lut, x, r_first, ch.r1, group, valid_words, values,
+                           tables, stage_addr, acc);
+    else
+        matvec_warp<4, DT>(packed, off0, ch.r0, words_per_row, perm, lut, x, r_first, ch.r1, group, valid_words, values,
+                           tables, stage_addr, acc);
+    __syncthreads();  // every warp is done with its tables: their space now stages the reduction
     // warps are summed in a fixed order; the staging is laid out so that both sides are conflict free
 #pragma unroll
-    for (int t = 0; t < 32; ++t) red[warp][lane * 33 + t] = acc[t];
+    for (int t = 0; t < 32; ++t) red[warp * kMvPad + lane * 33 + t] = acc[t];
     __syncthreads();
     float* out = partial + (int64_t)blockIdx.y * d_out + (int64_t)blockIdx.x * kMvCols;
     const int64_t cols_here = min((int64_t)kMvCols, d_out - (int64_t)blockIdx.x * kMvCols);
     for (int col = threadIdx.x; col < cols_here; col += kMvThreads) {
         float s = 0.0f;
 #pragma unroll
-        for (int wq = 0; wq < kMvWarps; ++wq) s += red[wq][col + (col >> 5)];
+        for (int wq = 0; wq < kMvWarps; ++wq) s += red[wq * kMvPad + col + (col >> 5)];
         out[col] = s;
     }
 }
@@ -212,14 +392,32 @@ matvec_finish_kernel(const float* __restrict__ partial, const int64_t* __restric
     const int64_t chunks = matvec_total_chunks(seg_rows, rows_per_block);
     float s = 0.0f;
     if (j < d_out) {
-        for (int64_t q = warp; q < chunks; q += kMvWarps) s += partial[q * d_out + j];
-        if (col_ptr != nullptr) {
-            float so = 0.0f;
-            const int64_t e1 = col_ptr[j + 1];
-            for (int64_t e = col_ptr[j] + warp; e < e1; e += kMvWarps)
-                so += widen16<DT>(x[c_rows[e]]) * widen16<DT>(c_vals[e]);
-            s += so;
+        // everything independent is requested before anything is added: the column's outlier range first,
+        // then four partial sums per step (absent ones read as 0; the additions keep their order)
+        const int64_t e0 = col_ptr != nullptr ? col_ptr[j] : 0, e1 = col_ptr != nullptr ? col_ptr[j + 1] : 0;
+        for (int64_t q = warp; q < chunks; q += 4 * kMvWarps) {
+            float pv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) pv[u] = (q + u * kMvWarps < chunks) ? partial[(q + u * kMvWarps) * d_out + j] : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) s += pv[u];
         }
+        float so = 0.0f;
+        for (int64_t e = e0 + warp; e < e1; e += 4 * kMvWarps) {
+            int32_t rw[4];
+            uint16_t vv[4], xv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool ok = e + u * kMvWarps < e1;
+                rw[u] = ok ? c_rows[e + u * kMvWarps] : -1;
+                vv[u] = ok ? c_vals[e + u * kMvWarps] : (uint16_t)0;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) xv[u] = rw[u] >= 0 ? x[rw[u]] : (uint16_t)0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) so += widen16<DT>(xv[u]) * widen16<DT>(vv[u]);
+        }
+        s += so;
     }
     part[warp][lane] = s;
     __syncthreads();
@@ -333,6 +531,21 @@ column_sort_kernel(const int64_t* __restrict__ col_ptr, int32_t* __restrict__ c_
     }
 }
 
+// The partial kernel needs more dynamic shared memory than the default limit: raise it once per device.
+static bool matvec_allow_shared_memory() {
+    static bool done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64 && done[dev]) return true;
+    if (cudaFuncSetAttribute(matvec_partial_kernel<CMPQ_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kMvSharedBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(matvec_partial_kernel<CMPQ_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kMvSharedBytes) != cudaSuccess)
+        return false;
+    if (dev >= 0 && dev < 64) done[dev] = true;
+    return true;
+}
+
 }  // namespace cmpq
 
 using namespace cmpq;
@@ -374,19 +587,19 @@ extern "C" cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_of
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int rb = matvec_rows_per_block(d_in, d_out);
     float* partial = static_cast<float*>(ws);
-    const int base_align = aligned_to(packed, 16) ? 16 : (aligned_to(packed, 8) ? 8 : 4);
+    if (!matvec_allow_shared_memory()) return CMPQ_ERR_CUDA;
     dim3 grid((unsigned)((d_out + kMvCols - 1) / kMvCols), (unsigned)matvec_max_chunks(d_in, rb));
     const unsigned fin_blocks = (unsigned)((d_out + 31) / 32);
     const uint16_t* xu = static_cast<const uint16_t*>(x);
     uint16_t* yu = static_cast<uint16_t*>(y16);
     if (dt == CMPQ_BF16) {
-        matvec_partial_kernel<CMPQ_BF16><<<grid, kMvThreads, 0, st>>>(packed, row_off, perm, seg_rows, lut, xu, d_out,
-                                                                      rb, base_align, partial);
+        matvec_partial_kernel<CMPQ_BF16><<<grid, kMvThreads, kMvSharedBytes, st>>>(packed, row_off, perm, seg_rows, lut,
+                                                                                   xu, d_out, rb, partial);
         matvec_finish_kernel<CMPQ_BF16><<<fin_blocks, kMvThreads, 0, st>>>(partial, seg_rows, rb, d_out, xu, col_ptr,
                                                                            c_rows, c_vals, y, yu);
     } else {
-        matvec_partial_kernel<CMPQ_F16><<<grid, kMvThreads, 0, st>>>(packed, row_off, perm, seg_rows, lut, xu, d_out,
-                                                                     rb, base_align, partial);
+        matvec_partial_kernel<CMPQ_F16><<<grid, kMvThreads, kMvSharedBytes, st>>>(packed, row_off, perm, seg_rows, lut,
+                                                                                  xu, d_out, rb, partial);
         matvec_finish_kernel<CMPQ_F16><<<fin_blocks, kMvThreads, 0, st>>>(partial, seg_rows, rb, d_out, xu, col_ptr,
                                                                           c_rows, c_vals, y, yu);
     }
