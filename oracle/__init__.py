@@ -87,6 +87,26 @@ def finalize_stats(sumsq):
     return a
 
 
+NORM_L2, NORM_L1, NORM_LINF = 0, 1, 2
+
+
+def collect_stats_norm(X_u16, dtype, norm, acc=None):
+    """Accumulates the l2 (sum of squares), l1 (sum of magnitudes) or l_inf (largest magnitude) statistic."""
+    X_u16 = _c(X_u16, np.uint16)
+    n, d_in = X_u16.shape
+    if acc is None:
+        acc = np.zeros(d_in, np.float64)
+    lib().oracle_collect_stats_norm(_p(X_u16), dtype, _i64(n), _i64(d_in), _i64(d_in), int(norm), _p(acc))
+    return acc
+
+
+def finalize_stats_norm(acc, norm):
+    acc = _c(acc, np.float64)
+    a = np.empty(acc.shape[0], np.float32)
+    lib().oracle_finalize_stats_norm(_p(acc), _i64(acc.shape[0]), int(norm), _p(a))
+    return a
+
+
 def alloc_counts(d_in, avg_bits):
     n2, n4 = ctypes.c_int64(), ctypes.c_int64()
     lib().oracle_alloc_counts(_i64(d_in), ctypes.c_double(avg_bits), ctypes.byref(n2),

@@ -89,6 +89,26 @@ void oracle_finalize_stats(const double* sumsq, int64_t d_in, float* a) {
     for (int64_t j = 0; j < d_in; ++j) a[j] = (float)sqrt(sumsq[j]);
 }
 
+/* Other activation norms as the allocation criterion (appendix, norm ablation table:
+ * the l1 and l_inf norms of the channel's activations are compared with l2).
+ * norm 1: acc_j += sum_t |X[t,j]| ; norm 2 (l_inf): acc_j = max(acc_j, max_t |X[t,j]|);
+ * norm 0 is the l2 statistic above.  The criterion a_j is acc_j itself (rounded to
+ * fp32) for l1 and l_inf, its square root for l2. */
+void oracle_collect_stats_norm(const uint16_t* X, int dtype, int64_t n_tokens, int64_t d_in,
+                               int64_t ldx, int norm, double* acc) {
+    for (int64_t t = 0; t < n_tokens; ++t)
+        for (int64_t j = 0; j < d_in; ++j) {
+            double x = (double)oracle_widen(X[t * ldx + j], dtype);
+            if (norm == 0) acc[j] += x * x;
+            else if (norm == 1) acc[j] += fabs(x);
+            else if (fabs(x) > acc[j]) acc[j] = fabs(x);
+        }
+}
+
+void oracle_finalize_stats_norm(const double* acc, int64_t d_in, int norm, float* a) {
+    for (int64_t j = 0; j < d_in; ++j) a[j] = (float)(norm == 0 ? sqrt(acc[j]) : acc[j]);
+}
+
 /* ---------------------------------------------------------------------------
  * Step 2.  Channel-wise precision allocation (Algorithm 1).
  *

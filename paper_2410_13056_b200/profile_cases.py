@@ -5,9 +5,12 @@
     python -m paper_2410_13056_b200.profile_cases pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
     python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
     python -m paper_2410_13056_b200.profile_cases matvec --d-in 8192 --d-out 28672 --budget 2.5 --launches 20
+    python -m paper_2410_13056_b200.profile_cases stack --config c4_stack7b --budget 3.0
     python -m paper_2410_13056_b200.profile_cases layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
 
 `layer` runs the whole pass on one layer of a named workload and prints the time per C-ABI call.
+`stack` quantizes every layer of a multi-block workload (all 32 x 7 layers of the Llama-7B-shaped stack) and
+prints the total device time of the passes; under torchrun the layers are dealt round-robin to the ranks.
 
 Each case prints the mean CUDA-event time per call; every run holds well under 1 GB on the device.
 """
@@ -52,6 +55,56 @@ def run_layer(a):
         print("   %-24s %.3f ms" % (name, t))
     print("   final-fit distance evaluations: %d, inexact rows: %d"
           % (int(q.counters[1].item()), int(q.counters[0].item() & 0xffffffff)))
+
+
+def run_stack(a):
+    """Every layer of the workload, each with its own seeded weights.  The calibration activations are
+    generated once per distinct input width and reused by the layers of that width (the statistic's cost
+    does not depend on the values, and regenerating a gigabyte per layer would only lengthen the untimed
+    part); weight generation is not timed, the passes are (CUDA events around each pass)."""
+    import os
+
+    from . import sharding
+    from .pipeline import LayerQuantizer
+
+    cfg = inputs.CONFIGS[a.config]
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", torch.cuda.current_device()))
+    layers = [(b, i, L) for b in range(cfg.repeat) for i, L in enumerate(cfg.layers)]
+    mine = [layers[k] for k in sharding.layers_of_rank(len(layers), rank, world)]
+    X, quant = {}, {}
+    for _, _, L in mine:
+        if L.d_in not in X:
+            X[L.d_in] = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, cfg.seed + L.d_in, device="cuda")
+        if (L.d_in, L.d_out) not in quant:
+            quant[(L.d_in, L.d_out)] = LayerQuantizer(L.d_in, L.d_out)
+    total_ms, params, inexact = 0.0, 0, 0
+    for n, (b, i, L) in enumerate(mine):
+        W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, cfg.seed + 7 * b + i, device="cuda")
+        q = quant[(L.d_in, L.d_out)]
+        if n < len(quant) * 2:  # first uses of a shape: one untimed pass (module and graph set-up)
+            q.run(X[L.d_in], W, a.budget, cfg.lloyd_iters)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        q.run(X[L.d_in], W, a.budget, cfg.lloyd_iters)
+        e1.record()
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+        params += L.d_in * L.d_out
+        inexact += int(q.counters[0].item() & 0xffffffff)
+    slowest = sharding.max_over_ranks(total_ms, device="cuda")
+    if world > 1:
+        t = torch.tensor([float(params)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t)
+        params = int(t.item())
+        dist.destroy_process_group()
+    if rank == 0:
+        print("stack %s: %d layers (%d blocks x %d), %.3f G weights, avg %.2f bits, T=%d, %d rank(s): %.1f ms of "
+              "passes on the slowest rank, %.0f Mparams/s; inexact rows on rank 0: %d"
+              % (a.config, len(layers), cfg.repeat, len(cfg.layers), params / 1e9, a.budget, cfg.lloyd_iters, world,
+                 slowest, params / slowest / 1e3, inexact))
 
 
 def run_matvec(a, dt):
@@ -110,7 +163,7 @@ def run_matvec(a, dt):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec"])
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec", "stack"])
     ap.add_argument("--config", default="c2_attn7b")
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--budget", type=float, default=3.0)
@@ -127,13 +180,17 @@ def main():
                     help="assignment method of the K-means kernels")
     a = ap.parse_args()
     dt = inputs.BF16 if a.dtype == "bf16" else inputs.F16
-    torch.cuda.set_device(0)
+    import os
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS if a.assign == "all_pairs" else B.ASSIGN_ORDERED)
     if a.case == "layer":
         run_layer(a)
         return
     if a.case == "matvec":
         run_matvec(a, dt)
+        return
+    if a.case == "stack":
+        run_stack(a)
         return
     d_in, d_out = a.d_in, a.d_out
     bits = torch.full((d_in,), a.bits, dtype=torch.uint8, device="cuda")
