@@ -50,6 +50,10 @@ typedef enum {
 
 typedef enum { CMPQ_F16 = 0, CMPQ_BF16 = 1 } cmpq_dtype;
 
+/* Which norm of a channel's activations serves as the allocation criterion.  L2 is the paper's
+ * choice (Section 3.2.1); L1 and LINF are the alternatives its norm-ablation table compares. */
+typedef enum { CMPQ_NORM_L2 = 0, CMPQ_NORM_L1 = 1, CMPQ_NORM_LINF = 2 } cmpq_norm;
+
 /* How Algorithm 1's "q-quantile" is read.  RANK: the floor(|b-3| d_in + 1/2)
  * channels with the smallest (b < 3) or largest (b > 3) statistic change width
  * (at b == 3 exactly: floor(0.01 d_in + 1/2) at each end); equal statistics are
@@ -112,6 +116,20 @@ cmpq_status cmpq_collect_stats_static(const void* X, cmpq_dtype dt, int64_t n_to
 
 /* a[j] = (float) sqrt(sumsq[j]). */
 cmpq_status cmpq_finalize_stats(const double* sumsq, int64_t d_in, float* a, void* stream);
+
+/* The statistic for another norm (appendix of the paper, norm-ablation table).  Same contract as
+ * cmpq_collect_stats / cmpq_finalize_stats with acc (fp64, d_in entries, zeroed by the caller
+ * before the first chunk) accumulating
+ *   CMPQ_NORM_L2    acc[j] += sum_t X[t][j]^2          a[j] = (float) sqrt(acc[j])   (identical to the calls above)
+ *   CMPQ_NORM_L1    acc[j] += sum_t |X[t][j]|          a[j] = (float) acc[j]
+ *   CMPQ_NORM_LINF  acc[j]  = max(acc[j], max_t |X[t][j]|)   a[j] = (float) acc[j]   (exact)
+ * The criterion a then feeds cmpq_allocate_bits and cmpq_extract_outliers unchanged.  An unknown
+ * norm is CMPQ_ERR_INVALID_ARG.  ws: cmpq_workspace_bytes(CMPQ_OP_COLLECT_STATS, d_in, 0). */
+cmpq_status cmpq_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                    int64_t ldx, cmpq_norm norm, double* acc, void* ws, size_t ws_bytes,
+                                    void* stream);
+cmpq_status cmpq_finalize_stats_norm(const double* acc, int64_t d_in, cmpq_norm norm, float* a,
+                                     void* stream);
 
 /* ---- allocation (Algorithm 1) ------------------------------------------------------------------
  * bits[i] in {2,3,4} from the statistic a (fp32, d_in entries, finite, >= 0) and the average

@@ -13,6 +13,7 @@ import torch
 
 F16, BF16 = 0, 1
 ALLOC_RANK, ALLOC_QUANTILE = 0, 1
+NORM_L2, NORM_L1, NORM_LINF = 0, 1, 2
 ASSIGN_ORDERED, ASSIGN_ALL_PAIRS = 0, 1
 (OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK, OP_PROTECT_AND_QUANTIZE,
  OP_OUTLIERS_BY_COLUMN, OP_MATVEC) = range(8)
@@ -24,6 +25,7 @@ EXPORTS = (
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
     "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment", "cmpq_lloyd_phase_events",
     "cmpq_protect_and_quantize", "cmpq_matvec", "cmpq_outliers_by_column",
+    "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -59,6 +61,10 @@ def lib():
         L.cmpq_protect_and_quantize.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
                                                 vp, vp, vp, vp, sz, vp]
         L.cmpq_protect_and_quantize.restype = ci
+        L.cmpq_collect_stats_norm.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, sz, vp]
+        L.cmpq_collect_stats_norm.restype = ci
+        L.cmpq_finalize_stats_norm.argtypes = [vp, i64, ci, vp, vp]
+        L.cmpq_finalize_stats_norm.restype = ci
         L.cmpq_matvec.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_matvec.restype = ci
         L.cmpq_outliers_by_column.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, sz, vp]
@@ -230,3 +236,15 @@ def cmpq_matvec(packed, row_off, perm, seg_rows, lut, x, col_ptr, c_rows, c_vals
     _check(lib().cmpq_matvec(_ptr(packed), _ptr(row_off), _ptr(perm), _ptr(seg_rows), _ptr(lut), d_in, d_out,
                              _ptr(x), dtype_code(x), _ptr(col_ptr), _ptr(c_rows), _ptr(c_vals), _ptr(y),
                              _ptr(y16), _ptr(ws), ws.numel(), _stream()), "cmpq_matvec")
+
+
+def cmpq_collect_stats_norm(X, norm, acc, ws):
+    """acc (float64 [d_in]) accumulates the l2 / l1 / l_inf statistic of X's columns (NORM_L2, NORM_L1, NORM_LINF)."""
+    n, d_in = X.shape
+    _check(lib().cmpq_collect_stats_norm(_ptr(X), dtype_code(X), n, d_in, X.stride(0) if n > 0 else d_in, int(norm),
+                                         _ptr(acc), _ptr(ws), ws.numel(), _stream()), "cmpq_collect_stats_norm")
+
+
+def cmpq_finalize_stats_norm(acc, norm, a):
+    _check(lib().cmpq_finalize_stats_norm(_ptr(acc), acc.numel(), int(norm), _ptr(a), _stream()),
+           "cmpq_finalize_stats_norm")

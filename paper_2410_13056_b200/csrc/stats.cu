@@ -48,24 +48,39 @@ size_t stats_ws_bytes(int64_t d_in) {
     return round_up((size_t)rb * (size_t)ct * kTileCols * sizeof(double), 256);
 }
 
-template <int DT>
+// One activation folded into a running fp32 value: x^2 added (l2, the paper's default), |x| added (l1) or
+// the larger of the two magnitudes (l_inf); the latter two are the criteria of the norm-ablation table.
+template <int NORM>
+__device__ __forceinline__ float fold(float x, float acc) {
+    if (NORM == CMPQ_NORM_L2) return fmaf(x, x, acc);
+    if (NORM == CMPQ_NORM_L1) return acc + fabsf(x);
+    return fmaxf(acc, fabsf(x));
+}
+
+// Two partial results combined: a sum, or a maximum for l_inf.
+template <int NORM>
+__device__ __forceinline__ double join(double a, double b) {
+    return NORM == CMPQ_NORM_LINF ? fmax(a, b) : a + b;
+}
+
+template <int DT, int NORM>
 __device__ __forceinline__ void accumulate8(const uint4& v, float (&acc)[8]) {
     float2 p0 = widen16x2<DT>(v.x), p1 = widen16x2<DT>(v.y);
     float2 p2 = widen16x2<DT>(v.z), p3 = widen16x2<DT>(v.w);
-    acc[0] = fmaf(p0.x, p0.x, acc[0]);
-    acc[1] = fmaf(p0.y, p0.y, acc[1]);
-    acc[2] = fmaf(p1.x, p1.x, acc[2]);
-    acc[3] = fmaf(p1.y, p1.y, acc[3]);
-    acc[4] = fmaf(p2.x, p2.x, acc[4]);
-    acc[5] = fmaf(p2.y, p2.y, acc[5]);
-    acc[6] = fmaf(p3.x, p3.x, acc[6]);
-    acc[7] = fmaf(p3.y, p3.y, acc[7]);
+    acc[0] = fold<NORM>(p0.x, acc[0]);
+    acc[1] = fold<NORM>(p0.y, acc[1]);
+    acc[2] = fold<NORM>(p1.x, acc[2]);
+    acc[3] = fold<NORM>(p1.y, acc[3]);
+    acc[4] = fold<NORM>(p2.x, acc[4]);
+    acc[5] = fold<NORM>(p2.y, acc[5]);
+    acc[6] = fold<NORM>(p3.x, acc[6]);
+    acc[7] = fold<NORM>(p3.y, acc[7]);
 }
 
 // partial[(row_block * tiles + tile) * kTileCols + c] = sum over the block's rows of X[t, tile*256+c]^2
 // The fp64 running totals live in shared memory (slot [warp][i][lane] for column lane*8+i: conflict
 // free), which keeps the register count low enough for 5 resident blocks per SM.
-template <int DT>
+template <int DT, int NORM>
 __global__ void __launch_bounds__(kStatsThreads, 5)
 stats_partial_vec_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64_t d_in, int64_t ldx,
                          int64_t rows_per_block, double* __restrict__ partial) {
@@ -91,35 +106,35 @@ stats_partial_vec_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64
             uint4 v1 = __ldcs(reinterpret_cast<const uint4*>(p + (r + kStatsWarps) * ldx));
             uint4 v2 = __ldcs(reinterpret_cast<const uint4*>(p + (r + 2 * kStatsWarps) * ldx));
             uint4 v3 = __ldcs(reinterpret_cast<const uint4*>(p + (r + 3 * kStatsWarps) * ldx));
-            accumulate8<DT>(v0, acc);
-            accumulate8<DT>(v1, acc);
-            accumulate8<DT>(v2, acc);
-            accumulate8<DT>(v3, acc);
+            accumulate8<DT, NORM>(v0, acc);
+            accumulate8<DT, NORM>(v1, acc);
+            accumulate8<DT, NORM>(v2, acc);
+            accumulate8<DT, NORM>(v3, acc);
             since_flush += 4;
             if (since_flush >= kFlushRows) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { red[warp][i][lane] += (double)acc[i]; acc[i] = 0.f; }
+                for (int i = 0; i < 8; ++i) { red[warp][i][lane] = join<NORM>(red[warp][i][lane], (double)acc[i]); acc[i] = 0.f; }
                 since_flush = 0;
             }
         }
         for (; r < r1; r += kStatsWarps) {
             uint4 v0 = __ldcs(reinterpret_cast<const uint4*>(p + r * ldx));
-            accumulate8<DT>(v0, acc);
+            accumulate8<DT, NORM>(v0, acc);
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) red[warp][i][lane] += (double)acc[i];
+        for (int i = 0; i < 8; ++i) red[warp][i][lane] = join<NORM>(red[warp][i][lane], (double)acc[i]);
     }
     __syncthreads();
     // thread c adds the eight warps' sums of column c in warp order
     const int c = threadIdx.x;
     double s = 0.0;
 #pragma unroll
-    for (int w = 0; w < kStatsWarps; ++w) s += red[w][c & 7][c >> 3];
+    for (int w = 0; w < kStatsWarps; ++w) s = join<NORM>(s, red[w][c & 7][c >> 3]);
     partial[((int64_t)blockIdx.y * gridDim.x + tile) * kTileCols + c] = s;
 }
 
 // Same contract for inputs that cannot be read with aligned 128-bit loads: one column per thread.
-template <int DT>
+template <int DT, int NORM>
 __global__ void __launch_bounds__(kStatsThreads)
 stats_partial_scalar_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, int64_t d_in,
                             int64_t ldx, int64_t rows_per_block, double* __restrict__ partial) {
@@ -134,52 +149,72 @@ stats_partial_scalar_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, in
         int since_flush = 0;
         for (int64_t r = r0; r < r1; ++r) {
             float x = widen16<DT>(X[r * ldx + col]);
-            acc = fmaf(x, x, acc);
-            if (++since_flush == kFlushRows) { total += (double)acc; acc = 0.f; since_flush = 0; }
+            acc = fold<NORM>(x, acc);
+            if (++since_flush == kFlushRows) { total = join<NORM>(total, (double)acc); acc = 0.f; since_flush = 0; }
         }
-        total += (double)acc;
+        total = join<NORM>(total, (double)acc);
     }
     partial[((int64_t)blockIdx.y * gridDim.x + tile) * kTileCols + threadIdx.x] = total;
 }
 
-// sumsq[j] += sum over row blocks (ascending) of partial[rb][j]
+// sumsq[j] += sum over row blocks (ascending) of partial[rb][j]   (l_inf: the maximum instead of the sum)
 __global__ void stats_combine_kernel(const double* __restrict__ partial, int64_t row_blocks,
-                                     int64_t padded_cols, int64_t d_in, double* __restrict__ sumsq) {
+                                     int64_t padded_cols, int64_t d_in, double* __restrict__ sumsq, int take_max) {
     int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= d_in) return;
     double s = 0.0;
-    for (int64_t rb = 0; rb < row_blocks; ++rb) s += partial[rb * padded_cols + j];
-    sumsq[j] += s;
+    if (take_max) {
+        for (int64_t rb = 0; rb < row_blocks; ++rb) s = fmax(s, partial[rb * padded_cols + j]);
+        sumsq[j] = fmax(sumsq[j], s);
+    } else {
+        for (int64_t rb = 0; rb < row_blocks; ++rb) s += partial[rb * padded_cols + j];
+        sumsq[j] += s;
+    }
 }
 
 __global__ void stats_finalize_kernel(const double* __restrict__ sumsq, int64_t d_in,
-                                      float* __restrict__ a) {
+                                      float* __restrict__ a, int take_root) {
     int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j < d_in) a[j] = (float)sqrt(sumsq[j]);
+    if (j < d_in) a[j] = (float)(take_root ? sqrt(sumsq[j]) : sumsq[j]);
+}
+
+template <int NORM>
+static void launch_partial(const uint16_t* Xp, cmpq_dtype dt, bool vec, dim3 grid, int64_t n_tokens, int64_t d_in,
+                           int64_t ldx, int64_t rows_per_block, double* partial, cudaStream_t st) {
+    if (vec) {
+        if (dt == CMPQ_F16)
+            stats_partial_vec_kernel<CMPQ_F16, NORM><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+        else
+            stats_partial_vec_kernel<CMPQ_BF16, NORM><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+    } else {
+        if (dt == CMPQ_F16)
+            stats_partial_scalar_kernel<CMPQ_F16, NORM><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+        else
+            stats_partial_scalar_kernel<CMPQ_BF16, NORM><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
+    }
 }
 
 // Launches the two statistic kernels with `partial` as scratch (row_blocks * tiles * 256 doubles).
-cmpq_status launch_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
-                                 int64_t ldx, double* sumsq, double* partial, int64_t row_blocks,
-                                 cudaStream_t st) {
+cmpq_status launch_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                      int64_t ldx, cmpq_norm norm, double* sumsq, double* partial,
+                                      int64_t row_blocks, cudaStream_t st) {
     const int64_t ct = col_tiles(d_in);
     const int64_t rows_per_block = (n_tokens + row_blocks - 1) / row_blocks;
     const bool vec = aligned_to(X, 16) && (ldx % 8 == 0) && (d_in % 8 == 0);
     dim3 grid((unsigned)ct, (unsigned)row_blocks);
     const uint16_t* Xp = static_cast<const uint16_t*>(X);
-    if (vec) {
-        if (dt == CMPQ_F16)
-            stats_partial_vec_kernel<CMPQ_F16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
-        else
-            stats_partial_vec_kernel<CMPQ_BF16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
-    } else {
-        if (dt == CMPQ_F16)
-            stats_partial_scalar_kernel<CMPQ_F16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
-        else
-            stats_partial_scalar_kernel<CMPQ_BF16><<<grid, kStatsThreads, 0, st>>>(Xp, n_tokens, d_in, ldx, rows_per_block, partial);
-    }
-    stats_combine_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, st>>>(partial, row_blocks, ct * kTileCols, d_in, sumsq);
+    if (norm == CMPQ_NORM_L2) launch_partial<CMPQ_NORM_L2>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
+    else if (norm == CMPQ_NORM_L1) launch_partial<CMPQ_NORM_L1>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
+    else launch_partial<CMPQ_NORM_LINF>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
+    stats_combine_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, st>>>(partial, row_blocks, ct * kTileCols, d_in, sumsq,
+                                                                          norm == CMPQ_NORM_LINF);
     return launch_status();
+}
+
+cmpq_status launch_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                 int64_t ldx, double* sumsq, double* partial, int64_t row_blocks,
+                                 cudaStream_t st) {
+    return launch_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, partial, row_blocks, st);
 }
 
 int64_t stats_row_blocks(int64_t d_in, int64_t n_tokens) {
@@ -192,23 +227,37 @@ int64_t stats_row_blocks(int64_t d_in, int64_t n_tokens) {
 
 using namespace cmpq;
 
-extern "C" cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
-                                          int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
-                                          void* stream) {
-    if (!sumsq || n_tokens < 0 || d_in < 1 || d_in > CMPQ_MAX_D_IN || ldx < d_in) return CMPQ_ERR_INVALID_ARG;
+extern "C" cmpq_status cmpq_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                               int64_t ldx, cmpq_norm norm, double* acc, void* ws, size_t ws_bytes,
+                                               void* stream) {
+    if (!acc || n_tokens < 0 || d_in < 1 || d_in > CMPQ_MAX_D_IN || ldx < d_in) return CMPQ_ERR_INVALID_ARG;
     if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
+    if (norm != CMPQ_NORM_L2 && norm != CMPQ_NORM_L1 && norm != CMPQ_NORM_LINF) return CMPQ_ERR_INVALID_ARG;
     if (n_tokens > 0 && !X) return CMPQ_ERR_INVALID_ARG;
-    if (!aligned_to(X, 2) || !aligned_to(sumsq, 8)) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(X, 2) || !aligned_to(acc, 8)) return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < stats_ws_bytes(d_in)) return CMPQ_ERR_WORKSPACE;
     if (n_tokens == 0) return CMPQ_OK;
     int64_t rb = stats_row_blocks(d_in, n_tokens);
     if (rb <= 0) return CMPQ_ERR_CUDA;
-    return launch_collect_stats(X, dt, n_tokens, d_in, ldx, sumsq, static_cast<double*>(ws), rb,
-                                static_cast<cudaStream_t>(stream));
+    return launch_collect_stats_norm(X, dt, n_tokens, d_in, ldx, norm, acc, static_cast<double*>(ws), rb,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+extern "C" cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
+                                          int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
+                                          void* stream) {
+    return cmpq_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, ws, ws_bytes, stream);
+}
+
+extern "C" cmpq_status cmpq_finalize_stats_norm(const double* acc, int64_t d_in, cmpq_norm norm, float* a,
+                                                void* stream) {
+    if (!acc || !a || d_in < 1 || d_in > CMPQ_MAX_D_IN) return CMPQ_ERR_INVALID_ARG;
+    if (norm != CMPQ_NORM_L2 && norm != CMPQ_NORM_L1 && norm != CMPQ_NORM_LINF) return CMPQ_ERR_INVALID_ARG;
+    stats_finalize_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        acc, d_in, a, norm == CMPQ_NORM_L2);
+    return launch_status();
 }
 
 extern "C" cmpq_status cmpq_finalize_stats(const double* sumsq, int64_t d_in, float* a, void* stream) {
-    if (!sumsq || !a || d_in < 1 || d_in > CMPQ_MAX_D_IN) return CMPQ_ERR_INVALID_ARG;
-    stats_finalize_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(sumsq, d_in, a);
-    return launch_status();
+    return cmpq_finalize_stats_norm(sumsq, d_in, CMPQ_NORM_L2, a, stream);
 }
