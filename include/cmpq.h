@@ -253,6 +253,15 @@ cmpq_status cmpq_outliers_by_column(const int32_t* rows, const int32_t* cols, co
                                     int64_t nnz, int64_t d_out, int64_t* col_ptr, int32_t* c_rows,
                                     uint16_t* c_vals, void* ws, size_t ws_bytes, void* stream);
 
+/* ---- layout conversion (Section 3.2.1: W in R^{d_in x d_out}, a channel is the row W_{i,:}) ----
+ * Frameworks store a linear layer output-major, [d_out][d_in]; every call above takes the paper's
+ * input-channel-major layout.  dst[c*ld_dst + r] = src[r*ld_src + c] for a [rows][cols] source of
+ * 16-bit elements (raw patterns, fp16 or bf16 alike): call it with rows = d_out, cols = d_in to get
+ * W [d_in][ld_dst >= d_out].  src and dst must not overlap.  1 <= rows, cols <= CMPQ_MAX_D_IN,
+ * ld_src >= cols, ld_dst >= rows, else CMPQ_ERR_INVALID_ARG.  No work space. */
+cmpq_status cmpq_transpose16(const void* src, int64_t rows, int64_t cols, int64_t ld_src, void* dst,
+                             int64_t ld_dst, void* stream);
+
 /* ---- host helpers (pure functions, no GPU work) ----------------------------------------------- */
 size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out);
 /* Algorithm 1 in rank form: how many channels get 2 and 4 bits. */

@@ -25,7 +25,7 @@ EXPORTS = (
     "cmpq_default_counts", "cmpq_packed_words", "cmpq_status_string",
     "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment", "cmpq_lloyd_phase_events",
     "cmpq_protect_and_quantize", "cmpq_matvec", "cmpq_outliers_by_column",
-    "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm",
+    "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -65,6 +65,8 @@ def lib():
         L.cmpq_collect_stats_norm.restype = ci
         L.cmpq_finalize_stats_norm.argtypes = [vp, i64, ci, vp, vp]
         L.cmpq_finalize_stats_norm.restype = ci
+        L.cmpq_transpose16.argtypes = [vp, i64, i64, i64, vp, i64, vp]
+        L.cmpq_transpose16.restype = ci
         L.cmpq_matvec.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_matvec.restype = ci
         L.cmpq_outliers_by_column.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp, sz, vp]
@@ -248,3 +250,14 @@ def cmpq_collect_stats_norm(X, norm, acc, ws):
 def cmpq_finalize_stats_norm(acc, norm, a):
     _check(lib().cmpq_finalize_stats_norm(_ptr(acc), acc.numel(), int(norm), _ptr(a), _stream()),
            "cmpq_finalize_stats_norm")
+
+
+def cmpq_transpose16(src, dst):
+    """dst[c][r] = src[r][c] for 2-D fp16/bf16 tensors with unit inner stride (e.g. a framework's [d_out][d_in]
+    weight into the [d_in][d_out] layout the other calls take)."""
+    rows, cols = src.shape
+    if src.stride(1) != 1 or dst.stride(1) != 1 or tuple(dst.shape) != (cols, rows) or src.dtype != dst.dtype:
+        raise ValueError("cmpq_transpose16 needs row-major 2-D tensors of one dtype with shapes [r][c] and [c][r]")
+    dtype_code(src)
+    _check(lib().cmpq_transpose16(_ptr(src), rows, cols, src.stride(0), _ptr(dst), dst.stride(0), _stream()),
+           "cmpq_transpose16")

@@ -328,6 +328,8 @@ matvec_partial_kernel(const uint32_t* __restrict__ packed, const int64_t* __rest
                       const float* __restrict__ lut, const uint16_t* __restrict__ x, int64_t d_out,
                       int rows_per_block, float* __restrict__ partial) {
     extern __shared__ __align__(16) unsigned char raw[];
+    // the finishing kernel may be scheduled from now on (it waits for this grid before it reads a partial sum)
+    asm volatile("griddepcontrol.launch_dependents;");
     const MvChunk ch = matvec_chunk(seg_rows, blockIdx.y, rows_per_block);
     if (ch.c == 0) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -390,20 +392,12 @@ matvec_finish_kernel(const float* __restrict__ partial, const int64_t* __restric
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t j = (int64_t)blockIdx.x * 32 + lane;
     const int64_t chunks = matvec_total_chunks(seg_rows, rows_per_block);
-    float s = 0.0f;
-    if (j < d_out) {
-        // everything independent is requested before anything is added: the column's outlier range first,
-        // then four partial sums per step (absent ones read as 0; the additions keep their order)
-        const int64_t e0 = col_ptr != nullptr ? col_ptr[j] : 0, e1 = col_ptr != nullptr ? col_ptr[j + 1] : 0;
-        for (int64_t q = warp; q < chunks; q += 4 * kMvWarps) {
-            float pv[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) pv[u] = (q + u * kMvWarps < chunks) ? partial[(q + u * kMvWarps) * d_out + j] : 0.0f;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) s += pv[u];
-        }
-        float so = 0.0f;
-        for (int64_t e = e0 + warp; e < e1; e += 4 * kMvWarps) {
+    // The outlier products need nothing from the partial kernel, so they run first: this kernel is launched
+    // as a programmatic dependent of the partial kernel and may start while that one is still running.
+    float so = 0.0f;
+    if (j < d_out && col_ptr != nullptr) {
+        const int64_t e0 = col_ptr[j], e1 = col_ptr[j + 1];
+        for (int64_t e = e0 + warp; e < e1; e += 4 * kMvWarps) {  // four entries in flight, additions in order
             int32_t rw[4];
             uint16_t vv[4], xv[4];
 #pragma unroll
@@ -416,6 +410,19 @@ matvec_finish_kernel(const float* __restrict__ partial, const int64_t* __restric
             for (int u = 0; u < 4; ++u) xv[u] = rw[u] >= 0 ? x[rw[u]] : (uint16_t)0;
 #pragma unroll
             for (int u = 0; u < 4; ++u) so += widen16<DT>(xv[u]) * widen16<DT>(vv[u]);
+        }
+    }
+    // From here on the partial sums are read: wait until the partial kernel has completed and its stores
+    // are visible (returns at once when the kernel was launched without the dependency).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    float s = 0.0f;
+    if (j < d_out) {
+        for (int64_t q = warp; q < chunks; q += 4 * kMvWarps) {  // absent partial sums read as 0
+            float pv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) pv[u] = (q + u * kMvWarps < chunks) ? __ldcg(partial + (q + u * kMvWarps) * d_out + j) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) s += pv[u];
         }
         s += so;
     }
@@ -592,16 +599,31 @@ extern "C" cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_of
     const unsigned fin_blocks = (unsigned)((d_out + 31) / 32);
     const uint16_t* xu = static_cast<const uint16_t*>(x);
     uint16_t* yu = static_cast<uint16_t*>(y16);
+    // the finishing kernel is a programmatic dependent of the partial kernel: its launch and its outlier
+    // products overlap the partial kernel, its griddepcontrol.wait orders the reads of the partial sums
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(fin_blocks);
+    cfg.blockDim = dim3(kMvThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float* partial_in = partial;
+    cudaError_t err;
     if (dt == CMPQ_BF16) {
         matvec_partial_kernel<CMPQ_BF16><<<grid, kMvThreads, kMvSharedBytes, st>>>(packed, row_off, perm, seg_rows, lut,
                                                                                    xu, d_out, rb, partial);
-        matvec_finish_kernel<CMPQ_BF16><<<fin_blocks, kMvThreads, 0, st>>>(partial, seg_rows, rb, d_out, xu, col_ptr,
-                                                                           c_rows, c_vals, y, yu);
+        err = cudaLaunchKernelEx(&cfg, matvec_finish_kernel<CMPQ_BF16>, partial_in, seg_rows, rb, d_out, xu, col_ptr,
+                                 c_rows, c_vals, y, yu);
     } else {
         matvec_partial_kernel<CMPQ_F16><<<grid, kMvThreads, kMvSharedBytes, st>>>(packed, row_off, perm, seg_rows, lut,
                                                                                   xu, d_out, rb, partial);
-        matvec_finish_kernel<CMPQ_F16><<<fin_blocks, kMvThreads, 0, st>>>(partial, seg_rows, rb, d_out, xu, col_ptr,
-                                                                          c_rows, c_vals, y, yu);
+        err = cudaLaunchKernelEx(&cfg, matvec_finish_kernel<CMPQ_F16>, partial_in, seg_rows, rb, d_out, xu, col_ptr,
+                                 c_rows, c_vals, y, yu);
     }
+    if (err != cudaSuccess) return CMPQ_ERR_CUDA;
     return launch_status();
 }

@@ -5,6 +5,7 @@
     python -m paper_2410_13056_b200.profile_cases pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
     python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
     python -m paper_2410_13056_b200.profile_cases matvec --d-in 8192 --d-out 28672 --budget 2.5 --launches 20
+    python -m paper_2410_13056_b200.profile_cases transpose --d-in 16384 --d-out 16384 --launches 10
     python -m paper_2410_13056_b200.profile_cases stack --config c4_stack7b --budget 3.0
     python -m paper_2410_13056_b200.profile_cases layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
 
@@ -163,7 +164,7 @@ def run_matvec(a, dt):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec", "stack"])
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec", "stack", "transpose"])
     ap.add_argument("--config", default="c2_attn7b")
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--budget", type=float, default=3.0)
@@ -195,7 +196,12 @@ def main():
     d_in, d_out = a.d_in, a.d_out
     bits = torch.full((d_in,), a.bits, dtype=torch.uint8, device="cuda")
 
-    if a.case == "stats":
+    if a.case == "transpose":  # a framework's [d_out][d_in] weight into the library's [d_in][d_out]
+        src = inputs.make_weight(d_out, d_in, dt, 1, device="cuda")
+        dst = torch.empty((d_in, d_out), dtype=src.dtype, device="cuda")
+        fn = lambda: B.cmpq_transpose16(src, dst)
+        work = "%.1f MB read + %.1f MB written" % (src.numel() * 2 / 1e6, src.numel() * 2 / 1e6)
+    elif a.case == "stats":
         X = inputs.make_activations(a.tokens, d_in, dt, 1, device="cuda")
         sumsq = torch.zeros(d_in, dtype=torch.float64, device="cuda")
         ws = B.workspace(B.OP_COLLECT_STATS, d_in)

@@ -24,7 +24,7 @@ def L():
 def test_every_declared_symbol_is_exported(L):
     header = open(os.path.join(ROOT, "include", "cmpq.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(cmpq_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(cmpq_[a-z0-9_]+)\s*\(", header))
     assert declared == set(B.EXPORTS)
     for name in declared:
         assert hasattr(L, name), name
