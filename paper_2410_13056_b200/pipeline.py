@@ -79,8 +79,23 @@ class LayerQuantizer:
         w = lambda c: (self.d_out * c + 31) // 32
         return n2 * w(2) + n3 * w(3) + n4 * w(4)
 
-    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None):
+    def run_budgets(self, X, W, budgets, lloyd_iters, on_result=None):
+        """The pass for several average budgets on the same layer (the paper's budget sweeps: any new
+        constraint means quantizing again).  The activation statistic does not depend on the budget, so it
+        is computed once and every budget re-runs only Algorithm 1, outlier protection, the K-means and the
+        packing; each budget's outputs are exactly those of a separate run().  The output buffers are
+        reused, so on_result(budget, result) is called after each budget's work has been enqueued (copy what
+        you need there, on the same stream).  Returns the last result."""
+        result = None
+        for k, b in enumerate(budgets):
+            result = self.run(X, W, b, lloyd_iters, reuse_statistic=k > 0)
+            if on_result is not None:
+                on_result(b, result)
+        return result
+
+    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None, reuse_statistic=False):
         """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
+        reuse_statistic: keep the statistic `a` of the previous run on the same X (see run_budgets).
         fused (default: True unless events are asked for): outlier protection and final fit through
         cmpq_protect_and_quantize, which derives the final fit's value tables from the provisional
         fit's; otherwise cmpq_extract_outliers and cmpq_quantize_layer one after the other (same
@@ -101,12 +116,13 @@ class LayerQuantizer:
             e1.record()
             events[name] = (e0, e1)
 
-        self.sumsq.zero_()
         self.counters.zero_()
         inexact = self.counters[0:1].view(torch.int32)[0:1]
         sweeps = self.counters[1:2]
-        call("cmpq_collect_stats", B.cmpq_collect_stats, X, self.sumsq, self.ws)
-        call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
+        if not reuse_statistic:
+            self.sumsq.zero_()
+            call("cmpq_collect_stats", B.cmpq_collect_stats, X, self.sumsq, self.ws)
+            call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
         call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
              self.ws)
         if fused:

@@ -6,6 +6,7 @@
     python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
     python -m paper_2410_13056_b200.profile_cases matvec --d-in 8192 --d-out 28672 --budget 2.5 --launches 20
     python -m paper_2410_13056_b200.profile_cases transpose --d-in 16384 --d-out 16384 --launches 10
+    python -m paper_2410_13056_b200.profile_cases sweep --config c3_mlp7b --layer 0 --launches 5
     python -m paper_2410_13056_b200.profile_cases stack --config c4_stack7b --budget 3.0
     python -m paper_2410_13056_b200.profile_cases layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
 
@@ -108,6 +109,35 @@ def run_stack(a):
                  slowest, params / slowest / 1e3, inexact))
 
 
+def run_sweep(a):
+    """All budgets of a workload on one layer: separate passes against run_budgets (statistic computed once)."""
+    from .pipeline import LayerQuantizer
+
+    cfg = inputs.CONFIGS[a.config]
+    L = cfg.layers[a.layer]
+    seed = inputs.layer_seed(cfg, a.layer)
+    W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, seed, device="cuda")
+    X = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, seed, device="cuda")
+    q = LayerQuantizer(L.d_in, L.d_out)
+    budgets = list(cfg.budgets)
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(a.launches):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / a.launches
+
+    separate = timed(lambda: [q.run(X, W, b, cfg.lloyd_iters) for b in budgets])
+    shared = timed(lambda: q.run_budgets(X, W, budgets, cfg.lloyd_iters))
+    print("sweep %s[%d] d_in=%d d_out=%d, budgets %s: %.3f ms as separate passes, %.3f ms with the statistic "
+          "computed once" % (a.config, a.layer, L.d_in, L.d_out, budgets, separate, shared))
+
+
 def run_matvec(a, dt):
     """The inference product on a random quantized layer (codes are random, so no quantization runs):
     widths split as the rank-form allocation splits them for the budget."""
@@ -164,7 +194,7 @@ def run_matvec(a, dt):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec", "stack", "transpose"])
+    ap.add_argument("case", choices=["lloyd", "stats", "pack", "outliers", "protect", "layer", "matvec", "stack", "transpose", "sweep"])
     ap.add_argument("--config", default="c2_attn7b")
     ap.add_argument("--layer", type=int, default=0)
     ap.add_argument("--budget", type=float, default=3.0)
@@ -192,6 +222,9 @@ def main():
         return
     if a.case == "stack":
         run_stack(a)
+        return
+    if a.case == "sweep":
+        run_sweep(a)
         return
     d_in, d_out = a.d_in, a.d_out
     bits = torch.full((d_in,), a.bits, dtype=torch.uint8, device="cuda")

@@ -198,3 +198,19 @@ def test_graph_replay_gives_the_same_bytes_as_the_eager_pass():
         assert np.array_equal(eager[k], first[k]), k
         assert np.array_equal(replay[k], again[k]), k
     assert not np.array_equal(eager["codes"], replay["codes"])
+
+
+def test_budget_sweep_shares_the_statistic():
+    """run_budgets computes the statistic once; every budget's outputs equal those of a separate pass."""
+    d_in, d_out, n, T = 192, 640, 1024, 6
+    W = inputs.make_weight(d_in, d_out, inputs.BF16, 61, device="cuda")
+    X = inputs.make_activations(n, d_in, inputs.BF16, 61, device="cuda")
+    budgets = [2.0, 2.5, 3.0, 3.5, 4.0]
+    q = LayerQuantizer(d_in, d_out)
+    got = {}
+    q.run_budgets(X, W, budgets, T, on_result=lambda b, r: got.__setitem__(b, {k: v.copy() for k, v in _np(r).items()}))
+    q2 = LayerQuantizer(d_in, d_out)
+    for b in budgets:
+        sep = _np(q2.run(X, W, b, T))
+        for k in sep:
+            assert np.array_equal(got[b][k], sep[k]), (b, k)

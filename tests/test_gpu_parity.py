@@ -303,17 +303,19 @@ def test_protect_and_quantize_equals_the_two_calls(dtype, d_in, d_out, n_act, n_
 
 
 # ----------------------------------------------------------------------------- layout conversion
-@pytest.mark.parametrize("shape", [(1, 1), (64, 64), (65, 63), (300, 1030), (4096, 11008), (11008, 4096)])
+@pytest.mark.parametrize("shape", [(1, 1), (64, 64), (65, 63), (300, 1030), (66, 2), (4096, 11008), (11008, 4096)])
+@pytest.mark.parametrize("pads", [(4, 6), (3, 5)])   # even leading dimensions: 32-bit accesses; odd: element-wise
 @pytest.mark.parametrize("tdt", [torch.float16, torch.bfloat16])
-def test_transpose16_is_the_transpose(shape, tdt):
+def test_transpose16_is_the_transpose(shape, pads, tdt):
     """Plain definition: dst[c][r] = src[r][c], raw 16-bit patterns (checked against numpy on the host)."""
     g = torch.Generator(device="cuda")
     g.manual_seed(shape[0] * 7 + shape[1])
     bits = torch.randint(-32768, 32768, shape, dtype=torch.int16, device="cuda", generator=g)
     src = bits.view(tdt)
-    dst = torch.full((shape[1], shape[0] + 3), 1.0, dtype=tdt, device="cuda")[:, : shape[0]]   # padded rows
+    full = torch.full((shape[1], shape[0] + pads[0]), 1.0, dtype=tdt, device="cuda")
+    dst = full[:, : shape[0]]                                                               # padded rows
     B.cmpq_transpose16(src, dst)
-    wide = torch.full((shape[0], shape[1] + 5), 1.0, dtype=tdt, device="cuda")
+    wide = torch.full((shape[0], shape[1] + pads[1]), 1.0, dtype=tdt, device="cuda")
     wide[:, : shape[1]] = src
     dst2 = torch.empty((shape[1], shape[0]), dtype=tdt, device="cuda")
     B.cmpq_transpose16(wide[:, : shape[1]], dst2)                                            # padded source
@@ -321,3 +323,4 @@ def test_transpose16_is_the_transpose(shape, tdt):
     ref = np.ascontiguousarray(bits.cpu().numpy().T)
     assert np.array_equal(dst.contiguous().view(torch.int16).cpu().numpy(), ref)
     assert np.array_equal(dst2.view(torch.int16).cpu().numpy(), ref)
+    assert torch.all(full[:, shape[0]:] == 1.0)                                             # padding untouched
