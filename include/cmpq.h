@@ -165,7 +165,14 @@ cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, in
  * exactly lloyd_iters updates (1..CMPQ_MAX_LLOYD_ITERS; 0 is allowed and returns the start),
  * then a last assignment.  lut: [d_in][CMPQ_LUT_STRIDE] fp32, the first K entries valid, the
  * rest 0.  codes: [d_in][d_out] uint8.
- * sens: must be NULL (the paper's K-means is unweighted); non-NULL gives CMPQ_ERR_UNSUPPORTED.
+ * sens: NULL for the paper's unweighted K-means.  Otherwise [d_in][d_out] fp32 sensitivities s >= 0
+ * (finite), one per weight: the update becomes the weighted mean  c_k = sum s x / sum s  over the
+ * members (a cluster whose members' sensitivities sum to 0 keeps c_k); start and assignment are
+ * unchanged.  The products s*x are not exact in fp64, so the sums depend on the order of summation:
+ * the result is deterministic, and agrees with a sequential sum to rounding (centroids to about
+ * 1e-7 relative; with all s equal it equals the unweighted fit bit for bit whenever inexact_rows
+ * stays 0 there).  The weighted fit evaluates all pairs whatever cmpq_set_lloyd_assignment says and
+ * leaves inexact_rows untouched.
  * inexact_rows (optional device int32, caller zeroes it): incremented for every channel whose
  * dynamic range is so wide that fp64 cluster sums may depend on the order of summation; when
  * it stays 0 the centroids are independent of the summation order, hence reproducible bit

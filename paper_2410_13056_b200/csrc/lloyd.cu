@@ -648,7 +648,7 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
     if (nnz < 0 || nnz > d_in * d_out || (nnz > 0 && (!rows || !cols))) return CMPQ_ERR_INVALID_ARG;
     if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
     if (!aligned_to(W, 2) || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
-    if (sens) return CMPQ_ERR_UNSUPPORTED;
+    if (sens && !aligned_to(sens, 4)) return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int64_t* row_ptr = static_cast<int64_t*>(ws);
@@ -665,6 +665,7 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
     a.codes = codes;
     a.inexact_rows = inexact_rows;
     a.sweeps = sweeps;
+    if (sens) return launch_lloyd_weighted(a, dt, sens, st);
     if (lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS) return launch_lloyd(a, dt, st);
     return launch_lloyd_ordered(a, dt, static_cast<char*>(ws) + row_ptr_bytes(d_in), lloyd_tables_bytes(d_in, d_out), st);
 }

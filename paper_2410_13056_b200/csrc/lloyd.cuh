@@ -57,6 +57,10 @@ void set_lloyd_phase_events(void* const* events);
 cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,
                                  cudaStream_t st);
 
+// Weighted fit (sens: [d_in][d_out] fp32 sensitivities): one block per channel, every (weight, centroid) pair
+// evaluated in every iteration; writes args.lut / args.codes / args.sweeps, ignores the other outputs.
+cmpq_status launch_lloyd_weighted(const LloydArgs& args, cmpq_dtype dt, const float* sens, cudaStream_t st);
+
 // Fills row_ptr[0..d_in] from a row-sorted coordinate list.
 cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64_t* row_ptr,
                            cudaStream_t st);

@@ -188,8 +188,11 @@ struct MvRows<C, kMvRowsPerWarp> {
     static __device__ __forceinline__ void run(const uint32_t (&)[kMvRowsPerWarp][C], uint32_t, float (&)[32]) {}
 };
 
+#ifndef CMPQ_MV_PAIR_MAX_BITS
+#define CMPQ_MV_PAIR_MAX_BITS 3  // widest channels that share a table between two channels
+#endif
 template <int C>
-constexpr bool kMvUsePairs = (C < 4);
+constexpr bool kMvUsePairs = (C <= CMPQ_MV_PAIR_MAX_BITS);
 
 // ---- staging of the code words: asynchronous copies into a per-lane slot of shared memory -------------
 // Every lane copies the C words of its own group for each row of a pass; word t of row q of lane l lands at

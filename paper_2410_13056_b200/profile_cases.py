@@ -207,6 +207,8 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16"])
     ap.add_argument("--fused", action="store_true",
                     help="layer case: outlier protection and final fit through cmpq_protect_and_quantize")
+    ap.add_argument("--weighted", action="store_true",
+                    help="lloyd case: the sensitivity-weighted fit (random sensitivities)")
     ap.add_argument("--assign", default="ordered", choices=["ordered", "all_pairs"],
                     help="assignment method of the K-means kernels")
     a = ap.parse_args()
@@ -257,7 +259,8 @@ def main():
             codes = torch.empty((d_in, d_out), dtype=torch.uint8, device="cuda")
             counters = torch.zeros(2, dtype=torch.int64, device="cuda")
             ws = B.workspace(B.OP_QUANTIZE_LAYER, d_in, d_out)
-            fn = lambda: B.cmpq_quantize_layer(W, bits, None, None, a.iters, lut, codes, ws,
+            sens = (torch.rand((d_in, d_out), device="cuda") + 0.5) if a.weighted else None
+            fn = lambda: B.cmpq_quantize_layer(W, bits, None, None, a.iters, lut, codes, ws, sens=sens,
                                                sweeps=counters[1:2])
             work = "%d channels x %d weights, K=%d, T=%d" % (d_in, d_out, 1 << a.bits, a.iters)
         else:

@@ -47,7 +47,7 @@ def gpu_extract(W, a_np, bits_np, n_act, n_q, T):
     return rows.cpu().numpy(), cols.cpu().numpy(), vals.cpu().numpy().view(np.uint16)
 
 
-def gpu_quantize(W, bits_np, rows_np, cols_np, T):
+def gpu_quantize(W, bits_np, rows_np, cols_np, T, sens=None):
     d_in, d_out = W.shape
     lut = torch.full((d_in, 16), -7.0, dtype=torch.float32, device="cuda")
     codes = torch.full((d_in, d_out), 255, dtype=torch.uint8, device="cuda")
@@ -55,7 +55,7 @@ def gpu_quantize(W, bits_np, rows_np, cols_np, T):
     rows = dev(rows_np) if len(rows_np) else None
     cols = dev(cols_np) if len(cols_np) else None
     B.cmpq_quantize_layer(W, dev(bits_np), rows, cols, T, lut, codes,
-                          B.workspace(B.OP_QUANTIZE_LAYER, d_in, d_out),
+                          B.workspace(B.OP_QUANTIZE_LAYER, d_in, d_out), sens=sens,
                           inexact_rows=counters[0:1].view(torch.int32)[0:1], sweeps=counters[1:2])
     torch.cuda.synchronize()
     c = counters.cpu().numpy()

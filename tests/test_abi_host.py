@@ -88,7 +88,7 @@ def test_bad_arguments_are_refused_on_the_host(L):
     assert L.cmpq_extract_outliers(*args(0, 0, 0, d_out=40000)) == INVALID                 # d_out too large
     # quantizer
     q = lambda sens=None, nnz=0, rows=None, d_out=16, iters=5: (p, 0, 8, d_out, d_out, p, rows, rows, nnz, iters, sens, p, p, None, None, ws, 1 << 30, None)
-    assert L.cmpq_quantize_layer(*q(sens=p)) == UNSUPPORTED
+    assert L.cmpq_quantize_layer(*q(sens=ctypes.c_void_p(p.value + 2))) == INVALID           # misaligned sensitivities
     assert L.cmpq_quantize_layer(*q(nnz=3)) == INVALID                                     # list missing
     assert L.cmpq_quantize_layer(*q(d_out=0)) == INVALID
     assert L.cmpq_quantize_layer(*q(iters=2000)) == INVALID
