@@ -7,7 +7,7 @@
 // One block per channel, the channel resident in shared memory as fp32 for all iterations (HBM traffic: the
 // weights and their sensitivities once per iteration from L2, codes once).  The products s_i x_i are not
 // exact in fp64, so cluster sums depend on the order of summation: the order here is fixed (thread-strided
-// partial sums, then a fixed tree), which makes the result deterministic, but it is not the index order of a
+// partial sums, a fixed tree inside each warp, the warps in order), which makes the result deterministic, but it is not the index order of a
 // sequential sum -- results agree with such a sum to rounding, not bit for bit.
 #include "common.cuh"
 #include "lloyd.cuh"
@@ -26,29 +26,6 @@ __device__ __forceinline__ uint16_t key_pattern(uint32_t key) {
     return (key & 0x8000u) ? (uint16_t)(key & 0x7fffu) : (uint16_t)~key;
 }
 
-// Deterministic block sum of two doubles (result valid in every thread).
-__device__ __forceinline__ void block_sum2(double& a, double& b, double (*scratch)[2]) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        a += __shfl_down_sync(0xffffffffu, a, o);
-        b += __shfl_down_sync(0xffffffffu, b, o);
-    }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();  // scratch free again
-    if (lane == 0) {
-        scratch[warp][0] = a;
-        scratch[warp][1] = b;
-    }
-    __syncthreads();
-    a = 0.0;
-    b = 0.0;
-#pragma unroll
-    for (int w = 0; w < kWWarps; ++w) {
-        a += scratch[w][0];
-        b += scratch[w][1];
-    }
-}
-
 template <int DT>
 __global__ void __launch_bounds__(kWThreads)
 lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw, const uint8_t* __restrict__ bits,
@@ -62,7 +39,7 @@ lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw
     __shared__ int hist_lo[16][256];
     __shared__ int bin_of[16], rank_in_bin[16];
     __shared__ float c[16];
-    __shared__ double scratch[kWWarps][2];
+    __shared__ double warp_sums[16][kWWarps][2];  // per cluster and warp: sum of s*x, sum of s
     __shared__ int changed;
     const int64_t i = blockIdx.x;
     const int tid = threadIdx.x;
@@ -133,7 +110,8 @@ lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw
             code[j] = (uint8_t)best;
         }
         __syncthreads();
-        // update: weighted mean of each cluster's members, clusters one after the other
+        // update: weighted mean of each cluster's members.  Every thread sums its own weights of cluster k,
+        // a warp adds its lanes in a fixed tree, and after ONE barrier thread k adds the warps in order.
         for (int k = 0; k < K; ++k) {
             double S = 0.0, n = 0.0;
             for (int j = tid; j < N; j += kWThreads)
@@ -142,11 +120,28 @@ lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw
                     S += sj * (double)x[j];
                     n += sj;
                 }
-            block_sum2(S, n, scratch);
-            if (tid == 0 && n > 0.0) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                S += __shfl_down_sync(0xffffffffu, S, o);
+                n += __shfl_down_sync(0xffffffffu, n, o);
+            }
+            if ((tid & 31) == 0) {
+                warp_sums[k][tid >> 5][0] = S;
+                warp_sums[k][tid >> 5][1] = n;
+            }
+        }
+        __syncthreads();
+        if (tid < K) {
+            double S = 0.0, n = 0.0;
+#pragma unroll
+            for (int wq = 0; wq < kWWarps; ++wq) {
+                S += warp_sums[tid][wq][0];
+                n += warp_sums[tid][wq][1];
+            }
+            if (n > 0.0) {
                 const float nc = (float)(S / n);
-                if (__float_as_uint(nc) != __float_as_uint(c[k])) changed = 1;
-                c[k] = nc;
+                if (__float_as_uint(nc) != __float_as_uint(c[tid])) changed = 1;
+                c[tid] = nc;
             }
         }
         __syncthreads();
