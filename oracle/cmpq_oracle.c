@@ -24,7 +24,10 @@
  * points, sklearn's Lloyd from the same start, full-sort top-k, pack/unpack
  * round trip, the storage figures the paper prints; for the inference product:
  * unit inputs, exactly representable layers, a dense float64 matrix product and
- * the reconstruction error of the same layer.
+ * the reconstruction error of the same layer; for the l1 / l_inf statistics:
+ * numpy's vector norms, closed forms, chunking and the norm inequalities; for
+ * the weighted update: constant weights change nothing, every non-empty
+ * centroid is its members' weighted mean.
  * Parity unpinned: none of the paper's perplexity tables can pin the
  * reconstruction error (no model weights exist here); oracle_recon_error is
  * pinned only against a dense float64 numpy evaluation of the same definition.
