@@ -72,6 +72,7 @@ def _check(q, dtype, y, y16=None, with_outliers=True):
     ((257, 1030), (100, 57, 100), 3, 300),     # two column tiles, ragged tail, odd word counts
     ((700, 2080), (3, 690, 7), 4, 900),        # several chunks per segment, short segments
     ((1200, 4096), (600, 200, 400), 5, 2400),
+    ((70, 32768), (20, 30, 20), 1, 500),       # the widest layer the library takes
 ])
 def test_matvec_against_the_checker(dtype, shape, counts, n_act, n_q):
     q = inputs.make_quantized_layer(shape[0], shape[1], counts, dtype, 17 + shape[0], n_act, n_q)

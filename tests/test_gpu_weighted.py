@@ -31,7 +31,8 @@ def _first_min_codes(x, lut, K):
 
 
 @pytest.mark.parametrize("dtype", [inputs.F16, inputs.BF16])
-@pytest.mark.parametrize("shape,T,nnz", [((24, 512), 10, 0), ((40, 1000), 20, 300), ((7, 4096), 20, 50), ((3, 16), 5, 4)])
+@pytest.mark.parametrize("shape,T,nnz", [((24, 512), 10, 0), ((40, 1000), 20, 300), ((7, 4096), 20, 50), ((3, 16), 5, 4),
+                                         ((5, 32768), 8, 100)])   # the widest channel the library takes
 def test_weighted_fit_against_the_checker(dtype, shape, T, nnz):
     d_in, d_out = shape
     W = inputs.make_weight(d_in, d_out, dtype, 100 + d_out, device="cuda")
