@@ -240,9 +240,12 @@ cmpq_status cmpq_pack(const uint8_t* codes, const uint8_t* bits, int64_t d_in, i
  * outliers grouped by column as written by cmpq_outliers_by_column (values of the same `dt`), or
  * three NULLs for a layer without outliers.  y: d_out fp32.  y16 (optional, may be NULL): the same
  * result rounded to nearest even into `dt` (the paper accumulates into 16-bit outputs).
- * Arithmetic: fp32; x[i]*lut[i][k] is formed once per table entry, a column's sum is taken over
- * blocks of channels in a fixed order, so the result is deterministic and differs from the exact
- * sum by at most a few hundred units of 2^-24 relative to sum_i |x[i] * w_ij|.
+ * Arithmetic: fp32; x[i]*lut[i][k] is formed once per table entry (for 2- and 3-bit channels the
+ * entries of two neighbouring channels are added into one table first), a column's sum is taken
+ * over blocks of channels in a fixed order, so the result is deterministic and differs from the
+ * exact sum by at most a few hundred units of 2^-24 relative to sum_i |x[i] * w_ij|.
+ * The call enqueues two kernels, the second as a programmatic dependent of the first (it starts
+ * early and waits for the first before it reads its results); both complete in stream order.
  * 1 <= d_out <= CMPQ_MAX_D_OUT.  ws: cmpq_workspace_bytes(CMPQ_OP_MATVEC, d_in, d_out). */
 cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
                         const int64_t* seg_rows, const float* lut, int64_t d_in, int64_t d_out,
