@@ -26,6 +26,35 @@ __device__ __forceinline__ uint16_t key_pattern(uint32_t key) {
     return (key & 0x8000u) ? (uint16_t)(key & 0x7fffu) : (uint16_t)~key;
 }
 
+// Nearest centroid of every weight of the channel (first minimum of fabsf(x - c_k), k ascending), the K
+// centroids held in registers.
+template <int K>
+__device__ __forceinline__ void assign_codes(const float* __restrict__ x, const float* c, int N, uint8_t* out) {
+    float cr[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) cr[k] = c[k];
+    for (int j = threadIdx.x; j < N; j += kWThreads) {
+        const float v = x[j];
+        int best = 0;
+        float bd = fabsf(v - cr[0]);
+#pragma unroll
+        for (int k = 1; k < K; ++k) {
+            const float d = fabsf(v - cr[k]);
+            if (d < bd) {
+                bd = d;
+                best = k;
+            }
+        }
+        out[j] = (uint8_t)best;
+    }
+}
+
+__device__ __forceinline__ void assign_codes(int K, const float* __restrict__ x, const float* c, int N, uint8_t* out) {
+    if (K == 4) assign_codes<4>(x, c, N, out);
+    else if (K == 8) assign_codes<8>(x, c, N, out);
+    else assign_codes<16>(x, c, N, out);
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kWThreads)
 lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw, const uint8_t* __restrict__ bits,
@@ -95,20 +124,7 @@ lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw
     int done = 0;
     for (int it = 0; it < iters; ++it) {
         if (tid == 0) changed = 0;  // ordered before the updates by the barrier after the assignment
-        // assignment: first k minimising fabsf(x - c_k)
-        for (int j = tid; j < N; j += kWThreads) {
-            const float v = x[j];
-            int best = 0;
-            float bd = fabsf(v - c[0]);
-            for (int k = 1; k < K; ++k) {
-                const float d = fabsf(v - c[k]);
-                if (d < bd) {
-                    bd = d;
-                    best = k;
-                }
-            }
-            code[j] = (uint8_t)best;
-        }
+        assign_codes(K, x, c, N, code);
         __syncthreads();
         // update: weighted mean of each cluster's members.  Every thread sums its own weights of cluster k,
         // a warp adds its lanes in a fixed tree, and after ONE barrier thread k adds the warps in order.
@@ -151,19 +167,7 @@ lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw
         if (!moved) break;         // every later iteration would repeat this one
     }
     // last assignment and outputs
-    for (int j = tid; j < N; j += kWThreads) {
-        const float v = x[j];
-        int best = 0;
-        float bd = fabsf(v - c[0]);
-        for (int k = 1; k < K; ++k) {
-            const float d = fabsf(v - c[k]);
-            if (d < bd) {
-                bd = d;
-                best = k;
-            }
-        }
-        codes[i * d_out + j] = (uint8_t)best;
-    }
+    assign_codes(K, x, c, N, codes + i * d_out);
     if (tid < CMPQ_LUT_STRIDE) lut[i * CMPQ_LUT_STRIDE + tid] = tid < K ? c[tid] : 0.0f;
     if (sweeps != nullptr && tid == 0) atomicAdd(sweeps, (unsigned long long)(done + 1) * (unsigned long long)N * K);
 }
