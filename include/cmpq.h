@@ -164,7 +164,7 @@ cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, in
  *   update      c_k = (float)(sum of members in fp64 / count); an empty cluster keeps c_k
  * exactly lloyd_iters updates (1..CMPQ_MAX_LLOYD_ITERS; 0 is allowed and returns the start),
  * then a last assignment.  lut: [d_in][CMPQ_LUT_STRIDE] fp32, the first K entries valid, the
- * rest 0.  codes: [d_in][d_out] uint8.
+ * rest 0.  codes: [d_in][d_out] uint8, 8-byte aligned (else CMPQ_ERR_INVALID_ARG).
  * sens: NULL for the paper's unweighted K-means.  Otherwise [d_in][d_out] fp32 sensitivities s >= 0
  * (finite), one per weight: the update becomes the weighted mean  c_k = sum s x / sum s  over the
  * members (a cluster whose members' sensitivities sum to 0 keeps c_k); start and assignment are

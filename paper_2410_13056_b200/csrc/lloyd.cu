@@ -648,6 +648,7 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
     if (nnz < 0 || nnz > d_in * d_out || (nnz > 0 && (!rows || !cols))) return CMPQ_ERR_INVALID_ARG;
     if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
     if (!aligned_to(W, 2) || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;  // eight codes leave in one store
     if (sens && !aligned_to(sens, 4)) return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

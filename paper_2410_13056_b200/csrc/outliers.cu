@@ -410,7 +410,7 @@ extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, i
                                                  void* stream) {
     cmpq_status s = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
     if (s != CMPQ_OK) return s;
-    if (!lut || !codes || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
+    if (!lut || !codes || !aligned_to(lut, 4) || !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < protect_quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     Workspace wsp(ws, ws_bytes);

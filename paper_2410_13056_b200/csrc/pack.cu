@@ -115,6 +115,7 @@ pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ bits,
     const int64_t j0 = g * 32;
     if (j0 >= d_out) return;
     const int c = bits[row];
+    if (c < 2 || c > 4) return;  // not a width of the method: the layout gave this row no words
     const uint8_t* src = codes + row * d_out + j0;
     const int cnt = (int)min((int64_t)32, d_out - j0);
     uint32_t b[8];  // 32 code bytes, little endian

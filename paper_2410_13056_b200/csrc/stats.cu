@@ -9,6 +9,8 @@
 // order, so the result does not depend on scheduling.
 #include "common.cuh"
 
+#include <atomic>
+
 namespace cmpq {
 
 constexpr int kStatsThreads = 256;
@@ -19,9 +21,14 @@ constexpr int kMaxRowBlocks = 2048;  // upper bound used to size the work space
 constexpr int kCtasPerSm = 5;       // resident blocks per SM of the vector kernel (48 registers)
 
 int sm_count() {
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cached[kMaxDevices];  // zero-initialised: 0 = not asked yet
     int dev = 0, n = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    if (slot && (n = cached[dev].load(std::memory_order_relaxed)) > 0) return n;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (slot) cached[dev].store(n, std::memory_order_relaxed);
     return n;
 }
 

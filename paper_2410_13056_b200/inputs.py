@@ -152,3 +152,46 @@ CONFIGS = {
 
 def layer_seed(cfg: Config, layer_index: int) -> int:
     return cfg.seed + layer_index
+
+
+def stack_layers(cfg: Config) -> List[Tuple[int, int, Layer]]:
+    """Every layer of a multi-block workload in order: (block, index inside the block, layer)."""
+    return [(b, i, L) for b in range(cfg.repeat) for i, L in enumerate(cfg.layers)]
+
+
+def stack_layer_seed(cfg: Config, block: int, index: int) -> int:
+    """Seed of one layer's weights in a multi-block workload (distinct for every layer)."""
+    return cfg.seed + len(cfg.layers) * block + index
+
+
+class StackInputs:
+    """Inputs of a multi-block workload, layer by layer: every layer has its own seeded weights (drawn
+    when asked for, into one buffer per shape so that addresses stay fixed); the calibration activations
+    are drawn once per distinct input width and shared by the layers of that width (the statistic's cost
+    does not depend on the values, and a gigabyte per layer would only lengthen the preparation)."""
+
+    def __init__(self, cfg: Config, device="cuda"):
+        self.cfg, self.device = cfg, device
+        self.layers = stack_layers(cfg)
+        self._X, self._W = {}, {}
+
+    def shapes(self) -> List[Tuple[int, int]]:
+        return [(L.d_in, L.d_out) for _, _, L in self.layers]
+
+    def activations(self, d_in: int) -> torch.Tensor:
+        if d_in not in self._X:
+            self._X[d_in] = make_activations(self.cfg.n_tokens, d_in, self.cfg.dtype, self.cfg.seed + d_in,
+                                             device=self.device)
+        return self._X[d_in]
+
+    def weights(self, shape: Tuple[int, int]) -> torch.Tensor:
+        """The buffer that holds the weights of the layer of this shape drawn last."""
+        return self._W[shape]
+
+    def __call__(self, k: int):
+        b, i, L = self.layers[k]
+        W = make_weight(L.d_in, L.d_out, self.cfg.dtype, stack_layer_seed(self.cfg, b, i), device=self.device)
+        buf = self._W.setdefault((L.d_in, L.d_out), W)
+        if buf is not W:
+            buf.copy_(W)
+        return self.activations(L.d_in), buf

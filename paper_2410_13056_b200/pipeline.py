@@ -149,7 +149,7 @@ class LayerQuantizer:
              self.lut, self.codes, self.ws, inexact_rows=inexact, sweeps=sweeps)
 
     def run_graphed(self, X, W, avg_bits, lloyd_iters):
-        """The same pass replayed from a CUDA graph: the 26 launches of a pass are short enough for launch
+        """The same pass replayed from a CUDA graph: the launches of a pass are short enough for launch
         overhead to show, and nothing in the pass depends on values read back by the host.  The graph is
         captured on the first call for a given (X, W, budget, iterations) and replayed afterwards; X
         and W must keep their addresses (their contents may change).  Results as in run()."""
@@ -197,6 +197,67 @@ class LayerQuantizer:
             t.copy_(src[k], non_blocking=True)
         torch.cuda.current_stream().synchronize()
         return host_out
+
+
+class StackQuantizer:
+    """The pass over a list of independent linear layers (Section 3.2.1 of the paper quantizes layer by
+    layer, so a transformer stack is just many such layers): this rank's share of them, one after the
+    other on the current stream, with one LayerQuantizer (output buffers and scratch) per distinct shape.
+
+    shapes: (d_in, d_out) of every layer of the stack, in order.  With world > 1 the layers are dealt
+    round-robin to the ranks (sharding.layers_of_rank); nothing is exchanged between ranks.
+    quantizer_factory(d_in, d_out) builds the per-shape quantizer (default: LayerQuantizer on `device`)."""
+
+    def __init__(self, shapes, rank=0, world=1, device="cuda", quantizer_factory=None):
+        from . import sharding
+
+        self.shapes = [(int(d_in), int(d_out)) for d_in, d_out in shapes]
+        self.rank, self.world = int(rank), int(world)
+        self.mine = sharding.layers_of_rank(len(self.shapes), self.rank, self.world)
+        self._factory = quantizer_factory or (lambda d_in, d_out: LayerQuantizer(d_in, d_out, device=device))
+        self._quantizers = {}
+
+    def quantizer(self, k):
+        """The quantizer that serves layer k (shared by all layers of that shape)."""
+        shape = self.shapes[k]
+        if shape not in self._quantizers:
+            self._quantizers[shape] = self._factory(*shape)
+        return self._quantizers[shape]
+
+    def params(self):
+        """Weights in this rank's layers."""
+        return sum(self.shapes[k][0] * self.shapes[k][1] for k in self.mine)
+
+    def run(self, inputs_of, avg_bits, lloyd_iters, on_result=None, timed=False, graphed=False):
+        """inputs_of(k) -> (X [n][d_in], W [d_in][d_out]) for layer k of this rank (called right before
+        the layer's pass; preparing the inputs is the caller's work and is not timed).  on_result(k, result)
+        is called after layer k's pass has been enqueued; the result's buffers are reused by the next layer
+        of the same shape, so copy what is kept there (on the same stream).  timed: CUDA events around every
+        pass; the returned dict then holds "ms" (the sum over this rank's passes) and "ms_by_shape".
+        graphed: passes through LayerQuantizer.run_graphed (inputs_of must then return tensors at fixed
+        addresses per shape).  Returns {"layers", "params"[, "ms", "ms_by_shape"]}."""
+        pairs = []
+        for k in self.mine:
+            X, W = inputs_of(k)
+            q = self.quantizer(k)
+            if timed:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            r = (q.run_graphed if graphed else q.run)(X, W, avg_bits, lloyd_iters)
+            if timed:
+                e1.record()
+                pairs.append((k, e0, e1))
+            if on_result is not None:
+                on_result(k, r)
+        out = {"layers": len(self.mine), "params": self.params()}
+        if timed:
+            torch.cuda.current_stream().synchronize()
+            by_shape = {}
+            for k, e0, e1 in pairs:
+                by_shape.setdefault(self.shapes[k], []).append(e0.elapsed_time(e1))
+            out["ms"] = sum(sum(v) for v in by_shape.values())
+            out["ms_by_shape"] = {shape: sum(v) / len(v) for shape, v in by_shape.items()}
+        return out
 
 
 class QuantizedLinear:

@@ -1,14 +1,14 @@
 """Small, self-ending runs of single C-ABI calls, meant to be captured by a profiler.
 
-    python -m paper_2410_13056_b200.profile_cases lloyd --d-in 1184 --d-out 4096 --bits 3 --launches 3
-    python -m paper_2410_13056_b200.profile_cases stats --tokens 32768 --d-in 4096 --launches 3
-    python -m paper_2410_13056_b200.profile_cases pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
-    python -m paper_2410_13056_b200.profile_cases outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
-    python -m paper_2410_13056_b200.profile_cases matvec --d-in 8192 --d-out 28672 --budget 2.5 --launches 20
-    python -m paper_2410_13056_b200.profile_cases transpose --d-in 16384 --d-out 16384 --launches 10
-    python -m paper_2410_13056_b200.profile_cases sweep --config c3_mlp7b --layer 0 --launches 5
-    python -m paper_2410_13056_b200.profile_cases stack --config c4_stack7b --budget 3.0
-    python -m paper_2410_13056_b200.profile_cases layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
+    python profile_cases.py lloyd --d-in 1184 --d-out 4096 --bits 3 --launches 3
+    python profile_cases.py stats --tokens 32768 --d-in 4096 --launches 3
+    python profile_cases.py pack  --d-in 16384 --d-out 8192 --bits 3 --launches 3
+    python profile_cases.py outliers --d-in 1184 --d-out 4096 --bits 3 --launches 2
+    python profile_cases.py matvec --d-in 8192 --d-out 28672 --budget 2.5 --launches 20
+    python profile_cases.py transpose --d-in 16384 --d-out 16384 --launches 10
+    python profile_cases.py sweep --config c3_mlp7b --layer 0 --launches 5
+    python profile_cases.py stack --config c4_stack7b --budget 3.0
+    python profile_cases.py layer --config c3_mlp7b --layer 0 --budget 3.0 --launches 5
 
 `layer` runs the whole pass on one layer of a named workload and prints the time per C-ABI call.
 `stack` quantizes every layer of a multi-block workload (all 32 x 7 layers of the Llama-7B-shaped stack) and
@@ -17,15 +17,21 @@ prints the total device time of the passes; under torchrun the layers are dealt 
 Each case prints the mean CUDA-event time per call; every run holds well under 1 GB on the device.
 """
 import argparse
+import os
+import sys
 
 import torch
 
-from . import binding as B
-from . import inputs
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2410_13056_b200 import binding as B
+from paper_2410_13056_b200 import inputs
 
 
 def run_layer(a):
-    from .pipeline import LayerQuantizer
+    from paper_2410_13056_b200.pipeline import LayerQuantizer
 
     cfg = inputs.CONFIGS[a.config]
     L = cfg.layers[a.layer]
@@ -60,43 +66,32 @@ def run_layer(a):
 
 
 def run_stack(a):
-    """Every layer of the workload, each with its own seeded weights.  The calibration activations are
-    generated once per distinct input width and reused by the layers of that width (the statistic's cost
-    does not depend on the values, and regenerating a gigabyte per layer would only lengthen the untimed
-    part); weight generation is not timed, the passes are (CUDA events around each pass)."""
-    import os
-
-    from . import sharding
-    from .pipeline import LayerQuantizer
+    """Every layer of a multi-block workload through pipeline.StackQuantizer (weights seeded per layer,
+    activations per input width; only the passes are timed); under torchrun the layers are dealt to the ranks."""
+    from paper_2410_13056_b200 import sharding
+    from paper_2410_13056_b200.pipeline import StackQuantizer
 
     cfg = inputs.CONFIGS[a.config]
     rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", torch.cuda.current_device()))
-    layers = [(b, i, L) for b in range(cfg.repeat) for i, L in enumerate(cfg.layers)]
-    mine = [layers[k] for k in sharding.layers_of_rank(len(layers), rank, world)]
-    X, quant = {}, {}
-    for _, _, L in mine:
-        if L.d_in not in X:
-            X[L.d_in] = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, cfg.seed + L.d_in, device="cuda")
-        if (L.d_in, L.d_out) not in quant:
-            quant[(L.d_in, L.d_out)] = LayerQuantizer(L.d_in, L.d_out)
-    total_ms, params, inexact = 0.0, 0, 0
-    for n, (b, i, L) in enumerate(mine):
-        W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, cfg.seed + 7 * b + i, device="cuda")
-        q = quant[(L.d_in, L.d_out)]
-        if n < len(quant) * 2:  # first uses of a shape: one untimed pass (module and graph set-up)
-            q.run(X[L.d_in], W, a.budget, cfg.lloyd_iters)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        q.run(X[L.d_in], W, a.budget, cfg.lloyd_iters)
-        e1.record()
-        torch.cuda.synchronize()
-        total_ms += e0.elapsed_time(e1)
-        params += L.d_in * L.d_out
-        inexact += int(q.counters[0].item() & 0xffffffff)
-    slowest = sharding.max_over_ranks(total_ms, device="cuda")
+    src = inputs.StackInputs(cfg)
+    stack = StackQuantizer(src.shapes(), rank, world)
+    seen = set()
+    for k in stack.mine:  # one untimed pass per shape: module and buffer set-up
+        if stack.shapes[k] not in seen:
+            seen.add(stack.shapes[k])
+            X, W = src(k)
+            stack.quantizer(k).run(X, W, a.budget, cfg.lloyd_iters)
+    inexact = [0]
+
+    def on_result(k, r):
+        inexact[0] += int(r.inexact_rows.item())
+
+    out = stack.run(src, a.budget, cfg.lloyd_iters, on_result=on_result, timed=True)
+    slowest = sharding.max_over_ranks(out["ms"], device="cuda")
+    params = out["params"]
     if world > 1:
         t = torch.tensor([float(params)], dtype=torch.float64, device="cuda")
         dist.all_reduce(t)
@@ -105,13 +100,15 @@ def run_stack(a):
     if rank == 0:
         print("stack %s: %d layers (%d blocks x %d), %.3f G weights, avg %.2f bits, T=%d, %d rank(s): %.1f ms of "
               "passes on the slowest rank, %.0f Mparams/s; inexact rows on rank 0: %d"
-              % (a.config, len(layers), cfg.repeat, len(cfg.layers), params / 1e9, a.budget, cfg.lloyd_iters, world,
-                 slowest, params / slowest / 1e3, inexact))
+              % (a.config, len(src.layers), cfg.repeat, len(cfg.layers), params / 1e9, a.budget, cfg.lloyd_iters,
+                 world, slowest, params / slowest / 1e3, inexact[0]))
+        for shape, ms in out["ms_by_shape"].items():
+            print("   %d x %d: %.3f ms per pass" % (shape[0], shape[1], ms))
 
 
 def run_sweep(a):
     """All budgets of a workload on one layer: separate passes against run_budgets (statistic computed once)."""
-    from .pipeline import LayerQuantizer
+    from paper_2410_13056_b200.pipeline import LayerQuantizer
 
     cfg = inputs.CONFIGS[a.config]
     L = cfg.layers[a.layer]
@@ -141,7 +138,7 @@ def run_sweep(a):
 def run_matvec(a, dt):
     """The inference product on a random quantized layer (codes are random, so no quantization runs):
     widths split as the rank-form allocation splits them for the budget."""
-    from .pipeline import QuantizedLinear
+    from paper_2410_13056_b200.pipeline import QuantizedLinear
 
     d_in, d_out = a.d_in, a.d_out
     n2, n4 = B.cmpq_alloc_counts(d_in, a.budget)
@@ -213,7 +210,6 @@ def main():
                     help="assignment method of the K-means kernels")
     a = ap.parse_args()
     dt = inputs.BF16 if a.dtype == "bf16" else inputs.F16
-    import os
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS if a.assign == "all_pairs" else B.ASSIGN_ORDERED)
     if a.case == "layer":

@@ -92,12 +92,17 @@ def test_bad_arguments_are_refused_on_the_host(L):
     assert L.cmpq_quantize_layer(*q(nnz=3)) == INVALID                                     # list missing
     assert L.cmpq_quantize_layer(*q(d_out=0)) == INVALID
     assert L.cmpq_quantize_layer(*q(iters=2000)) == INVALID
+    # eight codes leave in one store: an offset view of a code buffer is refused here, never launched
+    qc = lambda codes: (ws, 0, 8, 16, 16, ws, None, None, 0, 5, None, ws, codes, None, None, ws, 1 << 30, None)
+    assert L.cmpq_quantize_layer(*qc(ctypes.c_void_p(ws.value + 1))) == INVALID
+    assert L.cmpq_quantize_layer(*qc(ctypes.c_void_p(ws.value + 4))) == INVALID
     # outlier protection and final fit in one call: the checks of both
     f = lambda n_act=1, n_q=3, nnz=19, lut=p, codes=p, wsb=1 << 30: (p, 0, 8, 16, 16, p, p, n_act, n_q, 5, p, p, p, nnz, lut, codes, None, None, ws, wsb, None)
     assert L.cmpq_protect_and_quantize(*f(nnz=18)) == INVALID
     assert L.cmpq_protect_and_quantize(*f(lut=None)) == INVALID
     assert L.cmpq_protect_and_quantize(*f(codes=None)) == INVALID
     assert L.cmpq_protect_and_quantize(*f(wsb=64)) == WORKSPACE
+    assert L.cmpq_protect_and_quantize(*f(codes=ctypes.c_void_p(ws.value + 4))) == INVALID   # misaligned codes
     # pack
     assert L.cmpq_pack(p, p, 8, 16, None, p, p, p, ws, 1 << 30, None) == INVALID
     assert L.cmpq_pack(p, p, 8, 16, p, p, p, p, ws, 8, None) == WORKSPACE

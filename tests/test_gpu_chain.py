@@ -9,26 +9,14 @@ from paper_2410_13056_b200 import binding as B
 from paper_2410_13056_b200 import inputs
 from paper_2410_13056_b200.pipeline import LayerQuantizer
 
+from gpu_util import (assert_whole_layer_equal, chain_with_gpu_statistic, check_layer_sampled,
+                      check_statistic_columns, result_arrays)
+
 pytestmark = pytest.mark.gpu
 
 
-def _np(r):
-    out = {k: getattr(r, k).cpu().numpy() for k in ("a", "bits", "rows", "cols", "lut", "codes", "row_off",
-                                                     "perm", "seg_rows")}
-    out["vals"] = r.vals.cpu().numpy().view(np.uint16)
-    out["packed"] = r.packed.cpu().numpy().view(np.uint32)
-    return out
-
-
-def _chain_with_gpu_statistic(Wu, dtype, a_gpu, b, n_act, n_q, T):
-    """The checker's steps 2..8 fed with the statistic the GPU produced (the statistic itself is
-    compared within tolerance; everything after it must then agree bit for bit)."""
-    bits, _ = oracle.allocate_bits(a_gpu, b)
-    rows, cols, vals = oracle.extract_outliers(Wu, dtype, a_gpu, bits, n_act, n_q, T)
-    lut, codes = oracle.quantize_layer(Wu, dtype, bits, rows, cols, T)
-    packed, row_off, perm, seg = oracle.pack(codes, bits)
-    return dict(bits=bits, rows=rows, cols=cols, vals=vals, lut=lut, codes=codes, packed=packed,
-                row_off=row_off, perm=perm, seg_rows=seg)
+_np = result_arrays
+_chain_with_gpu_statistic = chain_with_gpu_statistic
 
 
 @pytest.fixture(params=["ordered", "all_pairs"])
@@ -88,10 +76,10 @@ def test_midsize_layer_all_budgets(b):
     assert abs(g["bits"].mean() - b) <= 0.5 / d_in or b == 3.0
 
 
-def _sampled_parity(cfg_name, layer_index, b):
-    """One full-size layer through the quantizer in the launch configuration the benchmark uses; the
-    checker verifies sampled channels and properties that hold at any size instead of re-running
-    everything (a full single-threaded run would take minutes)."""
+def _sampled_parity(cfg_name, layer_index, budgets, stripe=None, graphed=False):
+    """One full-size layer through the quantizer in the launch configuration the benchmark uses, at every
+    budget given (the statistic is checked once); the checker verifies sampled channels and properties
+    that hold at any size instead of re-running everything (a full single-threaded run takes minutes)."""
     cfg = inputs.CONFIGS[cfg_name]
     L = cfg.layers[layer_index]
     T = cfg.lloyd_iters
@@ -100,87 +88,47 @@ def _sampled_parity(cfg_name, layer_index, b):
     W = inputs.make_weight(d_in, d_out, cfg.dtype, seed, device="cuda")
     X = inputs.make_activations(cfg.n_tokens, d_in, cfg.dtype, seed, device="cuda")
     q = LayerQuantizer(d_in, d_out)
-    r = q.run(X, W, b, T)
-    g = _np(r)
-    assert int(q.counters[0].item()) == 0
     assert (q.n_act, q.n_q) == oracle.default_counts(d_in, d_out)
-    # statistic: sampled columns against the checker (fp64, token order)
-    colsel = np.unique(np.array([0, 1, 7, 8, 255, 256, d_in // 2, d_in - 1] + list(np.argsort(g["a"])[-4:])))
-    Xs = X[:, torch.from_numpy(colsel).cuda()].contiguous()
-    a_ref = oracle.finalize_stats(oracle.collect_stats(inputs.as_u16(Xs), cfg.dtype))
-    np.testing.assert_allclose(g["a"][colsel], a_ref, rtol=1e-5)
-    del X, Xs
-    # allocation: exact, from the GPU statistic
-    bits_ref, order_ref = oracle.allocate_bits(g["a"], b)
-    assert np.array_equal(g["bits"], bits_ref)
-    n2, n4 = oracle.alloc_counts(d_in, b)
-    assert (g["bits"] == 2).sum() == n2 and (g["bits"] == 4).sum() == n4
-    # outlier list: structure and O_act rows
-    lin = g["rows"].astype(np.int64) * d_out + g["cols"]
-    assert np.all(np.diff(lin) > 0)
-    Wu = inputs.as_u16(W)
-    assert np.array_equal(g["vals"], Wu[g["rows"], g["cols"]])
-    per_row = np.bincount(g["rows"], minlength=d_in)
-    act_rows = np.sort(order_ref[d_in - q.n_act:])
-    assert np.array_equal(np.flatnonzero(per_row == d_out), act_rows)
-    assert per_row[per_row < d_out].sum() == q.n_q
-    # O_q: the provisional fit of sampled rows reproduces exactly the entries taken in those rows,
-    # and no error left behind in a sampled row exceeds the smallest error taken in any sampled row
-    is_act = np.zeros(d_in, bool)
-    is_act[act_rows] = True
-    sample = [i for i in (0, 1, 17, d_in // 8, d_in // 2, d_in - 1, int(np.argmax(per_row * ~is_act))) if not is_act[i]]
-    taken_min, left_max = np.inf, 0.0
-    for i in sample:
-        xi = W[i].float().cpu().numpy()
-        _, _, err = oracle.lloyd(xi, 1 << int(bits_ref[i]), T)
-        mask = np.zeros(d_out, bool)
-        mask[g["cols"][g["rows"] == i]] = True
-        if mask.any():
-            taken_min = min(taken_min, err[mask].min())
-            assert err[mask].min() >= err[~mask].max()
-        left_max = max(left_max, err[~mask].max())
-    assert left_max <= taken_min
-    # final fit: sampled channels (every width present, an O_act row, the row with most O_q entries)
-    sample2 = sample + [int(act_rows[0])] + [int(np.flatnonzero(bits_ref == c)[k]) for c in (2, 3, 4)
-                                              for k in (0, -1) if (bits_ref == c).any()]
-    for i in sample2:
-        xi = W[i].float().cpu().numpy()
-        xi[g["cols"][g["rows"] == i]] = 0
-        lut, code, _ = oracle.lloyd(xi, 1 << int(bits_ref[i]), T)
-        assert np.array_equal(code, g["codes"][i]), i
-        np.testing.assert_allclose(g["lut"][i], lut, rtol=1e-4)
-        assert np.array_equal(g["lut"][i].view(np.uint32), lut.view(np.uint32)), i
-    assert np.all(g["codes"] < (1 << g["bits"].astype(np.int64))[:, None])
-    # packing: full comparison against the checker's packer
-    packed, row_off, perm, seg = oracle.pack(g["codes"], g["bits"])
-    assert np.array_equal(g["packed"], packed) and np.array_equal(g["row_off"], row_off)
-    assert np.array_equal(g["perm"], perm) and np.array_equal(g["seg_rows"], seg)
-    return g, q
+    out = {}
+    for k, b in enumerate(budgets):
+        r = (q.run_graphed if graphed else q.run)(X, W, b, T)
+        g = _np(r)
+        assert int(q.counters[0].item()) == 0
+        if k == 0:
+            check_statistic_columns(X, g["a"], cfg.dtype, extra=list(np.argsort(g["a"])[-4:]))
+        check_layer_sampled(W, g, cfg.dtype, b, T, q.n_act, q.n_q, stripe=stripe)
+        out[b] = g
+    return out, q
 
 
 def test_llama_attention_shape_sampled_parity():
     """The benchmark's workload shape (4096 x 4096 bf16, 131072 tokens, 20 iterations) at its own 2.2-bit
-    budget and at the metric's 3.0 bits."""
-    g, q = _sampled_parity("c2_attn7b", 0, 2.2)
+    budget and at the metric's 3.0 bits, eager calls (the graph-replayed path is compared in full in
+    test_gpu_full_parity.py)."""
+    out, q = _sampled_parity("c2_attn7b", 0, [2.2, 3.0])
     assert (q.n_act, q.n_q, q.nnz) == (18, 8388, 82116)
-    assert (g["bits"] == 2).sum() == 3277 and g["packed"].nbytes == 4613632
-    g, q = _sampled_parity("c2_attn7b", 0, 3.0)
-    assert g["packed"].nbytes == 4096 * 4096 * 3 // 8
+    assert (out[2.2]["bits"] == 2).sum() == 3277 and out[2.2]["packed"].nbytes == 4613632
+    assert out[3.0]["packed"].nbytes == 4096 * 4096 * 3 // 8
 
 
-@pytest.mark.parametrize("layer_index,b", [(0, 2.5), (1, 3.5)])
-def test_llama_mlp_shapes_sampled_parity(layer_index, b):
-    """4096 x 11008 (up) and 11008 x 4096 (down) with 131072 calibration tokens."""
-    g, q = _sampled_parity("c3_mlp7b", layer_index, b)
+@pytest.mark.parametrize("layer_index,budgets", [(0, [2.0, 2.5, 3.5, 4.0]), (1, [2.0, 2.5, 3.0, 3.5, 4.0])])
+def test_llama_mlp_shapes_sampled_parity(layer_index, budgets):
+    """4096 x 11008 (up) and 11008 x 4096 (down) with 131072 calibration tokens, every budget of the sweep
+    (the up projection at 3.0 bits is compared in full in test_gpu_full_parity.py)."""
+    out, q = _sampled_parity("c3_mlp7b", layer_index, budgets)
     assert q.nnz == (220688 if layer_index == 0 else 223248)
+    for b, g in out.items():
+        assert g["packed"].nbytes == round(4096 * 11008 * b / 8)
 
 
 @pytest.mark.parametrize("layer_index", [0, 1])
-def test_llama70b_mlp_shapes_sampled_parity(layer_index):
-    """8192 x 28672 and 28672 x 8192 with 65536 calibration tokens at 2.5 bits."""
-    g, q = _sampled_parity("c5_mlp70b", layer_index, 2.5)
+def test_llama70b_mlp_shapes_striped_parity(layer_index):
+    """8192 x 28672 and 28672 x 8192 with 65536 calibration tokens at 2.5 bits: every sixteenth channel is
+    fitted by the checker (provisional and final fit), and the entries kept in those channels must be
+    exactly the ones their errors select."""
+    out, q = _sampled_parity("c5_mlp70b", layer_index, [2.5], stripe=(5, 16))
     assert q.nnz == (1149632 if layer_index == 0 else 1174208)
-    assert g["packed"].nbytes == 8192 * 28672 * 5 // 16
+    assert out[2.5]["packed"].nbytes == 8192 * 28672 * 5 // 16
 
 
 def test_graph_replay_gives_the_same_bytes_as_the_eager_pass():

@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2410_13056_b200 import binding as B
 from paper_2410_13056_b200 import inputs
 
@@ -33,11 +34,14 @@ def test_static_scratch_matches_workspace_version_on_two_calls_in_a_row():
     X1 = inputs.make_activations(6000, 4096, inputs.BF16, 41, device="cuda")
     got1, ref1 = _both(X1)
     np.testing.assert_allclose(np.sqrt(got1), np.sqrt(ref1), rtol=STAT_RTOL)
+    # and against the CPU checker's sums (fp64, token order), not only against the library's other entry
+    np.testing.assert_allclose(got1, oracle.collect_stats(inputs.as_u16(X1), inputs.BF16), rtol=STAT_RTOL)
     # second call right after it: another shape and dtype, small values, ragged width (scalar
     # path); anything the first call left in the array must not leak into this result
     X2 = (inputs.make_activations(777, 1001, inputs.F16, 42, device="cuda").float() * 1e-3).to(torch.float16)
     got2, ref2 = _both(X2)
     np.testing.assert_allclose(np.sqrt(got2), np.sqrt(ref2), rtol=STAT_RTOL)
+    np.testing.assert_allclose(got2, oracle.collect_stats(inputs.as_u16(X2), inputs.F16), rtol=STAT_RTOL)
     # and the first input again gives the first answer again, bit for bit
     got3, _ = _both(X1)
     assert np.array_equal(got3, got1)
