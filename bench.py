@@ -27,13 +27,27 @@ METRIC_BUDGET = 3.0          # the metric is quoted at an average of 3.0 bits
 SM_COUNT, FP32_LANES_PER_SM = 148, 128
 CPU_BASELINE_CHANNELS = 4096   # cpu_baseline leg: the whole layer (about 15 s on one core)
 REFERENCE_ARM_CHANNELS = 1024  # --impl reference: a quarter of the layer per step
-# dram__bytes_read.sum and dram__bytes_write.sum of stats_partial_vec_kernel from the ncu capture summarised
-# under profiles/ (32768 x 4096 bf16 activations: 268.44 MB algorithmic).  Reads grow with the rows, the
-# written fp64 partial sums do not.  None while no capture of the current kernel exists.
-STATS_DRAM_READ_PER_INPUT_BYTE = 268.45e6 / (32768 * 4096 * 2)
-STATS_DRAM_WRITE_BYTES = 3.97e6
-# the same for lloyd_table_kernel, per weight
-LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT = 9761536 / (1184 * 4096)
+MIN_TIMED_SECONDS = 1.0        # the timed region is repeated until it has lasted this long
+
+
+def _traffic_records():
+    """DRAM traffic per kernel from the ncu captures summarised under profiles/ (profiles/traffic.json).
+    A record is used only while the kernel still has the register count it was captured with."""
+    from paper_2410_13056_b200 import binding as B
+
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    out = {}
+    if not os.path.exists(path):
+        return out
+    for name, rec in json.load(open(path)).items():
+        if name.startswith("_"):
+            continue
+        try:
+            regs, _ = B.cmpq_kernel_resources(rec["kernel_id"])
+        except Exception:
+            regs = None
+        out[name] = dict(rec, current=(regs == rec["registers"]), registers_now=regs)
+    return out
 
 
 def _peaks():
@@ -152,6 +166,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stack", action="store_true", help="skip the leg that quantizes the whole 7B-shaped stack")
     args = ap.parse_args()
 
     from paper_2410_13056_b200 import inputs
@@ -194,30 +209,39 @@ def main():
     q = LayerQuantizer(layer.d_in, layer.d_out)
     params = layer.d_in * layer.d_out
 
-    def timed(budget, k, ev=None):
+    def timed(budget, k, ev=None, min_seconds=0.0):
         """k passes; without ev through the graph-replaying call, with ev eagerly with CUDA events
-        around every C-ABI call and every K-means kernel of the final fit."""
+        around every C-ABI call and every K-means kernel of the final fit.  The k-step region (barrier and
+        synchronisation on both sides, CUDA events, maximum over ranks) is repeated until the regions
+        together have lasted min_seconds; returns (median ms per step, ms per step of every repeat)."""
         step = (lambda i: q.run_graphed(X, W, budget, cfg.lloyd_iters)) if ev is None else \
                (lambda i: q.run(X, W, budget, cfg.lloyd_iters, events=ev[i]))
         for _ in range(warmup):
             q.run_graphed(X, W, budget, cfg.lloyd_iters) if ev is None else q.run(X, W, budget, cfg.lloyd_iters)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(k):
-            step(i)
-        e1.record()
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1)) / k
+        per_step, total = [], 0.0
+        while True:
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(k):
+                step(i)
+            e1.record()
+            barrier()
+            region_ms = max_over_ranks(e0.elapsed_time(e1))
+            per_step.append(region_ms / k)
+            total += region_ms
+            if total >= min_seconds * 1e3 or len(per_step) >= 1000:
+                break
+        return statistics.median(per_step), per_step
 
     # device-resident throughput at the metric's budget; then the same steps again with events around
     # every call and kernel (those cost a few per cent, so they are kept out of `value`)
     sampler = ClockSampler(_visible_index(local_rank))
     sampler.start()
-    ms = timed(METRIC_BUDGET, steps)
-    events = [dict() for _ in range(steps)]
-    ms_instrumented = timed(METRIC_BUDGET, steps, events)
+    ms, ms_repeats = timed(METRIC_BUDGET, steps, min_seconds=MIN_TIMED_SECONDS)
     clocks = sampler.stop()
+    events = [dict() for _ in range(steps)]
+    ms_instrumented, _ = timed(METRIC_BUDGET, steps, events)
     value = world * params / (ms * 1e-3) / 1e6
     per_call = {}
     for name in events[0]:
@@ -229,7 +253,7 @@ def main():
         "lloyd_iterate_kernel": statistics.mean(p[1].elapsed_time(p[2]) for p in phases),
         "lloyd_assign_kernel": statistics.mean(p[2].elapsed_time(p[3]) for p in phases),
     }
-    ms_22 = timed(cfg.budgets[0], max(3, steps // 2))
+    ms_22, _ = timed(cfg.budgets[0], max(3, steps // 2))
 
     # Roofline of the dominant kernel.  By time per step the largest kernel is the statistic's column
     # reduction (about a quarter of the pass; the K-means work is spread over five smaller kernels).  It has
@@ -245,7 +269,21 @@ def main():
 
     # The all-pairs formulation (every weight against every centroid in every iteration), timed on
     # the same layer after the timed region: 2 ops (subtract, compare/select) per evaluation it executes.
-    alu_peak_tflops = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    alu_peak_derived = SM_COUNT * FP32_LANES_PER_SM * sm_max_mhz * 1e6 / 1e12
+    # measured in this run: the library's arithmetic probe (subtract + compare/select on registers only,
+    # independent chains, every SM full), best of 5 launches of about 2 ms
+    sink = torch.empty(SM_COUNT * 16 * 256, dtype=torch.float32, device="cuda")
+    B.cmpq_alu_probe(64, SM_COUNT * 16, sink)
+    torch.cuda.synchronize()
+    probe_tflops = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        pairs = B.cmpq_alu_probe(2048, SM_COUNT * 16, sink)
+        e1.record()
+        torch.cuda.synchronize()
+        probe_tflops.append(2.0 * pairs / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    alu_peak_tflops = max(probe_tflops)
     q.run(X, W, METRIC_BUDGET, cfg.lloyd_iters)  # bits and outlier list of the metric's budget
     B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS)
     try:
@@ -273,10 +311,18 @@ def main():
     ap_tflops = 2.0 * ap_evals / (ap_ms * 1e-3) / 1e12
 
     stats_bytes = X.numel() * 2
+    # ncu traffic of the two kernels, scaled from the captured small case to this launch; null once the
+    # kernel has changed since its capture
+    traffic = _traffic_records()
+    rec = traffic.get("stats_partial_vec_kernel")
+    stats_traffic = (rec["dram_read_bytes"] / rec["captured_input_bytes"] * stats_bytes + rec["dram_write_bytes"]
+                     if rec and rec["current"] else None)
+    rec = traffic.get("lloyd_table_kernel")
+    table_traffic = ((rec["dram_read_bytes"] + rec["dram_write_bytes"]) / rec["captured_weights"] * params
+                     if rec and rec["current"] else None)
     roofline = {"bound": "hbm", "kernel": "stats_partial_vec_kernel (cmpq_collect_stats)", "achieved": stats_gbs,
                 "peak": hbm_peak, "unit": "GB/s", "frac": stats_gbs / hbm_peak, "peak_kind": peak_kind,
-                "traffic": (STATS_DRAM_READ_PER_INPUT_BYTE * stats_bytes + STATS_DRAM_WRITE_BYTES
-                            if STATS_DRAM_READ_PER_INPUT_BYTE else None),
+                "traffic": stats_traffic,
                 "note": "algorithmic bytes: every 16-bit activation read once (%d bytes per launch); the largest "
                         "kernel of the step by time" % stats_bytes,
                 "ms": stats_ms, "share_of_step": stats_ms / ms,
@@ -285,7 +331,7 @@ def main():
                     "lloyd_table": {"bound": "hbm", "kernel": "lloyd_table_kernel (final fit, separate calls)",
                                     "achieved": table_gbs, "peak": hbm_peak, "unit": "GB/s",
                                     "frac": table_gbs / hbm_peak, "peak_kind": peak_kind,
-                                    "traffic": LLOYD_TABLE_DRAM_BYTES_PER_WEIGHT * params,
+                                    "traffic": table_traffic,
                                     "note": "each 16-bit weight read once; bound by shared-memory histogram "
                                             "work, not by HBM"},
                     "pack": {"bound": "hbm", "achieved": pack_gbs, "peak": hbm_peak, "unit": "GB/s",
@@ -296,7 +342,10 @@ def main():
                         "bound": "alu", "kernel": "lloyd_kernel (CMPQ_ASSIGN_ALL_PAIRS, final fit)",
                         "achieved": ap_tflops, "peak": alu_peak_tflops, "unit": "TFLOP/s",
                         "frac": ap_tflops / alu_peak_tflops, "ms": ap_ms,
-                        "peak_kind": "148 SMs x 128 fp32 lanes x %.0f MHz, one op per lane per clock" % sm_max_mhz,
+                        "peak_kind": "measured in this run by cmpq_alu_probe (subtract + compare/select per "
+                                     "pair, registers only); derived 148 SMs x 128 lanes x %.0f MHz x 1 op = "
+                                     "%.1f" % (sm_max_mhz, alu_peak_derived),
+                        "peak_derived": alu_peak_derived, "frac_of_derived": ap_tflops / alu_peak_derived,
                         "note": "brute-force formulation, not on the default path: the ordered "
                                 "assignment reaches the same codes and centroids without this work"}}}
 
@@ -349,6 +398,38 @@ def main():
                       "shared-memory table look-ups bound it, not HBM"}
     roofline["other_kernels"]["matvec"] = matvec
 
+    # The metric's own workload: every layer of the 32-block 7B-shaped stack at avg 3.0 bits through the stack
+    # driver (own seeded weights per layer, 131072 calibration tokens per layer; with N ranks the layers are
+    # dealt round-robin, no collective on the data path).  One untimed pass per shape first; CUDA events
+    # around every pass; the job's time is the slowest rank's sum.
+    stack_leg = None
+    n_act_q = (q.n_act, q.n_q)
+    if not args.no_stack:
+        from paper_2410_13056_b200.pipeline import StackQuantizer
+        del X, W, Xh, Wh, flush
+        q = qlin = res = None
+        torch.cuda.empty_cache()
+        scfg = inputs.CONFIGS["c4_stack7b"]
+        src = inputs.StackInputs(scfg)
+        stack = StackQuantizer(src.shapes(), rank, world)
+        seen = set()
+        for k in stack.mine:
+            if stack.shapes[k] not in seen:
+                seen.add(stack.shapes[k])
+                Xs, Ws = src(k)
+                stack.quantizer(k).run(Xs, Ws, METRIC_BUDGET, scfg.lloyd_iters)
+        barrier()
+        out = stack.run(src, METRIC_BUDGET, scfg.lloyd_iters, timed=True)
+        barrier()
+        stack_ms = max_over_ranks(out["ms"])
+        total_params = sum(a * b for a, b in src.shapes())
+        stack_leg = {"workload": "c4_stack7b: 32 blocks x (4 x 4096x4096, 2 x 4096x11008, 1 x 11008x4096) bf16, "
+                                 "131072 tokens per layer, avg 3.0 bits, 20 Lloyd iterations",
+                     "layers": len(src.shapes()), "params": total_params, "ms_total": stack_ms,
+                     "value": total_params / (stack_ms * 1e-3) / 1e6, "unit": UNIT,
+                     "scaling": "strong (the 224 layers are split over the ranks)", "launch": "eager calls",
+                     "ms_per_pass_by_shape": {"%dx%d" % shape: v for shape, v in out["ms_by_shape"].items()}}
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, sec, sample = time_cpu_reference(cfg, layer, METRIC_BUDGET, 1, 0, CPU_BASELINE_CHANNELS)
@@ -358,7 +439,7 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms, "repeats": len(ms_repeats), "ms_per_step_repeats": ms_repeats, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": "c2_attn7b: W 4096x4096 bf16, X 131072x4096 bf16, 20 Lloyd iterations, "
                                    "avg 3.0 bits (the metric's budget); one layer per step per GPU",
@@ -367,12 +448,14 @@ def main():
                                  "kernel_ms come from eager passes that call cmpq_extract_outliers and "
                                  "cmpq_quantize_layer separately (same results, the final fit rebuilds its tables)",
                        "l2": "inputs larger than L2 (X is 1 GiB per step)",
-                       "n_act": q.n_act, "n_q": q.n_q},
+                       "timing": "the region of `steps` passes is repeated until it has lasted %.0f s in all; value and "
+                                 "ms_per_step are the median region" % MIN_TIMED_SECONDS,
+                       "n_act": n_act_q[0], "n_q": n_act_q[1]},
             "at_config_budget": {"avg_bits": cfg.budgets[0], "value": world * params / (ms_22 * 1e-3) / 1e6,
                                  "unit": UNIT, "ms_per_step": ms_22},
             "per_call_ms": per_call, "ms_per_step_with_events": ms_instrumented,
             "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_per_run(B.ASSIGN_ORDERED, fused=True) * steps,
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "stack": stack_leg, "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
     if dist is not None:

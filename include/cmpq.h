@@ -272,6 +272,24 @@ cmpq_status cmpq_outliers_by_column(const int32_t* rows, const int32_t* cols, co
 cmpq_status cmpq_transpose16(const void* src, int64_t rows, int64_t cols, int64_t ld_src, void* dst,
                              int64_t ld_dst, void* stream);
 
+/* ---- measurement aids (no counterpart in the paper; nothing here is on the quantization path) ------
+ * cmpq_alu_probe enqueues a kernel that performs, on register operands only and in eight independent
+ * chains per thread, the arithmetic of a brute-force nearest-centroid assignment (Section 3): per
+ * (value, centroid) pair one fp32 subtract and one compare/select (min of magnitudes).  `blocks` blocks of
+ * 256 threads run `rounds` rounds of 8 x 16 pairs each; *evaluations (host, optional) receives the number
+ * of pairs the launch evaluates, so 2 * evaluations / (event-timed duration) is this GPU's ceiling, at the
+ * clocks of the moment, for the two-operation mix an all-pairs assignment needs.  sink: device scratch of
+ * blocks * 256 floats (never written in practice).  1 <= rounds <= 2^24, 1 <= blocks <= 2^20. */
+cmpq_status cmpq_alu_probe(int rounds, int blocks, float* sink, unsigned long long* evaluations, void* stream);
+
+/* Registers per thread and static shared memory of a kernel of this library, as compiled (host call, no
+ * GPU work).  Lets a stored profile of a kernel be recognised as stale after the kernel has changed. */
+typedef enum {
+    CMPQ_KERNEL_STATS_PARTIAL_VEC_BF16 = 0,   /* column reduction of cmpq_collect_stats, bf16, l2 */
+    CMPQ_KERNEL_LLOYD_TABLE_BF16_4096 = 1     /* value-table kernel, bf16, 2048 < d_out <= 4096 */
+} cmpq_kernel;
+cmpq_status cmpq_kernel_resources(cmpq_kernel k, int* registers, int* static_smem_bytes);
+
 /* ---- host helpers (pure functions, no GPU work) ----------------------------------------------- */
 size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out);
 /* Algorithm 1 in rank form: how many channels get 2 and 4 bits. */

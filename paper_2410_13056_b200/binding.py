@@ -26,6 +26,7 @@ EXPORTS = (
     "cmpq_set_lloyd_assignment", "cmpq_get_lloyd_assignment", "cmpq_lloyd_phase_events",
     "cmpq_protect_and_quantize", "cmpq_matvec", "cmpq_outliers_by_column",
     "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
+    "cmpq_alu_probe", "cmpq_kernel_resources",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -88,6 +89,10 @@ def lib():
         L.cmpq_get_lloyd_assignment.restype = ci
         L.cmpq_lloyd_phase_events.argtypes = [vp, vp, vp, vp]
         L.cmpq_lloyd_phase_events.restype = ci
+        L.cmpq_alu_probe.argtypes = [ci, ci, vp, ctypes.POINTER(ctypes.c_ulonglong), vp]
+        L.cmpq_alu_probe.restype = ci
+        L.cmpq_kernel_resources.argtypes = [ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.cmpq_kernel_resources.restype = ci
         L.cmpq_status_string.argtypes = [ci]
         L.cmpq_status_string.restype = ctypes.c_char_p
         _lib = L
@@ -144,6 +149,23 @@ def cmpq_lloyd_phase_events(events):
         ev.record()  # torch creates the CUDA event lazily: make sure the handle exists
         handles.append(ctypes.c_void_p(ev.cuda_event))
     _check(lib().cmpq_lloyd_phase_events(*handles), "cmpq_lloyd_phase_events")
+
+
+KERNEL_STATS_PARTIAL_VEC_BF16, KERNEL_LLOYD_TABLE_BF16_4096 = 0, 1
+
+
+def cmpq_alu_probe(rounds, blocks, sink):
+    """Enqueues the arithmetic-throughput probe; returns the (value, centroid) pairs it evaluates."""
+    n = ctypes.c_ulonglong()
+    _check(lib().cmpq_alu_probe(int(rounds), int(blocks), _ptr(sink), ctypes.byref(n), _stream()), "cmpq_alu_probe")
+    return int(n.value)
+
+
+def cmpq_kernel_resources(kernel):
+    """(registers per thread, static shared memory bytes) of one of the library's kernels as compiled."""
+    regs, smem = ctypes.c_int(), ctypes.c_int()
+    _check(lib().cmpq_kernel_resources(int(kernel), ctypes.byref(regs), ctypes.byref(smem)), "cmpq_kernel_resources")
+    return regs.value, smem.value
 
 
 def cmpq_alloc_counts(d_in, avg_bits):

@@ -1105,6 +1105,10 @@ static cmpq_status launch_table_dt(const LloydArgs& args, const Tables& t, cudaS
     return launch_table<DT, 32, 1024, 1>(args, t, threads_for(32), st);
 }
 
+const void* lloyd_table_kernel_address() {
+    return reinterpret_cast<const void*>(&lloyd_table_kernel<CMPQ_BF16, 16, 256, 4>);
+}
+
 // tables_ready: the value tables of every row to be fitted are in place already (skip the table kernel)
 template <int DT>
 static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, bool tables_ready, cudaStream_t st) {

@@ -224,6 +224,10 @@ cmpq_status launch_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens,
     return launch_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, partial, row_blocks, st);
 }
 
+const void* stats_kernel_address() {
+    return reinterpret_cast<const void*>(&stats_partial_vec_kernel<CMPQ_BF16, CMPQ_NORM_L2>);
+}
+
 int64_t stats_row_blocks(int64_t d_in, int64_t n_tokens) {
     int sms = sm_count();
     if (sms <= 0) return 0;
