@@ -203,6 +203,32 @@ cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in
                                       int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
                                       size_t ws_bytes, void* stream);
 
+/* ---- budget sweeps (the paper's limitations paragraph: a new memory budget means quantizing again) --
+ * The value tables of a layer's channels depend on the weights alone, and a channel's provisional
+ * K-means fit on its width and the iteration count alone.  A sweep over several budgets on the same
+ * weights therefore keeps both in a caller-owned cache:
+ *   cmpq_sweep_begin   counts the values of every channel of W once (no statistic needed) and marks the
+ *                      cache empty of fits; lloyd_iters is the count every later call will use.
+ *   cmpq_sweep_budget  is cmpq_protect_and_quantize -- same arguments, same outputs bit for bit -- except
+ *                      that the provisional fit reads the cached tables, copies the fits already made for
+ *                      a (channel, width) pair and adds the new ones to the cache.  W, d_in, d_out, ldw
+ *                      and lloyd_iters must be those of cmpq_sweep_begin (a different lloyd_iters is
+ *                      detected on the device and simply bypasses the kept fits); a, bits, n_act and n_q
+ *                      may change from call to call.
+ * cache: cmpq_sweep_cache_bytes(d_in, d_out) bytes of device memory, 256-byte aligned, untouched by the
+ * caller between the calls (else CMPQ_ERR_WORKSPACE).  Calls on one cache must be ordered (one stream).
+ * With CMPQ_ASSIGN_ALL_PAIRS selected the cache is ignored.
+ * ws of cmpq_sweep_budget: cmpq_workspace_bytes(CMPQ_OP_PROTECT_AND_QUANTIZE, d_in, d_out). */
+size_t cmpq_sweep_cache_bytes(int64_t d_in, int64_t d_out);
+cmpq_status cmpq_sweep_begin(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                             int lloyd_iters, void* cache, size_t cache_bytes, void* stream);
+cmpq_status cmpq_sweep_budget(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                              const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                              int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
+                              int64_t nnz_out, float* lut, uint8_t* codes, int32_t* inexact_rows,
+                              unsigned long long* sweeps, void* cache, size_t cache_bytes, void* ws,
+                              size_t ws_bytes, void* stream);
+
 /* Process-wide choice of the assignment method used by cmpq_extract_outliers and
  * cmpq_quantize_layer from the next call on (host state, no GPU work; thread-safe).
  * CMPQ_ERR_INVALID_ARG for an unknown value. */

@@ -27,6 +27,7 @@ EXPORTS = (
     "cmpq_protect_and_quantize", "cmpq_matvec", "cmpq_outliers_by_column",
     "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
     "cmpq_alu_probe", "cmpq_kernel_resources",
+    "cmpq_sweep_cache_bytes", "cmpq_sweep_begin", "cmpq_sweep_budget",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -89,6 +90,13 @@ def lib():
         L.cmpq_get_lloyd_assignment.restype = ci
         L.cmpq_lloyd_phase_events.argtypes = [vp, vp, vp, vp]
         L.cmpq_lloyd_phase_events.restype = ci
+        L.cmpq_sweep_cache_bytes.argtypes = [i64, i64]
+        L.cmpq_sweep_cache_bytes.restype = sz
+        L.cmpq_sweep_begin.argtypes = [vp, ci, i64, i64, i64, ci, vp, sz, vp]
+        L.cmpq_sweep_begin.restype = ci
+        L.cmpq_sweep_budget.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
+                                        vp, vp, vp, vp, sz, vp, sz, vp]
+        L.cmpq_sweep_budget.restype = ci
         L.cmpq_alu_probe.argtypes = [ci, ci, vp, ctypes.POINTER(ctypes.c_ulonglong), vp]
         L.cmpq_alu_probe.restype = ci
         L.cmpq_kernel_resources.argtypes = [ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
@@ -235,6 +243,28 @@ def cmpq_protect_and_quantize(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, v
                                            n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz,
                                            _ptr(lut), _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(ws),
                                            ws.numel(), _stream()), "cmpq_protect_and_quantize")
+
+
+def cmpq_sweep_cache_bytes(d_in, d_out):
+    return int(lib().cmpq_sweep_cache_bytes(d_in, d_out))
+
+
+def cmpq_sweep_begin(W, lloyd_iters, cache):
+    """Counts the values of every channel of W into `cache` (uint8 tensor of cmpq_sweep_cache_bytes bytes)."""
+    d_in, d_out = W.shape
+    _check(lib().cmpq_sweep_begin(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), lloyd_iters, _ptr(cache),
+                                  cache.numel(), _stream()), "cmpq_sweep_begin")
+
+
+def cmpq_sweep_budget(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, cache, ws,
+                      inexact_rows=None, sweeps=None):
+    """cmpq_protect_and_quantize with the value tables and provisional fits kept in `cache`."""
+    d_in, d_out = W.shape
+    nnz = n_act * d_out + n_q
+    _check(lib().cmpq_sweep_budget(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
+                                   n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz, _ptr(lut),
+                                   _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(cache), cache.numel(),
+                                   _ptr(ws), ws.numel(), _stream()), "cmpq_sweep_budget")
 
 
 def cmpq_pack(codes, bits, packed, row_off, perm, seg_rows, ws):

@@ -22,6 +22,11 @@ struct LloydArgs {
     uint8_t* codes;          // [d_in][d_out] or NULL
     int32_t* inexact_rows;   // optional counter
     unsigned long long* sweeps;  // optional counter of distance evaluations
+    // ordered formulation only: fits kept across calls on the same weights (budget sweeps).  fit_cache is
+    // the block lloyd_fit_cache_bytes() describes; a channel whose fit for its width is already there
+    // copies it instead of iterating, every other channel stores its fit there.
+    void* fit_cache;         // or NULL
+    bool tables_ready;       // the value tables of every row to be fitted are in place already
 };
 
 // The process-wide choice made by cmpq_set_lloyd_assignment.
@@ -33,6 +38,13 @@ cmpq_status launch_lloyd(const LloydArgs& args, cmpq_dtype dt, cudaStream_t st);
 // Ordered formulation: value table per channel, warp-per-channel iterations, streaming last
 // assignment.  `tables` is device scratch of lloyd_tables_bytes(d_in, d_out) bytes, 256-byte aligned.
 size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out);
+// Value tables of every row of args.W alone (no fit); args.skip_row / row_ptr are honoured.
+cmpq_status launch_lloyd_tables(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,
+                                cudaStream_t st);
+// Provisional fits per (width, channel) kept between calls: [header 256 B][valid 3 x d_in bytes]
+// [centroids 3 x d_in x 16 floats][thresholds 3 x d_in x 16 floats]; cleared by launch_fit_cache_clear.
+size_t lloyd_fit_cache_bytes(int64_t d_in);
+cmpq_status launch_fit_cache_clear(void* fit_cache, int64_t d_in, int iters, cudaStream_t st);
 // Final fit whose value tables are derived from those a provisional ordered fit of the same weights left
 // in prov_tables (args.row_ptr / args.cols: the positions removed since; skip_rebuild: d_in bytes of scratch).
 cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, void* prov_tables, void* tables,

@@ -325,8 +325,48 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
 // ------------------------------------------------------------------------------------------------
 // iterations: one warp per channel
 
+// fits kept between calls (see lloyd.cuh): slot (bits - 2) * d_in + row
+struct FitCacheHeader {
+    int iters;  // the iteration count the cached fits were made with
+};
+struct FitCache {
+    FitCacheHeader* hdr;  // NULL: no cache
+    uint8_t* valid;
+    float* lut;
+    float* thr;
+};
+
+static FitCache carve_fit_cache(void* p, int64_t d_in) {
+    FitCache c{};
+    if (!p) return c;
+    Workspace w(p, ~(size_t)0);
+    c.hdr = w.take<FitCacheHeader>(1);
+    c.valid = w.take<uint8_t>(3 * (size_t)d_in);
+    c.lut = w.take<float>(3 * (size_t)d_in * CMPQ_LUT_STRIDE);
+    c.thr = w.take<float>(3 * (size_t)d_in * CMPQ_LUT_STRIDE);
+    return c;
+}
+
+size_t lloyd_fit_cache_bytes(int64_t d_in) {
+    return 256 + round_up(3 * (size_t)d_in, 256) + 2 * round_up(3 * (size_t)d_in * CMPQ_LUT_STRIDE * sizeof(float), 256);
+}
+
+__global__ void fit_cache_clear_kernel(FitCache c, int64_t n, int iters) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) c.valid[i] = 0;
+    if (i == 0) c.hdr->iters = iters;
+}
+
+cmpq_status launch_fit_cache_clear(void* fit_cache, int64_t d_in, int iters, cudaStream_t st) {
+    const FitCache c = carve_fit_cache(fit_cache, d_in);
+    const int64_t n = 3 * d_in;
+    fit_cache_clear_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(c, n, iters);
+    return launch_status();
+}
+
 struct IterArgs {
     Tables t;
+    FitCache fc;
     const uint8_t* bits;
     const uint8_t* skip_row;
     int64_t d_in, d_out;
@@ -559,9 +599,31 @@ lloyd_iterate_kernel(const IterArgs a) {
     if (row >= a.d_in) return;
     if (a.skip_row && a.skip_row[row]) return;
     const int bits = a.bits[row];
+    const int lane = threadIdx.x & 31;
+    // a fit of this channel at this width kept from an earlier call on the same weights: copy it
+    const bool cached_ok = a.fc.hdr && a.fc.hdr->iters == a.iters;
+    const int64_t slot = (int64_t)(bits == 2 ? 0 : (bits == 3 ? 1 : 2)) * a.d_in + row;
+    if (cached_ok && a.fc.valid[slot]) {
+        if (lane < CMPQ_LUT_STRIDE) {
+            a.lut[row * CMPQ_LUT_STRIDE + lane] = a.fc.lut[slot * CMPQ_LUT_STRIDE + lane];
+            a.t.thr[row * CMPQ_LUT_STRIDE + lane] = a.fc.thr[slot * CMPQ_LUT_STRIDE + lane];
+        }
+        return;
+    }
     if (bits == 2) iterate_channel<DT, 4>(a, row, warp_smem);
     else if (bits == 3) iterate_channel<DT, 8>(a, row, warp_smem);
     else iterate_channel<DT, 16>(a, row, warp_smem);
+    if (cached_ok) {  // lane l wrote entry l of both rows above and reads its own writes back
+        if (lane < CMPQ_LUT_STRIDE) {
+            a.fc.lut[slot * CMPQ_LUT_STRIDE + lane] = a.lut[row * CMPQ_LUT_STRIDE + lane];
+            a.fc.thr[slot * CMPQ_LUT_STRIDE + lane] = a.t.thr[row * CMPQ_LUT_STRIDE + lane];
+        }
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence();
+            a.fc.valid[slot] = 1;
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1112,6 +1174,7 @@ const void* lloyd_table_kernel_address() {
 // tables_ready: the value tables of every row to be fitted are in place already (skip the table kernel)
 template <int DT>
 static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, bool tables_ready, cudaStream_t st) {
+    tables_ready = tables_ready || args.tables_ready;
     if (args.err && args.codes) return CMPQ_ERR_INTERNAL;  // the assign kernel writes one or the other
     cudaEvent_t ev[4];
     take_phase_events(ev);
@@ -1124,6 +1187,7 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
 
     IterArgs ia{};
     ia.t = t;
+    ia.fc = carve_fit_cache(args.fit_cache, args.d_in);
     ia.bits = args.bits;
     ia.skip_row = args.skip_row;
     ia.d_in = args.d_in;
@@ -1150,6 +1214,13 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
     s = launch_status();
     if (ev[3]) cudaEventRecord(ev[3], st);
     return s;
+}
+
+cmpq_status launch_lloyd_tables(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,
+                                cudaStream_t st) {
+    if (!tables || tables_bytes < lloyd_tables_bytes(args.d_in, args.d_out)) return CMPQ_ERR_WORKSPACE;
+    const Tables t = tables_at(tables, tables_bytes, args.d_in, args.d_out);
+    return dt == CMPQ_F16 ? launch_table_dt<CMPQ_F16>(args, t, st) : launch_table_dt<CMPQ_BF16>(args, t, st);
 }
 
 cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tables, size_t tables_bytes,

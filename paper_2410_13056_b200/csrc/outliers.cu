@@ -262,7 +262,8 @@ size_t outliers_ws_bytes(int64_t d_in, int64_t d_out) {
 
 cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw, const float* a,
                          const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
-                         int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st);
+                         int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st,
+                         void* fit_cache = nullptr, bool tables_ready = false);
 static cmpq_status check_extract_args(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
                                       const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
                                       int lloyd_iters, const int32_t* rows, const int32_t* cols,
@@ -295,7 +296,8 @@ namespace cmpq {
 
 cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw, const float* a,
                          const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
-                         int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st) {
+                         int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st,
+                         void* fit_cache, bool tables_ready) {
     const unsigned row_blocks = (unsigned)((d_in + 255) / 256);
 
     const bool all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
@@ -316,6 +318,8 @@ cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_o
         // all pairs: one fp32 error per weight is written; ordered: the fit alone, errors are then
         // taken from the value tables
         la.err = all_pairs ? o.err : nullptr;
+        la.fit_cache = fit_cache;
+        la.tables_ready = tables_ready;
         s = all_pairs ? launch_lloyd(la, dt, st) : launch_lloyd_ordered(la, dt, o.tables, tables_bytes, st);
         if (s != CMPQ_OK) return s;
     }
@@ -401,21 +405,49 @@ size_t protect_quantize_ws_bytes(int64_t d_in, int64_t d_out) {
 
 }  // namespace cmpq
 
-extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
-                                                 int64_t ldw, const float* a, const uint8_t* bits,
-                                                 int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
-                                                 int32_t* cols, uint16_t* vals, int64_t nnz_out, float* lut,
-                                                 uint8_t* codes, int32_t* inexact_rows,
-                                                 unsigned long long* sweeps, void* ws, size_t ws_bytes,
-                                                 void* stream) {
+namespace cmpq {
+
+// Sweep cache: [value tables of all channels][fits kept per (width, channel)]
+struct SweepCache {
+    char* tables;
+    char* fits;
+};
+
+static SweepCache carve_sweep(void* cache, int64_t d_in, int64_t d_out) {
+    Workspace w(cache, ~(size_t)0);
+    SweepCache c;
+    c.tables = w.take<char>(lloyd_tables_bytes(d_in, d_out));
+    c.fits = w.take<char>(lloyd_fit_cache_bytes(d_in));
+    return c;
+}
+
+static size_t sweep_cache_bytes(int64_t d_in, int64_t d_out) {
+    return round_up(lloyd_tables_bytes(d_in, d_out), 256) + round_up(lloyd_fit_cache_bytes(d_in), 256);
+}
+
+// Outlier protection and final fit; with a sweep cache the provisional fit takes its value tables (and the
+// fits already made) from there.
+static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                         const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                         int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
+                                         int64_t nnz_out, float* lut, uint8_t* codes, int32_t* inexact_rows,
+                                         unsigned long long* sweeps, void* ws, size_t ws_bytes, void* cache,
+                                         cudaStream_t st) {
     cmpq_status s = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
     if (s != CMPQ_OK) return s;
     if (!lut || !codes || !aligned_to(lut, 4) || !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < protect_quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     Workspace wsp(ws, ws_bytes);
-    const FusedWs f = carve_fused(wsp, d_in, d_out);
-    s = extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, f.o, st);
+    FusedWs f = carve_fused(wsp, d_in, d_out);
+    const bool ordered = lloyd_assignment() != CMPQ_ASSIGN_ALL_PAIRS;
+    void* fit_cache = nullptr;
+    if (cache && ordered) {  // the provisional fit reads the cache's tables instead of building its own
+        const SweepCache c = carve_sweep(cache, d_in, d_out);
+        f.o.tables = c.tables;
+        fit_cache = c.fits;
+    }
+    s = extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, f.o, st,
+                     fit_cache, fit_cache != nullptr);
     if (s != CMPQ_OK) return s;
     s = launch_row_ptr(rows, nnz_out, d_in, f.row_ptr, st);
     if (s != CMPQ_OK) return s;
@@ -431,9 +463,59 @@ extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, i
     la.inexact_rows = inexact_rows;
     la.sweeps = sweeps;
     const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
-    if (lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS) return launch_lloyd(la, dt, st);
-    // the provisional fit ran (and left its tables) only when entries had to be selected
-    if (n_q > 0) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, f.skip_rebuild, st);
+    if (!ordered) return launch_lloyd(la, dt, st);
+    // the provisional fit ran (and left its tables) only when entries had to be selected; a sweep cache
+    // holds the tables of all channels in any case
+    if (n_q > 0 || fit_cache) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, f.skip_rebuild, st);
     return launch_lloyd_ordered(la, dt, f.tables, tables_bytes, st);
 }
 
+}  // namespace cmpq
+
+extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                                 int64_t ldw, const float* a, const uint8_t* bits,
+                                                 int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
+                                                 int32_t* cols, uint16_t* vals, int64_t nnz_out, float* lut,
+                                                 uint8_t* codes, int32_t* inexact_rows,
+                                                 unsigned long long* sweeps, void* ws, size_t ws_bytes,
+                                                 void* stream) {
+    return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
+                                 lut, codes, inexact_rows, sweeps, ws, ws_bytes, nullptr,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t cmpq_sweep_cache_bytes(int64_t d_in, int64_t d_out) {
+    if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+    return sweep_cache_bytes(d_in, d_out);
+}
+
+extern "C" cmpq_status cmpq_sweep_begin(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                        int lloyd_iters, void* cache, size_t cache_bytes, void* stream) {
+    if (!W || (dt != CMPQ_F16 && dt != CMPQ_BF16) || !aligned_to(W, 2)) return CMPQ_ERR_INVALID_ARG;
+    if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT || ldw < d_out) return CMPQ_ERR_INVALID_ARG;
+    if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
+    if (!cache || !aligned_to(cache, 256) || cache_bytes < sweep_cache_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const SweepCache c = carve_sweep(cache, d_in, d_out);
+    LloydArgs la{};
+    la.W = static_cast<const uint16_t*>(W);
+    la.d_in = d_in; la.d_out = d_out; la.ldw = ldw;
+    cmpq_status s = launch_lloyd_tables(la, dt, c.tables, lloyd_tables_bytes(d_in, d_out), st);
+    if (s != CMPQ_OK) return s;
+    return launch_fit_cache_clear(c.fits, d_in, lloyd_iters, st);
+}
+
+extern "C" cmpq_status cmpq_sweep_budget(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                         const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                         int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
+                                         int64_t nnz_out, float* lut, uint8_t* codes, int32_t* inexact_rows,
+                                         unsigned long long* sweeps, void* cache, size_t cache_bytes, void* ws,
+                                         size_t ws_bytes, void* stream) {
+    if (!cache || !aligned_to(cache, 256)) return CMPQ_ERR_WORKSPACE;
+    if (d_in >= 1 && d_in <= CMPQ_MAX_D_IN && d_out >= 1 && d_out <= CMPQ_MAX_D_OUT &&
+        cache_bytes < sweep_cache_bytes(d_in, d_out))
+        return CMPQ_ERR_WORKSPACE;
+    return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
+                                 lut, codes, inexact_rows, sweeps, ws, ws_bytes, cache,
+                                 static_cast<cudaStream_t>(stream));
+}

@@ -79,23 +79,34 @@ class LayerQuantizer:
         w = lambda c: (self.d_out * c + 31) // 32
         return n2 * w(2) + n3 * w(3) + n4 * w(4)
 
-    def run_budgets(self, X, W, budgets, lloyd_iters, on_result=None):
+    def run_budgets(self, X, W, budgets, lloyd_iters, on_result=None, share_fits=True):
         """The pass for several average budgets on the same layer (the paper's budget sweeps: any new
-        constraint means quantizing again).  The activation statistic does not depend on the budget, so it
-        is computed once and every budget re-runs only Algorithm 1, outlier protection, the K-means and the
-        packing; each budget's outputs are exactly those of a separate run().  The output buffers are
-        reused, so on_result(budget, result) is called after each budget's work has been enqueued (copy what
-        you need there, on the same stream).  Returns the last result."""
+        constraint means quantizing again).  Three things do not depend on the budget and are computed once:
+        the activation statistic, the value tables of the channels (cmpq_sweep_begin) and the provisional
+        fit of a channel at a given width, which is kept the first time a budget needs it
+        (cmpq_sweep_budget).  Every budget re-runs Algorithm 1, the remaining provisional fits, the
+        selection, the final fit and the packing; each budget's outputs are exactly those of a separate
+        run().  share_fits=False shares the statistic only.  The output buffers are reused, so
+        on_result(budget, result) is called after each budget's work has been enqueued (copy what you need
+        there, on the same stream).  Returns the last result."""
         result = None
+        cache = None
+        if share_fits and B.cmpq_get_lloyd_assignment() == B.ASSIGN_ORDERED:
+            if getattr(self, "_sweep_cache", None) is None:
+                self._sweep_cache = torch.empty(B.cmpq_sweep_cache_bytes(self.d_in, self.d_out), dtype=torch.uint8,
+                                                device=self.device)
+            cache = self._sweep_cache
+            B.cmpq_sweep_begin(W, lloyd_iters, cache)
         for k, b in enumerate(budgets):
-            result = self.run(X, W, b, lloyd_iters, reuse_statistic=k > 0)
+            result = self.run(X, W, b, lloyd_iters, reuse_statistic=k > 0, sweep_cache=cache)
             if on_result is not None:
                 on_result(b, result)
         return result
 
-    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None, reuse_statistic=False):
+    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None, reuse_statistic=False, sweep_cache=None):
         """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
         reuse_statistic: keep the statistic `a` of the previous run on the same X (see run_budgets).
+        sweep_cache: a cache prepared by cmpq_sweep_begin for W (see run_budgets).
         fused (default: True unless events are asked for): outlier protection and final fit through
         cmpq_protect_and_quantize, which derives the final fit's value tables from the provisional
         fit's; otherwise cmpq_extract_outliers and cmpq_quantize_layer one after the other (same
@@ -125,7 +136,11 @@ class LayerQuantizer:
             call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
         call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
              self.ws)
-        if fused:
+        if sweep_cache is not None:
+            call("cmpq_sweep_budget", B.cmpq_sweep_budget, W, self.a, self.bits, self.n_act, self.n_q, lloyd_iters,
+                 self.rows, self.cols, self.vals, self.lut, self.codes, sweep_cache, self.ws,
+                 inexact_rows=inexact, sweeps=sweeps)
+        elif fused:
             call("cmpq_protect_and_quantize", B.cmpq_protect_and_quantize, W, self.a, self.bits, self.n_act,
                  self.n_q, lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.ws,
                  inexact_rows=inexact, sweeps=sweeps)

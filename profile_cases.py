@@ -130,9 +130,11 @@ def run_sweep(a):
         return e0.elapsed_time(e1) / a.launches
 
     separate = timed(lambda: [q.run(X, W, b, cfg.lloyd_iters) for b in budgets])
+    stat_only = timed(lambda: q.run_budgets(X, W, budgets, cfg.lloyd_iters, share_fits=False))
     shared = timed(lambda: q.run_budgets(X, W, budgets, cfg.lloyd_iters))
     print("sweep %s[%d] d_in=%d d_out=%d, budgets %s: %.3f ms as separate passes, %.3f ms with the statistic "
-          "computed once" % (a.config, a.layer, L.d_in, L.d_out, budgets, separate, shared))
+          "computed once, %.3f ms with the value tables and provisional fits kept as well"
+          % (a.config, a.layer, L.d_in, L.d_out, budgets, separate, stat_only, shared))
 
 
 def run_matvec(a, dt):

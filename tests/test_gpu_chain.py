@@ -148,17 +148,44 @@ def test_graph_replay_gives_the_same_bytes_as_the_eager_pass():
     assert not np.array_equal(eager["codes"], replay["codes"])
 
 
-def test_budget_sweep_shares_the_statistic():
-    """run_budgets computes the statistic once; every budget's outputs equal those of a separate pass."""
-    d_in, d_out, n, T = 192, 640, 1024, 6
+@pytest.mark.parametrize("d_in,d_out,n,T,budgets", [
+    (192, 640, 1024, 6, [2.0, 2.5, 3.0, 3.5, 4.0]),
+    (300, 2048, 512, 9, [3.5, 2.5, 3.5, 2.0, 3.0, 2.5]),      # budgets revisited: every fit comes from the cache
+    (64, 6000, 256, 4, [4.0, 3.0, 2.2]),
+])
+def test_budget_sweep_shares_statistic_tables_and_fits(d_in, d_out, n, T, budgets, assignment):
+    """run_budgets computes the statistic and the value tables once and keeps the provisional fits per
+    (channel, width); every budget's outputs equal those of a separate pass bit for bit, and those of the
+    checker fed the same statistic."""
     W = inputs.make_weight(d_in, d_out, inputs.BF16, 61, device="cuda")
     X = inputs.make_activations(n, d_in, inputs.BF16, 61, device="cuda")
-    budgets = [2.0, 2.5, 3.0, 3.5, 4.0]
     q = LayerQuantizer(d_in, d_out)
-    got = {}
-    q.run_budgets(X, W, budgets, T, on_result=lambda b, r: got.__setitem__(b, {k: v.copy() for k, v in _np(r).items()}))
+    got = []
+    q.run_budgets(X, W, budgets, T, on_result=lambda b, r: got.append({k: v.copy() for k, v in _np(r).items()}))
     q2 = LayerQuantizer(d_in, d_out)
-    for b in budgets:
+    Wu = inputs.as_u16(W)
+    for b, g in zip(budgets, got):
         sep = _np(q2.run(X, W, b, T))
         for k in sep:
-            assert np.array_equal(got[b][k], sep[k]), (b, k)
+            assert np.array_equal(g[k], sep[k]), (b, k)
+        assert_whole_layer_equal(g, _chain_with_gpu_statistic(Wu, inputs.BF16, g["a"], b, q.n_act, q.n_q, T))
+    # a sweep after the weights changed starts from a fresh cache (cmpq_sweep_begin): no stale fit is reused
+    W2 = inputs.make_weight(d_in, d_out, inputs.BF16, 62, device="cuda")
+    got2 = []
+    q.run_budgets(X, W2, budgets[:2], T, on_result=lambda b, r: got2.append({k: v.copy() for k, v in _np(r).items()}))
+    for b, g in zip(budgets[:2], got2):
+        sep = _np(q2.run(X, W2, b, T))
+        for k in sep:
+            assert np.array_equal(g[k], sep[k]), (b, k)
+
+
+def test_sweep_cache_with_another_iteration_count_is_bypassed_not_trusted():
+    d_in, d_out, n = 96, 1024, 512
+    W = inputs.make_weight(d_in, d_out, inputs.BF16, 63, device="cuda")
+    X = inputs.make_activations(n, d_in, inputs.BF16, 63, device="cuda")
+    q = LayerQuantizer(d_in, d_out)
+    q.run_budgets(X, W, [3.0], 3)                       # leaves fits made with 3 iterations in the cache
+    g = _np(q.run(X, W, 3.0, 8, reuse_statistic=True, sweep_cache=q._sweep_cache))
+    sep = _np(LayerQuantizer(d_in, d_out).run(X, W, 3.0, 8))
+    for k in sep:
+        assert np.array_equal(g[k], sep[k]), k
