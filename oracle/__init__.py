@@ -44,6 +44,8 @@ def lib():
         _lib.oracle_packed_words.restype = ctypes.c_int64
         _lib.oracle_metadata_bits_per_weight.restype = ctypes.c_double
         _lib.oracle_recon_error.restype = ctypes.c_double
+        _lib.oracle_float_to_half.restype = ctypes.c_uint16
+        _lib.oracle_float_to_half.argtypes = [ctypes.c_float]
     return _lib
 
 
@@ -221,6 +223,49 @@ def metadata_bits_per_weight(bits, d_out, tag_bits=4, lut_bits=16):
     bits = _c(bits, np.uint8)
     return float(lib().oracle_metadata_bits_per_weight(_p(bits), _i64(bits.shape[0]), _i64(d_out),
                                                        int(tag_bits), int(lut_bits)))
+
+
+def float_to_half(values):
+    """float32 -> binary16 bit patterns, round to nearest even (element by element through the C routine)."""
+    v = _c(values, np.float32).reshape(-1)
+    f = lib().oracle_float_to_half
+    return np.array([f(ctypes.c_float(float(x))) for x in v], np.uint16).reshape(np.shape(values))
+
+
+LUT_U4_BYTES = 12
+
+
+def lut_to_f16(lut, bits):
+    """Tables rounded to FP16 (Section 5.1): uint16 [d_in][16], entries beyond K are 0."""
+    lut = _c(lut, np.float32)
+    bits = _c(bits, np.uint8)
+    out = np.empty((bits.shape[0], 16), np.uint16)
+    lib().oracle_lut_to_f16(_p(lut), _p(bits), _i64(bits.shape[0]), _p(out))
+    return out
+
+
+def lut_from_f16(lut16):
+    lut16 = _c(lut16, np.uint16)
+    out = np.empty(lut16.shape, np.float32)
+    lib().oracle_lut_from_f16(_p(lut16), _i64(lut16.shape[0]), _p(out))
+    return out
+
+
+def lut_to_u4(lut, bits):
+    """Tables in 4 bits per centroid (Section 5.1 variant): uint8 [d_in][12] = 8 code bytes + FP16 lo, hi."""
+    lut = _c(lut, np.float32)
+    bits = _c(bits, np.uint8)
+    out = np.empty((bits.shape[0], LUT_U4_BYTES), np.uint8)
+    lib().oracle_lut_to_u4(_p(lut), _p(bits), _i64(bits.shape[0]), _p(out))
+    return out
+
+
+def lut_from_u4(stored, bits):
+    stored = _c(stored, np.uint8)
+    bits = _c(bits, np.uint8)
+    out = np.empty((bits.shape[0], 16), np.float32)
+    lib().oracle_lut_from_u4(_p(stored), _p(bits), _i64(bits.shape[0]), _p(out))
+    return out
 
 
 def recon_error(X_u16, W_u16, dtype, lut, codes, rows, cols, vals, t_step=1):

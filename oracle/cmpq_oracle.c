@@ -27,7 +27,9 @@
  * the reconstruction error of the same layer; for the l1 / l_inf statistics:
  * numpy's vector norms, closed forms, chunking and the norm inequalities; for
  * the weighted update: constant weights change nothing, every non-empty
- * centroid is its members' weighted mean.
+ * centroid is its members' weighted mean; for the stored table formats: numpy's
+ * float16 conversion on every binade and rounding case, the grid end points, the
+ * half-step error bound and a hand-worked channel.
  * Parity unpinned: none of the paper's perplexity tables can pin the
  * reconstruction error (no model weights exist here); oracle_recon_error is
  * pinned only against a dense float64 numpy evaluation of the same definition.
@@ -73,7 +75,7 @@ float oracle_widen(uint16_t h, int dtype) {
 }
 
 /* ---------------------------------------------------------------------------
- * Step 1.  Activation statistic (Section 3.2.1: "the per-channel L2-norm of X").
+ * Step 1.  Activation statistic (Section 3.2.1: the L2 norm of every column of X).
  *   sumsq_j += sum_t X[t,j]^2   in token order, fp64
  *   a_j      = (float) sqrt(sumsq_j)
  * The caller zeroes sumsq before the first chunk of tokens.
@@ -179,7 +181,7 @@ int oracle_allocate_bits(const float* a, int64_t d_in, double avg_bits, int mode
     if (!(avg_bits >= 2.0 && avg_bits <= 4.0) || d_in < 1) return 1;
     int32_t* order = (int32_t*)malloc((size_t)d_in * sizeof(int32_t));
     rank_channels(a, d_in, order);
-    for (int64_t i = 0; i < d_in; ++i) bits[i] = 3; /* c <- 3 * 1 */
+    for (int64_t i = 0; i < d_in; ++i) bits[i] = 3; /* every channel starts at 3 bits */
     if (mode == 0) {
         int64_t n2, n4;
         oracle_alloc_counts(d_in, avg_bits, &n2, &n4);
@@ -214,9 +216,9 @@ void oracle_default_counts(int64_t d_in, int64_t d_out, int64_t* n_act, int64_t*
 }
 
 /* ---------------------------------------------------------------------------
- * Channel-wise K-means (Section 3.2.1: "for each channel W_{i,:} ... we apply a
- * K-means clustering algorithm, where K is determined by the precision", K = 8
- * for 3 bits; quantizer of Section 3: Q(x_i) = argmin_j |x_i - q_j|).
+ * Channel-wise K-means (Section 3.2.1: every channel W_{i,:} is clustered on its
+ * own with K = 2^bits centroids, e.g. K = 8 at 3 bits; quantizer of Section 3:
+ * a value is replaced by the centroid nearest to it).
  *
  * The paper fixes neither the start, the iteration count, the handling of empty
  * clusters nor the rounding.  Reading taken:
@@ -450,8 +452,125 @@ double oracle_metadata_bits_per_weight(const uint8_t* bits, int64_t d_in, int64_
 }
 
 /* ---------------------------------------------------------------------------
- * Step 9.  Reconstruction and output error (Section 3.2.2: "W_q + O is used as
- * model weights"; Appendix, justification of the allocation: dY = X (W - W^)).
+ * Stored formats of the look-up tables (Section 5.1, memory usage: the tables are
+ * kept in FP16, 16 bits per centroid, and a variant keeps them in 4 bits).
+ *
+ * FP16: every centroid is rounded to the nearest binary16 value, ties to even
+ * (values beyond the binary16 range become infinities).
+ *
+ * 4 bit: the paper prints only the accounting, (1*4 + 8*4)/4096 bits per weight.
+ * Reading taken: the uniform quantizer of Section 3 with N = 4 applied to the K
+ * centroids of one channel.  lo and hi are the smallest and largest centroid of
+ * the channel, each rounded to FP16 (they are stored with the codes: 32 more bits
+ * per channel than the paper's accounting counts);  D = (hi - lo) / 15;
+ * code_k = clamp(round((c_k - lo) / D), 0, 15) with round-half-to-even; D == 0
+ * gives code 0.  Decoding: lo + code * D.  Every step is one fp32 operation
+ * (subtract, divide, round, multiply, add), nothing fused.
+ * Layout of a channel: 8 bytes of codes (code 2b in the low, code 2b+1 in the high
+ * nibble of byte b; codes at k >= K are 0), then lo and hi as little-endian
+ * binary16 patterns: 12 bytes.
+ * ------------------------------------------------------------------------- */
+static uint32_t float_to_bits(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return u;
+}
+
+/* float -> binary16, round to nearest, ties to even */
+static uint16_t float_to_half(float f) {
+    uint32_t u = float_to_bits(f);
+    uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    uint32_t mag = u & 0x7fffffffu;
+    if (mag > 0x7f800000u) return (uint16_t)(sign | 0x7e00u);            /* NaN */
+    if (mag == 0x7f800000u) return (uint16_t)(sign | 0x7c00u);           /* infinity */
+    double v = fabs((double)f);
+    if (v == 0.0) return sign;
+    /* position on the binary16 grid: subnormal spacing 2^-24 below 2^-14, else 2^(e-10) */
+    int e;
+    (void)frexp(v, &e);              /* v = m * 2^e, 0.5 <= m < 1, so v in [2^(e-1), 2^e) */
+    int ex = e - 1;                  /* floor(log2 v) */
+    if (ex < -14) ex = -14;
+    double ulp = ldexp(1.0, ex - 10);
+    double q = v / ulp;              /* exact: a power-of-two scaling */
+    double r = floor(q);
+    double frac = q - r;
+    if (frac > 0.5 || (frac == 0.5 && fmod(r, 2.0) == 1.0)) r += 1.0;
+    /* r in [0, 2048]: 0..1023 subnormal (ex == -14 and v < 2^-14), 1024..2047 normal, 2048 = next binade */
+    uint32_t n = (uint32_t)r;
+    uint32_t h;
+    if (ex == -14 && n < 1024u) {
+        h = n;                                           /* subnormal or zero */
+    } else {
+        int be = ex + 15;                                /* biased exponent */
+        if (n == 2048u) { n = 1024u; be += 1; }
+        if (be >= 31) return (uint16_t)(sign | 0x7c00u); /* overflow */
+        h = ((uint32_t)be << 10) | (n - 1024u);
+    }
+    return (uint16_t)(sign | h);
+}
+
+uint16_t oracle_float_to_half(float f) { return float_to_half(f); }
+
+void oracle_lut_to_f16(const float* lut, const uint8_t* bits, int64_t d_in, uint16_t* out) {
+    for (int64_t i = 0; i < d_in; ++i) {
+        int K = 1 << bits[i];
+        for (int k = 0; k < 16; ++k) out[i * 16 + k] = k < K ? float_to_half(lut[i * 16 + k]) : 0;
+    }
+}
+
+void oracle_lut_from_f16(const uint16_t* in, int64_t d_in, float* lut) {
+    for (int64_t i = 0; i < d_in * 16; ++i) lut[i] = half_to_float(in[i]);
+}
+
+void oracle_lut_to_u4(const float* lut, const uint8_t* bits, int64_t d_in, uint8_t* out) {
+    for (int64_t i = 0; i < d_in; ++i) {
+        const float* c = lut + i * 16;
+        int K = 1 << bits[i];
+        float lo = c[0], hi = c[0];
+        for (int k = 1; k < K; ++k) {
+            if (c[k] < lo) lo = c[k];
+            if (c[k] > hi) hi = c[k];
+        }
+        uint16_t lo16 = float_to_half(lo), hi16 = float_to_half(hi);
+        float flo = half_to_float(lo16), fhi = half_to_float(hi16);
+        float span = fhi - flo;
+        float D = span / 15.0f;
+        uint8_t* o = out + i * 12;
+        memset(o, 0, 8);
+        for (int k = 0; k < K; ++k) {
+            int code = 0;
+            if (D > 0.0f) {
+                float t = c[k] - flo;
+                float r = nearbyintf(t / D);          /* default rounding mode: half to even */
+                code = r < 0.0f ? 0 : (r > 15.0f ? 15 : (int)r);
+            }
+            o[k >> 1] |= (uint8_t)(code << (4 * (k & 1)));
+        }
+        o[8] = (uint8_t)(lo16 & 0xff); o[9] = (uint8_t)(lo16 >> 8);
+        o[10] = (uint8_t)(hi16 & 0xff); o[11] = (uint8_t)(hi16 >> 8);
+    }
+}
+
+void oracle_lut_from_u4(const uint8_t* in, const uint8_t* bits, int64_t d_in, float* lut) {
+    for (int64_t i = 0; i < d_in; ++i) {
+        const uint8_t* o = in + i * 12;
+        int K = 1 << bits[i];
+        float flo = half_to_float((uint16_t)(o[8] | (o[9] << 8)));
+        float fhi = half_to_float((uint16_t)(o[10] | (o[11] << 8)));
+        float span = fhi - flo;
+        float D = span / 15.0f;
+        for (int k = 0; k < 16; ++k) {
+            int code = (o[k >> 1] >> (4 * (k & 1))) & 15;
+            float step = (float)code * D;
+            lut[i * 16 + k] = k < K ? flo + step : 0.0f;
+        }
+    }
+}
+
+/* ---------------------------------------------------------------------------
+ * Step 9.  Reconstruction and output error (Section 3.2.2: inference uses the
+ * quantized weights plus the kept outliers; Appendix, justification of the
+ * allocation: the output changes by X (W - W^)).
  *   What_{ij} = lut_i[code_{ij}] + O_{ij},   E = || X (W - What) ||_F   in fp64.
  * t_step > 1 evaluates every t_step-th token only (a sample of the rows of X).
  * ------------------------------------------------------------------------- */
