@@ -289,6 +289,43 @@ cmpq_status cmpq_outliers_by_column(const int32_t* rows, const int32_t* cols, co
                                     int64_t nnz, int64_t d_out, int64_t* col_ptr, int32_t* c_rows,
                                     uint16_t* c_vals, void* ws, size_t ws_bytes, void* stream);
 
+/* The same product with the tables in their stored FP16 format (Section 5.1: 16 bits per centroid):
+ * lut16 is [d_in][16] binary16 patterns as written by cmpq_store_lut(CMPQ_LUT_F16), widened exactly
+ * when read; everything else as cmpq_matvec.  (4-bit tables are expanded with cmpq_load_lut first.) */
+cmpq_status cmpq_matvec_f16lut(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
+                               const int64_t* seg_rows, const uint16_t* lut16, int64_t d_in, int64_t d_out,
+                               const void* x, cmpq_dtype dt, const int64_t* col_ptr, const int32_t* c_rows,
+                               const uint16_t* c_vals, float* y, void* y16, void* ws, size_t ws_bytes,
+                               void* stream);
+
+/* ---- stored formats of the look-up tables (Section 5.1, memory usage) ----------------------------
+ * The final fit returns fp32 centroids.  The paper stores them in FP16 (one 4-bit width tag and K
+ * 16-bit centroids per channel: (4 + 8*16)/4096 = 0.03 bit per weight at 3 bits and 4096 weights per
+ * channel) and reports a variant with 4 bits per centroid ((4 + 8*4)/4096 < 0.01).
+ *   CMPQ_LUT_F16  uint16 [d_in][16]: every centroid rounded to the nearest binary16 value, ties to even
+ *                 (centroids beyond +-65504 become infinities); entries at k >= K are 0.
+ *   CMPQ_LUT_U4   12 bytes per channel.  The paper gives only the accounting; the reading taken is its own
+ *                 uniform quantizer (Section 3, N = 4) over the K centroids of the channel: lo / hi = the
+ *                 smallest / largest centroid, each rounded to binary16; D = (hi - lo)/15;
+ *                 code_k = clamp(round_half_even((c_k - lo)/D), 0, 15), 0 when D == 0; decoded centroid
+ *                 lo + code_k * D; every step one fp32 operation.  Bytes 0..7: code 2b in the low and code
+ *                 2b+1 in the high nibble of byte b (0 at k >= K); bytes 8..11: lo, hi as little-endian
+ *                 binary16.  The two grid ends cost 32 bits per channel more than the paper's accounting.
+ * cmpq_store_lut: lut [d_in][16] fp32 (16-byte aligned) -> stored (cmpq_lut_bytes(fmt, d_in) bytes, 4-byte
+ * aligned).  cmpq_load_lut: the inverse, fp32 tables that cmpq_matvec reads.  CMPQ_LUT_F32 is refused by
+ * both (nothing to convert).  cmpq_table_bits_per_weight (host, bits_host is a HOST array): the paper's
+ * accounting, (4 + K * bits per centroid [+ 32 for the 4-bit format's grid ends]) / d_out averaged over
+ * the channels. */
+typedef enum { CMPQ_LUT_F32 = 0, CMPQ_LUT_F16 = 1, CMPQ_LUT_U4 = 2 } cmpq_lut_format;
+#define CMPQ_LUT_U4_BYTES 12
+size_t cmpq_lut_bytes(cmpq_lut_format fmt, int64_t d_in);
+cmpq_status cmpq_store_lut(const float* lut, const uint8_t* bits, int64_t d_in, cmpq_lut_format fmt, void* stored,
+                           void* stream);
+cmpq_status cmpq_load_lut(const void* stored, cmpq_lut_format fmt, const uint8_t* bits, int64_t d_in, float* lut,
+                          void* stream);
+double cmpq_table_bits_per_weight(const uint8_t* bits_host, int64_t d_in, int64_t d_out, cmpq_lut_format fmt,
+                                  int count_grid_ends);
+
 /* ---- layout conversion (Section 3.2.1: W in R^{d_in x d_out}, a channel is the row W_{i,:}) ----
  * Frameworks store a linear layer output-major, [d_out][d_in]; every call above takes the paper's
  * input-channel-major layout.  dst[c*ld_dst + r] = src[r*ld_src + c] for a [rows][cols] source of

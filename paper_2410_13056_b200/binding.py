@@ -28,6 +28,7 @@ EXPORTS = (
     "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
     "cmpq_alu_probe", "cmpq_kernel_resources",
     "cmpq_sweep_cache_bytes", "cmpq_sweep_begin", "cmpq_sweep_budget",
+    "cmpq_matvec_f16lut", "cmpq_lut_bytes", "cmpq_store_lut", "cmpq_load_lut", "cmpq_table_bits_per_weight",
 )
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcmpq.so")
@@ -97,6 +98,16 @@ def lib():
         L.cmpq_sweep_budget.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
                                         vp, vp, vp, vp, sz, vp, sz, vp]
         L.cmpq_sweep_budget.restype = ci
+        L.cmpq_matvec_f16lut.argtypes = L.cmpq_matvec.argtypes
+        L.cmpq_matvec_f16lut.restype = ci
+        L.cmpq_lut_bytes.argtypes = [ci, i64]
+        L.cmpq_lut_bytes.restype = sz
+        L.cmpq_store_lut.argtypes = [vp, vp, i64, ci, vp, vp]
+        L.cmpq_store_lut.restype = ci
+        L.cmpq_load_lut.argtypes = [vp, ci, vp, i64, vp, vp]
+        L.cmpq_load_lut.restype = ci
+        L.cmpq_table_bits_per_weight.argtypes = [vp, i64, i64, ci, ci]
+        L.cmpq_table_bits_per_weight.restype = dbl
         L.cmpq_alu_probe.argtypes = [ci, ci, vp, ctypes.POINTER(ctypes.c_ulonglong), vp]
         L.cmpq_alu_probe.restype = ci
         L.cmpq_kernel_resources.argtypes = [ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
@@ -290,6 +301,40 @@ def cmpq_matvec(packed, row_off, perm, seg_rows, lut, x, col_ptr, c_rows, c_vals
     _check(lib().cmpq_matvec(_ptr(packed), _ptr(row_off), _ptr(perm), _ptr(seg_rows), _ptr(lut), d_in, d_out,
                              _ptr(x), dtype_code(x), _ptr(col_ptr), _ptr(c_rows), _ptr(c_vals), _ptr(y),
                              _ptr(y16), _ptr(ws), ws.numel(), _stream()), "cmpq_matvec")
+
+
+LUT_F32, LUT_F16, LUT_U4 = 0, 1, 2
+LUT_U4_BYTES = 12
+
+
+def cmpq_lut_bytes(fmt, d_in):
+    return int(lib().cmpq_lut_bytes(int(fmt), d_in))
+
+
+def cmpq_store_lut(lut, bits, fmt, stored):
+    """lut (float32 [d_in][16]) -> stored: int16 [d_in][16] (LUT_F16) or uint8 [d_in][12] (LUT_U4)."""
+    _check(lib().cmpq_store_lut(_ptr(lut), _ptr(bits), lut.shape[0], int(fmt), _ptr(stored), _stream()),
+           "cmpq_store_lut")
+
+
+def cmpq_load_lut(stored, fmt, bits, lut):
+    _check(lib().cmpq_load_lut(_ptr(stored), int(fmt), _ptr(bits), lut.shape[0], _ptr(lut), _stream()),
+           "cmpq_load_lut")
+
+
+def cmpq_table_bits_per_weight(bits_host, d_out, fmt, count_grid_ends=False):
+    """bits_host: a CPU uint8 tensor.  The table and width-tag overhead in bits per weight."""
+    b = bits_host.contiguous()
+    return float(lib().cmpq_table_bits_per_weight(ctypes.c_void_p(b.data_ptr()), b.numel(), d_out, int(fmt),
+                                                  1 if count_grid_ends else 0))
+
+
+def cmpq_matvec_f16lut(packed, row_off, perm, seg_rows, lut16, x, col_ptr, c_rows, c_vals, y, y16, ws):
+    """cmpq_matvec reading the tables in their stored FP16 format (int16 [d_in][16])."""
+    d_in, d_out = x.numel(), y.numel()
+    _check(lib().cmpq_matvec_f16lut(_ptr(packed), _ptr(row_off), _ptr(perm), _ptr(seg_rows), _ptr(lut16), d_in,
+                                    d_out, _ptr(x), dtype_code(x), _ptr(col_ptr), _ptr(c_rows), _ptr(c_vals),
+                                    _ptr(y), _ptr(y16), _ptr(ws), ws.numel(), _stream()), "cmpq_matvec_f16lut")
 
 
 def cmpq_collect_stats_norm(X, norm, acc, ws):

@@ -7,7 +7,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libcmpq.so")
-SOURCES = ["api.cu", "stats.cu", "stats_static.cu", "alloc.cu", "lloyd.cu", "lloyd_weighted.cu", "lloyd_hist.cu", "outliers.cu", "pack.cu", "matvec.cu", "transpose.cu", "probe.cu"]
+SOURCES = ["api.cu", "stats.cu", "stats_static.cu", "alloc.cu", "lloyd.cu", "lloyd_weighted.cu", "lloyd_hist.cu", "outliers.cu", "pack.cu", "matvec.cu", "transpose.cu", "probe.cu", "lut_store.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--fmad=false", "--cudart", "static", "-I", INCLUDE, "-I", CSRC]
 

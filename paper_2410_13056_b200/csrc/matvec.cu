@@ -250,14 +250,24 @@ __device__ __forceinline__ MvIds load_ids(const int32_t* __restrict__ perm, int6
     return ids;
 }
 
-__device__ __forceinline__ MvRaw load_raw(const MvIds& ids, const float* __restrict__ lut,
-                                          const uint16_t* __restrict__ x) {
+// The tables of a layer as the kernel reads them: fp32 as the final fit wrote them, or rounded to FP16
+// (the stored format of Section 5.1), widened on the fly.
+struct MvLut {
+    const void* p;
+    int is_f16;
+    __device__ __forceinline__ float at(int64_t idx) const {
+        return is_f16 ? __half2float(__ushort_as_half(static_cast<const uint16_t*>(p)[idx]))
+                      : static_cast<const float*>(p)[idx];
+    }
+};
+
+__device__ __forceinline__ MvRaw load_raw(const MvIds& ids, const MvLut& lut, const uint16_t* __restrict__ x) {
     const int lane = threadIdx.x & 31;
     MvRaw raw;
 #pragma unroll
     for (int q = 0; q < kMvRowsPerWarp / 2; ++q) {
         raw.x[q] = ids.i[q] >= 0 ? x[ids.i[q]] : (uint16_t)0;
-        raw.l[q] = ids.i[q] >= 0 ? lut[(int64_t)ids.i[q] * CMPQ_LUT_STRIDE + (lane & 15)] : 0.0f;
+        raw.l[q] = ids.i[q] >= 0 ? lut.at((int64_t)ids.i[q] * CMPQ_LUT_STRIDE + (lane & 15)) : 0.0f;
     }
     return raw;
 }
@@ -274,7 +284,7 @@ static_assert(kMvTableRegion >= kMvWarps * kMvPad * 4, "the reduction staging re
 template <int C, int DT>
 __device__ __forceinline__ void matvec_warp(const uint32_t* __restrict__ packed, int64_t off0, int64_t r0,
                                             int64_t words_per_row, const int32_t* __restrict__ perm,
-                                            const float* __restrict__ lut, const uint16_t* __restrict__ x,
+                                            const MvLut& lut, const uint16_t* __restrict__ x,
                                             int64_t r_first, int64_t r_end, int64_t group, int valid_words,
                                             float* values, float* tables, uint32_t stage_addr, float (&acc)[32]) {
     const int lane = threadIdx.x & 31;
@@ -328,7 +338,7 @@ template <int DT>
 __global__ void __launch_bounds__(kMvThreads, CMPQ_MV_MIN_BLOCKS)
 matvec_partial_kernel(const uint32_t* __restrict__ packed, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ perm, const int64_t* __restrict__ seg_rows,
-                      const float* __restrict__ lut, const uint16_t* __restrict__ x, int64_t d_out,
+                      const MvLut lut, const uint16_t* __restrict__ x, int64_t d_out,
                       int rows_per_block, float* __restrict__ partial) {
     extern __shared__ __align__(16) unsigned char raw[];
     // the finishing kernel may be scheduled from now on (it waits for this grid before it reads a partial sum)
@@ -581,16 +591,19 @@ extern "C" cmpq_status cmpq_outliers_by_column(const int32_t* rows, const int32_
     return launch_status();
 }
 
-extern "C" cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
-                                   const int64_t* seg_rows, const float* lut, int64_t d_in, int64_t d_out,
-                                   const void* x, cmpq_dtype dt, const int64_t* col_ptr, const int32_t* c_rows,
-                                   const uint16_t* c_vals, float* y, void* y16, void* ws, size_t ws_bytes,
-                                   void* stream) {
-    if (!packed || !row_off || !perm || !seg_rows || !lut || !x || !y) return CMPQ_ERR_INVALID_ARG;
+static cmpq_status matvec_impl(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
+                               const int64_t* seg_rows, const void* lut_p, int lut_is_f16, int64_t d_in, int64_t d_out,
+                               const void* x, cmpq_dtype dt, const int64_t* col_ptr, const int32_t* c_rows,
+                               const uint16_t* c_vals, float* y, void* y16, void* ws, size_t ws_bytes,
+                               void* stream) {
+    MvLut lut;
+    lut.p = lut_p;
+    lut.is_f16 = lut_is_f16;
+    if (!packed || !row_off || !perm || !seg_rows || !lut_p || !x || !y) return CMPQ_ERR_INVALID_ARG;
     if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT) return CMPQ_ERR_INVALID_ARG;
     if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
     if (col_ptr && (!c_rows || !c_vals)) return CMPQ_ERR_INVALID_ARG;
-    if (!aligned_to(packed, 4) || !aligned_to(row_off, 8) || !aligned_to(seg_rows, 8) || !aligned_to(lut, 4) ||
+    if (!aligned_to(packed, 4) || !aligned_to(row_off, 8) || !aligned_to(seg_rows, 8) || !aligned_to(lut_p, lut_is_f16 ? 2 : 4) ||
         !aligned_to(x, 2) || !aligned_to(y, 4) || (y16 && !aligned_to(y16, 2)) || (col_ptr && !aligned_to(col_ptr, 8)))
         return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < matvec_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
@@ -629,4 +642,22 @@ extern "C" cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_of
     }
     if (err != cudaSuccess) return CMPQ_ERR_CUDA;
     return launch_status();
+}
+
+extern "C" cmpq_status cmpq_matvec(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
+                                   const int64_t* seg_rows, const float* lut, int64_t d_in, int64_t d_out,
+                                   const void* x, cmpq_dtype dt, const int64_t* col_ptr, const int32_t* c_rows,
+                                   const uint16_t* c_vals, float* y, void* y16, void* ws, size_t ws_bytes,
+                                   void* stream) {
+    return matvec_impl(packed, row_off, perm, seg_rows, lut, 0, d_in, d_out, x, dt, col_ptr, c_rows, c_vals, y, y16, ws,
+                       ws_bytes, stream);
+}
+
+extern "C" cmpq_status cmpq_matvec_f16lut(const uint32_t* packed, const int64_t* row_off, const int32_t* perm,
+                                          const int64_t* seg_rows, const uint16_t* lut16, int64_t d_in,
+                                          int64_t d_out, const void* x, cmpq_dtype dt, const int64_t* col_ptr,
+                                          const int32_t* c_rows, const uint16_t* c_vals, float* y, void* y16,
+                                          void* ws, size_t ws_bytes, void* stream) {
+    return matvec_impl(packed, row_off, perm, seg_rows, lut16, 1, d_in, d_out, x, dt, col_ptr, c_rows, c_vals, y, y16,
+                       ws, ws_bytes, stream);
 }
