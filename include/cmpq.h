@@ -80,7 +80,9 @@ typedef enum {
     CMPQ_OP_PACK = 4,
     CMPQ_OP_PROTECT_AND_QUANTIZE = 5,
     CMPQ_OP_OUTLIERS_BY_COLUMN = 6, /* d_in is ignored */
-    CMPQ_OP_MATVEC = 7
+    CMPQ_OP_MATVEC = 7,
+    CMPQ_OP_QUANTIZE_LAYER_PACKED = 8,
+    CMPQ_OP_PROTECT_QUANTIZE_PACK = 9
 } cmpq_op;
 
 #define CMPQ_LUT_STRIDE 16      /* floats per channel in a look-up table */
@@ -254,6 +256,31 @@ cmpq_status cmpq_lloyd_phase_events(void* before_table, void* after_table, void*
 cmpq_status cmpq_pack(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
                       uint32_t* packed, int64_t* row_off, int32_t* perm, int64_t* seg_rows,
                       void* ws, size_t ws_bytes, void* stream);
+
+/* ---- final fit and packing in one call (Sections 3.2.1 / 3.2.2 with the storage of Section 5.1) ------
+ * cmpq_quantize_layer_packed = cmpq_quantize_layer followed by cmpq_pack, and
+ * cmpq_protect_quantize_pack = cmpq_protect_and_quantize followed by cmpq_pack: the same arguments and
+ * the same outputs bit for bit (lut, codes, packed, row_off, perm, seg_rows, ...).  The last assignment
+ * of the K-means writes the bit streams itself (the four threads that hold 32 neighbouring codes form
+ * the 2, 3 or 4 words of that group), so the byte codes need not exist: codes may be NULL, and then
+ * they are neither written nor read anywhere -- the call moves 2 bytes per weight less than the two
+ * separate calls.  With CMPQ_ASSIGN_ALL_PAIRS selected, or with sensitivities given, the kernels still
+ * produce byte codes: codes == NULL is then CMPQ_ERR_UNSUPPORTED, otherwise the packing runs as a
+ * separate step inside the call.  packed must hold cmpq_packed_words() words.
+ * ws: cmpq_workspace_bytes(CMPQ_OP_QUANTIZE_LAYER_PACKED / CMPQ_OP_PROTECT_QUANTIZE_PACK, d_in, d_out). */
+cmpq_status cmpq_quantize_layer_packed(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                       int64_t ldw, const uint8_t* bits, const int32_t* rows,
+                                       const int32_t* cols, int64_t nnz, int lloyd_iters, const float* sens,
+                                       float* lut, uint8_t* codes, uint32_t* packed, int64_t* row_off,
+                                       int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
+                                       unsigned long long* sweeps, void* ws, size_t ws_bytes, void* stream);
+cmpq_status cmpq_protect_quantize_pack(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                       const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                       int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
+                                       int64_t nnz_out, float* lut, uint8_t* codes, uint32_t* packed,
+                                       int64_t* row_off, int32_t* perm, int64_t* seg_rows,
+                                       int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
+                                       size_t ws_bytes, void* stream);
 
 /* ---- inference product of one token (Section 6: the figure of the real quantization process) ----
  * The input vector is split by the precision of its channels, every part multiplies its 2-, 3- or

@@ -16,7 +16,7 @@ ALLOC_RANK, ALLOC_QUANTILE = 0, 1
 NORM_L2, NORM_L1, NORM_LINF = 0, 1, 2
 ASSIGN_ORDERED, ASSIGN_ALL_PAIRS = 0, 1
 (OP_COLLECT_STATS, OP_ALLOCATE_BITS, OP_EXTRACT_OUTLIERS, OP_QUANTIZE_LAYER, OP_PACK, OP_PROTECT_AND_QUANTIZE,
- OP_OUTLIERS_BY_COLUMN, OP_MATVEC) = range(8)
+ OP_OUTLIERS_BY_COLUMN, OP_MATVEC, OP_QUANTIZE_LAYER_PACKED, OP_PROTECT_QUANTIZE_PACK) = range(10)
 LUT_STRIDE = 16
 
 EXPORTS = (
@@ -28,6 +28,7 @@ EXPORTS = (
     "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
     "cmpq_alu_probe", "cmpq_kernel_resources",
     "cmpq_sweep_cache_bytes", "cmpq_sweep_begin", "cmpq_sweep_budget",
+    "cmpq_quantize_layer_packed", "cmpq_protect_quantize_pack",
     "cmpq_matvec_f16lut", "cmpq_lut_bytes", "cmpq_store_lut", "cmpq_load_lut", "cmpq_table_bits_per_weight",
 )
 
@@ -98,6 +99,12 @@ def lib():
         L.cmpq_sweep_budget.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
                                         vp, vp, vp, vp, sz, vp, sz, vp]
         L.cmpq_sweep_budget.restype = ci
+        L.cmpq_quantize_layer_packed.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp, vp, vp,
+                                                 vp, vp, vp, vp, sz, vp]
+        L.cmpq_quantize_layer_packed.restype = ci
+        L.cmpq_protect_quantize_pack.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
+                                                 vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.cmpq_protect_quantize_pack.restype = ci
         L.cmpq_matvec_f16lut.argtypes = L.cmpq_matvec.argtypes
         L.cmpq_matvec_f16lut.restype = ci
         L.cmpq_lut_bytes.argtypes = [ci, i64]
@@ -254,6 +261,31 @@ def cmpq_protect_and_quantize(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, v
                                            n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz,
                                            _ptr(lut), _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(ws),
                                            ws.numel(), _stream()), "cmpq_protect_and_quantize")
+
+
+def cmpq_quantize_layer_packed(W, bits, rows, cols, lloyd_iters, lut, codes, packed, row_off, perm, seg_rows, ws,
+                               sens=None, inexact_rows=None, sweeps=None):
+    """cmpq_quantize_layer and cmpq_pack in one call; codes may be None (the byte codes are then never written)."""
+    d_in, d_out = W.shape
+    nnz = 0 if rows is None else rows.numel()
+    _check(lib().cmpq_quantize_layer_packed(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(bits),
+                                            _ptr(rows) if nnz else None, _ptr(cols) if nnz else None, nnz,
+                                            lloyd_iters, _ptr(sens), _ptr(lut), _ptr(codes), _ptr(packed),
+                                            _ptr(row_off), _ptr(perm), _ptr(seg_rows), _ptr(inexact_rows),
+                                            _ptr(sweeps), _ptr(ws), ws.numel(), _stream()),
+           "cmpq_quantize_layer_packed")
+
+
+def cmpq_protect_quantize_pack(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, packed, row_off,
+                               perm, seg_rows, ws, inexact_rows=None, sweeps=None):
+    """cmpq_protect_and_quantize and cmpq_pack in one call; codes may be None."""
+    d_in, d_out = W.shape
+    nnz = n_act * d_out + n_q
+    _check(lib().cmpq_protect_quantize_pack(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
+                                            n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz,
+                                            _ptr(lut), _ptr(codes), _ptr(packed), _ptr(row_off), _ptr(perm),
+                                            _ptr(seg_rows), _ptr(inexact_rows), _ptr(sweeps), _ptr(ws),
+                                            ws.numel(), _stream()), "cmpq_protect_quantize_pack")
 
 
 def cmpq_sweep_cache_bytes(d_in, d_out):

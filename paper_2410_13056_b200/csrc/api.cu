@@ -26,6 +26,12 @@ extern "C" size_t cmpq_workspace_bytes(cmpq_op op, int64_t d_in, int64_t d_out) 
         case CMPQ_OP_MATVEC:
             if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
             return matvec_ws_bytes(d_in, d_out);
+        case CMPQ_OP_QUANTIZE_LAYER_PACKED:
+            if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+            return quantize_packed_ws_bytes(d_in, d_out);
+        case CMPQ_OP_PROTECT_QUANTIZE_PACK:
+            if (d_out < 1 || d_out > CMPQ_MAX_D_OUT) return 0;
+            return protect_quantize_pack_ws_bytes(d_in, d_out);
     }
     return 0;
 }

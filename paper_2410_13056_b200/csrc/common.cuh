@@ -65,6 +65,8 @@ size_t outliers_ws_bytes(int64_t d_in, int64_t d_out);
 size_t quantize_ws_bytes(int64_t d_in, int64_t d_out);
 size_t pack_ws_bytes(int64_t d_in, int64_t d_out);
 size_t protect_quantize_ws_bytes(int64_t d_in, int64_t d_out);
+size_t quantize_packed_ws_bytes(int64_t d_in, int64_t d_out);
+size_t protect_quantize_pack_ws_bytes(int64_t d_in, int64_t d_out);
 size_t matvec_ws_bytes(int64_t d_in, int64_t d_out);
 size_t by_column_ws_bytes(int64_t d_out);
 

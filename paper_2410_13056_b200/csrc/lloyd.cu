@@ -635,26 +635,48 @@ extern "C" cmpq_status cmpq_lloyd_phase_events(void* before_table, void* after_t
     return CMPQ_OK;
 }
 
-extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
-                                           int64_t ldw, const uint8_t* bits, const int32_t* rows,
-                                           const int32_t* cols, int64_t nnz, int lloyd_iters,
-                                           const float* sens, float* lut, uint8_t* codes,
-                                           int32_t* inexact_rows, unsigned long long* sweeps,
-                                           void* ws, size_t ws_bytes, void* stream) {
-    if (!W || !bits || !lut || !codes) return CMPQ_ERR_INVALID_ARG;
+namespace cmpq {
+cmpq_status launch_pack_layout(const uint8_t* bits, int64_t d_in, int64_t d_out, int64_t* row_off, int32_t* perm,
+                               int64_t* seg_rows, int64_t* word_off, cudaStream_t st);
+cmpq_status launch_pack_codes(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
+                              const int64_t* word_off, uint32_t* packed, cudaStream_t st);
+
+size_t quantize_packed_ws_bytes(int64_t d_in, int64_t d_out) {
+    return quantize_ws_bytes(d_in, d_out) + pack_ws_bytes(d_in, d_out);
+}
+
+// The final fit; with `packed` also the packing, fused into the last assignment where the formulation allows.
+static cmpq_status quantize_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                 const uint8_t* bits, const int32_t* rows, const int32_t* cols, int64_t nnz,
+                                 int lloyd_iters, const float* sens, float* lut, uint8_t* codes, uint32_t* packed,
+                                 int64_t* row_off, int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
+                                 unsigned long long* sweeps, void* ws, size_t ws_bytes, void* stream) {
+    if (!W || !bits || !lut) return CMPQ_ERR_INVALID_ARG;
+    if (!codes && !packed) return CMPQ_ERR_INVALID_ARG;
     if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
     if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT || ldw < d_out)
         return CMPQ_ERR_INVALID_ARG;
     if (nnz < 0 || nnz > d_in * d_out || (nnz > 0 && (!rows || !cols))) return CMPQ_ERR_INVALID_ARG;
     if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
     if (!aligned_to(W, 2) || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
-    if (!aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;  // eight codes leave in one store
+    if (codes && !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;  // eight codes leave in one store
     if (sens && !aligned_to(sens, 4)) return CMPQ_ERR_INVALID_ARG;
-    if (!ws || !aligned_to(ws, 256) || ws_bytes < quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
+    if (packed && (!row_off || !perm || !seg_rows || !aligned_to(packed, 4) || !aligned_to(row_off, 8) ||
+                   !aligned_to(perm, 4) || !aligned_to(seg_rows, 8)))
+        return CMPQ_ERR_INVALID_ARG;
+    const bool fused_pack_ok = !sens && lloyd_assignment() != CMPQ_ASSIGN_ALL_PAIRS;
+    if (packed && !codes && !fused_pack_ok) return CMPQ_ERR_UNSUPPORTED;  // those kernels write byte codes
+    const size_t need = packed ? quantize_packed_ws_bytes(d_in, d_out) : quantize_ws_bytes(d_in, d_out);
+    if (!ws || !aligned_to(ws, 256) || ws_bytes < need) return CMPQ_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int64_t* row_ptr = static_cast<int64_t*>(ws);
+    int64_t* word_off = reinterpret_cast<int64_t*>(static_cast<char*>(ws) + quantize_ws_bytes(d_in, d_out));
     cmpq_status s = launch_row_ptr(rows, nnz, d_in, row_ptr, st);
     if (s != CMPQ_OK) return s;
+    if (packed) {
+        s = launch_pack_layout(bits, d_in, d_out, row_off, perm, seg_rows, word_off, st);
+        if (s != CMPQ_OK) return s;
+    }
     LloydArgs a{};
     a.W = static_cast<const uint16_t*>(W);
     a.d_in = d_in; a.d_out = d_out; a.ldw = ldw;
@@ -666,7 +688,37 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
     a.codes = codes;
     a.inexact_rows = inexact_rows;
     a.sweeps = sweeps;
-    if (sens) return launch_lloyd_weighted(a, dt, sens, st);
-    if (lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS) return launch_lloyd(a, dt, st);
+    if (!fused_pack_ok) {
+        s = sens ? launch_lloyd_weighted(a, dt, sens, st) : launch_lloyd(a, dt, st);
+        if (s != CMPQ_OK || !packed) return s;
+        return launch_pack_codes(codes, bits, d_in, d_out, word_off, packed, st);
+    }
+    a.packed = packed;
+    a.word_off = word_off;
     return launch_lloyd_ordered(a, dt, static_cast<char*>(ws) + row_ptr_bytes(d_in), lloyd_tables_bytes(d_in, d_out), st);
+}
+
+}  // namespace cmpq
+
+extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                           int64_t ldw, const uint8_t* bits, const int32_t* rows,
+                                           const int32_t* cols, int64_t nnz, int lloyd_iters,
+                                           const float* sens, float* lut, uint8_t* codes,
+                                           int32_t* inexact_rows, unsigned long long* sweeps,
+                                           void* ws, size_t ws_bytes, void* stream) {
+    if (!codes) return CMPQ_ERR_INVALID_ARG;
+    return quantize_impl(W, dt, d_in, d_out, ldw, bits, rows, cols, nnz, lloyd_iters, sens, lut, codes, nullptr,
+                         nullptr, nullptr, nullptr, inexact_rows, sweeps, ws, ws_bytes, stream);
+}
+
+extern "C" cmpq_status cmpq_quantize_layer_packed(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                                  int64_t ldw, const uint8_t* bits, const int32_t* rows,
+                                                  const int32_t* cols, int64_t nnz, int lloyd_iters,
+                                                  const float* sens, float* lut, uint8_t* codes, uint32_t* packed,
+                                                  int64_t* row_off, int32_t* perm, int64_t* seg_rows,
+                                                  int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
+                                                  size_t ws_bytes, void* stream) {
+    if (!packed) return CMPQ_ERR_INVALID_ARG;
+    return quantize_impl(W, dt, d_in, d_out, ldw, bits, rows, cols, nnz, lloyd_iters, sens, lut, codes, packed,
+                         row_off, perm, seg_rows, inexact_rows, sweeps, ws, ws_bytes, stream);
 }

@@ -20,6 +20,9 @@ struct LloydArgs {
     const int32_t* cols;     // [nnz] or NULL
     float* lut;              // [d_in][16] or NULL
     uint8_t* codes;          // [d_in][d_out] or NULL
+    // ordered formulation: the last assignment can write the packed bit streams itself (layout of cmpq_pack)
+    uint32_t* packed;        // or NULL
+    const int64_t* word_off; // [d_in] first word of every channel (with packed)
     int32_t* inexact_rows;   // optional counter
     unsigned long long* sweeps;  // optional counter of distance evaluations
     // ordered formulation only: fits kept across calls on the same weights (budget sweeps).  fit_cache is

@@ -30,6 +30,7 @@
 // Nothing here is a dense contraction, so no tensor cores are used.
 #include "lloyd.cuh"
 #include "lloyd_device.cuh"
+#include "pack_bits.cuh"
 #include "select.cuh"
 
 #include <cuda_bf16.h>
@@ -694,8 +695,9 @@ struct RemovedCols {
 template <int DT, int K, bool ERR>
 __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restrict__ lut,
                            const float* __restrict__ thr, const RemovedCols& rem, uint4 first) {
+    constexpr int C = K == 4 ? 2 : (K == 8 ? 3 : 4);
     const int N = (int)a.d_out;
-    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
     float c[K], t[K];
 #pragma unroll
     for (int k = 0; k < K; ++k) {
@@ -714,73 +716,98 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
     const bool vec_out = (N & 7) == 0;
     uint8_t* codes = a.codes ? a.codes + row * a.d_out : nullptr;
     float* err = a.err ? a.err + row * a.d_out : nullptr;
+    // packed output: the eight codes of a thread become a field of 8 C bits, four neighbouring threads
+    // hold 32 consecutive codes = C words
+    uint32_t* packed = (!ERR && a.packed) ? a.packed + a.word_off[row] : nullptr;
+    const int words_per_row = (N * C + 31) / 32;
 #pragma unroll 1
-    for (int j0 = tid * 8; j0 < N; j0 += nthr * 8) {
-        uint32_t pk[4] = {0u, 0u, 0u, 0u};  // 8 weights, two per word
-        if (j0 + 7 < N && vec_in) {
-            // the first step's weights were requested before anything else in the kernel
-            const uint4 v = j0 == tid * 8 ? first : __ldcs(reinterpret_cast<const uint4*>(w + j0));
-            pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
-        } else {
+    for (int base = 0; base < N; base += nthr * 8) {  // the same trip count in every thread of the block
+        const int j0 = base + tid * 8;
+        uint2 o = make_uint2(0u, 0u);  // eight codes, one per byte; zero beyond the end of the row
+        if (j0 < N) {
+            uint32_t pk[4] = {0u, 0u, 0u, 0u};  // 8 weights, two per word
+            if (j0 + 7 < N && vec_in) {
+                // the first step's weights were requested before anything else in the kernel
+                const uint4 v = base == 0 ? first : __ldcs(reinterpret_cast<const uint4*>(w + j0));
+                pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
+            } else {
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-                if (j0 + u < N) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
-        }
-        uint32_t mask = 0;  // removed positions among the 8
-        if (rem.nrem > kShortList) {
-            mask = (rem.bitmap[j0 >> 5] >> (j0 & 31)) & 0xffu;  // j0 is a multiple of 8
-        } else {
-            for (int i = 0; i < rem.nrem; ++i) {
-                const unsigned d = (unsigned)(rem.list[i] - j0);
-                if (d < 8u) mask |= 1u << d;
+                for (int u = 0; u < 8; ++u)
+                    if (j0 + u < N) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
             }
-        }
-        if (!ERR && codes && by_threshold && j0 + 7 < N && vec_out) {
-            uint32_t r[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t x2 = pk[q];
-                if ((mask >> (2 * q)) & 1u) x2 &= 0xffff0000u;      // removed positions become +0
-                if ((mask >> (2 * q + 1)) & 1u) x2 &= 0x0000ffffu;
-                uint32_t acc = acc0;
-#pragma unroll
-                for (int k = 1; k < K; ++k) acc = add_ge_x2<DT>(acc, x2, t2[k]);
-                r[q] = acc & 0x000f000fu;
-            }
-            uint2 o;
-            o.x = __byte_perm(r[0], r[1], 0x6420);
-            o.y = __byte_perm(r[2], r[3], 0x6420);
-            *reinterpret_cast<uint2*>(codes + j0) = o;
-            continue;
-        }
-        uint32_t code[8];
-        float dist[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            float x = widen16<DT>((uint16_t)(pk[u >> 1] >> (16 * (u & 1))));
-            if ((mask >> u) & 1u) x = 0.f;
-            x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
-            assign_one<K, ERR>(x, c, t, by_threshold, code[u], dist[u]);
-        }
-        if (j0 + 7 < N && vec_out) {
-            if (codes) {
-                uint2 o;
-                o.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
-                o.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
-                *reinterpret_cast<uint2*>(codes + j0) = o;
-            }
-            if (ERR && err) {
-                *reinterpret_cast<float4*>(err + j0) = make_float4(dist[0], dist[1], dist[2], dist[3]);
-                *reinterpret_cast<float4*>(err + j0 + 4) = make_float4(dist[4], dist[5], dist[6], dist[7]);
-            }
-        } else {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                if (j0 + u < N) {
-                    if (codes) codes[j0 + u] = (uint8_t)code[u];
-                    if (ERR && err) err[j0 + u] = dist[u];
+            uint32_t mask = 0;  // removed positions among the 8
+            if (rem.nrem > kShortList) {
+                mask = (rem.bitmap[j0 >> 5] >> (j0 & 31)) & 0xffu;  // j0 is a multiple of 8
+            } else {
+                for (int i = 0; i < rem.nrem; ++i) {
+                    const unsigned d = (unsigned)(rem.list[i] - j0);
+                    if (d < 8u) mask |= 1u << d;
                 }
             }
+            if (!ERR && by_threshold && j0 + 7 < N) {
+                uint32_t r[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t x2 = pk[q];
+                    if ((mask >> (2 * q)) & 1u) x2 &= 0xffff0000u;      // removed positions become +0
+                    if ((mask >> (2 * q + 1)) & 1u) x2 &= 0x0000ffffu;
+                    uint32_t acc = acc0;
+#pragma unroll
+                    for (int k = 1; k < K; ++k) acc = add_ge_x2<DT>(acc, x2, t2[k]);
+                    r[q] = acc & 0x000f000fu;
+                }
+                o.x = __byte_perm(r[0], r[1], 0x6420);
+                o.y = __byte_perm(r[2], r[3], 0x6420);
+                if (codes) {
+                    if (vec_out) {
+                        *reinterpret_cast<uint2*>(codes + j0) = o;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) codes[j0 + u] = (uint8_t)(((u < 4 ? o.x : o.y) >> (8 * (u & 3))) & 0xffu);
+                    }
+                }
+            } else {
+                uint32_t code[8];
+                float dist[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float x = widen16<DT>((uint16_t)(pk[u >> 1] >> (16 * (u & 1))));
+                    if ((mask >> u) & 1u) x = 0.f;
+                    x = (x == 0.f) ? 0.f : x;  // -0 and +0 are the same point
+                    assign_one<K, ERR>(x, c, t, by_threshold, code[u], dist[u]);
+                    if (j0 + u >= N) code[u] = 0u;
+                }
+                o.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
+                o.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
+                if (j0 + 7 < N && vec_out) {
+                    if (codes) *reinterpret_cast<uint2*>(codes + j0) = o;
+                    if (ERR && err) {
+                        *reinterpret_cast<float4*>(err + j0) = make_float4(dist[0], dist[1], dist[2], dist[3]);
+                        *reinterpret_cast<float4*>(err + j0 + 4) = make_float4(dist[4], dist[5], dist[6], dist[7]);
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (j0 + u < N) {
+                            if (codes) codes[j0 + u] = (uint8_t)code[u];
+                            if (ERR && err) err[j0 + u] = dist[u];
+                        }
+                    }
+                }
+            }
+        }
+        if (!ERR && packed) {
+            const uint32_t field = squeeze4<C>(o.x) | (squeeze4<C>(o.y) << (4 * C));
+            const uint32_t next = __shfl_down_sync(0xffffffffu, field, 1);  // the following eight codes
+            const int q = lane & 3;    // position in the group of 32 codes
+            const int g = j0 >> 5;
+            uint32_t word;
+            int widx;
+            bool mine;
+            if (C == 4) { word = field; widx = g * 4 + q; mine = true; }
+            else if (C == 2) { word = field | (next << 16); widx = g * 2 + (q >> 1); mine = (q & 1) == 0; }
+            else { word = (field >> (8 * q)) | (next << (24 - 8 * q)); widx = g * 3 + q; mine = q < 3; }
+            if (mine && widx < words_per_row) packed[widx] = word;
         }
     }
 }
@@ -1210,7 +1237,7 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
 
     // neither codes nor errors wanted: the fit alone (centroids and thresholds stay in the tables)
     if (args.err) lloyd_assign_kernel<DT, true><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
-    else if (args.codes) lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
+    else if (args.codes || args.packed) lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
     s = launch_status();
     if (ev[3]) cudaEventRecord(ev[3], st);
     return s;

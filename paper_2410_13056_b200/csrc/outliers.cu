@@ -403,6 +403,23 @@ size_t protect_quantize_ws_bytes(int64_t d_in, int64_t d_out) {
     return w.used;
 }
 
+size_t protect_quantize_pack_ws_bytes(int64_t d_in, int64_t d_out) {
+    return protect_quantize_ws_bytes(d_in, d_out) + pack_ws_bytes(d_in, d_out);
+}
+
+cmpq_status launch_pack_layout(const uint8_t* bits, int64_t d_in, int64_t d_out, int64_t* row_off, int32_t* perm,
+                               int64_t* seg_rows, int64_t* word_off, cudaStream_t st);
+cmpq_status launch_pack_codes(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
+                              const int64_t* word_off, uint32_t* packed, cudaStream_t st);
+
+// packed outputs of a call that also packs (all NULL otherwise)
+struct PackOut {
+    uint32_t* packed;
+    int64_t* row_off;
+    int32_t* perm;
+    int64_t* seg_rows;
+};
+
 }  // namespace cmpq
 
 namespace cmpq {
@@ -432,14 +449,26 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
                                          int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
                                          int64_t nnz_out, float* lut, uint8_t* codes, int32_t* inexact_rows,
                                          unsigned long long* sweeps, void* ws, size_t ws_bytes, void* cache,
-                                         cudaStream_t st) {
+                                         cudaStream_t st, const PackOut* po = nullptr) {
     cmpq_status s = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
     if (s != CMPQ_OK) return s;
-    if (!lut || !codes || !aligned_to(lut, 4) || !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;
-    if (!ws || !aligned_to(ws, 256) || ws_bytes < protect_quantize_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
+    if (!lut || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
+    if (!codes && !po) return CMPQ_ERR_INVALID_ARG;
+    if (codes && !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;
+    if (po && (!po->packed || !po->row_off || !po->perm || !po->seg_rows || !aligned_to(po->packed, 4) ||
+               !aligned_to(po->row_off, 8) || !aligned_to(po->perm, 4) || !aligned_to(po->seg_rows, 8)))
+        return CMPQ_ERR_INVALID_ARG;
+    const bool ordered = lloyd_assignment() != CMPQ_ASSIGN_ALL_PAIRS;
+    if (po && !codes && !ordered) return CMPQ_ERR_UNSUPPORTED;  // the all-pairs kernel writes byte codes
+    const size_t need = po ? protect_quantize_pack_ws_bytes(d_in, d_out) : protect_quantize_ws_bytes(d_in, d_out);
+    if (!ws || !aligned_to(ws, 256) || ws_bytes < need) return CMPQ_ERR_WORKSPACE;
     Workspace wsp(ws, ws_bytes);
     FusedWs f = carve_fused(wsp, d_in, d_out);
-    const bool ordered = lloyd_assignment() != CMPQ_ASSIGN_ALL_PAIRS;
+    int64_t* word_off = po ? wsp.take<int64_t>(d_in) : nullptr;
+    if (po) {  // the layout of the packed segments depends on the widths alone
+        s = launch_pack_layout(bits, d_in, d_out, po->row_off, po->perm, po->seg_rows, word_off, st);
+        if (s != CMPQ_OK) return s;
+    }
     void* fit_cache = nullptr;
     if (cache && ordered) {  // the provisional fit reads the cache's tables instead of building its own
         const SweepCache c = carve_sweep(cache, d_in, d_out);
@@ -463,7 +492,15 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
     la.inexact_rows = inexact_rows;
     la.sweeps = sweeps;
     const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
-    if (!ordered) return launch_lloyd(la, dt, st);
+    if (!ordered) {
+        s = launch_lloyd(la, dt, st);
+        if (s != CMPQ_OK || !po) return s;
+        return launch_pack_codes(codes, bits, d_in, d_out, word_off, po->packed, st);
+    }
+    if (po) {  // the last assignment writes the packed words itself
+        la.packed = po->packed;
+        la.word_off = word_off;
+    }
     // the provisional fit ran (and left its tables) only when entries had to be selected; a sweep cache
     // holds the tables of all channels in any case
     if (n_q > 0 || fit_cache) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, f.skip_rebuild, st);
@@ -482,6 +519,20 @@ extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, i
     return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
                                  lut, codes, inexact_rows, sweeps, ws, ws_bytes, nullptr,
                                  static_cast<cudaStream_t>(stream));
+}
+
+extern "C" cmpq_status cmpq_protect_quantize_pack(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
+                                                  int64_t ldw, const float* a, const uint8_t* bits,
+                                                  int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
+                                                  int32_t* cols, uint16_t* vals, int64_t nnz_out, float* lut,
+                                                  uint8_t* codes, uint32_t* packed, int64_t* row_off,
+                                                  int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
+                                                  unsigned long long* sweeps, void* ws, size_t ws_bytes,
+                                                  void* stream) {
+    const PackOut po{packed, row_off, perm, seg_rows};
+    return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
+                                 lut, codes, inexact_rows, sweeps, ws, ws_bytes, nullptr,
+                                 static_cast<cudaStream_t>(stream), &po);
 }
 
 extern "C" size_t cmpq_sweep_cache_bytes(int64_t d_in, int64_t d_out) {

@@ -6,6 +6,7 @@
 // a contiguous 256 to 512 bytes.  Every channel of a segment has the same length in words, so
 // its offset is segment base + (number of earlier channels of that width) * words.
 #include "common.cuh"
+#include "pack_bits.cuh"
 
 namespace cmpq {
 
@@ -74,38 +75,6 @@ pack_layout_kernel(const uint8_t* __restrict__ bits, int64_t d_in, int64_t d_out
     }
 }
 
-// Four codes held one per byte -> one 4C-bit field (C bits each, first code lowest).
-template <int C>
-__device__ __forceinline__ uint32_t squeeze4(uint32_t x) {
-    constexpr uint32_t m1 = ((1u << (2 * C)) - 1u) * 0x00010001u;
-    constexpr uint32_t m2 = (C == 4) ? 0xffffu : ((1u << (4 * C)) - 1u);
-    x &= ((1u << C) - 1u) * 0x01010101u;  // ignore anything above the channel's width
-    uint32_t t = (x | (x >> (8 - C))) & m1;
-    return (t | (t >> (16 - 2 * C))) & m2;
-}
-
-template <int C>
-__device__ __forceinline__ void pack32(const uint32_t (&b)[8], uint32_t (&w)[4]) {
-    uint32_t r[8];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) r[q] = squeeze4<C>(b[q]);
-    if (C == 2) {
-        w[0] = r[0] | (r[1] << 8) | (r[2] << 16) | (r[3] << 24);
-        w[1] = r[4] | (r[5] << 8) | (r[6] << 16) | (r[7] << 24);
-        w[2] = w[3] = 0;
-    } else if (C == 3) {
-        w[0] = r[0] | (r[1] << 12) | (r[2] << 24);
-        w[1] = (r[2] >> 8) | (r[3] << 4) | (r[4] << 16) | (r[5] << 28);
-        w[2] = (r[5] >> 4) | (r[6] << 8) | (r[7] << 20);
-        w[3] = 0;
-    } else {
-        w[0] = r[0] | (r[1] << 16);
-        w[1] = r[2] | (r[3] << 16);
-        w[2] = r[4] | (r[5] << 16);
-        w[3] = r[6] | (r[7] << 16);
-    }
-}
-
 // One thread packs 32 consecutive codes of one channel into C consecutive words.
 __global__ void __launch_bounds__(kPackThreads)
 pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ bits, int64_t d_out,
@@ -147,6 +116,23 @@ pack_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ bits,
         if (t < nwords) dst[t] = w[t];
 }
 
+// Layout of the packed segments from the widths alone: row_off / perm / seg_rows (outputs of cmpq_pack) and
+// word_off[i] = first word of channel i (d_in int64 of scratch).
+cmpq_status launch_pack_layout(const uint8_t* bits, int64_t d_in, int64_t d_out, int64_t* row_off, int32_t* perm,
+                               int64_t* seg_rows, int64_t* word_off, cudaStream_t st) {
+    pack_layout_kernel<<<1, 1024, 0, st>>>(bits, d_in, d_out, row_off, perm, seg_rows, word_off);
+    return launch_status();
+}
+
+cmpq_status launch_pack_codes(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
+                              const int64_t* word_off, uint32_t* packed, cudaStream_t st) {
+    const int64_t groups = (d_out + 31) / 32;
+    dim3 grid((unsigned)d_in, (unsigned)((groups + kPackThreads - 1) / kPackThreads));
+    const int vec_ok = aligned_to(codes, 16) && (d_out % 16 == 0);
+    pack_kernel<<<grid, kPackThreads, 0, st>>>(codes, bits, d_out, word_off, packed, vec_ok);
+    return launch_status();
+}
+
 }  // namespace cmpq
 
 using namespace cmpq;
@@ -168,10 +154,7 @@ extern "C" cmpq_status cmpq_pack(const uint8_t* codes, const uint8_t* bits, int6
     if (!ws || !aligned_to(ws, 256) || ws_bytes < pack_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int64_t* word_off = static_cast<int64_t*>(ws);
-    pack_layout_kernel<<<1, 1024, 0, st>>>(bits, d_in, d_out, row_off, perm, seg_rows, word_off);
-    const int64_t groups = (d_out + 31) / 32;
-    dim3 grid((unsigned)d_in, (unsigned)((groups + kPackThreads - 1) / kPackThreads));
-    const int vec_ok = aligned_to(codes, 16) && (d_out % 16 == 0);
-    pack_kernel<<<grid, kPackThreads, 0, st>>>(codes, bits, d_out, word_off, packed, vec_ok);
-    return launch_status();
+    const cmpq_status s = launch_pack_layout(bits, d_in, d_out, row_off, perm, seg_rows, word_off, st);
+    if (s != CMPQ_OK) return s;
+    return launch_pack_codes(codes, bits, d_in, d_out, word_off, packed, st);
 }

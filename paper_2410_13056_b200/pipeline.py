@@ -47,15 +47,19 @@ class LayerResult:
 
 
 class LayerQuantizer:
-    def __init__(self, d_in, d_out, device="cuda", n_act=None, n_q=None):
+    def __init__(self, d_in, d_out, device="cuda", n_act=None, n_q=None, keep_codes=True):
+        """keep_codes=False: the byte codes are never materialised (the last assignment of the final fit
+        writes the packed words directly); LayerResult.codes is then None."""
         self.d_in, self.d_out = int(d_in), int(d_out)
+        self.keep_codes = bool(keep_codes)
         self.device = torch.device(device)
         da, dq = B.cmpq_default_counts(self.d_in, self.d_out)
         self.n_act = da if n_act is None else int(n_act)
         self.n_q = dq if n_q is None else int(n_q)
         self.nnz = self.n_act * self.d_out + self.n_q
         dev = self.device
-        ws_bytes = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out) for op in range(6))
+        ws_bytes = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out)
+                       for op in list(range(6)) + [B.OP_PROTECT_QUANTIZE_PACK])
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
         self.sumsq = torch.empty(self.d_in, dtype=torch.float64, device=dev)
         self.a = torch.empty(self.d_in, dtype=torch.float32, device=dev)
@@ -64,7 +68,7 @@ class LayerQuantizer:
         self.cols = torch.empty(self.nnz, dtype=torch.int32, device=dev)
         self.vals = torch.empty(self.nnz, dtype=torch.int16, device=dev)
         self.lut = torch.empty((self.d_in, B.LUT_STRIDE), dtype=torch.float32, device=dev)
-        self.codes = torch.empty((self.d_in, self.d_out), dtype=torch.uint8, device=dev)
+        self.codes = torch.empty((self.d_in, self.d_out), dtype=torch.uint8, device=dev) if keep_codes else None
         max_words = self.d_in * ((self.d_out * 4 + 31) // 32)
         self.packed = torch.empty(max_words, dtype=torch.int32, device=dev)
         self.row_off = torch.empty(self.d_in + 1, dtype=torch.int64, device=dev)
@@ -107,14 +111,15 @@ class LayerQuantizer:
         """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
         reuse_statistic: keep the statistic `a` of the previous run on the same X (see run_budgets).
         sweep_cache: a cache prepared by cmpq_sweep_begin for W (see run_budgets).
-        fused (default: True unless events are asked for): outlier protection and final fit through
-        cmpq_protect_and_quantize, which derives the final fit's value tables from the provisional
-        fit's; otherwise cmpq_extract_outliers and cmpq_quantize_layer one after the other (same
-        results).  events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and,
+        fused (default: True unless events are asked for): outlier protection, final fit and packing through
+        cmpq_protect_quantize_pack, which derives the final fit's value tables from the provisional fit's
+        and lets the last assignment write the packed words; otherwise cmpq_extract_outliers,
+        cmpq_quantize_layer and cmpq_pack one after the other (same results; needs keep_codes).  events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and,
         when not fused, under "final_fit_kernels" the four events around the three kernels of the
         final K-means."""
         if fused is None:
-            fused = events is None
+            fused = events is None or not self.keep_codes
+        assert fused or self.keep_codes
         assert W.shape == (self.d_in, self.d_out) and X.shape[1] == self.d_in
 
         def call(name, fn, *args, **kw):
@@ -140,14 +145,16 @@ class LayerQuantizer:
             call("cmpq_sweep_budget", B.cmpq_sweep_budget, W, self.a, self.bits, self.n_act, self.n_q, lloyd_iters,
                  self.rows, self.cols, self.vals, self.lut, self.codes, sweep_cache, self.ws,
                  inexact_rows=inexact, sweeps=sweeps)
-        elif fused:
-            call("cmpq_protect_and_quantize", B.cmpq_protect_and_quantize, W, self.a, self.bits, self.n_act,
-                 self.n_q, lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.ws,
-                 inexact_rows=inexact, sweeps=sweeps)
+            call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
+                 self.seg_rows, self.ws)
+        elif fused:  # outlier protection, final fit and packing in one call
+            call("cmpq_protect_quantize_pack", B.cmpq_protect_quantize_pack, W, self.a, self.bits, self.n_act,
+                 self.n_q, lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.packed,
+                 self.row_off, self.perm, self.seg_rows, self.ws, inexact_rows=inexact, sweeps=sweeps)
         else:
             self._protect_then_quantize(call, W, lloyd_iters, events, inexact, sweeps)
-        call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
-             self.seg_rows, self.ws)
+            call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,
+                 self.seg_rows, self.ws)
         words = self.packed_words(avg_bits)
         return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
                            self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)
