@@ -84,6 +84,110 @@ __global__ void quantile_bits_kernel(const float* __restrict__ a, const int32_t*
     bits[i] = c;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Classification without a full rank.  Algorithm 1 in rank form and the choice of the O_act channels
+// (Section 3.2.2) only ask on which side of one or two rank cuts a channel lies.  One block finds, for
+// each cut k, the element of rank k in the ascending order of (a, id) by an exact radix select over the
+// order-preserving bit pattern of a (four 8-bit digits, both cuts at once), then every channel is
+// compared with the cut elements; equal statistics are ordered by channel id through a prefix count.
+constexpr int kCutThreads = 1024;
+
+__device__ __forceinline__ uint32_t ordered_bits(float v) {
+    const uint32_t u = __float_as_uint(v + 0.0f);  // -0 and +0 are the same value
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// out[i] = base + #{ t in {0,1} : channel i has rank >= k_t }.  k_t >= d_in: no channel reaches cut t.
+__global__ void __launch_bounds__(kCutThreads)
+rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long long k1, int base,
+                uint8_t* __restrict__ out) {
+    __shared__ unsigned int hist[2][256];
+    __shared__ uint32_t prefix[2];
+    __shared__ long long remaining[2];  // rank of the cut element among the elements matching the prefix
+    __shared__ unsigned long long warp_tot[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long k[2] = {k0, k1};
+    const bool live[2] = {k0 < d_in, k1 < d_in};
+    if (tid < 2) { prefix[tid] = 0u; remaining[tid] = k[tid] < 0 ? 0 : k[tid]; }
+    for (int pass = 3; pass >= 0; --pass) {
+        const int shift = 8 * pass;
+        const uint32_t mask = pass == 3 ? 0u : (0xffffffffu << (shift + 8));
+        for (int b = tid; b < 512; b += kCutThreads) (&hist[0][0])[b] = 0u;
+        __syncthreads();
+        const uint32_t p0 = prefix[0], p1 = prefix[1];
+        for (int64_t i = tid; i < d_in; i += kCutThreads) {
+            const uint32_t key = ordered_bits(a[i]);
+            const uint32_t d = (key >> shift) & 255u;
+            if (live[0] && (key & mask) == p0) atomicAdd(&hist[0][d], 1u);
+            if (live[1] && (key & mask) == p1) atomicAdd(&hist[1][d], 1u);
+        }
+        __syncthreads();
+        if (warp < 2 && live[warp]) {  // warp t walks the histogram of cut t upwards
+            unsigned int v[8], sum = 0;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { v[u] = hist[warp][lane * 8 + u]; sum += v[u]; }
+            unsigned int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            const long long rem = remaining[warp];
+            long long below = (long long)(incl - sum);
+            if (below <= rem && rem < (long long)incl) {  // exactly one lane
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (below <= rem && rem < below + (long long)v[u]) {
+                        prefix[warp] |= (uint32_t)(lane * 8 + u) << shift;
+                        remaining[warp] = rem - below;
+                        below = rem + 1;  // stop
+                    } else {
+                        below += v[u];
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    // every thread owns a contiguous range of channels: how many statistics equal to a cut value precede it
+    const int64_t per = (d_in + kCutThreads - 1) / kCutThreads;
+    const int64_t c0 = (int64_t)tid * per;
+    const int64_t c1 = c0 + per < d_in ? c0 + per : d_in;
+    const uint32_t v0 = prefix[0], v1 = prefix[1];
+    unsigned long long mine = 0;  // two counts of 32 bits
+    for (int64_t i = c0; i < c1; ++i) {
+        const uint32_t key = ordered_bits(a[i]);
+        mine += (key == v0 ? 1ull : 0ull) + (key == v1 ? (1ull << 32) : 0ull);
+    }
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    unsigned long long before = incl - mine;
+    for (int w = 0; w < warp; ++w) before += warp_tot[w];
+    long long eq0 = (long long)(before & 0xffffffffull), eq1 = (long long)(before >> 32);
+    const long long r0 = remaining[0], r1 = remaining[1];
+    for (int64_t i = c0; i < c1; ++i) {
+        const uint32_t key = ordered_bits(a[i]);
+        int cls = base;
+        if (live[0] && (key > v0 || (key == v0 && eq0 >= r0))) ++cls;
+        if (live[1] && (key > v1 || (key == v1 && eq1 >= r1))) ++cls;
+        eq0 += key == v0 ? 1 : 0;
+        eq1 += key == v1 ? 1 : 0;
+        out[i] = (uint8_t)cls;
+    }
+}
+
+cmpq_status launch_rank_cut(const float* a, int64_t d_in, int64_t k0, int64_t k1, int base, uint8_t* out,
+                            cudaStream_t st) {
+    rank_cut_kernel<<<1, kCutThreads, 0, st>>>(a, d_in, (long long)k0, (long long)k1, base, out);
+    return launch_status();
+}
+
 // rank[i] = position of channel i in the ascending order of (a, id).  rank must hold d_in ints.
 cmpq_status launch_rank(const float* a, int64_t d_in, int32_t* rank, cudaStream_t st) {
     if (cudaMemsetAsync(rank, 0, (size_t)d_in * sizeof(int32_t), st) != cudaSuccess) return CMPQ_ERR_CUDA;
@@ -120,10 +224,12 @@ extern "C" cmpq_status cmpq_allocate_bits(const float* a, int64_t d_in, double a
     Workspace w(ws, ws_bytes);
     int32_t* rank = w.take<int32_t>(d_in);
     int32_t* order_ws = w.take<int32_t>(d_in);
-    cmpq_status s = launch_rank(a, d_in, rank, st);
-    if (s != CMPQ_OK) return s;
     int64_t n2 = 0, n4 = 0;
     cmpq_alloc_counts(d_in, avg_bits, &n2, &n4);
+    // without the order only two rank cuts matter: 2 bits below rank n2, 4 bits from rank d_in - n4
+    if (mode == CMPQ_ALLOC_RANK && !order) return launch_rank_cut(a, d_in, n2, d_in - n4, 2, bits, st);
+    cmpq_status s = launch_rank(a, d_in, rank, st);
+    if (s != CMPQ_OK) return s;
     const unsigned blocks = (unsigned)((d_in + 255) / 256);
     if (mode == CMPQ_ALLOC_RANK) {
         rank_scatter_kernel<<<blocks, 256, 0, st>>>(rank, d_in, n2, n4, bits, order);

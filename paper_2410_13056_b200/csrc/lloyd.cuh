@@ -80,6 +80,11 @@ cmpq_status launch_lloyd_weighted(const LloydArgs& args, cmpq_dtype dt, const fl
 cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64_t* row_ptr,
                            cudaStream_t st);
 
+// out[i] = base + how many of the two rank cuts k0, k1 channel i reaches in the ascending order of (a, id)
+// (a cut >= d_in is reached by nobody).
+cmpq_status launch_rank_cut(const float* a, int64_t d_in, int64_t k0, int64_t k1, int base, uint8_t* out,
+                            cudaStream_t st);
+
 // rank[i] = position of channel i in the ascending order of (a, id).
 cmpq_status launch_rank(const float* a, int64_t d_in, int32_t* rank, cudaStream_t st);
 

@@ -21,12 +21,6 @@
 
 namespace cmpq {
 
-__global__ void mark_act_rows_kernel(const int32_t* __restrict__ rank, int64_t d_in, int64_t n_act,
-                                     uint8_t* __restrict__ is_act) {
-    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < d_in) is_act[i] = rank[i] >= d_in - n_act ? 1 : 0;
-}
-
 __global__ void select_init_kernel(SelectState* st, long long n_q) {
     st->prefix = 0; st->mask = 0; st->remaining = n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0;
 }
@@ -298,15 +292,13 @@ cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_o
                          const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
                          int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st,
                          void* fit_cache, bool tables_ready) {
-    const unsigned row_blocks = (unsigned)((d_in + 255) / 256);
-
     const bool all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
     const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
     const uint16_t* Wp = static_cast<const uint16_t*>(W);
 
-    cmpq_status s = launch_rank(a, d_in, o.rank, st);
+    // O_act: the channels of rank >= d_in - n_act in the ascending order of (a, id)
+    cmpq_status s = launch_rank_cut(a, d_in, d_in - n_act, d_in, 0, o.is_act, st);
     if (s != CMPQ_OK) return s;
-    mark_act_rows_kernel<<<row_blocks, 256, 0, st>>>(o.rank, d_in, n_act, o.is_act);
 
     if (n_q > 0) {
         LloydArgs la{};
