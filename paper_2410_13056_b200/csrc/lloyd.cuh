@@ -49,9 +49,9 @@ cmpq_status launch_lloyd_tables(const LloydArgs& args, cmpq_dtype dt, void* tabl
 size_t lloyd_fit_cache_bytes(int64_t d_in);
 cmpq_status launch_fit_cache_clear(void* fit_cache, int64_t d_in, int iters, cudaStream_t st);
 // Final fit whose value tables are derived from those a provisional ordered fit of the same weights left
-// in prov_tables (args.row_ptr / args.cols: the positions removed since; skip_rebuild: d_in bytes of scratch).
+// in prov_tables, which is only read (args.row_ptr / args.cols: the positions removed since).
 cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, void* prov_tables, void* tables,
-                                         size_t tables_bytes, uint8_t* skip_rebuild, cudaStream_t st);
+                                         size_t tables_bytes, cudaStream_t st);
 
 // Selection of the worst-fitted entries on the tables of a provisional ordered fit made with neither codes
 // nor errors requested (state: the radix select's SelectState; see outliers.cu for the procedure).

@@ -41,6 +41,7 @@ namespace cmpq {
 
 constexpr int kSlots = 32;       // high-byte buckets refined per pass of the second histogram level
 constexpr int kSlotWords = 128;  // 256 low-byte counters of 16 bits, two per word
+constexpr int kStageCap = 4096;  // table entries of one pass gathered in shared memory before they are stored
 static_assert(CMPQ_MAX_D_OUT < 65536, "second-level counters and count prefixes are 16 bits wide");
 
 struct ChannelHeader {
@@ -59,7 +60,8 @@ struct Tables {
     float* thr;          // [d_in][16] value thresholds of the last assignment ([0]: 1 if valid)
 };
 
-static int64_t table_stride(int64_t d_out) { return (d_out + 1 + 7) / 8 * 8; }
+// d_out + 1 entries and the sentinel, plus one entry of slack while a table is patched in place
+static int64_t table_stride(int64_t d_out) { return (d_out + 2 + 7) / 8 * 8; }
 
 static Tables carve_tables(Workspace& w, int64_t d_in, int64_t d_out) {
     Tables t;
@@ -106,6 +108,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     TableShared& sh = *reinterpret_cast<TableShared*>(smem_raw);
     uint32_t* h2 = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TableShared));
     uint32_t* bitmap = h2 + kSlots * kSlotWords;
+    uint16_t* st_keys = reinterpret_cast<uint16_t*>(bitmap + (a.d_out + 31) / 32);  // entries of one pass, gathered
+    uint16_t* st_cum = st_keys + kStageCap;
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = nthr >> 5;
     const int N = (int)a.d_out;
@@ -282,11 +286,13 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         const int w0 = (int)((long long)tid * words_total / nthr);
         const int w1 = (int)((long long)(tid + 1) * words_total / nthr);
         int nz = 0, cnt = 0;
+        uint32_t occupied = 0;  // bit 2 (w - w0) + half: that counter is not zero (ranges of at most 16 words)
         for (int w = w0; w < w1; ++w) {
             const uint32_t word = h2[w];
             const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
             nz += (c0 ? 1 : 0) + (c1 ? 1 : 0);
             cnt += c0 + c1;
+            if (w - w0 < 16) occupied |= ((c0 ? 1u : 0u) | (c1 ? 2u : 0u)) << (2 * (w - w0));
         }
         int inz = nz, icnt = cnt;
 #pragma unroll
@@ -299,17 +305,47 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         __syncthreads();
         run_nz = sh.base_nz + inz - nz;
         run_cnt = sh.base_cnt + icnt - cnt;
-        for (int wv = 0; wv < warp; ++wv) { run_nz += sh.w_nz[wv]; run_cnt += sh.w_cnt[wv]; }
-        for (int w = w0; w < w1; ++w) {
-            const uint32_t word = h2[w];
-            if (word) {
-                const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
-                const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-                if (c0) { keys[run_nz] = (uint16_t)kb; cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c0; }
-                if (c1) { keys[run_nz] = (uint16_t)(kb | 1u); cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c1; }
+        int pass_nz = 0;  // entries of this pass (all warps)
+        for (int wv = 0; wv < nwarps; ++wv) {
+            if (wv < warp) { run_nz += sh.w_nz[wv]; run_cnt += sh.w_cnt[wv]; }
+            pass_nz += sh.w_nz[wv];
+        }
+        // The entries of a pass are gathered in shared memory when they fit and leave in order with
+        // coalesced stores; a thread walks the set bits of its range instead of every counter.
+        const bool staged = pass_nz <= kStageCap;
+        const int stage_base = sh.base_nz;
+        uint16_t* out_keys = staged ? st_keys - stage_base : keys;
+        uint16_t* out_cum = staged ? st_cum - stage_base : cum;
+        if (w1 - w0 <= 16) {
+            while (occupied) {
+                const int b = __ffs(occupied) - 1;
+                occupied &= occupied - 1u;
+                const int w = w0 + (b >> 1);
+                const int c = (int)((h2[w] >> (16 * (b & 1))) & 0xffffu);
+                const uint32_t k = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1) | (uint32_t)(b & 1);
+                out_keys[run_nz] = (uint16_t)k;
+                out_cum[run_nz] = (uint16_t)run_cnt;
+                ++run_nz;
+                run_cnt += c;
+            }
+        } else {
+            for (int w = w0; w < w1; ++w) {
+                const uint32_t word = h2[w];
+                if (word) {
+                    const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
+                    const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
+                    if (c0) { out_keys[run_nz] = (uint16_t)kb; out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c0; }
+                    if (c1) { out_keys[run_nz] = (uint16_t)(kb | 1u); out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c1; }
+                }
             }
         }
         __syncthreads();  // every thread has read the bases and the counters of this pass
+        if (staged) {
+            for (int i = tid; i < pass_nz; i += nthr) {
+                keys[stage_base + i] = st_keys[i];
+                cum[stage_base + i] = st_cum[i];
+            }
+        }
         if (tid == nthr - 1) { sh.base_nz = run_nz; sh.base_cnt = run_cnt; }
     }
     if (tid == nthr - 1) {
@@ -324,7 +360,7 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// iterations: one warp per channel
+// fits kept between calls
 
 // fits kept between calls (see lloyd.cuh): slot (bits - 2) * d_in + row
 struct FitCacheHeader {
@@ -372,59 +408,113 @@ struct IterArgs {
     const uint8_t* skip_row;
     int64_t d_in, d_out;
     int iters;
-    int cap;     // table entries a warp can stage in shared memory (multiple of 8)
+    int cap;     // table entries a channel can stage in shared memory (multiple of 16)
     float* lut;  // [d_in][16]
     unsigned long long* sweeps;
+    // Final fit derived from the tables an earlier fit of the same weights left in `src`: this launch's
+    // table of a channel is src's with the positions row_ptr / cols removed (set to +0), built by the
+    // channel's lanes in shared memory (or in t, for tables too large to stage).  src.hdr == NULL: the
+    // tables in t are complete already.
+    Tables src;
+    const uint16_t* W;
+    int64_t ldw;
+    const int64_t* row_ptr;
+    const int32_t* cols;
+    int32_t* inexact_rows;
 };
 
-// Lane k (1..K-1) receives e_k = the number of table entries for whose value the predicate
-// fabsf(x - c_k) < fabsf(x - c_{k-1}) is false (a prefix of the table); lane 0 receives 0, lane K
-// receives M.  Every lane searches its own boundary: the warp's instruction stream then serves all
-// K-1 boundaries at once, which matters because the kernel is bound by instruction issue.  e_prev
-// (the lane's result of the previous iteration, or -1) starts a galloping search next to the old
-// boundary -- boundaries move by a few entries per iteration -- followed by bisection.
-template <int DT, int K>
-__device__ __forceinline__ int search_entries(const uint16_t* keys, int M, float ck_lane, int e_prev) {
-    const int lane = threadIdx.x & 31;
-    const float cm = __shfl_up_sync(0xffffffffu, ck_lane, 1);  // c_{k-1}
-    const float ck = ck_lane;
-    int lo = 0, hi = 0;  // the predicate is false for entries < lo and true for entries >= hi
-    if (lane > 0 && lane < K) {
-        hi = M;
-        auto pred = [&](int i) {
-            const float v = value_of_key16<DT>(keys[i]);
-            return fabsf(v - ck) < fabsf(v - cm);
-        };
-        if (e_prev >= 0) {
-            // gallop away from the old boundary p, downwards if the predicate holds at p and upwards if
-            // not, in one loop for both directions (lanes of both kinds then share the instructions)
-            const int p = e_prev < M ? e_prev : M;
-            const bool down = p >= M || pred(p);
-            if (down) hi = p; else lo = p + 1;
-            bool open = true;
-            for (int step = 1; open; step <<= 1) {
-                const int q = down ? hi - step : lo - 1 + step;
-                if (q < 0 || q >= M) break;  // ran off the table: the bracket is [0, hi] or [lo, M]
-                const bool t = pred(q);
-                if (t) hi = q; else lo = q + 1;
-                open = (t == down);          // closed by the first false (down) or the first true (up)
-            }
-        }
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if (pred(mid)) hi = mid; else lo = mid + 1;
-        }
-    }
-    __syncwarp();
-    return lane == K ? M : lo;
+// ------------------------------------------------------------------------------------------------
+// iterations: one half-warp per channel, two channels per warp
+//
+// While the centroids are strictly increasing with safe gaps, cluster k of a channel is the run of
+// table entries between two boundaries, and the boundary between clusters k-1 and k is a 16-bit KEY:
+// the first key b (in sort-key order) whose value is closer to c_k than to c_{k-1} under the defining
+// fp32 rule.  Between the two centroids fl(c_k - v) falls and fl(v - c_{k-1}) rises with v whatever the
+// rounding does, so the rule is monotone there and b is well defined; it lies next to the midpoint, so
+// b is found with two evaluations of the rule on register operands (no table access) in all but rare
+// cases, which fall back to bisection over keys.  The boundary as a table index -- how many table keys
+// lie below b -- is then read off the sixteen keys around the lane's previous boundary (boundaries move
+// by a few entries per iteration), with bisection over the rest of the table when it moved further.
+// The kernel is bound by the latency of this dependent chain (every channel of a layer is resident at
+// once), so the chain is kept short: no fp64 on the way to the boundary, the partial sums below a
+// boundary as a tree of independent products, one vote per iteration.
+
+constexpr int kGroup = 16;     // lanes that share one channel
+constexpr int kIterWarps = 2;  // warps per block: four channels
+constexpr int kKeyPad = 16;    // staged keys are followed by this many 0xffff entries
+
+// Shared memory of one channel: prefix sums at every eighth entry, keys (padded), count prefixes (table
+// of at most `cap` entries, cap a multiple of 16).
+constexpr int kPatchChunk = 64;  // removed positions of a channel handled per pass over its table (their keys
+                                 // borrow the space of the prefix sums, which are built afterwards)
+constexpr int kMinIterCap = 1536;  // smallest table capacity the host ever chooses
+static_assert(kPatchChunk * 4 <= (kMinIterCap / 8 + 2) * 8, "the prefix-sum area holds a chunk of removed keys");
+__host__ __device__ inline size_t iter_channel_bytes(int cap) {
+    const size_t b = (size_t)(cap / 8 + 2) * 8 + (size_t)(cap + kKeyPad) * 2 + (size_t)(cap + 8) * 2;
+    return (b + 15) / 16 * 16;
 }
 
-constexpr int kIterWarps = 4;
+__device__ __forceinline__ unsigned group_mask() { return 0xffffu << (threadIdx.x & 16); }
 
-// Shared memory of one warp of the iterate kernel: the channel's table when it has at most `cap`
-// distinct values (cap is a multiple of 8, chosen by the host from d_out).
-__host__ __device__ inline size_t iter_warp_bytes(int cap) {
-    return (size_t)cap * 2 + (size_t)(cap + 8) * 2 + (size_t)(cap / 8 + 1) * 8 + 8;  // keys, cum, coarse sums
+// Largest 16-bit storage value <= f / smallest >= f, as sort keys (f finite).
+__device__ __forceinline__ uint32_t key_of_pattern(uint32_t h) {
+    if ((h & 0x7fffu) == 0u) h = 0u;  // -0 and +0 are the same point
+    return (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+}
+template <int DT>
+__device__ __forceinline__ uint32_t key_floor(float f) {
+    uint32_t h;
+    if (DT == CMPQ_BF16) {
+        const uint32_t u = __float_as_uint(f);
+        h = (u & 0x80000000u) ? ((u + 0xffffu) >> 16) : (u >> 16);  // negative: the magnitude rounds up
+    } else {
+        h = __half_as_ushort(__float2half_rd(f));
+    }
+    return key_of_pattern(h);
+}
+template <int DT>
+__device__ __forceinline__ uint32_t key_ceil(float f) {
+    uint32_t h;
+    if (DT == CMPQ_BF16) {
+        const uint32_t u = __float_as_uint(f);
+        h = (u & 0x80000000u) ? (u >> 16) : ((u + 0xffffu) >> 16);
+    } else {
+        h = __half_as_ushort(__float2half_ru(f));
+    }
+    return key_of_pattern(h);
+}
+
+// The defining rule on one storage value given as a key: closer to ck than to cm (cm < ck)?
+template <int DT>
+__device__ __forceinline__ bool nearer_upper(uint32_t key, float cm, float ck) {
+    const float v = value_of_key16<DT>(key);
+    return fabsf(v - ck) < fabsf(v - cm);
+}
+
+// First key in [kfirst, kend] for which the rule holds, kend (one past the table's last key) counting as
+// true: every table key below the result goes to cluster k-1 or lower, every other one to k or higher.
+template <int DT>
+__device__ __forceinline__ uint32_t boundary_key(float cm, float ck, uint32_t kfirst, uint32_t kend) {
+    // candidate: the first storage value at or above the midpoint (fp32 is enough for a candidate)
+    uint32_t kc = key_ceil<DT>(0.5f * cm + 0.5f * ck);
+    kc = kc < kfirst ? kfirst : (kc > kend ? kend : kc);
+    const bool at = kc >= kend ? true : nearer_upper<DT>(kc, cm, ck);
+    const bool before = kc <= kfirst ? false : nearer_upper<DT>(kc - 1u, cm, ck);
+    if (at && !before) return kc;  // inside [cm, ck] the rule is monotone: this is the only change
+    // values <= cm are never nearer to ck; values >= ck inside the table's range always are
+    uint32_t lo = key_floor<DT>(cm) + 1u;
+    if (lo < kfirst) lo = kfirst;
+    uint32_t hi = key_ceil<DT>(ck);
+    if (hi > kend) hi = kend;
+    if (lo >= hi) return lo < kend ? lo : kend;
+    if (kc >= lo && kc <= hi) {  // use what the two evaluations told (kc - 1 holds the rule when kc does)
+        if (!at) lo = kc + 1u; else hi = kc - 1u;
+    }
+    while (lo < hi) {  // hi always names a key for which the rule holds
+        const uint32_t mid = (lo + hi) >> 1;
+        if (nearer_upper<DT>(mid, cm, ck)) hi = mid; else lo = mid + 1u;
+    }
+    return lo;
 }
 
 // Eight consecutive 16-bit table entries starting at a multiple of 8 (16-byte aligned), one load.
@@ -439,85 +529,265 @@ __device__ __forceinline__ Eight load_eight(const uint16_t* p) {
     return r;
 }
 
+// Number of table entries whose key is below b.  hint >= 0 (staged tables only: the keys are followed by
+// kKeyPad entries of 0xffff): the sixteen keys around entry `hint` are examined first.
+__device__ __forceinline__ int rank_of_key(const uint16_t* keys, int M, uint32_t b, int hint) {
+    int lo = 0, hi = M;
+    if (hint >= 0) {
+        int j0 = (hint & ~7) - 8;
+        if (j0 < 0) j0 = 0;
+        const Eight a8 = load_eight(keys + j0), b8 = load_eight(keys + j0 + 8);
+        int below = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) below += (a8.at(u) < b ? 1 : 0) + (b8.at(u) < b ? 1 : 0);
+        if (below == 0 && j0 > 0) hi = j0;                    // the boundary moved below the window
+        else if (below == 16 && j0 + 16 < M) lo = j0 + 16;    // ... or above it
+        else return j0 + below;                               // (entries past the table are 0xffff: never below)
+    }
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if ((uint32_t)keys[mid] < b) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// fp64 sum of count x value over the first r (0..7) of eight entries: independent products, added as a tree.
+template <int DT>
+__device__ __forceinline__ double partial_sum8(const Eight& k8, const Eight& c8, int r) {
+    double t[8];
+#pragma unroll
+    for (int u = 0; u < 7; ++u) {
+        const int cnt = (int)c8.at(u + 1) - (int)c8.at(u);
+        const double prod = (double)cnt * (double)value_of_key16<DT>(k8.at(u));
+        t[u] = u < r ? prod : 0.0;  // entries past the table may hold anything, NaN patterns included
+    }
+    return ((t[0] + t[1]) + (t[2] + t[3])) + ((t[4] + t[5]) + t[6]);
+}
+
 // fp64 sum of all weights below entry e (0 <= e <= M): the prefix stored for entry 8 (e / 8)
 // plus at most seven count x value products.
 template <int DT>
 __device__ __forceinline__ double prefix_sum_at(const uint16_t* keys, const uint16_t* cum, const double* coarse,
                                                 int e) {
-    const int j0 = e & ~7, r = e & 7;
-    double P = coarse[e >> 3];
+    const int j0 = e & ~7;
+    const double P = coarse[e >> 3];
     const Eight k8 = load_eight(keys + j0), c8 = load_eight(cum + j0);
-#pragma unroll
-    for (int u = 0; u < 7; ++u) {
-        if (u < r) {
-            const int cnt = (int)c8.at(u + 1) - (int)c8.at(u);
-            P += (double)cnt * (double)value_of_key16<DT>(k8.at(u));
-        }
-    }
-    return P;
+    return P + partial_sum8<DT>(k8, c8, e & 7);
 }
 
-template <int DT, int K>
-__device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* warp_smem) {
-    const int lane = threadIdx.x & 31;
-    const ChannelHeader h = a.t.hdr[row];
-    const int N = (int)a.d_out, T = a.iters;
-    const int M = h.M < 1 ? 1 : (h.M > N ? N : h.M);  // 1 <= M <= N by construction
-    const uint16_t* keys = a.t.keys + row * a.t.stride;
-    const uint16_t* cum = a.t.cum + row * a.t.stride;
-    double* coarse = a.t.sum + row * a.t.stride;  // global scratch, used when the table is too large
-    if (M <= a.cap) {  // the rows are 16-byte aligned and padded to a multiple of 8 entries
-        double* s_coarse = reinterpret_cast<double*>(warp_smem);
-        uint16_t* s_keys = reinterpret_cast<uint16_t*>(s_coarse + a.cap / 8 + 1 + 1);
-        uint16_t* s_cum = s_keys + a.cap;
-        for (int i = lane; i < (M + 7) / 8; i += 32)
-            reinterpret_cast<uint4*>(s_keys)[i] = __ldg(reinterpret_cast<const uint4*>(keys) + i);
-        for (int i = lane; i < (M + 1 + 7) / 8; i += 32)  // with the sentinel cum[M] = d_out
-            reinterpret_cast<uint4*>(s_cum)[i] = __ldg(reinterpret_cast<const uint4*>(cum) + i);
-        keys = s_keys;
-        cum = s_cum;
-        coarse = s_coarse;
+// Lane gl holds c_gl: is every centroid above its lower neighbour by more than `need`?  (per lane)
+__device__ __forceinline__ bool gap_ok(unsigned gmask, int gl, int K, float ck, double need) {
+    const float cp = __shfl_up_sync(gmask, ck, 1, kGroup);
+    return (gl == 0 || gl >= K) ? true : ((double)ck - (double)cp > need);
+}
+
+__device__ __forceinline__ double group_sum(unsigned gmask, double v) {
+#pragma unroll
+    for (int o = kGroup / 2; o > 0; o >>= 1) v += __shfl_xor_sync(gmask, v, o, kGroup);
+    return v;
+}
+__device__ __forceinline__ int group_sum(unsigned gmask, int v) {
+#pragma unroll
+    for (int o = kGroup / 2; o > 0; o >>= 1) v += __shfl_xor_sync(gmask, v, o, kGroup);
+    return v;
+}
+
+// W'' differs from W' only at the removed positions (the entries kept as outliers): the table of a row of
+// W'' is the table of the same row of W' with the counts of the removed values moved to the value +0.
+// One group of lanes does that in place on a writable copy (shared or global memory): keys[0..M) ascending,
+// cum[0..M] count prefixes with cum[M] = N.  Removed positions are taken kPatchChunk at a time; every pass
+// first makes sure an entry for +0 exists (entries above it move up by one, highest first), then adjusts
+// counts and prefixes and closes the gaps of entries whose count fell to zero (an entry never moves up, so
+// reading a chunk of sixteen entries before writing it keeps the pass in place).  Returns the new M.
+__device__ int patch_table(uint16_t* keys, uint16_t* cum, int M, int N, const uint16_t* __restrict__ wrow,
+                           const int32_t* __restrict__ cols, int nrem, uint32_t* rk) {
+    const unsigned gmask = group_mask();
+    const int gl = threadIdx.x & 15, gbase = threadIdx.x & 16;
+    const uint32_t kZeroKey = 0x8000u;  // sort key of +0
+    for (int c0 = 0; c0 < nrem; c0 += kPatchChunk) {
+        const int nr = nrem - c0 < kPatchChunk ? nrem - c0 : kPatchChunk;
+        for (int i = gl; i < nr; i += kGroup) {
+            uint32_t h = wrow[cols[c0 + i]];
+            if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
+            rk[i] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+        }
+        __syncwarp(gmask);
+        int lo = 0, hi = M;  // where +0 sits in the table, or would sit
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((uint32_t)keys[mid] >= kZeroKey) hi = mid; else lo = mid + 1;
+        }
+        const int pos0 = lo;
+        const bool present = pos0 < M && (uint32_t)keys[pos0] == kZeroKey;
+        __syncwarp(gmask);
+        if (!present) {  // entries pos0 .. M (the sentinel included) move up by one, highest chunk first
+            for (int base = pos0 + ((M - pos0) / kGroup) * kGroup; base >= pos0; base -= kGroup) {
+                const int j = base + gl;
+                const bool in = j <= M;
+                const uint16_t k = in ? keys[j] : (uint16_t)0, c = in ? cum[j] : (uint16_t)0;
+                __syncwarp(gmask);
+                if (in) { keys[j + 1] = k; cum[j + 1] = c; }
+                __syncwarp(gmask);
+            }
+            if (gl == 0) keys[pos0] = (uint16_t)kZeroKey;  // cum[pos0] already is the number of weights below +0
+            M += 1;
+            __syncwarp(gmask);
+        }
+        int deleted = 0;  // entries dropped so far in this pass
+        for (int base = 0; base < M; base += kGroup) {
+            const int i = base + gl;
+            const bool valid = i < M;
+            uint32_t key = kZeroKey;
+            int cnt = 0, below = 0;
+            if (valid) {
+                key = keys[i];
+                below = (int)cum[i];
+                cnt = (int)cum[i + 1] - below;
+                int eq = 0, lt = 0;
+                for (int r = 0; r < nr; ++r) {
+                    const uint32_t k = rk[r];
+                    eq += k == key ? 1 : 0;
+                    lt += k < key ? 1 : 0;
+                }
+                cnt -= eq;
+                below -= lt;
+                if (key == kZeroKey) cnt += nr;   // the removed weights are zeros now
+                if (key > kZeroKey) below += nr;
+            }
+            const bool keep = valid && cnt > 0;
+            const unsigned gone = (__ballot_sync(gmask, valid && !keep) >> gbase) & 0xffffu;
+            __syncwarp(gmask);  // every lane has read its entry (and the next prefix) before anyone writes
+            if (keep) {
+                const int o = i - deleted - __popc(gone & ((1u << gl) - 1u));
+                keys[o] = (uint16_t)key;
+                cum[o] = (uint16_t)below;
+            }
+            deleted += __popc(gone);
+            __syncwarp(gmask);
+        }
+        M -= deleted;
+        if (gl == 0) { keys[M] = 0xffffu; cum[M] = (uint16_t)N; }
+        __syncwarp(gmask);
     }
-    __syncwarp();
-    // prefix sums at every eighth entry: each lane sums a contiguous range of groups of eight entries,
-    // the lane totals are scanned, then every group receives its base
+    return M;
+}
+
+// The exactness test of the table kernel (see load_channel_keys) on a finished table.
+template <int DT>
+__device__ void count_if_inexact(const uint16_t* keys, int M, int N, int32_t* inexact_rows) {
+    const unsigned gmask = group_mask();
+    const int gl = threadIdx.x & 15;
+    uint32_t amax = 0u;
+    int q = 100000;
+    for (int i = gl; i < M; i += kGroup) {
+        const uint32_t ub = __float_as_uint(value_of_key16<DT>(keys[i])) & 0x7fffffffu;
+        if (ub) {
+            amax = max(amax, ub);
+            const int ex = (int)(ub >> 23);
+            const uint32_t m = ub & 0x7fffffu;
+            q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
+        }
+    }
+#pragma unroll
+    for (int o = kGroup / 2; o > 0; o >>= 1) {
+        amax = max(amax, __shfl_xor_sync(gmask, amax, o, kGroup));
+        q = min(q, __shfl_xor_sync(gmask, q, o, kGroup));
+    }
+    if (gl == 0 && amax != 0u) {
+        const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
+        const int ex_max = (int)(amax >> 23);
+        const int top = ex_max ? ex_max - 127 : (31 - __clz(amax)) - 149;
+        if (log2n + 1 + (top + 1 - q) > 53) atomicAdd(inexact_rows, 1);
+    }
+}
+
+// K = 2^bits of the channel is a run-time value on purpose: the two channels of a warp may differ in
+// width and still share one instruction stream (lanes >= K of a group idle).
+template <int DT>
+__device__ void iterate_channel(const IterArgs& a, int64_t row, const int K, unsigned char* smem) {
+    const unsigned gmask = group_mask();
+    const int gl = threadIdx.x & 15;
+    const int N = (int)a.d_out, T = a.iters;
+    double* s_coarse = reinterpret_cast<double*>(smem);
+    uint16_t* s_keys = reinterpret_cast<uint16_t*>(s_coarse + a.cap / 8 + 2);
+    uint16_t* s_cum = s_keys + a.cap + kKeyPad;
+    uint32_t* s_removed = reinterpret_cast<uint32_t*>(s_coarse);  // keys of removed weights: used before the sums exist
+    const bool patch = a.src.hdr != nullptr;
+    const Tables& from = patch ? a.src : a.t;
+    int64_t p0 = 0, nrem = 0;
+    if (patch) { p0 = a.row_ptr[row]; nrem = a.row_ptr[row + 1] - p0; }
+    int M = 1;
+    const uint16_t* keys = s_keys;
+    const uint16_t* cum = s_cum;
+    double* coarse = s_coarse;
+    bool staged = true;
+    if (patch && nrem >= N) {  // every position removed: an all-zero channel
+        if (gl == 0) { s_keys[0] = 0x8000u; s_cum[0] = 0; s_cum[1] = (uint16_t)N; }
+    } else {
+        const ChannelHeader h = from.hdr[row];
+        M = h.M < 1 ? 1 : (h.M > N ? N : h.M);  // 1 <= M <= N by construction
+        const uint16_t* g_keys = from.keys + row * from.stride;  // rows are 16-byte aligned, padded to 8 entries
+        const uint16_t* g_cum = from.cum + row * from.stride;
+        staged = M + (nrem > 0 ? 1 : 0) <= a.cap;  // removing weights can add the entry of +0
+        uint16_t* w_keys = staged ? s_keys : a.t.keys + row * a.t.stride;
+        uint16_t* w_cum = staged ? s_cum : a.t.cum + row * a.t.stride;
+        if (staged || patch) {  // copy: into shared memory, or into this launch's own table for patching
+            for (int i = gl; i < (M + 7) / 8; i += kGroup)
+                reinterpret_cast<uint4*>(w_keys)[i] = __ldg(reinterpret_cast<const uint4*>(g_keys) + i);
+            for (int i = gl; i < (M + 1 + 7) / 8; i += kGroup)  // with the sentinel cum[M] = d_out
+                reinterpret_cast<uint4*>(w_cum)[i] = __ldg(reinterpret_cast<const uint4*>(g_cum) + i);
+            __syncwarp(gmask);
+            if (nrem > 0) M = patch_table(w_keys, w_cum, M, N, a.W + row * a.ldw, a.cols + p0, (int)nrem, s_removed);
+            if (patch && a.inexact_rows && h.suspect) count_if_inexact<DT>(w_keys, M, N, a.inexact_rows);
+            keys = w_keys;
+            cum = w_cum;
+        } else {
+            keys = g_keys;
+            cum = g_cum;
+        }
+        if (!staged) coarse = a.t.sum + row * a.t.stride;  // global scratch for tables too large to stage
+    }
+    __syncwarp(gmask);
+    if (staged)  // nothing past the table
+        for (int i = M + gl; i < ((M + 7) & ~7) + kKeyPad; i += kGroup) s_keys[i] = 0xffffu;
+    __syncwarp(gmask);
+    // prefix sums at every eighth entry: each lane owns a contiguous range of groups of eight entries,
+    // sums each group (independent products), the lane totals are scanned, every group receives its base
     {
         const int groups = (M >> 3) + 1;  // coarse[g] for g = 0 .. M / 8
-        const int per_lane = (groups + 31) / 32;
-        const int g_begin = lane * per_lane;
+        const int per_lane = (groups + kGroup - 1) / kGroup;
+        const int g_begin = gl * per_lane;
         double local = 0.0;
         for (int g = g_begin; g < g_begin + per_lane && g < groups; ++g) {
-            coarse[g] = local;
             const Eight k8 = load_eight(keys + g * 8), c8 = load_eight(cum + g * 8);
-            const int c_end = g * 8 + 8 <= M ? (int)cum[g * 8 + 8] : 0;
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                if (g * 8 + u < M) {
-                    const int c_next = u < 7 ? (int)c8.at(u + 1) : c_end;
-                    local += (double)(c_next - (int)c8.at(u)) * (double)value_of_key16<DT>(k8.at(u));
-                }
-            }
+            const int left = M - g * 8;  // entries of this group that exist (may exceed 8)
+            double s7 = partial_sum8<DT>(k8, c8, left < 7 ? left : 7);
+            if (left >= 8) s7 += (double)((int)cum[g * 8 + 8] - (int)c8.at(7)) * (double)value_of_key16<DT>(k8.at(7));
+            coarse[g] = local;
+            local += s7;
         }
         double incl = local;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
+        for (int o = 1; o < kGroup; o <<= 1) {
+            const double up = __shfl_up_sync(gmask, incl, o, kGroup);
+            if (gl >= o) incl += up;
         }
-        double base = __shfl_up_sync(0xffffffffu, incl, 1);
-        if (lane == 0) base = 0.0;
+        double base = __shfl_up_sync(gmask, incl, 1, kGroup);
+        if (gl == 0) base = 0.0;
         for (int g = g_begin; g < g_begin + per_lane && g < groups; ++g) coarse[g] += base;
         __threadfence_block();  // the sums may live in global memory: make them visible to the other lanes
-        __syncwarp();
+        __syncwarp(gmask);
     }
+    const uint32_t kfirst = keys[0], kend = (uint32_t)keys[M - 1] + 1u;
     // range * 2^-22, the range being last minus first value of the table
-    const double need = ((double)value_of_key16<DT>(keys[M - 1]) - (double)value_of_key16<DT>(keys[0])) * (1.0 / 4194304.0);
+    const double need = ((double)value_of_key16<DT>(kend - 1u) - (double)value_of_key16<DT>(kfirst)) * (1.0 / 4194304.0);
+    const double p_total = prefix_sum_at<DT>(keys, cum, coarse, M);  // sum of all weights of the channel
 
     // start: K evenly spaced order statistics; the weight at sorted position pos has the value of the
     // entry e with cum[e] <= pos < cum[e + 1]
     float ck = 0.f;
-    if (lane < K) {
-        const int pos = (int)(((long long)(2 * lane + 1) * N) / (2 * K));
+    if (gl < K) {
+        const int pos = (int)(((long long)(2 * gl + 1) * N) / (2 * K));
         int lo = 0, hi = M;  // cum[lo] <= pos < cum[hi]   (cum[0] = 0, cum[M] = N)
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -525,102 +795,124 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, unsigned char* w
         }
         ck = value_of_key16<DT>(keys[lo]);
     }
-    __syncwarp();
+    __syncwarp(gmask);
 
+    // the boundary formulation needs strictly increasing centroids with gaps above `need`
+    bool ordered = __all_sync(gmask, gap_ok(gmask, gl, K, ck, need)) != 0;
     int updates = 0;
-    int e_prev = -1;  // this lane's boundary of the previous ordered search
+    int e_hint = -1;       // this lane's boundary of the previous ordered iteration (staged tables)
+    uint32_t b_last = 0;   // ... and its key
     while (updates < T) {
         float cn = ck;
-        if (counting_sweep_valid<K>(ck, need)) {
-            const int e = search_entries<DT, K>(keys, M, ck, e_prev);
-            e_prev = e;
+        if (ordered) {
+            const float cm = __shfl_up_sync(gmask, ck, 1, kGroup);  // c_{k-1}
+            int e = 0;  // first table entry of this lane's cluster
+            if (gl > 0 && gl < K) {
+                b_last = boundary_key<DT>(cm, ck, kfirst, kend);
+                e = b_last >= kend ? M : rank_of_key(keys, M, b_last, staged ? e_hint : -1);
+                e_hint = e;
+            }
             int B = 0;
             double P = 0.0;
-            if (lane <= K) { B = (int)cum[e]; P = prefix_sum_at<DT>(keys, cum, coarse, e); }
-            const int Bn = __shfl_down_sync(0xffffffffu, B, 1);
-            const double Pn = __shfl_down_sync(0xffffffffu, P, 1);
-            if (lane < K) {
+            if (gl < K) { B = (int)cum[e]; P = prefix_sum_at<DT>(keys, cum, coarse, e); }
+            int Bn = __shfl_down_sync(gmask, B, 1, kGroup);
+            double Pn = __shfl_down_sync(gmask, P, 1, kGroup);
+            if (gl == K - 1) { Bn = N; Pn = p_total; }  // the last cluster ends with the table
+            if (gl < K) {
                 const int cnt = Bn - B;
                 if (cnt > 0) cn = __double2float_rn(__ddiv_rn(Pn - P, (double)cnt));
             }
         } else {
+            e_hint = -1;
             // plain rule on every distinct value; cluster sums as count x value in fp64
-            float c[K];
+            float c[kMaxK];
 #pragma unroll
-            for (int k = 0; k < K; ++k) c[k] = __shfl_sync(0xffffffffu, ck, k);
-            double s[K];
-            int n[K];
+            for (int k = 0; k < kMaxK; ++k) c[k] = __shfl_sync(gmask, ck, k, kGroup);
+            double s[kMaxK];
+            int n[kMaxK];
 #pragma unroll
-            for (int k = 0; k < K; ++k) { s[k] = 0.0; n[k] = 0; }
-            for (int j = lane; j < M; j += 32) {
+            for (int k = 0; k < kMaxK; ++k) { s[k] = 0.0; n[k] = 0; }
+            for (int j = gl; j < M; j += kGroup) {
                 const float v = value_of_key16<DT>(keys[j]);
                 const int cnt = (int)cum[j + 1] - (int)cum[j];
-                const int code = nearest_scan<K>(v, c);
+                float best = fabsf(v - c[0]);
+                int code = 0;  // first k < K minimising |v - c_k|
+#pragma unroll
+                for (int k = 1; k < kMaxK; ++k) {
+                    const float d = fabsf(v - c[k]);
+                    if (k < K && d < best) { best = d; code = k; }
+                }
                 const double prod = (double)cnt * (double)v;
 #pragma unroll
-                for (int k = 0; k < K; ++k)
+                for (int k = 0; k < kMaxK; ++k)
                     if (code == k) { s[k] += prod; n[k] += cnt; }
             }
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
-                const double sk = warp_sum(s[k]);
-                const int nk = warp_sum(n[k]);
-                if (lane == k && nk > 0) cn = __double2float_rn(__ddiv_rn(sk, (double)nk));
+            for (int k = 0; k < kMaxK; ++k) {
+                if (k < K) {  // K is the same in every lane of the group
+                    const double sk = group_sum(gmask, s[k]);
+                    const int nk = group_sum(gmask, n[k]);
+                    if (gl == k && nk > 0) cn = __double2float_rn(__ddiv_rn(sk, (double)nk));
+                }
             }
         }
         ++updates;
-        const bool same = __all_sync(0xffffffffu, lane >= K || __float_as_uint(cn) == __float_as_uint(ck));
+        // one round of votes answers both questions about the new centroids
+        const bool ok = gap_ok(gmask, gl, K, cn, need);
+        const bool same_here = gl >= K || __float_as_uint(cn) == __float_as_uint(ck);
+        const unsigned full = gmask;
+        const bool same = __ballot_sync(gmask, same_here) == full;
+        const bool was_ordered = ordered;
+        ordered = __ballot_sync(gmask, ok) == full;
         ck = cn;
-        if (same) break;  // identical centroids: every later iteration repeats this one
-    }
-    if (lane < CMPQ_LUT_STRIDE) a.lut[row * CMPQ_LUT_STRIDE + lane] = lane < K ? ck : 0.f;
-    // Last assignment: when the final centroids pass the test, predicate k holds exactly for the values
-    // from the first entry where it is true, so the assign kernel only compares with K-1 thresholds.
-    {
-        const bool ok = counting_sweep_valid<K>(ck, need);
-        float thr = ok ? 1.f : 0.f;
-        if (ok) {
-            const int e = search_entries<DT, K>(keys, M, ck, e_prev);
-            if (lane > 0 && lane < K) thr = e < M ? value_of_key16<DT>(keys[e]) : __int_as_float(0x7f800000);
+        if (same) {  // identical centroids: every later iteration repeats this one
+            if (!was_ordered) e_hint = -1;
+            break;
         }
-        if (lane < CMPQ_LUT_STRIDE) a.t.thr[row * CMPQ_LUT_STRIDE + lane] = lane < K ? thr : 0.f;
+    }
+    a.lut[row * CMPQ_LUT_STRIDE + gl] = gl < K ? ck : 0.f;
+    // Last assignment: when the final centroids pass the test, a weight's code is the number of k >= 1
+    // whose boundary value it reaches, so the assign kernel only compares with K-1 thresholds.
+    {
+        const float cm = __shfl_up_sync(gmask, ck, 1, kGroup);
+        float thr = ordered ? 1.f : 0.f;
+        if (ordered && gl > 0 && gl < K) {
+            const uint32_t b = boundary_key<DT>(cm, ck, kfirst, kend);
+            thr = b < kend ? value_of_key16<DT>(b) : __int_as_float(0x7f800000);
+        }
+        a.t.thr[row * CMPQ_LUT_STRIDE + gl] = gl < K ? thr : 0.f;
     }
     // assignments made: one per update, and the last one by the assign kernel
-    if (a.sweeps && lane == 0)
+    if (a.sweeps && gl == 0)
         atomicAdd(a.sweeps, (unsigned long long)(updates + 1) * (unsigned long long)N * (unsigned long long)K);
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kIterWarps * 32, 7)
+__global__ void __launch_bounds__(kIterWarps * 32)
 lloyd_iterate_kernel(const IterArgs a) {
     extern __shared__ __align__(16) unsigned char iter_smem[];
-    const int warp = threadIdx.x >> 5;
-    unsigned char* warp_smem = iter_smem + (size_t)warp * iter_warp_bytes(a.cap);
-    const int64_t row = (int64_t)blockIdx.x * kIterWarps + warp;
+    const int group = threadIdx.x >> 4;  // channel of the block
+    unsigned char* smem = iter_smem + (size_t)group * iter_channel_bytes(a.cap);
+    const int64_t row = (int64_t)blockIdx.x * (kIterWarps * 2) + group;
     if (row >= a.d_in) return;
     if (a.skip_row && a.skip_row[row]) return;
+    const unsigned gmask = group_mask();
     const int bits = a.bits[row];
-    const int lane = threadIdx.x & 31;
+    const int gl = threadIdx.x & 15;
     // a fit of this channel at this width kept from an earlier call on the same weights: copy it
     const bool cached_ok = a.fc.hdr && a.fc.hdr->iters == a.iters;
     const int64_t slot = (int64_t)(bits == 2 ? 0 : (bits == 3 ? 1 : 2)) * a.d_in + row;
     if (cached_ok && a.fc.valid[slot]) {
-        if (lane < CMPQ_LUT_STRIDE) {
-            a.lut[row * CMPQ_LUT_STRIDE + lane] = a.fc.lut[slot * CMPQ_LUT_STRIDE + lane];
-            a.t.thr[row * CMPQ_LUT_STRIDE + lane] = a.fc.thr[slot * CMPQ_LUT_STRIDE + lane];
-        }
+        a.lut[row * CMPQ_LUT_STRIDE + gl] = a.fc.lut[slot * CMPQ_LUT_STRIDE + gl];
+        a.t.thr[row * CMPQ_LUT_STRIDE + gl] = a.fc.thr[slot * CMPQ_LUT_STRIDE + gl];
         return;
     }
-    if (bits == 2) iterate_channel<DT, 4>(a, row, warp_smem);
-    else if (bits == 3) iterate_channel<DT, 8>(a, row, warp_smem);
-    else iterate_channel<DT, 16>(a, row, warp_smem);
+    iterate_channel<DT>(a, row, bits == 2 ? 4 : (bits == 3 ? 8 : 16), smem);
     if (cached_ok) {  // lane l wrote entry l of both rows above and reads its own writes back
-        if (lane < CMPQ_LUT_STRIDE) {
-            a.fc.lut[slot * CMPQ_LUT_STRIDE + lane] = a.lut[row * CMPQ_LUT_STRIDE + lane];
-            a.fc.thr[slot * CMPQ_LUT_STRIDE + lane] = a.t.thr[row * CMPQ_LUT_STRIDE + lane];
-        }
-        __syncwarp();
-        if (lane == 0) {
+        a.fc.lut[slot * CMPQ_LUT_STRIDE + gl] = a.lut[row * CMPQ_LUT_STRIDE + gl];
+        a.fc.thr[slot * CMPQ_LUT_STRIDE + gl] = a.t.thr[row * CMPQ_LUT_STRIDE + gl];
+        __syncwarp(gmask);
+        if (gl == 0) {
             __threadfence();
             a.fc.valid[slot] = 1;
         }
@@ -1156,7 +1448,7 @@ cmpq_status launch_table_emit(void* tables, size_t tables_bytes, cmpq_dtype dt, 
 template <int DT, int E, int MAXT, int MINB>
 static cmpq_status launch_table(const LloydArgs& args, const Tables& t, int threads, cudaStream_t st) {
     const size_t smem = sizeof(TableShared) + (size_t)kSlots * kSlotWords * sizeof(uint32_t) +
-                        (((size_t)args.d_out + 31) / 32) * sizeof(uint32_t);
+                        (((size_t)args.d_out + 31) / 32) * sizeof(uint32_t) + (size_t)kStageCap * 2 * sizeof(uint16_t);
     auto kern = lloyd_table_kernel<DT, E, MAXT, MINB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
@@ -1200,7 +1492,8 @@ const void* lloyd_table_kernel_address() {
 
 // tables_ready: the value tables of every row to be fitted are in place already (skip the table kernel)
 template <int DT>
-static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, bool tables_ready, cudaStream_t st) {
+static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, bool tables_ready, cudaStream_t st,
+                                     const Tables* patch_from = nullptr) {
     tables_ready = tables_ready || args.tables_ready;
     if (args.err && args.codes) return CMPQ_ERR_INTERNAL;  // the assign kernel writes one or the other
     cudaEvent_t ev[4];
@@ -1222,14 +1515,22 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
     ia.iters = args.iters;
     ia.lut = args.lut ? args.lut : t.lut;
     ia.sweeps = args.sweeps;
+    if (patch_from) {
+        ia.src = *patch_from;
+        ia.W = args.W;
+        ia.ldw = args.ldw;
+        ia.row_ptr = args.row_ptr;
+        ia.cols = args.cols;
+        ia.inexact_rows = args.inexact_rows;
+    }
     // distinct 16-bit values grow slowly with the channel length (about 1400 at 4096 weights, 2300 at
     // 28672 for Gaussian-like bf16 weights); longer tables are read from global memory
-    ia.cap = N <= 4096 ? 1536 : (N <= 12288 ? 2048 : 3072);
-    const size_t iter_smem = (size_t)kIterWarps * iter_warp_bytes(ia.cap);
+    ia.cap = N <= 4096 ? kMinIterCap : (N <= 12288 ? 2048 : 3072);
+    const size_t iter_smem = (size_t)kIterWarps * 2 * iter_channel_bytes(ia.cap);
     if (cudaFuncSetAttribute(lloyd_iterate_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)iter_smem) !=
         cudaSuccess)
         return CMPQ_ERR_CUDA;
-    const unsigned iter_blocks = (unsigned)((args.d_in + kIterWarps - 1) / kIterWarps);
+    const unsigned iter_blocks = (unsigned)((args.d_in + kIterWarps * 2 - 1) / (kIterWarps * 2));
     lloyd_iterate_kernel<DT><<<iter_blocks, kIterWarps * 32, iter_smem, st>>>(ia);
     s = launch_status();
     if (s != CMPQ_OK) return s;
@@ -1259,172 +1560,19 @@ cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tab
 }
 
 // ------------------------------------------------------------------------------------------------
-// Final fit from the tables of the provisional fit.  W'' differs from W' only at the positions of
-// O_q (and the O_act rows are all zero in both), so the table of a row of W'' is the table of the
-// same row of W' with the counts of the removed values moved to the value +0.  One warp per row
-// does that for rows with at most kPatchCap removed positions; a row whose every position is
-// removed gets the one-entry table of an all-zero channel; the few other rows are flagged and
-// rebuilt from the weights by the table kernel.
-
-constexpr int kPatchCap = 64;
-constexpr int kPatchWarps = 4;
-
-template <int DT>
-__global__ void __launch_bounds__(kPatchWarps * 32)
-lloyd_patch_tables_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables src, const Tables dst,
-                          const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ cols, int64_t d_in,
-                          int64_t d_out, int32_t* inexact_rows, uint8_t* __restrict__ skip_rebuild, int cap) {
-    extern __shared__ __align__(16) unsigned char patch_smem[];  // per warp: cap keys, cap + 8 count prefixes
-    __shared__ uint32_t removed_keys[kPatchWarps][kPatchCap];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t row = (int64_t)blockIdx.x * kPatchWarps + warp;
-    if (row >= d_in) return;
-    const int N = (int)d_out;
-    const int64_t p0 = row_ptr[row];
-    const int64_t nrem64 = row_ptr[row + 1] - p0;
-    uint16_t* dkeys = dst.keys + row * dst.stride;
-    uint16_t* dcum = dst.cum + row * dst.stride;
-    const uint32_t kZeroKey = 0x8000u;  // sort key of +0
-    if (nrem64 >= N) {  // an all-zero channel
-        if (lane == 0) {
-            dkeys[0] = (uint16_t)kZeroKey; dcum[0] = 0;
-            dkeys[1] = 0xffffu; dcum[1] = (uint16_t)N;
-            ChannelHeader h; h.M = 1; h.suspect = 0; dst.hdr[row] = h;
-            skip_rebuild[row] = 1;
-        }
-        return;
-    }
-    if (nrem64 > kPatchCap) {
-        if (lane == 0) skip_rebuild[row] = 0;
-        return;
-    }
-    if (lane == 0) skip_rebuild[row] = 1;
-    const int nrem = (int)nrem64;
-    uint32_t* rk = removed_keys[warp];
-    for (int i = lane; i < nrem; i += 32) {
-        uint32_t h = W[row * ldw + cols[p0 + i]];
-        if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
-        rk[i] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
-    }
-    __syncwarp();
-    const int M = src.hdr[row].M;
-    const uint16_t* skeys = src.keys + row * src.stride;
-    const uint16_t* scum = src.cum + row * src.stride;
-    if (M <= cap) {  // stage the old table in shared memory: all its loads are in flight at once
-        uint16_t* s_keys = reinterpret_cast<uint16_t*>(patch_smem + (size_t)warp * (4 * (size_t)cap + 16));
-        uint16_t* s_cum = s_keys + cap;
-        for (int i = lane; i < (M + 7) / 8; i += 32)
-            reinterpret_cast<uint4*>(s_keys)[i] = __ldg(reinterpret_cast<const uint4*>(skeys) + i);
-        for (int i = lane; i < (M + 1 + 7) / 8; i += 32)
-            reinterpret_cast<uint4*>(s_cum)[i] = __ldg(reinterpret_cast<const uint4*>(scum) + i);
-        __syncwarp();
-        skeys = s_keys;
-        scum = s_cum;
-    }
-    // where +0 sits in the old table, or would sit
-    int lo = 0, hi = M;
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if ((uint32_t)skeys[mid] >= kZeroKey) hi = mid; else lo = mid + 1;
-    }
-    const int pos0 = lo;
-    const bool present = pos0 < M && (uint32_t)skeys[pos0] == kZeroKey;
-    const int ins = (nrem > 0 && !present) ? 1 : 0;  // +0 becomes a new entry
-    const int Mm = M + ins;
-    // The magnitude range of the old table proved its sums exact: so are those of any subset with zeros
-    // added, and the bit-by-bit test is skipped.
-    const bool test = inexact_rows && src.hdr[row].suspect;
-    int deleted = 0;  // entries dropped so far (their count fell to zero)
-    uint32_t amax = 0u;
-    int q = 100000;
-    for (int base = 0; base < Mm; base += 32) {
-        const int i = base + lane;
-        const bool valid = i < Mm;
-        uint32_t key = kZeroKey;
-        int cnt = 0, below = 0;  // weights with this value / with a smaller value in the old table
-        if (valid) {
-            if (ins && i == pos0) {
-                below = (int)scum[pos0];
-            } else {
-                const int j = (ins && i > pos0) ? i - 1 : i;
-                key = skeys[j];
-                below = (int)scum[j];
-                cnt = (int)scum[j + 1] - below;
-            }
-            int eq = 0, lt = 0;
-            for (int r = 0; r < nrem; ++r) {
-                const uint32_t k = rk[r];
-                eq += k == key ? 1 : 0;
-                lt += k < key ? 1 : 0;
-            }
-            cnt -= eq;
-            below -= lt;
-            if (key == kZeroKey) cnt += nrem;      // the removed weights are zeros now
-            if (key > kZeroKey) below += nrem;
-        }
-        const bool keep = cnt > 0;
-        const uint32_t gone = __ballot_sync(0xffffffffu, valid && !keep);
-        if (keep) {
-            const int o = i - deleted - __popc(gone & ((1u << lane) - 1u));
-            dkeys[o] = (uint16_t)key;
-            dcum[o] = (uint16_t)below;
-            if (test) {
-                const uint32_t ub = __float_as_uint(value_of_key16<DT>(key)) & 0x7fffffffu;
-                if (ub) {
-                    amax = max(amax, ub);
-                    const int ex = (int)(ub >> 23);
-                    const uint32_t m = ub & 0x7fffffu;
-                    q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
-                }
-            }
-        }
-        deleted += __popc(gone);
-    }
-    if (lane == 0) {
-        const int out = Mm - deleted;
-        dkeys[out] = 0xffffu;
-        dcum[out] = (uint16_t)N;
-        ChannelHeader h; h.M = out; h.suspect = src.hdr[row].suspect; dst.hdr[row] = h;
-    }
-    if (test) {  // the exactness test of the table kernel, on the new table
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-            q = min(q, __shfl_xor_sync(0xffffffffu, q, o));
-        }
-        if (lane == 0 && amax != 0u) {
-            const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
-            const int ex_max = (int)(amax >> 23);
-            const int top = ex_max ? ex_max - 127 : (31 - __clz(amax)) - 149;
-            if (log2n + 1 + (top + 1 - q) > 53) atomicAdd(inexact_rows, 1);
-        }
-    }
-}
+// Final fit from the tables of the provisional fit: the iterate kernel builds every channel's table
+// from the provisional one (see patch_table), so nothing is read from the weights and counted again.
 
 // args: the final fit (row_ptr / cols = the removed positions, skip_row unused).  prov_tables: the
-// tables the provisional fit left; tables: scratch of the final fit; skip_rebuild: d_in bytes.
+// tables the provisional fit left (read only); tables: scratch of the final fit.
 cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, void* prov_tables, void* tables,
-                                         size_t tables_bytes, uint8_t* skip_rebuild, cudaStream_t st) {
+                                         size_t tables_bytes, cudaStream_t st) {
     if (!prov_tables || !tables || tables_bytes < lloyd_tables_bytes(args.d_in, args.d_out)) return CMPQ_ERR_WORKSPACE;
+    if (!args.row_ptr) return CMPQ_ERR_INTERNAL;
     const Tables src = tables_at(prov_tables, tables_bytes, args.d_in, args.d_out);
     const Tables dst = tables_at(tables, tables_bytes, args.d_in, args.d_out);
-    const unsigned blocks = (unsigned)((args.d_in + kPatchWarps - 1) / kPatchWarps);
-    const int cap = args.d_out <= 4096 ? 1536 : (args.d_out <= 12288 ? 2048 : 3072);  // as in the iterate kernel
-    const size_t smem = (size_t)kPatchWarps * (4 * (size_t)cap + 16);
-    if (cudaFuncSetAttribute(lloyd_patch_tables_kernel<CMPQ_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute(lloyd_patch_tables_kernel<CMPQ_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return CMPQ_ERR_CUDA;
-    if (dt == CMPQ_F16)
-        lloyd_patch_tables_kernel<CMPQ_F16><<<blocks, kPatchWarps * 32, smem, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild, cap);
-    else
-        lloyd_patch_tables_kernel<CMPQ_BF16><<<blocks, kPatchWarps * 32, smem, st>>>(args.W, args.ldw, src, dst, args.row_ptr, args.cols, args.d_in, args.d_out, args.inexact_rows, skip_rebuild, cap);
-    cmpq_status s = launch_status();
-    if (s != CMPQ_OK) return s;
-    LloydArgs rebuild = args;  // rows with too many removed positions for the patch: from the weights
-    rebuild.skip_row = skip_rebuild;
-    s = dt == CMPQ_F16 ? launch_table_dt<CMPQ_F16>(rebuild, dst, st) : launch_table_dt<CMPQ_BF16>(rebuild, dst, st);
-    if (s != CMPQ_OK) return s;
-    return dt == CMPQ_F16 ? launch_ordered_dt<CMPQ_F16>(args, dst, true, st) : launch_ordered_dt<CMPQ_BF16>(args, dst, true, st);
+    return dt == CMPQ_F16 ? launch_ordered_dt<CMPQ_F16>(args, dst, true, st, &src)
+                          : launch_ordered_dt<CMPQ_BF16>(args, dst, true, st, &src);
 }
 
 }  // namespace cmpq

@@ -371,13 +371,11 @@ static cmpq_status check_extract_args(const void* W, cmpq_dtype dt, int64_t d_in
     return CMPQ_OK;
 }
 
-// work space of the fused call: the outlier step's, then the final fit's row index, tables and a
-// byte per row
+// work space of the fused call: the outlier step's, then the final fit's row index and tables
 struct FusedWs {
     OutlierWs o;
     int64_t* row_ptr;
     char* tables;
-    uint8_t* skip_rebuild;
 };
 
 static FusedWs carve_fused(Workspace& w, int64_t d_in, int64_t d_out) {
@@ -385,7 +383,6 @@ static FusedWs carve_fused(Workspace& w, int64_t d_in, int64_t d_out) {
     f.o = carve(w, d_in, d_out);
     f.row_ptr = w.take<int64_t>(d_in + 1);
     f.tables = w.take<char>(lloyd_tables_bytes(d_in, d_out));
-    f.skip_rebuild = w.take<uint8_t>(d_in);
     return f;
 }
 
@@ -470,14 +467,14 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
     s = extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, f.o, st,
                      fit_cache, fit_cache != nullptr);
     if (s != CMPQ_OK) return s;
-    s = launch_row_ptr(rows, nnz_out, d_in, f.row_ptr, st);
-    if (s != CMPQ_OK) return s;
+    // the list is sorted by row, so the first list position of a row is the start of the row's slice of
+    // the output: the row index of the final fit is the scan the outlier step has just made
     LloydArgs la{};
     la.W = static_cast<const uint16_t*>(W);
     la.d_in = d_in; la.d_out = d_out; la.ldw = ldw;
     la.bits = bits;
     la.iters = lloyd_iters;
-    la.row_ptr = f.row_ptr;
+    la.row_ptr = f.o.row_start;
     la.cols = cols;
     la.lut = lut;
     la.codes = codes;
@@ -495,7 +492,7 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
     }
     // the provisional fit ran (and left its tables) only when entries had to be selected; a sweep cache
     // holds the tables of all channels in any case
-    if (n_q > 0 || fit_cache) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, f.skip_rebuild, st);
+    if (n_q > 0 || fit_cache) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, st);
     return launch_lloyd_ordered(la, dt, f.tables, tables_bytes, st);
 }
 
