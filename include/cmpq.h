@@ -26,7 +26,12 @@
  *  - Arguments are checked on the host before anything is launched.  A call
  *    returns CMPQ_OK or an error code and never throws, aborts or prints;
  *    after an error no output has been written.
- *  - Inputs must be finite.
+ *  - Inputs must be finite.  Calls never look at their inputs on the host; the calls that read the
+ *    activations or the weights take an optional device word `nonfinite` (int32, zeroed by the caller,
+ *    may be NULL) into which the kernels OR bit 0 when an activation, and bit 1 when a weight, is a NaN or
+ *    an infinity (they read every value anyway, so the test costs nothing).  The outputs of such a call are
+ *    unspecified; the K-means iterations of the same call are skipped once the word is non-zero.
+ *    cmpq_check_finite waits for the stream and turns the word into a status.
  *  - Results are deterministic: the same inputs give the same bytes.
  */
 #ifndef CMPQ_H_
@@ -45,7 +50,8 @@ typedef enum {
     CMPQ_ERR_UNSUPPORTED = 2, /* legal but outside what the kernels handle (see each call) */
     CMPQ_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than cmpq_workspace_bytes */
     CMPQ_ERR_CUDA = 4,        /* a CUDA runtime call failed */
-    CMPQ_ERR_INTERNAL = 5
+    CMPQ_ERR_INTERNAL = 5,
+    CMPQ_ERR_NONFINITE = 6    /* an input held a NaN or an infinity (answer of cmpq_check_finite) */
 } cmpq_status;
 
 typedef enum { CMPQ_F16 = 0, CMPQ_BF16 = 1 } cmpq_dtype;
@@ -95,10 +101,17 @@ typedef enum {
  * calibration tokens after zeroing sumsq (fp64, d_in entries).  Squares are formed in fp32
  * (exact for 16-bit inputs), partial sums in fp32 over at most 32 rows, the rest in fp64 in
  * a fixed order.  n_tokens may be 0.  X is [n_tokens][ldx] of `dt`, ldx >= d_in.
+ * Because the squares are formed in fp32, a bf16 activation beyond about 1.8e19 in magnitude overflows
+ * to infinity although it is finite: it is reported through `nonfinite` like a true infinity (fp16
+ * inputs cannot get there).
  * ws: cmpq_workspace_bytes(CMPQ_OP_COLLECT_STATS, d_in, 0). */
 cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
-                               int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
+                               int64_t ldx, double* sumsq, int32_t* nonfinite, void* ws, size_t ws_bytes,
                                void* stream);
+
+/* Waits for `stream` and reads the word the calls above and below OR their findings into:
+ * CMPQ_OK if it is zero, CMPQ_ERR_NONFINITE otherwise (CMPQ_ERR_INVALID_ARG for NULL). */
+cmpq_status cmpq_check_finite(const int32_t* nonfinite, void* stream);
 
 /* Same result as cmpq_collect_stats without any work space: the partial sums live in a fixed
  * 2 MiB array inside the library (the paper has no counterpart; this exists for callers that
@@ -128,8 +141,8 @@ cmpq_status cmpq_finalize_stats(const double* sumsq, int64_t d_in, float* a, voi
  * The criterion a then feeds cmpq_allocate_bits and cmpq_extract_outliers unchanged.  An unknown
  * norm is CMPQ_ERR_INVALID_ARG.  ws: cmpq_workspace_bytes(CMPQ_OP_COLLECT_STATS, d_in, 0). */
 cmpq_status cmpq_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
-                                    int64_t ldx, cmpq_norm norm, double* acc, void* ws, size_t ws_bytes,
-                                    void* stream);
+                                    int64_t ldx, cmpq_norm norm, double* acc, int32_t* nonfinite, void* ws,
+                                    size_t ws_bytes, void* stream);
 cmpq_status cmpq_finalize_stats_norm(const double* acc, int64_t d_in, cmpq_norm norm, float* a,
                                      void* stream);
 
@@ -151,12 +164,15 @@ cmpq_status cmpq_allocate_bits(const float* a, int64_t d_in, double avg_bits, cm
  * patterns of W.  nnz_out must equal n_act*d_out + n_q (the arrays' length).
  * W is [d_in][ldw] of `dt`, ldw >= d_out, 1 <= d_out <= CMPQ_MAX_D_OUT.
  * 0 <= n_act <= d_in, 0 <= n_q <= (d_in - n_act)*d_out.
- * ws: cmpq_workspace_bytes(CMPQ_OP_EXTRACT_OUTLIERS, d_in, d_out)  (holds one fp32 per weight). */
+ * ws: cmpq_workspace_bytes(CMPQ_OP_EXTRACT_OUTLIERS, d_in, d_out): about 5 bytes per weight of value
+ * tables (2-byte key and 2-byte count prefix per possible distinct value, sums at every eighth), or one
+ * fp32 error per weight while CMPQ_ASSIGN_ALL_PAIRS is selected -- cmpq_workspace_bytes answers for the
+ * assignment method selected at the time it is asked. */
 cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
                                   int64_t ldw, const float* a, const uint8_t* bits, int64_t n_act,
                                   int64_t n_q, int lloyd_iters, int32_t* rows, int32_t* cols,
-                                  uint16_t* vals, int64_t nnz_out, void* ws, size_t ws_bytes,
-                                  void* stream);
+                                  uint16_t* vals, int64_t nnz_out, int32_t* nonfinite, void* ws,
+                                  size_t ws_bytes, void* stream);
 
 /* ---- channel-wise non-uniform quantization (Sections 3 and 3.2.1, final step of 3.2.2) -------
  * W'' = W with the nnz listed positions (sorted by (row, col), e.g. from cmpq_extract_outliers;
@@ -188,8 +204,8 @@ cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t d_in, int6
                                 int64_t ldw, const uint8_t* bits, const int32_t* rows,
                                 const int32_t* cols, int64_t nnz, int lloyd_iters,
                                 const float* sens, float* lut, uint8_t* codes,
-                                int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
-                                size_t ws_bytes, void* stream);
+                                int32_t* inexact_rows, unsigned long long* sweeps, int32_t* nonfinite,
+                                void* ws, size_t ws_bytes, void* stream);
 
 /* ---- outlier protection and quantization in one call (Section 3.2.2 with its final step) -------
  * Exactly cmpq_extract_outliers followed by cmpq_quantize_layer on the list it produced: the same
@@ -202,8 +218,8 @@ cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in
                                       int64_t ldw, const float* a, const uint8_t* bits, int64_t n_act,
                                       int64_t n_q, int lloyd_iters, int32_t* rows, int32_t* cols,
                                       uint16_t* vals, int64_t nnz_out, float* lut, uint8_t* codes,
-                                      int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
-                                      size_t ws_bytes, void* stream);
+                                      int32_t* inexact_rows, unsigned long long* sweeps, int32_t* nonfinite,
+                                      void* ws, size_t ws_bytes, void* stream);
 
 /* ---- budget sweeps (the paper's limitations paragraph: a new memory budget means quantizing again) --
  * The value tables of a layer's channels depend on the weights alone, and a channel's provisional
@@ -223,7 +239,7 @@ cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in
  * ws of cmpq_sweep_budget: cmpq_workspace_bytes(CMPQ_OP_PROTECT_AND_QUANTIZE, d_in, d_out). */
 size_t cmpq_sweep_cache_bytes(int64_t d_in, int64_t d_out);
 cmpq_status cmpq_sweep_begin(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
-                             int lloyd_iters, void* cache, size_t cache_bytes, void* stream);
+                             int lloyd_iters, int32_t* nonfinite, void* cache, size_t cache_bytes, void* stream);
 cmpq_status cmpq_sweep_budget(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
                               const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
                               int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
@@ -273,14 +289,15 @@ cmpq_status cmpq_quantize_layer_packed(const void* W, cmpq_dtype dt, int64_t d_i
                                        const int32_t* cols, int64_t nnz, int lloyd_iters, const float* sens,
                                        float* lut, uint8_t* codes, uint32_t* packed, int64_t* row_off,
                                        int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
-                                       unsigned long long* sweeps, void* ws, size_t ws_bytes, void* stream);
+                                       unsigned long long* sweeps, int32_t* nonfinite, void* ws, size_t ws_bytes,
+                                       void* stream);
 cmpq_status cmpq_protect_quantize_pack(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
                                        const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
                                        int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
                                        int64_t nnz_out, float* lut, uint8_t* codes, uint32_t* packed,
                                        int64_t* row_off, int32_t* perm, int64_t* seg_rows,
-                                       int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
-                                       size_t ws_bytes, void* stream);
+                                       int32_t* inexact_rows, unsigned long long* sweeps, int32_t* nonfinite,
+                                       void* ws, size_t ws_bytes, void* stream);
 
 /* ---- inference product of one token (Section 6: the figure of the real quantization process) ----
  * The input vector is split by the precision of its channels, every part multiplies its 2-, 3- or

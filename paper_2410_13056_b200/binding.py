@@ -28,7 +28,7 @@ EXPORTS = (
     "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
     "cmpq_alu_probe", "cmpq_kernel_resources",
     "cmpq_sweep_cache_bytes", "cmpq_sweep_begin", "cmpq_sweep_budget",
-    "cmpq_quantize_layer_packed", "cmpq_protect_quantize_pack",
+    "cmpq_quantize_layer_packed", "cmpq_protect_quantize_pack", "cmpq_check_finite",
     "cmpq_matvec_f16lut", "cmpq_lut_bytes", "cmpq_store_lut", "cmpq_load_lut", "cmpq_table_bits_per_weight",
 )
 
@@ -53,19 +53,21 @@ def lib():
         L = ctypes.CDLL(_LIB_PATH)
         i64, vp, dbl, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_double, ctypes.c_size_t
         ci = ctypes.c_int
-        L.cmpq_collect_stats.argtypes = [vp, ci, i64, i64, i64, vp, vp, sz, vp]
+        L.cmpq_collect_stats.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, sz, vp]
+        L.cmpq_check_finite.argtypes = [vp, vp]
+        L.cmpq_check_finite.restype = ci
         L.cmpq_collect_stats_static.argtypes = [vp, ci, i64, i64, i64, vp, vp]
         L.cmpq_finalize_stats.argtypes = [vp, i64, vp, vp]
         L.cmpq_allocate_bits.argtypes = [vp, i64, dbl, ci, vp, vp, vp, sz, vp]
         L.cmpq_extract_outliers.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp,
-                                            i64, vp, sz, vp]
+                                            i64, vp, vp, sz, vp]
         L.cmpq_quantize_layer.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp,
-                                          vp, vp, sz, vp]
+                                          vp, vp, vp, sz, vp]
         L.cmpq_pack.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_protect_and_quantize.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
-                                                vp, vp, vp, vp, sz, vp]
+                                                vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_protect_and_quantize.restype = ci
-        L.cmpq_collect_stats_norm.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, sz, vp]
+        L.cmpq_collect_stats_norm.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, sz, vp]
         L.cmpq_collect_stats_norm.restype = ci
         L.cmpq_finalize_stats_norm.argtypes = [vp, i64, ci, vp, vp]
         L.cmpq_finalize_stats_norm.restype = ci
@@ -94,16 +96,16 @@ def lib():
         L.cmpq_lloyd_phase_events.restype = ci
         L.cmpq_sweep_cache_bytes.argtypes = [i64, i64]
         L.cmpq_sweep_cache_bytes.restype = sz
-        L.cmpq_sweep_begin.argtypes = [vp, ci, i64, i64, i64, ci, vp, sz, vp]
+        L.cmpq_sweep_begin.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, sz, vp]
         L.cmpq_sweep_begin.restype = ci
         L.cmpq_sweep_budget.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
                                         vp, vp, vp, vp, sz, vp, sz, vp]
         L.cmpq_sweep_budget.restype = ci
         L.cmpq_quantize_layer_packed.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp, vp, vp,
-                                                 vp, vp, vp, vp, sz, vp]
+                                                 vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_quantize_layer_packed.restype = ci
         L.cmpq_protect_quantize_pack.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
-                                                 vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+                                                 vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_protect_quantize_pack.restype = ci
         L.cmpq_matvec_f16lut.argtypes = L.cmpq_matvec.argtypes
         L.cmpq_matvec_f16lut.restype = ci
@@ -212,11 +214,18 @@ def cmpq_packed_words(bits_host, d_out):
     return int(lib().cmpq_packed_words(ctypes.c_void_p(b.data_ptr()), b.numel(), d_out))
 
 
-def cmpq_collect_stats(X, sumsq, ws):
-    """sumsq (float64 [d_in]) += column sums of squares of X ([n_tokens][d_in], fp16/bf16)."""
+def cmpq_collect_stats(X, sumsq, ws, nonfinite=None):
+    """sumsq (float64 [d_in]) += column sums of squares of X ([n_tokens][d_in], fp16/bf16).
+    nonfinite (here and below): optional int32 device word the kernels OR their findings into
+    (bit 0: a NaN or infinity among the activations, bit 1: among the weights); see cmpq_check_finite."""
     n, d_in = X.shape
     _check(lib().cmpq_collect_stats(_ptr(X), dtype_code(X), n, d_in, X.stride(0) if n > 0 else d_in,
-                                    _ptr(sumsq), _ptr(ws), ws.numel(), _stream()), "cmpq_collect_stats")
+                                    _ptr(sumsq), _ptr(nonfinite), _ptr(ws), ws.numel(), _stream()), "cmpq_collect_stats")
+
+
+def cmpq_check_finite(nonfinite):
+    """Waits for the current stream; raises CmpqError (status 6) if the word is not zero."""
+    _check(lib().cmpq_check_finite(_ptr(nonfinite), _stream()), "cmpq_check_finite")
 
 
 def cmpq_collect_stats_static(X, sumsq):
@@ -236,35 +245,37 @@ def cmpq_allocate_bits(a, avg_bits, mode, bits, order, ws):
                                     _ptr(ws), ws.numel(), _stream()), "cmpq_allocate_bits")
 
 
-def cmpq_extract_outliers(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, ws):
+def cmpq_extract_outliers(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, ws, nonfinite=None):
     d_in, d_out = W.shape
     _check(lib().cmpq_extract_outliers(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
                                        n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals),
-                                       rows.numel(), _ptr(ws), ws.numel(), _stream()), "cmpq_extract_outliers")
+                                       rows.numel(), _ptr(nonfinite), _ptr(ws), ws.numel(), _stream()),
+           "cmpq_extract_outliers")
 
 
 def cmpq_quantize_layer(W, bits, rows, cols, lloyd_iters, lut, codes, ws, sens=None, inexact_rows=None,
-                        sweeps=None):
+                        sweeps=None, nonfinite=None):
     d_in, d_out = W.shape
     nnz = 0 if rows is None else rows.numel()
     _check(lib().cmpq_quantize_layer(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(bits),
                                      _ptr(rows) if nnz else None, _ptr(cols) if nnz else None, nnz,
                                      lloyd_iters, _ptr(sens), _ptr(lut), _ptr(codes), _ptr(inexact_rows),
-                                     _ptr(sweeps), _ptr(ws), ws.numel(), _stream()), "cmpq_quantize_layer")
+                                     _ptr(sweeps), _ptr(nonfinite), _ptr(ws), ws.numel(), _stream()),
+           "cmpq_quantize_layer")
 
 
 def cmpq_protect_and_quantize(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, ws,
-                              inexact_rows=None, sweeps=None):
+                              inexact_rows=None, sweeps=None, nonfinite=None):
     d_in, d_out = W.shape
     nnz = n_act * d_out + n_q
     _check(lib().cmpq_protect_and_quantize(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
                                            n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz,
-                                           _ptr(lut), _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(ws),
-                                           ws.numel(), _stream()), "cmpq_protect_and_quantize")
+                                           _ptr(lut), _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(nonfinite),
+                                           _ptr(ws), ws.numel(), _stream()), "cmpq_protect_and_quantize")
 
 
 def cmpq_quantize_layer_packed(W, bits, rows, cols, lloyd_iters, lut, codes, packed, row_off, perm, seg_rows, ws,
-                               sens=None, inexact_rows=None, sweeps=None):
+                               sens=None, inexact_rows=None, sweeps=None, nonfinite=None):
     """cmpq_quantize_layer and cmpq_pack in one call; codes may be None (the byte codes are then never written)."""
     d_in, d_out = W.shape
     nnz = 0 if rows is None else rows.numel()
@@ -272,31 +283,31 @@ def cmpq_quantize_layer_packed(W, bits, rows, cols, lloyd_iters, lut, codes, pac
                                             _ptr(rows) if nnz else None, _ptr(cols) if nnz else None, nnz,
                                             lloyd_iters, _ptr(sens), _ptr(lut), _ptr(codes), _ptr(packed),
                                             _ptr(row_off), _ptr(perm), _ptr(seg_rows), _ptr(inexact_rows),
-                                            _ptr(sweeps), _ptr(ws), ws.numel(), _stream()),
+                                            _ptr(sweeps), _ptr(nonfinite), _ptr(ws), ws.numel(), _stream()),
            "cmpq_quantize_layer_packed")
 
 
 def cmpq_protect_quantize_pack(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, packed, row_off,
-                               perm, seg_rows, ws, inexact_rows=None, sweeps=None):
+                               perm, seg_rows, ws, inexact_rows=None, sweeps=None, nonfinite=None):
     """cmpq_protect_and_quantize and cmpq_pack in one call; codes may be None."""
     d_in, d_out = W.shape
     nnz = n_act * d_out + n_q
     _check(lib().cmpq_protect_quantize_pack(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
                                             n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz,
                                             _ptr(lut), _ptr(codes), _ptr(packed), _ptr(row_off), _ptr(perm),
-                                            _ptr(seg_rows), _ptr(inexact_rows), _ptr(sweeps), _ptr(ws),
-                                            ws.numel(), _stream()), "cmpq_protect_quantize_pack")
+                                            _ptr(seg_rows), _ptr(inexact_rows), _ptr(sweeps), _ptr(nonfinite),
+                                            _ptr(ws), ws.numel(), _stream()), "cmpq_protect_quantize_pack")
 
 
 def cmpq_sweep_cache_bytes(d_in, d_out):
     return int(lib().cmpq_sweep_cache_bytes(d_in, d_out))
 
 
-def cmpq_sweep_begin(W, lloyd_iters, cache):
+def cmpq_sweep_begin(W, lloyd_iters, cache, nonfinite=None):
     """Counts the values of every channel of W into `cache` (uint8 tensor of cmpq_sweep_cache_bytes bytes)."""
     d_in, d_out = W.shape
-    _check(lib().cmpq_sweep_begin(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), lloyd_iters, _ptr(cache),
-                                  cache.numel(), _stream()), "cmpq_sweep_begin")
+    _check(lib().cmpq_sweep_begin(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), lloyd_iters, _ptr(nonfinite),
+                                  _ptr(cache), cache.numel(), _stream()), "cmpq_sweep_begin")
 
 
 def cmpq_sweep_budget(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, cache, ws,
@@ -369,11 +380,12 @@ def cmpq_matvec_f16lut(packed, row_off, perm, seg_rows, lut16, x, col_ptr, c_row
                                     _ptr(y), _ptr(y16), _ptr(ws), ws.numel(), _stream()), "cmpq_matvec_f16lut")
 
 
-def cmpq_collect_stats_norm(X, norm, acc, ws):
+def cmpq_collect_stats_norm(X, norm, acc, ws, nonfinite=None):
     """acc (float64 [d_in]) accumulates the l2 / l1 / l_inf statistic of X's columns (NORM_L2, NORM_L1, NORM_LINF)."""
     n, d_in = X.shape
     _check(lib().cmpq_collect_stats_norm(_ptr(X), dtype_code(X), n, d_in, X.stride(0) if n > 0 else d_in, int(norm),
-                                         _ptr(acc), _ptr(ws), ws.numel(), _stream()), "cmpq_collect_stats_norm")
+                                         _ptr(acc), _ptr(nonfinite), _ptr(ws), ws.numel(), _stream()),
+           "cmpq_collect_stats_norm")
 
 
 def cmpq_finalize_stats_norm(acc, norm, a):

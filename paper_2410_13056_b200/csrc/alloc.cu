@@ -5,6 +5,8 @@
 // is the number of channels that sort before it.  The count is exact, needs no sort network
 // and is spread over (channel tile) x (candidate slice) blocks that add integer partial counts.
 #include "common.cuh"
+#include "pack_bits.cuh"
+#include "select.cuh"
 
 namespace cmpq {
 
@@ -97,10 +99,24 @@ __device__ __forceinline__ uint32_t ordered_bits(float v) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Small per-layer steps that ride along with a rank-cut launch (one block, nothing else running yet):
+// the layout of the packed segments from the widths, and the start state of the radix select.
+struct CutExtras {
+    const uint8_t* bits;     // pack layout wanted: widths, and its five outputs
+    int64_t d_out;
+    int64_t* row_off;
+    int32_t* perm;
+    int64_t* seg_rows;
+    int64_t* word_off;
+    SelectState* select;     // select start state wanted: entries to take, histogram to clear
+    long long n_q;
+    unsigned int* hist;
+};
+
 // out[i] = base + #{ t in {0,1} : channel i has rank >= k_t }.  k_t >= d_in: no channel reaches cut t.
 __global__ void __launch_bounds__(kCutThreads)
 rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long long k1, int base,
-                uint8_t* __restrict__ out) {
+                uint8_t* __restrict__ out, const CutExtras x) {
     __shared__ unsigned int hist[2][256];
     __shared__ uint32_t prefix[2];
     __shared__ long long remaining[2];  // rank of the cut element among the elements matching the prefix
@@ -180,11 +196,41 @@ rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long lo
         eq1 += key == v1 ? 1 : 0;
         out[i] = (uint8_t)cls;
     }
+    if (x.select) {
+        if (tid == 0) {
+            SelectState* st = x.select;
+            st->prefix = 0; st->mask = 0; st->remaining = x.n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0;
+        }
+        for (int b = tid; b < kSelBins; b += kCutThreads) x.hist[b] = 0u;
+    }
+    if (x.bits) {
+        __syncthreads();  // warp_tot is free again
+        pack_layout_block(x.bits, d_in, x.d_out, x.row_off, x.perm, x.seg_rows, x.word_off, warp_tot);
+    }
 }
 
 cmpq_status launch_rank_cut(const float* a, int64_t d_in, int64_t k0, int64_t k1, int base, uint8_t* out,
                             cudaStream_t st) {
-    rank_cut_kernel<<<1, kCutThreads, 0, st>>>(a, d_in, (long long)k0, (long long)k1, base, out);
+    rank_cut_kernel<<<1, kCutThreads, 0, st>>>(a, d_in, (long long)k0, (long long)k1, base, out, CutExtras{});
+    return launch_status();
+}
+
+// The O_act cut of the outlier step with what else one block can prepare for it: the start state of the
+// select (state / hist / n_q) and, when bits is given, the layout of the packed segments.
+cmpq_status launch_act_cut(const float* a, int64_t d_in, int64_t n_act, uint8_t* is_act, void* select_state,
+                           long long n_q, unsigned int* hist, const uint8_t* bits, int64_t d_out, int64_t* row_off,
+                           int32_t* perm, int64_t* seg_rows, int64_t* word_off, cudaStream_t st) {
+    CutExtras x{};
+    x.select = static_cast<SelectState*>(select_state);
+    x.n_q = n_q;
+    x.hist = hist;
+    x.bits = bits;
+    x.d_out = d_out;
+    x.row_off = row_off;
+    x.perm = perm;
+    x.seg_rows = seg_rows;
+    x.word_off = word_off;
+    rank_cut_kernel<<<1, kCutThreads, 0, st>>>(a, d_in, (long long)(d_in - n_act), (long long)d_in, 0, is_act, x);
     return launch_status();
 }
 

@@ -44,6 +44,7 @@ extern "C" const char* cmpq_status_string(cmpq_status s) {
         case CMPQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case CMPQ_ERR_CUDA: return "CUDA runtime error";
         case CMPQ_ERR_INTERNAL: return "internal error";
+        case CMPQ_ERR_NONFINITE: return "an input held a NaN or an infinity";
     }
     return "unknown status";
 }

@@ -650,7 +650,8 @@ static cmpq_status quantize_impl(const void* W, cmpq_dtype dt, int64_t d_in, int
                                  const uint8_t* bits, const int32_t* rows, const int32_t* cols, int64_t nnz,
                                  int lloyd_iters, const float* sens, float* lut, uint8_t* codes, uint32_t* packed,
                                  int64_t* row_off, int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
-                                 unsigned long long* sweeps, void* ws, size_t ws_bytes, void* stream) {
+                                 unsigned long long* sweeps, int32_t* nonfinite, void* ws, size_t ws_bytes,
+                                 void* stream) {
     if (!W || !bits || !lut) return CMPQ_ERR_INVALID_ARG;
     if (!codes && !packed) return CMPQ_ERR_INVALID_ARG;
     if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
@@ -661,6 +662,7 @@ static cmpq_status quantize_impl(const void* W, cmpq_dtype dt, int64_t d_in, int
     if (!aligned_to(W, 2) || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
     if (codes && !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;  // eight codes leave in one store
     if (sens && !aligned_to(sens, 4)) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(nonfinite, 4)) return CMPQ_ERR_INVALID_ARG;
     if (packed && (!row_off || !perm || !seg_rows || !aligned_to(packed, 4) || !aligned_to(row_off, 8) ||
                    !aligned_to(perm, 4) || !aligned_to(seg_rows, 8)))
         return CMPQ_ERR_INVALID_ARG;
@@ -688,6 +690,7 @@ static cmpq_status quantize_impl(const void* W, cmpq_dtype dt, int64_t d_in, int
     a.codes = codes;
     a.inexact_rows = inexact_rows;
     a.sweeps = sweeps;
+    a.nonfinite = nonfinite;
     if (!fused_pack_ok) {
         s = sens ? launch_lloyd_weighted(a, dt, sens, st) : launch_lloyd(a, dt, st);
         if (s != CMPQ_OK || !packed) return s;
@@ -705,10 +708,10 @@ extern "C" cmpq_status cmpq_quantize_layer(const void* W, cmpq_dtype dt, int64_t
                                            const int32_t* cols, int64_t nnz, int lloyd_iters,
                                            const float* sens, float* lut, uint8_t* codes,
                                            int32_t* inexact_rows, unsigned long long* sweeps,
-                                           void* ws, size_t ws_bytes, void* stream) {
+                                           int32_t* nonfinite, void* ws, size_t ws_bytes, void* stream) {
     if (!codes) return CMPQ_ERR_INVALID_ARG;
     return quantize_impl(W, dt, d_in, d_out, ldw, bits, rows, cols, nnz, lloyd_iters, sens, lut, codes, nullptr,
-                         nullptr, nullptr, nullptr, inexact_rows, sweeps, ws, ws_bytes, stream);
+                         nullptr, nullptr, nullptr, inexact_rows, sweeps, nonfinite, ws, ws_bytes, stream);
 }
 
 extern "C" cmpq_status cmpq_quantize_layer_packed(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out,
@@ -716,9 +719,9 @@ extern "C" cmpq_status cmpq_quantize_layer_packed(const void* W, cmpq_dtype dt, 
                                                   const int32_t* cols, int64_t nnz, int lloyd_iters,
                                                   const float* sens, float* lut, uint8_t* codes, uint32_t* packed,
                                                   int64_t* row_off, int32_t* perm, int64_t* seg_rows,
-                                                  int32_t* inexact_rows, unsigned long long* sweeps, void* ws,
-                                                  size_t ws_bytes, void* stream) {
+                                                  int32_t* inexact_rows, unsigned long long* sweeps,
+                                                  int32_t* nonfinite, void* ws, size_t ws_bytes, void* stream) {
     if (!packed) return CMPQ_ERR_INVALID_ARG;
     return quantize_impl(W, dt, d_in, d_out, ldw, bits, rows, cols, nnz, lloyd_iters, sens, lut, codes, packed,
-                         row_off, perm, seg_rows, inexact_rows, sweeps, ws, ws_bytes, stream);
+                         row_off, perm, seg_rows, inexact_rows, sweeps, nonfinite, ws, ws_bytes, stream);
 }

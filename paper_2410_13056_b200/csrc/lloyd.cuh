@@ -25,6 +25,7 @@ struct LloydArgs {
     const int64_t* word_off; // [d_in] first word of every channel (with packed)
     int32_t* inexact_rows;   // optional counter
     unsigned long long* sweeps;  // optional counter of distance evaluations
+    int32_t* nonfinite;      // optional flag word: bit 1 is set when a weight is a NaN or an infinity
     // ordered formulation only: fits kept across calls on the same weights (budget sweeps).  fit_cache is
     // the block lloyd_fit_cache_bytes() describes; a channel whose fit for its width is already there
     // copies it instead of iterating, every other channel stores its fit there.
@@ -84,6 +85,10 @@ cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64
 // (a cut >= d_in is reached by nobody).
 cmpq_status launch_rank_cut(const float* a, int64_t d_in, int64_t k0, int64_t k1, int base, uint8_t* out,
                             cudaStream_t st);
+
+cmpq_status launch_act_cut(const float* a, int64_t d_in, int64_t n_act, uint8_t* is_act, void* select_state,
+                           long long n_q, unsigned int* hist, const uint8_t* bits, int64_t d_out, int64_t* row_off,
+                           int32_t* perm, int64_t* seg_rows, int64_t* word_off, cudaStream_t st);
 
 // rank[i] = position of channel i in the ascending order of (a, id).
 cmpq_status launch_rank(const float* a, int64_t d_in, int32_t* rank, cudaStream_t st);

@@ -172,6 +172,7 @@ __device__ __forceinline__ void load_channel_keys(const LloydArgs& a, int64_t ro
         // top = exponent of the largest magnitude, 2^q = smallest unit in the last place of a non-zero
         // weight.  First with a lower bound of q from the smallest magnitude's exponent and the trailing
         // zero bits every widened 16-bit value has; only a channel that fails this is examined bit by bit.
+        if (a.nonfinite && tid == 0 && amax >= 0x7f800000u) atomicOr(a.nonfinite, 2);  // a NaN or an infinity
         if (a.inexact_rows && amax != 0u) {
             const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
             const int ex_max = (int)(amax >> 23), ex_min = (int)((amin1 + 1u) >> 23);

@@ -41,6 +41,7 @@ namespace cmpq {
 
 constexpr int kSlots = 32;       // high-byte buckets refined per pass of the second histogram level
 constexpr int kSlotWords = 128;  // 256 low-byte counters of 16 bits, two per word
+constexpr uint32_t kZeroKeyOfTable = 0x8000u;  // sort key of +0
 constexpr int kStageCap = 4096;  // table entries of one pass gathered in shared memory before they are stored
 static_assert(CMPQ_MAX_D_OUT < 65536, "second-level counters and count prefixes are 16 bits wide");
 
@@ -55,7 +56,8 @@ struct Tables {
     ChannelHeader* hdr;  // [d_in]
     uint16_t* keys;      // [d_in][stride] sort keys of the distinct values, ascending
     uint16_t* cum;       // [d_in][stride] number of weights below the entry's value
-    double* sum;         // [d_in][stride] scratch of the iterate kernel for tables too large for shared memory
+    int64_t sum_stride;  // doubles per channel in `sum`
+    double* sum;         // [d_in][sum_stride] prefix sums at every eighth entry, for tables too large for shared memory
     float* lut;          // [d_in][16] centroids for the assign kernel when the caller wants no lut
     float* thr;          // [d_in][16] value thresholds of the last assignment ([0]: 1 if valid)
 };
@@ -69,7 +71,8 @@ static Tables carve_tables(Workspace& w, int64_t d_in, int64_t d_out) {
     t.hdr = w.take<ChannelHeader>(d_in);
     t.keys = w.take<uint16_t>((size_t)d_in * t.stride);
     t.cum = w.take<uint16_t>((size_t)d_in * t.stride);
-    t.sum = w.take<double>((size_t)d_in * t.stride);
+    t.sum_stride = t.stride / 8 + 2;
+    t.sum = w.take<double>((size_t)d_in * t.sum_stride);
     t.lut = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
     t.thr = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
     return t;
@@ -195,6 +198,9 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
     }
     if (lane == 0) { sh.wtop[warp] = (int)amax; sh.wulp[warp] = (int)amin1; }
+    // Every table holds an entry for +0, with count 0 if no weight is zero: a later fit of the same weights
+    // with some positions removed (set to +0) then only changes counts, never the list of entries.
+    if (tid == 0) sh.hist1[kZeroKeyOfTable >> 8] = 1;
     __syncthreads();
     if (warp == 0) {
         int flag[8], sum = 0;
@@ -227,6 +233,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
             amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
             amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
         }
+        // the largest magnitude pattern of the row tells whether any weight is a NaN or an infinity
+        if (a.nonfinite && tid == 0 && amax >= (DT == CMPQ_BF16 ? 0x7f80u : 0x7c00u)) atomicOr(a.nonfinite, 2);
         if (amax != 0u) {
             const uint32_t fmax = __float_as_uint(widen16<DT>((uint16_t)amax));
             const uint32_t fmin = __float_as_uint(widen16<DT>((uint16_t)(amin1 + 1u)));
@@ -286,13 +294,16 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         const int w0 = (int)((long long)tid * words_total / nthr);
         const int w1 = (int)((long long)(tid + 1) * words_total / nthr);
         int nz = 0, cnt = 0;
-        uint32_t occupied = 0;  // bit 2 (w - w0) + half: that counter is not zero (ranges of at most 16 words)
+        uint32_t occupied = 0;  // bit 2 (w - w0) + half: that counter makes an entry (ranges of at most 16 words)
+        const int r_zero = sh.bucket_rank[kZeroKeyOfTable >> 8] - g0;  // the counter of +0 always makes one
+        const int w_zero = (r_zero >= 0 && r_zero < nslots) ? r_zero * kSlotWords : -1;
         for (int w = w0; w < w1; ++w) {
             const uint32_t word = h2[w];
             const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-            nz += (c0 ? 1 : 0) + (c1 ? 1 : 0);
+            const bool e0 = c0 != 0 || w == w_zero, e1 = c1 != 0;
+            nz += (e0 ? 1 : 0) + (e1 ? 1 : 0);
             cnt += c0 + c1;
-            if (w - w0 < 16) occupied |= ((c0 ? 1u : 0u) | (c1 ? 2u : 0u)) << (2 * (w - w0));
+            if (w - w0 < 16) occupied |= ((e0 ? 1u : 0u) | (e1 ? 2u : 0u)) << (2 * (w - w0));
         }
         int inz = nz, icnt = cnt;
 #pragma unroll
@@ -331,10 +342,10 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         } else {
             for (int w = w0; w < w1; ++w) {
                 const uint32_t word = h2[w];
-                if (word) {
+                if (word || w == w_zero) {
                     const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
                     const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-                    if (c0) { out_keys[run_nz] = (uint16_t)kb; out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c0; }
+                    if (c0 || w == w_zero) { out_keys[run_nz] = (uint16_t)kb; out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c0; }
                     if (c1) { out_keys[run_nz] = (uint16_t)(kb | 1u); out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c1; }
                 }
             }
@@ -421,6 +432,7 @@ struct IterArgs {
     const int64_t* row_ptr;
     const int32_t* cols;
     int32_t* inexact_rows;
+    const int32_t* nonfinite;  // optional flag word of the call: once it is set the iterations are skipped
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -594,94 +606,49 @@ __device__ __forceinline__ int group_sum(unsigned gmask, int v) {
 
 // W'' differs from W' only at the removed positions (the entries kept as outliers): the table of a row of
 // W'' is the table of the same row of W' with the counts of the removed values moved to the value +0.
-// One group of lanes does that in place on a writable copy (shared or global memory): keys[0..M) ascending,
-// cum[0..M] count prefixes with cum[M] = N.  Removed positions are taken kPatchChunk at a time; every pass
-// first makes sure an entry for +0 exists (entries above it move up by one, highest first), then adjusts
-// counts and prefixes and closes the gaps of entries whose count fell to zero (an entry never moves up, so
-// reading a chunk of sixteen entries before writing it keeps the pass in place).  Returns the new M.
-__device__ int patch_table(uint16_t* keys, uint16_t* cum, int M, int N, const uint16_t* __restrict__ wrow,
-                           const int32_t* __restrict__ cols, int nrem, uint32_t* rk) {
-    const unsigned gmask = group_mask();
-    const int gl = threadIdx.x & 15, gbase = threadIdx.x & 16;
-    const uint32_t kZeroKey = 0x8000u;  // sort key of +0
-    for (int c0 = 0; c0 < nrem; c0 += kPatchChunk) {
-        const int nr = nrem - c0 < kPatchChunk ? nrem - c0 : kPatchChunk;
-        for (int i = gl; i < nr; i += kGroup) {
-            uint32_t h = wrow[cols[c0 + i]];
-            if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
-            rk[i] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
-        }
-        __syncwarp(gmask);
-        int lo = 0, hi = M;  // where +0 sits in the table, or would sit
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if ((uint32_t)keys[mid] >= kZeroKey) hi = mid; else lo = mid + 1;
-        }
-        const int pos0 = lo;
-        const bool present = pos0 < M && (uint32_t)keys[pos0] == kZeroKey;
-        __syncwarp(gmask);
-        if (!present) {  // entries pos0 .. M (the sentinel included) move up by one, highest chunk first
-            for (int base = pos0 + ((M - pos0) / kGroup) * kGroup; base >= pos0; base -= kGroup) {
-                const int j = base + gl;
-                const bool in = j <= M;
-                const uint16_t k = in ? keys[j] : (uint16_t)0, c = in ? cum[j] : (uint16_t)0;
-                __syncwarp(gmask);
-                if (in) { keys[j + 1] = k; cum[j + 1] = c; }
-                __syncwarp(gmask);
-            }
-            if (gl == 0) keys[pos0] = (uint16_t)kZeroKey;  // cum[pos0] already is the number of weights below +0
-            M += 1;
-            __syncwarp(gmask);
-        }
-        int deleted = 0;  // entries dropped so far in this pass
-        for (int base = 0; base < M; base += kGroup) {
-            const int i = base + gl;
-            const bool valid = i < M;
-            uint32_t key = kZeroKey;
-            int cnt = 0, below = 0;
-            if (valid) {
-                key = keys[i];
-                below = (int)cum[i];
-                cnt = (int)cum[i + 1] - below;
-                int eq = 0, lt = 0;
+// Every table has an entry for +0 and entries may have count 0, so the list of keys does not change: only
+// the count prefixes do, and the prefix of an entry with key k becomes
+//     cum(k) - #{removed weights with key < k} + (k > key of +0 ? number of removed weights : 0) ,
+// which is applied while the table is copied.  Copies keys[0..M) and cum[0..M] (eight entries per lane and
+// step), adjusting for the `nr` removed keys in rk.
+__device__ __forceinline__ void copy_table_removing(uint16_t* w_keys, uint16_t* w_cum, const uint16_t* g_keys,
+                                                    const uint16_t* g_cum, int M, const uint32_t* rk, int nr) {
+    const int gl = threadIdx.x & 15;
+    for (int i = gl; i < (M + 1 + 7) / 8; i += kGroup) {  // with the sentinel (key 0xffff, cum[M] = d_out)
+        // plain loads: after the first pass over a row the source is the copy itself, which may be shared memory
+        const uint4 kv = reinterpret_cast<const uint4*>(g_keys)[i];
+        uint4 cv = reinterpret_cast<const uint4*>(g_cum)[i];
+        if (nr > 0) {
+            const uint32_t kw[4] = {kv.x, kv.y, kv.z, kv.w};
+            uint32_t cw[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t k0 = kw[q] & 0xffffu, k1 = kw[q] >> 16;
+                int d0 = k0 > kZeroKeyOfTable ? nr : 0, d1 = k1 > kZeroKeyOfTable ? nr : 0;
                 for (int r = 0; r < nr; ++r) {
                     const uint32_t k = rk[r];
-                    eq += k == key ? 1 : 0;
-                    lt += k < key ? 1 : 0;
+                    d0 -= k < k0 ? 1 : 0;
+                    d1 -= k < k1 ? 1 : 0;
                 }
-                cnt -= eq;
-                below -= lt;
-                if (key == kZeroKey) cnt += nr;   // the removed weights are zeros now
-                if (key > kZeroKey) below += nr;
+                cw[q] = ((cw[q] + (uint32_t)d0) & 0xffffu) | ((((cw[q] >> 16) + (uint32_t)d1) & 0xffffu) << 16);
             }
-            const bool keep = valid && cnt > 0;
-            const unsigned gone = (__ballot_sync(gmask, valid && !keep) >> gbase) & 0xffffu;
-            __syncwarp(gmask);  // every lane has read its entry (and the next prefix) before anyone writes
-            if (keep) {
-                const int o = i - deleted - __popc(gone & ((1u << gl) - 1u));
-                keys[o] = (uint16_t)key;
-                cum[o] = (uint16_t)below;
-            }
-            deleted += __popc(gone);
-            __syncwarp(gmask);
+            cv = make_uint4(cw[0], cw[1], cw[2], cw[3]);
         }
-        M -= deleted;
-        if (gl == 0) { keys[M] = 0xffffu; cum[M] = (uint16_t)N; }
-        __syncwarp(gmask);
+        reinterpret_cast<uint4*>(w_keys)[i] = kv;
+        reinterpret_cast<uint4*>(w_cum)[i] = cv;
     }
-    return M;
 }
 
 // The exactness test of the table kernel (see load_channel_keys) on a finished table.
 template <int DT>
-__device__ void count_if_inexact(const uint16_t* keys, int M, int N, int32_t* inexact_rows) {
+__device__ void count_if_inexact(const uint16_t* keys, const uint16_t* cum, int M, int N, int32_t* inexact_rows) {
     const unsigned gmask = group_mask();
     const int gl = threadIdx.x & 15;
     uint32_t amax = 0u;
     int q = 100000;
     for (int i = gl; i < M; i += kGroup) {
         const uint32_t ub = __float_as_uint(value_of_key16<DT>(keys[i])) & 0x7fffffffu;
-        if (ub) {
+        if (ub && cum[i + 1] != cum[i]) {  // values that still occur
             amax = max(amax, ub);
             const int ex = (int)(ub >> 23);
             const uint32_t m = ub & 0x7fffffu;
@@ -722,30 +689,37 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, const int K, uns
     double* coarse = s_coarse;
     bool staged = true;
     if (patch && nrem >= N) {  // every position removed: an all-zero channel
-        if (gl == 0) { s_keys[0] = 0x8000u; s_cum[0] = 0; s_cum[1] = (uint16_t)N; }
+        if (gl == 0) { s_keys[0] = (uint16_t)kZeroKeyOfTable; s_cum[0] = 0; s_cum[1] = (uint16_t)N; }
     } else {
         const ChannelHeader h = from.hdr[row];
-        M = h.M < 1 ? 1 : (h.M > N ? N : h.M);  // 1 <= M <= N by construction
+        M = h.M < 1 ? 1 : (h.M > N + 1 ? N + 1 : h.M);  // 1 <= M <= N + 1 by construction (the entry of +0 may be empty)
         const uint16_t* g_keys = from.keys + row * from.stride;  // rows are 16-byte aligned, padded to 8 entries
         const uint16_t* g_cum = from.cum + row * from.stride;
-        staged = M + (nrem > 0 ? 1 : 0) <= a.cap;  // removing weights can add the entry of +0
+        staged = M <= a.cap;
         uint16_t* w_keys = staged ? s_keys : a.t.keys + row * a.t.stride;
         uint16_t* w_cum = staged ? s_cum : a.t.cum + row * a.t.stride;
-        if (staged || patch) {  // copy: into shared memory, or into this launch's own table for patching
-            for (int i = gl; i < (M + 7) / 8; i += kGroup)
-                reinterpret_cast<uint4*>(w_keys)[i] = __ldg(reinterpret_cast<const uint4*>(g_keys) + i);
-            for (int i = gl; i < (M + 1 + 7) / 8; i += kGroup)  // with the sentinel cum[M] = d_out
-                reinterpret_cast<uint4*>(w_cum)[i] = __ldg(reinterpret_cast<const uint4*>(g_cum) + i);
-            __syncwarp(gmask);
-            if (nrem > 0) M = patch_table(w_keys, w_cum, M, N, a.W + row * a.ldw, a.cols + p0, (int)nrem, s_removed);
-            if (patch && a.inexact_rows && h.suspect) count_if_inexact<DT>(w_keys, M, N, a.inexact_rows);
+        if (staged || patch) {  // copy: into shared memory, or into this launch's own table when patching
+            int done = 0;
+            do {  // removed weights are taken kPatchChunk at a time (one pass in all but pathological rows)
+                const int nr = (int)(nrem - done < kPatchChunk ? nrem - done : kPatchChunk);
+                for (int i = gl; i < nr; i += kGroup) {
+                    uint32_t hh = a.W[row * a.ldw + a.cols[p0 + done + i]];
+                    if (hh == 0x8000u) hh = 0u;  // -0 and +0 are the same point
+                    s_removed[i] = (hh & 0x8000u) ? (~hh & 0xffffu) : (hh | 0x8000u);
+                }
+                __syncwarp(gmask);
+                copy_table_removing(w_keys, w_cum, done == 0 ? g_keys : w_keys, done == 0 ? g_cum : w_cum, M, s_removed, nr);
+                __syncwarp(gmask);
+                done += nr;
+            } while (done < nrem);
+            if (patch && a.inexact_rows && h.suspect) count_if_inexact<DT>(w_keys, w_cum, M, N, a.inexact_rows);
             keys = w_keys;
             cum = w_cum;
         } else {
             keys = g_keys;
             cum = g_cum;
         }
-        if (!staged) coarse = a.t.sum + row * a.t.stride;  // global scratch for tables too large to stage
+        if (!staged) coarse = a.t.sum + row * a.t.sum_stride;  // global scratch for tables too large to stage
     }
     __syncwarp(gmask);
     if (staged)  // nothing past the table
@@ -896,6 +870,10 @@ lloyd_iterate_kernel(const IterArgs a) {
     const int64_t row = (int64_t)blockIdx.x * (kIterWarps * 2) + group;
     if (row >= a.d_in) return;
     if (a.skip_row && a.skip_row[row]) return;
+    // Non-finite inputs were found by an earlier kernel of the call: its outputs are unspecified anyway, and
+    // although every loop below is bounded whatever the values (bisections halve an interval, the update
+    // loop counts to the iteration limit), there is nothing worth computing.
+    if (a.nonfinite && *a.nonfinite) return;
     const unsigned gmask = group_mask();
     const int bits = a.bits[row];
     const int gl = threadIdx.x & 15;
@@ -1515,6 +1493,7 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
     ia.iters = args.iters;
     ia.lut = args.lut ? args.lut : t.lut;
     ia.sweeps = args.sweeps;
+    ia.nonfinite = args.nonfinite;
     if (patch_from) {
         ia.src = *patch_from;
         ia.W = args.W;
@@ -1564,7 +1543,9 @@ cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tab
 // from the provisional one (see patch_table), so nothing is read from the weights and counted again.
 
 // args: the final fit (row_ptr / cols = the removed positions, skip_row unused).  prov_tables: the
-// tables the provisional fit left (read only); tables: scratch of the final fit.
+// tables the provisional fit left; tables: scratch of the final fit for the channels whose table does not
+// fit in shared memory.  tables == prov_tables is allowed: those channels are then patched in place (the
+// update is element-wise), which destroys the provisional tables.
 cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, void* prov_tables, void* tables,
                                          size_t tables_bytes, cudaStream_t st) {
     if (!prov_tables || !tables || tables_bytes < lloyd_tables_bytes(args.d_in, args.d_out)) return CMPQ_ERR_WORKSPACE;

@@ -21,10 +21,6 @@
 
 namespace cmpq {
 
-__global__ void select_init_kernel(SelectState* st, long long n_q) {
-    st->prefix = 0; st->mask = 0; st->remaining = n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0;
-}
-
 // hist[d] += number of errors in non-act rows whose fixed bits match the prefix and whose
 // digit (err >> shift) & (bins-1) equals d.  One block handles whole rows.
 __global__ void __launch_bounds__(kSelThreads)
@@ -220,9 +216,16 @@ emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const float* __restrict
     }
 }
 
+// packed outputs of a call that also packs (all NULL otherwise)
+struct PackOut {
+    uint32_t* packed;
+    int64_t* row_off;
+    int32_t* perm;
+    int64_t* seg_rows;
+};
+
 struct OutlierWs {
-    float* err;
-    int32_t* rank;
+    float* err;     // one fp32 error per weight: only the all-pairs formulation materialises them
     uint8_t* is_act;
     unsigned int* hist;
     SelectState* state;
@@ -230,13 +233,15 @@ struct OutlierWs {
     int32_t* eq;
     int32_t* take_eq;
     int64_t* row_start;
-    char* tables;  // scratch of the ordered K-means
+    char* tables;  // value tables of the ordered K-means
 };
 
+// The layout depends on the assignment method selected when the call is made: the ordered formulation keeps
+// value tables (about 5 bytes per weight), the all-pairs formulation an fp32 error per weight.
 static OutlierWs carve(Workspace& w, int64_t d_in, int64_t d_out) {
+    const bool all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
     OutlierWs o;
-    o.err = w.take<float>((size_t)d_in * (size_t)d_out);
-    o.rank = w.take<int32_t>(d_in);
+    o.err = all_pairs ? w.take<float>((size_t)d_in * (size_t)d_out) : nullptr;
     o.is_act = w.take<uint8_t>(d_in);
     o.hist = w.take<unsigned int>(kSelBins);
     o.state = w.take<SelectState>(1);
@@ -244,7 +249,7 @@ static OutlierWs carve(Workspace& w, int64_t d_in, int64_t d_out) {
     o.eq = w.take<int32_t>(d_in);
     o.take_eq = w.take<int32_t>(d_in);
     o.row_start = w.take<int64_t>(d_in + 1);
-    o.tables = w.take<char>(lloyd_tables_bytes(d_in, d_out));
+    o.tables = all_pairs ? nullptr : w.take<char>(lloyd_tables_bytes(d_in, d_out));
     return o;
 }
 
@@ -257,7 +262,8 @@ size_t outliers_ws_bytes(int64_t d_in, int64_t d_out) {
 cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw, const float* a,
                          const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
                          int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st,
-                         void* fit_cache = nullptr, bool tables_ready = false);
+                         void* fit_cache = nullptr, bool tables_ready = false, const PackOut* po = nullptr,
+                         int64_t* word_off = nullptr, int32_t* nonfinite = nullptr);
 static cmpq_status check_extract_args(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
                                       const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
                                       int lloyd_iters, const int32_t* rows, const int32_t* cols,
@@ -276,14 +282,16 @@ extern "C" cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64
                                              int64_t ldw, const float* a, const uint8_t* bits,
                                              int64_t n_act, int64_t n_q, int lloyd_iters,
                                              int32_t* rows, int32_t* cols, uint16_t* vals,
-                                             int64_t nnz_out, void* ws, size_t ws_bytes, void* stream) {
+                                             int64_t nnz_out, int32_t* nonfinite, void* ws, size_t ws_bytes,
+                                             void* stream) {
+    if (!aligned_to(nonfinite, 4)) return CMPQ_ERR_INVALID_ARG;
     const cmpq_status chk = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
     if (chk != CMPQ_OK) return chk;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < outliers_ws_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
     Workspace wsp(ws, ws_bytes);
     OutlierWs o = carve(wsp, d_in, d_out);
     return extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, o,
-                        static_cast<cudaStream_t>(stream));
+                        static_cast<cudaStream_t>(stream), nullptr, false, nullptr, nullptr, nonfinite);
 }
 
 namespace cmpq {
@@ -291,13 +299,16 @@ namespace cmpq {
 cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw, const float* a,
                          const uint8_t* bits, int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
                          int32_t* cols, uint16_t* vals, int64_t nnz_out, const OutlierWs& o, cudaStream_t st,
-                         void* fit_cache, bool tables_ready) {
+                         void* fit_cache, bool tables_ready, const PackOut* po, int64_t* word_off, int32_t* nonfinite) {
     const bool all_pairs = lloyd_assignment() == CMPQ_ASSIGN_ALL_PAIRS;
     const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
     const uint16_t* Wp = static_cast<const uint16_t*>(W);
 
-    // O_act: the channels of rank >= d_in - n_act in the ascending order of (a, id)
-    cmpq_status s = launch_rank_cut(a, d_in, d_in - n_act, d_in, 0, o.is_act, st);
+    // O_act: the channels of rank >= d_in - n_act in the ascending order of (a, id).  The same block also
+    // resets the select and, for a call that packs, lays out the packed segments (widths alone decide it).
+    cmpq_status s = launch_act_cut(a, d_in, n_act, o.is_act, o.state, (long long)n_q, o.hist, po ? bits : nullptr, d_out,
+                                   po ? po->row_off : nullptr, po ? po->perm : nullptr, po ? po->seg_rows : nullptr,
+                                   word_off, st);
     if (s != CMPQ_OK) return s;
 
     if (n_q > 0) {
@@ -312,12 +323,11 @@ cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_o
         la.err = all_pairs ? o.err : nullptr;
         la.fit_cache = fit_cache;
         la.tables_ready = tables_ready;
+        la.nonfinite = nonfinite;
         s = all_pairs ? launch_lloyd(la, dt, st) : launch_lloyd_ordered(la, dt, o.tables, tables_bytes, st);
         if (s != CMPQ_OK) return s;
     }
 
-    select_init_kernel<<<1, 1, 0, st>>>(o.state, (long long)n_q);
-    if (cudaMemsetAsync(o.hist, 0, kSelBins * sizeof(unsigned int), st) != cudaSuccess) return CMPQ_ERR_CUDA;
     if (n_q > 0) {
         int sms = sm_count();
         if (sms <= 0) return CMPQ_ERR_CUDA;
@@ -371,18 +381,15 @@ static cmpq_status check_extract_args(const void* W, cmpq_dtype dt, int64_t d_in
     return CMPQ_OK;
 }
 
-// work space of the fused call: the outlier step's, then the final fit's row index and tables
+// Work space of the fused call: the outlier step's.  The final fit derives its tables from the provisional
+// ones: in shared memory for nearly every channel, in place in the provisional tables for the others.
 struct FusedWs {
     OutlierWs o;
-    int64_t* row_ptr;
-    char* tables;
 };
 
 static FusedWs carve_fused(Workspace& w, int64_t d_in, int64_t d_out) {
     FusedWs f;
     f.o = carve(w, d_in, d_out);
-    f.row_ptr = w.take<int64_t>(d_in + 1);
-    f.tables = w.take<char>(lloyd_tables_bytes(d_in, d_out));
     return f;
 }
 
@@ -401,13 +408,6 @@ cmpq_status launch_pack_layout(const uint8_t* bits, int64_t d_in, int64_t d_out,
 cmpq_status launch_pack_codes(const uint8_t* codes, const uint8_t* bits, int64_t d_in, int64_t d_out,
                               const int64_t* word_off, uint32_t* packed, cudaStream_t st);
 
-// packed outputs of a call that also packs (all NULL otherwise)
-struct PackOut {
-    uint32_t* packed;
-    int64_t* row_off;
-    int32_t* perm;
-    int64_t* seg_rows;
-};
 
 }  // namespace cmpq
 
@@ -437,11 +437,11 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
                                          const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
                                          int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
                                          int64_t nnz_out, float* lut, uint8_t* codes, int32_t* inexact_rows,
-                                         unsigned long long* sweeps, void* ws, size_t ws_bytes, void* cache,
-                                         cudaStream_t st, const PackOut* po = nullptr) {
+                                         unsigned long long* sweeps, int32_t* nonfinite, void* ws, size_t ws_bytes,
+                                         void* cache, cudaStream_t st, const PackOut* po = nullptr) {
     cmpq_status s = check_extract_args(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out);
     if (s != CMPQ_OK) return s;
-    if (!lut || !aligned_to(lut, 4)) return CMPQ_ERR_INVALID_ARG;
+    if (!lut || !aligned_to(lut, 4) || !aligned_to(nonfinite, 4)) return CMPQ_ERR_INVALID_ARG;
     if (!codes && !po) return CMPQ_ERR_INVALID_ARG;
     if (codes && !aligned_to(codes, 8)) return CMPQ_ERR_INVALID_ARG;
     if (po && (!po->packed || !po->row_off || !po->perm || !po->seg_rows || !aligned_to(po->packed, 4) ||
@@ -454,18 +454,15 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
     Workspace wsp(ws, ws_bytes);
     FusedWs f = carve_fused(wsp, d_in, d_out);
     int64_t* word_off = po ? wsp.take<int64_t>(d_in) : nullptr;
-    if (po) {  // the layout of the packed segments depends on the widths alone
-        s = launch_pack_layout(bits, d_in, d_out, po->row_off, po->perm, po->seg_rows, word_off, st);
-        if (s != CMPQ_OK) return s;
-    }
     void* fit_cache = nullptr;
-    if (cache && ordered) {  // the provisional fit reads the cache's tables instead of building its own
+    char* final_tables = f.o.tables;  // the provisional tables are patched in place ...
+    if (cache && ordered) {  // ... unless they are the cache's, which stay as they are: the work space's serve
         const SweepCache c = carve_sweep(cache, d_in, d_out);
         f.o.tables = c.tables;
         fit_cache = c.fits;
     }
     s = extract_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out, f.o, st,
-                     fit_cache, fit_cache != nullptr);
+                     fit_cache, fit_cache != nullptr, po, word_off, nonfinite);
     if (s != CMPQ_OK) return s;
     // the list is sorted by row, so the first list position of a row is the start of the row's slice of
     // the output: the row index of the final fit is the scan the outlier step has just made
@@ -480,6 +477,7 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
     la.codes = codes;
     la.inexact_rows = inexact_rows;
     la.sweeps = sweeps;
+    la.nonfinite = nonfinite;
     const size_t tables_bytes = lloyd_tables_bytes(d_in, d_out);
     if (!ordered) {
         s = launch_lloyd(la, dt, st);
@@ -492,8 +490,8 @@ static cmpq_status protect_quantize_impl(const void* W, cmpq_dtype dt, int64_t d
     }
     // the provisional fit ran (and left its tables) only when entries had to be selected; a sweep cache
     // holds the tables of all channels in any case
-    if (n_q > 0 || fit_cache) return launch_lloyd_ordered_patched(la, dt, f.o.tables, f.tables, tables_bytes, st);
-    return launch_lloyd_ordered(la, dt, f.tables, tables_bytes, st);
+    if (n_q > 0 || fit_cache) return launch_lloyd_ordered_patched(la, dt, f.o.tables, final_tables, tables_bytes, st);
+    return launch_lloyd_ordered(la, dt, final_tables, tables_bytes, st);
 }
 
 }  // namespace cmpq
@@ -503,10 +501,10 @@ extern "C" cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, i
                                                  int64_t n_act, int64_t n_q, int lloyd_iters, int32_t* rows,
                                                  int32_t* cols, uint16_t* vals, int64_t nnz_out, float* lut,
                                                  uint8_t* codes, int32_t* inexact_rows,
-                                                 unsigned long long* sweeps, void* ws, size_t ws_bytes,
-                                                 void* stream) {
+                                                 unsigned long long* sweeps, int32_t* nonfinite, void* ws,
+                                                 size_t ws_bytes, void* stream) {
     return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
-                                 lut, codes, inexact_rows, sweeps, ws, ws_bytes, nullptr,
+                                 lut, codes, inexact_rows, sweeps, nonfinite, ws, ws_bytes, nullptr,
                                  static_cast<cudaStream_t>(stream));
 }
 
@@ -516,11 +514,11 @@ extern "C" cmpq_status cmpq_protect_quantize_pack(const void* W, cmpq_dtype dt, 
                                                   int32_t* cols, uint16_t* vals, int64_t nnz_out, float* lut,
                                                   uint8_t* codes, uint32_t* packed, int64_t* row_off,
                                                   int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
-                                                  unsigned long long* sweeps, void* ws, size_t ws_bytes,
-                                                  void* stream) {
+                                                  unsigned long long* sweeps, int32_t* nonfinite, void* ws,
+                                                  size_t ws_bytes, void* stream) {
     const PackOut po{packed, row_off, perm, seg_rows};
     return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
-                                 lut, codes, inexact_rows, sweeps, ws, ws_bytes, nullptr,
+                                 lut, codes, inexact_rows, sweeps, nonfinite, ws, ws_bytes, nullptr,
                                  static_cast<cudaStream_t>(stream), &po);
 }
 
@@ -530,8 +528,9 @@ extern "C" size_t cmpq_sweep_cache_bytes(int64_t d_in, int64_t d_out) {
 }
 
 extern "C" cmpq_status cmpq_sweep_begin(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
-                                        int lloyd_iters, void* cache, size_t cache_bytes, void* stream) {
-    if (!W || (dt != CMPQ_F16 && dt != CMPQ_BF16) || !aligned_to(W, 2)) return CMPQ_ERR_INVALID_ARG;
+                                        int lloyd_iters, int32_t* nonfinite, void* cache, size_t cache_bytes,
+                                        void* stream) {
+    if (!W || (dt != CMPQ_F16 && dt != CMPQ_BF16) || !aligned_to(W, 2) || !aligned_to(nonfinite, 4)) return CMPQ_ERR_INVALID_ARG;
     if (d_in < 1 || d_in > CMPQ_MAX_D_IN || d_out < 1 || d_out > CMPQ_MAX_D_OUT || ldw < d_out) return CMPQ_ERR_INVALID_ARG;
     if (lloyd_iters < 0 || lloyd_iters > CMPQ_MAX_LLOYD_ITERS) return CMPQ_ERR_INVALID_ARG;
     if (!cache || !aligned_to(cache, 256) || cache_bytes < sweep_cache_bytes(d_in, d_out)) return CMPQ_ERR_WORKSPACE;
@@ -540,6 +539,7 @@ extern "C" cmpq_status cmpq_sweep_begin(const void* W, cmpq_dtype dt, int64_t d_
     LloydArgs la{};
     la.W = static_cast<const uint16_t*>(W);
     la.d_in = d_in; la.d_out = d_out; la.ldw = ldw;
+    la.nonfinite = nonfinite;
     cmpq_status s = launch_lloyd_tables(la, dt, c.tables, lloyd_tables_bytes(d_in, d_out), st);
     if (s != CMPQ_OK) return s;
     return launch_fit_cache_clear(c.fits, d_in, lloyd_iters, st);
@@ -556,6 +556,6 @@ extern "C" cmpq_status cmpq_sweep_budget(const void* W, cmpq_dtype dt, int64_t d
         cache_bytes < sweep_cache_bytes(d_in, d_out))
         return CMPQ_ERR_WORKSPACE;
     return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
-                                 lut, codes, inexact_rows, sweeps, ws, ws_bytes, cache,
+                                 lut, codes, inexact_rows, sweeps, nullptr, ws, ws_bytes, cache,
                                  static_cast<cudaStream_t>(stream));
 }

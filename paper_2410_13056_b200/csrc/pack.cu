@@ -16,63 +16,12 @@ size_t pack_ws_bytes(int64_t d_in, int64_t) {
     return round_up((size_t)d_in * sizeof(int64_t), 256);
 }
 
-// Single block: segment sizes, perm, row_off (segment order) and word_off (by channel id).
-// Thread t owns the consecutive channels [t R, t R + R); the three per-width counts travel through
-// one block-wide scan packed into a 64-bit integer (21 bits each, d_in <= 2^18).
 __global__ void __launch_bounds__(1024)
 pack_layout_kernel(const uint8_t* __restrict__ bits, int64_t d_in, int64_t d_out,
                    int64_t* __restrict__ row_off, int32_t* __restrict__ perm,
                    int64_t* __restrict__ seg_rows, int64_t* __restrict__ word_off) {
     __shared__ unsigned long long warp_tot[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    const int64_t R = (d_in + blockDim.x - 1) / blockDim.x;
-    const int64_t i0 = (int64_t)tid * R;
-    const int64_t i1 = i0 + R < d_in ? i0 + R : d_in;
-    unsigned long long mine = 0;
-    for (int64_t i = i0; i < i1; ++i) {
-        int c = bits[i];
-        if (c >= 2 && c <= 4) mine += 1ull << (21 * (c - 2));
-    }
-    unsigned long long incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    unsigned long long base = 0, total = 0;
-    for (int w = 0; w < nwarps; ++w) {
-        unsigned long long t = warp_tot[w];
-        if (w < warp) base += t;
-        total += t;
-    }
-    const unsigned long long before = base + incl - mine;
-    long long seen[3], count[3], words[3], seg_base[3], seg_word_base[3];
-    long long rb = 0, wb = 0;
-#pragma unroll
-    for (int sgm = 0; sgm < 3; ++sgm) {
-        seen[sgm] = (long long)((before >> (21 * sgm)) & 0x1fffffull);
-        count[sgm] = (long long)((total >> (21 * sgm)) & 0x1fffffull);
-        words[sgm] = (d_out * (sgm + 2) + 31) / 32;
-        seg_base[sgm] = rb;
-        seg_word_base[sgm] = wb;
-        rb += count[sgm];
-        wb += count[sgm] * words[sgm];
-    }
-    if (tid < 3) seg_rows[tid] = count[tid];
-    if (tid == 0) row_off[d_in] = wb;
-    for (int64_t i = i0; i < i1; ++i) {
-        int c = bits[i];
-        if (c < 2 || c > 4) continue;
-        int sgm = c - 2;
-        long long pos = seen[sgm]++;
-        long long r = seg_base[sgm] + pos;
-        long long off = seg_word_base[sgm] + pos * words[sgm];
-        perm[r] = (int32_t)i;
-        row_off[r] = off;
-        word_off[i] = off;
-    }
+    pack_layout_block(bits, d_in, d_out, row_off, perm, seg_rows, word_off, warp_tot);
 }
 
 // One thread packs 32 consecutive codes of one channel into C consecutive words.

@@ -61,13 +61,18 @@ template <int NORM>
 __device__ __forceinline__ float fold(float x, float acc) {
     if (NORM == CMPQ_NORM_L2) return fmaf(x, x, acc);
     if (NORM == CMPQ_NORM_L1) return acc + fabsf(x);
-    return fmaxf(acc, fabsf(x));
+    // the larger magnitude, as bit patterns (for finite values the order is the same): a NaN pattern sorts
+    // above every number and so survives to the end, where it is reported
+    return __uint_as_float(max(__float_as_uint(acc), __float_as_uint(x) & 0x7fffffffu));
 }
 
 // Two partial results combined: a sum, or a maximum for l_inf.
+// the larger of two non-negative values, a NaN in either winning
+__device__ __forceinline__ double max_keep_nan(double a, double b) { return (a != a) ? a : ((b != b || b > a) ? b : a); }
+
 template <int NORM>
 __device__ __forceinline__ double join(double a, double b) {
-    return NORM == CMPQ_NORM_LINF ? fmax(a, b) : a + b;
+    return NORM == CMPQ_NORM_LINF ? max_keep_nan(a, b) : a + b;
 }
 
 template <int DT, int NORM>
@@ -165,18 +170,22 @@ stats_partial_scalar_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, in
 }
 
 // sumsq[j] += sum over row blocks (ascending) of partial[rb][j]   (l_inf: the maximum instead of the sum)
+// A NaN or an infinity among the activations of a column (or an fp32 square beyond the fp32 range) makes
+// the column's partial result non-finite: bit 0 of *nonfinite is set (nonfinite may be NULL).
 __global__ void stats_combine_kernel(const double* __restrict__ partial, int64_t row_blocks,
-                                     int64_t padded_cols, int64_t d_in, double* __restrict__ sumsq, int take_max) {
+                                     int64_t padded_cols, int64_t d_in, double* __restrict__ sumsq, int take_max,
+                                     int32_t* nonfinite) {
     int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= d_in) return;
     double s = 0.0;
     if (take_max) {
-        for (int64_t rb = 0; rb < row_blocks; ++rb) s = fmax(s, partial[rb * padded_cols + j]);
-        sumsq[j] = fmax(sumsq[j], s);
+        for (int64_t rb = 0; rb < row_blocks; ++rb) s = max_keep_nan(s, partial[rb * padded_cols + j]);
+        sumsq[j] = max_keep_nan(sumsq[j], s);
     } else {
         for (int64_t rb = 0; rb < row_blocks; ++rb) s += partial[rb * padded_cols + j];
         sumsq[j] += s;
     }
+    if (nonfinite && !(fabs(s) <= 1.7976931348623157e308)) atomicOr(nonfinite, 1);
 }
 
 __global__ void stats_finalize_kernel(const double* __restrict__ sumsq, int64_t d_in,
@@ -204,7 +213,7 @@ static void launch_partial(const uint16_t* Xp, cmpq_dtype dt, bool vec, dim3 gri
 // Launches the two statistic kernels with `partial` as scratch (row_blocks * tiles * 256 doubles).
 cmpq_status launch_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
                                       int64_t ldx, cmpq_norm norm, double* sumsq, double* partial,
-                                      int64_t row_blocks, cudaStream_t st) {
+                                      int64_t row_blocks, cudaStream_t st, int32_t* nonfinite) {
     const int64_t ct = col_tiles(d_in);
     const int64_t rows_per_block = (n_tokens + row_blocks - 1) / row_blocks;
     const bool vec = aligned_to(X, 16) && (ldx % 8 == 0) && (d_in % 8 == 0);
@@ -214,14 +223,14 @@ cmpq_status launch_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_to
     else if (norm == CMPQ_NORM_L1) launch_partial<CMPQ_NORM_L1>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
     else launch_partial<CMPQ_NORM_LINF>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
     stats_combine_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, st>>>(partial, row_blocks, ct * kTileCols, d_in, sumsq,
-                                                                          norm == CMPQ_NORM_LINF);
+                                                                          norm == CMPQ_NORM_LINF, nonfinite);
     return launch_status();
 }
 
 cmpq_status launch_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
                                  int64_t ldx, double* sumsq, double* partial, int64_t row_blocks,
                                  cudaStream_t st) {
-    return launch_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, partial, row_blocks, st);
+    return launch_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, partial, row_blocks, st, nullptr);
 }
 
 const void* stats_kernel_address() {
@@ -239,25 +248,34 @@ int64_t stats_row_blocks(int64_t d_in, int64_t n_tokens) {
 using namespace cmpq;
 
 extern "C" cmpq_status cmpq_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
-                                               int64_t ldx, cmpq_norm norm, double* acc, void* ws, size_t ws_bytes,
-                                               void* stream) {
+                                               int64_t ldx, cmpq_norm norm, double* acc, int32_t* nonfinite, void* ws,
+                                               size_t ws_bytes, void* stream) {
     if (!acc || n_tokens < 0 || d_in < 1 || d_in > CMPQ_MAX_D_IN || ldx < d_in) return CMPQ_ERR_INVALID_ARG;
     if (dt != CMPQ_F16 && dt != CMPQ_BF16) return CMPQ_ERR_INVALID_ARG;
     if (norm != CMPQ_NORM_L2 && norm != CMPQ_NORM_L1 && norm != CMPQ_NORM_LINF) return CMPQ_ERR_INVALID_ARG;
     if (n_tokens > 0 && !X) return CMPQ_ERR_INVALID_ARG;
-    if (!aligned_to(X, 2) || !aligned_to(acc, 8)) return CMPQ_ERR_INVALID_ARG;
+    if (!aligned_to(X, 2) || !aligned_to(acc, 8) || !aligned_to(nonfinite, 4)) return CMPQ_ERR_INVALID_ARG;
     if (!ws || !aligned_to(ws, 256) || ws_bytes < stats_ws_bytes(d_in)) return CMPQ_ERR_WORKSPACE;
     if (n_tokens == 0) return CMPQ_OK;
     int64_t rb = stats_row_blocks(d_in, n_tokens);
     if (rb <= 0) return CMPQ_ERR_CUDA;
     return launch_collect_stats_norm(X, dt, n_tokens, d_in, ldx, norm, acc, static_cast<double*>(ws), rb,
-                                     static_cast<cudaStream_t>(stream));
+                                     static_cast<cudaStream_t>(stream), nonfinite);
 }
 
 extern "C" cmpq_status cmpq_collect_stats(const void* X, cmpq_dtype dt, int64_t n_tokens, int64_t d_in,
-                                          int64_t ldx, double* sumsq, void* ws, size_t ws_bytes,
+                                          int64_t ldx, double* sumsq, int32_t* nonfinite, void* ws, size_t ws_bytes,
                                           void* stream) {
-    return cmpq_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, ws, ws_bytes, stream);
+    return cmpq_collect_stats_norm(X, dt, n_tokens, d_in, ldx, CMPQ_NORM_L2, sumsq, nonfinite, ws, ws_bytes, stream);
+}
+
+extern "C" cmpq_status cmpq_check_finite(const int32_t* nonfinite, void* stream) {
+    if (!nonfinite) return CMPQ_ERR_INVALID_ARG;
+    int32_t word = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, nonfinite, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return CMPQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CMPQ_ERR_CUDA;
+    return word ? CMPQ_ERR_NONFINITE : CMPQ_OK;
 }
 
 extern "C" cmpq_status cmpq_finalize_stats_norm(const double* acc, int64_t d_in, cmpq_norm norm, float* a,

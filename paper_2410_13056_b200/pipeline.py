@@ -58,9 +58,8 @@ class LayerQuantizer:
         self.n_q = dq if n_q is None else int(n_q)
         self.nnz = self.n_act * self.d_out + self.n_q
         dev = self.device
-        ws_bytes = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out)
-                       for op in list(range(6)) + [B.OP_PROTECT_QUANTIZE_PACK])
-        self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+        self.ws = None
+        self._ensure_ws()
         self.sumsq = torch.empty(self.d_in, dtype=torch.float64, device=dev)
         self.a = torch.empty(self.d_in, dtype=torch.float32, device=dev)
         self.bits = torch.empty(self.d_in, dtype=torch.uint8, device=dev)
@@ -75,6 +74,21 @@ class LayerQuantizer:
         self.perm = torch.empty(self.d_in, dtype=torch.int32, device=dev)
         self.seg_rows = torch.empty(3, dtype=torch.int64, device=dev)
         self.counters = torch.zeros(4, dtype=torch.int64, device=dev)
+
+    def _ensure_ws(self):
+        """One scratch buffer large enough for every call of the pass.  The size depends on the assignment
+        method selected in the library (the all-pairs method keeps an fp32 error per weight), so it is
+        checked again before every run."""
+        need = max(B.cmpq_workspace_bytes(op, self.d_in, self.d_out)
+                   for op in list(range(6)) + [B.OP_PROTECT_QUANTIZE_PACK])
+        if self.ws is None or self.ws.numel() < need:
+            self.ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+            self._graphs = {}  # captured graphs hold the old buffer's address
+
+    def check_finite(self):
+        """Waits for the last run and raises binding.CmpqError (status 6) if its activations or weights
+        held a NaN or an infinity (the run's outputs are then unspecified)."""
+        B.cmpq_check_finite(self.nonfinite)
 
     def packed_words(self, avg_bits):
         """Words the rank-form allocation produces for this budget (no device read needed)."""
@@ -132,12 +146,14 @@ class LayerQuantizer:
             e1.record()
             events[name] = (e0, e1)
 
+        self._ensure_ws()
         self.counters.zero_()
         inexact = self.counters[0:1].view(torch.int32)[0:1]
         sweeps = self.counters[1:2]
+        nonfinite = self.nonfinite = self.counters[2:3].view(torch.int32)[0:1]
         if not reuse_statistic:
             self.sumsq.zero_()
-            call("cmpq_collect_stats", B.cmpq_collect_stats, X, self.sumsq, self.ws)
+            call("cmpq_collect_stats", B.cmpq_collect_stats, X, self.sumsq, self.ws, nonfinite=nonfinite)
             call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
         call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
              self.ws)
@@ -150,7 +166,8 @@ class LayerQuantizer:
         elif fused:  # outlier protection, final fit and packing in one call
             call("cmpq_protect_quantize_pack", B.cmpq_protect_quantize_pack, W, self.a, self.bits, self.n_act,
                  self.n_q, lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.packed,
-                 self.row_off, self.perm, self.seg_rows, self.ws, inexact_rows=inexact, sweeps=sweeps)
+                 self.row_off, self.perm, self.seg_rows, self.ws, inexact_rows=inexact, sweeps=sweeps,
+                 nonfinite=nonfinite)
         else:
             self._protect_then_quantize(call, W, lloyd_iters, events, inexact, sweeps)
             call("cmpq_pack", B.cmpq_pack, self.codes, self.bits, self.packed, self.row_off, self.perm,

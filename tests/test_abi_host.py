@@ -51,14 +51,24 @@ def test_default_counts_and_packed_words_match_the_checker(L):
 
 
 def test_workspace_sizes(L):
-    assert B.cmpq_workspace_bytes(B.OP_EXTRACT_OUTLIERS, 4096, 4096) >= 4 * 4096 * 4096
     assert B.cmpq_workspace_bytes(B.OP_COLLECT_STATS, 4096) <= 8 << 20
     for op in range(6):
         assert B.cmpq_workspace_bytes(op, 512, 512) % 256 == 0
         assert B.cmpq_workspace_bytes(op, 0, 512) == 0          # d_in out of range
     assert B.cmpq_workspace_bytes(B.OP_PACK, 512, 1 << 20) == 0   # d_out out of range
+    # the fused call needs no more than the outlier step alone: the final fit patches the provisional tables
     assert (B.cmpq_workspace_bytes(B.OP_PROTECT_AND_QUANTIZE, 512, 512)
-            > B.cmpq_workspace_bytes(B.OP_EXTRACT_OUTLIERS, 512, 512))
+            == B.cmpq_workspace_bytes(B.OP_EXTRACT_OUTLIERS, 512, 512))
+    assert (B.cmpq_workspace_bytes(B.OP_PROTECT_QUANTIZE_PACK, 512, 512)
+            > B.cmpq_workspace_bytes(B.OP_PROTECT_AND_QUANTIZE, 512, 512))
+    # the whole pass of the largest workload layer (8192 x 28672) fits in 8 bytes per weight of scratch ...
+    assert B.cmpq_workspace_bytes(B.OP_PROTECT_QUANTIZE_PACK, 8192, 28672) <= 8 * 8192 * 28672
+    # ... while the all-pairs formulation keeps an fp32 error per weight: the answer follows the selected method
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS)
+    try:
+        assert B.cmpq_workspace_bytes(B.OP_EXTRACT_OUTLIERS, 4096, 4096) >= 4 * 4096 * 4096
+    finally:
+        B.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED)
 
 
 def test_bad_arguments_are_refused_on_the_host(L):
@@ -67,19 +77,19 @@ def test_bad_arguments_are_refused_on_the_host(L):
     p = ctypes.cast(buf, ctypes.c_void_p)
     ws = ctypes.c_void_p((p.value + 255) // 256 * 256)
     # statistic
-    assert L.cmpq_collect_stats(p, 0, 4, 8, 8, None, ws, 1 << 30, None) == INVALID       # no sumsq
-    assert L.cmpq_collect_stats(p, 0, -1, 8, 8, p, ws, 1 << 30, None) == INVALID          # n < 0
-    assert L.cmpq_collect_stats(p, 0, 4, 8, 7, p, ws, 1 << 30, None) == INVALID           # ldx < d_in
-    assert L.cmpq_collect_stats(p, 5, 4, 8, 8, p, ws, 1 << 30, None) == INVALID           # dtype
-    assert L.cmpq_collect_stats(p, 0, 4, 8, 8, p, None, 1 << 30, None) == WORKSPACE
-    assert L.cmpq_collect_stats(p, 0, 4, 8, 8, p, ws, 16, None) == WORKSPACE
+    assert L.cmpq_collect_stats(p, 0, 4, 8, 8, None, None, ws, 1 << 30, None) == INVALID       # no sumsq
+    assert L.cmpq_collect_stats(p, 0, -1, 8, 8, p, None, ws, 1 << 30, None) == INVALID          # n < 0
+    assert L.cmpq_collect_stats(p, 0, 4, 8, 7, p, None, ws, 1 << 30, None) == INVALID           # ldx < d_in
+    assert L.cmpq_collect_stats(p, 5, 4, 8, 8, p, None, ws, 1 << 30, None) == INVALID           # dtype
+    assert L.cmpq_collect_stats(p, 0, 4, 8, 8, p, None, None, 1 << 30, None) == WORKSPACE
+    assert L.cmpq_collect_stats(p, 0, 4, 8, 8, p, None, ws, 16, None) == WORKSPACE
     # Algorithm 1 requires b in [2, 4]
     for b in (1.99, 4.01, float("nan")):
         assert L.cmpq_allocate_bits(p, 8, b, 0, p, None, ws, 1 << 30, None) == INVALID
     assert L.cmpq_allocate_bits(p, 8, 3.0, 7, p, None, ws, 1 << 30, None) == INVALID      # mode
     assert L.cmpq_allocate_bits(p, 8, 3.0, 0, p, None, ws, 8, None) == WORKSPACE
     # outliers: counts must be consistent
-    args = lambda n_act, n_q, nnz, iters=5, d_out=16: (p, 0, 8, d_out, d_out, p, p, n_act, n_q, iters, p, p, p, nnz, ws, 1 << 30, None)
+    args = lambda n_act, n_q, nnz, iters=5, d_out=16: (p, 0, 8, d_out, d_out, p, p, n_act, n_q, iters, p, p, p, nnz, None, ws, 1 << 30, None)
     assert L.cmpq_extract_outliers(*args(9, 0, 9 * 16)) == INVALID
     assert L.cmpq_extract_outliers(*args(1, 7 * 16 + 1, 16 + 7 * 16 + 1)) == INVALID
     assert L.cmpq_extract_outliers(*args(1, 3, 18)) == INVALID                             # nnz mismatch
@@ -87,17 +97,17 @@ def test_bad_arguments_are_refused_on_the_host(L):
     assert L.cmpq_extract_outliers(*args(1, 3, 19, iters=1001)) == INVALID
     assert L.cmpq_extract_outliers(*args(0, 0, 0, d_out=40000)) == INVALID                 # d_out too large
     # quantizer
-    q = lambda sens=None, nnz=0, rows=None, d_out=16, iters=5: (p, 0, 8, d_out, d_out, p, rows, rows, nnz, iters, sens, p, p, None, None, ws, 1 << 30, None)
+    q = lambda sens=None, nnz=0, rows=None, d_out=16, iters=5: (p, 0, 8, d_out, d_out, p, rows, rows, nnz, iters, sens, p, p, None, None, None, ws, 1 << 30, None)
     assert L.cmpq_quantize_layer(*q(sens=ctypes.c_void_p(p.value + 2))) == INVALID           # misaligned sensitivities
     assert L.cmpq_quantize_layer(*q(nnz=3)) == INVALID                                     # list missing
     assert L.cmpq_quantize_layer(*q(d_out=0)) == INVALID
     assert L.cmpq_quantize_layer(*q(iters=2000)) == INVALID
     # eight codes leave in one store: an offset view of a code buffer is refused here, never launched
-    qc = lambda codes: (ws, 0, 8, 16, 16, ws, None, None, 0, 5, None, ws, codes, None, None, ws, 1 << 30, None)
+    qc = lambda codes: (ws, 0, 8, 16, 16, ws, None, None, 0, 5, None, ws, codes, None, None, None, ws, 1 << 30, None)
     assert L.cmpq_quantize_layer(*qc(ctypes.c_void_p(ws.value + 1))) == INVALID
     assert L.cmpq_quantize_layer(*qc(ctypes.c_void_p(ws.value + 4))) == INVALID
     # outlier protection and final fit in one call: the checks of both
-    f = lambda n_act=1, n_q=3, nnz=19, lut=p, codes=p, wsb=1 << 30: (p, 0, 8, 16, 16, p, p, n_act, n_q, 5, p, p, p, nnz, lut, codes, None, None, ws, wsb, None)
+    f = lambda n_act=1, n_q=3, nnz=19, lut=p, codes=p, wsb=1 << 30: (p, 0, 8, 16, 16, p, p, n_act, n_q, 5, p, p, p, nnz, lut, codes, None, None, None, ws, wsb, None)
     assert L.cmpq_protect_and_quantize(*f(nnz=18)) == INVALID
     assert L.cmpq_protect_and_quantize(*f(lut=None)) == INVALID
     assert L.cmpq_protect_and_quantize(*f(codes=None)) == INVALID

@@ -74,3 +74,41 @@ def test_unknown_norm_is_rejected():
     with pytest.raises(B.CmpqError) as e:
         B.cmpq_collect_stats_norm(X, 3, acc, B.workspace(B.OP_COLLECT_STATS, 64))
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("norm", [B.NORM_L2, B.NORM_L1, B.NORM_LINF])
+@pytest.mark.parametrize("bad", [float("inf"), float("-inf"), float("nan")])
+def test_nonfinite_activation_sets_the_flag_and_nothing_else_changes(norm, bad):
+    """A NaN or an infinity among the activations: bit 0 of the caller's word is set (the reduction reads
+    every value anyway) and every other column's statistic is what it would be without it."""
+    X = inputs.make_activations(700, 512, inputs.BF16, 9, device="cuda")
+    ws = B.workspace(B.OP_COLLECT_STATS, 512)
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clean = torch.zeros(512, dtype=torch.float64, device="cuda")
+    B.cmpq_collect_stats_norm(X, norm, clean, ws, nonfinite=flag)
+    B.cmpq_check_finite(flag)                                   # finite input: no error
+    assert int(flag.item()) == 0
+    Xb = X.clone()
+    Xb[123, 45] = bad
+    acc = torch.zeros(512, dtype=torch.float64, device="cuda")
+    B.cmpq_collect_stats_norm(Xb, norm, acc, ws, nonfinite=flag)
+    with pytest.raises(B.CmpqError) as e:
+        B.cmpq_check_finite(flag)
+    assert e.value.status == 6 and int(flag.item()) == 1
+    keep = torch.ones(512, dtype=torch.bool, device="cuda")
+    keep[45] = False
+    assert torch.equal(acc[keep], clean[keep])
+    assert not torch.isfinite(acc[45])
+    # without a word to report into, the call still runs
+    B.cmpq_collect_stats_norm(Xb, norm, torch.zeros(512, dtype=torch.float64, device="cuda"), ws)
+    torch.cuda.synchronize()
+
+
+def test_bf16_square_beyond_fp32_is_reported_like_an_infinity():
+    X = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
+    X[3, 7] = 3.0e19                                            # finite in bf16, its square is not in fp32
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    acc = torch.zeros(256, dtype=torch.float64, device="cuda")
+    B.cmpq_collect_stats(X, acc, B.workspace(B.OP_COLLECT_STATS, 256), nonfinite=flag)
+    torch.cuda.synchronize()
+    assert int(flag.item()) == 1
