@@ -199,7 +199,7 @@ rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long lo
     if (x.select) {
         if (tid == 0) {
             SelectState* st = x.select;
-            st->prefix = 0; st->mask = 0; st->remaining = x.n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0;
+            st->prefix = 0; st->mask = 0; st->remaining = x.n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0; st->lower = 0;
         }
         for (int b = tid; b < kSelBins; b += kCutThreads) x.hist[b] = 0u;
     }

@@ -26,6 +26,10 @@ struct LloydArgs {
     int32_t* inexact_rows;   // optional counter
     unsigned long long* sweeps;  // optional counter of distance evaluations
     int32_t* nonfinite;      // optional flag word: bit 1 is set when a weight is a NaN or an infinity
+    // ordered formulation, provisional fit of the outlier step: every fitted channel leaves the limits of
+    // its clusters in the tables and adds the largest error of each cluster side to this histogram (by the
+    // top 12 bits of the error pattern), from which a lower bound of the selection threshold follows
+    unsigned int* side_hist; // [4096] or NULL
     // ordered formulation only: fits kept across calls on the same weights (budget sweeps).  fit_cache is
     // the block lloyd_fit_cache_bytes() describes; a channel whose fit for its width is already there
     // copies it instead of iterating, every other channel stores its fit there.
@@ -56,6 +60,9 @@ cmpq_status launch_lloyd_ordered_patched(const LloydArgs& args, cmpq_dtype dt, v
 
 // Selection of the worst-fitted entries on the tables of a provisional ordered fit made with neither codes
 // nor errors requested (state: the radix select's SelectState; see outliers.cu for the procedure).
+// state->lower = the lower edge of the histogram bin in which the n_q-th largest of the cluster-side
+// maxima lies (0 if there are fewer); clears the histogram.
+cmpq_status launch_select_lower(void* state, unsigned int* hist, cudaStream_t st);
 cmpq_status launch_table_select_hist(void* tables, size_t tables_bytes, cmpq_dtype dt, const uint8_t* bits,
                                      const uint8_t* is_act, int64_t d_in, int64_t d_out, void* state,
                                      int shift, int bins, int final_pass, unsigned int* hist, cudaStream_t st);

@@ -60,6 +60,8 @@ struct Tables {
     double* sum;         // [d_in][sum_stride] prefix sums at every eighth entry, for tables too large for shared memory
     float* lut;          // [d_in][16] centroids for the assign kernel when the caller wants no lut
     float* thr;          // [d_in][16] value thresholds of the last assignment ([0]: 1 if valid)
+    uint16_t* bnd;       // [d_in][32] provisional fit with valid thresholds: [2k] first entry of cluster k,
+                         // [2k+1] its first entry whose value is >= c_k (the cluster ends where the next begins)
 };
 
 // d_out + 1 entries and the sentinel, plus one entry of slack while a table is patched in place
@@ -75,6 +77,7 @@ static Tables carve_tables(Workspace& w, int64_t d_in, int64_t d_out) {
     t.sum = w.take<double>((size_t)d_in * t.sum_stride);
     t.lut = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
     t.thr = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
+    t.bnd = w.take<uint16_t>((size_t)d_in * 32);
     return t;
 }
 
@@ -382,6 +385,7 @@ struct FitCache {
     uint8_t* valid;
     float* lut;
     float* thr;
+    uint16_t* bnd;
 };
 
 static FitCache carve_fit_cache(void* p, int64_t d_in) {
@@ -392,11 +396,13 @@ static FitCache carve_fit_cache(void* p, int64_t d_in) {
     c.valid = w.take<uint8_t>(3 * (size_t)d_in);
     c.lut = w.take<float>(3 * (size_t)d_in * CMPQ_LUT_STRIDE);
     c.thr = w.take<float>(3 * (size_t)d_in * CMPQ_LUT_STRIDE);
+    c.bnd = w.take<uint16_t>(3 * (size_t)d_in * 32);
     return c;
 }
 
 size_t lloyd_fit_cache_bytes(int64_t d_in) {
-    return 256 + round_up(3 * (size_t)d_in, 256) + 2 * round_up(3 * (size_t)d_in * CMPQ_LUT_STRIDE * sizeof(float), 256);
+    return 256 + round_up(3 * (size_t)d_in, 256) + 2 * round_up(3 * (size_t)d_in * CMPQ_LUT_STRIDE * sizeof(float), 256) +
+           round_up(3 * (size_t)d_in * 32 * sizeof(uint16_t), 256);
 }
 
 __global__ void fit_cache_clear_kernel(FitCache c, int64_t n, int iters) {
@@ -433,6 +439,7 @@ struct IterArgs {
     const int32_t* cols;
     int32_t* inexact_rows;
     const int32_t* nonfinite;  // optional flag word of the call: once it is set the iterations are skipped
+    unsigned int* side_hist;   // provisional fit of the outlier step (see LloydArgs), else NULL
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -850,11 +857,37 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, const int K, uns
     {
         const float cm = __shfl_up_sync(gmask, ck, 1, kGroup);
         float thr = ordered ? 1.f : 0.f;
+        uint32_t b = kfirst;
         if (ordered && gl > 0 && gl < K) {
-            const uint32_t b = boundary_key<DT>(cm, ck, kfirst, kend);
+            b = boundary_key<DT>(cm, ck, kfirst, kend);
             thr = b < kend ? value_of_key16<DT>(b) : __int_as_float(0x7f800000);
         }
         a.t.thr[row * CMPQ_LUT_STRIDE + gl] = gl < K ? thr : 0.f;
+        // For the selection of the worst-fitted entries: cluster k is the run [first, next first) of the table;
+        // on each side of c_k the error grows towards the end of the run, so the largest error of a side sits
+        // at its outer end.  Those maxima (of entries that hold at least one weight) go into the histogram.
+        if (a.side_hist && ordered) {
+            int first = 0, mid = 0;
+            if (gl < K) {
+                if (gl > 0) first = b < kend ? rank_of_key(keys, M, b, staged ? e_hint : -1) : M;
+                const uint32_t kc = key_ceil<DT>(ck);  // the first storage value not below c_k
+                mid = kc >= kend ? M : (kc <= kfirst ? 0 : rank_of_key(keys, M, kc, staged ? first : -1));
+            }
+            int next = __shfl_down_sync(gmask, first, 1, kGroup);
+            if (gl == K - 1) next = M;
+            if (gl < K) {
+                mid = mid < first ? first : (mid > next ? next : mid);
+                uint16_t* bnd = a.t.bnd + row * 32;
+                bnd[2 * gl] = (uint16_t)first;
+                bnd[2 * gl + 1] = (uint16_t)mid;
+                int j = first;  // left side: [first, mid), largest error at its first entry that is not empty
+                if (j < mid && cum[j + 1] == cum[j]) ++j;
+                if (j < mid) atomicAdd(&a.side_hist[__float_as_uint(fabsf(value_of_key16<DT>(keys[j]) - ck)) >> 20], 1u);
+                j = next - 1;   // right side: [mid, next), largest error at its last entry that is not empty
+                if (j >= mid && cum[j + 1] == cum[j]) --j;
+                if (j >= mid) atomicAdd(&a.side_hist[__float_as_uint(fabsf(value_of_key16<DT>(keys[j]) - ck)) >> 20], 1u);
+            }
+        }
     }
     // assignments made: one per update, and the last one by the assign kernel
     if (a.sweeps && gl == 0)
@@ -883,12 +916,15 @@ lloyd_iterate_kernel(const IterArgs a) {
     if (cached_ok && a.fc.valid[slot]) {
         a.lut[row * CMPQ_LUT_STRIDE + gl] = a.fc.lut[slot * CMPQ_LUT_STRIDE + gl];
         a.t.thr[row * CMPQ_LUT_STRIDE + gl] = a.fc.thr[slot * CMPQ_LUT_STRIDE + gl];
+        reinterpret_cast<uint32_t*>(a.t.bnd + row * 32)[gl] = reinterpret_cast<const uint32_t*>(a.fc.bnd + slot * 32)[gl];
         return;
     }
     iterate_channel<DT>(a, row, bits == 2 ? 4 : (bits == 3 ? 8 : 16), smem);
     if (cached_ok) {  // lane l wrote entry l of both rows above and reads its own writes back
         a.fc.lut[slot * CMPQ_LUT_STRIDE + gl] = a.lut[row * CMPQ_LUT_STRIDE + gl];
         a.fc.thr[slot * CMPQ_LUT_STRIDE + gl] = a.t.thr[row * CMPQ_LUT_STRIDE + gl];
+        __syncwarp(gmask);  // lanes below K wrote the cluster limits (two 16-bit values each) just before
+        reinterpret_cast<uint32_t*>(a.fc.bnd + slot * 32)[gl] = reinterpret_cast<const uint32_t*>(a.t.bnd + row * 32)[gl];
         __syncwarp(gmask);
         if (gl == 0) {
             __threadfence();
@@ -1172,8 +1208,38 @@ __device__ __forceinline__ void table_hist_row(const Tables& t, int64_t row, uin
     }
 }
 
+// A row fitted with valid thresholds: lane 2k walks the left side of cluster k (values below c_k) upwards
+// from its first entry, lane 2k + 1 the right side downwards from its last entry.  Along such a walk the
+// error |v - c_k| (fp32, the rounding is monotone) never grows, so the walk ends at the first error below
+// `lo`: visit(error pattern, count, key) sees exactly the non-empty entries of the row with error >= lo.
+template <int DT, class Visit>
+__device__ __forceinline__ void walk_row_sides(const Tables& t, int64_t row, int K, uint32_t lo, Visit&& visit) {
+    const int lane = threadIdx.x & 31;
+    if (lane >= 2 * K) return;
+    const int k = lane >> 1;
+    const bool left = (lane & 1) == 0;
+    const uint16_t* bnd = t.bnd + row * 32;
+    const int M = t.hdr[row].M;
+    const int first = bnd[2 * k], mid = bnd[2 * k + 1], next = k + 1 < K ? (int)bnd[2 * k + 2] : M;
+    const float c = t.lut[row * CMPQ_LUT_STRIDE + k];
+    const uint16_t* keys = t.keys + row * t.stride;
+    const uint16_t* cum = t.cum + row * t.stride;
+    int j = left ? first : next - 1;
+    const int stop = left ? mid : mid - 1, step = left ? 1 : -1;
+    while (j != stop) {
+        const uint32_t key = keys[j], c0 = cum[j], c1 = cum[j + 1];
+        if (c1 != c0) {
+            const uint32_t e = __float_as_uint(fabsf(value_of_key16<DT>(key) - c));
+            if (e < lo) break;
+            visit(e, c1 - c0, key);
+        }
+        j += step;
+    }
+}
+
 // hist[d] += number of weights in non-act rows whose error has the fixed bits of the prefix and the
-// digit d at `shift`.  One warp per row, block-local histogram first.
+// digit d at `shift`.  One warp per row, block-local histogram first.  Errors below st->lower (a bound
+// known not to exceed the threshold sought) are left out wherever the row's fit allows the walk above.
 template <int DT>
 __global__ void __launch_bounds__(kTableSelWarps * 32)
 table_select_hist_kernel(const Tables t, const uint8_t* __restrict__ bits, const uint8_t* __restrict__ is_act,
@@ -1185,11 +1251,16 @@ table_select_hist_kernel(const Tables t, const uint8_t* __restrict__ bits, const
     for (int b = threadIdx.x; b < bins; b += blockDim.x) local[b] = 0;
     __syncthreads();
     const uint32_t prefix = st->prefix, mask = st->mask;
+    const uint32_t lo = st->lower > prefix ? st->lower : prefix;  // a matching error is at least the prefix
     const int warp = threadIdx.x >> 5;
     for (int64_t row = (int64_t)blockIdx.x * kTableSelWarps + warp; row < d_in; row += (int64_t)gridDim.x * kTableSelWarps) {
         if (is_act[row]) continue;
         const int b = bits[row];
-        if (b == 2) table_hist_row<DT, 4>(t, row, prefix, mask, shift, bins, local);
+        if (t.thr[row * CMPQ_LUT_STRIDE] != 0.f) {
+            walk_row_sides<DT>(t, row, 1 << b, lo, [&](uint32_t e, uint32_t cnt, uint32_t) {
+                if ((e & mask) == prefix) atomicAdd(&local[(e >> shift) & (bins - 1)], cnt);
+            });
+        } else if (b == 2) table_hist_row<DT, 4>(t, row, prefix, mask, shift, bins, local);
         else if (b == 3) table_hist_row<DT, 8>(t, row, prefix, mask, shift, bins, local);
         else table_hist_row<DT, 16>(t, row, prefix, mask, shift, bins, local);
     }
@@ -1207,6 +1278,43 @@ table_select_hist_kernel(const Tables t, const uint8_t* __restrict__ bits, const
         select_digit_block<kTableSelWarps * 32>(hist, shift, bins, st, final_pass, warp_totals, &found_digit, &found_above);
         if (threadIdx.x == 0) st->done = 0;
     }
+}
+
+// The histogram holds, by the top 12 bits of the error pattern, the largest error of every cluster side of
+// every fitted row: distinct entries that each stand for at least one weight.  If n_q or more of them lie in
+// bin d or above, so do n_q or more errors of the layer: the n_q-th largest error is at least the lower edge
+// of the bin in which the n_q-th largest of the maxima lies.  Clears the histogram for the select passes.
+__global__ void __launch_bounds__(1024)
+select_lower_kernel(unsigned int* hist, SelectState* st) {
+    __shared__ int warp_totals[32];
+    __shared__ uint32_t found;
+    constexpr int per = kSelBins / 1024;  // bins per thread, descending
+    const long long want = st->remaining;
+    int v[per], sum = 0;
+#pragma unroll
+    for (int u = 0; u < per; ++u) {
+        v[u] = (int)hist[kSelBins - 1 - (threadIdx.x * per + u)];
+        sum += v[u];
+    }
+    if (threadIdx.x == 0) found = 0u;
+    int total;
+    long long above = block_exclusive_scan(sum, warp_totals, total);  // maxima in higher bins (publishes `found`)
+    if (want > 0 && above < want && want <= above + sum) {  // at most one thread
+#pragma unroll
+        for (int u = 0; u < per; ++u) {
+            if (above < want && want <= above + v[u]) found = (uint32_t)(kSelBins - 1 - (threadIdx.x * per + u)) << 20;
+            above += v[u];
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) st->lower = found;
+#pragma unroll
+    for (int u = 0; u < per; ++u) hist[threadIdx.x * per + u] = 0u;
+}
+
+cmpq_status launch_select_lower(void* state, unsigned int* hist, cudaStream_t st) {
+    select_lower_kernel<<<1, 1024, 0, st>>>(hist, static_cast<SelectState*>(state));
+    return launch_status();
 }
 
 template <int DT, int K>
@@ -1244,7 +1352,12 @@ table_row_count_kernel(const Tables t, const uint8_t* __restrict__ bits, const u
     if (!is_act[row]) {
         const uint32_t tau = st->tau;
         const int b = bits[row];
-        if (b == 2) table_count_row<DT, 4>(t, row, tau, g, q);
+        if (t.thr[row * CMPQ_LUT_STRIDE] != 0.f) {
+            walk_row_sides<DT>(t, row, 1 << b, tau, [&](uint32_t e, uint32_t cnt, uint32_t) {
+                g += e > tau ? (int)cnt : 0;
+                q += e == tau ? (int)cnt : 0;
+            });
+        } else if (b == 2) table_count_row<DT, 4>(t, row, tau, g, q);
         else if (b == 3) table_count_row<DT, 8>(t, row, tau, g, q);
         else table_count_row<DT, 16>(t, row, tau, g, q);
     }
@@ -1494,6 +1607,7 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
     ia.lut = args.lut ? args.lut : t.lut;
     ia.sweeps = args.sweeps;
     ia.nonfinite = args.nonfinite;
+    ia.side_hist = args.side_hist;
     if (patch_from) {
         ia.src = *patch_from;
         ia.W = args.W;

@@ -324,6 +324,7 @@ cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_o
         la.fit_cache = fit_cache;
         la.tables_ready = tables_ready;
         la.nonfinite = nonfinite;
+        la.side_hist = all_pairs ? nullptr : o.hist;
         s = all_pairs ? launch_lloyd(la, dt, st) : launch_lloyd_ordered(la, dt, o.tables, tables_bytes, st);
         if (s != CMPQ_OK) return s;
     }
@@ -334,6 +335,10 @@ cmpq_status extract_impl(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_o
         unsigned hist_blocks = (unsigned)((int64_t)sms * 8 < d_in ? (int64_t)sms * 8 : d_in);
         const int shifts[3] = {20, 10, 0};
         const int bins[3] = {4096, 1024, 1024};
+        if (!all_pairs) {  // a lower bound of the threshold from the largest errors of the cluster sides
+            s = launch_select_lower(o.state, o.hist, st);
+            if (s != CMPQ_OK) return s;
+        }
         for (int p = 0; p < 3; ++p) {
             if (all_pairs) {
                 select_hist_kernel<<<hist_blocks, kSelThreads, 0, st>>>(o.err, o.is_act, d_in, d_out, o.state, shifts[p], bins[p], o.hist);

@@ -16,6 +16,7 @@ struct SelectState {
     uint32_t tau;           // final threshold pattern
     long long take_equal;   // entries equal to tau that belong to the set
     unsigned int done;      // blocks of the running histogram kernel that have added their counts
+    uint32_t lower;         // an error pattern known not to exceed tau (0: nothing known)
 };
 
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_totals, int& total) {
