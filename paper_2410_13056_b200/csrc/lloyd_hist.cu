@@ -62,6 +62,9 @@ struct Tables {
     float* thr;          // [d_in][16] value thresholds of the last assignment ([0]: 1 if valid)
     uint16_t* bnd;       // [d_in][32] provisional fit with valid thresholds: [2k] first entry of cluster k,
                          // [2k+1] its first entry whose value is >= c_k (the cluster ends where the next begins)
+    uint32_t* kept;      // [d_in][32] after the selection: [0] = n, then the n keys of the row's values that keep
+                         // entries (bit 16: only some of their entries, error equal to the threshold);
+                         // n = kKeptUnknown: not listed
 };
 
 // d_out + 1 entries and the sentinel, plus one entry of slack while a table is patched in place
@@ -78,6 +81,7 @@ static Tables carve_tables(Workspace& w, int64_t d_in, int64_t d_out) {
     t.lut = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
     t.thr = w.take<float>((size_t)d_in * CMPQ_LUT_STRIDE);
     t.bnd = w.take<uint16_t>((size_t)d_in * 32);
+    t.kept = w.take<uint32_t>((size_t)d_in * 32);
     return t;
 }
 
@@ -1183,6 +1187,8 @@ struct RowFit {
 };
 
 constexpr int kTableSelWarps = 8;
+constexpr int kKeptCap = 31;                  // values of a row listed for the emit step
+constexpr uint32_t kKeptUnknown = 0xffffffffu;
 
 template <int DT, int K>
 __device__ __forceinline__ void table_hist_row(const Tables& t, int64_t row, uint32_t prefix, uint32_t mask, int shift,
@@ -1352,14 +1358,36 @@ table_row_count_kernel(const Tables t, const uint8_t* __restrict__ bits, const u
     if (!is_act[row]) {
         const uint32_t tau = st->tau;
         const int b = bits[row];
+        uint32_t* kept = t.kept + row * 32;
         if (t.thr[row * CMPQ_LUT_STRIDE] != 0.f) {
+            int mine = 0;  // values this lane's walk finds at or above the threshold
             walk_row_sides<DT>(t, row, 1 << b, tau, [&](uint32_t e, uint32_t cnt, uint32_t) {
                 g += e > tau ? (int)cnt : 0;
                 q += e == tau ? (int)cnt : 0;
+                ++mine;
             });
-        } else if (b == 2) table_count_row<DT, 4>(t, row, tau, g, q);
-        else if (b == 3) table_count_row<DT, 8>(t, row, tau, g, q);
-        else table_count_row<DT, 16>(t, row, tau, g, q);
+            // the emit step only needs to know WHICH values keep entries: list them (second, identical walk)
+            const int lane = threadIdx.x & 31;
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            const int total = __shfl_sync(0xffffffffu, incl, 31);
+            if (total <= kKeptCap) {
+                int at = 1 + incl - mine;
+                walk_row_sides<DT>(t, row, 1 << b, tau, [&](uint32_t e, uint32_t, uint32_t key) {
+                    kept[at++] = key | (e == tau ? 0x10000u : 0u);
+                });
+            }
+            if (lane == 0) kept[0] = total <= kKeptCap ? (uint32_t)total : kKeptUnknown;
+        } else {
+            if ((threadIdx.x & 31) == 0) kept[0] = kKeptUnknown;
+            if (b == 2) table_count_row<DT, 4>(t, row, tau, g, q);
+            else if (b == 3) table_count_row<DT, 8>(t, row, tau, g, q);
+            else table_count_row<DT, 16>(t, row, tau, g, q);
+        }
     }
     g = warp_sum(g);
     q = warp_sum(q);
@@ -1453,6 +1481,69 @@ __device__ void table_emit_row(const uint16_t* __restrict__ w, int64_t d_out, co
     }
 }
 
+// Kept entries of a row whose entry-keeping values were listed by the count step: a weight is a candidate
+// exactly when its key is in the list, so no error is evaluated here.  Ordering as in table_emit_row.
+__device__ void table_emit_row_by_keys(const uint16_t* __restrict__ w, int64_t d_out, const uint32_t* __restrict__ kept,
+                                       int nkept, int64_t row, int te, int64_t out0, int32_t* __restrict__ rows,
+                                       int32_t* __restrict__ cols, uint16_t* __restrict__ vals, int* list_col,
+                                       unsigned char* list_eq, int* list_n, uint32_t* s_kept) {
+    if (threadIdx.x == 0) *list_n = 0;
+    if ((int)threadIdx.x < nkept) s_kept[threadIdx.x] = kept[1 + threadIdx.x];
+    __syncthreads();
+    const bool vec = ((reinterpret_cast<uintptr_t>(w) & 15) == 0);
+    for (int64_t j0 = (int64_t)threadIdx.x * 8; j0 < d_out; j0 += (int64_t)blockDim.x * 8) {
+        uint32_t pk[4] = {0u, 0u, 0u, 0u};
+        if (j0 + 7 < d_out && vec) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(w + j0));
+            pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
+        } else {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (j0 + u < d_out) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
+        }
+        uint32_t key[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            uint32_t h = (pk[u >> 1] >> (16 * (u & 1))) & 0xffffu;
+            if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
+            key[u] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+        }
+        for (int i = 0; i < nkept; ++i) {
+            const uint32_t kk = s_kept[i];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (key[u] == (kk & 0xffffu) && j0 + u < d_out) {
+                    const int p = atomicAdd(list_n, 1);
+                    if (p < kEmitListCap) {
+                        list_col[p] = (int)(j0 + u);
+                        list_eq[p] = (unsigned char)(kk >> 16);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    const int n = *list_n < kEmitListCap ? *list_n : kEmitListCap;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int c = list_col[i];
+        const int is_eq = list_eq[i];
+        int before = 0, eq_before = 0;  // candidates / threshold-candidates in lower columns
+        for (int u = 0; u < n; ++u) {
+            const int lower = list_col[u] < c ? 1 : 0;
+            before += lower;
+            eq_before += lower & list_eq[u];
+        }
+        const bool keep = !is_eq || eq_before < te;
+        if (keep) {
+            const int dropped_before = eq_before > te ? eq_before - te : 0;
+            const int64_t pos = out0 + before - dropped_before;
+            rows[pos] = (int32_t)row;
+            cols[pos] = c;
+            vals[pos] = w[c];
+        }
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kSelThreads)
 table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, const uint8_t* __restrict__ bits,
@@ -1464,6 +1555,7 @@ table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, c
     __shared__ int list_col[kEmitListCap];
     __shared__ unsigned char list_eq[kEmitListCap];
     __shared__ int list_n;
+    __shared__ uint32_t s_kept[32];
     const int64_t row = blockIdx.x;
     const int64_t out0 = row_start[row];
     if (row_start[row + 1] == out0) return;
@@ -1480,6 +1572,12 @@ table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, c
     const int te = take_eq[row];
     const int ncand = gt[row] + eq[row];
     const int b = bits[row];
+    const uint32_t nkept = t.kept[row * 32];
+    if (nkept != kKeptUnknown && ncand <= kEmitListCap) {
+        table_emit_row_by_keys(w, d_out, t.kept + row * 32, (int)nkept, row, te, out0, rows, cols, vals, list_col, list_eq,
+                               &list_n, s_kept);
+        return;
+    }
     if (b == 2) table_emit_row<DT, 4>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
     else if (b == 3) table_emit_row<DT, 8>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
     else table_emit_row<DT, 16>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
