@@ -15,10 +15,14 @@
  *
  * Conventions for every entry point
  *  - All array arguments are DEVICE pointers owned by the caller unless the
- *    parameter comment says "host".  The library keeps no state and allocates no
- *    memory; scratch space is the caller's `ws` buffer of at least
- *    cmpq_workspace_bytes(op, ...) bytes, 256-byte aligned, whose contents are
- *    undefined before and after the call.
+ *    parameter comment says "host".  The library allocates no memory; scratch space
+ *    is the caller's `ws` buffer of at least cmpq_workspace_bytes(op, ...) bytes,
+ *    256-byte aligned, whose contents are undefined before and after the call.
+ *    The only state it keeps between calls is host state that the caller sets
+ *    explicitly: the process-wide assignment method (cmpq_set_lloyd_assignment,
+ *    which also decides what cmpq_workspace_bytes answers) and the one-shot event
+ *    handles of cmpq_lloyd_phase_events; cmpq_collect_stats_static in addition
+ *    owns a fixed device array (see there).
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *    only enqueue work; outputs are valid once the stream has been synchronised.
  *  - Matrices are row-major with a leading dimension in elements (ldx, ldw).

@@ -12,20 +12,25 @@ import torch
 
 from . import binding as B
 
-# CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0.
-# ASSIGN_ALL_PAIRS: statistic 2 + finalize 1, allocation 2, outliers 13 (rank, mark, K-means, select init,
-# 3 x (histogram, digit), row count, row scan, emit), final fit 2 (row index, K-means), packing 2 = 22.
-# Default: the provisional fit is 2 kernels (table, iterate; its errors are never written), the three digit
-# steps run inside the histogram kernels, the final fit is row index + 3 (table, iterate, assign) = 22 as well.
-# Fused (cmpq_protect_and_quantize, default path): the final fit's table kernel is replaced by the patch
-# kernel plus a table-kernel launch that only rebuilds rows with many removed positions = 23.
+# CUDA kernels of this library launched by one LayerQuantizer.run with n_q > 0 and nnz > 0 (the two zero fills
+# of the counters and of the statistic's accumulator are torch's and not counted).
+# Fused, default assignment (cmpq_protect_quantize_pack): statistic 2 + finalize 1, allocation 1 (two rank cuts
+# in one block), outlier step 10 (O_act cut with select start and pack layout, value tables, provisional
+# iterations, lower bound, 3 select passes, row counts, row scan, emit), final fit 2 (iterations that patch the
+# tables, last assignment that packs) = 17.
+# Separate calls: the final fit builds its own tables (row index, tables, iterations, assignment = 4) and the
+# packing takes 2 more = 20.  All-pairs assignment: the provisional fit is one kernel and every select pass is
+# followed by a digit kernel (outlier step 11), the final fit is row index + one kernel, packing 2 = 19; fused
+# the packing still runs as its own step after the fit (layout with the O_act cut, pack 1) = 18.
 def kernels_per_run(assignment=None, fused=False):
     if assignment is None:
         assignment = B.cmpq_get_lloyd_assignment()
-    return 23 if (fused and assignment != B.ASSIGN_ALL_PAIRS) else 22
+    if assignment == B.ASSIGN_ALL_PAIRS:
+        return 18 if fused else 19
+    return 17 if fused else 20
 
 
-KERNELS_PER_RUN = 22
+KERNELS_PER_RUN = 20
 
 
 @dataclass
@@ -44,6 +49,7 @@ class LayerResult:
     seg_rows: torch.Tensor   # [3] int64 channels per width 2,3,4
     inexact_rows: torch.Tensor  # [1] int32
     sweeps: torch.Tensor     # [1] int64 distance evaluations of the final fit
+    d_out: int = 0           # weights per channel (codes may be None)
 
 
 class LayerQuantizer:
@@ -174,7 +180,7 @@ class LayerQuantizer:
                  self.seg_rows, self.ws)
         words = self.packed_words(avg_bits)
         return LayerResult(self.a, self.bits, self.rows, self.cols, self.vals, self.lut, self.codes,
-                           self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps)
+                           self.packed[:words], self.row_off, self.perm, self.seg_rows, inexact, sweeps, self.d_out)
 
     def _protect_then_quantize(self, call, W, lloyd_iters, events, inexact, sweeps):
         call("cmpq_extract_outliers", B.cmpq_extract_outliers, W, self.a, self.bits, self.n_act, self.n_q,
@@ -321,7 +327,7 @@ class QuantizedLinear:
 
     @classmethod
     def from_result(cls, r: "LayerResult"):
-        return cls(r.packed, r.row_off, r.perm, r.seg_rows, r.lut, r.rows, r.cols, r.vals, r.codes.shape[1])
+        return cls(r.packed, r.row_off, r.perm, r.seg_rows, r.lut, r.rows, r.cols, r.vals, r.d_out)
 
     def packed_bytes(self):
         return self.packed.numel() * 4

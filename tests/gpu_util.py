@@ -80,10 +80,13 @@ def gpu_pack(codes_np, bits_np):
 
 def result_arrays(r):
     """A LayerResult's buffers as host numpy arrays (16-bit values and packed words as unsigned)."""
-    out = {k: getattr(r, k).cpu().numpy() for k in ("a", "bits", "rows", "cols", "lut", "codes", "row_off",
-                                                     "perm", "seg_rows")}
+    out = {k: getattr(r, k).cpu().numpy() for k in ("a", "bits", "rows", "cols", "lut", "row_off", "perm", "seg_rows")}
     out["vals"] = r.vals.cpu().numpy().view(np.uint16)
     out["packed"] = r.packed.cpu().numpy().view(np.uint32)
+    if r.codes is not None:
+        out["codes"] = r.codes.cpu().numpy()
+    else:  # a pass that never materialised the byte codes: the checker's unpacker recovers them
+        out["codes"] = oracle.unpack(out["packed"], out["row_off"], out["perm"], out["bits"], int(r.d_out))
     return out
 
 

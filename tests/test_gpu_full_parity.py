@@ -24,7 +24,7 @@ def _whole_layer(cfg_name, layer_index, budgets, whole_statistic):
     seed = inputs.layer_seed(cfg, layer_index)
     W = inputs.make_weight(L.d_in, L.d_out, cfg.dtype, seed, device="cuda")
     X = inputs.make_activations(cfg.n_tokens, L.d_in, cfg.dtype, seed, device="cuda")
-    q = LayerQuantizer(L.d_in, L.d_out)
+    q = LayerQuantizer(L.d_in, L.d_out, keep_codes=False)   # as the benchmark: packed words only, no byte codes
     Wu = inputs.as_u16(W)
     for k, b in enumerate(budgets):
         q.run_graphed(X, W, b, cfg.lloyd_iters)            # captures
