@@ -90,9 +90,10 @@ __global__ void quantile_bits_kernel(const float* __restrict__ a, const int32_t*
 // Classification without a full rank.  Algorithm 1 in rank form and the choice of the O_act channels
 // (Section 3.2.2) only ask on which side of one or two rank cuts a channel lies.  One block finds, for
 // each cut k, the element of rank k in the ascending order of (a, id) by an exact radix select over the
-// order-preserving bit pattern of a (four 8-bit digits, both cuts at once), then every channel is
+// order-preserving bit pattern of a (8-bit digits, both cuts at once), then every channel is
 // compared with the cut elements; equal statistics are ordered by channel id through a prefix count.
 constexpr int kCutThreads = 1024;
+constexpr int kCutRegKeys = 8;  // statistics per thread held in registers
 
 __device__ __forceinline__ uint32_t ordered_bits(float v) {
     const uint32_t u = __float_as_uint(v + 0.0f);  // -0 and +0 are the same value
@@ -121,21 +122,62 @@ rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long lo
     __shared__ uint32_t prefix[2];
     __shared__ long long remaining[2];  // rank of the cut element among the elements matching the prefix
     __shared__ unsigned long long warp_tot[32];
+    __shared__ uint32_t warp_min[32], warp_max[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long k[2] = {k0, k1};
     const bool live[2] = {k0 < d_in, k1 < d_in};
     if (tid < 2) { prefix[tid] = 0u; remaining[tid] = k[tid] < 0 ? 0 : k[tid]; }
-    for (int pass = 3; pass >= 0; --pass) {
+    // Up to kCutRegKeys patterns per thread stay in registers (channel u * kCutThreads + tid in slot u); a
+    // longer statistic is read again in every pass.
+    const bool in_regs = d_in <= (int64_t)kCutRegKeys * kCutThreads;
+    const int n = (int)d_in;  // d_in <= CMPQ_MAX_D_IN fits
+    uint32_t rk[kCutRegKeys];
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    if (in_regs) {
+#pragma unroll
+        for (int u = 0; u < kCutRegKeys; ++u) {
+            const int i = u * kCutThreads + tid;
+            rk[u] = i < n ? ordered_bits(a[i]) : 0u;
+            if (i < n) { kmin = min(kmin, rk[u]); kmax = max(kmax, rk[u]); }
+        }
+    } else {
+        for (int i = tid; i < n; i += kCutThreads) {
+            const uint32_t key = ordered_bits(a[i]);
+            kmin = min(kmin, key);
+            kmax = max(kmax, key);
+        }
+    }
+    // The statistics of a layer share their leading bits.  The digits are therefore taken from the distance
+    // to the smallest pattern, and only as many 8-bit digits as the largest distance has: the counters of a
+    // pass are then hit evenly and a layer needs three passes rather than four.
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { warp_min[warp] = kmin; warp_max[warp] = kmax; }
+    __syncthreads();
+    kmin = __reduce_min_sync(0xffffffffu, warp_min[lane]);  // kCutThreads / 32 = 32 warps: one value per lane
+    kmax = __reduce_max_sync(0xffffffffu, warp_max[lane]);
+    if (in_regs) {
+#pragma unroll
+        for (int u = 0; u < kCutRegKeys; ++u) rk[u] -= kmin;
+    }
+    const int nbits = 32 - __clz(kmax - kmin);  // 0: all statistics are equal
+    for (int pass = (nbits + 7) / 8 - 1; pass >= 0; --pass) {
         const int shift = 8 * pass;
-        const uint32_t mask = pass == 3 ? 0u : (0xffffffffu << (shift + 8));
-        for (int b = tid; b < 512; b += kCutThreads) (&hist[0][0])[b] = 0u;
+        const uint32_t mask = shift + 8 >= 32 ? 0u : (0xffffffffu << (shift + 8));
+        if (tid < 512) (&hist[0][0])[tid] = 0u;
         __syncthreads();
         const uint32_t p0 = prefix[0], p1 = prefix[1];
-        for (int64_t i = tid; i < d_in; i += kCutThreads) {
-            const uint32_t key = ordered_bits(a[i]);
+        auto count = [&](uint32_t key) {
             const uint32_t d = (key >> shift) & 255u;
             if (live[0] && (key & mask) == p0) atomicAdd(&hist[0][d], 1u);
             if (live[1] && (key & mask) == p1) atomicAdd(&hist[1][d], 1u);
+        };
+        if (in_regs) {
+#pragma unroll
+            for (int u = 0; u < kCutRegKeys; ++u)
+                if (u * kCutThreads + tid < n) count(rk[u]);
+        } else {
+            for (int i = tid; i < n; i += kCutThreads) count(ordered_bits(a[i]) - kmin);
         }
         __syncthreads();
         if (warp < 2 && live[warp]) {  // warp t walks the histogram of cut t upwards
@@ -165,36 +207,51 @@ rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long lo
         }
         __syncthreads();
     }
-    // every thread owns a contiguous range of channels: how many statistics equal to a cut value precede it
-    const int64_t per = (d_in + kCutThreads - 1) / kCutThreads;
-    const int64_t c0 = (int64_t)tid * per;
-    const int64_t c1 = c0 + per < d_in ? c0 + per : d_in;
-    const uint32_t v0 = prefix[0], v1 = prefix[1];
-    unsigned long long mine = 0;  // two counts of 32 bits
-    for (int64_t i = c0; i < c1; ++i) {
-        const uint32_t key = ordered_bits(a[i]);
-        mine += (key == v0 ? 1ull : 0ull) + (key == v1 ? (1ull << 32) : 0ull);
-    }
-    unsigned long long incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    unsigned long long before = incl - mine;
-    for (int w = 0; w < warp; ++w) before += warp_tot[w];
-    long long eq0 = (long long)(before & 0xffffffffull), eq1 = (long long)(before >> 32);
+    const uint32_t v0 = prefix[0], v1 = prefix[1];  // the cut elements, as distances to the smallest pattern
     const long long r0 = remaining[0], r1 = remaining[1];
-    for (int64_t i = c0; i < c1; ++i) {
-        const uint32_t key = ordered_bits(a[i]);
-        int cls = base;
-        if (live[0] && (key > v0 || (key == v0 && eq0 >= r0))) ++cls;
-        if (live[1] && (key > v1 || (key == v1 && eq1 >= r1))) ++cls;
-        eq0 += key == v0 ? 1 : 0;
-        eq1 += key == v1 ? 1 : 0;
-        out[i] = (uint8_t)cls;
+    if ((!live[0] || r0 == 0) && (!live[1] || r1 == 0)) {
+        // The cut element is the first of those equal to it in channel order (always so without ties): every
+        // channel at or above the cut value is at or above the cut.
+        auto classify = [&](int i, uint32_t key) {
+            out[i] = (uint8_t)(base + ((live[0] && key >= v0) ? 1 : 0) + ((live[1] && key >= v1) ? 1 : 0));
+        };
+        if (in_regs) {
+#pragma unroll
+            for (int u = 0; u < kCutRegKeys; ++u)
+                if (u * kCutThreads + tid < n) classify(u * kCutThreads + tid, rk[u]);
+        } else {
+            for (int i = tid; i < n; i += kCutThreads) classify(i, ordered_bits(a[i]) - kmin);
+        }
+    } else {
+        // every thread owns a contiguous range of channels: how many statistics equal to a cut value precede it
+        const int64_t per = (d_in + kCutThreads - 1) / kCutThreads;
+        const int64_t c0 = (int64_t)tid * per;
+        const int64_t c1 = c0 + per < d_in ? c0 + per : d_in;
+        unsigned long long mine = 0;  // two counts of 32 bits
+        for (int64_t i = c0; i < c1; ++i) {
+            const uint32_t key = ordered_bits(a[i]) - kmin;
+            mine += (key == v0 ? 1ull : 0ull) + (key == v1 ? (1ull << 32) : 0ull);
+        }
+        unsigned long long incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        unsigned long long before = incl - mine;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        long long eq0 = (long long)(before & 0xffffffffull), eq1 = (long long)(before >> 32);
+        for (int64_t i = c0; i < c1; ++i) {
+            const uint32_t key = ordered_bits(a[i]) - kmin;
+            int cls = base;
+            if (live[0] && (key > v0 || (key == v0 && eq0 >= r0))) ++cls;
+            if (live[1] && (key > v1 || (key == v1 && eq1 >= r1))) ++cls;
+            eq0 += key == v0 ? 1 : 0;
+            eq1 += key == v1 ? 1 : 0;
+            out[i] = (uint8_t)cls;
+        }
     }
     if (x.select) {
         if (tid == 0) {

@@ -39,7 +39,6 @@
 
 namespace cmpq {
 
-constexpr int kSlots = 32;       // high-byte buckets refined per pass of the second histogram level
 constexpr int kSlotWords = 128;  // 256 low-byte counters of 16 bits, two per word
 constexpr uint32_t kZeroKeyOfTable = 0x8000u;  // sort key of +0
 constexpr int kStageCap = 4096;  // table entries of one pass gathered in shared memory before they are stored
@@ -95,21 +94,30 @@ size_t lloyd_tables_bytes(int64_t d_in, int64_t d_out) {
 // value table of one channel
 
 constexpr int kShortList = 16;  // removed positions of a row kept as a list up to this many, else as a bitmap
+constexpr int kScanWords = 16;  // counter words a thread owns at most on the register path of the scan
 
 struct alignas(16) TableShared {
-    int hist1[256];        // 1 where the high byte occurs
-    int bucket_rank[256];  // rank of a high-byte bucket among the non-empty ones, or -1
-    int slot_hi[256];      // the inverse: high byte of the r-th non-empty bucket
+    unsigned char hist1[256];  // 1 where the high byte occurs
+    int bucket_rank[256];      // rank of a high-byte bucket among the non-empty ones, or -1
+    int slot_hi[256];          // the inverse: high byte of the r-th non-empty bucket
     int n_nonempty;
-    int wtop[32], wulp[32];   // per-warp magnitude range (largest pattern, smallest non-zero pattern - 1)
-    int w_nz[32], w_cnt[32];  // per-warp totals of the block scan
-    int base_nz, base_cnt;    // entries / weights emitted by the previous passes
+    int wtop[32], wulp[32];  // per-warp magnitude range (largest pattern, smallest non-zero pattern - 1)
+    uint32_t w_scan[32];     // per-warp totals of the block scan: entries << 16 | weights
+    int base_nz, base_cnt;   // entries / weights emitted by the previous passes
     int rem_list[kShortList];
 };
-// dynamic shared memory after TableShared: kSlots * kSlotWords words of second-level counters, then
-// a bitmap of d_out bits for rows with many removed positions
+// dynamic shared memory after TableShared: SLOTS * kSlotWords words of second-level counters, then a bitmap of
+// d_out bits for rows with many removed positions, then the staging area of one pass (key | prefix << 16)
 
-template <int DT, int E, int MAXT, int MINB>
+// Sort keys of two 16-bit patterns at once (neither half is -0): a positive pattern gets its top bit set,
+// a negative one is complemented.
+__device__ __forceinline__ uint32_t keys_of_patterns_x2(uint32_t w) {
+    const uint32_t s = w & 0x80008000u;
+    return w ^ (0x80008000u | (s - (s >> 15)));
+}
+
+// E weights per thread, at most MAXT threads; SLOTS high-byte buckets are refined per pass.
+template <int DT, int E, int MAXT, int MINB, int SLOTS>
 __global__ void __launch_bounds__(MAXT, MINB)
 lloyd_table_kernel(const LloydArgs a, const Tables t) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -117,9 +125,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     if (a.skip_row && a.skip_row[row]) return;
     TableShared& sh = *reinterpret_cast<TableShared*>(smem_raw);
     uint32_t* h2 = reinterpret_cast<uint32_t*>(smem_raw + sizeof(TableShared));
-    uint32_t* bitmap = h2 + kSlots * kSlotWords;
-    uint16_t* st_keys = reinterpret_cast<uint16_t*>(bitmap + (a.d_out + 31) / 32);  // entries of one pass, gathered
-    uint16_t* st_cum = st_keys + kStageCap;
+    uint32_t* bitmap = h2 + SLOTS * kSlotWords;
+    uint32_t* stage = bitmap + (a.d_out + 31) / 32;  // entries of one pass, gathered
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = nthr >> 5;
     const int N = (int)a.d_out;
@@ -153,8 +160,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     int64_t p0 = 0, p1 = 0;
     if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
     const int nrem = (int)(p1 - p0);
-    for (int b = tid; b < 256; b += nthr) sh.hist1[b] = 0;
-    for (int i = tid; i < kSlots * kSlotWords / 4; i += nthr) reinterpret_cast<uint4*>(h2)[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < 64; i += nthr) reinterpret_cast<uint32_t*>(sh.hist1)[i] = 0u;
+    for (int i = tid; i < SLOTS * kSlotWords / 4; i += nthr) reinterpret_cast<uint4*>(h2)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (nrem > kShortList) {
         for (int i = tid; i < (N + 31) / 32; i += nthr) bitmap[i] = 0;
         __syncthreads();
@@ -167,10 +174,13 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     }
     __syncthreads();
 
-    // keys (removed positions and -0 become +0), which high bytes occur, range of the magnitudes
-    uint32_t key[E];
-    uint32_t valid = 0;  // bit e: key[e] is a weight of the row
+    // keys (removed positions and -0 become +0), which high bytes occur, range of the magnitudes.  A group of
+    // VEC weights that lies inside the row, has no removed position and no zero is handled two weights at a
+    // time; everything else weight by weight.
+    uint32_t kw[E / 2];  // two keys per word
+    uint32_t valid = 0;  // bit e: key e is a weight of the row
     uint32_t amax = 0u, amin1 = 0xffffffffu;
+    uint32_t amax2 = 0u, amin2 = 0xffffffffu;  // the same for the pairs: one magnitude per half
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         const int j0 = (g * nthr + tid) * VEC;
@@ -183,36 +193,62 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
                 if (d < (unsigned)VEC) rm |= 1u << d;
             }
         }
+        uint32_t has_zero = 0u;  // non-zero if some magnitude of the group is zero (may also be set without one)
 #pragma unroll
-        for (int u = 0; u < VEC; ++u) {
-            const int e = g * VEC + u;
-            uint32_t h = (raw[e >> 1] >> (16 * (e & 1))) & 0xffffu;
-            if ((rm >> u) & 1u) h = 0u;
-            if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
-            const uint32_t ub = h & 0x7fffu;
-            key[e] = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
-            if (j0 + u < N) {
-                valid |= 1u << e;
-                amax = max(amax, ub);
-                amin1 = min(amin1, ub - 1u);  // zero wraps to the largest value
-                sh.hist1[key[e] >> 8] = 1;
+        for (int u = 0; u < VEC / 2; ++u) {
+            const uint32_t m = raw[g * (VEC / 2) + u] & 0x7fff7fffu;
+            has_zero |= (m - 0x00010001u) & ~m & 0x80008000u;
+        }
+        if (j0 + VEC - 1 < N && rm == 0u && has_zero == 0u) {
+            valid |= ((1u << VEC) - 1u) << (g * VEC);
+#pragma unroll
+            for (int u = 0; u < VEC / 2; ++u) {
+                const uint32_t word = raw[g * (VEC / 2) + u];
+                const uint32_t m = word & 0x7fff7fffu;
+                const uint32_t k2 = keys_of_patterns_x2(word);
+                kw[g * (VEC / 2) + u] = k2;
+                amax2 = __vmaxu2(amax2, m);
+                amin2 = __vminu2(amin2, m - 0x00010001u);  // no half is zero: no borrow
+                sh.hist1[(k2 >> 8) & 0xffu] = 1;
+                sh.hist1[k2 >> 24] = 1;
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < VEC; ++u) {
+                const int e = g * VEC + u;
+                uint32_t h = (raw[e >> 1] >> (16 * (e & 1))) & 0xffffu;
+                if ((rm >> u) & 1u) h = 0u;
+                if (h == 0x8000u) h = 0u;  // -0 and +0 are the same point
+                const uint32_t ub = h & 0x7fffu;
+                const uint32_t key = (h & 0x8000u) ? (~h & 0xffffu) : (h | 0x8000u);
+                if (e & 1) kw[e >> 1] |= key << 16;
+                else kw[e >> 1] = key;
+                if (j0 + u < N) {
+                    valid |= 1u << e;
+                    amax = max(amax, ub);
+                    amin1 = min(amin1, ub - 1u);  // zero wraps to the largest value
+                    sh.hist1[key >> 8] = 1;
+                }
             }
         }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-        amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
-    }
+    amax = max(amax, max(amax2 & 0xffffu, amax2 >> 16));
+    amin1 = min(amin1, min(amin2 & 0xffffu, amin2 >> 16));  // untouched halves read 0xffff: above every pattern - 1
+    amax = __reduce_max_sync(0xffffffffu, amax);
+    amin1 = __reduce_min_sync(0xffffffffu, amin1);
     if (lane == 0) { sh.wtop[warp] = (int)amax; sh.wulp[warp] = (int)amin1; }
     // Every table holds an entry for +0, with count 0 if no weight is zero: a later fit of the same weights
     // with some positions removed (set to +0) then only changes counts, never the list of entries.
     if (tid == 0) sh.hist1[kZeroKeyOfTable >> 8] = 1;
     __syncthreads();
     if (warp == 0) {
+        const uint2 eight = reinterpret_cast<const uint2*>(sh.hist1)[lane];
         int flag[8], sum = 0;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { flag[u] = sh.hist1[lane * 8 + u]; sum += flag[u]; }
+        for (int u = 0; u < 8; ++u) {
+            flag[u] = (int)(((u < 4 ? eight.x : eight.y) >> (8 * (u & 3))) & 1u);
+            sum += flag[u];
+        }
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -233,13 +269,8 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     // the same in all threads.
     bool suspect = false;  // kept in the header: a later fit of a subset of these weights can skip the test
     {
-        amax = lane < nwarps ? (uint32_t)sh.wtop[lane] : 0u;
-        amin1 = lane < nwarps ? (uint32_t)sh.wulp[lane] : 0xffffffffu;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-            amin1 = min(amin1, __shfl_xor_sync(0xffffffffu, amin1, o));
-        }
+        amax = __reduce_max_sync(0xffffffffu, lane < nwarps ? (uint32_t)sh.wtop[lane] : 0u);
+        amin1 = __reduce_min_sync(0xffffffffu, lane < nwarps ? (uint32_t)sh.wulp[lane] : 0xffffffffu);
         // the largest magnitude pattern of the row tells whether any weight is a NaN or an infinity
         if (a.nonfinite && tid == 0 && amax >= (DT == CMPQ_BF16 ? 0x7f80u : 0x7c00u)) atomicOr(a.nonfinite, 2);
         if (amax != 0u) {
@@ -254,15 +285,15 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
                 int q = 100000;
 #pragma unroll
                 for (int e = 0; e < E; ++e) {
-                    const uint32_t ub = __float_as_uint(value_of_key16<DT>(key[e])) & 0x7fffffffu;
+                    const uint32_t key = (kw[e >> 1] >> (16 * (e & 1))) & 0xffffu;
+                    const uint32_t ub = __float_as_uint(value_of_key16<DT>(key)) & 0x7fffffffu;
                     if (((valid >> e) & 1u) && ub) {
                         const int ex = (int)(ub >> 23);
                         const uint32_t m = ub & 0x7fffffu;
                         q = min(q, ex ? ex - 150 + (__ffs(m | 0x800000u) - 1) : (__ffs(m) - 1) - 149);
                     }
                 }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) q = min(q, __shfl_xor_sync(0xffffffffu, q, o));
+                q = __reduce_min_sync(0xffffffffu, q);
                 __syncthreads();  // every warp has read wtop / wulp
                 if (lane == 0) sh.wulp[warp] = q;
                 __syncthreads();
@@ -278,9 +309,10 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
     uint16_t* keys = t.keys + row * t.stride;
     uint16_t* cum = t.cum + row * t.stride;
     const int n_nonempty = sh.n_nonempty;
+    constexpr uint32_t kAllValid = E == 32 ? 0xffffffffu : (1u << E) - 1u;
     int run_nz = 0, run_cnt = 0;
-    for (int g0 = 0; g0 < n_nonempty; g0 += kSlots) {
-        const int nslots = n_nonempty - g0 < kSlots ? n_nonempty - g0 : kSlots;
+    for (int g0 = 0; g0 < n_nonempty; g0 += SLOTS) {
+        const int nslots = n_nonempty - g0 < SLOTS ? n_nonempty - g0 : SLOTS;
         const int words_total = nslots * kSlotWords;
         // Second level: the low byte inside the buckets g0 .. g0 + nslots.  Two 16-bit counters share a
         // word (a channel has fewer than 2^16 weights, so the halves never carry into each other).
@@ -290,78 +322,112 @@ lloyd_table_kernel(const LloydArgs a, const Tables t) {
         }
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if ((valid >> e) & 1u) {
-                const int r = sh.bucket_rank[key[e] >> 8] - g0;
-                const uint32_t lo = key[e] & 0xffu;
-                if (r >= 0 && r < kSlots) atomicAdd(&h2[r * kSlotWords + (lo >> 1)], 1u << (16 * (lo & 1u)));
+            if (valid == kAllValid || ((valid >> e) & 1u)) {
+                const uint32_t key = (kw[e >> 1] >> (16 * (e & 1))) & 0xffffu;
+                const int r = sh.bucket_rank[key >> 8] - g0;
+                if ((unsigned)r < (unsigned)SLOTS) atomicAdd(&h2[r * kSlotWords + ((key & 0xffu) >> 1)], (key & 1u) ? 0x10000u : 1u);
             }
         }
         __syncthreads();
         // Every thread owns a contiguous range of counters: totals first, a block scan, then the entries.
-        const int w0 = (int)((long long)tid * words_total / nthr);
-        const int w1 = (int)((long long)(tid + 1) * words_total / nthr);
-        int nz = 0, cnt = 0;
-        uint32_t occupied = 0;  // bit 2 (w - w0) + half: that counter makes an entry (ranges of at most 16 words)
-        const int r_zero = sh.bucket_rank[kZeroKeyOfTable >> 8] - g0;  // the counter of +0 always makes one
+        // With at most kScanWords words per thread (a power of two, so a range stays inside one bucket) the
+        // counters of a thread are held in registers between the two steps.
+        int wpt = 4;
+        while (wpt * nthr < words_total) wpt *= 2;
+        const bool in_regs = wpt <= kScanWords;
+        const int w0 = in_regs ? min(tid * wpt, words_total) : (int)((unsigned)tid * (unsigned)words_total / (unsigned)nthr);
+        const int w1 = in_regs ? min(w0 + wpt, words_total) : (int)((unsigned)(tid + 1) * (unsigned)words_total / (unsigned)nthr);
+        const int r_zero = sh.bucket_rank[kZeroKeyOfTable >> 8] - g0;  // the counter of +0 always makes an entry
         const int w_zero = (r_zero >= 0 && r_zero < nslots) ? r_zero * kSlotWords : -1;
-        for (int w = w0; w < w1; ++w) {
-            const uint32_t word = h2[w];
-            const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-            const bool e0 = c0 != 0 || w == w_zero, e1 = c1 != 0;
-            nz += (e0 ? 1 : 0) + (e1 ? 1 : 0);
-            cnt += c0 + c1;
-            if (w - w0 < 16) occupied |= ((e0 ? 1u : 0u) | (e1 ? 2u : 0u)) << (2 * (w - w0));
-        }
-        int inz = nz, icnt = cnt;
+        uint32_t occupied = 0;  // bit 2 (w - w0) + half: that counter makes an entry (register path)
+        int nz = 0, cnt = 0;
+        if (in_regs) {
+            uint32_t total = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int unz = __shfl_up_sync(0xffffffffu, inz, o);
-            const int ucnt = __shfl_up_sync(0xffffffffu, icnt, o);
-            if (lane >= o) { inz += unz; icnt += ucnt; }
-        }
-        if (lane == 31) { sh.w_nz[warp] = inz; sh.w_cnt[warp] = icnt; }
-        __syncthreads();
-        run_nz = sh.base_nz + inz - nz;
-        run_cnt = sh.base_cnt + icnt - cnt;
-        int pass_nz = 0;  // entries of this pass (all warps)
-        for (int wv = 0; wv < nwarps; ++wv) {
-            if (wv < warp) { run_nz += sh.w_nz[wv]; run_cnt += sh.w_cnt[wv]; }
-            pass_nz += sh.w_nz[wv];
-        }
-        // The entries of a pass are gathered in shared memory when they fit and leave in order with
-        // coalesced stores; a thread walks the set bits of its range instead of every counter.
-        const bool staged = pass_nz <= kStageCap;
-        const int stage_base = sh.base_nz;
-        uint16_t* out_keys = staged ? st_keys - stage_base : keys;
-        uint16_t* out_cum = staged ? st_cum - stage_base : cum;
-        if (w1 - w0 <= 16) {
-            while (occupied) {
-                const int b = __ffs(occupied) - 1;
-                occupied &= occupied - 1u;
-                const int w = w0 + (b >> 1);
-                const int c = (int)((h2[w] >> (16 * (b & 1))) & 0xffffu);
-                const uint32_t k = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1) | (uint32_t)(b & 1);
-                out_keys[run_nz] = (uint16_t)k;
-                out_cum[run_nz] = (uint16_t)run_cnt;
-                ++run_nz;
-                run_cnt += c;
+            for (int q = 0; q < kScanWords / 4; ++q) {
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (w0 + 4 * q < w1) v = *reinterpret_cast<const uint4*>(h2 + w0 + 4 * q);
+                const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    total = __dp2a_lo(wd[i], 0x0101u, total);  // both halves added
+                    occupied |= ((wd[i] & 0xffffu) ? 1u : 0u) << (2 * (4 * q + i));
+                    occupied |= ((wd[i] >> 16) ? 1u : 0u) << (2 * (4 * q + i) + 1);
+                }
             }
+            if (w_zero >= w0 && w_zero < w1) occupied |= 1u << (2 * (w_zero - w0));
+            nz = __popc(occupied);
+            cnt = (int)total;
         } else {
             for (int w = w0; w < w1; ++w) {
                 const uint32_t word = h2[w];
-                if (word || w == w_zero) {
-                    const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
-                    const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
-                    if (c0 || w == w_zero) { out_keys[run_nz] = (uint16_t)kb; out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c0; }
-                    if (c1) { out_keys[run_nz] = (uint16_t)(kb | 1u); out_cum[run_nz] = (uint16_t)run_cnt; ++run_nz; run_cnt += c1; }
+                const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
+                nz += ((c0 != 0 || w == w_zero) ? 1 : 0) + (c1 != 0 ? 1 : 0);
+                cnt += c0 + c1;
+            }
+        }
+        // block scan of (entries, weights) in one word: neither total reaches 2^16
+        const uint32_t mine = ((uint32_t)nz << 16) | (uint32_t)cnt;
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) sh.w_scan[warp] = incl;
+        __syncthreads();
+        const uint32_t wv = lane < nwarps ? sh.w_scan[lane] : 0u;
+        const uint32_t before = __reduce_add_sync(0xffffffffu, lane < warp ? wv : 0u) + incl - mine;
+        const int pass_nz = (int)(__reduce_add_sync(0xffffffffu, wv) >> 16);  // entries of this pass (all warps)
+        run_nz = sh.base_nz + (int)(before >> 16);
+        run_cnt = sh.base_cnt + (int)(before & 0xffffu);
+        // The entries of a pass are gathered in shared memory when they fit and leave in order with
+        // coalesced stores.
+        const bool staged = pass_nz <= kStageCap;
+        const int stage_base = sh.base_nz;
+        auto emit_range = [&](auto&& put) {
+            if (in_regs) {  // a thread walks the set bits of its range instead of every counter
+                const uint32_t kb0 = w0 < words_total
+                    ? ((uint32_t)sh.slot_hi[g0 + (w0 >> 7)] << 8) | ((uint32_t)(w0 & 127) << 1) : 0u;
+                while (occupied) {
+                    const int b = __ffs(occupied) - 1;
+                    occupied &= occupied - 1u;
+                    const uint32_t word = h2[w0 + (b >> 1)];
+                    put(kb0 + (uint32_t)b, (int)((b & 1) ? word >> 16 : word & 0xffffu));
+                }
+            } else {
+                for (int w = w0; w < w1; ++w) {
+                    const uint32_t word = h2[w];
+                    if (word || w == w_zero) {
+                        const uint32_t kb = ((uint32_t)sh.slot_hi[g0 + (w >> 7)] << 8) | ((uint32_t)(w & 127) << 1);
+                        const int c0 = (int)(word & 0xffffu), c1 = (int)(word >> 16);
+                        if (c0 || w == w_zero) put(kb, c0);
+                        if (c1) put(kb | 1u, c1);
+                    }
                 }
             }
+        };
+        if (staged) {
+            uint32_t* out = stage - stage_base;
+            emit_range([&](uint32_t k, int c) {
+                out[run_nz] = k | ((uint32_t)run_cnt << 16);
+                ++run_nz;
+                run_cnt += c;
+            });
+        } else {
+            emit_range([&](uint32_t k, int c) {
+                keys[run_nz] = (uint16_t)k;
+                cum[run_nz] = (uint16_t)run_cnt;
+                ++run_nz;
+                run_cnt += c;
+            });
         }
         __syncthreads();  // every thread has read the bases and the counters of this pass
         if (staged) {
             for (int i = tid; i < pass_nz; i += nthr) {
-                keys[stage_base + i] = st_keys[i];
-                cum[stage_base + i] = st_cum[i];
+                const uint32_t en = stage[i];
+                keys[stage_base + i] = (uint16_t)en;
+                cum[stage_base + i] = (uint16_t)(en >> 16);
             }
         }
         if (tid == nthr - 1) { sh.base_nz = run_nz; sh.base_cnt = run_cnt; }
@@ -1214,10 +1280,12 @@ __device__ __forceinline__ void table_hist_row(const Tables& t, int64_t row, uin
     }
 }
 
-// A row fitted with valid thresholds: lane 2k walks the left side of cluster k (values below c_k) upwards
-// from its first entry, lane 2k + 1 the right side downwards from its last entry.  Along such a walk the
-// error |v - c_k| (fp32, the rounding is monotone) never grows, so the walk ends at the first error below
-// `lo`: visit(error pattern, count, key) sees exactly the non-empty entries of the row with error >= lo.
+// A row fitted with valid thresholds: lane 2k takes the left side of cluster k (entries below c_k), lane
+// 2k + 1 the right side.  Towards the centroid the error |v - c_k| (fp32, the rounding is monotone) never
+// grows, so the entries of a side with error >= lo are the ones at its outer end.  A lane reads its side
+// eight table entries at a time (two 128-bit loads), starting at the outer end, and stops after the first
+// group that holds a smaller error: visit(error pattern, count, key) sees exactly the non-empty entries of
+// the row with error >= lo, each once.
 template <int DT, class Visit>
 __device__ __forceinline__ void walk_row_sides(const Tables& t, int64_t row, int K, uint32_t lo, Visit&& visit) {
     const int lane = threadIdx.x & 31;
@@ -1227,19 +1295,28 @@ __device__ __forceinline__ void walk_row_sides(const Tables& t, int64_t row, int
     const uint16_t* bnd = t.bnd + row * 32;
     const int M = t.hdr[row].M;
     const int first = bnd[2 * k], mid = bnd[2 * k + 1], next = k + 1 < K ? (int)bnd[2 * k + 2] : M;
+    const int j_lo = left ? first : mid, j_hi = left ? mid : next;  // the side: entries [j_lo, j_hi)
+    if (j_lo >= j_hi) return;
     const float c = t.lut[row * CMPQ_LUT_STRIDE + k];
     const uint16_t* keys = t.keys + row * t.stride;
     const uint16_t* cum = t.cum + row * t.stride;
-    int j = left ? first : next - 1;
-    const int stop = left ? mid : mid - 1, step = left ? 1 : -1;
-    while (j != stop) {
-        const uint32_t key = keys[j], c0 = cum[j], c1 = cum[j + 1];
-        if (c1 != c0) {
-            const uint32_t e = __float_as_uint(fabsf(value_of_key16<DT>(key) - c));
-            if (e < lo) break;
-            visit(e, c1 - c0, key);
+    int g = (left ? j_lo : j_hi - 1) & ~7;
+    for (;;) {
+        const Eight k8 = load_eight(keys + g), c8 = load_eight(cum + g);
+        const uint32_t c_end = g + 8 <= M ? cum[g + 8] : 0u;
+        bool below = false;  // an entry of the side with error < lo: everything further in is smaller still
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t cnt = (u < 7 ? c8.at(u + 1) : c_end) - c8.at(u);
+            if (g + u >= j_lo && g + u < j_hi && cnt != 0u) {
+                const uint32_t e = __float_as_uint(fabsf(value_of_key16<DT>(k8.at(u)) - c));
+                if (e >= lo) visit(e, cnt, k8.at(u));
+                else below = true;
+            }
         }
-        j += step;
+        if (below) break;
+        g += left ? 8 : -8;
+        if (left ? g >= j_hi : g + 8 <= j_lo) break;
     }
 }
 
@@ -1486,21 +1563,40 @@ __device__ void table_emit_row(const uint16_t* __restrict__ w, int64_t d_out, co
 __device__ void table_emit_row_by_keys(const uint16_t* __restrict__ w, int64_t d_out, const uint32_t* __restrict__ kept,
                                        int nkept, int64_t row, int te, int64_t out0, int32_t* __restrict__ rows,
                                        int32_t* __restrict__ cols, uint16_t* __restrict__ vals, int* list_col,
-                                       unsigned char* list_eq, int* list_n, uint32_t* s_kept) {
+                                       unsigned char* list_eq, int* list_n, uint32_t* s_kept, const uint4 first) {
     if (threadIdx.x == 0) *list_n = 0;
-    if ((int)threadIdx.x < nkept) s_kept[threadIdx.x] = kept[1 + threadIdx.x];
+    // Almost no weight is a candidate, and candidates lie far from their centroids: a weight whose magnitude
+    // is below the smallest magnitude among the listed values cannot be one.
+    if (threadIdx.x < 32) {  // at most kKeptCap = 31 listed values: the last slot carries that magnitude
+        uint32_t mag = 0x7fffu;
+        if ((int)threadIdx.x < nkept) {
+            const uint32_t kk = kept[1 + threadIdx.x];
+            s_kept[threadIdx.x] = kk;
+            mag = (kk & 0xffffu) >= 0x8000u ? kk & 0x7fffu : 0x7fffu - (kk & 0xffffu);
+        }
+        mag = __reduce_min_sync(0xffffffffu, mag);
+        if (threadIdx.x == 31) s_kept[31] = mag;
+    }
     __syncthreads();
+    const uint32_t mag_bias = (0x8000u - s_kept[31]) * 0x00010001u;
     const bool vec = ((reinterpret_cast<uintptr_t>(w) & 15) == 0);
     for (int64_t j0 = (int64_t)threadIdx.x * 8; j0 < d_out; j0 += (int64_t)blockDim.x * 8) {
         uint32_t pk[4] = {0u, 0u, 0u, 0u};
         if (j0 + 7 < d_out && vec) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(w + j0));
+            // the first eight weights of a thread were requested when the kernel started
+            const uint4 v = j0 == (int64_t)threadIdx.x * 8 ? first : __ldg(reinterpret_cast<const uint4*>(w + j0));
             pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
         } else {
 #pragma unroll
             for (int u = 0; u < 8; ++u)
                 if (j0 + u < d_out) pk[u >> 1] |= (uint32_t)w[j0 + u] << (16 * (u & 1));
         }
+        // two magnitudes per word against the smallest listed one: bit 15 of a half survives the addition
+        // exactly when that weight is at least as large (no carry between the halves: both terms < 2^15 + 1)
+        uint32_t large = 0u;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) large |= ((pk[q] & 0x7fff7fffu) + mag_bias) & 0x80008000u;
+        if (!large) continue;
         uint32_t key[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -1557,9 +1653,13 @@ table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, c
     __shared__ int list_n;
     __shared__ uint32_t s_kept[32];
     const int64_t row = blockIdx.x;
+    const uint16_t* w = W + row * ldw;
+    // nearly every row keeps something: its weights are requested before anything else is looked at
+    uint4 first = make_uint4(0u, 0u, 0u, 0u);
+    if ((reinterpret_cast<uintptr_t>(w) & 15) == 0 && (int64_t)threadIdx.x * 8 + 7 < d_out)
+        first = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)threadIdx.x * 8));
     const int64_t out0 = row_start[row];
     if (row_start[row + 1] == out0) return;
-    const uint16_t* w = W + row * ldw;
     if (is_act[row]) {
         for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
             rows[out0 + j] = (int32_t)row;
@@ -1575,7 +1675,7 @@ table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, c
     const uint32_t nkept = t.kept[row * 32];
     if (nkept != kKeptUnknown && ncand <= kEmitListCap) {
         table_emit_row_by_keys(w, d_out, t.kept + row * 32, (int)nkept, row, te, out0, rows, cols, vals, list_col, list_eq,
-                               &list_n, s_kept);
+                               &list_n, s_kept, first);
         return;
     }
     if (b == 2) table_emit_row<DT, 4>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
@@ -1634,11 +1734,11 @@ cmpq_status launch_table_emit(void* tables, size_t tables_bytes, cmpq_dtype dt, 
 // ------------------------------------------------------------------------------------------------
 // host side
 
-template <int DT, int E, int MAXT, int MINB>
+template <int DT, int E, int MAXT, int MINB, int SLOTS>
 static cmpq_status launch_table(const LloydArgs& args, const Tables& t, int threads, cudaStream_t st) {
-    const size_t smem = sizeof(TableShared) + (size_t)kSlots * kSlotWords * sizeof(uint32_t) +
-                        (((size_t)args.d_out + 31) / 32) * sizeof(uint32_t) + (size_t)kStageCap * 2 * sizeof(uint16_t);
-    auto kern = lloyd_table_kernel<DT, E, MAXT, MINB>;
+    const size_t smem = sizeof(TableShared) + (size_t)SLOTS * kSlotWords * sizeof(uint32_t) +
+                        (((size_t)args.d_out + 31) / 32) * sizeof(uint32_t) + (size_t)kStageCap * sizeof(uint32_t);
+    auto kern = lloyd_table_kernel<DT, E, MAXT, MINB, SLOTS>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return CMPQ_ERR_CUDA;
     kern<<<(unsigned)args.d_in, threads, smem, st>>>(args, t);
@@ -1668,15 +1768,17 @@ static cmpq_status launch_table_dt(const LloydArgs& args, const Tables& t, cudaS
         th = (th + 31) / 32 * 32;
         return (int)(th < 32 ? 32 : th);
     };
-    if (N <= 2048) return launch_table<DT, 4, 512, 2>(args, t, threads_for(4), st);
-    if (N <= 4096) return launch_table<DT, 16, 256, 4>(args, t, threads_for(16), st);
-    if (N <= 8192) return launch_table<DT, 16, 512, 2>(args, t, threads_for(16), st);
-    if (N <= 16384) return launch_table<DT, 16, 1024, 1>(args, t, threads_for(16), st);
-    return launch_table<DT, 32, 1024, 1>(args, t, threads_for(32), st);
+    // 32 high-byte buckets per pass cover a zero-centred channel of a few thousand weights in one pass; longer
+    // rows reach further into the small magnitudes and get 64
+    if (N <= 2048) return launch_table<DT, 4, 512, 2, 32>(args, t, threads_for(4), st);
+    if (N <= 4096) return launch_table<DT, 16, 256, 4, 32>(args, t, threads_for(16), st);
+    if (N <= 8192) return launch_table<DT, 16, 512, 2, 32>(args, t, threads_for(16), st);
+    if (N <= 16384) return launch_table<DT, 16, 1024, 1, 64>(args, t, threads_for(16), st);
+    return launch_table<DT, 32, 1024, 1, 64>(args, t, threads_for(32), st);
 }
 
 const void* lloyd_table_kernel_address() {
-    return reinterpret_cast<const void*>(&lloyd_table_kernel<CMPQ_BF16, 16, 256, 4>);
+    return reinterpret_cast<const void*>(&lloyd_table_kernel<CMPQ_BF16, 16, 256, 4, 32>);
 }
 
 // tables_ready: the value tables of every row to be fitted are in place already (skip the table kernel)

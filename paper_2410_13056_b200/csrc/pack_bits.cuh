@@ -62,19 +62,18 @@ __device__ __forceinline__ void pack_layout_block(const uint8_t* __restrict__ bi
     }
     if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    unsigned long long base = 0, total = 0;
-    for (int w = 0; w < nwarps; ++w) {
-        unsigned long long t = warp_tot[w];
-        if (w < warp) base += t;
-        total += t;
-    }
-    const unsigned long long before = base + incl - mine;
+    // lane w holds the total of warp w: the three 21-bit fields are summed separately, over the warps below
+    // this one and over all of them
+    const unsigned long long wt = lane < nwarps ? warp_tot[lane] : 0ull;
+    const unsigned long long own = incl - mine;
     long long seen[3], count[3], words[3], seg_base[3], seg_word_base[3];
     long long rb = 0, wb = 0;
 #pragma unroll
     for (int sgm = 0; sgm < 3; ++sgm) {
-        seen[sgm] = (long long)((before >> (21 * sgm)) & 0x1fffffull);
-        count[sgm] = (long long)((total >> (21 * sgm)) & 0x1fffffull);
+        const unsigned f = (unsigned)((wt >> (21 * sgm)) & 0x1fffffull);
+        seen[sgm] = (long long)(__reduce_add_sync(0xffffffffu, lane < warp ? f : 0u) +
+                                (unsigned)((own >> (21 * sgm)) & 0x1fffffull));
+        count[sgm] = (long long)__reduce_add_sync(0xffffffffu, f);
         words[sgm] = (d_out * (sgm + 2) + 31) / 32;
         seg_base[sgm] = rb;
         seg_word_base[sgm] = wb;

@@ -30,14 +30,9 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_totals, int
     __syncthreads();  // warp_totals may still be read from a previous call
     if (lane == 31) warp_totals[warp] = incl;
     __syncthreads();
-    int base = 0, all = 0;
-    for (int w = 0; w < nwarps; ++w) {
-        int t = warp_totals[w];
-        if (w < warp) base += t;
-        all += t;
-    }
-    total = all;
-    return base + incl - v;
+    const int t = lane < nwarps ? warp_totals[lane] : 0;  // at most 32 warps: one total per lane
+    total = __reduce_add_sync(0xffffffffu, t);
+    return __reduce_add_sync(0xffffffffu, lane < warp ? t : 0) + incl - v;
 }
 
 // One block: walks the histogram from the largest digit down to the one that holds the

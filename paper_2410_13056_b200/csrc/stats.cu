@@ -169,22 +169,33 @@ stats_partial_scalar_kernel(const uint16_t* __restrict__ X, int64_t n_tokens, in
     partial[((int64_t)blockIdx.y * gridDim.x + tile) * kTileCols + threadIdx.x] = total;
 }
 
-// sumsq[j] += sum over row blocks (ascending) of partial[rb][j]   (l_inf: the maximum instead of the sum)
+// sumsq[j] += sum over the row blocks of partial[rb][j]   (l_inf: the maximum instead of the sum), always in
+// the same order: warp p of a block adds the row blocks p, p + 8, p + 16, ... of 32 columns (one per lane), then
+// warp 0 adds the eight part sums in ascending p.
 // A NaN or an infinity among the activations of a column (or an fp32 square beyond the fp32 range) makes
 // the column's partial result non-finite: bit 0 of *nonfinite is set (nonfinite may be NULL).
-__global__ void stats_combine_kernel(const double* __restrict__ partial, int64_t row_blocks,
-                                     int64_t padded_cols, int64_t d_in, double* __restrict__ sumsq, int take_max,
-                                     int32_t* nonfinite) {
-    int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= d_in) return;
+constexpr int kCombineParts = 8;
+__global__ void __launch_bounds__(32 * kCombineParts)
+stats_combine_kernel(const double* __restrict__ partial, int64_t row_blocks, int64_t padded_cols, int64_t d_in,
+                     double* __restrict__ sumsq, int take_max, int32_t* nonfinite) {
+    __shared__ double part_sum[kCombineParts][32];
+    const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+    const int64_t j = (int64_t)blockIdx.x * 32 + lane;
     double s = 0.0;
-    if (take_max) {
-        for (int64_t rb = 0; rb < row_blocks; ++rb) s = max_keep_nan(s, partial[rb * padded_cols + j]);
-        sumsq[j] = max_keep_nan(sumsq[j], s);
-    } else {
-        for (int64_t rb = 0; rb < row_blocks; ++rb) s += partial[rb * padded_cols + j];
-        sumsq[j] += s;
+    if (j < d_in) {
+        if (take_max) {
+            for (int64_t rb = part; rb < row_blocks; rb += kCombineParts) s = max_keep_nan(s, partial[rb * padded_cols + j]);
+        } else {
+            for (int64_t rb = part; rb < row_blocks; rb += kCombineParts) s += partial[rb * padded_cols + j];
+        }
     }
+    part_sum[part][lane] = s;
+    __syncthreads();
+    if (part != 0 || j >= d_in) return;
+    s = part_sum[0][lane];
+#pragma unroll
+    for (int p = 1; p < kCombineParts; ++p) s = take_max ? max_keep_nan(s, part_sum[p][lane]) : s + part_sum[p][lane];
+    sumsq[j] = take_max ? max_keep_nan(sumsq[j], s) : sumsq[j] + s;
     if (nonfinite && !(fabs(s) <= 1.7976931348623157e308)) atomicOr(nonfinite, 1);
 }
 
@@ -222,8 +233,8 @@ cmpq_status launch_collect_stats_norm(const void* X, cmpq_dtype dt, int64_t n_to
     if (norm == CMPQ_NORM_L2) launch_partial<CMPQ_NORM_L2>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
     else if (norm == CMPQ_NORM_L1) launch_partial<CMPQ_NORM_L1>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
     else launch_partial<CMPQ_NORM_LINF>(Xp, dt, vec, grid, n_tokens, d_in, ldx, rows_per_block, partial, st);
-    stats_combine_kernel<<<(unsigned)((d_in + 255) / 256), 256, 0, st>>>(partial, row_blocks, ct * kTileCols, d_in, sumsq,
-                                                                          norm == CMPQ_NORM_LINF, nonfinite);
+    stats_combine_kernel<<<(unsigned)((d_in + 31) / 32), 32 * kCombineParts, 0, st>>>(partial, row_blocks, ct * kTileCols, d_in,
+                                                                                   sumsq, norm == CMPQ_NORM_LINF, nonfinite);
     return launch_status();
 }
 
