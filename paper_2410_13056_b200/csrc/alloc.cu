@@ -100,7 +100,7 @@ __device__ __forceinline__ uint32_t ordered_bits(float v) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Small per-layer steps that ride along with a rank-cut launch (one block, nothing else running yet):
+// Small per-layer steps that ride along with a rank-cut launch (a second block, nothing else running yet):
 // the layout of the packed segments from the widths, and the start state of the radix select.
 struct CutExtras {
     const uint8_t* bits;     // pack layout wanted: widths, and its five outputs
@@ -124,6 +124,17 @@ rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long lo
     __shared__ unsigned long long warp_tot[32];
     __shared__ uint32_t warp_min[32], warp_max[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (blockIdx.x == 1) {  // the steps that ride along need nothing from the cut: a block of their own
+        if (x.select) {
+            if (tid == 0) {
+                SelectState* st = x.select;
+                st->prefix = 0; st->mask = 0; st->remaining = x.n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0; st->lower = 0;
+            }
+            for (int b = tid; b < kSelBins; b += kCutThreads) x.hist[b] = 0u;
+        }
+        if (x.bits) pack_layout_block(x.bits, d_in, x.d_out, x.row_off, x.perm, x.seg_rows, x.word_off, warp_tot);
+        return;
+    }
     const long long k[2] = {k0, k1};
     const bool live[2] = {k0 < d_in, k1 < d_in};
     if (tid < 2) { prefix[tid] = 0u; remaining[tid] = k[tid] < 0 ? 0 : k[tid]; }
@@ -253,17 +264,6 @@ rank_cut_kernel(const float* __restrict__ a, int64_t d_in, long long k0, long lo
             out[i] = (uint8_t)cls;
         }
     }
-    if (x.select) {
-        if (tid == 0) {
-            SelectState* st = x.select;
-            st->prefix = 0; st->mask = 0; st->remaining = x.n_q; st->tau = 0xffffffffu; st->take_equal = 0; st->done = 0; st->lower = 0;
-        }
-        for (int b = tid; b < kSelBins; b += kCutThreads) x.hist[b] = 0u;
-    }
-    if (x.bits) {
-        __syncthreads();  // warp_tot is free again
-        pack_layout_block(x.bits, d_in, x.d_out, x.row_off, x.perm, x.seg_rows, x.word_off, warp_tot);
-    }
 }
 
 cmpq_status launch_rank_cut(const float* a, int64_t d_in, int64_t k0, int64_t k1, int base, uint8_t* out,
@@ -287,7 +287,7 @@ cmpq_status launch_act_cut(const float* a, int64_t d_in, int64_t n_act, uint8_t*
     x.perm = perm;
     x.seg_rows = seg_rows;
     x.word_off = word_off;
-    rank_cut_kernel<<<1, kCutThreads, 0, st>>>(a, d_in, (long long)(d_in - n_act), (long long)d_in, 0, is_act, x);
+    rank_cut_kernel<<<2, kCutThreads, 0, st>>>(a, d_in, (long long)(d_in - n_act), (long long)d_in, 0, is_act, x);
     return launch_status();
 }
 
