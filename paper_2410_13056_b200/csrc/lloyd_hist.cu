@@ -1076,11 +1076,15 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
     float c[K], t[K];
 #pragma unroll
-    for (int k = 0; k < K; ++k) {
-        c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
-        t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
-    }
+    for (int k = 0; k < K; ++k) t[k] = __ldg(thr + row * CMPQ_LUT_STRIDE + k);
     const bool by_threshold = t[0] != 0.f;
+    if (ERR || !by_threshold) {  // codes by thresholds never look at the centroids
+#pragma unroll
+        for (int k = 0; k < K; ++k) c[k] = __ldg(lut + row * CMPQ_LUT_STRIDE + k);
+    } else {
+#pragma unroll
+        for (int k = 0; k < K; ++k) c[k] = 0.f;
+    }
     // codes only, by thresholds: two weights per compare in the storage type.  A count c sits in
     // the low mantissa bits of 128 + c (bf16) or 1024 + c (fp16).
     uint32_t t2[K];
@@ -1121,12 +1125,17 @@ __device__ void assign_row(const LloydArgs& a, int64_t row, const float* __restr
                 }
             }
             if (!ERR && by_threshold && j0 + 7 < N) {
+                if (mask) {  // rare: removed positions become +0
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if ((mask >> (2 * q)) & 1u) pk[q] &= 0xffff0000u;
+                        if ((mask >> (2 * q + 1)) & 1u) pk[q] &= 0x0000ffffu;
+                    }
+                }
                 uint32_t r[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    uint32_t x2 = pk[q];
-                    if ((mask >> (2 * q)) & 1u) x2 &= 0xffff0000u;      // removed positions become +0
-                    if ((mask >> (2 * q + 1)) & 1u) x2 &= 0x0000ffffu;
+                    const uint32_t x2 = pk[q];
                     uint32_t acc = acc0;
 #pragma unroll
                     for (int k = 1; k < K; ++k) acc = add_ge_x2<DT>(acc, x2, t2[k]);
@@ -1830,8 +1839,11 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
     if (ev[2]) cudaEventRecord(ev[2], st);
 
     // neither codes nor errors wanted: the fit alone (centroids and thresholds stay in the tables)
-    if (args.err) lloyd_assign_kernel<DT, true><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
-    else if (args.codes || args.packed) lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, kAssignThreads, 0, st>>>(args, ia.lut, t.thr);
+    // a short row keeps fewer threads busy for longer: the per-row set-up (centroids, thresholds, removed
+    // columns) is paid once per thread
+    const int assign_threads = N <= 4096 ? kAssignThreads / 2 : kAssignThreads;
+    if (args.err) lloyd_assign_kernel<DT, true><<<(unsigned)args.d_in, assign_threads, 0, st>>>(args, ia.lut, t.thr);
+    else if (args.codes || args.packed) lloyd_assign_kernel<DT, false><<<(unsigned)args.d_in, assign_threads, 0, st>>>(args, ia.lut, t.thr);
     s = launch_status();
     if (ev[3]) cudaEventRecord(ev[3], st);
     return s;
