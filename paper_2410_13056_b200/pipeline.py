@@ -17,7 +17,7 @@ from . import binding as B
 # Fused, default assignment (cmpq_protect_quantize_pack): statistic 2 + finalize 1, allocation 1 (two rank cuts
 # in one block), outlier step 10 (O_act cut with select start and pack layout, value tables, provisional
 # iterations, lower bound, 3 select passes, row counts, row scan, emit), final fit 2 (iterations that patch the
-# tables, last assignment that packs) = 17.
+# tables, last assignment that packs) = 16.
 # Separate calls: the final fit builds its own tables (row index, tables, iterations, assignment = 4) and the
 # packing takes 2 more = 20.  All-pairs assignment: the provisional fit is one kernel and every select pass is
 # followed by a digit kernel (outlier step 11), the final fit is row index + one kernel, packing 2 = 19; fused
@@ -27,7 +27,7 @@ def kernels_per_run(assignment=None, fused=False):
         assignment = B.cmpq_get_lloyd_assignment()
     if assignment == B.ASSIGN_ALL_PAIRS:
         return 18 if fused else 19
-    return 17 if fused else 20
+    return 16 if fused else 20
 
 
 KERNELS_PER_RUN = 20
