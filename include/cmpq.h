@@ -190,11 +190,16 @@ cmpq_status cmpq_extract_outliers(const void* W, cmpq_dtype dt, int64_t d_in, in
  * sens: NULL for the paper's unweighted K-means.  Otherwise [d_in][d_out] fp32 sensitivities s >= 0
  * (finite), one per weight: the update becomes the weighted mean  c_k = sum s x / sum s  over the
  * members (a cluster whose members' sensitivities sum to 0 keeps c_k); start and assignment are
- * unchanged.  The products s*x are not exact in fp64, so the sums depend on the order of summation:
- * the result is deterministic, and agrees with a sequential sum to rounding (centroids to about
- * 1e-7 relative; with all s equal it equals the unweighted fit bit for bit whenever inexact_rows
- * stays 0 there).  The weighted fit evaluates all pairs whatever cmpq_set_lloyd_assignment says and
- * leaves inexact_rows untouched.
+ * unchanged.  The weighted sums are not exact in fp64, so they depend on the order of summation: the
+ * result is deterministic (the same inputs give the same bytes) and agrees with a sequential sum to
+ * rounding (centroids to about 1e-7 relative); with all s equal to one power of two it equals the
+ * unweighted fit bit for bit whenever inexact_rows stays 0 there.  With CMPQ_ASSIGN_ORDERED the fit
+ * works on the value tables: the sensitivities of the weights that share a value are added in 64-bit
+ * fixed point (scaled by a power of two so that a channel's total stays below 2^52; a sensitivity
+ * below 2^-(52 - ceil(log2 d_out)) of the channel's largest loses its low bits), and cluster sums are
+ * differences of fp64 prefix sums over the distinct values.  With CMPQ_ASSIGN_ALL_PAIRS, and for a
+ * channel with more than 11264 distinct values, every weight is scanned against every centroid in
+ * every iteration.  inexact_rows is left untouched.
  * inexact_rows (optional device int32, caller zeroes it): incremented for every channel whose
  * dynamic range is so wide that fp64 cluster sums may depend on the order of summation; when
  * it stays 0 the centroids are independent of the summation order, hence reproducible bit

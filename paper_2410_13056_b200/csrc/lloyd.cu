@@ -692,7 +692,11 @@ static cmpq_status quantize_impl(const void* W, cmpq_dtype dt, int64_t d_in, int
     a.sweeps = sweeps;
     a.nonfinite = nonfinite;
     if (!fused_pack_ok) {
-        s = sens ? launch_lloyd_weighted(a, dt, sens, st) : launch_lloyd(a, dt, st);
+        if (sens && lloyd_assignment() != CMPQ_ASSIGN_ALL_PAIRS)
+            s = launch_lloyd_weighted_tables(a, dt, sens, static_cast<char*>(ws) + row_ptr_bytes(d_in),
+                                             lloyd_tables_bytes(d_in, d_out), st);
+        else
+            s = sens ? launch_lloyd_weighted(a, dt, sens, st) : launch_lloyd(a, dt, st);
         if (s != CMPQ_OK || !packed) return s;
         return launch_pack_codes(codes, bits, d_in, d_out, word_off, packed, st);
     }

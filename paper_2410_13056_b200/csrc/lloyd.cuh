@@ -83,6 +83,9 @@ cmpq_status launch_lloyd_ordered(const LloydArgs& args, cmpq_dtype dt, void* tab
 // Weighted fit (sens: [d_in][d_out] fp32 sensitivities): one block per channel, every (weight, centroid) pair
 // evaluated in every iteration; writes args.lut / args.codes / args.sweeps, ignores the other outputs.
 cmpq_status launch_lloyd_weighted(const LloydArgs& args, cmpq_dtype dt, const float* sens, cudaStream_t st);
+// the same fit on the value tables (tables: as for launch_lloyd_ordered); args.skip_row is not used
+cmpq_status launch_lloyd_weighted_tables(const LloydArgs& args, cmpq_dtype dt, const float* sens, void* tables,
+                                         size_t tables_bytes, cudaStream_t st);
 
 // Fills row_ptr[0..d_in] from a row-sorted coordinate list.
 cmpq_status launch_row_ptr(const int32_t* rows, int64_t nnz, int64_t d_in, int64_t* row_ptr,

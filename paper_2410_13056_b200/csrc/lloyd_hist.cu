@@ -1004,6 +1004,252 @@ lloyd_iterate_kernel(const IterArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// sensitivity-weighted fit on the value tables
+//
+// With sensitivities the update is the weighted mean  c_k = sum s x / sum s  over a cluster's members.
+// Members with the same value contribute  value * (sum of their s), so the table of a channel carries the
+// weighted fit as well once every entry knows the sum S of its members' sensitivities: cluster sums are again
+// differences of prefix sums over the ascending entries, and the boundaries are found exactly as in the
+// unweighted iterations.  S is accumulated in 64-bit fixed point (scale: a power of two chosen from the
+// channel's largest sensitivity so that the total stays below 2^52), which makes the sums independent of the
+// order in which the threads add them: the same inputs give the same bytes.  A sensitivity smaller than
+// 2^-(52 - log2 d_out) of the channel's largest loses its low bits; nothing else is rounded before the fp64
+// prefix sums.
+//
+// One block per channel: table and prefix sums in shared memory, the block accumulates S (one search in the
+// table per weight), then a half-warp iterates.  The kernel is launched twice: with a capacity that fits the
+// tables of nearly all channels and lets several blocks share an SM, then, for the channels that exceeded it,
+// with the largest capacity shared memory allows.  Channels beyond that are left to the kernel that scans
+// every weight (flags tell which).
+constexpr int kWtThreads = 128;
+
+__host__ __device__ inline size_t weighted_table_smem(int cap, int64_t d_out) {
+    return (size_t)(cap + 1) * 16 + (size_t)(cap + kKeyPad + 8) * 2 + (size_t)(cap + 8) * 2 + ((size_t)d_out + 31) / 32 * 4 + 16;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kWtThreads, 8)
+lloyd_weighted_table_kernel(const LloydArgs a, const Tables t, const float* __restrict__ sens, int cap, int second_try,
+                            uint8_t* fitted, uint8_t* not_fitted) {
+    extern __shared__ __align__(16) unsigned char wt_smem[];
+    __shared__ unsigned long long warp_s[kWtThreads / 32];
+    __shared__ double warp_sx[kWtThreads / 32];
+    __shared__ uint32_t warp_max[kWtThreads / 32];
+    double* s_ps = reinterpret_cast<double*>(wt_smem);  // [cap + 1] fixed-point sums first, then their prefix
+    double* s_psx = s_ps + cap + 1;                     // [cap + 1] prefix of value * S
+    uint16_t* s_keys = reinterpret_cast<uint16_t*>(s_psx + cap + 1);  // [cap + kKeyPad + 8]
+    uint16_t* s_cum = s_keys + cap + kKeyPad + 8;                     // [cap + 8]
+    uint32_t* bitmap = reinterpret_cast<uint32_t*>(s_cum + cap + 8);  // removed columns of the row
+    unsigned long long* s_fix = reinterpret_cast<unsigned long long*>(s_ps);
+    const int64_t row = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int N = (int)a.d_out, T = a.iters;
+    if (second_try && fitted[row]) return;  // the launch with the small capacity did this channel
+    const ChannelHeader h = t.hdr[row];
+    const int M = h.M < 1 ? 1 : (h.M > N + 1 ? N + 1 : h.M);
+    if (M > cap) {
+        if (tid == 0) { fitted[row] = 0; not_fitted[row] = 1; }
+        return;
+    }
+    const uint16_t* g_keys = t.keys + row * t.stride;
+    const uint16_t* g_cum = t.cum + row * t.stride;
+    for (int i = tid; i <= M; i += kWtThreads) { s_keys[i] = g_keys[i]; s_cum[i] = g_cum[i]; s_fix[i] = 0ull; }
+    for (int i = M + 1 + tid; i < ((M + 8) & ~7) + kKeyPad; i += kWtThreads) s_keys[i] = 0xffffu;
+    int64_t p0 = 0, p1 = 0;
+    if (a.row_ptr) { p0 = a.row_ptr[row]; p1 = a.row_ptr[row + 1]; }
+    if (p1 > p0) for (int i = tid; i < (N + 31) / 32; i += kWtThreads) bitmap[i] = 0u;
+    // largest sensitivity of the channel (s >= 0: the bit patterns order like the values)
+    const float* s_row = sens + row * a.d_out;
+    uint32_t smax = 0u;
+    for (int j = tid; j < N; j += kWtThreads) smax = max(smax, __float_as_uint(s_row[j]));
+    smax = __reduce_max_sync(0xffffffffu, smax);
+    if (lane == 0) warp_max[warp] = smax;
+    __syncthreads();
+    if (p1 > p0)
+        for (int64_t p = p0 + tid; p < p1; p += kWtThreads) {
+            const int col = a.cols[p];
+            atomicOr(&bitmap[col >> 5], 1u << (col & 31));
+        }
+    smax = __reduce_max_sync(0xffffffffu, lane < kWtThreads / 32 ? warp_max[lane] : 0u);
+    double scale = 0.0;  // all sensitivities zero: every sum stays zero and the centroids stay at the start
+    if (smax != 0u) {
+        int ex;
+        frexpf(__uint_as_float(smax), &ex);  // largest sensitivity < 2^ex
+        const int log2n = 32 - __clz(N - 1 > 0 ? N - 1 : 1);
+        scale = ldexp(1.0, 52 - ex - log2n);
+    }
+    __syncthreads();
+    // S of every entry: the entry of a weight is found by bisection (its key is in the table).  The number of
+    // steps depends on the table alone, so four searches run side by side.
+    const uint16_t* w = a.W + row * a.ldw;
+    constexpr int kSide = 4;
+    for (int j0 = tid; j0 < N; j0 += kWtThreads * kSide) {
+        uint32_t key[kSide];
+        int base[kSide];
+#pragma unroll
+        for (int u = 0; u < kSide; ++u) {
+            const int j = j0 + u * kWtThreads;
+            uint32_t hh = j < N ? w[j] : 0u;
+            if (j < N && p1 > p0 && ((bitmap[j >> 5] >> (j & 31)) & 1u)) hh = 0u;
+            if (hh == 0x8000u) hh = 0u;  // -0 and +0 are the same point
+            key[u] = (hh & 0x8000u) ? (~hh & 0xffffu) : (hh | 0x8000u);
+            base[u] = 0;
+        }
+        for (int n = M; n > 1;) {  // first entry whose key is not below the weight's
+            const int half = n >> 1;
+#pragma unroll
+            for (int u = 0; u < kSide; ++u) base[u] = (uint32_t)s_keys[base[u] + half - 1] < key[u] ? base[u] + half : base[u];
+            n -= half;
+        }
+#pragma unroll
+        for (int u = 0; u < kSide; ++u) {
+            const int j = j0 + u * kWtThreads;
+            if (j < N) {
+                const unsigned long long fx = __double2ull_rn((double)s_row[j] * scale);
+                if (fx) atomicAdd(&s_fix[base[u]], fx);
+            }
+        }
+    }
+    __syncthreads();
+    // prefix sums over the entries, every thread a contiguous range, always in the same order
+    {
+        const int chunk = (M + kWtThreads - 1) / kWtThreads;
+        const int e0 = min(tid * chunk, M), e1 = min(e0 + chunk, M);
+        unsigned long long ls = 0ull;
+        double lsx = 0.0;
+        for (int e = e0; e < e1; ++e) {
+            const unsigned long long S = s_fix[e];
+            ls += S;
+            lsx += (double)S * (double)value_of_key16<DT>(s_keys[e]);
+        }
+        unsigned long long is = ls;
+        double isx = lsx;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long us = __shfl_up_sync(0xffffffffu, is, o);
+            const double ux = __shfl_up_sync(0xffffffffu, isx, o);
+            if (lane >= o) { is += us; isx += ux; }
+        }
+        if (lane == 31) { warp_s[warp] = is; warp_sx[warp] = isx; }
+        __syncthreads();
+        unsigned long long run_s = is - ls;
+        double run_sx = 0.0, tot_sx = 0.0;
+        unsigned long long tot_s = 0ull;
+        for (int wv = 0; wv < kWtThreads / 32; ++wv) {  // the warps in order
+            if (wv < warp) { run_s += warp_s[wv]; run_sx += warp_sx[wv]; }
+            tot_s += warp_s[wv];
+            tot_sx += warp_sx[wv];
+        }
+        run_sx += isx - lsx;
+        for (int e = e0; e < e1; ++e) {
+            const unsigned long long S = s_fix[e];
+            s_ps[e] = (double)run_s;  // below 2^52: exact
+            s_psx[e] = run_sx;
+            run_s += S;
+            run_sx += (double)S * (double)value_of_key16<DT>(s_keys[e]);
+        }
+        __syncthreads();  // every range is written before the totals replace the sentinel's slot
+        if (tid == 0) { s_ps[M] = (double)tot_s; s_psx[M] = tot_sx; }
+    }
+    __syncthreads();
+    if (tid >= kGroup) return;
+
+    // iterations: lane k of the half-warp owns centroid k (as in iterate_channel, sums from the prefixes above)
+    const unsigned gmask = 0xffffu;
+    const int gl = tid;
+    const int width = a.bits[row];
+    const int K = width == 2 ? 4 : (width == 3 ? 8 : 16);
+    const uint32_t kfirst = s_keys[0], kend = (uint32_t)s_keys[M - 1] + 1u;
+    const double need = ((double)value_of_key16<DT>(kend - 1u) - (double)value_of_key16<DT>(kfirst)) * (1.0 / 4194304.0);
+    float ck = 0.f;
+    if (gl < K) {
+        const int pos = (int)(((long long)(2 * gl + 1) * N) / (2 * K));
+        int lo = 0, hi = M;  // cum[lo] <= pos < cum[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((int)s_cum[mid] <= pos) lo = mid; else hi = mid;
+        }
+        ck = value_of_key16<DT>(s_keys[lo]);
+    }
+    bool ordered = __all_sync(gmask, gap_ok(gmask, gl, K, ck, need)) != 0;
+    int updates = 0, e_hint = -1;
+    while (updates < T) {
+        float cn = ck;
+        if (ordered) {
+            const float cm = __shfl_up_sync(gmask, ck, 1, kGroup);
+            int e = 0;
+            if (gl > 0 && gl < K) {
+                const uint32_t b = boundary_key<DT>(cm, ck, kfirst, kend);
+                e = b >= kend ? M : rank_of_key(s_keys, M, b, e_hint);
+                e_hint = e;
+            }
+            double P = 0.0, Q = 0.0;
+            if (gl < K) { P = s_ps[e]; Q = s_psx[e]; }
+            double Pn = __shfl_down_sync(gmask, P, 1, kGroup);
+            double Qn = __shfl_down_sync(gmask, Q, 1, kGroup);
+            if (gl == K - 1) { Pn = s_ps[M]; Qn = s_psx[M]; }
+            if (gl < K && Pn - P > 0.0) cn = __double2float_rn(__ddiv_rn(Qn - Q, Pn - P));
+        } else {
+            e_hint = -1;
+            float c[kMaxK];
+#pragma unroll
+            for (int k = 0; k < kMaxK; ++k) c[k] = __shfl_sync(gmask, ck, k, kGroup);
+            double s[kMaxK], n[kMaxK];
+#pragma unroll
+            for (int k = 0; k < kMaxK; ++k) { s[k] = 0.0; n[k] = 0.0; }
+            for (int j = gl; j < M; j += kGroup) {
+                const float v = value_of_key16<DT>(s_keys[j]);
+                const double S = s_ps[j + 1] - s_ps[j];  // integers below 2^52: exact
+                float best = fabsf(v - c[0]);
+                int code = 0;
+#pragma unroll
+                for (int k = 1; k < kMaxK; ++k) {
+                    const float d = fabsf(v - c[k]);
+                    if (k < K && d < best) { best = d; code = k; }
+                }
+#pragma unroll
+                for (int k = 0; k < kMaxK; ++k)
+                    if (code == k) { s[k] += S * (double)v; n[k] += S; }
+            }
+#pragma unroll
+            for (int k = 0; k < kMaxK; ++k) {
+                if (k < K) {
+                    const double sk = group_sum(gmask, s[k]);
+                    const double nk = group_sum(gmask, n[k]);
+                    if (gl == k && nk > 0.0) cn = __double2float_rn(__ddiv_rn(sk, nk));
+                }
+            }
+        }
+        ++updates;
+        const bool ok = gap_ok(gmask, gl, K, cn, need);
+        const bool same_here = gl >= K || __float_as_uint(cn) == __float_as_uint(ck);
+        const bool same = __ballot_sync(gmask, same_here) == gmask;
+        const bool was_ordered = ordered;
+        ordered = __ballot_sync(gmask, ok) == gmask;
+        ck = cn;
+        if (same) {
+            if (!was_ordered) e_hint = -1;
+            break;
+        }
+    }
+    a.lut[row * CMPQ_LUT_STRIDE + gl] = gl < K ? ck : 0.f;
+    {
+        const float cm = __shfl_up_sync(gmask, ck, 1, kGroup);
+        float thr = ordered ? 1.f : 0.f;
+        if (ordered && gl > 0 && gl < K) {
+            const uint32_t b = boundary_key<DT>(cm, ck, kfirst, kend);
+            thr = b < kend ? value_of_key16<DT>(b) : __int_as_float(0x7f800000);
+        }
+        t.thr[row * CMPQ_LUT_STRIDE + gl] = gl < K ? thr : 0.f;
+    }
+    if (gl == 0) {
+        fitted[row] = 1;
+        not_fitted[row] = 0;
+        if (a.sweeps) atomicAdd(a.sweeps, (unsigned long long)(updates + 1) * (unsigned long long)N * (unsigned long long)K);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // last assignment
 
 constexpr int kAssignThreads = 256;
@@ -1788,6 +2034,49 @@ static cmpq_status launch_table_dt(const LloydArgs& args, const Tables& t, cudaS
 
 const void* lloyd_table_kernel_address() {
     return reinterpret_cast<const void*>(&lloyd_table_kernel<CMPQ_BF16, 16, 256, 4, 32>);
+}
+
+// Sensitivity-weighted fit (see lloyd_weighted_table_kernel): value tables, the weighted iterations on them,
+// the all-weights kernel for channels whose tables are too long for shared memory, then the last assignment
+// of the channels fitted on tables.  The two flag arrays live in the tables' list area, unused here.
+cmpq_status launch_lloyd_weighted_tables(const LloydArgs& args, cmpq_dtype dt, const float* sens, void* tables,
+                                         size_t tables_bytes, cudaStream_t st) {
+    const Tables t = tables_at(tables, tables_bytes, args.d_in, args.d_out);
+    const int64_t N = args.d_out;
+    LloydArgs ta = args;
+    ta.inexact_rows = nullptr;  // the exactness diagnostic belongs to the unweighted sums
+    cmpq_status s = dt == CMPQ_F16 ? launch_table_dt<CMPQ_F16>(ta, t, st) : launch_table_dt<CMPQ_BF16>(ta, t, st);
+    if (s != CMPQ_OK) return s;
+    const int fit = (int)((N + 2 + 15) / 16 * 16);  // a table has at most d_out + 1 entries
+    int caps[2] = {N <= 4096 ? 1536 : (N <= 12288 ? 2560 : 3584), fit < 11264 ? fit : 11264};
+    if (caps[0] > fit) caps[0] = fit;
+    uint8_t* fitted = reinterpret_cast<uint8_t*>(t.kept);
+    uint8_t* not_fitted = fitted + args.d_in;
+    const size_t smem_max = weighted_table_smem(caps[1], N);
+    if (cudaFuncSetAttribute(lloyd_weighted_table_kernel<CMPQ_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max) != cudaSuccess ||
+        cudaFuncSetAttribute(lloyd_weighted_table_kernel<CMPQ_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max) != cudaSuccess)
+        return CMPQ_ERR_CUDA;
+    for (int pass = 0; pass < 2; ++pass) {
+        if (pass == 1 && caps[1] <= caps[0]) break;
+        const size_t smem = weighted_table_smem(caps[pass], N);
+        if (dt == CMPQ_F16)
+            lloyd_weighted_table_kernel<CMPQ_F16><<<(unsigned)args.d_in, kWtThreads, smem, st>>>(ta, t, sens, caps[pass], pass, fitted, not_fitted);
+        else
+            lloyd_weighted_table_kernel<CMPQ_BF16><<<(unsigned)args.d_in, kWtThreads, smem, st>>>(ta, t, sens, caps[pass], pass, fitted, not_fitted);
+        s = launch_status();
+        if (s != CMPQ_OK) return s;
+    }
+    LloydArgs oa = args;
+    oa.skip_row = fitted;
+    s = launch_lloyd_weighted(oa, dt, sens, st);
+    if (s != CMPQ_OK) return s;
+    LloydArgs aa = args;
+    aa.skip_row = not_fitted;
+    aa.packed = nullptr;
+    const int assign_threads = N <= 4096 ? kAssignThreads / 2 : kAssignThreads;
+    if (dt == CMPQ_F16) lloyd_assign_kernel<CMPQ_F16, false><<<(unsigned)args.d_in, assign_threads, 0, st>>>(aa, args.lut, t.thr);
+    else lloyd_assign_kernel<CMPQ_BF16, false><<<(unsigned)args.d_in, assign_threads, 0, st>>>(aa, args.lut, t.thr);
+    return launch_status();
 }
 
 // tables_ready: the value tables of every row to be fitted are in place already (skip the table kernel)

@@ -60,8 +60,10 @@ __global__ void __launch_bounds__(kWThreads)
 lloyd_weighted_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t ldw, const uint8_t* __restrict__ bits,
                       const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ cols,
                       const float* __restrict__ sens, int iters, float* __restrict__ lut,
-                      uint8_t* __restrict__ codes, unsigned long long* __restrict__ sweeps) {
+                      uint8_t* __restrict__ codes, unsigned long long* __restrict__ sweeps,
+                      const uint8_t* __restrict__ skip_row) {
     extern __shared__ __align__(16) unsigned char smem[];
+    if (skip_row != nullptr && skip_row[blockIdx.x]) return;  // fitted elsewhere (the whole block leaves)
     float* x = reinterpret_cast<float*>(smem);                       // [d_out]
     uint8_t* code = reinterpret_cast<uint8_t*>(x + d_out);           // [d_out]
     __shared__ int hist_hi[256];
@@ -186,10 +188,10 @@ cmpq_status launch_lloyd_weighted(const LloydArgs& a, cmpq_dtype dt, const float
     }
     if (dt == CMPQ_F16)
         lloyd_weighted_kernel<CMPQ_F16><<<(unsigned)a.d_in, kWThreads, smem, st>>>(
-            a.W, a.d_out, a.ldw, a.bits, a.row_ptr, a.cols, sens, a.iters, a.lut, a.codes, a.sweeps);
+            a.W, a.d_out, a.ldw, a.bits, a.row_ptr, a.cols, sens, a.iters, a.lut, a.codes, a.sweeps, a.skip_row);
     else
         lloyd_weighted_kernel<CMPQ_BF16><<<(unsigned)a.d_in, kWThreads, smem, st>>>(
-            a.W, a.d_out, a.ldw, a.bits, a.row_ptr, a.cols, sens, a.iters, a.lut, a.codes, a.sweeps);
+            a.W, a.d_out, a.ldw, a.bits, a.row_ptr, a.cols, sens, a.iters, a.lut, a.codes, a.sweeps, a.skip_row);
     return launch_status();
 }
 

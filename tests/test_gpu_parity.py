@@ -312,8 +312,10 @@ def test_protect_and_quantize_equals_the_two_calls(dtype, d_in, d_out, n_act, n_
 
 
 # ----------------------------------------------------------------------------- layout conversion
-@pytest.mark.parametrize("shape", [(1, 1), (64, 64), (65, 63), (300, 1030), (66, 2), (4096, 11008), (11008, 4096)])
-@pytest.mark.parametrize("pads", [(4, 6), (3, 5)])   # even leading dimensions: 32-bit accesses; odd: element-wise
+@pytest.mark.parametrize("shape", [(1, 1), (64, 64), (65, 63), (300, 1030), (66, 2), (8, 200), (72, 136), (4096, 11008),
+                                   (11008, 4096)])
+# leading dimensions that are multiples of 8 (with extents that are): 128-bit accesses; even: 32-bit; odd: element-wise
+@pytest.mark.parametrize("pads", [(8, 16), (4, 6), (3, 5)])
 @pytest.mark.parametrize("tdt", [torch.float16, torch.bfloat16])
 def test_transpose16_is_the_transpose(shape, pads, tdt):
     """Plain definition: dst[c][r] = src[r][c], raw 16-bit patterns (checked against numpy on the host)."""

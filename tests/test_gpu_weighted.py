@@ -90,3 +90,35 @@ def test_zero_sensitivity_cluster_keeps_its_centroid():
     lut, codes, _, _ = G.gpu_quantize(W, bits, none, none, 6, sens=sens)
     start, start_codes, _, _ = G.gpu_quantize(W, bits, none, none, 0)
     assert np.array_equal(lut.view(np.uint32), start.view(np.uint32)) and np.array_equal(codes, start_codes)
+
+
+@pytest.mark.parametrize("dtype,shape", [(inputs.BF16, (64, 4096)), (inputs.F16, (12, 4096)), (inputs.F16, (3, 24576))])
+def test_table_formulation_agrees_with_the_all_weights_kernel(dtype, shape):
+    """The default weighted fit works on the value tables (sums of sensitivities per distinct value); the kernel
+    that scans every weight stays selectable through the all-pairs switch.  Same method, different orders of
+    summation: centroids agree to rounding, codes wherever the centroids are bit-equal.  bf16 channels of 4096
+    weights fit the small table capacity, fp16 ones need the large one, and a 24576-wide fp16 channel has more
+    distinct values than shared memory holds and is handed to the all-weights kernel."""
+    from paper_2410_13056_b200 import binding as B
+    d_in, d_out = shape
+    W = inputs.make_weight(d_in, d_out, dtype, 31 + d_out, device="cuda")
+    bits = _bits(d_in, 5)
+    rows, cols = _outliers(d_in, d_out, 40, 11)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(17)
+    sens = (torch.rand((d_in, d_out), device="cuda", generator=g) * 3 + 0.05).float()
+    lut_t, codes_t, _, _ = G.gpu_quantize(W, bits, rows, cols, 12, sens=sens)
+    B.cmpq_set_lloyd_assignment(B.ASSIGN_ALL_PAIRS)
+    try:
+        lut_a, codes_a, _, _ = G.gpu_quantize(W, bits, rows, cols, 12, sens=sens)
+    finally:
+        B.cmpq_set_lloyd_assignment(B.ASSIGN_ORDERED)
+    scale = np.abs(lut_a).max(axis=1, keepdims=True)
+    assert np.all(np.abs(lut_t - lut_a) <= 1e-5 * scale)
+    equal = [i for i in range(d_in) if np.array_equal(lut_t[i].view(np.uint32), lut_a[i].view(np.uint32))]
+    assert len(equal) >= 0.8 * d_in
+    for i in equal:
+        assert np.array_equal(codes_t[i], codes_a[i]), i
+    # and the run is reproducible byte for byte
+    lut_2, codes_2, _, _ = G.gpu_quantize(W, bits, rows, cols, 12, sens=sens)
+    assert np.array_equal(lut_2.view(np.uint32), lut_t.view(np.uint32)) and np.array_equal(codes_2, codes_t)
