@@ -401,7 +401,8 @@ def main():
 
     # The metric's own workload: every layer of the 32-block 7B-shaped stack at avg 3.0 bits through the stack
     # driver (own seeded weights per layer, 131072 calibration tokens per layer; with N ranks the layers are
-    # dealt round-robin, no collective on the data path).  One untimed pass per shape first; CUDA events
+    # dealt round-robin, no collective on the data path).  One untimed pass per shape first (it captures the
+    # shape's graph); CUDA events
     # around every pass; the job's time is the slowest rank's sum.
     stack_leg = None
     n_act_q = (q.n_act, q.n_q)
@@ -412,15 +413,18 @@ def main():
         torch.cuda.empty_cache()
         scfg = inputs.CONFIGS["c4_stack7b"]
         src = inputs.StackInputs(scfg)
-        stack = StackQuantizer(src.shapes(), rank, world)
+        # as the headline pass: packed words only, every shape's pass captured once in a CUDA graph (the stack
+        # inputs keep one buffer per shape, so the addresses stay fixed) and replayed for each layer
+        stack = StackQuantizer(src.shapes(), rank, world,
+                               quantizer_factory=lambda d_in, d_out: LayerQuantizer(d_in, d_out, keep_codes=False))
         seen = set()
         for k in stack.mine:
             if stack.shapes[k] not in seen:
                 seen.add(stack.shapes[k])
                 Xs, Ws = src(k)
-                stack.quantizer(k).run(Xs, Ws, METRIC_BUDGET, scfg.lloyd_iters)
+                stack.quantizer(k).run_graphed(Xs, Ws, METRIC_BUDGET, scfg.lloyd_iters)
         barrier()
-        out = stack.run(src, METRIC_BUDGET, scfg.lloyd_iters, timed=True)
+        out = stack.run(src, METRIC_BUDGET, scfg.lloyd_iters, timed=True, graphed=True)
         barrier()
         stack_ms = max_over_ranks(out["ms"])
         total_params = sum(a * b for a, b in src.shapes())
@@ -428,7 +432,8 @@ def main():
                                  "131072 tokens per layer, avg 3.0 bits, 20 Lloyd iterations",
                      "layers": len(src.shapes()), "params": total_params, "ms_total": stack_ms,
                      "value": total_params / (stack_ms * 1e-3) / 1e6, "unit": UNIT,
-                     "scaling": "strong (the 224 layers are split over the ranks)", "launch": "eager calls",
+                     "scaling": "strong (the 224 layers are split over the ranks)",
+                     "launch": "one CUDA graph per layer shape, replayed for every layer of that shape",
                      "ms_per_pass_by_shape": {"%dx%d" % shape: v for shape, v in out["ms_by_shape"].items()}}
 
     cpu_baseline = None
