@@ -626,9 +626,17 @@ __device__ __forceinline__ int rank_of_key(const uint16_t* keys, int M, uint32_t
         int j0 = (hint & ~7) - 8;
         if (j0 < 0) j0 = 0;
         const Eight a8 = load_eight(keys + j0), b8 = load_eight(keys + j0 + 8);
-        int below = 0;
-#pragma unroll
-        for (int u = 0; u < 8; ++u) below += (a8.at(u) < b ? 1 : 0) + (b8.at(u) < b ? 1 : 0);
+        // the sixteen keys ascend: bisection on registers (a word holds two keys, the lower one in its low half)
+        const bool hi8 = b8.at(0) < b;  // at least eight keys below b?
+        const uint32_t w0 = hi8 ? b8.w[0] : a8.w[0], w1 = hi8 ? b8.w[1] : a8.w[1];
+        const uint32_t w2 = hi8 ? b8.w[2] : a8.w[2], w3 = hi8 ? b8.w[3] : a8.w[3];
+        const bool hi4 = (w2 & 0xffffu) < b;  // key 4 of those eight
+        const uint32_t v0 = hi4 ? w2 : w0, v1 = hi4 ? w3 : w1;
+        const bool hi2 = (v1 & 0xffffu) < b;  // key 2 of those four
+        const uint32_t u0 = hi2 ? v1 : v0;
+        const bool hi1 = (u0 >> 16) < b;      // key 1 of those two
+        const uint32_t last = hi1 ? (u0 >> 16) : (u0 & 0xffffu);
+        const int below = (hi8 ? 8 : 0) + (hi4 ? 4 : 0) + (hi2 ? 2 : 0) + (hi1 ? 1 : 0) + (last < b ? 1 : 0);
         if (below == 0 && j0 > 0) hi = j0;                    // the boundary moved below the window
         else if (below == 16 && j0 + 16 < M) lo = j0 + 16;    // ... or above it
         else return j0 + below;                               // (entries past the table are 0xffff: never below)
@@ -691,28 +699,42 @@ __device__ __forceinline__ int group_sum(unsigned gmask, int v) {
 __device__ __forceinline__ void copy_table_removing(uint16_t* w_keys, uint16_t* w_cum, const uint16_t* g_keys,
                                                     const uint16_t* g_cum, int M, const uint32_t* rk, int nr) {
     const int gl = threadIdx.x & 15;
-    for (int i = gl; i < (M + 1 + 7) / 8; i += kGroup) {  // with the sentinel (key 0xffff, cum[M] = d_out)
+    const int steps = (M + 1 + 7) / 8;  // with the sentinel (key 0xffff, cum[M] = d_out)
+    constexpr int kAhead = 4;           // groups of eight a lane requests before it stores any (the loads are L2 latency)
+    for (int i0 = gl; i0 < steps; i0 += kGroup * kAhead) {
         // plain loads: after the first pass over a row the source is the copy itself, which may be shared memory
-        const uint4 kv = reinterpret_cast<const uint4*>(g_keys)[i];
-        uint4 cv = reinterpret_cast<const uint4*>(g_cum)[i];
-        if (nr > 0) {
-            const uint32_t kw[4] = {kv.x, kv.y, kv.z, kv.w};
-            uint32_t cw[4] = {cv.x, cv.y, cv.z, cv.w};
+        uint4 kv[kAhead], cv[kAhead];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t k0 = kw[q] & 0xffffu, k1 = kw[q] >> 16;
-                int d0 = k0 > kZeroKeyOfTable ? nr : 0, d1 = k1 > kZeroKeyOfTable ? nr : 0;
-                for (int r = 0; r < nr; ++r) {
-                    const uint32_t k = rk[r];
-                    d0 -= k < k0 ? 1 : 0;
-                    d1 -= k < k1 ? 1 : 0;
-                }
-                cw[q] = ((cw[q] + (uint32_t)d0) & 0xffffu) | ((((cw[q] >> 16) + (uint32_t)d1) & 0xffffu) << 16);
+        for (int q = 0; q < kAhead; ++q) {
+            const int i = i0 + q * kGroup;
+            if (i < steps) {
+                kv[q] = reinterpret_cast<const uint4*>(g_keys)[i];
+                cv[q] = reinterpret_cast<const uint4*>(g_cum)[i];
             }
-            cv = make_uint4(cw[0], cw[1], cw[2], cw[3]);
         }
-        reinterpret_cast<uint4*>(w_keys)[i] = kv;
-        reinterpret_cast<uint4*>(w_cum)[i] = cv;
+#pragma unroll
+        for (int q = 0; q < kAhead; ++q) {
+            const int i = i0 + q * kGroup;
+            if (i >= steps) continue;
+            if (nr > 0) {
+                const uint32_t kw[4] = {kv[q].x, kv[q].y, kv[q].z, kv[q].w};
+                uint32_t cw[4] = {cv[q].x, cv[q].y, cv[q].z, cv[q].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const uint32_t k0 = kw[h] & 0xffffu, k1 = kw[h] >> 16;
+                    int d0 = k0 > kZeroKeyOfTable ? nr : 0, d1 = k1 > kZeroKeyOfTable ? nr : 0;
+                    for (int r = 0; r < nr; ++r) {
+                        const uint32_t k = rk[r];
+                        d0 -= k < k0 ? 1 : 0;
+                        d1 -= k < k1 ? 1 : 0;
+                    }
+                    cw[h] = ((cw[h] + (uint32_t)d0) & 0xffffu) | ((((cw[h] >> 16) + (uint32_t)d1) & 0xffffu) << 16);
+                }
+                cv[q] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            }
+            reinterpret_cast<uint4*>(w_keys)[i] = kv[q];
+            reinterpret_cast<uint4*>(w_cum)[i] = cv[q];
+        }
     }
 }
 
@@ -759,6 +781,7 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, const int K, uns
     const bool patch = a.src.hdr != nullptr;
     const Tables& from = patch ? a.src : a.t;
     int64_t p0 = 0, nrem = 0;
+    const ChannelHeader h = from.hdr[row];  // requested together with the row's list limits
     if (patch) { p0 = a.row_ptr[row]; nrem = a.row_ptr[row + 1] - p0; }
     int M = 1;
     const uint16_t* keys = s_keys;
@@ -768,7 +791,6 @@ __device__ void iterate_channel(const IterArgs& a, int64_t row, const int K, uns
     if (patch && nrem >= N) {  // every position removed: an all-zero channel
         if (gl == 0) { s_keys[0] = (uint16_t)kZeroKeyOfTable; s_cum[0] = 0; s_cum[1] = (uint16_t)N; }
     } else {
-        const ChannelHeader h = from.hdr[row];
         M = h.M < 1 ? 1 : (h.M > N + 1 ? N + 1 : h.M);  // 1 <= M <= N + 1 by construction (the entry of +0 may be empty)
         const uint16_t* g_keys = from.keys + row * from.stride;  // rows are 16-byte aligned, padded to 8 entries
         const uint16_t* g_cum = from.cum + row * from.stride;
@@ -972,16 +994,20 @@ lloyd_iterate_kernel(const IterArgs a) {
     unsigned char* smem = iter_smem + (size_t)group * iter_channel_bytes(a.cap);
     const int64_t row = (int64_t)blockIdx.x * (kIterWarps * 2) + group;
     if (row >= a.d_in) return;
-    if (a.skip_row && a.skip_row[row]) return;
+    // the per-row words are all requested before any of them is looked at (each is a round trip to L2)
+    const int skip = a.skip_row ? (int)a.skip_row[row] : 0;
+    const int bad = a.nonfinite ? *a.nonfinite : 0;
+    const int bits = a.bits[row];
+    const int cache_iters = a.fc.hdr ? a.fc.hdr->iters : -1;
+    if (skip) return;
     // Non-finite inputs were found by an earlier kernel of the call: its outputs are unspecified anyway, and
     // although every loop below is bounded whatever the values (bisections halve an interval, the update
     // loop counts to the iteration limit), there is nothing worth computing.
-    if (a.nonfinite && *a.nonfinite) return;
+    if (bad) return;
     const unsigned gmask = group_mask();
-    const int bits = a.bits[row];
     const int gl = threadIdx.x & 15;
     // a fit of this channel at this width kept from an earlier call on the same weights: copy it
-    const bool cached_ok = a.fc.hdr && a.fc.hdr->iters == a.iters;
+    const bool cached_ok = a.fc.hdr && cache_iters == a.iters;
     const int64_t slot = (int64_t)(bits == 2 ? 0 : (bits == 3 ? 1 : 2)) * a.d_in + row;
     if (cached_ok && a.fc.valid[slot]) {
         a.lut[row * CMPQ_LUT_STRIDE + gl] = a.fc.lut[slot * CMPQ_LUT_STRIDE + gl];
