@@ -719,16 +719,33 @@ __device__ __forceinline__ void copy_table_removing(uint16_t* w_keys, uint16_t* 
             if (nr > 0) {
                 const uint32_t kw[4] = {kv[q].x, kv[q].y, kv[q].z, kv[q].w};
                 uint32_t cw[4] = {cv[q].x, cv[q].y, cv[q].z, cv[q].w};
+                // Both parts of the shift are monotone in the key, so if the first and the last of the eight
+                // ascending keys get the same parts, all eight get the same shift (nearly every group does).
+                const uint32_t k_lo = kw[0] & 0xffffu, k_hi = kw[3] >> 16;
+                int below_lo = 0, below_hi = 0;
+                for (int r = 0; r < nr; ++r) {
+                    const uint32_t k = rk[r];
+                    below_lo += k < k_lo ? 1 : 0;
+                    below_hi += k < k_hi ? 1 : 0;
+                }
+                // (a group that reaches past the sentinel holds unordered left-overs: entry by entry)
+                if (8 * i + 7 <= M && below_lo == below_hi && (k_lo > kZeroKeyOfTable) == (k_hi > kZeroKeyOfTable)) {
+                    const uint32_t d = (uint32_t)((k_lo > kZeroKeyOfTable ? nr : 0) - below_lo);
 #pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    const uint32_t k0 = kw[h] & 0xffffu, k1 = kw[h] >> 16;
-                    int d0 = k0 > kZeroKeyOfTable ? nr : 0, d1 = k1 > kZeroKeyOfTable ? nr : 0;
-                    for (int r = 0; r < nr; ++r) {
-                        const uint32_t k = rk[r];
-                        d0 -= k < k0 ? 1 : 0;
-                        d1 -= k < k1 ? 1 : 0;
+                    for (int h = 0; h < 4; ++h)
+                        cw[h] = ((cw[h] + d) & 0xffffu) | ((((cw[h] >> 16) + d) & 0xffffu) << 16);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const uint32_t k0 = kw[h] & 0xffffu, k1 = kw[h] >> 16;
+                        int d0 = k0 > kZeroKeyOfTable ? nr : 0, d1 = k1 > kZeroKeyOfTable ? nr : 0;
+                        for (int r = 0; r < nr; ++r) {
+                            const uint32_t k = rk[r];
+                            d0 -= k < k0 ? 1 : 0;
+                            d1 -= k < k1 ? 1 : 0;
+                        }
+                        cw[h] = ((cw[h] + (uint32_t)d0) & 0xffffu) | ((((cw[h] >> 16) + (uint32_t)d1) & 0xffffu) << 16);
                     }
-                    cw[h] = ((cw[h] + (uint32_t)d0) & 0xffffu) | ((((cw[h] >> 16) + (uint32_t)d1) & 0xffffu) << 16);
                 }
                 cv[q] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
             }
