@@ -1858,17 +1858,17 @@ __device__ void table_emit_row(const uint16_t* __restrict__ w, int64_t d_out, co
 
 // Kept entries of a row whose entry-keeping values were listed by the count step: a weight is a candidate
 // exactly when its key is in the list, so no error is evaluated here.  Ordering as in table_emit_row.
-__device__ void table_emit_row_by_keys(const uint16_t* __restrict__ w, int64_t d_out, const uint32_t* __restrict__ kept,
+__device__ void table_emit_row_by_keys(const uint16_t* __restrict__ w, int64_t d_out, const uint32_t my_kept /* list slot threadIdx.x */,
                                        int nkept, int64_t row, int te, int64_t out0, int32_t* __restrict__ rows,
                                        int32_t* __restrict__ cols, uint16_t* __restrict__ vals, int* list_col,
-                                       unsigned char* list_eq, int* list_n, uint32_t* s_kept, const uint4 first) {
+                                       unsigned char* list_eq, int* list_n, uint32_t* s_kept, const uint4 first, const uint4 second) {
     if (threadIdx.x == 0) *list_n = 0;
     // Almost no weight is a candidate, and candidates lie far from their centroids: a weight whose magnitude
     // is below the smallest magnitude among the listed values cannot be one.
     if (threadIdx.x < 32) {  // at most kKeptCap = 31 listed values: the last slot carries that magnitude
         uint32_t mag = 0x7fffu;
         if ((int)threadIdx.x < nkept) {
-            const uint32_t kk = kept[1 + threadIdx.x];
+            const uint32_t kk = my_kept;
             s_kept[threadIdx.x] = kk;
             mag = (kk & 0xffffu) >= 0x8000u ? kk & 0x7fffu : 0x7fffu - (kk & 0xffffu);
         }
@@ -1881,8 +1881,9 @@ __device__ void table_emit_row_by_keys(const uint16_t* __restrict__ w, int64_t d
     for (int64_t j0 = (int64_t)threadIdx.x * 8; j0 < d_out; j0 += (int64_t)blockDim.x * 8) {
         uint32_t pk[4] = {0u, 0u, 0u, 0u};
         if (j0 + 7 < d_out && vec) {
-            // the first eight weights of a thread were requested when the kernel started
-            const uint4 v = j0 == (int64_t)threadIdx.x * 8 ? first : __ldg(reinterpret_cast<const uint4*>(w + j0));
+            // the first two groups of eight of a thread were requested when the kernel started
+            const uint4 v = j0 == (int64_t)threadIdx.x * 8 ? first
+                          : (j0 == (int64_t)(blockDim.x + threadIdx.x) * 8 ? second : __ldg(reinterpret_cast<const uint4*>(w + j0)));
             pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
         } else {
 #pragma unroll
@@ -1953,12 +1954,21 @@ table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, c
     const int64_t row = blockIdx.x;
     const uint16_t* w = W + row * ldw;
     // nearly every row keeps something: its weights are requested before anything else is looked at
-    uint4 first = make_uint4(0u, 0u, 0u, 0u);
-    if ((reinterpret_cast<uintptr_t>(w) & 15) == 0 && (int64_t)threadIdx.x * 8 + 7 < d_out)
-        first = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)threadIdx.x * 8));
-    const int64_t out0 = row_start[row];
-    if (row_start[row + 1] == out0) return;
-    if (is_act[row]) {
+    uint4 first = make_uint4(0u, 0u, 0u, 0u), second = make_uint4(0u, 0u, 0u, 0u);
+    if ((reinterpret_cast<uintptr_t>(w) & 15) == 0) {
+        if ((int64_t)threadIdx.x * 8 + 7 < d_out) first = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)threadIdx.x * 8));
+        if ((int64_t)(blockDim.x + threadIdx.x) * 8 + 7 < d_out)
+            second = __ldg(reinterpret_cast<const uint4*>(w + (int64_t)(blockDim.x + threadIdx.x) * 8));
+    }
+    // ... and so are the row's few words (each a round trip to L2 when asked for one after the other)
+    const int64_t out0 = row_start[row], out1 = row_start[row + 1];
+    const int act = is_act[row];
+    const int te = take_eq[row];
+    const int ncand = gt[row] + eq[row];
+    const uint32_t nkept = t.kept[row * 32];
+    const uint32_t my_kept = threadIdx.x < (unsigned)kKeptCap ? t.kept[row * 32 + 1 + threadIdx.x] : 0u;  // slot of the list, if used
+    if (out1 == out0) return;
+    if (act) {
         for (int64_t j = threadIdx.x; j < d_out; j += blockDim.x) {
             rows[out0 + j] = (int32_t)row;
             cols[out0 + j] = (int32_t)j;
@@ -1966,16 +1976,13 @@ table_emit_kernel(const uint16_t* __restrict__ W, int64_t ldw, const Tables t, c
         }
         return;
     }
-    const uint32_t tau = st->tau;
-    const int te = take_eq[row];
-    const int ncand = gt[row] + eq[row];
-    const int b = bits[row];
-    const uint32_t nkept = t.kept[row * 32];
     if (nkept != kKeptUnknown && ncand <= kEmitListCap) {
-        table_emit_row_by_keys(w, d_out, t.kept + row * 32, (int)nkept, row, te, out0, rows, cols, vals, list_col, list_eq,
-                               &list_n, s_kept, first);
+        table_emit_row_by_keys(w, d_out, my_kept, (int)nkept, row, te, out0, rows, cols, vals, list_col, list_eq,
+                               &list_n, s_kept, first, second);
         return;
     }
+    const uint32_t tau = st->tau;
+    const int b = bits[row];
     if (b == 2) table_emit_row<DT, 4>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
     else if (b == 3) table_emit_row<DT, 8>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
     else table_emit_row<DT, 16>(w, d_out, t, row, tau, te, ncand, out0, rows, cols, vals, warp_totals, list_col, list_eq, &list_n);
