@@ -37,6 +37,19 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Number of SMs of the current device (queried once per device and cached).
 int sm_count();
 
+// Raises a kernel's dynamic shared-memory limit to `bytes` once per device (the limit is an upper bound, so
+// callers pass the largest amount any launch of the kernel can ask for); later calls on the same device return
+// at once.  `done` is the caller's flag array for this kernel, one entry per device.
+template <class Kernel>
+inline bool raise_smem_limit_once(Kernel kern, size_t bytes, bool (&done)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64 && done[dev]) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64) done[dev] = true;
+    return true;
+}
+
 // Converts the last CUDA launch error into a status.
 inline cmpq_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? CMPQ_OK : CMPQ_ERR_CUDA;

@@ -2044,8 +2044,10 @@ static cmpq_status launch_table(const LloydArgs& args, const Tables& t, int thre
     const size_t smem = sizeof(TableShared) + (size_t)SLOTS * kSlotWords * sizeof(uint32_t) +
                         (((size_t)args.d_out + 31) / 32) * sizeof(uint32_t) + (size_t)kStageCap * sizeof(uint32_t);
     auto kern = lloyd_table_kernel<DT, E, MAXT, MINB, SLOTS>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return CMPQ_ERR_CUDA;
+    static bool raised[64] = {};  // per instance of this template, hence per kernel
+    const size_t smem_limit = sizeof(TableShared) + (size_t)SLOTS * kSlotWords * sizeof(uint32_t) +
+                              (((size_t)CMPQ_MAX_D_OUT + 31) / 32) * sizeof(uint32_t) + (size_t)kStageCap * sizeof(uint32_t);
+    if (!raise_smem_limit_once(kern, smem_limit, raised)) return CMPQ_ERR_CUDA;
     kern<<<(unsigned)args.d_in, threads, smem, st>>>(args, t);
     return launch_status();
 }
@@ -2103,8 +2105,11 @@ cmpq_status launch_lloyd_weighted_tables(const LloydArgs& args, cmpq_dtype dt, c
     uint8_t* fitted = reinterpret_cast<uint8_t*>(t.kept);
     uint8_t* not_fitted = fitted + args.d_in;
     const size_t smem_max = weighted_table_smem(caps[1], N);
-    if (cudaFuncSetAttribute(lloyd_weighted_table_kernel<CMPQ_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max) != cudaSuccess ||
-        cudaFuncSetAttribute(lloyd_weighted_table_kernel<CMPQ_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max) != cudaSuccess)
+    static bool raised_f16[64] = {}, raised_bf16[64] = {};
+    const size_t smem_limit = weighted_table_smem(11264, CMPQ_MAX_D_OUT);
+    if (smem_max > smem_limit) return CMPQ_ERR_INTERNAL;
+    if (!raise_smem_limit_once(lloyd_weighted_table_kernel<CMPQ_F16>, smem_limit, raised_f16) ||
+        !raise_smem_limit_once(lloyd_weighted_table_kernel<CMPQ_BF16>, smem_limit, raised_bf16))
         return CMPQ_ERR_CUDA;
     for (int pass = 0; pass < 2; ++pass) {
         if (pass == 1 && caps[1] <= caps[0]) break;
@@ -2168,8 +2173,8 @@ static cmpq_status launch_ordered_dt(const LloydArgs& args, const Tables& t, boo
     // 28672 for Gaussian-like bf16 weights); longer tables are read from global memory
     ia.cap = N <= 4096 ? kMinIterCap : (N <= 12288 ? 2048 : 3072);
     const size_t iter_smem = (size_t)kIterWarps * 2 * iter_channel_bytes(ia.cap);
-    if (cudaFuncSetAttribute(lloyd_iterate_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)iter_smem) !=
-        cudaSuccess)
+    static bool raised[64] = {};  // per instance of this template, hence per kernel
+    if (!raise_smem_limit_once(lloyd_iterate_kernel<DT>, (size_t)kIterWarps * 2 * iter_channel_bytes(3072), raised))
         return CMPQ_ERR_CUDA;
     const unsigned iter_blocks = (unsigned)((args.d_in + kIterWarps * 2 - 1) / (kIterWarps * 2));
     lloyd_iterate_kernel<DT><<<iter_blocks, kIterWarps * 32, iter_smem, st>>>(ia);
