@@ -245,7 +245,10 @@ cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in
  * cache: cmpq_sweep_cache_bytes(d_in, d_out) bytes of device memory, 256-byte aligned, untouched by the
  * caller between the calls (else CMPQ_ERR_WORKSPACE).  Calls on one cache must be ordered (one stream).
  * With CMPQ_ASSIGN_ALL_PAIRS selected the cache is ignored.
- * ws of cmpq_sweep_budget: cmpq_workspace_bytes(CMPQ_OP_PROTECT_AND_QUANTIZE, d_in, d_out). */
+ *   cmpq_sweep_budget_pack  is cmpq_protect_quantize_pack with the same use of the cache (the last assignment
+ *                      writes the packed words; codes may be NULL).
+ * ws of cmpq_sweep_budget: cmpq_workspace_bytes(CMPQ_OP_PROTECT_AND_QUANTIZE, d_in, d_out); of
+ * cmpq_sweep_budget_pack: cmpq_workspace_bytes(CMPQ_OP_PROTECT_QUANTIZE_PACK, d_in, d_out). */
 size_t cmpq_sweep_cache_bytes(int64_t d_in, int64_t d_out);
 cmpq_status cmpq_sweep_begin(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
                              int lloyd_iters, int32_t* nonfinite, void* cache, size_t cache_bytes, void* stream);
@@ -255,6 +258,13 @@ cmpq_status cmpq_sweep_budget(const void* W, cmpq_dtype dt, int64_t d_in, int64_
                               int64_t nnz_out, float* lut, uint8_t* codes, int32_t* inexact_rows,
                               unsigned long long* sweeps, void* cache, size_t cache_bytes, void* ws,
                               size_t ws_bytes, void* stream);
+cmpq_status cmpq_sweep_budget_pack(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                   const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                   int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
+                                   int64_t nnz_out, float* lut, uint8_t* codes, uint32_t* packed,
+                                   int64_t* row_off, int32_t* perm, int64_t* seg_rows, int32_t* inexact_rows,
+                                   unsigned long long* sweeps, void* cache, size_t cache_bytes, void* ws,
+                                   size_t ws_bytes, void* stream);
 
 /* Process-wide choice of the assignment method used by cmpq_extract_outliers and
  * cmpq_quantize_layer from the next call on (host state, no GPU work; thread-safe).

@@ -27,7 +27,7 @@ EXPORTS = (
     "cmpq_protect_and_quantize", "cmpq_matvec", "cmpq_outliers_by_column",
     "cmpq_collect_stats_norm", "cmpq_finalize_stats_norm", "cmpq_transpose16",
     "cmpq_alu_probe", "cmpq_kernel_resources",
-    "cmpq_sweep_cache_bytes", "cmpq_sweep_begin", "cmpq_sweep_budget",
+    "cmpq_sweep_cache_bytes", "cmpq_sweep_begin", "cmpq_sweep_budget", "cmpq_sweep_budget_pack",
     "cmpq_quantize_layer_packed", "cmpq_protect_quantize_pack", "cmpq_check_finite",
     "cmpq_matvec_f16lut", "cmpq_lut_bytes", "cmpq_store_lut", "cmpq_load_lut", "cmpq_table_bits_per_weight",
 )
@@ -101,6 +101,9 @@ def lib():
         L.cmpq_sweep_budget.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
                                         vp, vp, vp, vp, sz, vp, sz, vp]
         L.cmpq_sweep_budget.restype = ci
+        L.cmpq_sweep_budget_pack.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, i64, ci, vp, vp, vp, i64, vp,
+                                             vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp]
+        L.cmpq_sweep_budget_pack.restype = ci
         L.cmpq_quantize_layer_packed.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, i64, ci, vp, vp, vp, vp, vp, vp,
                                                  vp, vp, vp, vp, vp, sz, vp]
         L.cmpq_quantize_layer_packed.restype = ci
@@ -319,6 +322,18 @@ def cmpq_sweep_budget(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut
                                    n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz, _ptr(lut),
                                    _ptr(codes), _ptr(inexact_rows), _ptr(sweeps), _ptr(cache), cache.numel(),
                                    _ptr(ws), ws.numel(), _stream()), "cmpq_sweep_budget")
+
+
+def cmpq_sweep_budget_pack(W, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, lut, codes, packed, row_off, perm,
+                           seg_rows, cache, ws, inexact_rows=None, sweeps=None):
+    """cmpq_protect_quantize_pack with the value tables and provisional fits kept in `cache`; codes may be None."""
+    d_in, d_out = W.shape
+    nnz = n_act * d_out + n_q
+    _check(lib().cmpq_sweep_budget_pack(_ptr(W), dtype_code(W), d_in, d_out, W.stride(0), _ptr(a), _ptr(bits),
+                                        n_act, n_q, lloyd_iters, _ptr(rows), _ptr(cols), _ptr(vals), nnz, _ptr(lut),
+                                        _ptr(codes), _ptr(packed), _ptr(row_off), _ptr(perm), _ptr(seg_rows),
+                                        _ptr(inexact_rows), _ptr(sweeps), _ptr(cache), cache.numel(), _ptr(ws),
+                                        ws.numel(), _stream()), "cmpq_sweep_budget_pack")
 
 
 def cmpq_pack(codes, bits, packed, row_off, perm, seg_rows, ws):

@@ -564,3 +564,20 @@ extern "C" cmpq_status cmpq_sweep_budget(const void* W, cmpq_dtype dt, int64_t d
                                  lut, codes, inexact_rows, sweeps, nullptr, ws, ws_bytes, cache,
                                  static_cast<cudaStream_t>(stream));
 }
+
+extern "C" cmpq_status cmpq_sweep_budget_pack(const void* W, cmpq_dtype dt, int64_t d_in, int64_t d_out, int64_t ldw,
+                                              const float* a, const uint8_t* bits, int64_t n_act, int64_t n_q,
+                                              int lloyd_iters, int32_t* rows, int32_t* cols, uint16_t* vals,
+                                              int64_t nnz_out, float* lut, uint8_t* codes, uint32_t* packed,
+                                              int64_t* row_off, int32_t* perm, int64_t* seg_rows,
+                                              int32_t* inexact_rows, unsigned long long* sweeps, void* cache,
+                                              size_t cache_bytes, void* ws, size_t ws_bytes, void* stream) {
+    if (!cache || !aligned_to(cache, 256)) return CMPQ_ERR_WORKSPACE;
+    if (d_in >= 1 && d_in <= CMPQ_MAX_D_IN && d_out >= 1 && d_out <= CMPQ_MAX_D_OUT &&
+        cache_bytes < sweep_cache_bytes(d_in, d_out))
+        return CMPQ_ERR_WORKSPACE;
+    const PackOut po{packed, row_off, perm, seg_rows};
+    return protect_quantize_impl(W, dt, d_in, d_out, ldw, a, bits, n_act, n_q, lloyd_iters, rows, cols, vals, nnz_out,
+                                 lut, codes, inexact_rows, sweeps, nullptr, ws, ws_bytes, cache,
+                                 static_cast<cudaStream_t>(stream), &po);
+}

@@ -163,7 +163,11 @@ class LayerQuantizer:
             call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
         call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
              self.ws)
-        if sweep_cache is not None:
+        if sweep_cache is not None and fused:
+            call("cmpq_sweep_budget_pack", B.cmpq_sweep_budget_pack, W, self.a, self.bits, self.n_act, self.n_q,
+                 lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.packed, self.row_off,
+                 self.perm, self.seg_rows, sweep_cache, self.ws, inexact_rows=inexact, sweeps=sweeps)
+        elif sweep_cache is not None:
             call("cmpq_sweep_budget", B.cmpq_sweep_budget, W, self.a, self.bits, self.n_act, self.n_q, lloyd_iters,
                  self.rows, self.cols, self.vals, self.lut, self.codes, sweep_cache, self.ws,
                  inexact_rows=inexact, sweeps=sweeps)
