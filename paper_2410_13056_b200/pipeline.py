@@ -22,11 +22,15 @@ from . import binding as B
 # packing takes 2 more = 20.  All-pairs assignment: the provisional fit is one kernel and every select pass is
 # followed by a digit kernel (outlier step 11), the final fit is row index + one kernel, packing 2 = 19; fused
 # the packing still runs as its own step after the fit (layout with the O_act cut, pack 1) = 18.
-def kernels_per_run(assignment=None, fused=False):
+# With overlap_tables the value tables come from cmpq_sweep_begin on a second stream (table kernel and the
+# kernel that empties the cache of fits) and the rest from cmpq_sweep_budget_pack: one kernel more, 17.
+def kernels_per_run(assignment=None, fused=False, overlap_tables=False):
     if assignment is None:
         assignment = B.cmpq_get_lloyd_assignment()
     if assignment == B.ASSIGN_ALL_PAIRS:
         return 18 if fused else 19
+    if fused and overlap_tables:
+        return 17
     return 16 if fused else 20
 
 
@@ -127,14 +131,19 @@ class LayerQuantizer:
                 on_result(b, result)
         return result
 
-    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None, reuse_statistic=False, sweep_cache=None):
+    def run(self, X, W, avg_bits, lloyd_iters, events=None, fused=None, reuse_statistic=False, sweep_cache=None,
+            overlap_tables=False):
         """Enqueue the pass for calibration activations X [n][d_in] and weights W [d_in][d_out].
         reuse_statistic: keep the statistic `a` of the previous run on the same X (see run_budgets).
         sweep_cache: a cache prepared by cmpq_sweep_begin for W (see run_budgets).
         fused (default: True unless events are asked for): outlier protection, final fit and packing through
         cmpq_protect_quantize_pack, which derives the final fit's value tables from the provisional fit's
         and lets the last assignment write the packed words; otherwise cmpq_extract_outliers,
-        cmpq_quantize_layer and cmpq_pack one after the other (same results; needs keep_codes).  events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and,
+        cmpq_quantize_layer and cmpq_pack one after the other (same results; needs keep_codes).
+        overlap_tables (fused runs of the default assignment without events): the value tables depend on the
+        weights alone, so they are built on a second stream (cmpq_sweep_begin into a cache this object keeps)
+        while the current stream computes the statistic and the allocation; the streams join before
+        cmpq_sweep_budget_pack.  Same results; one table set more of device memory.  events (optional dict) receives a (start, end) CUDA event pair per C-ABI call and,
         when not fused, under "final_fit_kernels" the four events around the three kernels of the
         final K-means."""
         if fused is None:
@@ -157,12 +166,30 @@ class LayerQuantizer:
         inexact = self.counters[0:1].view(torch.int32)[0:1]
         sweeps = self.counters[1:2]
         nonfinite = self.nonfinite = self.counters[2:3].view(torch.int32)[0:1]
+        side = None
+        if (overlap_tables and fused and events is None and sweep_cache is None and not reuse_statistic
+                and B.cmpq_get_lloyd_assignment() == B.ASSIGN_ORDERED):
+            if getattr(self, "_overlap_cache", None) is None:
+                self._overlap_cache = torch.empty(B.cmpq_sweep_cache_bytes(self.d_in, self.d_out), dtype=torch.uint8,
+                                                  device=self.device)
+                self._side_stream = torch.cuda.Stream(device=self.device)
+            sweep_cache, side = self._overlap_cache, self._side_stream
         if not reuse_statistic:
             self.sumsq.zero_()
+            if side is not None:
+                # The previous pass may still be reading the cache.  The fork comes directly before the
+                # statistic: both kernels then depend on the same predecessor and the statistic, enqueued
+                # first, gets its blocks placed first (the other order leaves nothing to overlap).
+                side.wait_stream(torch.cuda.current_stream())
             call("cmpq_collect_stats", B.cmpq_collect_stats, X, self.sumsq, self.ws, nonfinite=nonfinite)
+            if side is not None:  # enqueued after the statistic so that its blocks are placed first
+                with torch.cuda.stream(side):
+                    B.cmpq_sweep_begin(W, lloyd_iters, sweep_cache, nonfinite=nonfinite)
             call("cmpq_finalize_stats", B.cmpq_finalize_stats, self.sumsq, self.a)
         call("cmpq_allocate_bits", B.cmpq_allocate_bits, self.a, avg_bits, B.ALLOC_RANK, self.bits, None,
              self.ws)
+        if side is not None:
+            torch.cuda.current_stream().wait_stream(side)
         if sweep_cache is not None and fused:
             call("cmpq_sweep_budget_pack", B.cmpq_sweep_budget_pack, W, self.a, self.bits, self.n_act, self.n_q,
                  lloyd_iters, self.rows, self.cols, self.vals, self.lut, self.codes, self.packed, self.row_off,
@@ -197,13 +224,13 @@ class LayerQuantizer:
         call("cmpq_quantize_layer", B.cmpq_quantize_layer, W, self.bits, self.rows, self.cols, lloyd_iters,
              self.lut, self.codes, self.ws, inexact_rows=inexact, sweeps=sweeps)
 
-    def run_graphed(self, X, W, avg_bits, lloyd_iters):
+    def run_graphed(self, X, W, avg_bits, lloyd_iters, overlap_tables=False):
         """The same pass replayed from a CUDA graph: the launches of a pass are short enough for launch
         overhead to show, and nothing in the pass depends on values read back by the host.  The graph is
         captured on the first call for a given (X, W, budget, iterations) and replayed afterwards; X
         and W must keep their addresses (their contents may change).  Results as in run()."""
         key = (X.data_ptr(), W.data_ptr(), tuple(X.shape), float(avg_bits), int(lloyd_iters),
-               B.cmpq_get_lloyd_assignment())
+               B.cmpq_get_lloyd_assignment(), bool(overlap_tables))
         if not hasattr(self, "_graphs"):
             self._graphs = {}
         entry = self._graphs.get(key)
@@ -212,11 +239,11 @@ class LayerQuantizer:
             side = torch.cuda.Stream()
             side.wait_stream(cur)
             with torch.cuda.stream(side):  # first-use initialisation must not be captured
-                self.run(X, W, avg_bits, lloyd_iters)
+                self.run(X, W, avg_bits, lloyd_iters, overlap_tables=overlap_tables)
             cur.wait_stream(side)
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
-                result = self.run(X, W, avg_bits, lloyd_iters)
+                result = self.run(X, W, avg_bits, lloyd_iters, overlap_tables=overlap_tables)
             entry = (graph, result)
             self._graphs[key] = entry
         entry[0].replay()
@@ -277,14 +304,14 @@ class StackQuantizer:
         """Weights in this rank's layers."""
         return sum(self.shapes[k][0] * self.shapes[k][1] for k in self.mine)
 
-    def run(self, inputs_of, avg_bits, lloyd_iters, on_result=None, timed=False, graphed=False):
+    def run(self, inputs_of, avg_bits, lloyd_iters, on_result=None, timed=False, graphed=False, overlap_tables=False):
         """inputs_of(k) -> (X [n][d_in], W [d_in][d_out]) for layer k of this rank (called right before
         the layer's pass; preparing the inputs is the caller's work and is not timed).  on_result(k, result)
         is called after layer k's pass has been enqueued; the result's buffers are reused by the next layer
         of the same shape, so copy what is kept there (on the same stream).  timed: CUDA events around every
         pass; the returned dict then holds "ms" (the sum over this rank's passes) and "ms_by_shape".
         graphed: passes through LayerQuantizer.run_graphed (inputs_of must then return tensors at fixed
-        addresses per shape).  Returns {"layers", "params"[, "ms", "ms_by_shape"]}."""
+        addresses per shape).  overlap_tables: as in LayerQuantizer.run.  Returns {"layers", "params"[, "ms", "ms_by_shape"]}."""
         pairs = []
         for k in self.mine:
             X, W = inputs_of(k)
@@ -292,7 +319,8 @@ class StackQuantizer:
             if timed:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-            r = (q.run_graphed if graphed else q.run)(X, W, avg_bits, lloyd_iters)
+            extra = {"overlap_tables": True} if overlap_tables else {}  # (a stand-in quantizer need not know the option)
+            r = (q.run_graphed if graphed else q.run)(X, W, avg_bits, lloyd_iters, **extra)
             if timed:
                 e1.record()
                 pairs.append((k, e0, e1))

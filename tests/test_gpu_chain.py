@@ -148,6 +148,29 @@ def test_graph_replay_gives_the_same_bytes_as_the_eager_pass():
     assert not np.array_equal(eager["codes"], replay["codes"])
 
 
+@pytest.mark.parametrize("keep_codes", [True, False])
+def test_tables_built_on_a_second_stream_give_the_same_bytes(keep_codes):
+    """overlap_tables: the value tables are counted on a second stream while the statistic runs; eager and
+    replayed from a graph, with new weights at the same address and with a budget change in between, every
+    output equals the plain pass's (and hence the checker's, which the plain pass is compared with above)."""
+    d_in, d_out, n, T = 200, 1536, 1024, 8
+    W = inputs.make_weight(d_in, d_out, inputs.BF16, 17, device="cuda")
+    X = inputs.make_activations(n, d_in, inputs.BF16, 17, device="cuda")
+    plain, over = LayerQuantizer(d_in, d_out, keep_codes=keep_codes), LayerQuantizer(d_in, d_out, keep_codes=keep_codes)
+    for step, b in enumerate([3.0, 2.3, 3.0]):
+        if step == 2:
+            W.copy_(inputs.make_weight(d_in, d_out, inputs.BF16, 18, device="cuda"))   # same address, new contents
+        ref = _np(plain.run(X, W, b, T))
+        eager = _np(over.run(X, W, b, T, overlap_tables=True))
+        graphed = _np(over.run_graphed(X, W, b, T, overlap_tables=True))
+        replay = _np(over.run_graphed(X, W, b, T, overlap_tables=True))
+        for k in ref:
+            assert np.array_equal(ref[k], eager[k]), (step, k)
+            assert np.array_equal(ref[k], graphed[k]), (step, k)
+            assert np.array_equal(ref[k], replay[k]), (step, k)
+        assert int(over.counters[0].item()) == int(plain.counters[0].item())
+
+
 @pytest.mark.parametrize("d_in,d_out,n,T,budgets", [
     (192, 640, 1024, 6, [2.0, 2.5, 3.0, 3.5, 4.0]),
     (300, 2048, 512, 9, [3.5, 2.5, 3.5, 2.0, 3.0, 2.5]),      # budgets revisited: every fit comes from the cache
