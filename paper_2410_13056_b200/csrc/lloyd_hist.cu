@@ -1027,9 +1027,31 @@ lloyd_iterate_kernel(const IterArgs a) {
     const bool cached_ok = a.fc.hdr && cache_iters == a.iters;
     const int64_t slot = (int64_t)(bits == 2 ? 0 : (bits == 3 ? 1 : 2)) * a.d_in + row;
     if (cached_ok && a.fc.valid[slot]) {
-        a.lut[row * CMPQ_LUT_STRIDE + gl] = a.fc.lut[slot * CMPQ_LUT_STRIDE + gl];
+        const float ck = a.fc.lut[slot * CMPQ_LUT_STRIDE + gl];
+        const float thr0 = a.fc.thr[slot * CMPQ_LUT_STRIDE];
+        const uint32_t limits = reinterpret_cast<const uint32_t*>(a.fc.bnd + slot * 32)[gl];  // first | mid << 16
+        a.lut[row * CMPQ_LUT_STRIDE + gl] = ck;
         a.t.thr[row * CMPQ_LUT_STRIDE + gl] = a.fc.thr[slot * CMPQ_LUT_STRIDE + gl];
-        reinterpret_cast<uint32_t*>(a.t.bnd + row * 32)[gl] = reinterpret_cast<const uint32_t*>(a.fc.bnd + slot * 32)[gl];
+        reinterpret_cast<uint32_t*>(a.t.bnd + row * 32)[gl] = limits;
+        // the selection's lower bound counts the largest error of every cluster side (see iterate_channel):
+        // a copied fit contributes them too, read off the table at the copied cluster limits
+        if (a.side_hist && thr0 != 0.f) {
+            const int K = bits == 2 ? 4 : (bits == 3 ? 8 : 16);
+            const int M = a.t.hdr[row].M;
+            const int first = (int)(limits & 0xffffu), mid = (int)(limits >> 16);
+            int next = (int)(__shfl_down_sync(gmask, limits, 1, kGroup) & 0xffffu);
+            if (gl == K - 1) next = M;
+            if (gl < K) {
+                const uint16_t* keys = a.t.keys + row * a.t.stride;
+                const uint16_t* cum = a.t.cum + row * a.t.stride;
+                int j = first;
+                if (j < mid && cum[j + 1] == cum[j]) ++j;
+                if (j < mid) atomicAdd(&a.side_hist[__float_as_uint(fabsf(value_of_key16<DT>(keys[j]) - ck)) >> 20], 1u);
+                j = next - 1;
+                if (j >= mid && cum[j + 1] == cum[j]) --j;
+                if (j >= mid) atomicAdd(&a.side_hist[__float_as_uint(fabsf(value_of_key16<DT>(keys[j]) - ck)) >> 20], 1u);
+            }
+        }
         return;
     }
     iterate_channel<DT>(a, row, bits == 2 ? 4 : (bits == 3 ? 8 : 16), smem);
