@@ -243,7 +243,8 @@ cmpq_status cmpq_protect_and_quantize(const void* W, cmpq_dtype dt, int64_t d_in
  *                      detected on the device and simply bypasses the kept fits); a, bits, n_act and n_q
  *                      may change from call to call.
  * cache: cmpq_sweep_cache_bytes(d_in, d_out) bytes of device memory, 256-byte aligned, untouched by the
- * caller between the calls (else CMPQ_ERR_WORKSPACE).  Calls on one cache must be ordered (one stream).
+ * caller between the calls (else CMPQ_ERR_WORKSPACE).  Calls on one cache must be ordered (one stream, or
+ * streams joined by events: cmpq_sweep_begin needs the weights alone and may run beside the statistic).
  * With CMPQ_ASSIGN_ALL_PAIRS selected the cache is ignored.
  *   cmpq_sweep_budget_pack  is cmpq_protect_quantize_pack with the same use of the cache (the last assignment
  *                      writes the packed words; codes may be NULL).
